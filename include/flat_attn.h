@@ -1,0 +1,131 @@
+/*
+ * flat_attn.h -- C ABI of the fused exact-attention library for NVIDIA B200 (sm_100a).
+ *
+ * The library computes O = softmax(scale * Q K^T) V for multi-head attention
+ * (paper Section 2, "Computation operators", steps 2-4: Logit, Softmax along
+ * the key index, Attend) in two ways:
+ *
+ *   - fused (the paper's FLAT dataflow, Section 5 and 5.1): the outer loops over
+ *     batch, head and query-row tile are shared by the Logit and Attend
+ *     operators, the slice of the logit tensor produced by Logit is consumed by
+ *     Softmax and Attend on chip, and only Q, K, V are read and O is written;
+ *   - naive (the paper's baseline, Section 4.2 and Fig. 7(a)): operator by
+ *     operator, with the [B,H,Nq,Nk] logit tensor L and weight tensor A written
+ *     to and read back from device memory.
+ *
+ * Conventions for every entry point
+ *   - Tensors are dense, row-major, innermost dimension contiguous:
+ *       Q, O : [B, H, Nq, d]      K, V : [B, H, Nk, d]      L, A : [B, H, Nq, Nk]
+ *   - Unless an argument says HOST, pointers are DEVICE pointers owned by the
+ *     caller, 16-byte aligned.  The library allocates and frees no device memory
+ *     and keeps no pointer after a call returns.
+ *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*; NULL is
+ *     the default stream); the library does not synchronise unless stated.
+ *   - Return value: FLAT_OK or one of the error codes below.  On an argument
+ *     error nothing is launched.  There is no CPU fallback: an unsupported
+ *     request is an error.
+ *   - Supported sizes: B, H, Nq, Nk >= 1; d in {16, 32, 64, 128} (tensor-core
+ *     kernels need d in {64, 128} and bf16); B*H*Nq*Nk and all byte counts must
+ *     fit in 63 bits; B*H <= 65535 * 32768.
+ *   - scale multiplies the logits before the softmax and must be finite.  The
+ *     paper does not mention a scale (scale = 1 is its literal text); 1/sqrt(d)
+ *     is the usual choice.
+ *   - Key-padding mask (k_valid_len, optional): key j of batch b takes part iff
+ *     j < k_valid_len[b], for all heads and query rows; values must lie in
+ *     [0, Nk].  Masked K/V entries must be finite and are otherwise ignored.  A
+ *     batch with k_valid_len[b] == 0 gets O = 0 (and A = 0).
+ */
+#ifndef FLAT_ATTN_H_
+#define FLAT_ATTN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+    FLAT_OK = 0,
+    FLAT_ERR_NULL = 1,         /* a required pointer is NULL                                  */
+    FLAT_ERR_SHAPE = 2,        /* a size is < 1, overflows, or k_valid_len is out of range     */
+    FLAT_ERR_UNSUPPORTED = 3,  /* d, dtype or variant not supported by any kernel              */
+    FLAT_ERR_ALIGN = 4,        /* a pointer is not 16-byte aligned                             */
+    FLAT_ERR_WORKSPACE = 5,    /* caller-provided workspace too small                          */
+    FLAT_ERR_CUDA = 6,         /* a CUDA runtime/driver call failed (launch, tensor map, copy) */
+    FLAT_ERR_TIMEOUT = 7       /* a bounded device-side wait gave up (reported via `status`)   */
+};
+
+enum { FLAT_DTYPE_BF16 = 0, FLAT_DTYPE_F32 = 1 };
+
+/* Kernel choice for the fused path. AUTO picks the tensor-core kernel when it applies. */
+enum {
+    FLAT_VARIANT_AUTO = 0,
+    FLAT_VARIANT_SIMT = 1,     /* fp32 FFMA kernel, any supported d and dtype                  */
+    FLAT_VARIANT_TC = 2        /* tcgen05 + TMEM + TMA kernel: bf16, d in {64,128}             */
+};
+
+typedef struct flat_attn_params {
+    const void* Q;             /* [B,H,Nq,d]                                                   */
+    const void* K;             /* [B,H,Nk,d]                                                   */
+    const void* V;             /* [B,H,Nk,d]                                                   */
+    void* O;                   /* [B,H,Nq,d], same dtype as the inputs                         */
+    int B, H, Nq, Nk, d;
+    float scale;
+    int dtype;                 /* FLAT_DTYPE_BF16 or FLAT_DTYPE_F32 (storage of Q,K,V,O);
+                                  accumulation is always fp32                                 */
+    const int32_t* k_valid_len;/* device, [B], or NULL = all keys valid                        */
+    int32_t* status;           /* optional device word; a kernel that gives up on a bounded
+                                  wait stores a non-zero code here (never traps or hangs)      */
+    int variant;               /* FLAT_VARIANT_*                                               */
+} flat_attn_params_t;
+
+/*
+ * Fused attention, bf16 in / bf16 out, fp32 accumulation, no mask.
+ * Operation: paper Section 5 (fused Logit-Softmax-Attend loop nest, row granularity,
+ * Section 5.2) applied to the operators of Section 2 steps 2-4.
+ * Equivalent to flat_attn_fwd_ex with dtype = BF16, k_valid_len = NULL, variant = AUTO.
+ */
+int flat_attn_fwd(const void* Q, const void* K, const void* V, void* O,
+                  int B, int H, int Nq, int Nk, int d, float scale, void* stream);
+
+/* Fused attention with dtype choice, optional key-padding mask and kernel choice (same
+ * operation as flat_attn_fwd).  `p` is a HOST pointer, read before the call returns. */
+int flat_attn_fwd_ex(const flat_attn_params_t* p, void* stream);
+
+/*
+ * The paper's unfused baseline (Section 4.2; Fig. 7(a)): three kernels,
+ *   L = scale * Q K^T   written to device memory as fp32 [B,H,Nq,Nk],
+ *   A = softmax_row(L)  written as bf16 (dtype BF16) or fp32 (dtype F32) [B,H,Nq,Nk],
+ *   O = A V.
+ * L and A are caller-allocated device buffers; their contents after the call are
+ * the logits (all columns, masked ones included, unmasked values) and the weights
+ * (masked columns 0).
+ */
+int flat_attn_naive_fwd(const void* Q, const void* K, const void* V, void* O, void* L, void* A,
+                        int B, int H, int Nq, int Nk, int d, float scale, void* stream);
+int flat_attn_naive_fwd_ex(const flat_attn_params_t* p, void* L, void* A, void* stream);
+
+/*
+ * End-to-end convenience call with HOST tensors: copies Q, K, V (and k_valid_len if
+ * non-NULL) from host memory into `workspace`, runs the fused kernel, copies O back
+ * to `O_host`, all on `stream`, and returns without synchronising (use pinned host
+ * memory for true asynchrony; the caller synchronises the stream before reading O).
+ * p->Q, p->K, p->V, p->O and p->k_valid_len are HOST pointers here; p->status is
+ * still a device pointer or NULL.  `workspace` is a caller-owned DEVICE buffer of at
+ * least flat_attn_host_workspace_bytes(...) bytes, 256-byte aligned.
+ * The operation is that of flat_attn_fwd_ex; the paper has no counterpart for the copies.
+ */
+int flat_attn_fwd_host(const flat_attn_params_t* p, void* workspace, size_t workspace_bytes, void* stream);
+size_t flat_attn_host_workspace_bytes(int B, int H, int Nq, int Nk, int d, int dtype);
+
+/* Number of kernels the most recent successful call on this thread launched. */
+int flat_attn_last_launch_count(void);
+
+const char* flat_attn_status_string(int code);
+int flat_attn_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FLAT_ATTN_H_ */

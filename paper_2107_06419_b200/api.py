@@ -1,0 +1,183 @@
+"""ctypes binding of libflat_attn.so: argument marshalling only, same names as include/flat_attn.h.
+
+Importing this module loads the CUDA library and raises if it is missing -- there is no
+CPU fallback.  Tensor arguments are torch tensors (device memory and streams are all
+PyTorch is used for); every computation happens inside the library's kernels.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libflat_attn.so")
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(
+        "libflat_attn.so is not built (run `python -m paper_2107_06419_b200.build` or "
+        "`__graft_entry__.build()`); there is no fallback path")
+
+_lib = ctypes.CDLL(LIB_PATH)
+
+FLAT_OK = 0
+FLAT_DTYPE_BF16, FLAT_DTYPE_F32 = 0, 1
+FLAT_VARIANT_AUTO, FLAT_VARIANT_SIMT, FLAT_VARIANT_TC = 0, 1, 2
+
+EXPORTS = ["flat_attn_fwd", "flat_attn_fwd_ex", "flat_attn_naive_fwd", "flat_attn_naive_fwd_ex",
+           "flat_attn_fwd_host", "flat_attn_host_workspace_bytes", "flat_attn_last_launch_count",
+           "flat_attn_status_string", "flat_attn_version"]
+
+
+class flat_attn_params_t(ctypes.Structure):
+    _fields_ = [("Q", ctypes.c_void_p), ("K", ctypes.c_void_p), ("V", ctypes.c_void_p), ("O", ctypes.c_void_p),
+                ("B", ctypes.c_int), ("H", ctypes.c_int), ("Nq", ctypes.c_int), ("Nk", ctypes.c_int),
+                ("d", ctypes.c_int), ("scale", ctypes.c_float), ("dtype", ctypes.c_int),
+                ("k_valid_len", ctypes.c_void_p), ("status", ctypes.c_void_p), ("variant", ctypes.c_int)]
+
+
+_vp, _i, _f = ctypes.c_void_p, ctypes.c_int, ctypes.c_float
+_lib.flat_attn_fwd.argtypes = [_vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _f, _vp]
+_lib.flat_attn_fwd.restype = _i
+_lib.flat_attn_fwd_ex.argtypes = [ctypes.POINTER(flat_attn_params_t), _vp]
+_lib.flat_attn_fwd_ex.restype = _i
+_lib.flat_attn_naive_fwd.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _f, _vp]
+_lib.flat_attn_naive_fwd.restype = _i
+_lib.flat_attn_naive_fwd_ex.argtypes = [ctypes.POINTER(flat_attn_params_t), _vp, _vp, _vp]
+_lib.flat_attn_naive_fwd_ex.restype = _i
+_lib.flat_attn_fwd_host.argtypes = [ctypes.POINTER(flat_attn_params_t), _vp, ctypes.c_size_t, _vp]
+_lib.flat_attn_fwd_host.restype = _i
+_lib.flat_attn_host_workspace_bytes.argtypes = [_i, _i, _i, _i, _i, _i]
+_lib.flat_attn_host_workspace_bytes.restype = ctypes.c_size_t
+_lib.flat_attn_last_launch_count.restype = _i
+_lib.flat_attn_status_string.argtypes = [_i]
+_lib.flat_attn_status_string.restype = ctypes.c_char_p
+_lib.flat_attn_version.restype = _i
+
+
+class FlatAttnError(RuntimeError):
+    def __init__(self, code: int):
+        self.code = code
+        super().__init__("flat_attn error %d: %s" % (code, flat_attn_status_string(code)))
+
+
+def flat_attn_status_string(code: int) -> str:
+    return _lib.flat_attn_status_string(int(code)).decode()
+
+
+def flat_attn_version() -> int:
+    return int(_lib.flat_attn_version())
+
+
+def flat_attn_last_launch_count() -> int:
+    return int(_lib.flat_attn_last_launch_count())
+
+
+def _stream_ptr(stream):
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream))
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _dtype_code(t) -> int:
+    if t.dtype == torch.bfloat16:
+        return FLAT_DTYPE_BF16
+    if t.dtype == torch.float32:
+        return FLAT_DTYPE_F32
+    raise TypeError("Q/K/V/O must be bfloat16 or float32")
+
+
+def _params(Q, K, V, O, scale, k_valid_len, status, variant, host=False):
+    B, H, Nq, d = Q.shape
+    Nk = K.shape[2]
+    if tuple(K.shape) != (B, H, Nk, d) or tuple(V.shape) != (B, H, Nk, d) or tuple(O.shape) != (B, H, Nq, d):
+        raise ValueError("expected Q,O [B,H,Nq,d] and K,V [B,H,Nk,d]")
+    for t in (Q, K, V, O):
+        if not t.is_contiguous():
+            raise ValueError("tensors must be contiguous")
+        if t.dtype != Q.dtype:
+            raise TypeError("Q, K, V, O must share a dtype")
+        if t.is_cuda == host:
+            raise ValueError("tensors must be %s tensors" % ("host" if host else "CUDA"))
+    if k_valid_len is not None:
+        if k_valid_len.dtype != torch.int32 or tuple(k_valid_len.shape) != (B,) or k_valid_len.is_cuda == host:
+            raise ValueError("k_valid_len must be int32 [B] on the same side as Q")
+    p = flat_attn_params_t()
+    p.Q, p.K, p.V, p.O = Q.data_ptr(), K.data_ptr(), V.data_ptr(), O.data_ptr()
+    p.B, p.H, p.Nq, p.Nk, p.d = B, H, Nq, Nk, d
+    p.scale = float(scale)
+    p.dtype = _dtype_code(Q)
+    p.k_valid_len = None if k_valid_len is None else k_valid_len.data_ptr()
+    p.status = None if status is None else status.data_ptr()
+    p.variant = int(variant)
+    return p
+
+
+def _check(rc: int):
+    if rc != FLAT_OK:
+        raise FlatAttnError(rc)
+
+
+def flat_attn_fwd(Q, K, V, O, scale, stream=None):
+    """Fused attention, bf16 CUDA tensors Q,O [B,H,Nq,d] and K,V [B,H,Nk,d]; writes O in place."""
+    p = _params(Q, K, V, O, scale, None, None, FLAT_VARIANT_AUTO)
+    if p.dtype != FLAT_DTYPE_BF16:
+        raise TypeError("flat_attn_fwd takes bfloat16 tensors; use flat_attn_fwd_ex for float32")
+    _check(_lib.flat_attn_fwd(p.Q, p.K, p.V, p.O, p.B, p.H, p.Nq, p.Nk, p.d, p.scale, _stream_ptr(stream)))
+    return O
+
+
+def flat_attn_fwd_ex(Q, K, V, O, scale, k_valid_len=None, status=None, variant=FLAT_VARIANT_AUTO, stream=None):
+    p = _params(Q, K, V, O, scale, k_valid_len, status, variant)
+    _check(_lib.flat_attn_fwd_ex(ctypes.byref(p), _stream_ptr(stream)))
+    return O
+
+
+def flat_attn_naive_fwd(Q, K, V, O, L, A, scale, stream=None):
+    """The unfused baseline: L (fp32) and A (bf16) [B,H,Nq,Nk] are caller-allocated CUDA tensors."""
+    p = _params(Q, K, V, O, scale, None, None, FLAT_VARIANT_AUTO)
+    _check_la(p, L, A)
+    _check(_lib.flat_attn_naive_fwd(p.Q, p.K, p.V, p.O, _ptr(L), _ptr(A), p.B, p.H, p.Nq, p.Nk, p.d, p.scale,
+                                    _stream_ptr(stream)))
+    return O
+
+
+def flat_attn_naive_fwd_ex(Q, K, V, O, L, A, scale, k_valid_len=None, stream=None):
+    p = _params(Q, K, V, O, scale, k_valid_len, None, FLAT_VARIANT_AUTO)
+    _check_la(p, L, A)
+    _check(_lib.flat_attn_naive_fwd_ex(ctypes.byref(p), _ptr(L), _ptr(A), _stream_ptr(stream)))
+    return O
+
+
+def _check_la(p, L, A):
+    shape = (p.B, p.H, p.Nq, p.Nk)
+    if tuple(L.shape) != shape or tuple(A.shape) != shape or not L.is_contiguous() or not A.is_contiguous():
+        raise ValueError("L and A must be contiguous [B,H,Nq,Nk]")
+    if L.dtype != torch.float32:
+        raise TypeError("L must be float32")
+    want = torch.bfloat16 if p.dtype == FLAT_DTYPE_BF16 else torch.float32
+    if A.dtype != want:
+        raise TypeError("A must have the dtype of Q")
+    if not (L.is_cuda and A.is_cuda):
+        raise ValueError("L and A must be CUDA tensors")
+
+
+def flat_attn_host_workspace_bytes(B, H, Nq, Nk, d, dtype=FLAT_DTYPE_BF16) -> int:
+    return int(_lib.flat_attn_host_workspace_bytes(B, H, Nq, Nk, d, dtype))
+
+
+def flat_attn_fwd_host(Q, K, V, O, scale, workspace, k_valid_len=None, status=None,
+                       variant=FLAT_VARIANT_AUTO, stream=None):
+    """Q, K, V, O (and k_valid_len) are HOST tensors (pinned for asynchrony); `workspace` is a CUDA
+    uint8 tensor of at least flat_attn_host_workspace_bytes(...) bytes.  Asynchronous on `stream`."""
+    p = _params(Q, K, V, O, scale, k_valid_len, status, variant, host=True)
+    if not workspace.is_cuda:
+        raise ValueError("workspace must be a CUDA tensor")
+    _check(_lib.flat_attn_fwd_host(ctypes.byref(p), _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                   _stream_ptr(stream)))
+    return O

@@ -1,0 +1,152 @@
+// C ABI of libflat_attn: argument validation and dispatch.  No kernel code here.
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdint.h>
+
+#include "flat_internal.cuh"
+
+namespace {
+
+thread_local int g_last_launches = 0;
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int validate(const flat_attn_params_t* p, flat::Problem* out) {
+    if (!p) return FLAT_ERR_NULL;
+    if (!p->Q || !p->K || !p->V || !p->O) return FLAT_ERR_NULL;
+    if (p->B < 1 || p->H < 1 || p->Nq < 1 || p->Nk < 1 || p->d < 1) return FLAT_ERR_SHAPE;
+    if (!isfinite(p->scale)) return FLAT_ERR_SHAPE;
+    const int64_t bh = static_cast<int64_t>(p->B) * p->H;
+    if (bh > 65535) return FLAT_ERR_SHAPE;
+    // B*H*Nq*Nk < 2^16 * 2^31 * 2^31 could overflow 63 bits: check stepwise.
+    const int64_t lim = INT64_MAX / 16;
+    if (bh * p->Nq > lim / p->Nk) return FLAT_ERR_SHAPE;
+    if (bh * static_cast<int64_t>(p->Nq > p->Nk ? p->Nq : p->Nk) > lim / p->d) return FLAT_ERR_SHAPE;
+    if (p->dtype != FLAT_DTYPE_BF16 && p->dtype != FLAT_DTYPE_F32) return FLAT_ERR_UNSUPPORTED;
+    if (p->d != 16 && p->d != 32 && p->d != 64 && p->d != 128) return FLAT_ERR_UNSUPPORTED;
+    if (p->variant != FLAT_VARIANT_AUTO && p->variant != FLAT_VARIANT_SIMT && p->variant != FLAT_VARIANT_TC)
+        return FLAT_ERR_UNSUPPORTED;
+    if (!aligned16(p->Q) || !aligned16(p->K) || !aligned16(p->V) || !aligned16(p->O)) return FLAT_ERR_ALIGN;
+    if (p->k_valid_len && (reinterpret_cast<uintptr_t>(p->k_valid_len) & 3u)) return FLAT_ERR_ALIGN;
+    if (p->status && (reinterpret_cast<uintptr_t>(p->status) & 3u)) return FLAT_ERR_ALIGN;
+    *out = flat::Problem{p->Q, p->K, p->V, p->O, p->B, p->H, p->Nq, p->Nk, p->d,
+                         p->scale, p->dtype, p->k_valid_len, p->status};
+    return FLAT_OK;
+}
+
+bool tc_applies(const flat::Problem& q) {
+    return q.dtype == FLAT_DTYPE_BF16 && (q.d == 64 || q.d == 128);
+}
+
+int run_fused(const flat::Problem& q, int variant, cudaStream_t st) {
+    int v = variant;
+    if (v == FLAT_VARIANT_AUTO) v = tc_applies(q) ? FLAT_VARIANT_TC : FLAT_VARIANT_SIMT;
+    if (v == FLAT_VARIANT_TC) {
+        if (!tc_applies(q)) return FLAT_ERR_UNSUPPORTED;
+        return flat::launch_fused_tc(q, st);
+    }
+    return flat::launch_fused_simt(q, st);
+}
+
+inline size_t round256(size_t x) { return (x + 255) & ~static_cast<size_t>(255); }
+
+}  // namespace
+
+extern "C" {
+
+int flat_attn_fwd_ex(const flat_attn_params_t* p, void* stream) {
+    flat::Problem q;
+    const int rc = validate(p, &q);
+    if (rc != FLAT_OK) return rc;
+    const int r = run_fused(q, p->variant, static_cast<cudaStream_t>(stream));
+    if (r == FLAT_OK) g_last_launches = 1;
+    return r;
+}
+
+int flat_attn_fwd(const void* Q, const void* K, const void* V, void* O, int B, int H, int Nq, int Nk, int d,
+                  float scale, void* stream) {
+    flat_attn_params_t p{Q, K, V, O, B, H, Nq, Nk, d, scale, FLAT_DTYPE_BF16, nullptr, nullptr, FLAT_VARIANT_AUTO};
+    return flat_attn_fwd_ex(&p, stream);
+}
+
+int flat_attn_naive_fwd_ex(const flat_attn_params_t* p, void* L, void* A, void* stream) {
+    flat::Problem q;
+    const int rc = validate(p, &q);
+    if (rc != FLAT_OK) return rc;
+    if (!L || !A) return FLAT_ERR_NULL;
+    if (!aligned16(L) || !aligned16(A)) return FLAT_ERR_ALIGN;
+    const int r = flat::launch_naive(q, L, A, static_cast<cudaStream_t>(stream));
+    if (r == FLAT_OK) g_last_launches = 3;
+    return r;
+}
+
+int flat_attn_naive_fwd(const void* Q, const void* K, const void* V, void* O, void* L, void* A, int B, int H,
+                        int Nq, int Nk, int d, float scale, void* stream) {
+    flat_attn_params_t p{Q, K, V, O, B, H, Nq, Nk, d, scale, FLAT_DTYPE_BF16, nullptr, nullptr, FLAT_VARIANT_AUTO};
+    return flat_attn_naive_fwd_ex(&p, L, A, stream);
+}
+
+size_t flat_attn_host_workspace_bytes(int B, int H, int Nq, int Nk, int d, int dtype) {
+    if (B < 1 || H < 1 || Nq < 1 || Nk < 1 || d < 1) return 0;
+    const size_t es = dtype == FLAT_DTYPE_F32 ? 4 : 2;
+    const size_t q = round256(es * B * H * static_cast<size_t>(Nq) * d);
+    const size_t k = round256(es * B * H * static_cast<size_t>(Nk) * d);
+    return 2 * q + 2 * k + round256(sizeof(int32_t) * static_cast<size_t>(B));
+}
+
+int flat_attn_fwd_host(const flat_attn_params_t* p, void* workspace, size_t workspace_bytes, void* stream) {
+    if (!p || !workspace) return FLAT_ERR_NULL;
+    if (reinterpret_cast<uintptr_t>(workspace) & 255u) return FLAT_ERR_ALIGN;
+    if (!p->Q || !p->K || !p->V || !p->O) return FLAT_ERR_NULL;
+    if (p->B < 1 || p->H < 1 || p->Nq < 1 || p->Nk < 1 || p->d < 1) return FLAT_ERR_SHAPE;
+    if (p->dtype != FLAT_DTYPE_BF16 && p->dtype != FLAT_DTYPE_F32) return FLAT_ERR_UNSUPPORTED;
+    const size_t need = flat_attn_host_workspace_bytes(p->B, p->H, p->Nq, p->Nk, p->d, p->dtype);
+    if (workspace_bytes < need) return FLAT_ERR_WORKSPACE;
+    const size_t es = p->dtype == FLAT_DTYPE_F32 ? 4 : 2;
+    const size_t qb = es * p->B * p->H * static_cast<size_t>(p->Nq) * p->d;
+    const size_t kb = es * p->B * p->H * static_cast<size_t>(p->Nk) * p->d;
+    char* w = static_cast<char*>(workspace);
+    char* dQ = w;
+    char* dK = dQ + round256(qb);
+    char* dV = dK + round256(kb);
+    char* dO = dV + round256(kb);
+    char* dLen = dO + round256(qb);
+    flat_attn_params_t dev = *p;
+    dev.Q = dQ; dev.K = dK; dev.V = dV; dev.O = dO;
+    dev.k_valid_len = p->k_valid_len ? reinterpret_cast<const int32_t*>(dLen) : nullptr;
+    flat::Problem q;
+    const int rc = validate(&dev, &q);
+    if (rc != FLAT_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(dQ, p->Q, qb, cudaMemcpyHostToDevice, st) != cudaSuccess) return FLAT_ERR_CUDA;
+    if (cudaMemcpyAsync(dK, p->K, kb, cudaMemcpyHostToDevice, st) != cudaSuccess) return FLAT_ERR_CUDA;
+    if (cudaMemcpyAsync(dV, p->V, kb, cudaMemcpyHostToDevice, st) != cudaSuccess) return FLAT_ERR_CUDA;
+    if (p->k_valid_len &&
+        cudaMemcpyAsync(dLen, p->k_valid_len, sizeof(int32_t) * p->B, cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return FLAT_ERR_CUDA;
+    const int r = run_fused(q, p->variant, st);
+    if (r != FLAT_OK) return r;
+    if (cudaMemcpyAsync(p->O, dO, qb, cudaMemcpyDeviceToHost, st) != cudaSuccess) return FLAT_ERR_CUDA;
+    g_last_launches = 1;
+    return FLAT_OK;
+}
+
+int flat_attn_last_launch_count(void) { return g_last_launches; }
+
+const char* flat_attn_status_string(int code) {
+    switch (code) {
+        case FLAT_OK: return "ok";
+        case FLAT_ERR_NULL: return "required pointer is NULL";
+        case FLAT_ERR_SHAPE: return "bad size or scale";
+        case FLAT_ERR_UNSUPPORTED: return "unsupported d, dtype or variant";
+        case FLAT_ERR_ALIGN: return "pointer not aligned";
+        case FLAT_ERR_WORKSPACE: return "workspace too small";
+        case FLAT_ERR_CUDA: return "CUDA call failed";
+        case FLAT_ERR_TIMEOUT: return "device-side wait timed out";
+    }
+    return "unknown status";
+}
+
+int flat_attn_version(void) { return 100; }
+
+}  // extern "C"

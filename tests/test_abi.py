@@ -1,0 +1,120 @@
+"""Host-side checks of the C ABI that need no GPU: the library loads, exports every symbol the
+header declares, and rejects bad arguments before touching the device."""
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+HEADER = os.path.join(ROOT, "include", "flat_attn.h")
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2107_06419_b200 import build
+    return ctypes.CDLL(build.build())
+
+
+@pytest.fixture(scope="module")
+def api(lib):
+    from paper_2107_06419_b200 import api as _api
+    return _api
+
+
+def declared_functions():
+    src = open(HEADER).read()
+    src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
+    return sorted(set(re.findall(r"\b(flat_attn_\w+)\s*\(", src)))
+
+
+def test_header_declares_and_library_exports(lib, api):
+    names = declared_functions()
+    assert "flat_attn_fwd" in names and "flat_attn_naive_fwd" in names and len(names) >= 9
+    for n in names:
+        assert hasattr(lib, n), "library does not export " + n
+    assert sorted(api.EXPORTS) == [n for n in names if n != "flat_attn_params"]
+    for n in api.EXPORTS:
+        assert callable(getattr(api, n)), "binding lacks " + n
+
+
+def test_status_strings_and_version(api):
+    assert api.flat_attn_version() >= 100
+    seen = {api.flat_attn_status_string(c) for c in range(8)}
+    assert len(seen) == 8 and api.flat_attn_status_string(0) == "ok"
+    assert api.flat_attn_status_string(99) == "unknown status"
+
+
+def _params(api, **kw):
+    p = api.flat_attn_params_t()
+    p.Q, p.K, p.V, p.O = 0x10000, 0x20000, 0x30000, 0x40000     # never dereferenced on the host
+    p.B, p.H, p.Nq, p.Nk, p.d = 1, 2, 128, 128, 64
+    p.scale, p.dtype, p.variant = 0.125, 0, 0
+    for k, v in kw.items():
+        setattr(p, k, v)
+    return p
+
+
+@pytest.mark.parametrize("kw,code", [
+    (dict(Q=None), 1), (dict(O=None), 1),
+    (dict(B=0), 2), (dict(Nk=-3), 2), (dict(scale=float("inf")), 2), (dict(scale=float("nan")), 2),
+    (dict(B=70000), 2), (dict(B=60000, Nq=2 ** 31 - 1, Nk=2 ** 31 - 1), 2),
+    (dict(d=48), 3), (dict(d=256), 3), (dict(dtype=2), 3), (dict(variant=9), 3),
+    (dict(dtype=1, variant=2), 3),                               # tensor-core kernel is bf16 only
+    (dict(d=32, variant=2), 3),
+    (dict(K=0x20008), 4), (dict(k_valid_len=0x50002), 4),
+])
+def test_fused_argument_errors(lib, api, kw, code):
+    p = _params(api, **kw)
+    assert api._lib.flat_attn_fwd_ex(ctypes.byref(p), None) == code
+    assert api._lib.flat_attn_fwd_ex(None, None) == 1
+
+
+def test_naive_and_host_argument_errors(api):
+    p = _params(api)
+    assert api._lib.flat_attn_naive_fwd_ex(ctypes.byref(p), None, 0x60000, None) == 1
+    assert api._lib.flat_attn_naive_fwd_ex(ctypes.byref(p), 0x60004, 0x70000, None) == 4
+    assert api._lib.flat_attn_naive_fwd(0x10000, 0x20000, 0x30000, 0x40000, 0x50000, 0x60000, 1, 1, 0, 5, 64, 1.0, None) == 2
+    need = api.flat_attn_host_workspace_bytes(1, 2, 128, 128, 64)
+    assert need == 4 * 2 * 128 * 64 * 2 + 256
+    assert api.flat_attn_host_workspace_bytes(1, 2, 128, 128, 64, 1) == 4 * 2 * 128 * 64 * 4 + 256
+    assert api.flat_attn_host_workspace_bytes(0, 2, 128, 128, 64) == 0
+    assert api._lib.flat_attn_fwd_host(ctypes.byref(p), None, need, None) == 1
+    assert api._lib.flat_attn_fwd_host(ctypes.byref(p), 0x100010, need, None) == 4
+    assert api._lib.flat_attn_fwd_host(ctypes.byref(p), 0x100000, need - 1, None) == 5
+
+
+def test_binding_rejects_bad_tensors(api):
+    import torch
+    q = torch.zeros(1, 1, 4, 64, dtype=torch.bfloat16)
+    with pytest.raises(ValueError):
+        api.flat_attn_fwd(q, q, q, q, 1.0)                      # host tensors on the device entry point
+    with pytest.raises(TypeError):
+        api._params(q.to(torch.float16), q, q, q, 1.0, None, None, 0, host=True)
+    with pytest.raises(ValueError):
+        api._params(q, q[:, :, :, :32], q, q, 1.0, None, None, 0, host=True)
+
+
+def test_missing_library_fails_loudly(tmp_path):
+    """Importing the binding without the built library raises; nothing falls back to the CPU."""
+    import subprocess
+    import sys
+    pkg = tmp_path / "paper_2107_06419_b200"
+    pkg.mkdir()
+    for f in ("__init__.py", "api.py"):
+        (pkg / f).write_text(open(os.path.join(ROOT, "paper_2107_06419_b200", f)).read())
+    r = subprocess.run([sys.executable, "-c", "import paper_2107_06419_b200.api"], cwd=tmp_path,
+                       capture_output=True, text=True, env={**os.environ, "PYTHONPATH": str(tmp_path)})
+    assert r.returncode != 0 and "libflat_attn.so is not built" in r.stderr
+
+
+def test_product_path_never_touches_the_oracle():
+    pkg = os.path.join(ROOT, "paper_2107_06419_b200")
+    for dirpath, _, files in os.walk(pkg):
+        for f in files:
+            if f.endswith((".py", ".cu", ".cuh", ".h")):
+                text = open(os.path.join(dirpath, f)).read()
+                assert "oracle" not in text.lower() or f == "inputs.py", f
+    for f in os.listdir(os.path.join(ROOT, "oracle")):
+        if f.endswith((".py", ".cpp")):
+            assert "paper_2107_06419_b200" not in open(os.path.join(ROOT, "oracle", f)).read()

@@ -1,0 +1,211 @@
+"""CUDA path vs CPU oracle, element by element on the same seeded inputs, through the C ABI."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2107_06419_b200 import inputs
+from helpers import bf16_tensor, bf16_to_f64, check_bf16, check_f32, rand_bits
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def api():
+    from paper_2107_06419_b200 import api as _api
+    return _api
+
+
+def run_fused_bf16(api, Qb, Kb, Vb, scale, vl=None, variant=0):
+    Q, K, V = bf16_tensor(Qb), bf16_tensor(Kb), bf16_tensor(Vb)
+    O = torch.full(Q.shape, float("nan"), dtype=torch.bfloat16, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    vlt = None if vl is None else torch.from_numpy(vl).cuda()
+    api.flat_attn_fwd_ex(Q, K, V, O, scale, k_valid_len=vlt, status=status, variant=variant)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0, "device status 0x%x" % int(status.item())
+    return bf16_to_f64(O)
+
+
+SMALL = [
+    # B, H, Nq, Nk, d  -- several 128-tiles plus ragged tails in both Nq and Nk
+    (1, 1, 128, 128, 64),
+    (1, 2, 256, 384, 64),
+    (2, 3, 300, 517, 64),
+    (1, 2, 129, 1, 64),
+    (1, 1, 1, 700, 64),
+    (2, 2, 200, 333, 128),
+    (1, 1, 128, 256, 128),
+]
+
+
+@pytest.mark.parametrize("shape", SMALL)
+@pytest.mark.parametrize("variant", [1, 2], ids=["simt", "tc"])
+def test_fused_bf16_small(api, shape, variant):
+    B, H, Nq, Nk, d = shape
+    rng = np.random.default_rng(abs(hash(shape)) % (2 ** 31))
+    Qb, Kb, Vb = rand_bits(rng, (B, H, Nq, d)), rand_bits(rng, (B, H, Nk, d)), rand_bits(rng, (B, H, Nk, d))
+    scale = 1 / math.sqrt(d)
+    ref = oracle.attention(Qb, Kb, Vb, scale)["O"]
+    got = run_fused_bf16(api, Qb, Kb, Vb, scale, variant=variant)
+    check_bf16(got, ref, "fused bf16 %s v%d" % (shape, variant))
+
+
+@pytest.mark.parametrize("variant", [1, 2], ids=["simt", "tc"])
+@pytest.mark.parametrize("d", [64, 128])
+def test_fused_bf16_masked(api, variant, d):
+    B, H, Nq, Nk = 5, 2, 200, 600
+    rng = np.random.default_rng(77 + d)
+    Qb, Kb, Vb = rand_bits(rng, (B, H, Nq, d)), rand_bits(rng, (B, H, Nk, d)), rand_bits(rng, (B, H, Nk, d))
+    vl = np.array([600, 1, 128, 385, 0], dtype=np.int32)    # full, single key, tile edge, ragged, none
+    # finite garbage in masked rows must not matter
+    Kf, Vf = inputs.bf16_bits_to_f32(Kb).reshape(Kb.shape).copy(), inputs.bf16_bits_to_f32(Vb).reshape(Vb.shape).copy()
+    for b in range(B):
+        Kf[b, :, vl[b]:] = 1000.0
+        Vf[b, :, vl[b]:] = -3000.0
+    Kb, Vb = inputs.f32_to_bf16_bits(Kf).reshape(Kb.shape), inputs.f32_to_bf16_bits(Vf).reshape(Vb.shape)
+    scale = 1 / math.sqrt(d)
+    ref = oracle.attention(Qb, Kb, Vb, scale, valid_len=vl)["O"]
+    got = run_fused_bf16(api, Qb, Kb, Vb, scale, vl=vl, variant=variant)
+    check_bf16(got, ref, "masked d=%d v%d" % (d, variant))
+    assert np.all(got[4] == 0.0)                            # no valid key: O = 0
+
+
+@pytest.mark.parametrize("variant", [1, 2], ids=["simt", "tc"])
+def test_fused_bf16_planted_keys(api, variant):
+    """Peaked softmax on a planted key with position-coded V: a dropped, duplicated, shifted or
+    mis-masked key tile moves O by O(1)."""
+    w = inputs.Workload("planted", 2, 2, 384, 1000, 64, masked=True)
+    Qb, Kb, Vb, planted = inputs.make_planted_qkv_bf16(w, seed=5)
+    vl = inputs.make_valid_len(w, seed=5)
+    ref = oracle.attention(Qb, Kb, Vb, w.scale, valid_len=vl, want_weights=True)
+    # the construction does what it says: the planted key dominates
+    A = ref["A"]
+    for b in range(w.B):
+        top = A[b, 0].argmax(-1)
+        assert np.mean(top == planted[b]) > 0.95
+    got = run_fused_bf16(api, Qb, Kb, Vb, w.scale, vl=vl, variant=variant)
+    check_bf16(got, ref["O"], "planted v%d" % variant)
+
+
+@pytest.mark.parametrize("scale", [1.0, 0.05, -0.125, 3.0])
+def test_fused_bf16_scales_tc(api, scale):
+    B, H, Nq, Nk, d = 1, 2, 256, 512, 64
+    rng = np.random.default_rng(5)
+    Qb, Kb, Vb = rand_bits(rng, (B, H, Nq, d)), rand_bits(rng, (B, H, Nk, d)), rand_bits(rng, (B, H, Nk, d))
+    ref = oracle.attention(Qb, Kb, Vb, scale)["O"]
+    got = run_fused_bf16(api, Qb, Kb, Vb, scale, variant=2)
+    check_bf16(got, ref, "scale %g" % scale)
+
+
+def test_rising_maximum_forces_rescale(api):
+    """Keys ordered so that the row maximum keeps rising tile after tile (logits grow with j)."""
+    B, H, Nq, Nk, d = 1, 1, 128, 1024, 64
+    rng = np.random.default_rng(9)
+    Qf = np.abs(rng.standard_normal((B, H, Nq, d))).astype(np.float32)
+    ramp = (np.arange(Nk, dtype=np.float32) / Nk * 6.0)[None, None, :, None]
+    Kf = (np.abs(rng.standard_normal((B, H, Nk, d))) * 0.2 + ramp * 0.25).astype(np.float32)
+    Vf = rng.standard_normal((B, H, Nk, d)).astype(np.float32)
+    Qb, Kb, Vb = (inputs.f32_to_bf16_bits(x).reshape(x.shape) for x in (Qf, Kf, Vf))
+    ref = oracle.attention(Qb, Kb, Vb, 1.0, want_logits=True)
+    L = ref["L"].reshape(Nq, Nk)
+    assert np.all(L[:, -128:].max(1) - L[:, :128].max(1) > 20)      # > 8 log2 units per several tiles
+    for variant in (1, 2):
+        got = run_fused_bf16(api, Qb, Kb, Vb, 1.0, variant=variant)
+        check_bf16(got, ref["O"], "rising max v%d" % variant)
+
+
+@pytest.mark.parametrize("shape", [(1, 2, 200, 333, 64), (2, 1, 128, 257, 128), (1, 1, 70, 130, 32), (1, 2, 65, 64, 16)])
+def test_fused_f32(api, shape):
+    B, H, Nq, Nk, d = shape
+    rng = np.random.default_rng(31 + d)
+    Q = rng.standard_normal((B, H, Nq, d)).astype(np.float32)
+    K = rng.standard_normal((B, H, Nk, d)).astype(np.float32)
+    V = rng.standard_normal((B, H, Nk, d)).astype(np.float32)
+    vl = np.array([Nk, max(1, Nk // 3)], dtype=np.int32)[:B]
+    scale = 1 / math.sqrt(d)
+    ref = oracle.attention(Q, K, V, scale, valid_len=vl)["O"]
+    Qt, Kt, Vt = (torch.from_numpy(x).cuda() for x in (Q, K, V))
+    O = torch.full(Qt.shape, float("nan"), device="cuda")
+    api.flat_attn_fwd_ex(Qt, Kt, Vt, O, scale, k_valid_len=torch.from_numpy(vl).cuda())
+    torch.cuda.synchronize()
+    check_f32(O.cpu().numpy().astype(np.float64), ref, "fused f32 %s" % (shape,))
+
+
+@pytest.mark.parametrize("d", [64, 128])
+def test_naive_bf16(api, d):
+    B, H, Nq, Nk = 2, 2, 200, 333
+    rng = np.random.default_rng(13 + d)
+    Qb, Kb, Vb = rand_bits(rng, (B, H, Nq, d)), rand_bits(rng, (B, H, Nk, d)), rand_bits(rng, (B, H, Nk, d))
+    vl = np.array([333, 130], dtype=np.int32)
+    scale = 1 / math.sqrt(d)
+    ref = oracle.attention(Qb, Kb, Vb, scale, valid_len=vl, want_logits=True, want_weights=True)
+    Q, K, V = bf16_tensor(Qb), bf16_tensor(Kb), bf16_tensor(Vb)
+    O = torch.full(Q.shape, float("nan"), dtype=torch.bfloat16, device="cuda")
+    L = torch.full((B, H, Nq, Nk), float("nan"), dtype=torch.float32, device="cuda")
+    A = torch.full((B, H, Nq, Nk), float("nan"), dtype=torch.bfloat16, device="cuda")
+    api.flat_attn_naive_fwd_ex(Q, K, V, O, L, A, scale, k_valid_len=torch.from_numpy(vl).cuda())
+    torch.cuda.synchronize()
+    check_bf16(bf16_to_f64(O), ref["O"], "naive O d=%d" % d)
+    Lg, Ag = L.cpu().numpy().astype(np.float64), bf16_to_f64(A)
+    for b in range(B):
+        n = vl[b]
+        assert np.max(np.abs(Lg[b, :, :, :n] - ref["L"][b, :, :, :n])) < 1e-4
+        assert np.all(Ag[b, :, :, n:] == 0.0)
+    assert np.max(np.abs(Ag - ref["A"])) < 4e-3          # bf16 rounding of weights <= 1
+    # unmasked entry point agrees with the fused kernel's result on the same data
+    api.flat_attn_naive_fwd(Q, K, V, O, L, A, scale)
+    torch.cuda.synchronize()
+    check_bf16(bf16_to_f64(O), oracle.attention(Qb, Kb, Vb, scale)["O"], "naive unmasked d=%d" % d)
+
+
+def test_naive_f32(api):
+    B, H, Nq, Nk, d = 1, 2, 130, 200, 64
+    rng = np.random.default_rng(17)
+    Q = rng.standard_normal((B, H, Nq, d)).astype(np.float32)
+    K = rng.standard_normal((B, H, Nk, d)).astype(np.float32)
+    V = rng.standard_normal((B, H, Nk, d)).astype(np.float32)
+    ref = oracle.attention(Q, K, V, 0.125, want_weights=True)
+    Qt, Kt, Vt = (torch.from_numpy(x).cuda() for x in (Q, K, V))
+    O = torch.empty_like(Qt)
+    L = torch.empty((B, H, Nq, Nk), device="cuda")
+    A = torch.empty((B, H, Nq, Nk), device="cuda")
+    api.flat_attn_naive_fwd_ex(Qt, Kt, Vt, O, L, A, 0.125)
+    torch.cuda.synchronize()
+    check_f32(O.cpu().numpy().astype(np.float64), ref["O"], "naive f32")
+    assert np.max(np.abs(A.cpu().numpy().astype(np.float64) - ref["A"])) < 1e-6
+
+
+def test_host_entry_point(api):
+    B, H, Nq, Nk, d = 2, 2, 256, 300, 64
+    rng = np.random.default_rng(23)
+    Qb, Kb, Vb = rand_bits(rng, (B, H, Nq, d)), rand_bits(rng, (B, H, Nk, d)), rand_bits(rng, (B, H, Nk, d))
+    vl = np.array([300, 77], dtype=np.int32)
+    Q, K, V = (bf16_tensor(x, device=None).pin_memory() for x in (Qb, Kb, Vb))
+    O = torch.empty(Q.shape, dtype=torch.bfloat16).pin_memory()
+    ws = torch.empty(api.flat_attn_host_workspace_bytes(B, H, Nq, Nk, d), dtype=torch.uint8, device="cuda")
+    api.flat_attn_fwd_host(Q, K, V, O, 0.125, ws, k_valid_len=torch.from_numpy(vl).pin_memory())
+    torch.cuda.synchronize()
+    ref = oracle.attention(Qb, Kb, Vb, 0.125, valid_len=vl)["O"]
+    check_bf16(bf16_to_f64(O), ref, "host entry")
+    with pytest.raises(api.FlatAttnError) as e:
+        api.flat_attn_fwd_host(Q, K, V, O, 0.125, ws[:1024])
+    assert e.value.code == 5
+
+
+def test_output_padding_untouched(api):
+    """Canary rows around O: the kernels write exactly B*H*Nq*d elements."""
+    B, H, Nq, Nk, d = 1, 3, 130, 140, 64
+    rng = np.random.default_rng(29)
+    Qb, Kb, Vb = rand_bits(rng, (B, H, Nq, d)), rand_bits(rng, (B, H, Nk, d)), rand_bits(rng, (B, H, Nk, d))
+    Q, K, V = bf16_tensor(Qb), bf16_tensor(Kb), bf16_tensor(Vb)
+    n = B * H * Nq * d
+    for variant in (1, 2):
+        buf = torch.full((n + 2048,), 7.0, dtype=torch.bfloat16, device="cuda")
+        O = buf[1024:1024 + n].view(B, H, Nq, d)
+        api.flat_attn_fwd_ex(Q, K, V, O, 0.125, variant=variant)
+        torch.cuda.synchronize()
+        assert torch.all(buf[:1024] == 7.0) and torch.all(buf[1024 + n:] == 7.0)
+        check_bf16(bf16_to_f64(O), oracle.attention(Qb, Kb, Vb, 0.125)["O"], "canary v%d" % variant)
