@@ -26,7 +26,7 @@
  *     request is an error.
  *   - Supported sizes: B, H, Nq, Nk >= 1; d in {16, 32, 64, 128} (tensor-core
  *     kernels need d in {64, 128} and bf16); B*H*Nq*Nk and all byte counts must
- *     fit in 63 bits; B*H <= 65535 * 32768.
+ *     fit in 63 bits; B*H <= 65535.
  *   - scale multiplies the logits before the softmax and must be finite.  The
  *     paper does not mention a scale (scale = 1 is its literal text); 1/sqrt(d)
  *     is the usual choice.
@@ -118,6 +118,38 @@ int flat_attn_naive_fwd_ex(const flat_attn_params_t* p, void* L, void* A, void* 
  */
 int flat_attn_fwd_host(const flat_attn_params_t* p, void* workspace, size_t workspace_bytes, void* stream);
 size_t flat_attn_host_workspace_bytes(int B, int H, int Nq, int Nk, int d, int dtype);
+
+/*
+ * The unfused baseline for callers that cannot allocate device memory.
+ *
+ * (The paper has no counterpart for this entry point; the arithmetic is that of
+ * flat_attn_naive_fwd: bf16 in and out, no mask.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- a plugin handed a
+ * fixed memory budget by its host application, a real-time or safety-reviewed loop
+ * that must not enter the driver's allocator (it can block, fail, or fragment the
+ * budget), a process whose device memory was carved up at start-up.  Such a caller
+ * can own Q, K, V and O but has nowhere to put the [B,H,Nq,Nk] logit and weight
+ * tensors that the baseline materialises.  Here they live in a device array that is
+ * part of the library image itself: fp32 logits followed by bf16 weights,
+ * 6 * FLAT_STATIC_MAX_ELEMS bytes (24 MiB), resident on every GPU that loads the
+ * library until the process exits.  The call path performs no cudaMalloc, cudaFree
+ * or other allocating call.
+ *
+ *   - Limit: B*H*Nq*Nk <= FLAT_STATIC_MAX_ELEMS, otherwise FLAT_ERR_WORKSPACE is
+ *     returned before anything touches the device.  Other argument rules and error
+ *     codes are those of flat_attn_naive_fwd; Q, K, V, O stay caller-owned.
+ *   - The first call on each device looks up the array's device address (with that
+ *     device current, which is the caller's job as for every entry point).  Make that
+ *     first call outside any stream capture.
+ *   - All calls on a device share the one array, and it keeps whatever the last call
+ *     left in it.  The three kernels overwrite every element they later read, so
+ *     nothing has to be cleared, but two calls whose kernels overlap on the GPU
+ *     (different streams, different host threads) race on it: serialise them.
+ */
+#define FLAT_STATIC_MAX_ELEMS (4 * 1024 * 1024)
+int flat_attn_naive_fwd_static(const void* Q, const void* K, const void* V, void* O,
+                               int B, int H, int Nq, int Nk, int d, float scale, void* stream);
 
 /* Number of kernels the most recent successful call on this thread launched. */
 int flat_attn_last_launch_count(void);

@@ -26,6 +26,7 @@ FLAT_DTYPE_BF16, FLAT_DTYPE_F32 = 0, 1
 FLAT_VARIANT_AUTO, FLAT_VARIANT_SIMT, FLAT_VARIANT_TC = 0, 1, 2
 
 EXPORTS = ["flat_attn_fwd", "flat_attn_fwd_ex", "flat_attn_naive_fwd", "flat_attn_naive_fwd_ex",
+           "flat_attn_naive_fwd_static",
            "flat_attn_fwd_host", "flat_attn_host_workspace_bytes", "flat_attn_last_launch_count",
            "flat_attn_status_string", "flat_attn_version"]
 
@@ -46,6 +47,8 @@ _lib.flat_attn_naive_fwd.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _
 _lib.flat_attn_naive_fwd.restype = _i
 _lib.flat_attn_naive_fwd_ex.argtypes = [ctypes.POINTER(flat_attn_params_t), _vp, _vp, _vp]
 _lib.flat_attn_naive_fwd_ex.restype = _i
+_lib.flat_attn_naive_fwd_static.argtypes = [_vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _f, _vp]
+_lib.flat_attn_naive_fwd_static.restype = _i
 _lib.flat_attn_fwd_host.argtypes = [ctypes.POINTER(flat_attn_params_t), _vp, ctypes.c_size_t, _vp]
 _lib.flat_attn_fwd_host.restype = _i
 _lib.flat_attn_host_workspace_bytes.argtypes = [_i, _i, _i, _i, _i, _i]
@@ -151,6 +154,22 @@ def flat_attn_naive_fwd_ex(Q, K, V, O, L, A, scale, k_valid_len=None, stream=Non
     p = _params(Q, K, V, O, scale, k_valid_len, None, FLAT_VARIANT_AUTO)
     _check_la(p, L, A)
     _check(_lib.flat_attn_naive_fwd_ex(ctypes.byref(p), _ptr(L), _ptr(A), _stream_ptr(stream)))
+    return O
+
+
+FLAT_STATIC_MAX_ELEMS = 4 * 1024 * 1024
+
+
+def flat_attn_naive_fwd_static(Q, K, V, O, scale, stream=None):
+    """The unfused baseline without caller-provided L and A: for callers that may not allocate
+    device memory, the two [B,H,Nq,Nk] intermediates live in a 24 MiB array inside the library.
+    bf16 CUDA tensors; B*H*Nq*Nk must not exceed FLAT_STATIC_MAX_ELEMS (error 5 otherwise).
+    Calls on one device share that array: do not let two of them overlap on the GPU."""
+    p = _params(Q, K, V, O, scale, None, None, FLAT_VARIANT_AUTO)
+    if p.dtype != FLAT_DTYPE_BF16:
+        raise TypeError("flat_attn_naive_fwd_static takes bfloat16 tensors")
+    _check(_lib.flat_attn_naive_fwd_static(p.Q, p.K, p.V, p.O, p.B, p.H, p.Nq, p.Nk, p.d, p.scale,
+                                           _stream_ptr(stream)))
     return O
 
 
