@@ -24,8 +24,7 @@ int validate(const flat_attn_params_t* p, flat::Problem* out) {
     if (bh * static_cast<int64_t>(p->Nq > p->Nk ? p->Nq : p->Nk) > lim / p->d) return FLAT_ERR_SHAPE;
     if (p->dtype != FLAT_DTYPE_BF16 && p->dtype != FLAT_DTYPE_F32) return FLAT_ERR_UNSUPPORTED;
     if (p->d != 16 && p->d != 32 && p->d != 64 && p->d != 128) return FLAT_ERR_UNSUPPORTED;
-    if (p->variant != FLAT_VARIANT_AUTO && p->variant != FLAT_VARIANT_SIMT && p->variant != FLAT_VARIANT_TC)
-        return FLAT_ERR_UNSUPPORTED;
+    if (p->variant < FLAT_VARIANT_AUTO || p->variant > FLAT_VARIANT_TC2) return FLAT_ERR_UNSUPPORTED;
     if (!aligned16(p->Q) || !aligned16(p->K) || !aligned16(p->V) || !aligned16(p->O)) return FLAT_ERR_ALIGN;
     if (p->k_valid_len && (reinterpret_cast<uintptr_t>(p->k_valid_len) & 3u)) return FLAT_ERR_ALIGN;
     if (p->status && (reinterpret_cast<uintptr_t>(p->status) & 3u)) return FLAT_ERR_ALIGN;
@@ -38,12 +37,33 @@ bool tc_applies(const flat::Problem& q) {
     return q.dtype == FLAT_DTYPE_BF16 && (q.d == 64 || q.d == 128);
 }
 
+int sm_count() {
+    thread_local int cached_dev = -1, cached_sms = 0;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+    if (dev != cached_dev) {
+        int sms = 0;
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) return 148;
+        cached_dev = dev; cached_sms = sms;
+    }
+    return cached_sms;
+}
+
 int run_fused(const flat::Problem& q, int variant, cudaStream_t st) {
     int v = variant;
-    if (v == FLAT_VARIANT_AUTO) v = tc_applies(q) ? FLAT_VARIANT_TC : FLAT_VARIANT_SIMT;
-    if (v == FLAT_VARIANT_TC) {
+    if (v == FLAT_VARIANT_AUTO) {
+        if (!tc_applies(q)) {
+            v = FLAT_VARIANT_SIMT;
+        } else {
+            // Two-tile CTAs (256 query rows) once they fill every SM; otherwise 128-row CTAs,
+            // which give twice as many CTAs for small problems.
+            const int64_t ctas2 = static_cast<int64_t>((q.Nq + 255) / 256) * q.B * q.H;
+            v = ctas2 >= sm_count() ? FLAT_VARIANT_TC2 : FLAT_VARIANT_TC;
+        }
+    }
+    if (v == FLAT_VARIANT_TC || v == FLAT_VARIANT_TC2) {
         if (!tc_applies(q)) return FLAT_ERR_UNSUPPORTED;
-        return flat::launch_fused_tc(q, st);
+        return v == FLAT_VARIANT_TC ? flat::launch_fused_tc(q, st) : flat::launch_fused_tc2(q, st);
     }
     return flat::launch_fused_simt(q, st);
 }

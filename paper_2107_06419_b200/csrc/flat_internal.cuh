@@ -22,5 +22,6 @@ struct Problem {
 int launch_fused_simt(const Problem& p, cudaStream_t st);
 int launch_naive(const Problem& p, void* L, void* A, cudaStream_t st);
 int launch_fused_tc(const Problem& p, cudaStream_t st);
+int launch_fused_tc2(const Problem& p, cudaStream_t st);
 
 }  // namespace flat

@@ -25,10 +25,12 @@
 
 #include "flat_internal.cuh"
 #include "ptx_sm100.cuh"
+#include "tc_common.cuh"
 
 namespace flat {
 
 using namespace ptx;
+using namespace tc;
 
 namespace {
 
@@ -37,8 +39,6 @@ constexpr int BN = 128;              // keys per step
 constexpr int STAGES = 2;
 constexpr int TC_THREADS = 192;
 constexpr uint32_t TMEM_COLS = 256;
-constexpr long long WAIT_CYCLES = 2000000000ll;   // ~1 s at 2 GHz
-constexpr float RESCALE_THRESHOLD = 8.0f;         // log2 units: P stays <= 2^8
 
 template <int D> struct TcLayout {
     static constexpr int Q_BYTES = BM * D * 2;
@@ -52,39 +52,6 @@ template <int D> struct TcLayout {
 
 enum { BAR_Q_FULL = 0, BAR_KV_FULL = 1, BAR_KV_EMPTY = 1 + STAGES, BAR_S_FULL = 1 + 2 * STAGES,
        BAR_P_FULL, BAR_PV_DONE, NUM_BARS };
-
-__device__ __forceinline__ bool bounded_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
-                                             int32_t* status, int code) {
-    if (mbar_try_wait(bar, parity)) return true;
-    const long long t0 = clock64();
-    for (;;) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if (*abort_flag) return false;
-        if (clock64() - t0 > WAIT_CYCLES) {
-            *abort_flag = 1;
-            if (status) atomicExch(status, code);
-            return false;
-        }
-    }
-}
-
-// Teardown helper: wait for a copy this thread started, with a time limit and no side effects.
-__device__ __forceinline__ void drain_wait(uint64_t* bar, uint32_t parity) {
-    const long long t0 = clock64();
-    while (!mbar_try_wait(bar, parity))
-        if (clock64() - t0 > WAIT_CYCLES) return;
-}
-
-__device__ __forceinline__ float ex2_approx(float x) {
-    float y;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
-
-__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
-    __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
-    return *reinterpret_cast<uint32_t*>(&h);
-}
 
 template <int D>
 __global__ void __launch_bounds__(TC_THREADS, (D == 64) ? 2 : 1)
@@ -294,35 +261,6 @@ fused_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 }
 
 // ---------------------------------------------------------------- host side
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn get_encode_fn() {
-    static EncodeTiledFn fn = [] {
-        void* p = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess ||
-            qres != cudaDriverEntryPointSuccess)
-            p = nullptr;
-        return reinterpret_cast<EncodeTiledFn>(p);
-    }();
-    return fn;
-}
-
-// bf16 tensor [BH, N, d] (d contiguous) viewed as 3-D {d, N, BH}; box = 64 x rows x 1, 128-byte swizzle.
-bool make_map(CUtensorMap* m, const void* ptr, int BH, int N, int d, int box_rows) {
-    EncodeTiledFn enc = get_encode_fn();
-    if (!enc) return false;
-    cuuint64_t dims[3] = {static_cast<cuuint64_t>(d), static_cast<cuuint64_t>(N), static_cast<cuuint64_t>(BH)};
-    cuuint64_t strides[2] = {static_cast<cuuint64_t>(d) * 2, static_cast<cuuint64_t>(N) * d * 2};
-    cuuint32_t box[3] = {64, static_cast<cuuint32_t>(box_rows), 1};
-    cuuint32_t estr[3] = {1, 1, 1};
-    return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
-               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 template <int D>
 int launch_tc_d(const Problem& p, cudaStream_t st) {
     using LY = TcLayout<D>;

@@ -1,0 +1,380 @@
+// Fused Logit-Softmax-Attend, pipelined: two 128-row query tiles per CTA ping-pong on the tensor
+// pipe so that the softmax of one tile overlaps the MMAs of the other (bf16 in, fp32 accumulate).
+//
+// Paper mapping (Section 5, 5.1, 5.2): shared outer loops = (batch, head) on blockIdx.y and a
+// 256-row slab of query rows on blockIdx.x (R-granularity, Rx = 2 x 128); inner loops Logit and
+// Attend run interleaved over 128-key tiles with the streaming softmax between them (the running
+// maximum / sum replaces the paper's full-row on-chip slice; same function).
+//
+// CTA = 384 threads (three warpgroups; registers are moved from the third to the first two):
+//   warps 0-3  softmax of query tile A   (thread r <-> row r of the tile <-> TMEM lane r)
+//   warps 4-7  softmax of query tile B
+//   warp  8    TMA producer (one lane): Q tiles once, then K and V tiles into separate rings
+//   warp  9    MMA issuer   (one lane): S_t = Q_t K^T and O_t += P_t V, t in {A, B}
+//   warps 10-11 idle (they only complete the warpgroup for the register hand-over)
+// A softmax thread pulls its 128 logits into registers, releases the S buffer at once (so the next
+// S_t is computed while it works), takes the row maximum, writes bf16 weights P_t to TMEM and adds
+// to its row sum.  O_t is rescaled in TMEM only when a row maximum exceeds the reference by 2^8.
+//
+// TMEM columns (512): S_A 0, S_B 128, O_A 256, O_B 256+d, and for d = 64 P_A 384, P_B 448; at
+// d = 128 TMEM is full and P_t overlays the first 64 columns of S_t, so S_t(j+1) is issued behind
+// O_t += P_t(j) V_j instead of ahead of it.
+// Every wait is bounded (see tc_common.cuh); on expiry the CTA aborts cleanly and reports a code.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "flat_internal.cuh"
+#include "ptx_sm100.cuh"
+#include "tc_common.cuh"
+
+namespace flat {
+
+using namespace ptx;
+using namespace tc;
+
+namespace {
+
+constexpr int BM = 128;              // rows per query tile (two tiles per CTA)
+constexpr int BN = 128;              // keys per step
+constexpr int THREADS = 384;          // 3 warpgroups: softmax A, softmax B, {TMA, MMA, 2 idle warps}
+
+template <int D> struct L2 {
+    static constexpr bool ALIAS = (D == 128);            // P overlays S
+    static constexpr int KS = (D == 64) ? 3 : 2;         // K ring depth
+    static constexpr int VS = (D == 64) ? 3 : 2;         // V ring depth
+    static constexpr int Q_BYTES = BM * D * 2;           // one query tile
+    static constexpr int KV_BYTES = BN * D * 2;
+    static constexpr int TILE_BYTES = 2 * Q_BYTES + (KS + VS) * KV_BYTES;
+    static constexpr int SMEM_BYTES = TILE_BYTES + 512 + 1024;
+    __host__ __device__ static constexpr uint32_t S_COL(int t) { return 128u * t; }
+    __host__ __device__ static constexpr uint32_t O_COL(int t) { return 256u + D * t; }
+    __host__ __device__ static constexpr uint32_t P_COL(int t) { return ALIAS ? 128u * t : 384u + 64u * t; }
+    // barrier indices
+    static constexpr int Q_FULL = 0;                     // [2]
+    static constexpr int K_FULL = 2, K_EMPTY = K_FULL + KS;
+    static constexpr int V_FULL = K_EMPTY + KS, V_EMPTY = V_FULL + VS;
+    static constexpr int S_FULL = V_EMPTY + VS;          // [2]
+    static constexpr int S_FREE = S_FULL + 2, P_FULL = S_FREE + 2, PV_DONE = P_FULL + 2;
+    static constexpr int NUM_BARS = PV_DONE + 2;
+};
+
+template <int D>
+__global__ void __launch_bounds__(THREADS, 1)
+fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                 const __grid_constant__ CUtensorMap tmV, __nv_bfloat16* __restrict__ O, int H, int Nq, int Nk,
+                 float scale_log2e, const int32_t* __restrict__ valid_len, int32_t* status) {
+    using LY = L2<D>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t* Qs = base;                                  // 2 tiles
+    uint8_t* Ks = Qs + 2 * LY::Q_BYTES;                  // KS tiles
+    uint8_t* Vs = Ks + LY::KS * LY::KV_BYTES;            // VS tiles
+    uint64_t* bars = reinterpret_cast<uint64_t*>(base + LY::TILE_BYTES);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + LY::NUM_BARS);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int bh = blockIdx.y;
+    const int row0 = blockIdx.x * (2 * BM);
+    int n = Nk;
+    if (valid_len) { n = valid_len[bh / H]; n = n < 0 ? 0 : (n > Nk ? Nk : n); }
+    const int ntiles = (n + BN - 1) / BN;
+
+    if (threadIdx.x == 8 * 32) {
+        for (int i = 0; i < LY::NUM_BARS; ++i) {
+            const bool by_softmax = (i >= LY::S_FREE && i < LY::PV_DONE);
+            mbar_init(&bars[i], by_softmax ? 128 : 1);
+        }
+        *abort_flag = 0;
+        fence_mbar_init();
+    }
+    if (warp == 0) { tmem_alloc(tmem_slot, 512); tmem_relinquish(); }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    if (warp >= 8) {
+      asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
+      if (warp == 8) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0 && ntiles > 0) {
+            prefetch_tensormap(&tmQ); prefetch_tensormap(&tmK); prefetch_tensormap(&tmV);
+            bool ok = true;
+            int k_issued = 0, v_issued = 0;
+            auto load_k = [&](int j) {
+                const int s = j % LY::KS;
+                ok = bounded_wait(&bars[LY::K_EMPTY + s], ((j / LY::KS) & 1) ^ 1, abort_flag, status, 0x100 + s);
+                if (!ok) return;
+                mbar_arrive_expect_tx(&bars[LY::K_FULL + s], LY::KV_BYTES);
+#pragma unroll
+                for (int c = 0; c < D / 64; ++c)
+                    tma_load_3d(Ks + s * LY::KV_BYTES + c * BN * 128, &tmK, &bars[LY::K_FULL + s], c * 64, j * BN, bh);
+                k_issued = j + 1;
+            };
+            auto load_v = [&](int j) {
+                const int s = j % LY::VS;
+                ok = bounded_wait(&bars[LY::V_EMPTY + s], ((j / LY::VS) & 1) ^ 1, abort_flag, status, 0x110 + s);
+                if (!ok) return;
+                mbar_arrive_expect_tx(&bars[LY::V_FULL + s], LY::KV_BYTES);
+#pragma unroll
+                for (int c = 0; c < D / 64; ++c)
+                    tma_load_3d(Vs + s * LY::KV_BYTES + c * BN * 128, &tmV, &bars[LY::V_FULL + s], c * 64, j * BN, bh);
+                v_issued = j + 1;
+            };
+            mbar_arrive_expect_tx(&bars[LY::Q_FULL + 0], LY::Q_BYTES);
+#pragma unroll
+            for (int c = 0; c < D / 64; ++c)
+                tma_load_3d(Qs + c * BM * 128, &tmQ, &bars[LY::Q_FULL + 0], c * 64, row0, bh);
+            load_k(0);
+            mbar_arrive_expect_tx(&bars[LY::Q_FULL + 1], LY::Q_BYTES);
+#pragma unroll
+            for (int c = 0; c < D / 64; ++c)
+                tma_load_3d(Qs + LY::Q_BYTES + c * BM * 128, &tmQ, &bars[LY::Q_FULL + 1], c * 64, row0 + BM, bh);
+            for (int j = 0; j < ntiles && ok; ++j) {
+                if (j + 1 < ntiles) load_k(j + 1);
+                if (ok) load_v(j);
+            }
+            if (!ok) {
+                drain_wait(&bars[LY::Q_FULL + 0], 0);
+                drain_wait(&bars[LY::Q_FULL + 1], 0);
+                for (int j = k_issued > LY::KS ? k_issued - LY::KS : 0; j < k_issued; ++j)
+                    drain_wait(&bars[LY::K_FULL + j % LY::KS], (j / LY::KS) & 1);
+                for (int j = v_issued > LY::VS ? v_issued - LY::VS : 0; j < v_issued; ++j)
+                    drain_wait(&bars[LY::V_FULL + j % LY::VS], (j / LY::VS) & 1);
+            }
+        }
+      } else if (warp == 9) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0 && ntiles > 0) {
+            constexpr uint32_t IDESC_S = make_idesc_bf16(BM, BN, 0, 0);
+            constexpr uint32_t IDESC_PV = make_idesc_bf16(BM, D, 0, 1);
+            const uint32_t q_addr = smem_u32(Qs), k_base = smem_u32(Ks), v_base = smem_u32(Vs);
+            bool ok = true;
+            auto wait = [&](int bar, uint32_t parity, int code) {
+                if (ok) ok = bounded_wait(&bars[bar], parity, abort_flag, status, code);
+                if (ok) tc_fence_after();
+            };
+            auto issue_s = [&](int t, int j) {           // S_t = Q_t K_j^T
+                const uint32_t qa = q_addr + t * LY::Q_BYTES, ka = k_base + (j % LY::KS) * LY::KV_BYTES;
+#pragma unroll
+                for (int k = 0; k < D / 16; ++k) {
+                    const uint32_t off = (k / 4) * (BM * 128) + (k % 4) * 32;
+                    mma_ss(tmem + LY::S_COL(t), make_smem_desc_sw128(qa + off, 16, 1024),
+                           make_smem_desc_sw128(ka + off, 16, 1024), IDESC_S, k > 0);
+                }
+                tc_commit(&bars[LY::S_FULL + t]);
+            };
+            auto issue_pv = [&](int t, int j) {          // O_t += P_t V_j
+                const uint32_t va = v_base + (j % LY::VS) * LY::KV_BYTES;
+#pragma unroll
+                for (int k = 0; k < BN / 16; ++k)
+                    mma_ts(tmem + LY::O_COL(t), tmem + LY::P_COL(t) + k * 8,
+                           make_smem_desc_sw128(va + k * 2048, BN * 128, 1024), IDESC_PV, (j > 0 || k > 0));
+                tc_commit(&bars[LY::PV_DONE + t]);
+            };
+            wait(LY::Q_FULL + 0, 0, 0x200);
+            wait(LY::K_FULL + 0, 0, 0x201);
+            if (ok) issue_s(0, 0);
+            wait(LY::Q_FULL + 1, 0, 0x202);
+            if (ok) { issue_s(1, 0); tc_commit(&bars[LY::K_EMPTY + 0]); }
+            for (int j = 0; j < ntiles && ok; ++j) {
+                const bool more = j + 1 < ntiles;
+                const int ks = (j + 1) % LY::KS, vs = j % LY::VS;
+                const uint32_t kph = ((j + 1) / LY::KS) & 1, vph = (j / LY::VS) & 1;
+                if (!LY::ALIAS) {
+                    if (more) {
+                        wait(LY::K_FULL + ks, kph, 0x210);
+                        wait(LY::S_FREE + 0, j & 1, 0x211);
+                        if (ok) issue_s(0, j + 1);
+                        wait(LY::S_FREE + 1, j & 1, 0x212);
+                        if (ok) { issue_s(1, j + 1); tc_commit(&bars[LY::K_EMPTY + ks]); }
+                    }
+                    wait(LY::V_FULL + vs, vph, 0x220);
+                    wait(LY::P_FULL + 0, j & 1, 0x221);
+                    if (ok) issue_pv(0, j);
+                    wait(LY::P_FULL + 1, j & 1, 0x222);
+                    if (ok) { issue_pv(1, j); tc_commit(&bars[LY::V_EMPTY + vs]); }
+                } else {
+                    wait(LY::V_FULL + vs, vph, 0x230);
+                    wait(LY::P_FULL + 0, j & 1, 0x231);
+                    if (ok) issue_pv(0, j);
+                    if (more) {
+                        wait(LY::K_FULL + ks, kph, 0x232);
+                        if (ok) issue_s(0, j + 1);
+                    }
+                    wait(LY::P_FULL + 1, j & 1, 0x233);
+                    if (ok) { issue_pv(1, j); tc_commit(&bars[LY::V_EMPTY + vs]); }
+                    if (more && ok) { issue_s(1, j + 1); tc_commit(&bars[LY::K_EMPTY + ks]); }
+                }
+            }
+        }
+      }
+    } else {
+        // ------------------------------------------------------------ softmax + epilogue (warps 0-7)
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
+        const int t = warp >> 2;                         // query tile of this warpgroup
+        const int row = row0 + t * BM + (warp & 3) * 32 + lane;
+        const uint32_t tl = tmem + (static_cast<uint32_t>((warp & 3) * 32) << 16);
+        const bool neg_scale = scale_log2e < 0.f;
+        float m_ref = -INFINITY, l = 0.f;
+        bool ok = true;
+        for (int j = 0; j < ntiles; ++j) {
+            ok = bounded_wait(&bars[LY::S_FULL + t], j & 1, abort_flag, status, 0x300 + t);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tc_fence_after();
+            uint32_t s[128];
+#pragma unroll
+            for (int c = 0; c < 4; ++c) tmem_ld_x32(tl + LY::S_COL(t) + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
+            tc_wait_ld();
+            tc_fence_before();
+            mbar_arrive(&bars[LY::S_FREE + t]);          // S_t may be overwritten (d = 64: by the next S_t)
+
+            const int col0 = j * BN;
+            const bool tail = col0 + BN > n;
+            if (tail) {
+                const uint32_t excl = __float_as_uint(neg_scale ? INFINITY : -INFINITY);
+#pragma unroll
+                for (int i = 0; i < 128; ++i) if (col0 + i >= n) s[i] = excl;
+            }
+            // row extremum of the raw logits, then scaled: max over j of scale * s_j
+            float e0 = __uint_as_float(s[0]), e1 = __uint_as_float(s[1]), e2 = __uint_as_float(s[2]), e3 = __uint_as_float(s[3]);
+            if (!neg_scale) {
+#pragma unroll
+                for (int i = 4; i < 128; i += 4) {
+                    e0 = fmaxf(e0, __uint_as_float(s[i])); e1 = fmaxf(e1, __uint_as_float(s[i + 1]));
+                    e2 = fmaxf(e2, __uint_as_float(s[i + 2])); e3 = fmaxf(e3, __uint_as_float(s[i + 3]));
+                }
+                e0 = fmaxf(fmaxf(e0, e1), fmaxf(e2, e3));
+            } else {
+#pragma unroll
+                for (int i = 4; i < 128; i += 4) {
+                    e0 = fminf(e0, __uint_as_float(s[i])); e1 = fminf(e1, __uint_as_float(s[i + 1]));
+                    e2 = fminf(e2, __uint_as_float(s[i + 2])); e3 = fminf(e3, __uint_as_float(s[i + 3]));
+                }
+                e0 = fminf(fminf(e0, e1), fminf(e2, e3));
+            }
+            const float mx = e0 * scale_log2e;
+            if (__any_sync(0xffffffffu, mx > m_ref + RESCALE_THRESHOLD)) {
+                const float m_new = fmaxf(m_ref, mx);
+                const float alpha = ex2_approx(m_ref - m_new);     // 0 on the first tile
+                l *= alpha;
+                if (j > 0) {
+                    ok = bounded_wait(&bars[LY::PV_DONE + t], (j - 1) & 1, abort_flag, status, 0x310 + t);
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok) break;
+                    tc_fence_after();
+#pragma unroll
+                    for (int c = 0; c < D / 32; ++c) {
+                        uint32_t r[32];
+                        tmem_ld_x32(tl + LY::O_COL(t) + c * 32, r);
+                        tc_wait_ld();
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
+                        tmem_st_x32(tl + LY::O_COL(t) + c * 32, r);
+                    }
+                }
+                m_ref = m_new;
+            }
+            if (!LY::ALIAS && j > 0) {
+                // P_t is a single buffer: O_t += P_t(j-1) V must have consumed it
+                ok = bounded_wait(&bars[LY::PV_DONE + t], (j - 1) & 1, abort_flag, status, 0x320 + t);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+            }
+            // p = 2^(scale*s - m_ref); row sum in fp32 from the unrounded p; P rounded to bf16
+            const float neg_m = -m_ref;
+            float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                uint32_t pk[16];
+#pragma unroll
+                for (int i = 0; i < 32; i += 4) {
+                    float p0 = ex2_approx(fmaf(__uint_as_float(s[c * 32 + i + 0]), scale_log2e, neg_m));
+                    float p1 = ex2_approx(fmaf(__uint_as_float(s[c * 32 + i + 1]), scale_log2e, neg_m));
+                    float p2 = ex2_approx(fmaf(__uint_as_float(s[c * 32 + i + 2]), scale_log2e, neg_m));
+                    float p3 = ex2_approx(fmaf(__uint_as_float(s[c * 32 + i + 3]), scale_log2e, neg_m));
+                    if (tail) {                           // also covers scale == 0 (inf * 0 = NaN)
+                        if (col0 + c * 32 + i + 0 >= n) p0 = 0.f;
+                        if (col0 + c * 32 + i + 1 >= n) p1 = 0.f;
+                        if (col0 + c * 32 + i + 2 >= n) p2 = 0.f;
+                        if (col0 + c * 32 + i + 3 >= n) p3 = 0.f;
+                    }
+                    l0 += p0; l1 += p1; l2 += p2; l3 += p3;
+                    pk[i / 2] = pack_bf16x2(p0, p1);
+                    pk[i / 2 + 1] = pack_bf16x2(p2, p3);
+                }
+                tmem_st_x16(tl + LY::P_COL(t) + c * 16, pk);
+            }
+            l += (l0 + l1) + (l2 + l3);
+            tc_wait_st();
+            tc_fence_before();
+            mbar_arrive(&bars[LY::P_FULL + t]);
+        }
+        if (ok && ntiles > 0) {
+            ok = bounded_wait(&bars[LY::PV_DONE + t], (ntiles - 1) & 1, abort_flag, status, 0x330 + t);
+            ok = __all_sync(0xffffffffu, ok);
+        }
+        if (ok) {
+            const float inv = l > 0.f ? 1.f / l : 0.f;
+            tc_fence_after();
+            __nv_bfloat16* orow = O + (static_cast<int64_t>(bh) * Nq + row) * D;
+#pragma unroll
+            for (int c = 0; c < D / 32; ++c) {
+                uint32_t r[32];
+                if (ntiles > 0) {
+                    tmem_ld_x32(tl + LY::O_COL(t) + c * 32, r);
+                    tc_wait_ld();
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) r[i] = 0u;      // no valid key: O = 0
+                }
+                if (row < Nq) {
+#pragma unroll
+                    for (int v = 0; v < 4; ++v) {
+                        uint4 w;
+                        w.x = pack_bf16x2(__uint_as_float(r[8 * v + 0]) * inv, __uint_as_float(r[8 * v + 1]) * inv);
+                        w.y = pack_bf16x2(__uint_as_float(r[8 * v + 2]) * inv, __uint_as_float(r[8 * v + 3]) * inv);
+                        w.z = pack_bf16x2(__uint_as_float(r[8 * v + 4]) * inv, __uint_as_float(r[8 * v + 5]) * inv);
+                        w.w = pack_bf16x2(__uint_as_float(r[8 * v + 6]) * inv, __uint_as_float(r[8 * v + 7]) * inv);
+                        *reinterpret_cast<uint4*>(orow + c * 32 + v * 8) = w;
+                    }
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem, 512);
+}
+
+template <int D>
+int launch_tc2_d(const Problem& p, cudaStream_t st) {
+    using LY = L2<D>;
+    CUtensorMap tmQ, tmK, tmV;
+    const int BH = p.B * p.H;
+    if (!make_map(&tmQ, p.Q, BH, p.Nq, D, BM) || !make_map(&tmK, p.K, BH, p.Nk, D, BN) ||
+        !make_map(&tmV, p.V, BH, p.Nk, D, BN))
+        return FLAT_ERR_CUDA;
+    auto kern = fused_tc2_kernel<D>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, LY::SMEM_BYTES) != cudaSuccess)
+        return FLAT_ERR_CUDA;
+    dim3 grid((p.Nq + 2 * BM - 1) / (2 * BM), BH);
+    kern<<<grid, THREADS, LY::SMEM_BYTES, st>>>(tmQ, tmK, tmV, static_cast<__nv_bfloat16*>(p.O), p.H, p.Nq, p.Nk,
+                                                p.scale * 1.4426950408889634f, p.k_valid_len, p.status);
+    return cudaGetLastError() == cudaSuccess ? FLAT_OK : FLAT_ERR_CUDA;
+}
+
+}  // namespace
+
+int launch_fused_tc2(const Problem& p, cudaStream_t st) {
+    if (p.dtype != FLAT_DTYPE_BF16) return FLAT_ERR_UNSUPPORTED;
+    if (p.d == 64) return launch_tc2_d<64>(p, st);
+    if (p.d == 128) return launch_tc2_d<128>(p, st);
+    return FLAT_ERR_UNSUPPORTED;
+}
+
+}  // namespace flat

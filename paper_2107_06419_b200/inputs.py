@@ -102,6 +102,9 @@ WORKLOADS = {
     "c3_16k": Workload("c3_16k", 4, 16, 16384, 16384, 64),
     "c4_64k_d128": Workload("c4_64k_d128", 1, 8, 65536, 65536, 128),
     "c5_cross_masked": Workload("c5_cross_masked", 8, 12, 1024, 16384, 64, masked=True),
+    # reduced copies of c2 / c4 for profiler captures (same tile shapes, a few hundred MB at most)
+    "p_4k_small": Workload("p_4k_small", 4, 16, 4096, 4096, 64),
+    "p_16k_d128_small": Workload("p_16k_d128_small", 1, 4, 16384, 16384, 128),
 }
 
 

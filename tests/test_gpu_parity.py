@@ -42,7 +42,7 @@ SMALL = [
 
 
 @pytest.mark.parametrize("shape", SMALL)
-@pytest.mark.parametrize("variant", [1, 2], ids=["simt", "tc"])
+@pytest.mark.parametrize("variant", [1, 2, 3], ids=["simt", "tc", "tc2"])
 def test_fused_bf16_small(api, shape, variant):
     B, H, Nq, Nk, d = shape
     rng = np.random.default_rng(abs(hash(shape)) % (2 ** 31))
@@ -53,7 +53,7 @@ def test_fused_bf16_small(api, shape, variant):
     check_bf16(got, ref, "fused bf16 %s v%d" % (shape, variant))
 
 
-@pytest.mark.parametrize("variant", [1, 2], ids=["simt", "tc"])
+@pytest.mark.parametrize("variant", [1, 2, 3], ids=["simt", "tc", "tc2"])
 @pytest.mark.parametrize("d", [64, 128])
 def test_fused_bf16_masked(api, variant, d):
     B, H, Nq, Nk = 5, 2, 200, 600
@@ -73,7 +73,7 @@ def test_fused_bf16_masked(api, variant, d):
     assert np.all(got[4] == 0.0)                            # no valid key: O = 0
 
 
-@pytest.mark.parametrize("variant", [1, 2], ids=["simt", "tc"])
+@pytest.mark.parametrize("variant", [1, 2, 3], ids=["simt", "tc", "tc2"])
 def test_fused_bf16_planted_keys(api, variant):
     """Peaked softmax on a planted key with position-coded V: a dropped, duplicated, shifted or
     mis-masked key tile moves O by O(1)."""
@@ -90,14 +90,15 @@ def test_fused_bf16_planted_keys(api, variant):
     check_bf16(got, ref["O"], "planted v%d" % variant)
 
 
-@pytest.mark.parametrize("scale", [1.0, 0.05, -0.125, 3.0])
+@pytest.mark.parametrize("scale", [1.0, 0.05, -0.125, 3.0, 0.0])
 def test_fused_bf16_scales_tc(api, scale):
     B, H, Nq, Nk, d = 1, 2, 256, 512, 64
     rng = np.random.default_rng(5)
     Qb, Kb, Vb = rand_bits(rng, (B, H, Nq, d)), rand_bits(rng, (B, H, Nk, d)), rand_bits(rng, (B, H, Nk, d))
     ref = oracle.attention(Qb, Kb, Vb, scale)["O"]
-    got = run_fused_bf16(api, Qb, Kb, Vb, scale, variant=2)
-    check_bf16(got, ref, "scale %g" % scale)
+    for variant in (2, 3):
+        got = run_fused_bf16(api, Qb, Kb, Vb, scale, variant=variant)
+        check_bf16(got, ref, "scale %g v%d" % (scale, variant))
 
 
 def test_rising_maximum_forces_rescale(api):
@@ -112,7 +113,7 @@ def test_rising_maximum_forces_rescale(api):
     ref = oracle.attention(Qb, Kb, Vb, 1.0, want_logits=True)
     L = ref["L"].reshape(Nq, Nk)
     assert np.all(L[:, -128:].max(1) - L[:, :128].max(1) > 20)      # > 8 log2 units per several tiles
-    for variant in (1, 2):
+    for variant in (1, 2, 3):
         got = run_fused_bf16(api, Qb, Kb, Vb, 1.0, variant=variant)
         check_bf16(got, ref["O"], "rising max v%d" % variant)
 
@@ -202,7 +203,7 @@ def test_output_padding_untouched(api):
     Qb, Kb, Vb = rand_bits(rng, (B, H, Nq, d)), rand_bits(rng, (B, H, Nk, d)), rand_bits(rng, (B, H, Nk, d))
     Q, K, V = bf16_tensor(Qb), bf16_tensor(Kb), bf16_tensor(Vb)
     n = B * H * Nq * d
-    for variant in (1, 2):
+    for variant in (1, 2, 3):
         buf = torch.full((n + 2048,), 7.0, dtype=torch.bfloat16, device="cuda")
         O = buf[1024:1024 + n].view(B, H, Nq, d)
         api.flat_attn_fwd_ex(Q, K, V, O, 0.125, variant=variant)
