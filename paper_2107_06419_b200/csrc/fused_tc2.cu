@@ -60,6 +60,74 @@ template <int D> struct L2 {
     static constexpr int NUM_BARS = PV_DONE + 2;
 };
 
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+__device__ __forceinline__ float min3(float a, float b, float c) {
+    float d;
+    asm("min.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+__device__ __forceinline__ float row_max(const uint32_t (&s)[128]) {
+    float e0 = __uint_as_float(s[0]), e1 = __uint_as_float(s[1]), e2 = __uint_as_float(s[2]), e3 = __uint_as_float(s[3]);
+#pragma unroll
+    for (int i = 4; i < 124; i += 8) {
+        e0 = max3(e0, __uint_as_float(s[i]), __uint_as_float(s[i + 1]));
+        e1 = max3(e1, __uint_as_float(s[i + 2]), __uint_as_float(s[i + 3]));
+        e2 = max3(e2, __uint_as_float(s[i + 4]), __uint_as_float(s[i + 5]));
+        e3 = max3(e3, __uint_as_float(s[i + 6]), __uint_as_float(s[i + 7]));
+    }
+    e0 = max3(e0, __uint_as_float(s[124]), __uint_as_float(s[125]));
+    e1 = max3(e1, __uint_as_float(s[126]), __uint_as_float(s[127]));
+    return fmaxf(fmaxf(e0, e1), fmaxf(e2, e3));
+}
+__device__ __forceinline__ float row_min(const uint32_t (&s)[128]) {
+    float e0 = __uint_as_float(s[0]), e1 = __uint_as_float(s[1]), e2 = __uint_as_float(s[2]), e3 = __uint_as_float(s[3]);
+#pragma unroll
+    for (int i = 4; i < 124; i += 8) {
+        e0 = min3(e0, __uint_as_float(s[i]), __uint_as_float(s[i + 1]));
+        e1 = min3(e1, __uint_as_float(s[i + 2]), __uint_as_float(s[i + 3]));
+        e2 = min3(e2, __uint_as_float(s[i + 4]), __uint_as_float(s[i + 5]));
+        e3 = min3(e3, __uint_as_float(s[i + 6]), __uint_as_float(s[i + 7]));
+    }
+    e0 = min3(e0, __uint_as_float(s[124]), __uint_as_float(s[125]));
+    e1 = min3(e1, __uint_as_float(s[126]), __uint_as_float(s[127]));
+    return fminf(fminf(e0, e1), fminf(e2, e3));
+}
+
+// p_i = 2^(s_i * scale + neg_m) for one row of 128 logits; stores bf16(p) to 64 TMEM columns at
+// `p_addr` and returns the fp32 sum of the unrounded p.  TAIL: only the first `nvalid` columns
+// take part, the rest get p = 0 (this also removes the NaN of inf * 0 when scale == 0).
+template <bool TAIL>
+__device__ __forceinline__ float exp_store(const uint32_t (&s)[128], float scale_log2e, float neg_m, uint32_t p_addr,
+                                           int nvalid) {
+    float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+        uint32_t pk[16];
+#pragma unroll
+        for (int i = 0; i < 32; i += 4) {
+            float p0 = ex2_approx(fmaf(__uint_as_float(s[c * 32 + i + 0]), scale_log2e, neg_m));
+            float p1 = ex2_approx(fmaf(__uint_as_float(s[c * 32 + i + 1]), scale_log2e, neg_m));
+            float p2 = ex2_approx(fmaf(__uint_as_float(s[c * 32 + i + 2]), scale_log2e, neg_m));
+            float p3 = ex2_approx(fmaf(__uint_as_float(s[c * 32 + i + 3]), scale_log2e, neg_m));
+            if (TAIL) {
+                if (c * 32 + i + 0 >= nvalid) p0 = 0.f;
+                if (c * 32 + i + 1 >= nvalid) p1 = 0.f;
+                if (c * 32 + i + 2 >= nvalid) p2 = 0.f;
+                if (c * 32 + i + 3 >= nvalid) p3 = 0.f;
+            }
+            l0 += p0; l1 += p1; l2 += p2; l3 += p3;
+            pk[i / 2] = pack_bf16x2(p0, p1);
+            pk[i / 2 + 1] = pack_bf16x2(p2, p3);
+        }
+        tmem_st_x16(p_addr + c * 16, pk);
+    }
+    return (l0 + l1) + (l2 + l3);
+}
+
 template <int D>
 __global__ void __launch_bounds__(THREADS, 1)
 fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
@@ -85,7 +153,7 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     if (threadIdx.x == 8 * 32) {
         for (int i = 0; i < LY::NUM_BARS; ++i) {
             const bool by_softmax = (i >= LY::S_FREE && i < LY::PV_DONE);
-            mbar_init(&bars[i], by_softmax ? 128 : 1);
+            mbar_init(&bars[i], by_softmax ? 4 : 1);         // one arrival per softmax warp
         }
         *abort_flag = 0;
         fence_mbar_init();
@@ -231,7 +299,8 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             for (int c = 0; c < 4; ++c) tmem_ld_x32(tl + LY::S_COL(t) + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
             tc_wait_ld();
             tc_fence_before();
-            mbar_arrive(&bars[LY::S_FREE + t]);          // S_t may be overwritten (d = 64: by the next S_t)
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&bars[LY::S_FREE + t]);   // S_t may be overwritten (d = 64: by the next S_t)
 
             const int col0 = j * BN;
             const bool tail = col0 + BN > n;
@@ -240,24 +309,8 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
 #pragma unroll
                 for (int i = 0; i < 128; ++i) if (col0 + i >= n) s[i] = excl;
             }
-            // row extremum of the raw logits, then scaled: max over j of scale * s_j
-            float e0 = __uint_as_float(s[0]), e1 = __uint_as_float(s[1]), e2 = __uint_as_float(s[2]), e3 = __uint_as_float(s[3]);
-            if (!neg_scale) {
-#pragma unroll
-                for (int i = 4; i < 128; i += 4) {
-                    e0 = fmaxf(e0, __uint_as_float(s[i])); e1 = fmaxf(e1, __uint_as_float(s[i + 1]));
-                    e2 = fmaxf(e2, __uint_as_float(s[i + 2])); e3 = fmaxf(e3, __uint_as_float(s[i + 3]));
-                }
-                e0 = fmaxf(fmaxf(e0, e1), fmaxf(e2, e3));
-            } else {
-#pragma unroll
-                for (int i = 4; i < 128; i += 4) {
-                    e0 = fminf(e0, __uint_as_float(s[i])); e1 = fminf(e1, __uint_as_float(s[i + 1]));
-                    e2 = fminf(e2, __uint_as_float(s[i + 2])); e3 = fminf(e3, __uint_as_float(s[i + 3]));
-                }
-                e0 = fminf(fminf(e0, e1), fminf(e2, e3));
-            }
-            const float mx = e0 * scale_log2e;
+            // row maximum of the scaled logits: scale * (max or min of the raw logits)
+            const float mx = (neg_scale ? row_min(s) : row_max(s)) * scale_log2e;
             if (__any_sync(0xffffffffu, mx > m_ref + RESCALE_THRESHOLD)) {
                 const float m_new = fmaxf(m_ref, mx);
                 const float alpha = ex2_approx(m_ref - m_new);     // 0 on the first tile
@@ -286,33 +339,12 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                 if (!ok) break;
             }
             // p = 2^(scale*s - m_ref); row sum in fp32 from the unrounded p; P rounded to bf16
-            const float neg_m = -m_ref;
-            float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                uint32_t pk[16];
-#pragma unroll
-                for (int i = 0; i < 32; i += 4) {
-                    float p0 = ex2_approx(fmaf(__uint_as_float(s[c * 32 + i + 0]), scale_log2e, neg_m));
-                    float p1 = ex2_approx(fmaf(__uint_as_float(s[c * 32 + i + 1]), scale_log2e, neg_m));
-                    float p2 = ex2_approx(fmaf(__uint_as_float(s[c * 32 + i + 2]), scale_log2e, neg_m));
-                    float p3 = ex2_approx(fmaf(__uint_as_float(s[c * 32 + i + 3]), scale_log2e, neg_m));
-                    if (tail) {                           // also covers scale == 0 (inf * 0 = NaN)
-                        if (col0 + c * 32 + i + 0 >= n) p0 = 0.f;
-                        if (col0 + c * 32 + i + 1 >= n) p1 = 0.f;
-                        if (col0 + c * 32 + i + 2 >= n) p2 = 0.f;
-                        if (col0 + c * 32 + i + 3 >= n) p3 = 0.f;
-                    }
-                    l0 += p0; l1 += p1; l2 += p2; l3 += p3;
-                    pk[i / 2] = pack_bf16x2(p0, p1);
-                    pk[i / 2 + 1] = pack_bf16x2(p2, p3);
-                }
-                tmem_st_x16(tl + LY::P_COL(t) + c * 16, pk);
-            }
-            l += (l0 + l1) + (l2 + l3);
+            if (tail) l += exp_store<true>(s, scale_log2e, -m_ref, tl + LY::P_COL(t), n - col0);
+            else      l += exp_store<false>(s, scale_log2e, -m_ref, tl + LY::P_COL(t), BN);
             tc_wait_st();
             tc_fence_before();
-            mbar_arrive(&bars[LY::P_FULL + t]);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&bars[LY::P_FULL + t]);
         }
         if (ok && ntiles > 0) {
             ok = bounded_wait(&bars[LY::PV_DONE + t], (ntiles - 1) & 1, abort_flag, status, 0x330 + t);
