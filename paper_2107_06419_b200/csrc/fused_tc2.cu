@@ -34,10 +34,30 @@ namespace flat {
 using namespace ptx;
 using namespace tc;
 
+#ifdef FLAT_TRACE
+// Developer tracing (off in the product build): CTA (0,0) records SM-clock timestamps.
+__device__ long long* g_trace = nullptr;
+extern "C" int flat_debug_set_trace(long long* p) {
+    return cudaMemcpyToSymbol(g_trace, &p, sizeof(p)) == cudaSuccess ? 0 : 6;
+}
+#define TRACE(role, iter, point)                                                              \
+    do {                                                                                      \
+        if (g_trace && blockIdx.x == 0 && blockIdx.y == 0 && (iter) < 64)                     \
+            g_trace[((role) * 64 + (iter)) * 8 + (point)] = clock64();                        \
+    } while (0)
+#else
+#define TRACE(role, iter, point) do { } while (0)
+#endif
+
 namespace {
 
 constexpr int BM = 128;              // rows per query tile (two tiles per CTA)
 constexpr int BN = 128;              // keys per step
+constexpr float OVERFLOW_SUM = 1.0995116e12f;   // 2^40: a tile row sum beyond this means m_ref is stale
+#ifndef FLAT_TURNS
+#define FLAT_TURNS 0
+#endif
+constexpr bool TAKE_TURNS = FLAT_TURNS != 0;
 constexpr int THREADS = 384;          // 3 warpgroups: softmax A, softmax B, {TMA, MMA, 2 idle warps}
 
 template <int D> struct L2 {
@@ -57,7 +77,8 @@ template <int D> struct L2 {
     static constexpr int V_FULL = K_EMPTY + KS, V_EMPTY = V_FULL + VS;
     static constexpr int S_FULL = V_EMPTY + VS;          // [2]
     static constexpr int S_FREE = S_FULL + 2, P_FULL = S_FREE + 2, PV_DONE = P_FULL + 2;
-    static constexpr int NUM_BARS = PV_DONE + 2;
+    static constexpr int TURN = PV_DONE + 2;             // [2][4]: exp-phase hand-over between the tiles, per warp
+    static constexpr int NUM_BARS = TURN + 8;
 };
 
 __device__ __forceinline__ float max3(float a, float b, float c) {
@@ -103,27 +124,30 @@ __device__ __forceinline__ float row_min(const uint32_t (&s)[128]) {
 template <bool TAIL>
 __device__ __forceinline__ float exp_store(const uint32_t (&s)[128], float scale_log2e, float neg_m, uint32_t p_addr,
                                            int nvalid) {
+    // Written as a software pipeline over the row: the scale-and-shift FFMA runs AHEAD elements in
+    // front of the ex2, whose results are summed and packed BEHIND elements later, so that
+    // consecutive ex2 never wait on a neighbour and the special-function unit stays fed.  The
+    // logits s[] are left intact (a stale reference maximum may force a second pass over them).
+    constexpr int AHEAD = 16, BEHIND = 16;
     float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
+    float q[128];                                       // short-lived: about AHEAD + BEHIND live at a time
+    uint32_t pk[16];
 #pragma unroll
-    for (int c = 0; c < 4; ++c) {
-        uint32_t pk[16];
+    for (int i = 0; i < AHEAD; ++i) q[i] = fmaf(__uint_as_float(s[i]), scale_log2e, neg_m);
 #pragma unroll
-        for (int i = 0; i < 32; i += 4) {
-            float p0 = ex2_approx(fmaf(__uint_as_float(s[c * 32 + i + 0]), scale_log2e, neg_m));
-            float p1 = ex2_approx(fmaf(__uint_as_float(s[c * 32 + i + 1]), scale_log2e, neg_m));
-            float p2 = ex2_approx(fmaf(__uint_as_float(s[c * 32 + i + 2]), scale_log2e, neg_m));
-            float p3 = ex2_approx(fmaf(__uint_as_float(s[c * 32 + i + 3]), scale_log2e, neg_m));
-            if (TAIL) {
-                if (c * 32 + i + 0 >= nvalid) p0 = 0.f;
-                if (c * 32 + i + 1 >= nvalid) p1 = 0.f;
-                if (c * 32 + i + 2 >= nvalid) p2 = 0.f;
-                if (c * 32 + i + 3 >= nvalid) p3 = 0.f;
-            }
-            l0 += p0; l1 += p1; l2 += p2; l3 += p3;
-            pk[i / 2] = pack_bf16x2(p0, p1);
-            pk[i / 2 + 1] = pack_bf16x2(p2, p3);
+    for (int i = 0; i < 128 + BEHIND; ++i) {
+        if (i + AHEAD < 128) q[i + AHEAD] = fmaf(__uint_as_float(s[i + AHEAD]), scale_log2e, neg_m);
+        if (i < 128) {
+            q[i] = ex2_approx(q[i]);
+            if (TAIL && i >= nvalid) q[i] = 0.f;
         }
-        tmem_st_x16(p_addr + c * 16, pk);
+        const int k = i - BEHIND;                       // element whose ex2 was issued BEHIND steps ago
+        if (k >= 0) {
+            const float p = q[k];
+            if ((k & 3) == 0) l0 += p; else if ((k & 3) == 1) l1 += p; else if ((k & 3) == 2) l2 += p; else l3 += p;
+            if (k & 1) pk[(k & 31) >> 1] = pack_bf16x2(q[k - 1], p);
+            if ((k & 31) == 31) tmem_st_x16(p_addr + (k >> 5) * 16, pk);
+        }
     }
     return (l0 + l1) + (l2 + l3);
 }
@@ -234,6 +258,7 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                            make_smem_desc_sw128(ka + off, 16, 1024), IDESC_S, k > 0);
                 }
                 tc_commit(&bars[LY::S_FULL + t]);
+                TRACE(2, j, t);
             };
             auto issue_pv = [&](int t, int j) {          // O_t += P_t V_j
                 const uint32_t va = v_base + (j % LY::VS) * LY::KV_BYTES;
@@ -242,6 +267,7 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                     mma_ts(tmem + LY::O_COL(t), tmem + LY::P_COL(t) + k * 8,
                            make_smem_desc_sw128(va + k * 2048, BN * 128, 1024), IDESC_PV, (j > 0 || k > 0));
                 tc_commit(&bars[LY::PV_DONE + t]);
+                TRACE(2, j, 2 + t);
             };
             wait(LY::Q_FULL + 0, 0, 0x200);
             wait(LY::K_FULL + 0, 0, 0x201);
@@ -289,11 +315,14 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         const bool neg_scale = scale_log2e < 0.f;
         float m_ref = -INFINITY, l = 0.f;
         bool ok = true;
+        if (TAKE_TURNS && t == 1 && lane == 0) mbar_arrive(&bars[LY::TURN + (warp & 3)]);   // tile A goes first
         for (int j = 0; j < ntiles; ++j) {
+            if ((warp & 3) == 0 && lane == 0) TRACE(t, j, 0);
             ok = bounded_wait(&bars[LY::S_FULL + t], j & 1, abort_flag, status, 0x300 + t);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
+            if ((warp & 3) == 0 && lane == 0) TRACE(t, j, 1);
             uint32_t s[128];
 #pragma unroll
             for (int c = 0; c < 4; ++c) tmem_ld_x32(tl + LY::S_COL(t) + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
@@ -301,6 +330,7 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&bars[LY::S_FREE + t]);   // S_t may be overwritten (d = 64: by the next S_t)
+            if ((warp & 3) == 0 && lane == 0) TRACE(t, j, 2);
 
             const int col0 = j * BN;
             const bool tail = col0 + BN > n;
@@ -309,42 +339,68 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
 #pragma unroll
                 for (int i = 0; i < 128; ++i) if (col0 + i >= n) s[i] = excl;
             }
-            // row maximum of the scaled logits: scale * (max or min of the raw logits)
-            const float mx = (neg_scale ? row_min(s) : row_max(s)) * scale_log2e;
-            if (__any_sync(0xffffffffu, mx > m_ref + RESCALE_THRESHOLD)) {
-                const float m_new = fmaxf(m_ref, mx);
-                const float alpha = ex2_approx(m_ref - m_new);     // 0 on the first tile
-                l *= alpha;
-                if (j > 0) {
-                    ok = bounded_wait(&bars[LY::PV_DONE + t], (j - 1) & 1, abort_flag, status, 0x310 + t);
-                    ok = __all_sync(0xffffffffu, ok);
-                    if (!ok) break;
-                    tc_fence_after();
-#pragma unroll
-                    for (int c = 0; c < D / 32; ++c) {
-                        uint32_t r[32];
-                        tmem_ld_x32(tl + LY::O_COL(t) + c * 32, r);
-                        tc_wait_ld();
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
-                        tmem_st_x32(tl + LY::O_COL(t) + c * 32, r);
-                    }
-                }
-                m_ref = m_new;
+            // Optional: the exponentials of the two query tiles take strict turns on each SM
+            // sub-partition's special-function unit (measured slower than free running: one warp
+            // alone does not keep that unit busy).
+            if (TAKE_TURNS) {
+                ok = bounded_wait(&bars[LY::TURN + t * 4 + (warp & 3)], j & 1, abort_flag, status, 0x340 + t);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
             }
+            if ((warp & 3) == 0 && lane == 0) TRACE(t, j, 3);
             if (!LY::ALIAS && j > 0) {
                 // P_t is a single buffer: O_t += P_t(j-1) V must have consumed it
                 ok = bounded_wait(&bars[LY::PV_DONE + t], (j - 1) & 1, abort_flag, status, 0x320 + t);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
             }
-            // p = 2^(scale*s - m_ref); row sum in fp32 from the unrounded p; P rounded to bf16
-            if (tail) l += exp_store<true>(s, scale_log2e, -m_ref, tl + LY::P_COL(t), n - col0);
-            else      l += exp_store<false>(s, scale_log2e, -m_ref, tl + LY::P_COL(t), BN);
+            if ((warp & 3) == 0 && lane == 0) TRACE(t, j, 4);
+            // p = 2^(scale*s - m_ref); row sum in fp32 from the unrounded p; P rounded to bf16.
+            // Any reference m_ref gives the exact softmax, so the common case reuses the one in
+            // hand and takes no row maximum at all; a row sum beyond 2^40 (or inf/NaN) shows that
+            // the reference fell too far behind, and the tile is then redone the careful way.
+            bool careful = (j == 0) || tail;
+            float lt = 0.f;
+            if (!careful) {
+                lt = exp_store<false>(s, scale_log2e, -m_ref, tl + LY::P_COL(t), BN);
+                careful = __any_sync(0xffffffffu, !(lt <= OVERFLOW_SUM));
+            }
+            if (careful) {
+                const float mx = (neg_scale ? row_min(s) : row_max(s)) * scale_log2e;
+                if (__any_sync(0xffffffffu, mx > m_ref + RESCALE_THRESHOLD)) {
+                    const float m_new = fmaxf(m_ref, mx);
+                    const float alpha = ex2_approx(m_ref - m_new);     // 0 on the first tile
+                    l *= alpha;
+                    if (j > 0) {
+                        ok = bounded_wait(&bars[LY::PV_DONE + t], (j - 1) & 1, abort_flag, status, 0x310 + t);
+                        ok = __all_sync(0xffffffffu, ok);
+                        if (!ok) break;
+                        tc_fence_after();
+#pragma unroll
+                        for (int c = 0; c < D / 32; ++c) {
+                            uint32_t r[32];
+                            tmem_ld_x32(tl + LY::O_COL(t) + c * 32, r);
+                            tc_wait_ld();
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
+                            tmem_st_x32(tl + LY::O_COL(t) + c * 32, r);
+                        }
+                    }
+                    m_ref = m_new;
+                }
+                lt = exp_store<true>(s, scale_log2e, -m_ref, tl + LY::P_COL(t), tail ? n - col0 : BN);
+            }
+            l += lt;
+            if (TAKE_TURNS) {
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&bars[LY::TURN + (t ^ 1) * 4 + (warp & 3)]);   // the other tile's turn
+            }
+            if ((warp & 3) == 0 && lane == 0) TRACE(t, j, 5);
             tc_wait_st();
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&bars[LY::P_FULL + t]);
+            if ((warp & 3) == 0 && lane == 0) TRACE(t, j, 6);
         }
         if (ok && ntiles > 0) {
             ok = bounded_wait(&bars[LY::PV_DONE + t], (ntiles - 1) & 1, abort_flag, status, 0x330 + t);
