@@ -10,8 +10,9 @@
 //   warps 0-3  softmax of query tile A   (thread r <-> row r of the tile <-> TMEM lane r)
 //   warps 4-7  softmax of query tile B
 //   warp  8    TMA producer (one lane): Q tiles once, then K and V tiles into separate rings
-//   warp  9    MMA issuer   (one lane): S_t = Q_t K^T and O_t += P_t V, t in {A, B}
-//   warps 10-11 idle (they only complete the warpgroup for the register hand-over)
+//   warp  9    MMA issuer of tile A (one elected lane): S_A = Q_A K^T and O_A += P_A V
+//   warp  10   MMA issuer of tile B
+//   warp  11   idle (it only completes the warpgroup for the register hand-over)
 // A softmax thread pulls its 128 logits into registers, releases the S buffer at once (so the next
 // S_t is computed while it works), takes the row maximum, writes bf16 weights P_t to TMEM and adds
 // to its row sum.  O_t is rescaled in TMEM only when a row maximum exceeds the reference by 2^8.
@@ -35,17 +36,20 @@ using namespace ptx;
 using namespace tc;
 
 #ifdef FLAT_TRACE
-// Developer tracing (off in the product build): CTA (0,0) records SM-clock timestamps.
-__device__ long long* g_trace = nullptr;
-extern "C" int flat_debug_set_trace(long long* p) {
+// Developer tracing (off in the product build): CTA (0,0) keeps SM-clock stamps in shared memory
+// and copies them to a global buffer when it ends.
+__device__ unsigned* g_trace = nullptr;
+extern "C" int flat_debug_set_trace(unsigned* p) {
     return cudaMemcpyToSymbol(g_trace, &p, sizeof(p)) == cudaSuccess ? 0 : 6;
 }
+#define TRACE_WORDS (3 * 64 * 8)
 #define TRACE(role, iter, point)                                                              \
     do {                                                                                      \
-        if (g_trace && blockIdx.x == 0 && blockIdx.y == 0 && (iter) < 64)                     \
-            g_trace[((role) * 64 + (iter)) * 8 + (point)] = clock64();                        \
+        if (blockIdx.x == 0 && blockIdx.y == 0 && (iter) < 64)                                \
+            trace_buf[((role) * 64 + (iter)) * 8 + (point)] = static_cast<unsigned>(clock64()); \
     } while (0)
 #else
+#define TRACE_WORDS 0
 #define TRACE(role, iter, point) do { } while (0)
 #endif
 
@@ -67,7 +71,7 @@ template <int D> struct L2 {
     static constexpr int Q_BYTES = BM * D * 2;           // one query tile
     static constexpr int KV_BYTES = BN * D * 2;
     static constexpr int TILE_BYTES = 2 * Q_BYTES + (KS + VS) * KV_BYTES;
-    static constexpr int SMEM_BYTES = TILE_BYTES + 512 + 1024;
+    static constexpr int SMEM_BYTES = TILE_BYTES + 512 + 1024 + 4 * TRACE_WORDS;
     __host__ __device__ static constexpr uint32_t S_COL(int t) { return 128u * t; }
     __host__ __device__ static constexpr uint32_t O_COL(int t) { return 256u + D * t; }
     __host__ __device__ static constexpr uint32_t P_COL(int t) { return ALIAS ? 128u * t : 384u + 64u * t; }
@@ -166,6 +170,10 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     uint64_t* bars = reinterpret_cast<uint64_t*>(base + LY::TILE_BYTES);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + LY::NUM_BARS);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+#ifdef FLAT_TRACE
+    volatile unsigned* trace_buf = reinterpret_cast<volatile unsigned*>(base + LY::TILE_BYTES + 512);
+    for (int i = threadIdx.x; i < TRACE_WORDS; i += THREADS) trace_buf[i] = 0;
+#endif
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int bh = blockIdx.y;
@@ -176,8 +184,9 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
 
     if (threadIdx.x == 8 * 32) {
         for (int i = 0; i < LY::NUM_BARS; ++i) {
-            const bool by_softmax = (i >= LY::S_FREE && i < LY::PV_DONE);
-            mbar_init(&bars[i], by_softmax ? 4 : 1);         // one arrival per softmax warp
+            const bool by_softmax = (i >= LY::S_FREE && i < LY::PV_DONE);      // one arrival per softmax warp
+            const bool by_issuers = (i >= LY::K_EMPTY && i < LY::V_FULL) || (i >= LY::V_EMPTY && i < LY::S_FULL);
+            mbar_init(&bars[i], by_softmax ? 4 : by_issuers ? 2 : 1);
         }
         *abort_flag = 0;
         fence_mbar_init();
@@ -238,70 +247,71 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                     drain_wait(&bars[LY::V_FULL + j % LY::VS], (j / LY::VS) & 1);
             }
         }
-      } else if (warp == 9) {
-        // ------------------------------------------------------------ MMA issuer
-        if (lane == 0 && ntiles > 0) {
+      } else if (warp == 9 || warp == 10) {
+        // ------------------------------------------------------------ MMA issuer of tile t
+        // The whole warp runs this loop (uniform control flow); one elected lane issues.
+        const int t = warp - 9;
+        if (ntiles > 0) {
             constexpr uint32_t IDESC_S = make_idesc_bf16(BM, BN, 0, 0);
             constexpr uint32_t IDESC_PV = make_idesc_bf16(BM, D, 0, 1);
-            const uint32_t q_addr = smem_u32(Qs), k_base = smem_u32(Ks), v_base = smem_u32(Vs);
+            const uint64_t q_desc = make_smem_desc_sw128(smem_u32(Qs) + t * LY::Q_BYTES, 16, 1024);
+            const uint64_t k_desc = make_smem_desc_sw128(smem_u32(Ks), 16, 1024);
+            const uint64_t v_desc = make_smem_desc_sw128(smem_u32(Vs), BN * 128, 1024);
+            const uint32_t s_tmem = tmem + LY::S_COL(t), o_tmem = tmem + LY::O_COL(t), p_tmem = tmem + LY::P_COL(t);
             bool ok = true;
             auto wait = [&](int bar, uint32_t parity, int code) {
-                if (ok) ok = bounded_wait(&bars[bar], parity, abort_flag, status, code);
+                if (ok) ok = __all_sync(0xffffffffu, bounded_wait(&bars[bar], parity, abort_flag, status, code));
                 if (ok) tc_fence_after();
             };
-            auto issue_s = [&](int t, int j) {           // S_t = Q_t K_j^T
-                const uint32_t qa = q_addr + t * LY::Q_BYTES, ka = k_base + (j % LY::KS) * LY::KV_BYTES;
+            auto issue_s = [&](int j) {                  // S_t = Q_t K_j^T, then release the K stage
+                const int ks = j % LY::KS;
+                if (elect_one()) {
+                    const uint64_t kd = k_desc + static_cast<uint64_t>((ks * LY::KV_BYTES) >> 4);
 #pragma unroll
-                for (int k = 0; k < D / 16; ++k) {
-                    const uint32_t off = (k / 4) * (BM * 128) + (k % 4) * 32;
-                    mma_ss(tmem + LY::S_COL(t), make_smem_desc_sw128(qa + off, 16, 1024),
-                           make_smem_desc_sw128(ka + off, 16, 1024), IDESC_S, k > 0);
+                    for (int k = 0; k < D / 16; ++k) {
+                        const uint64_t off = static_cast<uint64_t>(((k / 4) * (BM * 128) + (k % 4) * 32) >> 4);
+                        mma_ss(s_tmem, q_desc + off, kd + off, IDESC_S, k > 0);
+                    }
+                    tc_commit(&bars[LY::S_FULL + t]);
+                    tc_commit(&bars[LY::K_EMPTY + ks]);
+                    TRACE(2, j, t);
                 }
-                tc_commit(&bars[LY::S_FULL + t]);
-                TRACE(2, j, t);
+                __syncwarp();
             };
-            auto issue_pv = [&](int t, int j) {          // O_t += P_t V_j
-                const uint32_t va = v_base + (j % LY::VS) * LY::KV_BYTES;
+            auto issue_pv = [&](int j) {                 // O_t += P_t V_j, then release the V stage
+                const int vs = j % LY::VS;
+                if (elect_one()) {
+                    const uint64_t vd = v_desc + static_cast<uint64_t>((vs * LY::KV_BYTES) >> 4);
 #pragma unroll
-                for (int k = 0; k < BN / 16; ++k)
-                    mma_ts(tmem + LY::O_COL(t), tmem + LY::P_COL(t) + k * 8,
-                           make_smem_desc_sw128(va + k * 2048, BN * 128, 1024), IDESC_PV, (j > 0 || k > 0));
-                tc_commit(&bars[LY::PV_DONE + t]);
-                TRACE(2, j, 2 + t);
+                    for (int k = 0; k < BN / 16; ++k)
+                        mma_ts(o_tmem, p_tmem + k * 8, vd + static_cast<uint64_t>((k * 2048) >> 4), IDESC_PV,
+                               (j > 0 || k > 0));
+                    tc_commit(&bars[LY::PV_DONE + t]);
+                    tc_commit(&bars[LY::V_EMPTY + vs]);
+                    TRACE(2, j, 2 + t);
+                }
+                __syncwarp();
             };
-            wait(LY::Q_FULL + 0, 0, 0x200);
-            wait(LY::K_FULL + 0, 0, 0x201);
-            if (ok) issue_s(0, 0);
-            wait(LY::Q_FULL + 1, 0, 0x202);
-            if (ok) { issue_s(1, 0); tc_commit(&bars[LY::K_EMPTY + 0]); }
+            wait(LY::Q_FULL + t, 0, 0x200 + t);
+            wait(LY::K_FULL + 0, 0, 0x202);
+            if (ok) issue_s(0);
             for (int j = 0; j < ntiles && ok; ++j) {
                 const bool more = j + 1 < ntiles;
                 const int ks = (j + 1) % LY::KS, vs = j % LY::VS;
                 const uint32_t kph = ((j + 1) / LY::KS) & 1, vph = (j / LY::VS) & 1;
-                if (!LY::ALIAS) {
-                    if (more) {
-                        wait(LY::K_FULL + ks, kph, 0x210);
-                        wait(LY::S_FREE + 0, j & 1, 0x211);
-                        if (ok) issue_s(0, j + 1);
-                        wait(LY::S_FREE + 1, j & 1, 0x212);
-                        if (ok) { issue_s(1, j + 1); tc_commit(&bars[LY::K_EMPTY + ks]); }
-                    }
-                    wait(LY::V_FULL + vs, vph, 0x220);
-                    wait(LY::P_FULL + 0, j & 1, 0x221);
-                    if (ok) issue_pv(0, j);
-                    wait(LY::P_FULL + 1, j & 1, 0x222);
-                    if (ok) { issue_pv(1, j); tc_commit(&bars[LY::V_EMPTY + vs]); }
-                } else {
-                    wait(LY::V_FULL + vs, vph, 0x230);
-                    wait(LY::P_FULL + 0, j & 1, 0x231);
-                    if (ok) issue_pv(0, j);
-                    if (more) {
-                        wait(LY::K_FULL + ks, kph, 0x232);
-                        if (ok) issue_s(0, j + 1);
-                    }
-                    wait(LY::P_FULL + 1, j & 1, 0x233);
-                    if (ok) { issue_pv(1, j); tc_commit(&bars[LY::V_EMPTY + vs]); }
-                    if (more && ok) { issue_s(1, j + 1); tc_commit(&bars[LY::K_EMPTY + ks]); }
+                if (!LY::ALIAS && more) {
+                    // P has columns of its own: the next S_t only needs the softmax to have taken S_t(j)
+                    wait(LY::K_FULL + ks, kph, 0x210);
+                    wait(LY::S_FREE + t, j & 1, 0x211);
+                    if (ok) issue_s(j + 1);
+                }
+                wait(LY::V_FULL + vs, vph, 0x220);
+                wait(LY::P_FULL + t, j & 1, 0x221);
+                if (ok) issue_pv(j);
+                if (LY::ALIAS && more) {
+                    // P overlays S: the next S_t goes behind the MMA that reads P_t(j)
+                    wait(LY::K_FULL + ks, kph, 0x230);
+                    if (ok) issue_s(j + 1);
                 }
             }
         }
@@ -316,6 +326,9 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         float m_ref = -INFINITY, l = 0.f;
         bool ok = true;
         if (TAKE_TURNS && t == 1 && lane == 0) mbar_arrive(&bars[LY::TURN + (warp & 3)]);   // tile A goes first
+#ifdef FLAT_STAGGER_NS
+        if (t == 1) __nanosleep(FLAT_STAGGER_NS);
+#endif
         for (int j = 0; j < ntiles; ++j) {
             if ((warp & 3) == 0 && lane == 0) TRACE(t, j, 0);
             ok = bounded_wait(&bars[LY::S_FULL + t], j & 1, abort_flag, status, 0x300 + t);
@@ -437,6 +450,10 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     tc_fence_before();
     __syncthreads();
     if (warp == 0) tmem_dealloc(tmem, 512);
+#ifdef FLAT_TRACE
+    if (g_trace && blockIdx.x == 0 && blockIdx.y == 0)
+        for (int i = threadIdx.x; i < TRACE_WORDS; i += THREADS) g_trace[i] = trace_buf[i];
+#endif
 }
 
 template <int D>
