@@ -42,11 +42,11 @@ __device__ unsigned* g_trace = nullptr;
 extern "C" int flat_debug_set_trace(unsigned* p) {
     return cudaMemcpyToSymbol(g_trace, &p, sizeof(p)) == cudaSuccess ? 0 : 6;
 }
-#define TRACE_WORDS (3 * 64 * 8)
+#define TRACE_WORDS (3 * 64 * 16)
 #define TRACE(role, iter, point)                                                              \
     do {                                                                                      \
         if (blockIdx.x == 0 && blockIdx.y == 0 && (iter) < 64)                                \
-            trace_buf[((role) * 64 + (iter)) * 8 + (point)] = static_cast<unsigned>(clock64()); \
+            trace_buf[((role) * 64 + (iter)) * 16 + (point)] = static_cast<unsigned>(clock64()); \
     } while (0)
 #else
 #define TRACE_WORDS 0
@@ -58,10 +58,6 @@ namespace {
 constexpr int BM = 128;              // rows per query tile (two tiles per CTA)
 constexpr int BN = 128;              // keys per step
 constexpr float OVERFLOW_SUM = 1.0995116e12f;   // 2^40: a tile row sum beyond this means m_ref is stale
-#ifndef FLAT_TURNS
-#define FLAT_TURNS 0
-#endif
-constexpr bool TAKE_TURNS = FLAT_TURNS != 0;
 constexpr int THREADS = 384;          // 3 warpgroups: softmax A, softmax B, {TMA, MMA, 2 idle warps}
 
 template <int D> struct L2 {
@@ -81,8 +77,7 @@ template <int D> struct L2 {
     static constexpr int V_FULL = K_EMPTY + KS, V_EMPTY = V_FULL + VS;
     static constexpr int S_FULL = V_EMPTY + VS;          // [2]
     static constexpr int S_FREE = S_FULL + 2, P_FULL = S_FREE + 2, PV_DONE = P_FULL + 2;
-    static constexpr int TURN = PV_DONE + 2;             // [2][4]: exp-phase hand-over between the tiles, per warp
-    static constexpr int NUM_BARS = TURN + 8;
+    static constexpr int NUM_BARS = PV_DONE + 2;
 };
 
 __device__ __forceinline__ float max3(float a, float b, float c) {
@@ -125,13 +120,16 @@ __device__ __forceinline__ float row_min(const uint32_t (&s)[128]) {
 // p_i = 2^(s_i * scale + neg_m) for one row of 128 logits; stores bf16(p) to 64 TMEM columns at
 // `p_addr` and returns the fp32 sum of the unrounded p.  TAIL: only the first `nvalid` columns
 // take part, the rest get p = 0 (this also removes the NaN of inf * 0 when scale == 0).
-template <bool TAIL>
+template <bool TAIL, typename BeforeFirstStore>
 __device__ __forceinline__ float exp_store(const uint32_t (&s)[128], float scale_log2e, float neg_m, uint32_t p_addr,
-                                           int nvalid) {
+                                           int nvalid, BeforeFirstStore&& before_first_store,
+                                           volatile unsigned* trace_row = nullptr) {
     // Written as a software pipeline over the row: the scale-and-shift FFMA runs AHEAD elements in
     // front of the ex2, whose results are summed and packed BEHIND elements later, so that
     // consecutive ex2 never wait on a neighbour and the special-function unit stays fed.  The
     // logits s[] are left intact (a stale reference maximum may force a second pass over them).
+    // `before_first_store` runs once, just before the first write to the P buffer: by then a
+    // third of the row's ex2 have been issued, which hides the wait for the buffer to be free.
     constexpr int AHEAD = 16, BEHIND = 16;
     float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
     float q[128];                                       // short-lived: about AHEAD + BEHIND live at a time
@@ -150,7 +148,11 @@ __device__ __forceinline__ float exp_store(const uint32_t (&s)[128], float scale
             const float p = q[k];
             if ((k & 3) == 0) l0 += p; else if ((k & 3) == 1) l1 += p; else if ((k & 3) == 2) l2 += p; else l3 += p;
             if (k & 1) pk[(k & 31) >> 1] = pack_bf16x2(q[k - 1], p);
+            if (k == 31) before_first_store();
             if ((k & 31) == 31) tmem_st_x16(p_addr + (k >> 5) * 16, pk);
+#ifdef FLAT_TRACE
+            if ((k & 31) == 31 && trace_row != nullptr && (threadIdx.x & 127) == 0) trace_row[8 + (k >> 5)] = static_cast<unsigned>(clock64());
+#endif
         }
     }
     return (l0 + l1) + (l2 + l3);
@@ -260,7 +262,11 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             const uint32_t s_tmem = tmem + LY::S_COL(t), o_tmem = tmem + LY::O_COL(t), p_tmem = tmem + LY::P_COL(t);
             bool ok = true;
             auto wait = [&](int bar, uint32_t parity, int code) {
+#ifdef FLAT_MMA_SPIN
+                if (ok) ok = __all_sync(0xffffffffu, bounded_spin_wait(&bars[bar], parity, abort_flag, status, code));
+#else
                 if (ok) ok = __all_sync(0xffffffffu, bounded_wait(&bars[bar], parity, abort_flag, status, code));
+#endif
                 if (ok) tc_fence_after();
             };
             auto issue_s = [&](int j) {                  // S_t = Q_t K_j^T, then release the K stage
@@ -325,10 +331,6 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         const bool neg_scale = scale_log2e < 0.f;
         float m_ref = -INFINITY, l = 0.f;
         bool ok = true;
-        if (TAKE_TURNS && t == 1 && lane == 0) mbar_arrive(&bars[LY::TURN + (warp & 3)]);   // tile A goes first
-#ifdef FLAT_STAGGER_NS
-        if (t == 1) __nanosleep(FLAT_STAGGER_NS);
-#endif
         for (int j = 0; j < ntiles; ++j) {
             if ((warp & 3) == 0 && lane == 0) TRACE(t, j, 0);
             ok = bounded_wait(&bars[LY::S_FULL + t], j & 1, abort_flag, status, 0x300 + t);
@@ -352,21 +354,17 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
 #pragma unroll
                 for (int i = 0; i < 128; ++i) if (col0 + i >= n) s[i] = excl;
             }
-            // Optional: the exponentials of the two query tiles take strict turns on each SM
-            // sub-partition's special-function unit (measured slower than free running: one warp
-            // alone does not keep that unit busy).
-            if (TAKE_TURNS) {
-                ok = bounded_wait(&bars[LY::TURN + t * 4 + (warp & 3)], j & 1, abort_flag, status, 0x340 + t);
-                ok = __all_sync(0xffffffffu, ok);
-                if (!ok) break;
-            }
-            if ((warp & 3) == 0 && lane == 0) TRACE(t, j, 3);
-            if (!LY::ALIAS && j > 0) {
-                // P_t is a single buffer: O_t += P_t(j-1) V must have consumed it
-                ok = bounded_wait(&bars[LY::PV_DONE + t], (j - 1) & 1, abort_flag, status, 0x320 + t);
-                ok = __all_sync(0xffffffffu, ok);
-                if (!ok) break;
-            }
+            // At d = 64 P_t is a single buffer: O_t += P_t(j-1) V must have consumed it before the
+            // first store of P_t(j).  The wait sits inside the exponential pipeline (see exp_store).
+            bool pv_waited = LY::ALIAS || j == 0;
+            auto wait_p_free = [&]() {
+                if (!pv_waited) {
+                    ok = __all_sync(0xffffffffu, bounded_wait(&bars[LY::PV_DONE + t], (j - 1) & 1, abort_flag,
+                                                             status, 0x320 + t));
+                    pv_waited = true;
+                    if ((warp & 3) == 0 && lane == 0) TRACE(t, j, 3);
+                }
+            };
             if ((warp & 3) == 0 && lane == 0) TRACE(t, j, 4);
             // p = 2^(scale*s - m_ref); row sum in fp32 from the unrounded p; P rounded to bf16.
             // Any reference m_ref gives the exact softmax, so the common case reuses the one in
@@ -375,7 +373,13 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             bool careful = (j == 0) || tail;
             float lt = 0.f;
             if (!careful) {
-                lt = exp_store<false>(s, scale_log2e, -m_ref, tl + LY::P_COL(t), BN);
+#ifdef FLAT_TRACE
+                lt = exp_store<false>(s, scale_log2e, -m_ref, tl + LY::P_COL(t), BN, wait_p_free,
+                                      (blockIdx.x == 0 && blockIdx.y == 0 && j < 64) ? trace_buf + (t * 64 + j) * 16 : nullptr);
+#else
+                lt = exp_store<false>(s, scale_log2e, -m_ref, tl + LY::P_COL(t), BN, wait_p_free);
+#endif
+                if (!ok) break;                           // (a failed wait means the stores went nowhere useful)
                 careful = __any_sync(0xffffffffu, !(lt <= OVERFLOW_SUM));
             }
             if (careful) {
@@ -385,9 +389,10 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                     const float alpha = ex2_approx(m_ref - m_new);     // 0 on the first tile
                     l *= alpha;
                     if (j > 0) {
-                        ok = bounded_wait(&bars[LY::PV_DONE + t], (j - 1) & 1, abort_flag, status, 0x310 + t);
-                        ok = __all_sync(0xffffffffu, ok);
+                        ok = __all_sync(0xffffffffu, bounded_wait(&bars[LY::PV_DONE + t], (j - 1) & 1, abort_flag,
+                                                                 status, 0x310 + t));
                         if (!ok) break;
+                        pv_waited = true;
                         tc_fence_after();
 #pragma unroll
                         for (int c = 0; c < D / 32; ++c) {
@@ -401,13 +406,10 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                     }
                     m_ref = m_new;
                 }
-                lt = exp_store<true>(s, scale_log2e, -m_ref, tl + LY::P_COL(t), tail ? n - col0 : BN);
+                lt = exp_store<true>(s, scale_log2e, -m_ref, tl + LY::P_COL(t), tail ? n - col0 : BN, wait_p_free);
+                if (!ok) break;
             }
             l += lt;
-            if (TAKE_TURNS) {
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&bars[LY::TURN + (t ^ 1) * 4 + (warp & 3)]);   // the other tile's turn
-            }
             if ((warp & 3) == 0 && lane == 0) TRACE(t, j, 5);
             tc_wait_st();
             tc_fence_before();
