@@ -3,6 +3,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "../../include/flat_attn.h"
 
 namespace flat {
@@ -23,5 +25,21 @@ int launch_fused_simt(const Problem& p, cudaStream_t st);
 int launch_naive(const Problem& p, void* L, void* A, cudaStream_t st);
 int launch_fused_tc(const Problem& p, cudaStream_t st);
 int launch_fused_tc2(const Problem& p, cudaStream_t st);
+
+// Raises the dynamic shared-memory limit of `Kernel` once per device (the attribute is sticky,
+// and setting it on every call costs microseconds that small problems notice).
+template <auto Kernel>
+inline bool ensure_dynamic_smem(size_t bytes) {
+    static std::atomic<uint64_t> done{0};               // bit i: set for device ordinal i (< 64)
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return false;
+    const uint64_t bit = dev >= 0 && dev < 64 ? (1ull << dev) : 0;
+    if (bit && (done.load(std::memory_order_acquire) & bit)) return true;
+    if (cudaFuncSetAttribute(Kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(bytes)) !=
+        cudaSuccess)
+        return false;
+    if (bit) done.fetch_or(bit, std::memory_order_release);
+    return true;
+}
 
 }  // namespace flat

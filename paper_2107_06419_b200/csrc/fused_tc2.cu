@@ -467,8 +467,7 @@ int launch_tc2_d(const Problem& p, cudaStream_t st) {
         !make_map(&tmV, p.V, BH, p.Nk, D, BN))
         return FLAT_ERR_CUDA;
     auto kern = fused_tc2_kernel<D>;
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, LY::SMEM_BYTES) != cudaSuccess)
-        return FLAT_ERR_CUDA;
+    if (!ensure_dynamic_smem<fused_tc2_kernel<D>>(LY::SMEM_BYTES)) return FLAT_ERR_CUDA;
     dim3 grid((p.Nq + 2 * BM - 1) / (2 * BM), BH);
     kern<<<grid, THREADS, LY::SMEM_BYTES, st>>>(tmQ, tmK, tmV, static_cast<__nv_bfloat16*>(p.O), p.H, p.Nq, p.Nk,
                                                 p.scale * 1.4426950408889634f, p.k_valid_len, p.status);

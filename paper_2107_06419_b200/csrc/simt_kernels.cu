@@ -137,7 +137,7 @@ __global__ void __launch_bounds__(NTHREADS) fused_simt_kernel(const T* __restric
     const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
     const int64_t bh = blockIdx.y;
     const int64_t row0 = static_cast<int64_t>(blockIdx.x) * TM;
-    const int n = valid_len ? valid_len[bh / H] : Nk;
+    const int n = valid_len ? min(max(valid_len[bh / H], 0), Nk) : Nk;
     const T* Qg = Q + bh * Nq * D;
     const T* Kg = K + bh * Nk * D;
     const T* Vg = V + bh * Nk * D;
@@ -230,7 +230,7 @@ __global__ void __launch_bounds__(NTHREADS) naive_softmax_kernel(const float* __
                                                                  const int32_t* __restrict__ valid_len) {
     __shared__ float red_m[NTHREADS / 32], red_l[NTHREADS / 32];
     const int64_t row = blockIdx.x;
-    const int n = valid_len ? valid_len[(row / Nq) / H] : Nk;
+    const int n = valid_len ? min(max(valid_len[(row / Nq) / H], 0), Nk) : Nk;
     const float* Lr = L + row * Nk;
     TA* Ar = A + row * Nk;
     constexpr float LOG2E = 1.4426950408889634f;
@@ -271,7 +271,7 @@ __global__ void __launch_bounds__(NTHREADS) naive_attend_kernel(const TA* __rest
     const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
     const int64_t bh = blockIdx.y;
     const int64_t row0 = static_cast<int64_t>(blockIdx.x) * TM;
-    const int n = valid_len ? valid_len[bh / H] : Nk;
+    const int n = valid_len ? min(max(valid_len[bh / H], 0), Nk) : Nk;
     const TA* Ag = A + bh * Nq * Nk;
     float o[4][D / 16];
 #pragma unroll
@@ -299,15 +299,11 @@ __global__ void __launch_bounds__(NTHREADS) naive_attend_kernel(const TA* __rest
     }
 }
 
-template <typename K> static cudaError_t opt_in_smem(K kernel, size_t bytes) {
-    return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(bytes));
-}
-
 template <typename T, int D>
 static int launch_fused_simt_td(const Problem& p, cudaStream_t st) {
     auto kern = fused_simt_kernel<T, D>;
     const size_t smem = fused_smem_bytes<D>();
-    if (opt_in_smem(kern, smem) != cudaSuccess) return FLAT_ERR_CUDA;
+    if (!ensure_dynamic_smem<fused_simt_kernel<T, D>>(smem)) return FLAT_ERR_CUDA;
     dim3 grid((p.Nq + TM - 1) / TM, p.B * p.H);
     kern<<<grid, NTHREADS, smem, st>>>(static_cast<const T*>(p.Q), static_cast<const T*>(p.K),
                                        static_cast<const T*>(p.V), static_cast<T*>(p.O), p.H, p.Nq, p.Nk,
@@ -320,7 +316,7 @@ static int launch_naive_td(const Problem& p, float* L, void* A, cudaStream_t st)
     {
         auto kern = naive_logit_kernel<T, D>;
         const size_t smem = sizeof(float) * 2 * 64 * (D + 4);
-        if (opt_in_smem(kern, smem) != cudaSuccess) return FLAT_ERR_CUDA;
+        if (!ensure_dynamic_smem<naive_logit_kernel<T, D>>(smem)) return FLAT_ERR_CUDA;
         dim3 grid((p.Nk + TN - 1) / TN, (p.Nq + TM - 1) / TM, p.B * p.H);
         kern<<<grid, NTHREADS, smem, st>>>(static_cast<const T*>(p.Q), static_cast<const T*>(p.K), L, p.Nq, p.Nk,
                                            p.scale);
@@ -335,7 +331,7 @@ static int launch_naive_td(const Problem& p, float* L, void* A, cudaStream_t st)
     {
         auto kern = naive_attend_kernel<T, TA, D>;
         const size_t smem = sizeof(float) * (64 * D + 64 * PSTRIDE);
-        if (opt_in_smem(kern, smem) != cudaSuccess) return FLAT_ERR_CUDA;
+        if (!ensure_dynamic_smem<naive_attend_kernel<T, TA, D>>(smem)) return FLAT_ERR_CUDA;
         dim3 grid((p.Nq + TM - 1) / TM, p.B * p.H);
         kern<<<grid, NTHREADS, smem, st>>>(static_cast<const TA*>(A), static_cast<const T*>(p.V),
                                            static_cast<T*>(p.O), p.H, p.Nq, p.Nk, p.k_valid_len);
