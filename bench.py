@@ -182,6 +182,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--variant", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--with-naive", action="store_true",
+                    help="also time the unfused baseline (L and A materialised in device memory)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -292,6 +294,21 @@ def main():
                          "traffic": load_traffic(w.name, KERNEL_NAMES.get(args.variant, "fused_tc2_kernel")),
                          "algorithmic_bytes": w.qkvo_bytes()},
         }
+        if args.with_naive and world == 1:
+            # The paper's unfused baseline on the same inputs: L (fp32) and A (bf16) go through HBM.
+            elems = w.B * w.H * w.Nq * w.Nk
+            L = torch.empty((w.B, w.H, w.Nq, w.Nk), dtype=torch.float32, device=dev)
+            A = torch.empty((w.B, w.H, w.Nq, w.Nk), dtype=torch.bfloat16, device=dev)
+            O2 = torch.empty_like(Q)
+            naive = lambda: api.flat_attn_naive_fwd_ex(Q, K, V, O2, L, A, w.scale, k_valid_len=vld)
+            naive()
+            n_ms, _ = timed(naive, 3)
+            n_ms /= 3
+            out["naive"] = {"ms_per_step": n_ms, "value": float(w.flops) / (n_ms * 1e-3) / 1e12, "unit": UNIT,
+                            "kernels_per_step": 3, "materialised_bytes": 6 * elems,
+                            "algorithmic_bytes": 12 * elems + w.qkvo_bytes(),
+                            "max_abs_diff_vs_fused": float((O2.float() - O.float()).abs().max())}
+            del L, A, O2
         if not args.no_cpu_baseline and world == 1:
             cb, rows, Oref = cpu_baseline(w, Qb, Kb, Vb, vl)
             got = O.view(-1, w.d)[torch.from_numpy(rows).to(dev)].float().cpu().numpy().astype(np.float64)
