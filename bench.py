@@ -41,14 +41,16 @@ def load_peaks():
     return {"bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "hbm_gbs": 6650.0, "source": "fallback"}
 
 
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel, copied from
+# the ncu capture summarised in profiles/fused_tc2_kernel_dram_and_pipes.md (None where nothing was captured).
+MEASURED_DRAM_TRAFFIC = {
+    ("fused_tc2_kernel", "c2_bert_large_4k"): 514_700_000,
+    ("fused_tc2_kernel", "p_4k_small"): 117_000_000,
+}
+
+
 def load_traffic(workload, kernel="fused_tc2_kernel"):
-    """DRAM bytes per launch of the dominant kernel, from the committed ncu summary (or None)."""
-    path = os.path.join(ROOT, "profiles", "dram_traffic.json")
-    if not os.path.exists(path):
-        return None
-    with open(path) as f:
-        t = json.load(f)
-    return t.get(kernel, {}).get(workload)
+    return MEASURED_DRAM_TRAFFIC.get((kernel, workload))
 
 
 class ClockSampler:
@@ -64,7 +66,7 @@ class ClockSampler:
              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), "--query-gpu=" + q,
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "20"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
