@@ -57,6 +57,10 @@ namespace {
 
 constexpr int BM = 128;              // rows per query tile (two tiles per CTA)
 constexpr int BN = 128;              // keys per step
+#ifndef FLAT_POLY_LANE
+#define FLAT_POLY_LANE 3
+#endif
+constexpr int POLY_LANE = FLAT_POLY_LANE;       // element index mod 4 that uses ex2_poly; -1 = none
 constexpr float OVERFLOW_SUM = 1.0995116e12f;   // 2^40: a tile row sum beyond this means m_ref is stale
 constexpr int THREADS = 384;          // 3 warpgroups: softmax A, softmax B, {TMA, MMA, 2 idle warps}
 
@@ -124,36 +128,43 @@ template <bool TAIL, typename BeforeFirstStore>
 __device__ __forceinline__ float exp_store(const uint32_t (&s)[128], float scale_log2e, float neg_m, uint32_t p_addr,
                                            int nvalid, BeforeFirstStore&& before_first_store,
                                            volatile unsigned* trace_row = nullptr) {
-    // Written as a software pipeline over the row: the scale-and-shift FFMA runs AHEAD elements in
-    // front of the ex2, whose results are summed and packed BEHIND elements later, so that
-    // consecutive ex2 never wait on a neighbour and the special-function unit stays fed.  The
+    // Four chunks of 32 logits.  Within a chunk all FFMAs come first, then all exponentials, then
+    // the sums and the bf16 packing, so that consecutive ex2 never wait on a neighbour.  The
     // logits s[] are left intact (a stale reference maximum may force a second pass over them).
-    // `before_first_store` runs once, just before the first write to the P buffer: by then a
-    // third of the row's ex2 have been issued, which hides the wait for the buffer to be free.
-    constexpr int AHEAD = 16, BEHIND = 16;
+    // The first chunk's weights are held in registers until the second chunk is done:
+    // `before_first_store` (the wait for the P buffer to be free) then runs with a third of the
+    // row already computed, late enough for the previous tile's O += P V to have finished.
     float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
-    float q[128];                                       // short-lived: about AHEAD + BEHIND live at a time
-    uint32_t pk[16];
+    uint32_t pk0[16];
 #pragma unroll
-    for (int i = 0; i < AHEAD; ++i) q[i] = fmaf(__uint_as_float(s[i]), scale_log2e, neg_m);
+    for (int c = 0; c < 4; ++c) {
+        uint32_t pk[16];
+        float p[32];
 #pragma unroll
-    for (int i = 0; i < 128 + BEHIND; ++i) {
-        if (i + AHEAD < 128) q[i + AHEAD] = fmaf(__uint_as_float(s[i + AHEAD]), scale_log2e, neg_m);
-        if (i < 128) {
-            q[i] = ex2_approx(q[i]);
-            if (TAIL && i >= nvalid) q[i] = 0.f;
+        for (int i = 0; i < 32; ++i) p[i] = fmaf(__uint_as_float(s[c * 32 + i]), scale_log2e, neg_m);
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+            // One element in four takes the polynomial route (FMA pipe) to unload the ex2 unit,
+            // the binding pipe at d = 64; the careful/tail pass keeps to ex2 throughout.
+            p[i] = (!TAIL && (i & 3) == POLY_LANE) ? ex2_poly(p[i]) : ex2_approx(p[i]);
+            if (TAIL && c * 32 + i >= nvalid) p[i] = 0.f;
         }
-        const int k = i - BEHIND;                       // element whose ex2 was issued BEHIND steps ago
-        if (k >= 0) {
-            const float p = q[k];
-            if ((k & 3) == 0) l0 += p; else if ((k & 3) == 1) l1 += p; else if ((k & 3) == 2) l2 += p; else l3 += p;
-            if (k & 1) pk[(k & 31) >> 1] = pack_bf16x2(q[k - 1], p);
-            if (k == 31) before_first_store();
-            if ((k & 31) == 31) tmem_st_x16(p_addr + (k >> 5) * 16, pk);
+#pragma unroll
+        for (int i = 0; i < 32; i += 4) {
+            l0 += p[i]; l1 += p[i + 1]; l2 += p[i + 2]; l3 += p[i + 3];
+            pk[i / 2] = pack_bf16x2(p[i], p[i + 1]);
+            pk[i / 2 + 1] = pack_bf16x2(p[i + 2], p[i + 3]);
+        }
+        if (c == 0) {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) pk0[i] = pk[i];
+        } else {
+            if (c == 1) { before_first_store(); tmem_st_x16(p_addr, pk0); }
+            tmem_st_x16(p_addr + c * 16, pk);
+        }
 #ifdef FLAT_TRACE
-            if ((k & 31) == 31 && trace_row != nullptr && (threadIdx.x & 127) == 0) trace_row[8 + (k >> 5)] = static_cast<unsigned>(clock64());
+        if (trace_row != nullptr && (threadIdx.x & 127) == 0) trace_row[8 + c] = static_cast<unsigned>(clock64());
 #endif
-        }
     }
     return (l0 + l1) + (l2 + l3);
 }
@@ -287,11 +298,13 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             auto issue_pv = [&](int j) {                 // O_t += P_t V_j, then release the V stage
                 const int vs = j % LY::VS;
                 if (elect_one()) {
+                    if (t == 0) TRACE(2, j, 4);
                     const uint64_t vd = v_desc + static_cast<uint64_t>((vs * LY::KV_BYTES) >> 4);
 #pragma unroll
                     for (int k = 0; k < BN / 16; ++k)
                         mma_ts(o_tmem, p_tmem + k * 8, vd + static_cast<uint64_t>((k * 2048) >> 4), IDESC_PV,
                                (j > 0 || k > 0));
+                    if (t == 0) TRACE(2, j, 5);
                     tc_commit(&bars[LY::PV_DONE + t]);
                     tc_commit(&bars[LY::V_EMPTY + vs]);
                     TRACE(2, j, 2 + t);
@@ -312,7 +325,9 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                     if (ok) issue_s(j + 1);
                 }
                 wait(LY::V_FULL + vs, vph, 0x220);
+                if (t == 0 && lane == 0) TRACE(2, j, 6);
                 wait(LY::P_FULL + t, j & 1, 0x221);
+                if (t == 0 && lane == 0) TRACE(2, j, 7);
                 if (ok) issue_pv(j);
                 if (LY::ALIAS && more) {
                     // P overlays S: the next S_t goes behind the MMA that reads P_t(j)
@@ -359,6 +374,7 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             bool pv_waited = LY::ALIAS || j == 0;
             auto wait_p_free = [&]() {
                 if (!pv_waited) {
+                    if ((warp & 3) == 0 && lane == 0) TRACE(t, j, 7);
                     ok = __all_sync(0xffffffffu, bounded_wait(&bars[LY::PV_DONE + t], (j - 1) & 1, abort_flag,
                                                              status, 0x320 + t));
                     pv_waited = true;

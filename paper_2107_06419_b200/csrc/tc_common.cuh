@@ -68,6 +68,23 @@ __device__ __forceinline__ float ex2_approx(float x) {
     return y;
 }
 
+// 2^x on the FMA and integer pipes instead of the ex2 unit: x = r + f with r = round(x) and
+// f in [-0.5, 0.5]; 2^f by a cubic (max relative error 7.7e-5, far below the bf16 rounding that
+// the weights undergo next) and 2^r by adding r to the exponent field.  x is clamped to
+// [-127, 126] so that the exponent arithmetic cannot wrap: below, the result is ~2^-127 (as good
+// as 0 next to a row maximum of order 1); above, it is 2^126, which trips the caller's overflow
+// check exactly like the ex2 unit's +inf would.
+__device__ __forceinline__ float ex2_poly(float x) {
+    x = fminf(fmaxf(x, -127.f), 126.f);
+    const float t = x + 12582912.f;                    // 1.5 * 2^23: the low mantissa bits now hold round(x)
+    const float r = t - 12582912.f;
+    const float f = x - r;
+    float p = fmaf(0.05508868f, f, 0.24260405f);
+    p = fmaf(p, f, 0.69327624f);
+    p = fmaf(p, f, 0.99992894f);
+    return __uint_as_float(__float_as_uint(p) + (__float_as_uint(t) << 23));
+}
+
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t*>(&h);
