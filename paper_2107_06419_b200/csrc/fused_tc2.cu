@@ -57,6 +57,13 @@ namespace {
 
 constexpr int BM = 128;              // rows per query tile (two tiles per CTA)
 constexpr int BN = 128;              // keys per step
+#ifndef FLAT_TURNS_EXPR
+#define FLAT_TURNS_EXPR (D == 128)
+#endif
+#ifndef FLAT_PASS_AT
+#define FLAT_PASS_AT 3
+#endif
+constexpr int PASS_AT_CHUNK = FLAT_PASS_AT;     // the other tile gets its turn once this chunk's ex2 are issued
 #ifndef FLAT_POLY_LANE
 #define FLAT_POLY_LANE 3
 #endif
@@ -81,7 +88,13 @@ template <int D> struct L2 {
     static constexpr int V_FULL = K_EMPTY + KS, V_EMPTY = V_FULL + VS;
     static constexpr int S_FULL = V_EMPTY + VS;          // [2]
     static constexpr int S_FREE = S_FULL + 2, P_FULL = S_FREE + 2, PV_DONE = P_FULL + 2;
-    static constexpr int NUM_BARS = PV_DONE + 2;
+    static constexpr int TURN = PV_DONE + 2;             // [2][4]: per warp pair, "tile t may run its exponentials"
+    static constexpr int NUM_BARS = TURN + 8;
+    // Strict alternation of the two tiles' exponential phases.  At d = 128 the chain of a tile is
+    // softmax -> (O += P V, next S) -> softmax with nothing to overlap inside the tile, so the tiles
+    // must interleave: one computes exponentials while the other's MMAs run.  Left to themselves
+    // they fall into lockstep and the phases add up instead.
+    static constexpr bool TURNS = FLAT_TURNS_EXPR;
 };
 
 __device__ __forceinline__ float max3(float a, float b, float c) {
@@ -124,10 +137,10 @@ __device__ __forceinline__ float row_min(const uint32_t (&s)[128]) {
 // p_i = 2^(s_i * scale + neg_m) for one row of 128 logits; stores bf16(p) to 64 TMEM columns at
 // `p_addr` and returns the fp32 sum of the unrounded p.  TAIL: only the first `nvalid` columns
 // take part, the rest get p = 0 (this also removes the NaN of inf * 0 when scale == 0).
-template <bool TAIL, typename BeforeFirstStore>
+template <bool TAIL, typename BeforeFirstStore, typename AfterLastExp>
 __device__ __forceinline__ float exp_store(const uint32_t (&s)[128], float scale_log2e, float neg_m, uint32_t p_addr,
                                            int nvalid, BeforeFirstStore&& before_first_store,
-                                           volatile unsigned* trace_row = nullptr) {
+                                           AfterLastExp&& after_last_exp, volatile unsigned* trace_row = nullptr) {
     // Four chunks of 32 logits.  Within a chunk all FFMAs come first, then all exponentials, then
     // the sums and the bf16 packing, so that consecutive ex2 never wait on a neighbour.  The
     // logits s[] are left intact (a stale reference maximum may force a second pass over them).
@@ -149,6 +162,7 @@ __device__ __forceinline__ float exp_store(const uint32_t (&s)[128], float scale
             p[i] = (!TAIL && (i & 3) == POLY_LANE) ? ex2_poly(p[i]) : ex2_approx(p[i]);
             if (TAIL && c * 32 + i >= nvalid) p[i] = 0.f;
         }
+        if (c == PASS_AT_CHUNK) after_last_exp();       // (nearly) every ex2 of the row has been issued
 #pragma unroll
         for (int i = 0; i < 32; i += 4) {
             l0 += p[i]; l1 += p[i + 1]; l2 += p[i + 2]; l3 += p[i + 3];
@@ -346,6 +360,7 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         const bool neg_scale = scale_log2e < 0.f;
         float m_ref = -INFINITY, l = 0.f;
         bool ok = true;
+        if (LY::TURNS && t == 1 && lane == 0) mbar_arrive(&bars[LY::TURN + (warp & 3)]);   // tile A goes first
         for (int j = 0; j < ntiles; ++j) {
             if ((warp & 3) == 0 && lane == 0) TRACE(t, j, 0);
             ok = bounded_wait(&bars[LY::S_FULL + t], j & 1, abort_flag, status, 0x300 + t);
@@ -381,6 +396,19 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                     if ((warp & 3) == 0 && lane == 0) TRACE(t, j, 3);
                 }
             };
+            bool turn_passed = !LY::TURNS;
+            auto pass_turn = [&]() {
+                if (!turn_passed) {
+                    turn_passed = true;
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&bars[LY::TURN + (t ^ 1) * 4 + (warp & 3)]);
+                }
+            };
+            if (LY::TURNS) {
+                ok = __all_sync(0xffffffffu, bounded_wait(&bars[LY::TURN + t * 4 + (warp & 3)], j & 1, abort_flag,
+                                                         status, 0x340 + t));
+                if (!ok) break;
+            }
             if ((warp & 3) == 0 && lane == 0) TRACE(t, j, 4);
             // p = 2^(scale*s - m_ref); row sum in fp32 from the unrounded p; P rounded to bf16.
             // Any reference m_ref gives the exact softmax, so the common case reuses the one in
@@ -390,10 +418,10 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             float lt = 0.f;
             if (!careful) {
 #ifdef FLAT_TRACE
-                lt = exp_store<false>(s, scale_log2e, -m_ref, tl + LY::P_COL(t), BN, wait_p_free,
+                lt = exp_store<false>(s, scale_log2e, -m_ref, tl + LY::P_COL(t), BN, wait_p_free, pass_turn,
                                       (blockIdx.x == 0 && blockIdx.y == 0 && j < 64) ? trace_buf + (t * 64 + j) * 16 : nullptr);
 #else
-                lt = exp_store<false>(s, scale_log2e, -m_ref, tl + LY::P_COL(t), BN, wait_p_free);
+                lt = exp_store<false>(s, scale_log2e, -m_ref, tl + LY::P_COL(t), BN, wait_p_free, pass_turn);
 #endif
                 if (!ok) break;                           // (a failed wait means the stores went nowhere useful)
                 careful = __any_sync(0xffffffffu, !(lt <= OVERFLOW_SUM));
@@ -422,7 +450,8 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                     }
                     m_ref = m_new;
                 }
-                lt = exp_store<true>(s, scale_log2e, -m_ref, tl + LY::P_COL(t), tail ? n - col0 : BN, wait_p_free);
+                lt = exp_store<true>(s, scale_log2e, -m_ref, tl + LY::P_COL(t), tail ? n - col0 : BN, wait_p_free,
+                                     pass_turn);
                 if (!ok) break;
             }
             l += lt;
