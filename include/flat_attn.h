@@ -112,8 +112,14 @@ int flat_attn_naive_fwd_ex(const flat_attn_params_t* p, void* L, void* A, void* 
 /*
  * End-to-end convenience call with HOST tensors: copies Q, K, V (and k_valid_len if
  * non-NULL) from host memory into `workspace`, runs the fused kernel, copies O back
- * to `O_host`, all on `stream`, and returns without synchronising (use pinned host
- * memory for true asynchrony; the caller synchronises the stream before reading O).
+ * to `O_host`, and returns without synchronising (use pinned host memory for true
+ * asynchrony; the caller synchronises `stream` before reading O).  The work is cut
+ * into up to 8 independent slices (whole batches, or groups of heads when B == 1)
+ * that run on two internal side streams forked from and joined back into `stream`,
+ * so that the transfer of one slice overlaps the kernel and the read-back of its
+ * neighbours; to the caller it behaves like work enqueued on `stream`.  The side
+ * streams and events are created once per device and host thread and never freed
+ * (no device memory is allocated).
  * p->Q, p->K, p->V, p->O and p->k_valid_len are HOST pointers here; p->status is
  * still a device pointer or NULL.  `workspace` is a caller-owned DEVICE buffer of at
  * least flat_attn_host_workspace_bytes(...) bytes, 256-byte aligned.

@@ -70,6 +70,30 @@ int run_fused(const flat::Problem& q, int variant, cudaStream_t st) {
 
 inline size_t round256(size_t x) { return (x + 255) & ~static_cast<size_t>(255); }
 
+// Side streams and events of flat_attn_fwd_host, one set per device and host thread, created on
+// first use and kept until the process exits.
+struct HostPipe {
+    cudaStream_t side[2];
+    cudaEvent_t fork, join[2];
+};
+
+HostPipe* host_pipe() {
+    thread_local HostPipe pipes[16];
+    thread_local bool ready[16] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 16) return nullptr;
+    if (!ready[dev]) {
+        HostPipe& h = pipes[dev];
+        if (cudaStreamCreateWithFlags(&h.side[0], cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+        if (cudaStreamCreateWithFlags(&h.side[1], cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+        if (cudaEventCreateWithFlags(&h.fork, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+        if (cudaEventCreateWithFlags(&h.join[0], cudaEventDisableTiming) != cudaSuccess) return nullptr;
+        if (cudaEventCreateWithFlags(&h.join[1], cudaEventDisableTiming) != cudaSuccess) return nullptr;
+        ready[dev] = true;
+    }
+    return &pipes[dev];
+}
+
 }  // namespace
 
 extern "C" {
@@ -138,16 +162,57 @@ int flat_attn_fwd_host(const flat_attn_params_t* p, void* workspace, size_t work
     const int rc = validate(&dev, &q);
     if (rc != FLAT_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (cudaMemcpyAsync(dQ, p->Q, qb, cudaMemcpyHostToDevice, st) != cudaSuccess) return FLAT_ERR_CUDA;
-    if (cudaMemcpyAsync(dK, p->K, kb, cudaMemcpyHostToDevice, st) != cudaSuccess) return FLAT_ERR_CUDA;
-    if (cudaMemcpyAsync(dV, p->V, kb, cudaMemcpyHostToDevice, st) != cudaSuccess) return FLAT_ERR_CUDA;
     if (p->k_valid_len &&
         cudaMemcpyAsync(dLen, p->k_valid_len, sizeof(int32_t) * p->B, cudaMemcpyHostToDevice, st) != cudaSuccess)
         return FLAT_ERR_CUDA;
-    const int r = run_fused(q, p->variant, st);
-    if (r != FLAT_OK) return r;
-    if (cudaMemcpyAsync(p->O, dO, qb, cudaMemcpyDeviceToHost, st) != cudaSuccess) return FLAT_ERR_CUDA;
-    g_last_launches = 1;
+
+    // Pipeline over independent slices (whole batches, or groups of heads when B == 1): the copy of
+    // slice c+1 overlaps the kernel of slice c and the read-back of slice c-1.  Two side streams
+    // (created once per device; streams and events are not device memory) fork from `stream` and
+    // join it again, so the caller sees ordinary stream semantics.
+    HostPipe* hp = host_pipe();
+    const int units = p->B > 1 ? p->B : p->H;            // slices are cut along this axis
+    int nslices = units < 8 ? units : 8;
+    if (!hp || nslices < 2) {
+        if (cudaMemcpyAsync(dQ, p->Q, qb, cudaMemcpyHostToDevice, st) != cudaSuccess) return FLAT_ERR_CUDA;
+        if (cudaMemcpyAsync(dK, p->K, kb, cudaMemcpyHostToDevice, st) != cudaSuccess) return FLAT_ERR_CUDA;
+        if (cudaMemcpyAsync(dV, p->V, kb, cudaMemcpyHostToDevice, st) != cudaSuccess) return FLAT_ERR_CUDA;
+        const int r = run_fused(q, p->variant, st);
+        if (r != FLAT_OK) return r;
+        if (cudaMemcpyAsync(p->O, dO, qb, cudaMemcpyDeviceToHost, st) != cudaSuccess) return FLAT_ERR_CUDA;
+        g_last_launches = 1;
+        return FLAT_OK;
+    }
+    if (cudaEventRecord(hp->fork, st) != cudaSuccess) return FLAT_ERR_CUDA;
+    for (int i = 0; i < 2; ++i)
+        if (cudaStreamWaitEvent(hp->side[i], hp->fork, 0) != cudaSuccess) return FLAT_ERR_CUDA;
+    const size_t q_unit = qb / units, k_unit = kb / units;   // bytes per batch (or per head when B == 1)
+    int launches = 0;
+    for (int c = 0; c < nslices; ++c) {
+        const int u0 = static_cast<int>(static_cast<int64_t>(units) * c / nslices);
+        const int u1 = static_cast<int>(static_cast<int64_t>(units) * (c + 1) / nslices);
+        if (u1 == u0) continue;
+        cudaStream_t ss = hp->side[c & 1];
+        const size_t qo = q_unit * u0, ko = k_unit * u0, qn = q_unit * (u1 - u0), kn = k_unit * (u1 - u0);
+        if (cudaMemcpyAsync(dQ + qo, static_cast<const char*>(p->Q) + qo, qn, cudaMemcpyHostToDevice, ss) != cudaSuccess ||
+            cudaMemcpyAsync(dK + ko, static_cast<const char*>(p->K) + ko, kn, cudaMemcpyHostToDevice, ss) != cudaSuccess ||
+            cudaMemcpyAsync(dV + ko, static_cast<const char*>(p->V) + ko, kn, cudaMemcpyHostToDevice, ss) != cudaSuccess)
+            return FLAT_ERR_CUDA;
+        flat::Problem sub = q;
+        sub.Q = dQ + qo; sub.K = dK + ko; sub.V = dV + ko; sub.O = dO + qo;
+        if (p->B > 1) { sub.B = u1 - u0; if (sub.k_valid_len) sub.k_valid_len += u0; }
+        else          { sub.H = u1 - u0; }
+        const int r = run_fused(sub, p->variant, ss);
+        if (r != FLAT_OK) return r;
+        ++launches;
+        if (cudaMemcpyAsync(static_cast<char*>(p->O) + qo, dO + qo, qn, cudaMemcpyDeviceToHost, ss) != cudaSuccess)
+            return FLAT_ERR_CUDA;
+    }
+    for (int i = 0; i < 2; ++i) {
+        if (cudaEventRecord(hp->join[i], hp->side[i]) != cudaSuccess) return FLAT_ERR_CUDA;
+        if (cudaStreamWaitEvent(st, hp->join[i], 0) != cudaSuccess) return FLAT_ERR_CUDA;
+    }
+    g_last_launches = launches;
     return FLAT_OK;
 }
 

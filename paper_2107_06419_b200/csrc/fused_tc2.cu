@@ -203,6 +203,9 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
 #endif
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+#ifdef FLAT_TRACE
+    const unsigned t_entry = static_cast<unsigned>(clock64());
+#endif
     const int bh = blockIdx.y;
     const int row0 = blockIdx.x * (2 * BM);
     int n = Nk;
@@ -223,6 +226,9 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
+#ifdef FLAT_TRACE
+    if (threadIdx.x == 0) { TRACE(2, 63, 0); trace_buf[(2 * 64 + 63) * 16 + 1] = t_entry; }
+#endif
 
     if (warp >= 8) {
       asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
@@ -494,8 +500,14 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             }
         }
     }
+#ifdef FLAT_TRACE
+    if (threadIdx.x == 0) TRACE(2, 63, 2);               // softmax warp 0 done with its epilogue
+#endif
     tc_fence_before();
     __syncthreads();
+#ifdef FLAT_TRACE
+    if (threadIdx.x == 0) TRACE(2, 63, 3);
+#endif
     if (warp == 0) tmem_dealloc(tmem, 512);
 #ifdef FLAT_TRACE
     if (g_trace && blockIdx.x == 0 && blockIdx.y == 0)
