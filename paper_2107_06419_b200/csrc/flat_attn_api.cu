@@ -37,18 +37,6 @@ bool tc_applies(const flat::Problem& q) {
     return q.dtype == FLAT_DTYPE_BF16 && (q.d == 64 || q.d == 128);
 }
 
-int sm_count() {
-    thread_local int cached_dev = -1, cached_sms = 0;
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
-    if (dev != cached_dev) {
-        int sms = 0;
-        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) return 148;
-        cached_dev = dev; cached_sms = sms;
-    }
-    return cached_sms;
-}
-
 int run_fused(const flat::Problem& q, int variant, cudaStream_t st) {
     int v = variant;
     if (v == FLAT_VARIANT_AUTO) {
@@ -58,7 +46,7 @@ int run_fused(const flat::Problem& q, int variant, cudaStream_t st) {
             // Two-tile CTAs (256 query rows) once they fill every SM; otherwise 128-row CTAs,
             // which give twice as many CTAs for small problems.
             const int64_t ctas2 = static_cast<int64_t>((q.Nq + 255) / 256) * q.B * q.H;
-            v = ctas2 >= sm_count() ? FLAT_VARIANT_TC2 : FLAT_VARIANT_TC;
+            v = ctas2 >= flat::device_sm_count() ? FLAT_VARIANT_TC2 : FLAT_VARIANT_TC;
         }
     }
     if (v == FLAT_VARIANT_TC || v == FLAT_VARIANT_TC2) {

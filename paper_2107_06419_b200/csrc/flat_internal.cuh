@@ -42,4 +42,18 @@ inline bool ensure_dynamic_smem(size_t bytes) {
     return true;
 }
 
+// Number of SMs of the current device (cached per host thread); 148 if the query fails.
+inline int device_sm_count() {
+    thread_local int cached_dev = -1, cached_sms = 0;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+    if (dev != cached_dev) {
+        int sms = 0;
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) return 148;
+        cached_dev = dev;
+        cached_sms = sms;
+    }
+    return cached_sms;
+}
+
 }  // namespace flat
