@@ -28,7 +28,8 @@ METRIC = "fused attention TFLOP/s"
 UNIT = "TFLOP/s"
 DEFAULT_WORKLOAD = "c2_bert_large_4k"
 L2_FLUSH_BELOW = 256 << 20          # workloads smaller than this get an L2 flush before every timed launch
-KERNEL_NAMES = {0: "fused_tc2_kernel", 1: "fused_simt_kernel", 2: "fused_tc_kernel", 3: "fused_tc2_kernel"}
+KERNEL_NAMES = {0: "fused_tc2_kernel", 1: "fused_simt_kernel", 2: "fused_tc_kernel", 3: "fused_tc2_kernel",
+                4: "fused_tc2_kernel"}
 
 
 def load_peaks():

@@ -64,8 +64,10 @@ enum {
     FLAT_VARIANT_SIMT = 1,     /* fp32 FFMA kernel, any supported d and dtype                  */
     FLAT_VARIANT_TC = 2,       /* tcgen05 + TMEM + TMA kernel, one 128-row tile per CTA:
                                   bf16, d in {64,128}                                          */
-    FLAT_VARIANT_TC2 = 3       /* same, two 128-row tiles per CTA ping-ponging on the tensor
+    FLAT_VARIANT_TC2 = 3,      /* same, two 128-row tiles per CTA ping-ponging on the tensor
                                   pipe (the default for problems that fill the GPU)            */
+    FLAT_VARIANT_TC2_SINGLE = 4 /* the TC2 pipeline with one 128-row tile per CTA and two CTAs
+                                  per SM: bf16, d = 64 only                                    */
 };
 
 typedef struct flat_attn_params {

@@ -25,6 +25,7 @@ int launch_fused_simt(const Problem& p, cudaStream_t st);
 int launch_naive(const Problem& p, void* L, void* A, cudaStream_t st);
 int launch_fused_tc(const Problem& p, cudaStream_t st);
 int launch_fused_tc2(const Problem& p, cudaStream_t st);
+int launch_fused_tc2_single(const Problem& p, cudaStream_t st);
 
 // Raises the dynamic shared-memory limit of `Kernel` once per device (the attribute is sticky,
 // and setting it on every call costs microseconds that small problems notice).

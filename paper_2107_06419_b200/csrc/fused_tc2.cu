@@ -69,32 +69,34 @@ constexpr int PASS_AT_CHUNK = FLAT_PASS_AT;     // the other tile gets its turn 
 #endif
 constexpr int POLY_LANE = FLAT_POLY_LANE;       // element index mod 4 that uses ex2_poly; -1 = none
 constexpr float OVERFLOW_SUM = 1.0995116e12f;   // 2^40: a tile row sum beyond this means m_ref is stale
-constexpr int THREADS = 384;          // 3 warpgroups: softmax A, softmax B, {TMA, MMA, 2 idle warps}
 
-template <int D> struct L2 {
+template <int D, int NT> struct L2 {
     static constexpr bool ALIAS = (D == 128);            // P overlays S
-    static constexpr int KS = (D == 64) ? 3 : 2;         // K ring depth
-    static constexpr int VS = (D == 64) ? 3 : 2;         // V ring depth
+    static constexpr int KS = (NT == 1) ? 2 : (D == 64) ? 3 : 2;   // K ring depth
+    static constexpr int VS = KS;                        // V ring depth
+    static constexpr int THREADS = 128 * NT + 128;       // NT softmax warpgroups + {TMA, NT MMA issuers, idle}
+    static constexpr int SOFT_WARPS = 4 * NT;
+    static constexpr uint32_t TMEM_COLS = (NT == 2) ? 512 : 256;
     static constexpr int Q_BYTES = BM * D * 2;           // one query tile
     static constexpr int KV_BYTES = BN * D * 2;
-    static constexpr int TILE_BYTES = 2 * Q_BYTES + (KS + VS) * KV_BYTES;
+    static constexpr int TILE_BYTES = NT * Q_BYTES + (KS + VS) * KV_BYTES;
     static constexpr int SMEM_BYTES = TILE_BYTES + 512 + 1024 + 4 * TRACE_WORDS;
     __host__ __device__ static constexpr uint32_t S_COL(int t) { return 128u * t; }
-    __host__ __device__ static constexpr uint32_t O_COL(int t) { return 256u + D * t; }
-    __host__ __device__ static constexpr uint32_t P_COL(int t) { return ALIAS ? 128u * t : 384u + 64u * t; }
+    __host__ __device__ static constexpr uint32_t O_COL(int t) { return 128u * NT + D * t; }
+    __host__ __device__ static constexpr uint32_t P_COL(int t) { return ALIAS ? 128u * t : 128u * NT + D * NT + 64u * t; }
     // barrier indices
-    static constexpr int Q_FULL = 0;                     // [2]
-    static constexpr int K_FULL = 2, K_EMPTY = K_FULL + KS;
+    static constexpr int Q_FULL = 0;                     // [NT]
+    static constexpr int K_FULL = NT, K_EMPTY = K_FULL + KS;
     static constexpr int V_FULL = K_EMPTY + KS, V_EMPTY = V_FULL + VS;
-    static constexpr int S_FULL = V_EMPTY + VS;          // [2]
-    static constexpr int S_FREE = S_FULL + 2, P_FULL = S_FREE + 2, PV_DONE = P_FULL + 2;
-    static constexpr int TURN = PV_DONE + 2;             // [2][4]: per warp pair, "tile t may run its exponentials"
+    static constexpr int S_FULL = V_EMPTY + VS;          // [NT]
+    static constexpr int S_FREE = S_FULL + NT, P_FULL = S_FREE + NT, PV_DONE = P_FULL + NT;
+    static constexpr int TURN = PV_DONE + NT;            // [2][4]: per warp pair, "tile t may run its exponentials"
     static constexpr int NUM_BARS = TURN + 8;
     // Strict alternation of the two tiles' exponential phases.  At d = 128 the chain of a tile is
     // softmax -> (O += P V, next S) -> softmax with nothing to overlap inside the tile, so the tiles
     // must interleave: one computes exponentials while the other's MMAs run.  Left to themselves
     // they fall into lockstep and the phases add up instead.
-    static constexpr bool TURNS = FLAT_TURNS_EXPR;
+    static constexpr bool TURNS = (NT == 2) && FLAT_TURNS_EXPR;
 };
 
 __device__ __forceinline__ float max3(float a, float b, float c) {
@@ -183,16 +185,17 @@ __device__ __forceinline__ float exp_store(const uint32_t (&s)[128], float scale
     return (l0 + l1) + (l2 + l3);
 }
 
-template <int D>
-__global__ void __launch_bounds__(THREADS, 1)
+template <int D, int NT>
+__global__ void __launch_bounds__(128 * NT + 128, NT == 1 ? 2 : 1)
 fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                  const __grid_constant__ CUtensorMap tmV, __nv_bfloat16* __restrict__ O, int H, int Nq, int Nk,
                  float scale_log2e, const int32_t* __restrict__ valid_len, int32_t* status) {
-    using LY = L2<D>;
+    using LY = L2<D, NT>;
+    constexpr int THREADS = LY::THREADS;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    uint8_t* Qs = base;                                  // 2 tiles
-    uint8_t* Ks = Qs + 2 * LY::Q_BYTES;                  // KS tiles
+    uint8_t* Qs = base;                                  // NT tiles
+    uint8_t* Ks = Qs + NT * LY::Q_BYTES;                  // KS tiles
     uint8_t* Vs = Ks + LY::KS * LY::KV_BYTES;            // VS tiles
     uint64_t* bars = reinterpret_cast<uint64_t*>(base + LY::TILE_BYTES);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + LY::NUM_BARS);
@@ -207,21 +210,21 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     const unsigned t_entry = static_cast<unsigned>(clock64());
 #endif
     const int bh = blockIdx.y;
-    const int row0 = blockIdx.x * (2 * BM);
+    const int row0 = blockIdx.x * (NT * BM);
     int n = Nk;
     if (valid_len) { n = valid_len[bh / H]; n = n < 0 ? 0 : (n > Nk ? Nk : n); }
     const int ntiles = (n + BN - 1) / BN;
 
-    if (threadIdx.x == 8 * 32) {
+    if (threadIdx.x == LY::SOFT_WARPS * 32) {
         for (int i = 0; i < LY::NUM_BARS; ++i) {
             const bool by_softmax = (i >= LY::S_FREE && i < LY::PV_DONE);      // one arrival per softmax warp
             const bool by_issuers = (i >= LY::K_EMPTY && i < LY::V_FULL) || (i >= LY::V_EMPTY && i < LY::S_FULL);
-            mbar_init(&bars[i], by_softmax ? 4 : by_issuers ? 2 : 1);
+            mbar_init(&bars[i], by_softmax ? 4 : by_issuers ? NT : 1);
         }
         *abort_flag = 0;
         fence_mbar_init();
     }
-    if (warp == 0) { tmem_alloc(tmem_slot, 512); tmem_relinquish(); }
+    if (warp == 0) { tmem_alloc(tmem_slot, LY::TMEM_COLS); tmem_relinquish(); }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -230,9 +233,10 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     if (threadIdx.x == 0) { TRACE(2, 63, 0); trace_buf[(2 * 64 + 63) * 16 + 1] = t_entry; }
 #endif
 
-    if (warp >= 8) {
-      asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
-      if (warp == 8) {
+    if (warp >= LY::SOFT_WARPS) {
+      if (NT == 2) asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
+      else         asm volatile("setmaxnreg.dec.sync.aligned.u32 48;");
+      if (warp == LY::SOFT_WARPS) {
         // ------------------------------------------------------------ TMA producer
         if (lane == 0 && ntiles > 0) {
             prefetch_tensormap(&tmQ); prefetch_tensormap(&tmK); prefetch_tensormap(&tmV);
@@ -263,27 +267,30 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             for (int c = 0; c < D / 64; ++c)
                 tma_load_3d(Qs + c * BM * 128, &tmQ, &bars[LY::Q_FULL + 0], c * 64, row0, bh);
             load_k(0);
-            mbar_arrive_expect_tx(&bars[LY::Q_FULL + 1], LY::Q_BYTES);
+            if (NT == 2) {
+                mbar_arrive_expect_tx(&bars[LY::Q_FULL + NT - 1], LY::Q_BYTES);
 #pragma unroll
-            for (int c = 0; c < D / 64; ++c)
-                tma_load_3d(Qs + LY::Q_BYTES + c * BM * 128, &tmQ, &bars[LY::Q_FULL + 1], c * 64, row0 + BM, bh);
+                for (int c = 0; c < D / 64; ++c)
+                    tma_load_3d(Qs + (NT - 1) * LY::Q_BYTES + c * BM * 128, &tmQ, &bars[LY::Q_FULL + NT - 1], c * 64,
+                                row0 + BM, bh);
+            }
             for (int j = 0; j < ntiles && ok; ++j) {
                 if (j + 1 < ntiles) load_k(j + 1);
                 if (ok) load_v(j);
             }
             if (!ok) {
                 drain_wait(&bars[LY::Q_FULL + 0], 0);
-                drain_wait(&bars[LY::Q_FULL + 1], 0);
+                if (NT == 2) drain_wait(&bars[LY::Q_FULL + NT - 1], 0);
                 for (int j = k_issued > LY::KS ? k_issued - LY::KS : 0; j < k_issued; ++j)
                     drain_wait(&bars[LY::K_FULL + j % LY::KS], (j / LY::KS) & 1);
                 for (int j = v_issued > LY::VS ? v_issued - LY::VS : 0; j < v_issued; ++j)
                     drain_wait(&bars[LY::V_FULL + j % LY::VS], (j / LY::VS) & 1);
             }
         }
-      } else if (warp == 9 || warp == 10) {
+      } else if (warp <= LY::SOFT_WARPS + NT) {
         // ------------------------------------------------------------ MMA issuer of tile t
         // The whole warp runs this loop (uniform control flow); one elected lane issues.
-        const int t = warp - 9;
+        const int t = warp - LY::SOFT_WARPS - 1;
         if (ntiles > 0) {
             constexpr uint32_t IDESC_S = make_idesc_bf16(BM, BN, 0, 0);
             constexpr uint32_t IDESC_PV = make_idesc_bf16(BM, D, 0, 1);
@@ -359,7 +366,8 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       }
     } else {
         // ------------------------------------------------------------ softmax + epilogue (warps 0-7)
-        asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
+        if (NT == 2) asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
+        else         asm volatile("setmaxnreg.inc.sync.aligned.u32 208;");
         const int t = warp >> 2;                         // query tile of this warpgroup
         const int row = row0 + t * BM + (warp & 3) * 32 + lane;
         const uint32_t tl = tmem + (static_cast<uint32_t>((warp & 3) * 32) << 16);
@@ -508,26 +516,26 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
 #ifdef FLAT_TRACE
     if (threadIdx.x == 0) TRACE(2, 63, 3);
 #endif
-    if (warp == 0) tmem_dealloc(tmem, 512);
+    if (warp == 0) tmem_dealloc(tmem, LY::TMEM_COLS);
 #ifdef FLAT_TRACE
     if (g_trace && blockIdx.x == 0 && blockIdx.y == 0)
         for (int i = threadIdx.x; i < TRACE_WORDS; i += THREADS) g_trace[i] = trace_buf[i];
 #endif
 }
 
-template <int D>
+template <int D, int NT>
 int launch_tc2_d(const Problem& p, cudaStream_t st) {
-    using LY = L2<D>;
+    using LY = L2<D, NT>;
     CUtensorMap tmQ, tmK, tmV;
     const int BH = p.B * p.H;
     if (!make_map(&tmQ, p.Q, BH, p.Nq, D, BM) || !make_map(&tmK, p.K, BH, p.Nk, D, BN) ||
         !make_map(&tmV, p.V, BH, p.Nk, D, BN))
         return FLAT_ERR_CUDA;
-    auto kern = fused_tc2_kernel<D>;
-    if (!ensure_dynamic_smem<fused_tc2_kernel<D>>(LY::SMEM_BYTES)) return FLAT_ERR_CUDA;
-    dim3 grid((p.Nq + 2 * BM - 1) / (2 * BM), BH);
-    kern<<<grid, THREADS, LY::SMEM_BYTES, st>>>(tmQ, tmK, tmV, static_cast<__nv_bfloat16*>(p.O), p.H, p.Nq, p.Nk,
-                                                p.scale * 1.4426950408889634f, p.k_valid_len, p.status);
+    auto kern = fused_tc2_kernel<D, NT>;
+    if (!ensure_dynamic_smem<fused_tc2_kernel<D, NT>>(LY::SMEM_BYTES)) return FLAT_ERR_CUDA;
+    dim3 grid((p.Nq + NT * BM - 1) / (NT * BM), BH);
+    kern<<<grid, LY::THREADS, LY::SMEM_BYTES, st>>>(tmQ, tmK, tmV, static_cast<__nv_bfloat16*>(p.O), p.H, p.Nq,
+                                                    p.Nk, p.scale * 1.4426950408889634f, p.k_valid_len, p.status);
     return cudaGetLastError() == cudaSuccess ? FLAT_OK : FLAT_ERR_CUDA;
 }
 
@@ -535,8 +543,15 @@ int launch_tc2_d(const Problem& p, cudaStream_t st) {
 
 int launch_fused_tc2(const Problem& p, cudaStream_t st) {
     if (p.dtype != FLAT_DTYPE_BF16) return FLAT_ERR_UNSUPPORTED;
-    if (p.d == 64) return launch_tc2_d<64>(p, st);
-    if (p.d == 128) return launch_tc2_d<128>(p, st);
+    if (p.d == 64) return launch_tc2_d<64, 2>(p, st);
+    if (p.d == 128) return launch_tc2_d<128, 2>(p, st);
+    return FLAT_ERR_UNSUPPORTED;
+}
+
+// One 128-row tile per CTA, two CTAs per SM (d = 64 only: at d = 128 two CTAs do not fit in shared memory).
+int launch_fused_tc2_single(const Problem& p, cudaStream_t st) {
+    if (p.dtype != FLAT_DTYPE_BF16) return FLAT_ERR_UNSUPPORTED;
+    if (p.d == 64) return launch_tc2_d<64, 1>(p, st);
     return FLAT_ERR_UNSUPPORTED;
 }
 

@@ -42,9 +42,11 @@ SMALL = [
 
 
 @pytest.mark.parametrize("shape", SMALL)
-@pytest.mark.parametrize("variant", [1, 2, 3], ids=["simt", "tc", "tc2"])
+@pytest.mark.parametrize("variant", [1, 2, 3, 4], ids=["simt", "tc", "tc2", "tc2single"])
 def test_fused_bf16_small(api, shape, variant):
     B, H, Nq, Nk, d = shape
+    if variant == 4 and d != 64:
+        pytest.skip("single-tile TC2 CTAs exist for d = 64 only")
     rng = np.random.default_rng(abs(hash(shape)) % (2 ** 31))
     Qb, Kb, Vb = rand_bits(rng, (B, H, Nq, d)), rand_bits(rng, (B, H, Nk, d)), rand_bits(rng, (B, H, Nk, d))
     scale = 1 / math.sqrt(d)
@@ -53,9 +55,11 @@ def test_fused_bf16_small(api, shape, variant):
     check_bf16(got, ref, "fused bf16 %s v%d" % (shape, variant))
 
 
-@pytest.mark.parametrize("variant", [1, 2, 3], ids=["simt", "tc", "tc2"])
+@pytest.mark.parametrize("variant", [1, 2, 3, 4], ids=["simt", "tc", "tc2", "tc2single"])
 @pytest.mark.parametrize("d", [64, 128])
 def test_fused_bf16_masked(api, variant, d):
+    if variant == 4 and d != 64:
+        pytest.skip("single-tile TC2 CTAs exist for d = 64 only")
     B, H, Nq, Nk = 5, 2, 200, 600
     rng = np.random.default_rng(77 + d)
     Qb, Kb, Vb = rand_bits(rng, (B, H, Nq, d)), rand_bits(rng, (B, H, Nk, d)), rand_bits(rng, (B, H, Nk, d))
@@ -73,7 +77,7 @@ def test_fused_bf16_masked(api, variant, d):
     assert np.all(got[4] == 0.0)                            # no valid key: O = 0
 
 
-@pytest.mark.parametrize("variant", [1, 2, 3], ids=["simt", "tc", "tc2"])
+@pytest.mark.parametrize("variant", [1, 2, 3, 4], ids=["simt", "tc", "tc2", "tc2single"])
 def test_fused_bf16_planted_keys(api, variant):
     """Peaked softmax on a planted key with position-coded V: a dropped, duplicated, shifted or
     mis-masked key tile moves O by O(1)."""
@@ -96,7 +100,7 @@ def test_fused_bf16_scales_tc(api, scale):
     rng = np.random.default_rng(5)
     Qb, Kb, Vb = rand_bits(rng, (B, H, Nq, d)), rand_bits(rng, (B, H, Nk, d)), rand_bits(rng, (B, H, Nk, d))
     ref = oracle.attention(Qb, Kb, Vb, scale)["O"]
-    for variant in (2, 3):
+    for variant in (2, 3, 4):
         got = run_fused_bf16(api, Qb, Kb, Vb, scale, variant=variant)
         check_bf16(got, ref, "scale %g v%d" % (scale, variant))
 
@@ -113,7 +117,7 @@ def test_rising_maximum_forces_rescale(api):
     ref = oracle.attention(Qb, Kb, Vb, 1.0, want_logits=True)
     L = ref["L"].reshape(Nq, Nk)
     assert np.all(L[:, -128:].max(1) - L[:, :128].max(1) > 20)      # > 8 log2 units per several tiles
-    for variant in (1, 2, 3):
+    for variant in (1, 2, 3, 4):
         got = run_fused_bf16(api, Qb, Kb, Vb, 1.0, variant=variant)
         check_bf16(got, ref["O"], "rising max v%d" % variant)
 
