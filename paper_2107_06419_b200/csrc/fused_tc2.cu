@@ -139,7 +139,7 @@ __device__ __forceinline__ float row_min(const uint32_t (&s)[128]) {
 // p_i = 2^(s_i * scale + neg_m) for one row of 128 logits; stores bf16(p) to 64 TMEM columns at
 // `p_addr` and returns the fp32 sum of the unrounded p.  TAIL: only the first `nvalid` columns
 // take part, the rest get p = 0 (this also removes the NaN of inf * 0 when scale == 0).
-template <bool TAIL, typename BeforeFirstStore, typename AfterLastExp>
+template <bool TAIL, bool POLY, typename BeforeFirstStore, typename AfterLastExp>
 __device__ __forceinline__ float exp_store(const uint32_t (&s)[128], float scale_log2e, float neg_m, uint32_t p_addr,
                                            int nvalid, BeforeFirstStore&& before_first_store,
                                            AfterLastExp&& after_last_exp, volatile unsigned* trace_row = nullptr) {
@@ -160,8 +160,10 @@ __device__ __forceinline__ float exp_store(const uint32_t (&s)[128], float scale
 #pragma unroll
         for (int i = 0; i < 32; ++i) {
             // One element in four takes the polynomial route (FMA pipe) to unload the ex2 unit,
-            // the binding pipe at d = 64; the careful/tail pass keeps to ex2 throughout.
-            p[i] = (!TAIL && (i & 3) == POLY_LANE) ? ex2_poly(p[i]) : ex2_approx(p[i]);
+            // the binding pipe at d = 64; the careful/tail pass keeps to ex2 throughout, and so do
+            // the tiles that take turns (POLY off): a warp running alone is short of issue slots,
+            // not of ex2 throughput.
+            p[i] = (!TAIL && POLY && (i & 3) == POLY_LANE) ? ex2_poly(p[i]) : ex2_approx(p[i]);
             if (TAIL && c * 32 + i >= nvalid) p[i] = 0.f;
         }
         if (c == PASS_AT_CHUNK) after_last_exp();       // (nearly) every ex2 of the row has been issued
@@ -432,10 +434,10 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             float lt = 0.f;
             if (!careful) {
 #ifdef FLAT_TRACE
-                lt = exp_store<false>(s, scale_log2e, -m_ref, tl + LY::P_COL(t), BN, wait_p_free, pass_turn,
+                lt = exp_store<false, !LY::TURNS>(s, scale_log2e, -m_ref, tl + LY::P_COL(t), BN, wait_p_free, pass_turn,
                                       (blockIdx.x == 0 && blockIdx.y == 0 && j < 64) ? trace_buf + (t * 64 + j) * 16 : nullptr);
 #else
-                lt = exp_store<false>(s, scale_log2e, -m_ref, tl + LY::P_COL(t), BN, wait_p_free, pass_turn);
+                lt = exp_store<false, !LY::TURNS>(s, scale_log2e, -m_ref, tl + LY::P_COL(t), BN, wait_p_free, pass_turn);
 #endif
                 if (!ok) break;                           // (a failed wait means the stores went nowhere useful)
                 careful = __any_sync(0xffffffffu, !(lt <= OVERFLOW_SUM));
@@ -464,7 +466,7 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                     }
                     m_ref = m_new;
                 }
-                lt = exp_store<true>(s, scale_log2e, -m_ref, tl + LY::P_COL(t), tail ? n - col0 : BN, wait_p_free,
+                lt = exp_store<true, false>(s, scale_log2e, -m_ref, tl + LY::P_COL(t), tail ? n - col0 : BN, wait_p_free,
                                      pass_turn);
                 if (!ok) break;
             }
