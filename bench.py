@@ -45,8 +45,9 @@ def load_peaks():
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel, copied from
 # the ncu capture summarised in profiles/fused_tc2_kernel_dram_and_pipes.md (None where nothing was captured).
 MEASURED_DRAM_TRAFFIC = {
-    ("fused_tc2_kernel", "c2_bert_large_4k"): 514_700_000,
-    ("fused_tc2_kernel", "p_4k_small"): 117_000_000,
+    ("fused_tc2_kernel", "c2_bert_large_4k"): 516_000_000,
+    ("fused_tc2_kernel", "p_4k_small"): 117_600_000,
+    ("fused_tc2_kernel", "p_16k_d128_small"): 51_900_000,
 }
 
 
