@@ -26,6 +26,10 @@ int launch_naive(const Problem& p, void* L, void* A, cudaStream_t st);
 int launch_fused_tc(const Problem& p, cudaStream_t st);
 int launch_fused_tc2(const Problem& p, cudaStream_t st);
 int launch_fused_tc2_single(const Problem& p, cudaStream_t st);
+// Tensor-core versions of the baseline's two contractions (bf16, d in {64,128}, Nk % 8 == 0).
+bool naive_tc_applies(const Problem& p);
+int launch_naive_logit_tc(const Problem& p, float* L, cudaStream_t st);
+int launch_naive_attend_tc(const Problem& p, const void* A, cudaStream_t st);
 
 // Raises the dynamic shared-memory limit of `Kernel` once per device (the attribute is sticky,
 // and setting it on every call costs microseconds that small problems notice).

@@ -357,6 +357,16 @@ int launch_fused_simt(const Problem& p, cudaStream_t st) {
 
 int launch_naive(const Problem& p, void* L, void* A, cudaStream_t st) {
     float* Lf = static_cast<float*>(L);
+    if (naive_tc_applies(p)) {
+        // contractions on the tensor cores, row softmax between them as below
+        int rc = launch_naive_logit_tc(p, Lf, st);
+        if (rc != FLAT_OK) return rc;
+        const int64_t rows = static_cast<int64_t>(p.B) * p.H * p.Nq;
+        naive_softmax_kernel<__nv_bfloat16><<<static_cast<unsigned>(rows), NTHREADS, 0, st>>>(
+            Lf, static_cast<__nv_bfloat16*>(A), p.H, p.Nq, p.Nk, p.k_valid_len);
+        if (cudaGetLastError() != cudaSuccess) return FLAT_ERR_CUDA;
+        return launch_naive_attend_tc(p, A, st);
+    }
     if (p.dtype == FLAT_DTYPE_BF16) {
         switch (p.d) {
             case 16: return launch_naive_td<__nv_bfloat16, __nv_bfloat16, 16>(p, Lf, A, st);

@@ -139,12 +139,14 @@ def test_fused_f32(api, shape):
     check_f32(O.cpu().numpy().astype(np.float64), ref, "fused f32 %s" % (shape,))
 
 
+@pytest.mark.parametrize("Nk", [333, 336, 1024], ids=["ffma", "tc-ragged", "tc"])
 @pytest.mark.parametrize("d", [64, 128])
-def test_naive_bf16(api, d):
-    B, H, Nq, Nk = 2, 2, 200, 333
+def test_naive_bf16(api, d, Nk):
+    """Nk % 8 == 0 takes the tensor-core contractions, otherwise the FFMA kernels."""
+    B, H, Nq = 2, 2, 200
     rng = np.random.default_rng(13 + d)
     Qb, Kb, Vb = rand_bits(rng, (B, H, Nq, d)), rand_bits(rng, (B, H, Nk, d)), rand_bits(rng, (B, H, Nk, d))
-    vl = np.array([333, 130], dtype=np.int32)
+    vl = np.array([Nk, 130], dtype=np.int32)
     scale = 1 / math.sqrt(d)
     ref = oracle.attention(Qb, Kb, Vb, scale, valid_len=vl, want_logits=True, want_weights=True)
     Q, K, V = bf16_tensor(Qb), bf16_tensor(Kb), bf16_tensor(Vb)
