@@ -162,6 +162,16 @@ size_t flat_attn_host_workspace_bytes(int B, int H, int Nq, int Nk, int d, int d
 int flat_attn_naive_fwd_static(const void* Q, const void* K, const void* V, void* O,
                                int B, int H, int Nq, int Nk, int d, float scale, void* stream);
 
+/*
+ * Self-test of the device-side give-up path (the paper has no counterpart).  Every wait inside the
+ * tensor-core kernels is bounded; when one runs out, the kernel stores a non-zero code in the
+ * caller's `status` word and returns normally.  This call launches a one-warp kernel that waits,
+ * for about 0.1 s, on a barrier nothing completes, and must leave FLAT_SELFTEST_TIMEOUT_CODE in
+ * *status (a device int32, zeroed by the caller) with the context still usable afterwards.
+ */
+#define FLAT_SELFTEST_TIMEOUT_CODE 0x7e57
+int flat_attn_selftest_wait_timeout(int32_t* status, void* stream);
+
 /* Number of kernels the most recent successful call on this thread launched. */
 int flat_attn_last_launch_count(void);
 

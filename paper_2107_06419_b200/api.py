@@ -26,7 +26,7 @@ FLAT_DTYPE_BF16, FLAT_DTYPE_F32 = 0, 1
 FLAT_VARIANT_AUTO, FLAT_VARIANT_SIMT, FLAT_VARIANT_TC, FLAT_VARIANT_TC2, FLAT_VARIANT_TC2_SINGLE = 0, 1, 2, 3, 4
 
 EXPORTS = ["flat_attn_fwd", "flat_attn_fwd_ex", "flat_attn_naive_fwd", "flat_attn_naive_fwd_ex",
-           "flat_attn_naive_fwd_static",
+           "flat_attn_naive_fwd_static", "flat_attn_selftest_wait_timeout",
            "flat_attn_fwd_host", "flat_attn_host_workspace_bytes", "flat_attn_last_launch_count",
            "flat_attn_status_string", "flat_attn_version"]
 
@@ -49,6 +49,8 @@ _lib.flat_attn_naive_fwd_ex.argtypes = [ctypes.POINTER(flat_attn_params_t), _vp,
 _lib.flat_attn_naive_fwd_ex.restype = _i
 _lib.flat_attn_naive_fwd_static.argtypes = [_vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _f, _vp]
 _lib.flat_attn_naive_fwd_static.restype = _i
+_lib.flat_attn_selftest_wait_timeout.argtypes = [_vp, _vp]
+_lib.flat_attn_selftest_wait_timeout.restype = _i
 _lib.flat_attn_fwd_host.argtypes = [ctypes.POINTER(flat_attn_params_t), _vp, ctypes.c_size_t, _vp]
 _lib.flat_attn_fwd_host.restype = _i
 _lib.flat_attn_host_workspace_bytes.argtypes = [_i, _i, _i, _i, _i, _i]
@@ -171,6 +173,16 @@ def flat_attn_naive_fwd_static(Q, K, V, O, scale, stream=None):
     _check(_lib.flat_attn_naive_fwd_static(p.Q, p.K, p.V, p.O, p.B, p.H, p.Nq, p.Nk, p.d, p.scale,
                                            _stream_ptr(stream)))
     return O
+
+
+FLAT_SELFTEST_TIMEOUT_CODE = 0x7E57
+
+
+def flat_attn_selftest_wait_timeout(status, stream=None):
+    """Runs the bounded-wait self-test; `status` is a zeroed CUDA int32 tensor of one element."""
+    if not status.is_cuda or status.dtype != torch.int32:
+        raise ValueError("status must be a CUDA int32 tensor")
+    _check(_lib.flat_attn_selftest_wait_timeout(_ptr(status), _stream_ptr(stream)))
 
 
 def _check_la(p, L, A):

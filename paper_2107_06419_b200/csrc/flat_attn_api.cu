@@ -210,6 +210,14 @@ int flat_attn_fwd_host(const flat_attn_params_t* p, void* workspace, size_t work
     return FLAT_OK;
 }
 
+int flat_attn_selftest_wait_timeout(int32_t* status, void* stream) {
+    if (!status) return FLAT_ERR_NULL;
+    if (reinterpret_cast<uintptr_t>(status) & 3u) return FLAT_ERR_ALIGN;
+    const int r = flat::launch_wait_timeout_selftest(status, static_cast<cudaStream_t>(stream));
+    if (r == FLAT_OK) g_last_launches = 1;
+    return r;
+}
+
 int flat_attn_last_launch_count(void) { return g_last_launches; }
 
 const char* flat_attn_status_string(int code) {

@@ -541,7 +541,24 @@ int launch_tc2_d(const Problem& p, cudaStream_t st) {
     return cudaGetLastError() == cudaSuccess ? FLAT_OK : FLAT_ERR_CUDA;
 }
 
+// Self-test of the give-up path: one warp waits on a barrier that nothing will ever complete, with
+// a limit of about a tenth of a second.  The wait must run out, record its code and let the kernel
+// end normally (no trap, no hang), leaving the context usable.
+__global__ void wait_timeout_selftest_kernel(int32_t* status) {
+    __shared__ uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) { mbar_init(&bar, 1); abort_flag = 0; fence_mbar_init(); }
+    __syncthreads();
+    const bool ok = bounded_wait(&bar, 0, &abort_flag, status, 0x7e57, 200000000ll);
+    if (ok && threadIdx.x == 0 && status) atomicExch(status, -1);   // would mean the wait "succeeded"
+}
+
 }  // namespace
+
+int launch_wait_timeout_selftest(int32_t* status, cudaStream_t st) {
+    wait_timeout_selftest_kernel<<<1, 32, 0, st>>>(status);
+    return cudaGetLastError() == cudaSuccess ? FLAT_OK : FLAT_ERR_CUDA;
+}
 
 int launch_fused_tc2(const Problem& p, cudaStream_t st) {
     if (p.dtype != FLAT_DTYPE_BF16) return FLAT_ERR_UNSUPPORTED;

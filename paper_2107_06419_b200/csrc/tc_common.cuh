@@ -18,7 +18,7 @@ constexpr float RESCALE_THRESHOLD = 8.0f;         // log2 units: P stays <= 2^8
 // raised the abort flag or after WAIT_CYCLES; the first thread to time out raises the flag and
 // records `code` in *status.  Never traps, never spins without limit.
 __device__ __forceinline__ bool bounded_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
-                                             int32_t* status, int code) {
+                                             int32_t* status, int code, long long limit = WAIT_CYCLES) {
     if (ptx::mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     for (;;) {
@@ -28,7 +28,7 @@ __device__ __forceinline__ bool bounded_wait(uint64_t* bar, uint32_t parity, vol
         for (int i = 0; i < 32; ++i)
             if (ptx::mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
-        if (clock64() - t0 > WAIT_CYCLES) {
+        if (clock64() - t0 > limit) {
             *abort_flag = 1;
             if (status) atomicExch(status, code);
             return false;

@@ -216,3 +216,16 @@ def test_output_padding_untouched(api):
         torch.cuda.synchronize()
         assert torch.all(buf[:1024] == 7.0) and torch.all(buf[1024 + n:] == 7.0)
         check_bf16(bf16_to_f64(O), oracle.attention(Qb, Kb, Vb, 0.125)["O"], "canary v%d" % variant)
+
+
+def test_bounded_wait_gives_up_cleanly(api):
+    """A wait that nothing satisfies runs out, reports its code and leaves the GPU usable."""
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    api.flat_attn_selftest_wait_timeout(status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == api.FLAT_SELFTEST_TIMEOUT_CODE
+    # the context is still healthy: a normal call right after gives the right answer
+    rng = np.random.default_rng(99)
+    Qb, Kb, Vb = rand_bits(rng, (1, 1, 128, 64)), rand_bits(rng, (1, 1, 256, 64)), rand_bits(rng, (1, 1, 256, 64))
+    got = run_fused_bf16(api, Qb, Kb, Vb, 0.125, variant=3)
+    check_bf16(got, oracle.attention(Qb, Kb, Vb, 0.125)["O"], "after timeout self-test")
