@@ -1,25 +1,28 @@
-// Fused Logit-Softmax-Attend, pipelined: two 128-row query tiles per CTA ping-pong on the tensor
-// pipe so that the softmax of one tile overlaps the MMAs of the other (bf16 in, fp32 accumulate).
+// Fused Logit-Softmax-Attend, pipelined (bf16 in, fp32 accumulate, bf16 out): NT = 2 query tiles
+// of 128 rows per CTA share the tensor pipe, the K/V stream and the SM's exponent unit (NT = 1: one
+// tile per CTA, two CTAs per SM, for problems too small to fill the SMs with 256-row CTAs).
 //
 // Paper mapping (Section 5, 5.1, 5.2): shared outer loops = (batch, head) on blockIdx.y and a
-// 256-row slab of query rows on blockIdx.x (R-granularity, Rx = 2 x 128); inner loops Logit and
-// Attend run interleaved over 128-key tiles with the streaming softmax between them (the running
-// maximum / sum replaces the paper's full-row on-chip slice; same function).
+// slab of NT x 128 query rows on blockIdx.x (R-granularity); inner loops Logit and Attend run
+// interleaved over 128-key tiles with the streaming softmax between them (a reference maximum and
+// a running sum replace the paper's full-row on-chip slice; same function).
 //
-// CTA = 384 threads (three warpgroups; registers are moved from the third to the first two):
+// CTA (NT = 2) = 384 threads, three warpgroups; registers are moved from the third to the first two:
 //   warps 0-3  softmax of query tile A   (thread r <-> row r of the tile <-> TMEM lane r)
 //   warps 4-7  softmax of query tile B
 //   warp  8    TMA producer (one lane): Q tiles once, then K and V tiles into separate rings
 //   warp  9    MMA issuer of tile A (one elected lane): S_A = Q_A K^T and O_A += P_A V
 //   warp  10   MMA issuer of tile B
 //   warp  11   idle (it only completes the warpgroup for the register hand-over)
-// A softmax thread pulls its 128 logits into registers, releases the S buffer at once (so the next
-// S_t is computed while it works), takes the row maximum, writes bf16 weights P_t to TMEM and adds
-// to its row sum.  O_t is rescaled in TMEM only when a row maximum exceeds the reference by 2^8.
+// A softmax thread pulls its 128 logits into registers and releases the S buffer at once (so the
+// next S_t is computed while it works), computes p = 2^(scale*log2e*s - m_ref) with the reference
+// maximum it already has -- no row maximum per tile: a tile whose row sum overflows 2^40 is redone
+// with an exact maximum, and O_t, l are rescaled -- writes bf16 weights P_t to TMEM and adds to its
+// row sum.  One exponential in four goes through a polynomial on the FMA pipe (d = 64).
 //
-// TMEM columns (512): S_A 0, S_B 128, O_A 256, O_B 256+d, and for d = 64 P_A 384, P_B 448; at
+// TMEM columns (NT = 2): S_A 0, S_B 128, O_A 256, O_B 256+d, and for d = 64 P_A 384, P_B 448; at
 // d = 128 TMEM is full and P_t overlays the first 64 columns of S_t, so S_t(j+1) is issued behind
-// O_t += P_t(j) V_j instead of ahead of it.
+// O_t += P_t(j) V_j instead of ahead of it, and the two tiles take strict turns at the exponentials.
 // Every wait is bounded (see tc_common.cuh); on expiry the CTA aborts cleanly and reports a code.
 #include <cuda.h>
 #include <cuda_bf16.h>
@@ -302,11 +305,7 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             const uint32_t s_tmem = tmem + LY::S_COL(t), o_tmem = tmem + LY::O_COL(t), p_tmem = tmem + LY::P_COL(t);
             bool ok = true;
             auto wait = [&](int bar, uint32_t parity, int code) {
-#ifdef FLAT_MMA_SPIN
-                if (ok) ok = __all_sync(0xffffffffu, bounded_spin_wait(&bars[bar], parity, abort_flag, status, code));
-#else
                 if (ok) ok = __all_sync(0xffffffffu, bounded_wait(&bars[bar], parity, abort_flag, status, code));
-#endif
                 if (ok) tc_fence_after();
             };
             auto issue_s = [&](int j) {                  // S_t = Q_t K_j^T, then release the K stage

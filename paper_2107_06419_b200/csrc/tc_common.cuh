@@ -36,25 +36,6 @@ __device__ __forceinline__ bool bounded_wait(uint64_t* bar, uint32_t parity, vol
     }
 }
 
-// Same contract, but probes without parking the thread: lower wake-up latency, for a warp whose
-// only job is to react to the barrier (the MMA issuers).
-__device__ __forceinline__ bool bounded_spin_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
-                                                  int32_t* status, int code) {
-    if (ptx::mbar_test_wait(bar, parity)) return true;
-    const long long t0 = clock64();
-    for (;;) {
-#pragma unroll 1
-        for (int i = 0; i < 64; ++i)
-            if (ptx::mbar_test_wait(bar, parity)) return true;
-        if (*abort_flag) return false;
-        if (clock64() - t0 > WAIT_CYCLES) {
-            *abort_flag = 1;
-            if (status) atomicExch(status, code);
-            return false;
-        }
-    }
-}
-
 // Teardown helper: wait for a copy this thread started, with a time limit and no side effects.
 __device__ __forceinline__ void drain_wait(uint64_t* bar, uint32_t parity) {
     const long long t0 = clock64();
