@@ -229,3 +229,40 @@ def test_bounded_wait_gives_up_cleanly(api):
     Qb, Kb, Vb = rand_bits(rng, (1, 1, 128, 64)), rand_bits(rng, (1, 1, 256, 64)), rand_bits(rng, (1, 1, 256, 64))
     got = run_fused_bf16(api, Qb, Kb, Vb, 0.125, variant=3)
     check_bf16(got, oracle.attention(Qb, Kb, Vb, 0.125)["O"], "after timeout self-test")
+
+
+@pytest.mark.parametrize("sigma,scale", [(3.0, 1.0), (1.0, 20.0), (6.0, 0.5)])
+def test_wide_dynamic_range(api, sigma, scale):
+    """Logits with a standard deviation of dozens to hundreds: row maxima jump by far more than the
+    exponent range between tiles, so the stale-reference check, the rescale of O and the clamps of
+    the polynomial exponential all fire; softmax rows are nearly one-hot."""
+    B, H, Nq, Nk, d = 1, 2, 256, 1536, 64
+    rng = np.random.default_rng(int(sigma * 10 + scale))
+    Qb, Kb = rand_bits(rng, (B, H, Nq, d), sigma), rand_bits(rng, (B, H, Nk, d), sigma)
+    Vb = rand_bits(rng, (B, H, Nk, d))
+    ref = oracle.attention(Qb, Kb, Vb, scale, want_logits=True)
+    spread = ref["L"].max(-1) - np.median(ref["L"], -1)
+    assert np.median(spread) > 100                                  # far beyond 2^126 in base-2 terms
+    for variant in (1, 2, 3, 4):
+        got = run_fused_bf16(api, Qb, Kb, Vb, scale, variant=variant)
+        check_bf16(got, ref["O"], "wide range sigma=%g scale=%g v%d" % (sigma, scale, variant))
+
+
+def test_spike_on_polynomial_lane(api):
+    """One key far above all others (hundreds of log2 units), sitting in a later tile on a column
+    that the kernel evaluates with the polynomial exponential and not with the ex2 unit: the clamp
+    must turn it into an overflow that forces the careful pass, not into garbage."""
+    B, H, Nq, Nk, d = 1, 1, 256, 1280, 64
+    rng = np.random.default_rng(4242)
+    u = np.ones(d, dtype=np.float32)
+    Qf = (u[None, :] * (1.0 + rng.random((Nq, 1), dtype=np.float32)) + 0.1 * rng.standard_normal((Nq, d))).astype(np.float32)
+    Kf = (0.01 * rng.standard_normal((Nk, d))).astype(np.float32)
+    Kf[131] = 2.0 * u           # tile 1, column 3
+    Kf[1027] = 6.0 * u          # tile 8, column 3: 4 * 64 * (1..2) = 256..512 above the first spike
+    Vf = rng.standard_normal((Nk, d)).astype(np.float32)
+    Qb, Kb, Vb = (inputs.f32_to_bf16_bits(x).reshape(1, 1, *x.shape) for x in (Qf, Kf, Vf))
+    ref = oracle.attention(Qb, Kb, Vb, 1.0, want_weights=True)
+    assert np.all(ref["A"][0, 0].argmax(-1) == 1027)
+    for variant in (2, 3, 4):
+        got = run_fused_bf16(api, Qb, Kb, Vb, 1.0, variant=variant)
+        check_bf16(got, ref["O"], "spike v%d" % variant)
