@@ -172,6 +172,13 @@ int flat_attn_naive_fwd_static(const void* Q, const void* K, const void* V, void
 #define FLAT_SELFTEST_TIMEOUT_CODE 0x7e57
 int flat_attn_selftest_wait_timeout(int32_t* status, void* stream);
 
+/*
+ * Self-test of the polynomial 2^x that the fused kernel uses for a quarter of its exponentials
+ * (the paper has no counterpart): y[i] = 2^clamp(x[i], -126, 126) evaluated by that routine, for
+ * n device floats.  Relative error <= 1e-4 inside the clamp range.
+ */
+int flat_attn_selftest_exp2_poly(const float* x, float* y, int n, void* stream);
+
 /* Number of kernels the most recent successful call on this thread launched. */
 int flat_attn_last_launch_count(void);
 

@@ -26,7 +26,7 @@ FLAT_DTYPE_BF16, FLAT_DTYPE_F32 = 0, 1
 FLAT_VARIANT_AUTO, FLAT_VARIANT_SIMT, FLAT_VARIANT_TC, FLAT_VARIANT_TC2, FLAT_VARIANT_TC2_SINGLE = 0, 1, 2, 3, 4
 
 EXPORTS = ["flat_attn_fwd", "flat_attn_fwd_ex", "flat_attn_naive_fwd", "flat_attn_naive_fwd_ex",
-           "flat_attn_naive_fwd_static", "flat_attn_selftest_wait_timeout",
+           "flat_attn_naive_fwd_static", "flat_attn_selftest_wait_timeout", "flat_attn_selftest_exp2_poly",
            "flat_attn_fwd_host", "flat_attn_host_workspace_bytes", "flat_attn_last_launch_count",
            "flat_attn_status_string", "flat_attn_version"]
 
@@ -49,6 +49,8 @@ _lib.flat_attn_naive_fwd_ex.argtypes = [ctypes.POINTER(flat_attn_params_t), _vp,
 _lib.flat_attn_naive_fwd_ex.restype = _i
 _lib.flat_attn_naive_fwd_static.argtypes = [_vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _f, _vp]
 _lib.flat_attn_naive_fwd_static.restype = _i
+_lib.flat_attn_selftest_exp2_poly.argtypes = [_vp, _vp, _i, _vp]
+_lib.flat_attn_selftest_exp2_poly.restype = _i
 _lib.flat_attn_selftest_wait_timeout.argtypes = [_vp, _vp]
 _lib.flat_attn_selftest_wait_timeout.restype = _i
 _lib.flat_attn_fwd_host.argtypes = [ctypes.POINTER(flat_attn_params_t), _vp, ctypes.c_size_t, _vp]
@@ -176,6 +178,16 @@ def flat_attn_naive_fwd_static(Q, K, V, O, scale, stream=None):
 
 
 FLAT_SELFTEST_TIMEOUT_CODE = 0x7E57
+
+
+def flat_attn_selftest_exp2_poly(x, y, stream=None):
+    """y = the kernel's polynomial 2^x of the CUDA float32 tensor x (same shape, contiguous)."""
+    if not (x.is_cuda and y.is_cuda and x.dtype == torch.float32 and y.dtype == torch.float32):
+        raise ValueError("x and y must be CUDA float32 tensors")
+    if x.numel() != y.numel() or not x.is_contiguous() or not y.is_contiguous():
+        raise ValueError("x and y must be contiguous and of equal size")
+    _check(_lib.flat_attn_selftest_exp2_poly(_ptr(x), _ptr(y), x.numel(), _stream_ptr(stream)))
+    return y
 
 
 def flat_attn_selftest_wait_timeout(status, stream=None):

@@ -210,6 +210,14 @@ int flat_attn_fwd_host(const flat_attn_params_t* p, void* workspace, size_t work
     return FLAT_OK;
 }
 
+int flat_attn_selftest_exp2_poly(const float* x, float* y, int n, void* stream) {
+    if (!x || !y) return FLAT_ERR_NULL;
+    if (n < 1) return FLAT_ERR_SHAPE;
+    const int r = flat::launch_exp2_poly_selftest(x, y, n, static_cast<cudaStream_t>(stream));
+    if (r == FLAT_OK) g_last_launches = 1;
+    return r;
+}
+
 int flat_attn_selftest_wait_timeout(int32_t* status, void* stream) {
     if (!status) return FLAT_ERR_NULL;
     if (reinterpret_cast<uintptr_t>(status) & 3u) return FLAT_ERR_ALIGN;

@@ -552,7 +552,18 @@ __global__ void wait_timeout_selftest_kernel(int32_t* status) {
     if (ok && threadIdx.x == 0 && status) atomicExch(status, -1);   // would mean the wait "succeeded"
 }
 
+// Self-test of the polynomial exponential: y[i] = ex2_poly(x[i]).
+__global__ void exp2_poly_selftest_kernel(const float* __restrict__ x, float* __restrict__ y, int n) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) y[i] = ex2_poly(x[i]);
+}
+
 }  // namespace
+
+int launch_exp2_poly_selftest(const float* x, float* y, int n, cudaStream_t st) {
+    exp2_poly_selftest_kernel<<<(n + 255) / 256, 256, 0, st>>>(x, y, n);
+    return cudaGetLastError() == cudaSuccess ? FLAT_OK : FLAT_ERR_CUDA;
+}
 
 int launch_wait_timeout_selftest(int32_t* status, cudaStream_t st) {
     wait_timeout_selftest_kernel<<<1, 32, 0, st>>>(status);

@@ -52,11 +52,12 @@ __device__ __forceinline__ float ex2_approx(float x) {
 // 2^x on the FMA and integer pipes instead of the ex2 unit: x = r + f with r = round(x) and
 // f in [-0.5, 0.5]; 2^f by a cubic (max relative error 7.7e-5, far below the bf16 rounding that
 // the weights undergo next) and 2^r by adding r to the exponent field.  x is clamped to
-// [-127, 126] so that the exponent arithmetic cannot wrap: below, the result is ~2^-127 (as good
-// as 0 next to a row maximum of order 1); above, it is 2^126, which trips the caller's overflow
-// check exactly like the ex2 unit's +inf would.
+// [-126, 126] so that the exponent arithmetic cannot wrap (the cubic lies in [0.70, 1.42], biased
+// exponent 126 or 127, so r >= -126 keeps the field at 0 or above): below, the result is a
+// denormal of about 2^-126 (as good as 0 next to a row maximum of order 1); above, it is 2^126,
+// which trips the caller's overflow check exactly like the ex2 unit's +inf would.
 __device__ __forceinline__ float ex2_poly(float x) {
-    x = fminf(fmaxf(x, -127.f), 126.f);
+    x = fminf(fmaxf(x, -126.f), 126.f);
     const float t = x + 12582912.f;                    // 1.5 * 2^23: the low mantissa bits now hold round(x)
     const float r = t - 12582912.f;
     const float f = x - r;

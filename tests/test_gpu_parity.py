@@ -266,3 +266,17 @@ def test_spike_on_polynomial_lane(api):
     for variant in (2, 3, 4):
         got = run_fused_bf16(api, Qb, Kb, Vb, 1.0, variant=variant)
         check_bf16(got, ref["O"], "spike v%d" % variant)
+
+
+def test_polynomial_exp2_accuracy_and_clamps(api):
+    x = np.concatenate([np.linspace(-126.0, 126.0, 200001), np.linspace(-1.0, 1.0, 50001),
+                        np.arange(-126, 127, dtype=np.float64) + 0.5, np.arange(-126, 127, dtype=np.float64),
+                        [-1e30, -500.0, -127.0, -126.5, 126.5, 127.0, 500.0, 1e30]]).astype(np.float32)
+    xt = torch.from_numpy(x).cuda()
+    y = api.flat_attn_selftest_exp2_poly(xt, torch.empty_like(xt)).cpu().numpy().astype(np.float64)
+    ref = np.exp2(np.clip(x.astype(np.float64), -126.0, 126.0))
+    assert np.all(np.isfinite(y)) and np.all(y > 0)
+    normal = ref >= 2.0 ** -125
+    assert np.max(np.abs(y[normal] / ref[normal] - 1.0)) < 1e-4
+    assert np.all(y[~normal] < 2.0 ** -124)                # the bottom of the range may come out denormal
+    assert y[-1] >= 2.0 ** 125 and y[-2] >= 2.0 ** 125     # far above the range: a huge finite value
