@@ -196,7 +196,9 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                  const __grid_constant__ CUtensorMap tmV, __nv_bfloat16* __restrict__ O, int H, int Nq, int Nk,
                  float scale_log2e, const int32_t* __restrict__ valid_len, int32_t* status) {
     using LY = L2<D, NT>;
+#ifdef FLAT_TRACE
     constexpr int THREADS = LY::THREADS;
+#endif
     extern __shared__ uint8_t smem_raw[];
     uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* Qs = base;                                  // NT tiles
