@@ -1,0 +1,82 @@
+"""Granularity sweep: times every fused kernel variant on a set of shapes (CUDA events).
+
+The paper explores, per workload, how many query rows a fused tile should hold (its R-granularity
+trade-off, Section 5.3: fewer rows mean more K/V re-fetches and a worse-filled compute array) and
+picks the best mapping by search (Section 6.1).  On B200 the candidates are the compiled kernel
+variants: 64-row FFMA tiles, 128-row tensor-core CTAs (one or two per SM) and 256-row CTAs.
+
+    python -m paper_2107_06419_b200.tune [--workloads c1_bert_base_512,c2_bert_large_4k,...] [--steps 10]
+
+Prints one JSON line per (workload, variant) and the winner per workload; inputs are random bf16
+(timing only -- parity is the tests' business).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+
+import torch
+
+from . import api, inputs
+
+VARIANTS = {
+    api.FLAT_VARIANT_SIMT: "simt: 64-row FFMA tiles",
+    api.FLAT_VARIANT_TC: "tc: 128-row CTA, exact running maximum",
+    api.FLAT_VARIANT_TC2_SINGLE: "tc2_single: 128-row CTA, two per SM (d = 64)",
+    api.FLAT_VARIANT_TC2: "tc2: 256-row CTA (two tiles ping-pong)",
+    api.FLAT_VARIANT_AUTO: "auto (the dispatcher's choice)",
+}
+
+
+def time_variant(w, variant, steps, warmup=2):
+    dev = torch.device("cuda")
+    Q = torch.randn(w.B, w.H, w.Nq, w.d, device=dev, dtype=torch.bfloat16)
+    K = torch.randn(w.B, w.H, w.Nk, w.d, device=dev, dtype=torch.bfloat16)
+    V = torch.randn_like(K)
+    O = torch.empty_like(Q)
+    vl = None
+    if w.masked:
+        vl = torch.from_numpy(inputs.make_valid_len(w)).to(dev)
+    try:
+        for _ in range(warmup):
+            api.flat_attn_fwd_ex(Q, K, V, O, w.scale, k_valid_len=vl, variant=variant)
+    except api.FlatAttnError as e:
+        return None, str(e)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(steps):
+        api.flat_attn_fwd_ex(Q, K, V, O, w.scale, k_valid_len=vl, variant=variant)
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / steps, None
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--workloads", default="c1_bert_base_512,c2_bert_large_4k,c3_16k,c4_64k_d128,c5_cross_masked")
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--skip-simt-above", type=float, default=2e12,
+                    help="skip the FFMA variant for workloads above this many FLOP (it takes long)")
+    args = ap.parse_args()
+    for name in args.workloads.split(","):
+        w = inputs.WORKLOADS[name]
+        best = None
+        for variant, label in VARIANTS.items():
+            if variant == api.FLAT_VARIANT_SIMT and w.flops > args.skip_simt_above:
+                continue
+            ms, err = time_variant(w, variant, args.steps if variant != api.FLAT_VARIANT_SIMT else 2)
+            row = {"workload": name, "variant": variant, "kernel": label}
+            if ms is None:
+                row["unsupported"] = err
+            else:
+                row.update(ms=round(ms, 4), tflops=round(w.flops / ms / 1e9, 1))
+                if variant != api.FLAT_VARIANT_AUTO and (best is None or ms < best[0]):
+                    best = (ms, variant)
+            print(json.dumps(row), flush=True)
+        if best:
+            print(json.dumps({"workload": name, "best_variant": best[1], "ms": round(best[0], 4)}), flush=True)
+
+
+if __name__ == "__main__":
+    main()
