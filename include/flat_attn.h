@@ -66,8 +66,11 @@ enum {
                                   bf16, d in {64,128}                                          */
     FLAT_VARIANT_TC2 = 3,      /* same, two 128-row tiles per CTA ping-ponging on the tensor
                                   pipe (the default for problems that fill the GPU)            */
-    FLAT_VARIANT_TC2_SINGLE = 4 /* the TC2 pipeline with one 128-row tile per CTA and two CTAs
+    FLAT_VARIANT_TC2_SINGLE = 4, /* the TC2 pipeline with one 128-row tile per CTA and two CTAs
                                   per SM: bf16, d = 64 only                                    */
+    FLAT_VARIANT_TC3 = 5       /* two tiles per CTA, the softmax of every row split over two
+                                  threads (sixteen softmax warps), logit tiles computed three
+                                  tile-steps ahead in rotating TMEM buffers: bf16, d = 64 only */
 };
 
 typedef struct flat_attn_params {

@@ -26,6 +26,7 @@ int launch_naive(const Problem& p, void* L, void* A, cudaStream_t st);
 int launch_fused_tc(const Problem& p, cudaStream_t st);
 int launch_fused_tc2(const Problem& p, cudaStream_t st);
 int launch_fused_tc2_single(const Problem& p, cudaStream_t st);
+int launch_fused_tc3(const Problem& p, cudaStream_t st);
 int launch_wait_timeout_selftest(int32_t* status, cudaStream_t st);
 int launch_exp2_poly_selftest(const float* x, float* y, int n, cudaStream_t st);
 // Tensor-core versions of the baseline's two contractions (bf16, d in {64,128}, Nk % 8 == 0).

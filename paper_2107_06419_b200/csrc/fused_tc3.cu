@@ -1,0 +1,534 @@
+// Fused Logit-Softmax-Attend for d = 64 with the softmax of each query tile split over two warps
+// per row group and the logit tiles computed three tile-steps ahead (bf16 in, fp32 accumulate,
+// bf16 out).  Two query tiles of 128 rows per CTA, as in fused_tc2.cu, but
+//   * sixteen softmax warps instead of eight: a thread owns HALF a row of a 128-key step (64
+//     logits, exponentiated in place), so every scheduler of the SM holds four softmax warps whose
+//     waits (barrier, TMEM load, store completion) hide behind the exponentials of the others;
+//   * TMEM holds O_A, O_B (64 columns each) and THREE logit buffers X0..X2 of 128 columns that the
+//     tile-steps u = 0, 1, 2, ... (u even: tile A, u odd: tile B, key step u / 2) use in rotation;
+//     the weights P(u) overlay the logits S(u) they came from, and S(u + 3) is issued as soon as
+//     the MMAs that read P(u) have completed, so the logits of a tile's next step are in TMEM long
+//     before its softmax asks for them.
+//
+// Paper mapping (Section 5, 5.1, 5.2): shared outer loops = (batch, head) on blockIdx.y and a slab
+// of 256 query rows on blockIdx.x (R-granularity); inner loops Logit and Attend interleaved over
+// 128-key tiles, the streaming softmax between them.
+//
+// CTA = 640 threads, five warpgroups; registers move from the fifth to the first four:
+//   warps 0-15  softmax: warp w serves row group q = w % 4 (TMEM lanes 32q..32q+31) of tile
+//               t = w / 8, key half h = (w / 4) % 2 of every step
+//   warp  16    TMA producer (one lane): Q tiles once, then K and V tiles into separate rings
+//   warp  17/18 MMA issuers of O_t += P V for tile A / B (one elected lane each)
+//   warp  19    MMA issuer of every S = Q K^T
+// The two warps that share a row keep the same reference maximum m_ref: the first step fixes it
+// from the exact maximum of both halves (exchanged through shared memory); later steps reuse it and
+// vote, with one reducing named barrier per step, on whether either half's row sum overflowed 2^40,
+// in which case both redo the step with a fresh common maximum (the logits are still in TMEM: the
+// vote comes before the weights are stored over them) and O_t, l are rescaled.
+// Every wait is bounded (see tc_common.cuh); on expiry the CTA aborts cleanly and reports a code.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "flat_internal.cuh"
+#include "ptx_sm100.cuh"
+#include "tc_common.cuh"
+
+namespace flat {
+
+using namespace ptx;
+using namespace tc;
+
+#ifdef FLAT_TRACE3
+// Developer tracing (off in the product build): CTA (0,0) keeps SM-clock stamps in shared memory
+// and copies them to a global buffer when it ends.
+__device__ unsigned* g_trace3 = nullptr;
+extern "C" int flat_debug_set_trace3(unsigned* p) {
+    return cudaMemcpyToSymbol(g_trace3, &p, sizeof(p)) == cudaSuccess ? 0 : 6;
+}
+#define TRACE3_WORDS (6 * 64 * 16)
+#define TRACE(role, iter, point)                                                              \
+    do {                                                                                      \
+        if (blockIdx.x == 0 && blockIdx.y == 0 && (iter) < 64)                                \
+            trace_buf[((role) * 64 + (iter)) * 16 + (point)] = static_cast<unsigned>(clock64()); \
+    } while (0)
+#else
+#define TRACE3_WORDS 0
+#define TRACE(role, iter, point) do { } while (0)
+#endif
+
+namespace {
+
+constexpr int BM = 128;              // rows per query tile (two tiles per CTA)
+constexpr int BN = 128;              // keys per step
+constexpr int HN = 64;               // keys per step and softmax thread
+constexpr float OVERFLOW_SUM = 1.0995116e12f;   // 2^40: a row sum beyond this means m_ref is stale
+// Registers per thread after the hand-over: 640 threads start with 96 each; 512 * 104 + 128 * 64 uses them all.
+#ifndef FLAT_TC3_SOFT_REGS
+#define FLAT_TC3_SOFT_REGS 104
+#define FLAT_TC3_OTHER_REGS 64
+#endif
+#ifndef FLAT_TC3_POLY
+#define FLAT_TC3_POLY true
+#endif
+constexpr int SOFT_REGS = FLAT_TC3_SOFT_REGS, OTHER_REGS = FLAT_TC3_OTHER_REGS;
+static_assert(512 * SOFT_REGS + 128 * OTHER_REGS <= 640 * 96, "register hand-over exceeds the CTA's allocation");
+
+constexpr int D = 64;                // head size of this kernel
+
+struct L3 {
+    static constexpr int KS = 4;                         // K ring depth (S runs 1.5 key steps ahead of P V)
+    static constexpr int VS = 3;                         // V ring depth
+    static constexpr int SOFT_WARPS = 16;
+    static constexpr int THREADS = 32 * SOFT_WARPS + 128;
+    static constexpr uint32_t TMEM_COLS = 512;
+    static constexpr int Q_BYTES = BM * D * 2;           // one query tile
+    static constexpr int KV_BYTES = BN * D * 2;
+    static constexpr int TILE_BYTES = 2 * Q_BYTES + (KS + VS) * KV_BYTES;
+    static constexpr int XCH_BYTES = 2 * 2 * 2 * BM * 4; // [maximum | row sum][tile][half][row] floats
+    static constexpr int SMEM_BYTES = TILE_BYTES + XCH_BYTES + 512 + 1024 + 4 * TRACE3_WORDS;
+    __host__ __device__ static constexpr uint32_t O_COL(int t) { return 64u * t; }
+    __host__ __device__ static constexpr uint32_t X_COL(int b) { return 128u + 128u * b; }   // logit / weight buffer b
+    // barrier indices
+    static constexpr int Q_FULL = 0;                     // [2]
+    static constexpr int K_FULL = 2, K_EMPTY = K_FULL + KS;
+    static constexpr int V_FULL = K_EMPTY + KS, V_EMPTY = V_FULL + VS;
+    // S_FULL / P_FULL / PV_DONE [tile][buffer]: S(u) is in the buffer / P(u) is in the buffer (the 8
+    // softmax warps of the tile arrive) / the MMAs that read P(u) have completed.  Tile u & 1 uses
+    // buffer u % 3 every sixth tile-step, in phase u / 6.  A buffer's next use starts only behind its
+    // PV_DONE, and a tile's softmax warps can be at most two key steps apart, so a waiter never finds
+    // one of these barriers more than one phase ahead of the phase it asks for (parity waits are safe).
+    static constexpr int S_FULL = V_EMPTY + VS, P_FULL = S_FULL + 6, PV_DONE = P_FULL + 6;
+    static constexpr int NUM_BARS = PV_DONE + 6;
+};
+
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+__device__ __forceinline__ float min3(float a, float b, float c) {
+    float d;
+    asm("min.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+__device__ __forceinline__ float half_max(const uint32_t (&s)[HN]) {
+    float e0 = __uint_as_float(s[0]), e1 = __uint_as_float(s[1]), e2 = __uint_as_float(s[2]), e3 = __uint_as_float(s[3]);
+#pragma unroll
+    for (int i = 4; i < 60; i += 8) {
+        e0 = max3(e0, __uint_as_float(s[i]), __uint_as_float(s[i + 1]));
+        e1 = max3(e1, __uint_as_float(s[i + 2]), __uint_as_float(s[i + 3]));
+        e2 = max3(e2, __uint_as_float(s[i + 4]), __uint_as_float(s[i + 5]));
+        e3 = max3(e3, __uint_as_float(s[i + 6]), __uint_as_float(s[i + 7]));
+    }
+    e0 = max3(e0, __uint_as_float(s[60]), __uint_as_float(s[61]));
+    e1 = max3(e1, __uint_as_float(s[62]), __uint_as_float(s[63]));
+    return fmaxf(fmaxf(e0, e1), fmaxf(e2, e3));
+}
+__device__ __forceinline__ float half_min(const uint32_t (&s)[HN]) {
+    float e0 = __uint_as_float(s[0]), e1 = __uint_as_float(s[1]), e2 = __uint_as_float(s[2]), e3 = __uint_as_float(s[3]);
+#pragma unroll
+    for (int i = 4; i < 60; i += 8) {
+        e0 = min3(e0, __uint_as_float(s[i]), __uint_as_float(s[i + 1]));
+        e1 = min3(e1, __uint_as_float(s[i + 2]), __uint_as_float(s[i + 3]));
+        e2 = min3(e2, __uint_as_float(s[i + 4]), __uint_as_float(s[i + 5]));
+        e3 = min3(e3, __uint_as_float(s[i + 6]), __uint_as_float(s[i + 7]));
+    }
+    e0 = min3(e0, __uint_as_float(s[60]), __uint_as_float(s[61]));
+    e1 = min3(e1, __uint_as_float(s[62]), __uint_as_float(s[63]));
+    return fminf(fminf(e0, e1), fminf(e2, e3));
+}
+
+// Named barrier of the two warps (64 threads) that share a row group of a tile.
+__device__ __forceinline__ void pair_sync(int id) {
+    asm volatile("bar.sync %0, 64;" ::"r"(id) : "memory");
+}
+// The same barrier, returning the OR of `flag` over its 64 threads.
+__device__ __forceinline__ bool pair_any(int id, bool flag) {
+    uint32_t r;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.u32 q, %2, 0;\n\t"
+        "bar.red.or.pred p, %1, 64, q;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(r)
+        : "r"(id), "r"(static_cast<uint32_t>(flag))
+        : "memory");
+    return r != 0;
+}
+
+// p_i = 2^(r_i * scale + neg_m) for 32 logits of a row: adds the unrounded p to the four partial
+// sums l[] and packs bf16(p) into pk[].  TAIL: only the first `nvalid` logits take part, the rest
+// get p = 0 (this also removes the NaN of inf * 0 when scale == 0).  All FFMAs come first, then all
+// exponentials, then the sums and the packing, so that consecutive ex2 never wait on a neighbour.
+template <bool TAIL, bool POLY>
+__device__ __forceinline__ void exp_pack32(const uint32_t (&r)[32], float scale_log2e, float neg_m, int nvalid,
+                                           float (&l)[4], uint32_t (&pk)[16]) {
+    float p[32];
+#pragma unroll
+    for (int i = 0; i < 32; ++i) p[i] = fmaf(__uint_as_float(r[i]), scale_log2e, neg_m);
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+        // One element in four takes the polynomial route (FMA pipe) to unload the ex2 unit.
+        p[i] = (!TAIL && POLY && (i & 3) == 3) ? ex2_poly(p[i]) : ex2_approx(p[i]);
+        if (TAIL && i >= nvalid) p[i] = 0.f;
+    }
+#pragma unroll
+    for (int i = 0; i < 32; i += 4) {
+        l[0] += p[i]; l[1] += p[i + 1]; l[2] += p[i + 2]; l[3] += p[i + 3];
+        pk[i / 2] = pack_bf16x2(p[i], p[i + 1]);
+        pk[i / 2 + 1] = pack_bf16x2(p[i + 2], p[i + 3]);
+    }
+}
+
+__global__ void __launch_bounds__(L3::THREADS, 1)
+fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                 const __grid_constant__ CUtensorMap tmV, __nv_bfloat16* __restrict__ O, int H, int Nq, int Nk,
+                 float scale_log2e, const int32_t* __restrict__ valid_len, int32_t* status) {
+    using LY = L3;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t* Qs = base;                                  // 2 tiles
+    uint8_t* Ks = Qs + 2 * LY::Q_BYTES;                  // KS tiles
+    uint8_t* Vs = Ks + LY::KS * LY::KV_BYTES;            // VS tiles
+    float* xch = reinterpret_cast<float*>(base + LY::TILE_BYTES);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(base + LY::TILE_BYTES + LY::XCH_BYTES);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + LY::NUM_BARS);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+#ifdef FLAT_TRACE3
+    volatile unsigned* trace_buf = reinterpret_cast<volatile unsigned*>(base + LY::TILE_BYTES + LY::XCH_BYTES + 512);
+    for (int i = threadIdx.x; i < TRACE3_WORDS; i += LY::THREADS) trace_buf[i] = 0;
+#endif
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int bh = blockIdx.y;
+    const int row0 = blockIdx.x * (2 * BM);
+    int n = Nk;
+    if (valid_len) { n = valid_len[bh / H]; n = n < 0 ? 0 : (n > Nk ? Nk : n); }
+    const int ntiles = (n + BN - 1) / BN;
+
+    if (threadIdx.x == LY::SOFT_WARPS * 32) {
+        for (int i = 0; i < LY::NUM_BARS; ++i)
+            mbar_init(&bars[i], (i >= LY::P_FULL && i < LY::PV_DONE) ? 8               // one arrival per softmax warp of the tile
+                                : (i >= LY::V_EMPTY && i < LY::S_FULL) ? 2 : 1);     // V_EMPTY: both P V issuers
+        *abort_flag = 0;
+        fence_mbar_init();
+    }
+    if (warp == 0) { tmem_alloc(tmem_slot, LY::TMEM_COLS); tmem_relinquish(); }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    if (warp >= LY::SOFT_WARPS) {
+      asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(OTHER_REGS));
+      if (warp == LY::SOFT_WARPS) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0 && ntiles > 0) {
+            prefetch_tensormap(&tmQ); prefetch_tensormap(&tmK); prefetch_tensormap(&tmV);
+            bool ok = true;
+            int k_issued = 0, v_issued = 0;
+            auto load_k = [&](int j) {
+                const int s = j % LY::KS;
+                ok = bounded_wait(&bars[LY::K_EMPTY + s], ((j / LY::KS) & 1) ^ 1, abort_flag, status, 0x100 + s);
+                if (!ok) return;
+                mbar_arrive_expect_tx(&bars[LY::K_FULL + s], LY::KV_BYTES);
+                tma_load_3d(Ks + s * LY::KV_BYTES, &tmK, &bars[LY::K_FULL + s], 0, j * BN, bh);
+                k_issued = j + 1;
+            };
+            auto load_v = [&](int j) {
+                const int s = j % LY::VS;
+                ok = bounded_wait(&bars[LY::V_EMPTY + s], ((j / LY::VS) & 1) ^ 1, abort_flag, status, 0x110 + s);
+                if (!ok) return;
+                mbar_arrive_expect_tx(&bars[LY::V_FULL + s], LY::KV_BYTES);
+                tma_load_3d(Vs + s * LY::KV_BYTES, &tmV, &bars[LY::V_FULL + s], 0, j * BN, bh);
+                v_issued = j + 1;
+            };
+            mbar_arrive_expect_tx(&bars[LY::Q_FULL + 0], LY::Q_BYTES);
+            tma_load_3d(Qs, &tmQ, &bars[LY::Q_FULL + 0], 0, row0, bh);
+            load_k(0);
+            mbar_arrive_expect_tx(&bars[LY::Q_FULL + 1], LY::Q_BYTES);
+            tma_load_3d(Qs + LY::Q_BYTES, &tmQ, &bars[LY::Q_FULL + 1], 0, row0 + BM, bh);
+            if (ntiles > 1) load_k(1);
+            // S runs ahead of P V: K_{j+2} is wanted before V_{j+1}
+            for (int j = 0; j < ntiles && ok; ++j) {
+                load_v(j);
+                if (ok && j + 2 < ntiles) load_k(j + 2);
+            }
+            if (!ok) {
+                drain_wait(&bars[LY::Q_FULL + 0], 0);
+                drain_wait(&bars[LY::Q_FULL + 1], 0);
+                for (int j = k_issued > LY::KS ? k_issued - LY::KS : 0; j < k_issued; ++j)
+                    drain_wait(&bars[LY::K_FULL + j % LY::KS], (j / LY::KS) & 1);
+                for (int j = v_issued > LY::VS ? v_issued - LY::VS : 0; j < v_issued; ++j)
+                    drain_wait(&bars[LY::V_FULL + j % LY::VS], (j / LY::VS) & 1);
+            }
+        }
+      } else {
+        // ------------------------------------------------------------ MMA issuers
+        // warp 17 / 18: O_t += P V of tile A / B; warp 19: every S = Q K^T.  A whole warp runs its
+        // loop (uniform control flow); one elected lane issues.
+        // Tile-step u: tile u & 1, key step u >> 1, logit/weight buffer u % 3 in its phase u / 3.
+        if (ntiles > 0) {
+            const int steps = 2 * ntiles;
+            bool ok = true;
+            auto wait = [&](int bar, uint32_t parity, int code) {
+                if (ok) ok = __all_sync(0xffffffffu, bounded_wait(&bars[bar], parity, abort_flag, status, code));
+                if (ok) tc_fence_after();
+            };
+            if (warp == LY::SOFT_WARPS + 3) {
+                constexpr uint32_t IDESC_S = make_idesc_bf16(BM, BN, 0, 0);
+                const uint64_t q_desc = make_smem_desc_sw128(smem_u32(Qs), 16, 1024);
+                const uint64_t k_desc = make_smem_desc_sw128(smem_u32(Ks), 16, 1024);
+                int b = 0;
+                for (int u = 0; u < steps && ok; ++u, b = (b == 2 ? 0 : b + 1)) {
+                    const int t = u & 1, j = u >> 1, ks = j % LY::KS;
+                    if (u >= 3) wait(LY::PV_DONE + (t ^ 1) * 3 + b, ((u - 3) / 6) & 1, 0x230 + b);   // the MMAs that read P(u - 3) are done
+                    if (j == 0) wait(LY::Q_FULL + t, 0, 0x200 + t);
+                    if (t == 0) wait(LY::K_FULL + ks, (j / LY::KS) & 1, 0x210);
+                    if (!ok) break;
+                    if (elect_one()) {
+                        const uint64_t qd = q_desc + static_cast<uint64_t>((t * LY::Q_BYTES) >> 4);
+                        const uint64_t kd = k_desc + static_cast<uint64_t>((ks * LY::KV_BYTES) >> 4);
+#pragma unroll
+                        for (int k = 0; k < D / 16; ++k)
+                            mma_ss(tmem + LY::X_COL(b), qd + static_cast<uint64_t>((k * 32) >> 4),
+                                   kd + static_cast<uint64_t>((k * 32) >> 4), IDESC_S, k > 0);
+                        tc_commit(&bars[LY::S_FULL + t * 3 + b]);
+                        if (t == 1) tc_commit(&bars[LY::K_EMPTY + ks]);   // both tiles have used K_j
+                        TRACE(4, u, 1);
+                    }
+                    __syncwarp();
+                }
+            } else {
+                constexpr uint32_t IDESC_PV = make_idesc_bf16(BM, D, 0, 1);
+                const uint64_t v_desc = make_smem_desc_sw128(smem_u32(Vs), BN * 128, 1024);
+                const int t = warp - LY::SOFT_WARPS - 1;
+                int b = t;
+                for (int j = 0; j < ntiles && ok; ++j, b = (b == 0 ? 2 : b - 1)) {
+                    const int u = 2 * j + t, vs = j % LY::VS;
+                    wait(LY::V_FULL + vs, (j / LY::VS) & 1, 0x220);
+                    wait(LY::P_FULL + t * 3 + b, (u / 6) & 1, 0x221);
+                    if (lane == 0) TRACE(4, u, 2);
+                    if (!ok) break;
+                    if (elect_one()) {
+                        const uint64_t vd = v_desc + static_cast<uint64_t>((vs * LY::KV_BYTES) >> 4);
+                        // the two halves of P(u) overlay the first 32 columns of each half of S(u)
+#pragma unroll
+                        for (int k = 0; k < BN / 16; ++k)
+                            mma_ts(tmem + LY::O_COL(t), tmem + LY::X_COL(b) + (k / 4) * HN + (k % 4) * 8,
+                                   vd + static_cast<uint64_t>((k * 2048) >> 4), IDESC_PV, (j > 0 || k > 0));
+                        tc_commit(&bars[LY::PV_DONE + t * 3 + b]);
+                        tc_commit(&bars[LY::V_EMPTY + vs]);
+                        TRACE(4, u, 3);
+                    }
+                    __syncwarp();
+                }
+            }
+        }
+      }
+    } else {
+        // ------------------------------------------------------------ softmax + epilogue (warps 0-15)
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(SOFT_REGS));
+        const int q = warp & 3;                          // row group = TMEM lane quarter
+        const int t = warp >> 3;                         // query tile
+        const int h = (warp >> 2) & 1;                   // key half of every step
+        const int row = row0 + t * BM + q * 32 + lane;
+        const uint32_t tl = tmem + (static_cast<uint32_t>(q * 32) << 16);
+        const int pair_id = 1 + t * 4 + q;               // named barrier of the two warps sharing these rows
+        float* xm_own = xch + ((t * 2 + h) * BM + q * 32 + lane);          // exchanged maxima
+        float* xm_oth = xch + ((t * 2 + (h ^ 1)) * BM + q * 32 + lane);
+        float* xl_own = xm_own + 4 * BM;                                   // exchanged row sums
+        float* xl_oth = xm_oth + 4 * BM;
+        const bool neg_scale = scale_log2e < 0.f;
+        float m_ref = -INFINITY, l = 0.f;
+        bool ok = true;
+        const int trole = t * 2 + h;
+        (void)trole;
+        int b = t;                                       // buffer of tile-step u = 2 j + t: u % 3
+        for (int j = 0; j < ntiles; ++j, b = (b == 0 ? 2 : b - 1)) {      // u += 2  <=>  b -= 1 (mod 3)
+            // this warp's 64 logits of S(u); its 32 packed columns of P(u) go over the first half of them
+            const uint32_t s_addr = tl + LY::X_COL(b) + h * HN;
+            if (q == 0 && lane == 0) TRACE(trole, j, 0);
+            const uint32_t xph = static_cast<uint32_t>((2 * j + t) / 6) & 1u;   // phase parity of this tile's use of the buffer
+            ok = bounded_wait(&bars[LY::S_FULL + t * 3 + b], xph, abort_flag, status, 0x300 + t);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tc_fence_after();
+            if (q == 0 && lane == 0) TRACE(trole, j, 1);
+            const int col0 = j * BN + h * HN;
+            const bool tail = col0 + HN > n;
+            const int nvalid = tail ? (n > col0 ? n - col0 : 0) : HN;
+            // p = 2^(scale*s - m_ref); row sum in fp32 from the unrounded p; P rounded to bf16.  Any
+            // reference m_ref gives the exact softmax, so the common case takes no row maximum; a sum
+            // beyond 2^40 (or inf/NaN) in either half shows that the reference fell too far behind,
+            // and both halves then redo the step the careful way.  The logits stay in TMEM until the
+            // two warps have voted, so the redo reads them again instead of holding them in registers.
+            uint32_t pk[2][16];
+            float ls[4] = {0.f, 0.f, 0.f, 0.f};
+#ifdef FLAT_TC3_ALWAYS_CAREFUL
+            bool careful = true;
+#else
+            bool careful = (j == 0);
+#endif
+            if (!careful) {
+                uint32_t r[2][32];
+                tmem_ld_x32(s_addr, r[0]);
+                tmem_ld_x32(s_addr + 32, r[1]);
+                tc_wait_ld();
+                if (q == 0 && lane == 0) TRACE(trole, j, 2);
+                if (tail) {
+                    exp_pack32<true, false>(r[0], scale_log2e, -m_ref, nvalid, ls, pk[0]);
+                    exp_pack32<true, false>(r[1], scale_log2e, -m_ref, nvalid - 32, ls, pk[1]);
+                } else {
+                    exp_pack32<false, FLAT_TC3_POLY>(r[0], scale_log2e, -m_ref, 32, ls, pk[0]);
+                    exp_pack32<false, FLAT_TC3_POLY>(r[1], scale_log2e, -m_ref, 32, ls, pk[1]);
+                }
+                const float lt = (ls[0] + ls[1]) + (ls[2] + ls[3]);
+                if (q == 0 && lane == 0) TRACE(trole, j, 3);
+#ifdef FLAT_TC3_NOVOTE
+                careful = __any_sync(0xffffffffu, !(lt <= OVERFLOW_SUM));
+#else
+                careful = pair_any(pair_id, !(lt <= OVERFLOW_SUM));
+#endif
+            }
+            if (q == 0 && lane == 0) TRACE(trole, j, 4);
+            if (careful) {
+                float mx = -INFINITY;
+                {
+                    uint32_t s[HN];
+                    tmem_ld_x32(s_addr, *reinterpret_cast<uint32_t(*)[32]>(&s[0]));
+                    tmem_ld_x32(s_addr + 32, *reinterpret_cast<uint32_t(*)[32]>(&s[32]));
+                    tc_wait_ld();
+                    if (tail) {
+                        const uint32_t excl = __float_as_uint(neg_scale ? INFINITY : -INFINITY);
+#pragma unroll
+                        for (int i = 0; i < HN; ++i) if (i >= nvalid) s[i] = excl;
+                    }
+                    if (nvalid > 0) mx = (neg_scale ? half_min(s) : half_max(s)) * scale_log2e;
+                }
+                *xm_own = mx;
+                pair_sync(pair_id);
+                mx = fmaxf(mx, *xm_oth);
+                if (__any_sync(0xffffffffu, mx > m_ref + RESCALE_THRESHOLD)) {
+                    const float m_new = fmaxf(m_ref, mx);
+                    const float alpha = ex2_approx(m_ref - m_new);     // 0 on the first step
+                    l *= alpha;
+                    if (j > 0) {
+                        // each half rescales its half of the columns of O_t
+                        // (O_t += P(u - 2) V must be complete; that tile-step used buffer b + 1 mod 3)
+                        const int u2 = 2 * j + t - 2;
+                        ok = __all_sync(0xffffffffu, bounded_wait(&bars[LY::PV_DONE + t * 3 + (b == 2 ? 0 : b + 1)],
+                                                                 static_cast<uint32_t>(u2 / 6) & 1u, abort_flag, status,
+                                                                 0x310 + t));
+                        if (ok) {
+                            tc_fence_after();
+#pragma unroll
+                            for (int c = 0; c < D / 64; ++c) {
+                                uint32_t r[32];
+                                const uint32_t addr = tl + LY::O_COL(t) + h * (D / 2) + c * 32;
+                                tmem_ld_x32(addr, r);
+                                tc_wait_ld();
+#pragma unroll
+                                for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
+                                tmem_st_x32(addr, r);
+                            }
+                        }
+                    }
+                    m_ref = m_new;
+                }
+                ls[0] = ls[1] = ls[2] = ls[3] = 0.f;
+#pragma unroll
+                for (int c = 0; c < 2; ++c) {            // the logits are read again, 32 at a time
+                    uint32_t r[32];
+                    tmem_ld_x32(s_addr + c * 32, r);
+                    tc_wait_ld();
+                    exp_pack32<true, false>(r, scale_log2e, -m_ref, nvalid - c * 32, ls, pk[c]);
+                }
+            }
+            // a failed wait is voted on so that the two warps leave the loop together (only the
+            // careful path waits for anything)
+            if (careful && pair_any(pair_id, !ok)) ok = false;
+            if (!ok) break;
+            if (q == 0 && lane == 0) TRACE(trole, j, 5);
+            tmem_st_x16(s_addr, pk[0]);
+            tmem_st_x16(s_addr + 16, pk[1]);
+            l += (ls[0] + ls[1]) + (ls[2] + ls[3]);
+            tc_wait_st();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&bars[LY::P_FULL + t * 3 + b]);
+            if (q == 0 && lane == 0) TRACE(trole, j, 7);
+        }
+        if (ok && ntiles > 0) {
+            // the last O_t += P V (the issuer's MMAs complete in order)
+            const int ul = 2 * (ntiles - 1) + t;
+            ok = bounded_wait(&bars[LY::PV_DONE + t * 3 + ul % 3], static_cast<uint32_t>(ul / 6) & 1u, abort_flag, status,
+                              0x330 + t);
+            ok = __all_sync(0xffffffffu, ok);
+        }
+        // row sum of both halves (a warp that gave up still takes part, so that its partner is not left waiting)
+        *xl_own = l;
+        pair_sync(pair_id);
+        l += *xl_oth;
+        if (ok) {
+            const float inv = l > 0.f ? 1.f / l : 0.f;
+            tc_fence_after();
+            __nv_bfloat16* orow = O + (static_cast<int64_t>(bh) * Nq + row) * D + h * (D / 2);
+#pragma unroll
+            for (int c = 0; c < D / 64; ++c) {
+                uint32_t r[32];
+                if (ntiles > 0) {
+                    tmem_ld_x32(tl + LY::O_COL(t) + h * (D / 2) + c * 32, r);
+                    tc_wait_ld();
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) r[i] = 0u;      // no valid key: O = 0
+                }
+                if (row < Nq) {
+#pragma unroll
+                    for (int v = 0; v < 4; ++v) {
+                        uint4 w;
+                        w.x = pack_bf16x2(__uint_as_float(r[8 * v + 0]) * inv, __uint_as_float(r[8 * v + 1]) * inv);
+                        w.y = pack_bf16x2(__uint_as_float(r[8 * v + 2]) * inv, __uint_as_float(r[8 * v + 3]) * inv);
+                        w.z = pack_bf16x2(__uint_as_float(r[8 * v + 4]) * inv, __uint_as_float(r[8 * v + 5]) * inv);
+                        w.w = pack_bf16x2(__uint_as_float(r[8 * v + 6]) * inv, __uint_as_float(r[8 * v + 7]) * inv);
+                        *reinterpret_cast<uint4*>(orow + c * 32 + v * 8) = w;
+                    }
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem, LY::TMEM_COLS);
+#ifdef FLAT_TRACE3
+    if (g_trace3 && blockIdx.x == 0 && blockIdx.y == 0)
+        for (int i = threadIdx.x; i < TRACE3_WORDS; i += LY::THREADS) g_trace3[i] = trace_buf[i];
+#endif
+}
+
+int launch_tc3(const Problem& p, cudaStream_t st) {
+    using LY = L3;
+    CUtensorMap tmQ, tmK, tmV;
+    const int BH = p.B * p.H;
+    if (!make_map(&tmQ, p.Q, BH, p.Nq, D, BM) || !make_map(&tmK, p.K, BH, p.Nk, D, BN) ||
+        !make_map(&tmV, p.V, BH, p.Nk, D, BN))
+        return FLAT_ERR_CUDA;
+    if (!ensure_dynamic_smem<fused_tc3_kernel>(LY::SMEM_BYTES)) return FLAT_ERR_CUDA;
+    dim3 grid((p.Nq + 2 * BM - 1) / (2 * BM), BH);
+    fused_tc3_kernel<<<grid, LY::THREADS, LY::SMEM_BYTES, st>>>(tmQ, tmK, tmV, static_cast<__nv_bfloat16*>(p.O), p.H,
+                                                                p.Nq, p.Nk, p.scale * 1.4426950408889634f,
+                                                                p.k_valid_len, p.status);
+    return cudaGetLastError() == cudaSuccess ? FLAT_OK : FLAT_ERR_CUDA;
+}
+
+}  // namespace
+
+int launch_fused_tc3(const Problem& p, cudaStream_t st) {
+    if (p.dtype != FLAT_DTYPE_BF16 || p.d != D) return FLAT_ERR_UNSUPPORTED;
+    return launch_tc3(p, st);
+}
+
+}  // namespace flat

@@ -42,10 +42,10 @@ SMALL = [
 
 
 @pytest.mark.parametrize("shape", SMALL)
-@pytest.mark.parametrize("variant", [1, 2, 3, 4], ids=["simt", "tc", "tc2", "tc2single"])
+@pytest.mark.parametrize("variant", [1, 2, 3, 4, 5], ids=["simt", "tc", "tc2", "tc2single", "tc3"])
 def test_fused_bf16_small(api, shape, variant):
     B, H, Nq, Nk, d = shape
-    if variant == 4 and d != 64:
+    if variant in (4, 5) and d != 64:
         pytest.skip("single-tile TC2 CTAs exist for d = 64 only")
     rng = np.random.default_rng(abs(hash(shape)) % (2 ** 31))
     Qb, Kb, Vb = rand_bits(rng, (B, H, Nq, d)), rand_bits(rng, (B, H, Nk, d)), rand_bits(rng, (B, H, Nk, d))
@@ -55,10 +55,10 @@ def test_fused_bf16_small(api, shape, variant):
     check_bf16(got, ref, "fused bf16 %s v%d" % (shape, variant))
 
 
-@pytest.mark.parametrize("variant", [1, 2, 3, 4], ids=["simt", "tc", "tc2", "tc2single"])
+@pytest.mark.parametrize("variant", [1, 2, 3, 4, 5], ids=["simt", "tc", "tc2", "tc2single", "tc3"])
 @pytest.mark.parametrize("d", [64, 128])
 def test_fused_bf16_masked(api, variant, d):
-    if variant == 4 and d != 64:
+    if variant in (4, 5) and d != 64:
         pytest.skip("single-tile TC2 CTAs exist for d = 64 only")
     B, H, Nq, Nk = 5, 2, 200, 600
     rng = np.random.default_rng(77 + d)
@@ -77,7 +77,7 @@ def test_fused_bf16_masked(api, variant, d):
     assert np.all(got[4] == 0.0)                            # no valid key: O = 0
 
 
-@pytest.mark.parametrize("variant", [1, 2, 3, 4], ids=["simt", "tc", "tc2", "tc2single"])
+@pytest.mark.parametrize("variant", [1, 2, 3, 4, 5], ids=["simt", "tc", "tc2", "tc2single", "tc3"])
 def test_fused_bf16_planted_keys(api, variant):
     """Peaked softmax on a planted key with position-coded V: a dropped, duplicated, shifted or
     mis-masked key tile moves O by O(1)."""
@@ -100,7 +100,7 @@ def test_fused_bf16_scales_tc(api, scale):
     rng = np.random.default_rng(5)
     Qb, Kb, Vb = rand_bits(rng, (B, H, Nq, d)), rand_bits(rng, (B, H, Nk, d)), rand_bits(rng, (B, H, Nk, d))
     ref = oracle.attention(Qb, Kb, Vb, scale)["O"]
-    for variant in (2, 3, 4):
+    for variant in (2, 3, 4, 5):
         got = run_fused_bf16(api, Qb, Kb, Vb, scale, variant=variant)
         check_bf16(got, ref, "scale %g v%d" % (scale, variant))
 
@@ -117,7 +117,7 @@ def test_rising_maximum_forces_rescale(api):
     ref = oracle.attention(Qb, Kb, Vb, 1.0, want_logits=True)
     L = ref["L"].reshape(Nq, Nk)
     assert np.all(L[:, -128:].max(1) - L[:, :128].max(1) > 20)      # > 8 log2 units per several tiles
-    for variant in (1, 2, 3, 4):
+    for variant in (1, 2, 3, 4, 5):
         got = run_fused_bf16(api, Qb, Kb, Vb, 1.0, variant=variant)
         check_bf16(got, ref["O"], "rising max v%d" % variant)
 
@@ -209,7 +209,7 @@ def test_output_padding_untouched(api):
     Qb, Kb, Vb = rand_bits(rng, (B, H, Nq, d)), rand_bits(rng, (B, H, Nk, d)), rand_bits(rng, (B, H, Nk, d))
     Q, K, V = bf16_tensor(Qb), bf16_tensor(Kb), bf16_tensor(Vb)
     n = B * H * Nq * d
-    for variant in (1, 2, 3):
+    for variant in (1, 2, 3, 5):
         buf = torch.full((n + 2048,), 7.0, dtype=torch.bfloat16, device="cuda")
         O = buf[1024:1024 + n].view(B, H, Nq, d)
         api.flat_attn_fwd_ex(Q, K, V, O, 0.125, variant=variant)
@@ -243,12 +243,13 @@ def test_wide_dynamic_range(api, sigma, scale):
     ref = oracle.attention(Qb, Kb, Vb, scale, want_logits=True)
     spread = ref["L"].max(-1) - np.median(ref["L"], -1)
     assert np.median(spread) > 100                                  # far beyond 2^126 in base-2 terms
-    for variant in (1, 2, 3, 4):
+    for variant in (1, 2, 3, 4, 5):
         got = run_fused_bf16(api, Qb, Kb, Vb, scale, variant=variant)
         check_bf16(got, ref["O"], "wide range sigma=%g scale=%g v%d" % (sigma, scale, variant))
 
 
-def test_spike_on_polynomial_lane(api):
+@pytest.mark.parametrize("spike_col", [3, 67, 127], ids=["col3", "col67", "col127"])
+def test_spike_on_polynomial_lane(api, spike_col):
     """One key far above all others (hundreds of log2 units), sitting in a later tile on a column
     that the kernel evaluates with the polynomial exponential and not with the ex2 unit: the clamp
     must turn it into an overflow that forces the careful pass, not into garbage."""
@@ -257,13 +258,16 @@ def test_spike_on_polynomial_lane(api):
     u = np.ones(d, dtype=np.float32)
     Qf = (u[None, :] * (1.0 + rng.random((Nq, 1), dtype=np.float32)) + 0.1 * rng.standard_normal((Nq, d))).astype(np.float32)
     Kf = (0.01 * rng.standard_normal((Nk, d))).astype(np.float32)
+    # (column 3 and 67: polynomial lanes of the first / second half of a 128-key step, which the
+    # kernel that splits a row over two threads handles in different warps; 127: last ex2 lane)
     Kf[131] = 2.0 * u           # tile 1, column 3
-    Kf[1027] = 6.0 * u          # tile 8, column 3: 4 * 64 * (1..2) = 256..512 above the first spike
+    big = 1024 + spike_col
+    Kf[big] = 6.0 * u           # tile 8: 4 * 64 * (1..2) = 256..512 above the first spike
     Vf = rng.standard_normal((Nk, d)).astype(np.float32)
     Qb, Kb, Vb = (inputs.f32_to_bf16_bits(x).reshape(1, 1, *x.shape) for x in (Qf, Kf, Vf))
     ref = oracle.attention(Qb, Kb, Vb, 1.0, want_weights=True)
-    assert np.all(ref["A"][0, 0].argmax(-1) == 1027)
-    for variant in (2, 3, 4):
+    assert np.all(ref["A"][0, 0].argmax(-1) == big)
+    for variant in (2, 3, 4, 5):
         got = run_fused_bf16(api, Qb, Kb, Vb, 1.0, variant=variant)
         check_bf16(got, ref["O"], "spike v%d" % variant)
 
