@@ -6,9 +6,9 @@
 //     waits (barrier, TMEM load, store completion) hide behind the exponentials of the others;
 //   * TMEM holds O_A, O_B (64 columns each) and THREE logit buffers X0..X2 of 128 columns that the
 //     tile-steps u = 0, 1, 2, ... (u even: tile A, u odd: tile B, key step u / 2) use in rotation;
-//     the weights P(u) overlay the logits S(u) they came from, and S(u + 3) is issued as soon as
-//     the MMAs that read P(u) have completed, so the logits of a tile's next step are in TMEM long
-//     before its softmax asks for them.
+//     the weights P(u) overlay the logits S(u) they came from, and S(u + 3) is issued right behind
+//     the MMAs that read P(u) (same thread, so the tensor pipe keeps the order): the logits of a
+//     tile's next step are computed while the other tile's softmax runs.
 //
 // Paper mapping (Section 5, 5.1, 5.2): shared outer loops = (batch, head) on blockIdx.y and a slab
 // of 256 query rows on blockIdx.x (R-granularity); inner loops Logit and Attend interleaved over
@@ -18,8 +18,9 @@
 //   warps 0-15  softmax: warp w serves row group q = w % 4 (TMEM lanes 32q..32q+31) of tile
 //               t = w / 8, key half h = (w / 4) % 2 of every step
 //   warp  16    TMA producer (one lane): Q tiles once, then K and V tiles into separate rings
-//   warp  17/18 MMA issuers of O_t += P V for tile A / B (one elected lane each)
-//   warp  19    MMA issuer of every S = Q K^T
+//   warp  17/18 MMA issuers (one elected lane each): O_t += P(u) V for the tile-steps of tile A / B,
+//               each followed by the logits S(u + 3) of the other tile into the buffer just read
+//   warp  19    idle (it completes the warpgroup for the register hand-over)
 // The two warps that share a row keep the same reference maximum m_ref: the first step fixes it
 // from the exact maximum of both halves (exchanged through shared memory); later steps reuse it and
 // vote, with one reducing named barrier per step, on whether either half's row sum overflowed 2^40,
@@ -71,6 +72,9 @@ constexpr float OVERFLOW_SUM = 1.0995116e12f;   // 2^40: a row sum beyond this m
 #endif
 #ifndef FLAT_TC3_POLY
 #define FLAT_TC3_POLY true
+#endif
+#ifndef FLAT_TC3_POLY_PAIRS
+#define FLAT_TC3_POLY_PAIRS 0x0202   // bit i: pair i of each 16 pairs (32 logits) takes the polynomial; two pairs = one element in eight
 #endif
 constexpr int SOFT_REGS = FLAT_TC3_SOFT_REGS, OTHER_REGS = FLAT_TC3_OTHER_REGS;
 static_assert(512 * SOFT_REGS + 128 * OTHER_REGS <= 640 * 96, "register hand-over exceeds the CTA's allocation");
@@ -140,6 +144,15 @@ __device__ __forceinline__ float half_min(const uint32_t (&s)[HN]) {
     return fminf(fminf(e0, e1), fminf(e2, e3));
 }
 
+__device__ __forceinline__ void st_shared_f32(uint32_t addr, float v) {
+    asm volatile("st.shared::cta.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
+}
+__device__ __forceinline__ float ld_shared_f32(uint32_t addr) {
+    float v;
+    asm volatile("ld.shared::cta.f32 %0, [%1];" : "=f"(v) : "r"(addr) : "memory");
+    return v;
+}
+
 // Named barrier of the two warps (64 threads) that share a row group of a tile.
 __device__ __forceinline__ void pair_sync(int id) {
     asm volatile("bar.sync %0, 64;" ::"r"(id) : "memory");
@@ -156,6 +169,75 @@ __device__ __forceinline__ bool pair_any(int id, bool flag) {
         : "r"(id), "r"(static_cast<uint32_t>(flag))
         : "memory");
     return r != 0;
+}
+
+// Two fp32 values in one 64-bit register pair, for the packed fp32 instructions of sm_100
+// (fma / add / sub .f32x2: two results per issue slot).
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+    uint64_t v;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(v) : "f"(lo), "f"(hi));
+    return v;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+// ex2_poly (see tc_common.cuh) without the upper clamp: the caller keeps the maximum of the
+// arguments and treats one above 126 as an overflow of the row.  Scalar on purpose: the constants
+// ride along as immediates, where packed instructions would want them in registers.
+__device__ __forceinline__ float ex2_poly_lo(float x) {
+    x = fmaxf(x, -126.f);
+    const float t = x + 12582912.f;                    // 1.5 * 2^23: the low mantissa bits now hold round(x)
+    const float f = x - (t - 12582912.f);
+    float p = fmaf(0.05508868f, f, 0.24260405f);
+    p = fmaf(p, f, 0.69327624f);
+    p = fmaf(p, f, 0.99992894f);
+    return __uint_as_float(__float_as_uint(p) + (__float_as_uint(t) << 23));
+}
+
+// The common case (all 32 logits of a chunk valid) in two parts, so that the registers of the
+// logits are free for the next TMEM load while the exponentials run.
+// Part 1: x = r * scale + neg_m as packed pairs.
+__device__ __forceinline__ void scale32(const uint32_t (&r)[32], uint64_t scale2, uint64_t neg_m2, uint64_t (&x2)[16]) {
+#pragma unroll
+    for (int i = 0; i < 16; ++i)
+        x2[i] = fma2(pack2(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1])), scale2, neg_m2);
+}
+// Part 2: p = 2^x, packed row sums, bf16 packing.  With POLY, pairs 1, 5, 9, 13 (one element in
+// four) take the polynomial instead of the ex2 unit and `xmax` follows the largest argument given
+// to it.  l2[0] sums elements 0, 1 (mod 4), l2[1] elements 2, 3.
+template <bool POLY>
+__device__ __forceinline__ void exp_pack_x2(const uint64_t (&x2)[16], uint64_t (&l2)[2], float& xmax, uint32_t (&pk)[16]) {
+    float p[32];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+        float a, b;
+        unpack2(x2[i], a, b);
+        if (POLY && ((FLAT_TC3_POLY_PAIRS >> i) & 1)) {
+            xmax = max3(xmax, a, b);
+            p[2 * i] = ex2_poly_lo(a);
+            p[2 * i + 1] = ex2_poly_lo(b);
+        } else {
+            p[2 * i] = ex2_approx(a);
+            p[2 * i + 1] = ex2_approx(b);
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < 32; i += 4) {
+        l2[0] = add2(l2[0], pack2(p[i], p[i + 1]));
+        l2[1] = add2(l2[1], pack2(p[i + 2], p[i + 3]));
+        pk[i / 2] = pack_bf16x2(p[i], p[i + 1]);
+        pk[i / 2 + 1] = pack_bf16x2(p[i + 2], p[i + 3]);
+    }
 }
 
 // p_i = 2^(r_i * scale + neg_m) for 32 logits of a row: adds the unrounded p to the four partial
@@ -211,7 +293,7 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     if (threadIdx.x == LY::SOFT_WARPS * 32) {
         for (int i = 0; i < LY::NUM_BARS; ++i)
             mbar_init(&bars[i], (i >= LY::P_FULL && i < LY::PV_DONE) ? 8               // one arrival per softmax warp of the tile
-                                : (i >= LY::V_EMPTY && i < LY::S_FULL) ? 2 : 1);     // V_EMPTY: both P V issuers
+                                : (i >= LY::K_EMPTY && i < LY::V_FULL) || (i >= LY::V_EMPTY && i < LY::S_FULL) ? 2 : 1);   // K/V_EMPTY: both issuers
         *abort_flag = 0;
         fence_mbar_init();
     }
@@ -267,64 +349,66 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         }
       } else {
         // ------------------------------------------------------------ MMA issuers
-        // warp 17 / 18: O_t += P V of tile A / B; warp 19: every S = Q K^T.  A whole warp runs its
-        // loop (uniform control flow); one elected lane issues.
-        // Tile-step u: tile u & 1, key step u >> 1, logit/weight buffer u % 3 in its phase u / 3.
-        if (ntiles > 0) {
+        // Warp 17 / 18 serves the tile-steps u of tile A / B: O_t += P(u) V, then, into the buffer
+        // that these MMAs have just read (same thread: the tensor pipe keeps the order), the logits
+        // S(u + 3) of the OTHER tile.  A whole warp runs the loop (uniform control flow); one elected
+        // lane issues.  Tile-step u: tile u & 1, key step u >> 1, buffer u % 3.
+        if (ntiles > 0 && warp <= LY::SOFT_WARPS + 2) {
+            constexpr uint32_t IDESC_S = make_idesc_bf16(BM, BN, 0, 0);
+            constexpr uint32_t IDESC_PV = make_idesc_bf16(BM, D, 0, 1);
+            const int t = warp - LY::SOFT_WARPS - 1;
+            // logits are always those of the other tile
+            const uint64_t q_desc = make_smem_desc_sw128(smem_u32(Qs) + (t ^ 1) * LY::Q_BYTES, 16, 1024);
+            const uint64_t k_desc = make_smem_desc_sw128(smem_u32(Ks), 16, 1024);
+            const uint64_t v_desc = make_smem_desc_sw128(smem_u32(Vs), BN * 128, 1024);
             const int steps = 2 * ntiles;
             bool ok = true;
             auto wait = [&](int bar, uint32_t parity, int code) {
                 if (ok) ok = __all_sync(0xffffffffu, bounded_wait(&bars[bar], parity, abort_flag, status, code));
                 if (ok) tc_fence_after();
             };
-            if (warp == LY::SOFT_WARPS + 3) {
-                constexpr uint32_t IDESC_S = make_idesc_bf16(BM, BN, 0, 0);
-                const uint64_t q_desc = make_smem_desc_sw128(smem_u32(Qs), 16, 1024);
-                const uint64_t k_desc = make_smem_desc_sw128(smem_u32(Ks), 16, 1024);
-                int b = 0;
-                for (int u = 0; u < steps && ok; ++u, b = (b == 2 ? 0 : b + 1)) {
-                    const int t = u & 1, j = u >> 1, ks = j % LY::KS;
-                    if (u >= 3) wait(LY::PV_DONE + (t ^ 1) * 3 + b, ((u - 3) / 6) & 1, 0x230 + b);   // the MMAs that read P(u - 3) are done
-                    if (j == 0) wait(LY::Q_FULL + t, 0, 0x200 + t);
-                    if (t == 0) wait(LY::K_FULL + ks, (j / LY::KS) & 1, 0x210);
-                    if (!ok) break;
-                    if (elect_one()) {
-                        const uint64_t qd = q_desc + static_cast<uint64_t>((t * LY::Q_BYTES) >> 4);
-                        const uint64_t kd = k_desc + static_cast<uint64_t>((ks * LY::KV_BYTES) >> 4);
+            auto issue_s = [&](int us, int bs) {         // S(us) of tile t ^ 1 into buffer bs
+                const int js = us >> 1, ks = js % LY::KS;
+                if (js == 0) wait(LY::Q_FULL + (t ^ 1), 0, 0x200 + t);
+                wait(LY::K_FULL + ks, (js / LY::KS) & 1, 0x210);
+                if (!ok) return;
+                if (elect_one()) {
+                    const uint64_t kd = k_desc + static_cast<uint64_t>((ks * LY::KV_BYTES) >> 4);
 #pragma unroll
-                        for (int k = 0; k < D / 16; ++k)
-                            mma_ss(tmem + LY::X_COL(b), qd + static_cast<uint64_t>((k * 32) >> 4),
-                                   kd + static_cast<uint64_t>((k * 32) >> 4), IDESC_S, k > 0);
-                        tc_commit(&bars[LY::S_FULL + t * 3 + b]);
-                        if (t == 1) tc_commit(&bars[LY::K_EMPTY + ks]);   // both tiles have used K_j
-                        TRACE(4, u, 1);
-                    }
-                    __syncwarp();
+                    for (int k = 0; k < D / 16; ++k)
+                        mma_ss(tmem + LY::X_COL(bs), q_desc + static_cast<uint64_t>((k * 32) >> 4),
+                               kd + static_cast<uint64_t>((k * 32) >> 4), IDESC_S, k > 0);
+                    tc_commit(&bars[LY::S_FULL + (t ^ 1) * 3 + bs]);
+                    tc_commit(&bars[LY::K_EMPTY + ks]);   // (counts 2: both tiles' logits have used K_j)
+                    TRACE(4, us, 1);
                 }
-            } else {
-                constexpr uint32_t IDESC_PV = make_idesc_bf16(BM, D, 0, 1);
-                const uint64_t v_desc = make_smem_desc_sw128(smem_u32(Vs), BN * 128, 1024);
-                const int t = warp - LY::SOFT_WARPS - 1;
-                int b = t;
-                for (int j = 0; j < ntiles && ok; ++j, b = (b == 0 ? 2 : b - 1)) {
-                    const int u = 2 * j + t, vs = j % LY::VS;
-                    wait(LY::V_FULL + vs, (j / LY::VS) & 1, 0x220);
-                    wait(LY::P_FULL + t * 3 + b, (u / 6) & 1, 0x221);
-                    if (lane == 0) TRACE(4, u, 2);
-                    if (!ok) break;
-                    if (elect_one()) {
-                        const uint64_t vd = v_desc + static_cast<uint64_t>((vs * LY::KV_BYTES) >> 4);
-                        // the two halves of P(u) overlay the first 32 columns of each half of S(u)
+                __syncwarp();
+            };
+            // the first three logit tiles need no buffer to be freed: S(0), S(2) (tile A) come from
+            // tile B's issuer, S(1) from tile A's
+            if (t == 1) { issue_s(0, 0); if (steps > 2) issue_s(2, 2); }
+            else issue_s(1, 1);
+            int b = t;
+            for (int j = 0; j < ntiles && ok; ++j, b = (b == 0 ? 2 : b - 1)) {
+                const int u = 2 * j + t, vs = j % LY::VS;
+                if (lane == 0) TRACE(4, u, 0);
+                wait(LY::V_FULL + vs, (j / LY::VS) & 1, 0x220);
+                wait(LY::P_FULL + t * 3 + b, (u / 6) & 1, 0x221);
+                if (lane == 0) TRACE(4, u, 2);
+                if (!ok) break;
+                if (elect_one()) {
+                    const uint64_t vd = v_desc + static_cast<uint64_t>((vs * LY::KV_BYTES) >> 4);
+                    // the two halves of P(u) overlay the first 32 columns of each half of S(u)
 #pragma unroll
-                        for (int k = 0; k < BN / 16; ++k)
-                            mma_ts(tmem + LY::O_COL(t), tmem + LY::X_COL(b) + (k / 4) * HN + (k % 4) * 8,
-                                   vd + static_cast<uint64_t>((k * 2048) >> 4), IDESC_PV, (j > 0 || k > 0));
-                        tc_commit(&bars[LY::PV_DONE + t * 3 + b]);
-                        tc_commit(&bars[LY::V_EMPTY + vs]);
-                        TRACE(4, u, 3);
-                    }
-                    __syncwarp();
+                    for (int k = 0; k < BN / 16; ++k)
+                        mma_ts(tmem + LY::O_COL(t), tmem + LY::X_COL(b) + (k / 4) * HN + (k % 4) * 8,
+                               vd + static_cast<uint64_t>((k * 2048) >> 4), IDESC_PV, (j > 0 || k > 0));
+                    tc_commit(&bars[LY::PV_DONE + t * 3 + b]);
+                    tc_commit(&bars[LY::V_EMPTY + vs]);
+                    TRACE(4, u, 3);
                 }
+                __syncwarp();
+                if (u + 3 < steps) issue_s(u + 3, b);
             }
         }
       }
@@ -337,10 +421,10 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         const int row = row0 + t * BM + q * 32 + lane;
         const uint32_t tl = tmem + (static_cast<uint32_t>(q * 32) << 16);
         const int pair_id = 1 + t * 4 + q;               // named barrier of the two warps sharing these rows
-        float* xm_own = xch + ((t * 2 + h) * BM + q * 32 + lane);          // exchanged maxima
-        float* xm_oth = xch + ((t * 2 + (h ^ 1)) * BM + q * 32 + lane);
-        float* xl_own = xm_own + 4 * BM;                                   // exchanged row sums
-        float* xl_oth = xm_oth + 4 * BM;
+        // shared-window addresses: the barriers, the abort flag, and this thread's slot for exchanged
+        // maxima (its partner's is BM floats away: flip bit 9; the row sums sit 4 * BM floats further)
+        const uint32_t bars_s = smem_u32(bars), abort_s = smem_u32(const_cast<int*>(abort_flag));
+        const uint32_t xm_own = smem_u32(xch + ((t * 2 + h) * BM + q * 32 + lane));
         const bool neg_scale = scale_log2e < 0.f;
         float m_ref = -INFINITY, l = 0.f;
         bool ok = true;
@@ -352,7 +436,7 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             const uint32_t s_addr = tl + LY::X_COL(b) + h * HN;
             if (q == 0 && lane == 0) TRACE(trole, j, 0);
             const uint32_t xph = static_cast<uint32_t>((2 * j + t) / 6) & 1u;   // phase parity of this tile's use of the buffer
-            ok = bounded_wait(&bars[LY::S_FULL + t * 3 + b], xph, abort_flag, status, 0x300 + t);
+            ok = bounded_wait_s(bars_s + 8 * (LY::S_FULL + t * 3 + b), xph, abort_s, status, 0x300 + t);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
@@ -373,25 +457,38 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             bool careful = (j == 0);
 #endif
             if (!careful) {
-                uint32_t r[2][32];
-                tmem_ld_x32(s_addr, r[0]);
-                tmem_ld_x32(s_addr + 32, r[1]);
+                // (the logits come in two loads of 32 so that few registers are live at a time)
+                uint32_t r[32];
+                float lt;
+                tmem_ld_x32(s_addr, r);
                 tc_wait_ld();
                 if (q == 0 && lane == 0) TRACE(trole, j, 2);
                 if (tail) {
-                    exp_pack32<true, false>(r[0], scale_log2e, -m_ref, nvalid, ls, pk[0]);
-                    exp_pack32<true, false>(r[1], scale_log2e, -m_ref, nvalid - 32, ls, pk[1]);
+                    exp_pack32<true, false>(r, scale_log2e, -m_ref, nvalid, ls, pk[0]);
+                    tmem_ld_x32(s_addr + 32, r);
+                    tc_wait_ld();
+                    exp_pack32<true, false>(r, scale_log2e, -m_ref, nvalid - 32, ls, pk[1]);
+                    lt = (ls[0] + ls[1]) + (ls[2] + ls[3]);
                 } else {
-                    exp_pack32<false, FLAT_TC3_POLY>(r[0], scale_log2e, -m_ref, 32, ls, pk[0]);
-                    exp_pack32<false, FLAT_TC3_POLY>(r[1], scale_log2e, -m_ref, 32, ls, pk[1]);
+                    const uint64_t scale2 = pack2(scale_log2e, scale_log2e), neg_m2 = pack2(-m_ref, -m_ref);
+                    uint64_t l2[2] = {0ull, 0ull};
+                    uint64_t x2[16];
+                    float xmax = 0.f;
+                    scale32(r, scale2, neg_m2, x2);
+                    tmem_ld_x32(s_addr + 32, r);         // the second 32 logits arrive during the first 32 exponentials
+                    exp_pack_x2<FLAT_TC3_POLY>(x2, l2, xmax, pk[0]);
+                    tc_wait_ld();
+                    scale32(r, scale2, neg_m2, x2);
+                    exp_pack_x2<FLAT_TC3_POLY>(x2, l2, xmax, pk[1]);
+                    float a, b2, c, d2;
+                    unpack2(l2[0], a, b2);
+                    unpack2(l2[1], c, d2);
+                    lt = (a + b2) + (c + d2);
+                    ls[0] = lt;
+                    if (xmax > 126.f) lt = INFINITY;      // the polynomial was fed an argument beyond its range
                 }
-                const float lt = (ls[0] + ls[1]) + (ls[2] + ls[3]);
                 if (q == 0 && lane == 0) TRACE(trole, j, 3);
-#ifdef FLAT_TC3_NOVOTE
-                careful = __any_sync(0xffffffffu, !(lt <= OVERFLOW_SUM));
-#else
                 careful = pair_any(pair_id, !(lt <= OVERFLOW_SUM));
-#endif
             }
             if (q == 0 && lane == 0) TRACE(trole, j, 4);
             if (careful) {
@@ -408,9 +505,9 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                     }
                     if (nvalid > 0) mx = (neg_scale ? half_min(s) : half_max(s)) * scale_log2e;
                 }
-                *xm_own = mx;
+                st_shared_f32(xm_own, mx);
                 pair_sync(pair_id);
-                mx = fmaxf(mx, *xm_oth);
+                mx = fmaxf(mx, ld_shared_f32(xm_own ^ (BM * 4)));
                 if (__any_sync(0xffffffffu, mx > m_ref + RESCALE_THRESHOLD)) {
                     const float m_new = fmaxf(m_ref, mx);
                     const float alpha = ex2_approx(m_ref - m_new);     // 0 on the first step
@@ -419,9 +516,9 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                         // each half rescales its half of the columns of O_t
                         // (O_t += P(u - 2) V must be complete; that tile-step used buffer b + 1 mod 3)
                         const int u2 = 2 * j + t - 2;
-                        ok = __all_sync(0xffffffffu, bounded_wait(&bars[LY::PV_DONE + t * 3 + (b == 2 ? 0 : b + 1)],
-                                                                 static_cast<uint32_t>(u2 / 6) & 1u, abort_flag, status,
-                                                                 0x310 + t));
+                        ok = __all_sync(0xffffffffu,
+                                        bounded_wait_s(bars_s + 8 * (LY::PV_DONE + t * 3 + (b == 2 ? 0 : b + 1)),
+                                                       static_cast<uint32_t>(u2 / 6) & 1u, abort_s, status, 0x310 + t));
                         if (ok) {
                             tc_fence_after();
 #pragma unroll
@@ -458,20 +555,21 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             tc_wait_st();
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&bars[LY::P_FULL + t * 3 + b]);
+            if (lane == 0) mbar_arrive_s(bars_s + 8 * (LY::P_FULL + t * 3 + b));
             if (q == 0 && lane == 0) TRACE(trole, j, 7);
+            if (lane == 0) TRACE(trole, j, 8 + q);
         }
         if (ok && ntiles > 0) {
             // the last O_t += P V (the issuer's MMAs complete in order)
             const int ul = 2 * (ntiles - 1) + t;
-            ok = bounded_wait(&bars[LY::PV_DONE + t * 3 + ul % 3], static_cast<uint32_t>(ul / 6) & 1u, abort_flag, status,
-                              0x330 + t);
+            ok = bounded_wait_s(bars_s + 8 * (LY::PV_DONE + t * 3 + ul % 3), static_cast<uint32_t>(ul / 6) & 1u, abort_s,
+                                status, 0x330 + t);
             ok = __all_sync(0xffffffffu, ok);
         }
         // row sum of both halves (a warp that gave up still takes part, so that its partner is not left waiting)
-        *xl_own = l;
+        st_shared_f32(xm_own + 4 * BM * 4, l);
         pair_sync(pair_id);
-        l += *xl_oth;
+        l += ld_shared_f32((xm_own ^ (BM * 4)) + 4 * BM * 4);
         if (ok) {
             const float inv = l > 0.f ? 1.f / l : 0.f;
             tc_fence_after();

@@ -36,6 +36,26 @@ __device__ __forceinline__ bool bounded_wait(uint64_t* bar, uint32_t parity, vol
     }
 }
 
+// The same wait with the barrier and the abort flag given as 32-bit shared-window addresses.
+__device__ __forceinline__ bool bounded_wait_s(uint32_t bar_addr, uint32_t parity, uint32_t abort_addr,
+                                               int32_t* status, int code, long long limit = WAIT_CYCLES) {
+    if (ptx::mbar_try_wait_s(bar_addr, parity)) return true;
+    const long long t0 = clock64();
+    for (;;) {
+#pragma unroll 1
+        for (int i = 0; i < 32; ++i)
+            if (ptx::mbar_try_wait_s(bar_addr, parity)) return true;
+        int aborted;
+        asm volatile("ld.volatile.shared::cta.s32 %0, [%1];" : "=r"(aborted) : "r"(abort_addr) : "memory");
+        if (aborted) return false;
+        if (clock64() - t0 > limit) {
+            asm volatile("st.volatile.shared::cta.s32 [%0], %1;" ::"r"(abort_addr), "r"(1) : "memory");
+            if (status) atomicExch(status, code);
+            return false;
+        }
+    }
+}
+
 // Teardown helper: wait for a copy this thread started, with a time limit and no side effects.
 __device__ __forceinline__ void drain_wait(uint64_t* bar, uint32_t parity) {
     const long long t0 = clock64();
