@@ -28,8 +28,18 @@ METRIC = "fused attention TFLOP/s"
 UNIT = "TFLOP/s"
 DEFAULT_WORKLOAD = "c2_bert_large_4k"
 L2_FLUSH_BELOW = 256 << 20          # workloads smaller than this get an L2 flush before every timed launch
-KERNEL_NAMES = {0: "fused_tc2_kernel", 1: "fused_simt_kernel", 2: "fused_tc_kernel", 3: "fused_tc2_kernel",
-                4: "fused_tc2_kernel"}
+KERNEL_NAMES = {1: "fused_simt_kernel", 2: "fused_tc_kernel", 3: "fused_tc2_kernel", 4: "fused_tc2_kernel",
+                5: "fused_tc3_kernel"}
+
+
+def kernel_name(variant, w):
+    """The kernel a launch of this workload runs (variant 0: the dispatcher's choice for problems that fill the GPU)."""
+    if variant in KERNEL_NAMES:
+        return KERNEL_NAMES[variant]
+    ctas = ((w.Nq + 255) // 256) * w.B * w.H            # 256-row CTAs; the dispatcher's rule with 148 SMs
+    if w.d == 64:
+        return "fused_tc3_kernel" if 2 * ctas >= 148 else "fused_tc2_kernel"
+    return "fused_tc2_kernel" if ctas >= 148 else "fused_tc_kernel"
 
 
 def load_peaks():
@@ -43,8 +53,11 @@ def load_peaks():
 
 
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel, copied from
-# the ncu capture summarised in profiles/fused_tc2_kernel_dram_and_pipes.md (None where nothing was captured).
+# the ncu captures summarised in profiles/fused_tc3_kernel_dram_and_pipes.md and
+# profiles/fused_tc2_kernel_dram_and_pipes.md (None where nothing was captured).
 MEASURED_DRAM_TRAFFIC = {
+    ("fused_tc3_kernel", "c2_bert_large_4k"): 515_600_000,
+    ("fused_tc3_kernel", "p_4k_small"): 118_300_000,
     ("fused_tc2_kernel", "c2_bert_large_4k"): 516_000_000,
     ("fused_tc2_kernel", "p_4k_small"): 117_600_000,
     ("fused_tc2_kernel", "p_16k_d128_small"): 51_900_000,
@@ -289,13 +302,13 @@ def main():
                     "d2h_bytes_per_step": int(2 * Oh.numel())},
             "gpu_launches": launches,
             "clocks": clocks,
-            "roofline": {"bound": "tensor", "kernel": KERNEL_NAMES.get(args.variant, "fused_tc2_kernel"),
+            "roofline": {"bound": "tensor", "kernel": kernel_name(args.variant, w),
                          "achieved": achieved,
                          "peak": peaks["bf16_tflops"], "unit": UNIT, "frac": achieved / peaks["bf16_tflops"],
                          "peak_kind": "burst bf16 matmul, of " + peaks["source"],
                          "frac_of_sustained": achieved / peaks["bf16_tflops_sustained"],
                          "kernel_ms": kernel_ms, "flops_per_launch": w.flops,
-                         "traffic": load_traffic(w.name, KERNEL_NAMES.get(args.variant, "fused_tc2_kernel")),
+                         "traffic": load_traffic(w.name, kernel_name(args.variant, w)),
                          "algorithmic_bytes": w.qkvo_bytes()},
         }
         if args.with_naive and world == 1:

@@ -313,7 +313,7 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             int k_issued = 0, v_issued = 0;
             auto load_k = [&](int j) {
                 const int s = j % LY::KS;
-                ok = bounded_wait(&bars[LY::K_EMPTY + s], ((j / LY::KS) & 1) ^ 1, abort_flag, status, 0x100 + s);
+                ok = bounded_wait_s(smem_u32(&bars[LY::K_EMPTY + s]), ((j / LY::KS) & 1) ^ 1, smem_u32(const_cast<int*>(abort_flag)), status, 0x100 + s);
                 if (!ok) return;
                 mbar_arrive_expect_tx(&bars[LY::K_FULL + s], LY::KV_BYTES);
                 tma_load_3d(Ks + s * LY::KV_BYTES, &tmK, &bars[LY::K_FULL + s], 0, j * BN, bh);
@@ -321,7 +321,7 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             };
             auto load_v = [&](int j) {
                 const int s = j % LY::VS;
-                ok = bounded_wait(&bars[LY::V_EMPTY + s], ((j / LY::VS) & 1) ^ 1, abort_flag, status, 0x110 + s);
+                ok = bounded_wait_s(smem_u32(&bars[LY::V_EMPTY + s]), ((j / LY::VS) & 1) ^ 1, smem_u32(const_cast<int*>(abort_flag)), status, 0x110 + s);
                 if (!ok) return;
                 mbar_arrive_expect_tx(&bars[LY::V_FULL + s], LY::KV_BYTES);
                 tma_load_3d(Vs + s * LY::KV_BYTES, &tmV, &bars[LY::V_FULL + s], 0, j * BN, bh);
@@ -364,7 +364,7 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             const int steps = 2 * ntiles;
             bool ok = true;
             auto wait = [&](int bar, uint32_t parity, int code) {
-                if (ok) ok = __all_sync(0xffffffffu, bounded_wait(&bars[bar], parity, abort_flag, status, code));
+                if (ok) ok = __all_sync(0xffffffffu, bounded_wait_s(smem_u32(&bars[bar]), parity, smem_u32(const_cast<int*>(abort_flag)), status, code));
                 if (ok) tc_fence_after();
             };
             auto issue_s = [&](int us, int bs) {         // S(us) of tile t ^ 1 into buffer bs

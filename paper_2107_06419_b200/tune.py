@@ -3,7 +3,8 @@
 The paper explores, per workload, how many query rows a fused tile should hold (its R-granularity
 trade-off, Section 5.3: fewer rows mean more K/V re-fetches and a worse-filled compute array) and
 picks the best mapping by search (Section 6.1).  On B200 the candidates are the compiled kernel
-variants: 64-row FFMA tiles, 128-row tensor-core CTAs (one or two per SM) and 256-row CTAs.
+variants: 64-row FFMA tiles, 128-row tensor-core CTAs (one or two per SM) and 256-row CTAs
+(with one or two softmax threads per row).
 
     python -m paper_2107_06419_b200.tune [--workloads c1_bert_base_512,c2_bert_large_4k,...] [--steps 10]
 
@@ -24,6 +25,7 @@ VARIANTS = {
     api.FLAT_VARIANT_TC: "tc: 128-row CTA, exact running maximum",
     api.FLAT_VARIANT_TC2_SINGLE: "tc2_single: 128-row CTA, two per SM (d = 64)",
     api.FLAT_VARIANT_TC2: "tc2: 256-row CTA (two tiles ping-pong)",
+    api.FLAT_VARIANT_TC3: "tc3: 256-row CTA, half-row softmax threads, logits three tile-steps ahead (d = 64)",
     api.FLAT_VARIANT_AUTO: "auto (the dispatcher's choice)",
 }
 
