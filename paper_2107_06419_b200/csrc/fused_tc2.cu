@@ -152,14 +152,18 @@ __device__ __forceinline__ float exp_store(const uint32_t (&s)[128], float scale
     // The first chunk's weights are held in registers until the second chunk is done:
     // `before_first_store` (the wait for the P buffer to be free) then runs with a third of the
     // row already computed, late enough for the previous tile's O += P V to have finished.
-    float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
+    // Scale/shift and the row sums run on packed pairs (fma / add .f32x2: half the issue slots).
+    uint64_t lsum0 = 0ull, lsum1 = 0ull;             // (l0, l1) and (l2, l3)
+    const uint64_t scale2 = pack2(scale_log2e, scale_log2e), neg_m2 = pack2(neg_m, neg_m);
     uint32_t pk0[16];
 #pragma unroll
     for (int c = 0; c < 4; ++c) {
         uint32_t pk[16];
         float p[32];
 #pragma unroll
-        for (int i = 0; i < 32; ++i) p[i] = fmaf(__uint_as_float(s[c * 32 + i]), scale_log2e, neg_m);
+        for (int i = 0; i < 32; i += 2)
+            unpack2(fma2(pack2(__uint_as_float(s[c * 32 + i]), __uint_as_float(s[c * 32 + i + 1])), scale2, neg_m2),
+                    p[i], p[i + 1]);
 #pragma unroll
         for (int i = 0; i < 32; ++i) {
             // One element in four takes the polynomial route (FMA pipe) to unload the ex2 unit,
@@ -172,7 +176,8 @@ __device__ __forceinline__ float exp_store(const uint32_t (&s)[128], float scale
         if (c == PASS_AT_CHUNK) after_last_exp();       // (nearly) every ex2 of the row has been issued
 #pragma unroll
         for (int i = 0; i < 32; i += 4) {
-            l0 += p[i]; l1 += p[i + 1]; l2 += p[i + 2]; l3 += p[i + 3];
+            lsum0 = add2(lsum0, pack2(p[i], p[i + 1]));
+            lsum1 = add2(lsum1, pack2(p[i + 2], p[i + 3]));
             pk[i / 2] = pack_bf16x2(p[i], p[i + 1]);
             pk[i / 2 + 1] = pack_bf16x2(p[i + 2], p[i + 3]);
         }
@@ -187,6 +192,9 @@ __device__ __forceinline__ float exp_store(const uint32_t (&s)[128], float scale
         if (trace_row != nullptr && (threadIdx.x & 127) == 0) trace_row[8 + c] = static_cast<unsigned>(clock64());
 #endif
     }
+    float l0, l1, l2, l3;
+    unpack2(lsum0, l0, l1);
+    unpack2(lsum1, l2, l3);
     return (l0 + l1) + (l2 + l3);
 }
 

@@ -171,26 +171,6 @@ __device__ __forceinline__ bool pair_any(int id, bool flag) {
     return r != 0;
 }
 
-// Two fp32 values in one 64-bit register pair, for the packed fp32 instructions of sm_100
-// (fma / add / sub .f32x2: two results per issue slot).
-__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
-    uint64_t v;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(v) : "f"(lo), "f"(hi));
-    return v;
-}
-__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
-    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
-}
-__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
-    uint64_t d;
-    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
-    return d;
-}
-__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
-    uint64_t d;
-    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-    return d;
-}
 // ex2_poly (see tc_common.cuh) without the upper clamp: the caller keeps the maximum of the
 // arguments and treats one above 126 as an overflow of the row.  Scalar on purpose: the constants
 // ride along as immediates, where packed instructions would want them in registers.
@@ -284,6 +264,9 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
 #endif
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+#ifdef FLAT_TRACE3
+    const unsigned t_entry = static_cast<unsigned>(clock64());
+#endif
     const int bh = blockIdx.y;
     const int row0 = blockIdx.x * (2 * BM);
     int n = Nk;
@@ -296,21 +279,38 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                                 : (i >= LY::K_EMPTY && i < LY::V_FULL) || (i >= LY::V_EMPTY && i < LY::S_FULL) ? 2 : 1);   // K/V_EMPTY: both issuers
         *abort_flag = 0;
         fence_mbar_init();
+        // This thread is the TMA producer: the first tiles leave at once, before the CTA-wide
+        // synchronisation and the TMEM allocation (their stages are free and need no wait).
+        if (ntiles > 0) {
+            prefetch_tensormap(&tmQ); prefetch_tensormap(&tmK); prefetch_tensormap(&tmV);
+            mbar_arrive_expect_tx(&bars[LY::Q_FULL + 0], LY::Q_BYTES);
+            tma_load_3d(Qs, &tmQ, &bars[LY::Q_FULL + 0], 0, row0, bh);
+            mbar_arrive_expect_tx(&bars[LY::K_FULL + 0], LY::KV_BYTES);
+            tma_load_3d(Ks, &tmK, &bars[LY::K_FULL + 0], 0, 0, bh);
+            mbar_arrive_expect_tx(&bars[LY::Q_FULL + 1], LY::Q_BYTES);
+            tma_load_3d(Qs + LY::Q_BYTES, &tmQ, &bars[LY::Q_FULL + 1], 0, row0 + BM, bh);
+            if (ntiles > 1) {
+                mbar_arrive_expect_tx(&bars[LY::K_FULL + 1], LY::KV_BYTES);
+                tma_load_3d(Ks + LY::KV_BYTES, &tmK, &bars[LY::K_FULL + 1], 0, BN, bh);
+            }
+        }
     }
     if (warp == 0) { tmem_alloc(tmem_slot, LY::TMEM_COLS); tmem_relinquish(); }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
+#ifdef FLAT_TRACE3
+    if (threadIdx.x == 0) { trace_buf[(5 * 64) * 16 + 0] = t_entry; TRACE(5, 0, 1); }
+#endif
 
     if (warp >= LY::SOFT_WARPS) {
       asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(OTHER_REGS));
       if (warp == LY::SOFT_WARPS) {
         // ------------------------------------------------------------ TMA producer
         if (lane == 0 && ntiles > 0) {
-            prefetch_tensormap(&tmQ); prefetch_tensormap(&tmK); prefetch_tensormap(&tmV);
             bool ok = true;
-            int k_issued = 0, v_issued = 0;
+            int k_issued = ntiles > 1 ? 2 : 1, v_issued = 0;     // Q_A, K_0, Q_B, K_1 left before the CTA synchronised
             auto load_k = [&](int j) {
                 const int s = j % LY::KS;
                 ok = bounded_wait_s(smem_u32(&bars[LY::K_EMPTY + s]), ((j / LY::KS) & 1) ^ 1, smem_u32(const_cast<int*>(abort_flag)), status, 0x100 + s);
@@ -327,12 +327,6 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                 tma_load_3d(Vs + s * LY::KV_BYTES, &tmV, &bars[LY::V_FULL + s], 0, j * BN, bh);
                 v_issued = j + 1;
             };
-            mbar_arrive_expect_tx(&bars[LY::Q_FULL + 0], LY::Q_BYTES);
-            tma_load_3d(Qs, &tmQ, &bars[LY::Q_FULL + 0], 0, row0, bh);
-            load_k(0);
-            mbar_arrive_expect_tx(&bars[LY::Q_FULL + 1], LY::Q_BYTES);
-            tma_load_3d(Qs + LY::Q_BYTES, &tmQ, &bars[LY::Q_FULL + 1], 0, row0 + BM, bh);
-            if (ntiles > 1) load_k(1);
             // S runs ahead of P V: K_{j+2} is wanted before V_{j+1}
             for (int j = 0; j < ntiles && ok; ++j) {
                 load_v(j);
@@ -535,13 +529,34 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                     }
                     m_ref = m_new;
                 }
+                // the logits are read again, 32 at a time; with the fresh maximum every argument is <= 0,
+                // so the ordinary routine (polynomial lanes included) applies unless part of the half is masked
                 ls[0] = ls[1] = ls[2] = ls[3] = 0.f;
+                if (tail) {
 #pragma unroll
-                for (int c = 0; c < 2; ++c) {            // the logits are read again, 32 at a time
-                    uint32_t r[32];
-                    tmem_ld_x32(s_addr + c * 32, r);
-                    tc_wait_ld();
-                    exp_pack32<true, false>(r, scale_log2e, -m_ref, nvalid - c * 32, ls, pk[c]);
+                    for (int c = 0; c < 2; ++c) {
+                        uint32_t r[32];
+                        tmem_ld_x32(s_addr + c * 32, r);
+                        tc_wait_ld();
+                        exp_pack32<true, false>(r, scale_log2e, -m_ref, nvalid - c * 32, ls, pk[c]);
+                    }
+                } else {
+                    const uint64_t scale2 = pack2(scale_log2e, scale_log2e), neg_m2 = pack2(-m_ref, -m_ref);
+                    uint64_t l2[2] = {0ull, 0ull};
+                    float xmax = 0.f;
+#pragma unroll
+                    for (int c = 0; c < 2; ++c) {
+                        uint32_t r[32];
+                        uint64_t x2[16];
+                        tmem_ld_x32(s_addr + c * 32, r);
+                        tc_wait_ld();
+                        scale32(r, scale2, neg_m2, x2);
+                        exp_pack_x2<FLAT_TC3_POLY>(x2, l2, xmax, pk[c]);
+                    }
+                    float a, b2, c2, d2;
+                    unpack2(l2[0], a, b2);
+                    unpack2(l2[1], c2, d2);
+                    ls[0] = (a + b2) + (c2 + d2);
                 }
             }
             // a failed wait is voted on so that the two warps leave the loop together (only the
@@ -598,10 +613,14 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             }
         }
     }
+#ifdef FLAT_TRACE3
+    if (threadIdx.x == 0) TRACE(5, 0, 2);
+#endif
     tc_fence_before();
     __syncthreads();
     if (warp == 0) tmem_dealloc(tmem, LY::TMEM_COLS);
 #ifdef FLAT_TRACE3
+    if (threadIdx.x == 0) TRACE(5, 0, 3);
     if (g_trace3 && blockIdx.x == 0 && blockIdx.y == 0)
         for (int i = threadIdx.x; i < TRACE3_WORDS; i += LY::THREADS) g_trace3[i] = trace_buf[i];
 #endif
