@@ -104,7 +104,8 @@ struct L3 {
     // PV_DONE, and a tile's softmax warps can be at most two key steps apart, so a waiter never finds
     // one of these barriers more than one phase ahead of the phase it asks for (parity waits are safe).
     static constexpr int S_FULL = V_EMPTY + VS, P_FULL = S_FULL + 6, PV_DONE = P_FULL + 6;
-    static constexpr int NUM_BARS = PV_DONE + 6;
+    static constexpr int Q_EMPTY = PV_DONE + 6;          // [2] the item's logit MMAs are done with the Q tile
+    static constexpr int NUM_BARS = Q_EMPTY + 2;
 };
 
 __device__ __forceinline__ float max3(float a, float b, float c) {
@@ -244,10 +245,58 @@ __device__ __forceinline__ void exp_pack32(const uint32_t (&r)[32], float scale_
     }
 }
 
+// One work item = (batch, head, slab of 256 query rows).  A CTA takes the items blockIdx.x,
+// blockIdx.x + gridDim.x, ... one after the other without draining its pipeline in between.
+struct Item {
+    int bh, row0, n, ntiles;                             // n = number of valid keys, ntiles = key steps
+};
+__device__ __forceinline__ Item get_item(int idx, int slabs, int H, int Nk, const int32_t* __restrict__ valid_len) {
+    Item it;
+    it.bh = idx / slabs;
+    it.row0 = (idx - it.bh * slabs) * (2 * BM);
+    int n = Nk;
+    if (valid_len) { n = valid_len[it.bh / H]; n = n < 0 ? 0 : (n > Nk ? Nk : n); }
+    it.n = n;
+    it.ntiles = (n + BN - 1) / BN;
+    return it;
+}
+// Position of a role in the CTA's sequence of key steps.  Items without a valid key have no steps
+// and are skipped (their rows are written as zeros by the softmax warps).  J counts the key steps
+// of all items so far: the rings, the buffers and the barrier phases are indexed with it, so the
+// pipeline runs on across item boundaries; q counts the items that had steps (phase of the Q tiles).
+struct Cursor {
+    int idx, j, J, q;
+    Item it;
+    bool valid;
+};
+__device__ __forceinline__ void cursor_seek(Cursor& c, int items, int slabs, int H, int Nk,
+                                            const int32_t* __restrict__ valid_len) {
+    c.valid = false;
+    while (c.idx < items) {
+        c.it = get_item(c.idx, slabs, H, Nk, valid_len);
+        if (c.it.ntiles > 0) { c.valid = true; return; }
+        c.idx += gridDim.x;
+    }
+}
+__device__ __forceinline__ void cursor_init(Cursor& c, int items, int slabs, int H, int Nk,
+                                            const int32_t* __restrict__ valid_len) {
+    c.idx = blockIdx.x; c.j = 0; c.J = 0; c.q = 0;
+    cursor_seek(c, items, slabs, H, Nk, valid_len);
+}
+__device__ __forceinline__ void cursor_next(Cursor& c, int items, int slabs, int H, int Nk,
+                                            const int32_t* __restrict__ valid_len) {
+    ++c.j; ++c.J;
+    if (c.j == c.it.ntiles) {
+        c.j = 0; ++c.q;
+        c.idx += gridDim.x;
+        cursor_seek(c, items, slabs, H, Nk, valid_len);
+    }
+}
+
 __global__ void __launch_bounds__(L3::THREADS, 1)
 fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                  const __grid_constant__ CUtensorMap tmV, __nv_bfloat16* __restrict__ O, int H, int Nq, int Nk,
-                 float scale_log2e, const int32_t* __restrict__ valid_len, int32_t* status) {
+                 int items, int slabs, float scale_log2e, const int32_t* __restrict__ valid_len, int32_t* status) {
     using LY = L3;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -267,11 +316,6 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
 #ifdef FLAT_TRACE3
     const unsigned t_entry = static_cast<unsigned>(clock64());
 #endif
-    const int bh = blockIdx.y;
-    const int row0 = blockIdx.x * (2 * BM);
-    int n = Nk;
-    if (valid_len) { n = valid_len[bh / H]; n = n < 0 ? 0 : (n > Nk ? Nk : n); }
-    const int ntiles = (n + BN - 1) / BN;
 
     if (threadIdx.x == LY::SOFT_WARPS * 32) {
         for (int i = 0; i < LY::NUM_BARS; ++i)
@@ -279,21 +323,6 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                                 : (i >= LY::K_EMPTY && i < LY::V_FULL) || (i >= LY::V_EMPTY && i < LY::S_FULL) ? 2 : 1);   // K/V_EMPTY: both issuers
         *abort_flag = 0;
         fence_mbar_init();
-        // This thread is the TMA producer: the first tiles leave at once, before the CTA-wide
-        // synchronisation and the TMEM allocation (their stages are free and need no wait).
-        if (ntiles > 0) {
-            prefetch_tensormap(&tmQ); prefetch_tensormap(&tmK); prefetch_tensormap(&tmV);
-            mbar_arrive_expect_tx(&bars[LY::Q_FULL + 0], LY::Q_BYTES);
-            tma_load_3d(Qs, &tmQ, &bars[LY::Q_FULL + 0], 0, row0, bh);
-            mbar_arrive_expect_tx(&bars[LY::K_FULL + 0], LY::KV_BYTES);
-            tma_load_3d(Ks, &tmK, &bars[LY::K_FULL + 0], 0, 0, bh);
-            mbar_arrive_expect_tx(&bars[LY::Q_FULL + 1], LY::Q_BYTES);
-            tma_load_3d(Qs + LY::Q_BYTES, &tmQ, &bars[LY::Q_FULL + 1], 0, row0 + BM, bh);
-            if (ntiles > 1) {
-                mbar_arrive_expect_tx(&bars[LY::K_FULL + 1], LY::KV_BYTES);
-                tma_load_3d(Ks + LY::KV_BYTES, &tmK, &bars[LY::K_FULL + 1], 0, BN, bh);
-            }
-        }
     }
     if (warp == 0) { tmem_alloc(tmem_slot, LY::TMEM_COLS); tmem_relinquish(); }
     tc_fence_before();
@@ -306,104 +335,128 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
 
     if (warp >= LY::SOFT_WARPS) {
       asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(OTHER_REGS));
+      const uint32_t bars_s = smem_u32(bars), abort_s = smem_u32(const_cast<int*>(abort_flag));
       if (warp == LY::SOFT_WARPS) {
         // ------------------------------------------------------------ TMA producer
-        if (lane == 0 && ntiles > 0) {
+        // Per item: Q_A, K_0, Q_B, K_1, then V_j and K_{j+2} in turn (S runs ahead of P V, so K_{j+2} is
+        // wanted before V_{j+1}).  The rings are indexed with the global key step J.
+        if (lane == 0) {
+            prefetch_tensormap(&tmQ); prefetch_tensormap(&tmK); prefetch_tensormap(&tmV);
             bool ok = true;
-            int k_issued = ntiles > 1 ? 2 : 1, v_issued = 0;     // Q_A, K_0, Q_B, K_1 left before the CTA synchronised
-            auto load_k = [&](int j) {
-                const int s = j % LY::KS;
-                ok = bounded_wait_s(smem_u32(&bars[LY::K_EMPTY + s]), ((j / LY::KS) & 1) ^ 1, smem_u32(const_cast<int*>(abort_flag)), status, 0x100 + s);
+            int q_loaded[2] = {0, 0}, k_issued = 0, v_issued = 0;    // (for the drain after a failed wait)
+            auto load_q = [&](int t, int q, int row, int bh) {
+                // the logit MMAs of the previous item must have finished with this tile of shared memory
+                if (q > 0) ok = bounded_wait_s(bars_s + 8 * (LY::Q_EMPTY + t), (q - 1) & 1, abort_s, status, 0x120 + t);
+                if (!ok) return;
+                mbar_arrive_expect_tx(&bars[LY::Q_FULL + t], LY::Q_BYTES);
+                tma_load_3d(Qs + t * LY::Q_BYTES, &tmQ, &bars[LY::Q_FULL + t], 0, row, bh);
+                q_loaded[t] = q + 1;
+            };
+            auto load_k = [&](int J, int j, int bh) {
+                const int s = J % LY::KS;
+                ok = bounded_wait_s(bars_s + 8 * (LY::K_EMPTY + s), ((J / LY::KS) & 1) ^ 1, abort_s, status, 0x100 + s);
                 if (!ok) return;
                 mbar_arrive_expect_tx(&bars[LY::K_FULL + s], LY::KV_BYTES);
                 tma_load_3d(Ks + s * LY::KV_BYTES, &tmK, &bars[LY::K_FULL + s], 0, j * BN, bh);
-                k_issued = j + 1;
+                k_issued = J + 1;
             };
-            auto load_v = [&](int j) {
-                const int s = j % LY::VS;
-                ok = bounded_wait_s(smem_u32(&bars[LY::V_EMPTY + s]), ((j / LY::VS) & 1) ^ 1, smem_u32(const_cast<int*>(abort_flag)), status, 0x110 + s);
+            auto load_v = [&](int J, int j, int bh) {
+                const int s = J % LY::VS;
+                ok = bounded_wait_s(bars_s + 8 * (LY::V_EMPTY + s), ((J / LY::VS) & 1) ^ 1, abort_s, status, 0x110 + s);
                 if (!ok) return;
                 mbar_arrive_expect_tx(&bars[LY::V_FULL + s], LY::KV_BYTES);
                 tma_load_3d(Vs + s * LY::KV_BYTES, &tmV, &bars[LY::V_FULL + s], 0, j * BN, bh);
-                v_issued = j + 1;
+                v_issued = J + 1;
             };
-            // S runs ahead of P V: K_{j+2} is wanted before V_{j+1}
-            for (int j = 0; j < ntiles && ok; ++j) {
-                load_v(j);
-                if (ok && j + 2 < ntiles) load_k(j + 2);
+            int J0 = 0, q = 0;
+            for (int idx = blockIdx.x; idx < items && ok; idx += gridDim.x) {
+                const Item it = get_item(idx, slabs, H, Nk, valid_len);
+                if (it.ntiles == 0) continue;
+                load_q(0, q, it.row0, it.bh);
+                if (ok) load_k(J0, 0, it.bh);
+                if (ok) load_q(1, q, it.row0 + BM, it.bh);
+                if (ok && it.ntiles > 1) load_k(J0 + 1, 1, it.bh);
+                for (int j = 0; j < it.ntiles && ok; ++j) {
+                    load_v(J0 + j, j, it.bh);
+                    if (ok && j + 2 < it.ntiles) load_k(J0 + j + 2, j + 2, it.bh);
+                }
+                J0 += it.ntiles;
+                ++q;
             }
             if (!ok) {
-                drain_wait(&bars[LY::Q_FULL + 0], 0);
-                drain_wait(&bars[LY::Q_FULL + 1], 0);
-                for (int j = k_issued > LY::KS ? k_issued - LY::KS : 0; j < k_issued; ++j)
-                    drain_wait(&bars[LY::K_FULL + j % LY::KS], (j / LY::KS) & 1);
-                for (int j = v_issued > LY::VS ? v_issued - LY::VS : 0; j < v_issued; ++j)
-                    drain_wait(&bars[LY::V_FULL + j % LY::VS], (j / LY::VS) & 1);
+                for (int t = 0; t < 2; ++t)
+                    if (q_loaded[t] > 0) drain_wait(&bars[LY::Q_FULL + t], (q_loaded[t] - 1) & 1);
+                for (int J = k_issued > LY::KS ? k_issued - LY::KS : 0; J < k_issued; ++J)
+                    drain_wait(&bars[LY::K_FULL + J % LY::KS], (J / LY::KS) & 1);
+                for (int J = v_issued > LY::VS ? v_issued - LY::VS : 0; J < v_issued; ++J)
+                    drain_wait(&bars[LY::V_FULL + J % LY::VS], (J / LY::VS) & 1);
             }
         }
-      } else {
+      } else if (warp <= LY::SOFT_WARPS + 2) {
         // ------------------------------------------------------------ MMA issuers
-        // Warp 17 / 18 serves the tile-steps u of tile A / B: O_t += P(u) V, then, into the buffer
-        // that these MMAs have just read (same thread: the tensor pipe keeps the order), the logits
-        // S(u + 3) of the OTHER tile.  A whole warp runs the loop (uniform control flow); one elected
-        // lane issues.  Tile-step u: tile u & 1, key step u >> 1, buffer u % 3.
-        if (ntiles > 0 && warp <= LY::SOFT_WARPS + 2) {
-            constexpr uint32_t IDESC_S = make_idesc_bf16(BM, BN, 0, 0);
-            constexpr uint32_t IDESC_PV = make_idesc_bf16(BM, D, 0, 1);
-            const int t = warp - LY::SOFT_WARPS - 1;
-            // logits are always those of the other tile
-            const uint64_t q_desc = make_smem_desc_sw128(smem_u32(Qs) + (t ^ 1) * LY::Q_BYTES, 16, 1024);
-            const uint64_t k_desc = make_smem_desc_sw128(smem_u32(Ks), 16, 1024);
-            const uint64_t v_desc = make_smem_desc_sw128(smem_u32(Vs), BN * 128, 1024);
-            const int steps = 2 * ntiles;
-            bool ok = true;
-            auto wait = [&](int bar, uint32_t parity, int code) {
-                if (ok) ok = __all_sync(0xffffffffu, bounded_wait_s(smem_u32(&bars[bar]), parity, smem_u32(const_cast<int*>(abort_flag)), status, code));
-                if (ok) tc_fence_after();
-            };
-            auto issue_s = [&](int us, int bs) {         // S(us) of tile t ^ 1 into buffer bs
-                const int js = us >> 1, ks = js % LY::KS;
-                if (js == 0) wait(LY::Q_FULL + (t ^ 1), 0, 0x200 + t);
-                wait(LY::K_FULL + ks, (js / LY::KS) & 1, 0x210);
-                if (!ok) return;
-                if (elect_one()) {
-                    const uint64_t kd = k_desc + static_cast<uint64_t>((ks * LY::KV_BYTES) >> 4);
+        // Warp 17 / 18 serves the tile-steps of tile A / B: O_t += P(g) V, then, into the buffer that
+        // these MMAs have just read (same thread: the tensor pipe keeps the order), the logits S(g + 3)
+        // of the OTHER tile.  A whole warp runs the loop (uniform control flow); one elected lane
+        // issues.  Tile-step g = 2 J + tile (J: global key step), buffer g % 3, barrier phase g / 6.
+        constexpr uint32_t IDESC_S = make_idesc_bf16(BM, BN, 0, 0);
+        constexpr uint32_t IDESC_PV = make_idesc_bf16(BM, D, 0, 1);
+        const int t = warp - LY::SOFT_WARPS - 1, ts = t ^ 1;     // ts: the tile whose logits this warp issues
+        const uint64_t q_desc = make_smem_desc_sw128(smem_u32(Qs) + ts * LY::Q_BYTES, 16, 1024);
+        const uint64_t k_desc = make_smem_desc_sw128(smem_u32(Ks), 16, 1024);
+        const uint64_t v_desc = make_smem_desc_sw128(smem_u32(Vs), BN * 128, 1024);
+        bool ok = true;
+        auto wait = [&](int bar, uint32_t parity, int code) {
+            if (ok) ok = __all_sync(0xffffffffu, bounded_wait_s(bars_s + 8 * bar, parity, abort_s, status, code));
+            if (ok) tc_fence_after();
+        };
+        Cursor cs, cp;                                   // where the logits / the O += P V of this warp stand
+        cursor_init(cs, items, slabs, H, Nk, valid_len);
+        cursor_init(cp, items, slabs, H, Nk, valid_len);
+        auto issue_s = [&]() {                           // S of tile ts at cursor cs, then advance it
+            if (!cs.valid || !ok) return;
+            const int g = 2 * cs.J + ts, bs = g % 3, ks = cs.J % LY::KS;
+            if (cs.j == 0) wait(LY::Q_FULL + ts, cs.q & 1, 0x200 + t);
+            wait(LY::K_FULL + ks, (cs.J / LY::KS) & 1, 0x210);
+            if (!ok) return;
+            if (elect_one()) {
+                const uint64_t kd = k_desc + static_cast<uint64_t>((ks * LY::KV_BYTES) >> 4);
 #pragma unroll
-                    for (int k = 0; k < D / 16; ++k)
-                        mma_ss(tmem + LY::X_COL(bs), q_desc + static_cast<uint64_t>((k * 32) >> 4),
-                               kd + static_cast<uint64_t>((k * 32) >> 4), IDESC_S, k > 0);
-                    tc_commit(&bars[LY::S_FULL + (t ^ 1) * 3 + bs]);
-                    tc_commit(&bars[LY::K_EMPTY + ks]);   // (counts 2: both tiles' logits have used K_j)
-                    TRACE(4, us, 1);
-                }
-                __syncwarp();
-            };
-            // the first three logit tiles need no buffer to be freed: S(0), S(2) (tile A) come from
-            // tile B's issuer, S(1) from tile A's
-            if (t == 1) { issue_s(0, 0); if (steps > 2) issue_s(2, 2); }
-            else issue_s(1, 1);
-            int b = t;
-            for (int j = 0; j < ntiles && ok; ++j, b = (b == 0 ? 2 : b - 1)) {
-                const int u = 2 * j + t, vs = j % LY::VS;
-                if (lane == 0) TRACE(4, u, 0);
-                wait(LY::V_FULL + vs, (j / LY::VS) & 1, 0x220);
-                wait(LY::P_FULL + t * 3 + b, (u / 6) & 1, 0x221);
-                if (lane == 0) TRACE(4, u, 2);
-                if (!ok) break;
-                if (elect_one()) {
-                    const uint64_t vd = v_desc + static_cast<uint64_t>((vs * LY::KV_BYTES) >> 4);
-                    // the two halves of P(u) overlay the first 32 columns of each half of S(u)
-#pragma unroll
-                    for (int k = 0; k < BN / 16; ++k)
-                        mma_ts(tmem + LY::O_COL(t), tmem + LY::X_COL(b) + (k / 4) * HN + (k % 4) * 8,
-                               vd + static_cast<uint64_t>((k * 2048) >> 4), IDESC_PV, (j > 0 || k > 0));
-                    tc_commit(&bars[LY::PV_DONE + t * 3 + b]);
-                    tc_commit(&bars[LY::V_EMPTY + vs]);
-                    TRACE(4, u, 3);
-                }
-                __syncwarp();
-                if (u + 3 < steps) issue_s(u + 3, b);
+                for (int k = 0; k < D / 16; ++k)
+                    mma_ss(tmem + LY::X_COL(bs), q_desc + static_cast<uint64_t>((k * 32) >> 4),
+                           kd + static_cast<uint64_t>((k * 32) >> 4), IDESC_S, k > 0);
+                tc_commit(&bars[LY::S_FULL + ts * 3 + bs]);
+                tc_commit(&bars[LY::K_EMPTY + ks]);       // (counts 2: both tiles' logits have used K_j)
+                if (cs.j == cs.it.ntiles - 1) tc_commit(&bars[LY::Q_EMPTY + ts]);   // the item's last use of Q_ts
+                TRACE(4, g, 1);
             }
+            __syncwarp();
+            cursor_next(cs, items, slabs, H, Nk, valid_len);
+        };
+        // the first three logit tiles need no buffer to be freed: S(0), S(2) (tile A, key steps 0 and 1)
+        // come from tile B's issuer, S(1) (tile B, key step 0) from tile A's
+        issue_s();
+        if (t == 1) issue_s();
+        while (cp.valid && ok) {
+            const int g = 2 * cp.J + t, b = g % 3, vs = cp.J % LY::VS;
+            if (lane == 0) TRACE(4, g, 0);
+            wait(LY::V_FULL + vs, (cp.J / LY::VS) & 1, 0x220);
+            wait(LY::P_FULL + t * 3 + b, (g / 6) & 1, 0x221);
+            if (lane == 0) TRACE(4, g, 2);
+            if (!ok) break;
+            if (elect_one()) {
+                const uint64_t vd = v_desc + static_cast<uint64_t>((vs * LY::KV_BYTES) >> 4);
+                // the two halves of P(g) overlay the first 32 columns of each half of S(g)
+#pragma unroll
+                for (int k = 0; k < BN / 16; ++k)
+                    mma_ts(tmem + LY::O_COL(t), tmem + LY::X_COL(b) + (k / 4) * HN + (k % 4) * 8,
+                           vd + static_cast<uint64_t>((k * 2048) >> 4), IDESC_PV, (cp.j > 0 || k > 0));
+                tc_commit(&bars[LY::PV_DONE + t * 3 + b]);
+                tc_commit(&bars[LY::V_EMPTY + vs]);
+                TRACE(4, g, 3);
+            }
+            __syncwarp();
+            cursor_next(cp, items, slabs, H, Nk, valid_len);
+            issue_s();                                   // into buffer b: 2 J_s + ts = g + 3
         }
       }
     } else {
@@ -412,7 +465,6 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         const int q = warp & 3;                          // row group = TMEM lane quarter
         const int t = warp >> 3;                         // query tile
         const int h = (warp >> 2) & 1;                   // key half of every step
-        const int row = row0 + t * BM + q * 32 + lane;
         const uint32_t tl = tmem + (static_cast<uint32_t>(q * 32) << 16);
         const int pair_id = 1 + t * 4 + q;               // named barrier of the two warps sharing these rows
         // shared-window addresses: the barriers, the abort flag, and this thread's slot for exchanged
@@ -420,16 +472,20 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         const uint32_t bars_s = smem_u32(bars), abort_s = smem_u32(const_cast<int*>(abort_flag));
         const uint32_t xm_own = smem_u32(xch + ((t * 2 + h) * BM + q * 32 + lane));
         const bool neg_scale = scale_log2e < 0.f;
-        float m_ref = -INFINITY, l = 0.f;
         bool ok = true;
         const int trole = t * 2 + h;
         (void)trole;
-        int b = t;                                       // buffer of tile-step u = 2 j + t: u % 3
-        for (int j = 0; j < ntiles; ++j, b = (b == 0 ? 2 : b - 1)) {      // u += 2  <=>  b -= 1 (mod 3)
-            // this warp's 64 logits of S(u); its 32 packed columns of P(u) go over the first half of them
+        int b = t;                                       // buffer of tile-step g = 2 J + t: g % 3
+        int g = t;                                       // this tile's next tile-step (J: key steps of all items so far)
+        for (int idx = blockIdx.x; idx < items; idx += gridDim.x) {
+        const Item it = get_item(idx, slabs, H, Nk, valid_len);
+        const int n = it.n, ntiles = it.ntiles;
+        float m_ref = -INFINITY, l = 0.f;
+        for (int j = 0; j < ntiles; ++j, g += 2, b = (b == 0 ? 2 : b - 1)) {      // g += 2  <=>  b -= 1 (mod 3)
+            // this warp's 64 logits of S(g); its 32 packed columns of P(g) go over the first half of them
             const uint32_t s_addr = tl + LY::X_COL(b) + h * HN;
             if (q == 0 && lane == 0) TRACE(trole, j, 0);
-            const uint32_t xph = static_cast<uint32_t>((2 * j + t) / 6) & 1u;   // phase parity of this tile's use of the buffer
+            const uint32_t xph = static_cast<uint32_t>(g / 6) & 1u;   // phase parity of this tile's use of the buffer
             ok = bounded_wait_s(bars_s + 8 * (LY::S_FULL + t * 3 + b), xph, abort_s, status, 0x300 + t);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
@@ -508,8 +564,8 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                     l *= alpha;
                     if (j > 0) {
                         // each half rescales its half of the columns of O_t
-                        // (O_t += P(u - 2) V must be complete; that tile-step used buffer b + 1 mod 3)
-                        const int u2 = 2 * j + t - 2;
+                        // (O_t += P(g - 2) V must be complete; that tile-step used buffer b + 1 mod 3)
+                        const int u2 = g - 2;
                         ok = __all_sync(0xffffffffu,
                                         bounded_wait_s(bars_s + 8 * (LY::PV_DONE + t * 3 + (b == 2 ? 0 : b + 1)),
                                                        static_cast<uint32_t>(u2 / 6) & 1u, abort_s, status, 0x310 + t));
@@ -575,20 +631,22 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             if (lane == 0) TRACE(trole, j, 8 + q);
         }
         if (ok && ntiles > 0) {
-            // the last O_t += P V (the issuer's MMAs complete in order)
-            const int ul = 2 * (ntiles - 1) + t;
-            ok = bounded_wait_s(bars_s + 8 * (LY::PV_DONE + t * 3 + ul % 3), static_cast<uint32_t>(ul / 6) & 1u, abort_s,
-                                status, 0x330 + t);
+            // the last O_t += P V of the item (the issuer's MMAs complete in order)
+            const int ul = g - 2;
+            ok = bounded_wait_s(bars_s + 8 * (LY::PV_DONE + t * 3 + (b == 2 ? 0 : b + 1)), static_cast<uint32_t>(ul / 6) & 1u,
+                                abort_s, status, 0x330 + t);
             ok = __all_sync(0xffffffffu, ok);
         }
-        // row sum of both halves (a warp that gave up still takes part, so that its partner is not left waiting)
+        // The two warps of a row leave together if either gave up; otherwise they add up their row sums.
+        if (pair_any(pair_id, !ok)) { ok = false; break; }
         st_shared_f32(xm_own + 4 * BM * 4, l);
         pair_sync(pair_id);
         l += ld_shared_f32((xm_own ^ (BM * 4)) + 4 * BM * 4);
-        if (ok) {
+        {
+            const int row = it.row0 + t * BM + q * 32 + lane;
             const float inv = l > 0.f ? 1.f / l : 0.f;
             tc_fence_after();
-            __nv_bfloat16* orow = O + (static_cast<int64_t>(bh) * Nq + row) * D + h * (D / 2);
+            __nv_bfloat16* orow = O + (static_cast<int64_t>(it.bh) * Nq + row) * D + h * (D / 2);
 #pragma unroll
             for (int c = 0; c < D / 64; ++c) {
                 uint32_t r[32];
@@ -611,6 +669,10 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                     }
                 }
             }
+            // (the reads of O_t above are complete -- tcgen05.wait::ld -- before this warp's next P_FULL
+            // arrival, which the first, overwriting O_t = P V of the next item waits for)
+            tc_fence_before();
+        }
         }
     }
 #ifdef FLAT_TRACE3
@@ -634,10 +696,15 @@ int launch_tc3(const Problem& p, cudaStream_t st) {
         !make_map(&tmV, p.V, BH, p.Nk, D, BN))
         return FLAT_ERR_CUDA;
     if (!ensure_dynamic_smem<fused_tc3_kernel>(LY::SMEM_BYTES)) return FLAT_ERR_CUDA;
-    dim3 grid((p.Nq + 2 * BM - 1) / (2 * BM), BH);
+    // One CTA per SM at most; each walks over its share of the (head, 256-row slab) items, slabs of
+    // a head next to each other so that CTAs running at the same time share K and V in L2.
+    const int slabs = (p.Nq + 2 * BM - 1) / (2 * BM);
+    const int64_t items = static_cast<int64_t>(slabs) * BH;
+    const int sms = device_sm_count();
+    const int grid = static_cast<int>(items < sms ? items : sms);
     fused_tc3_kernel<<<grid, LY::THREADS, LY::SMEM_BYTES, st>>>(tmQ, tmK, tmV, static_cast<__nv_bfloat16*>(p.O), p.H,
-                                                                p.Nq, p.Nk, p.scale * 1.4426950408889634f,
-                                                                p.k_valid_len, p.status);
+                                                                p.Nq, p.Nk, static_cast<int>(items), slabs,
+                                                                p.scale * 1.4426950408889634f, p.k_valid_len, p.status);
     return cudaGetLastError() == cudaSuccess ? FLAT_OK : FLAT_ERR_CUDA;
 }
 
