@@ -94,6 +94,25 @@ def test_fused_bf16_planted_keys(api, variant):
     check_bf16(got, ref["O"], "planted v%d" % variant)
 
 
+@pytest.mark.parametrize("variant", [0, 5], ids=["auto", "tc3"])
+def test_many_items_per_cta(api, variant):
+    """More (head, row-slab) work items than SMs, so the persistent CTAs of the d = 64 kernel take several
+    items each, one behind the other: ragged query slabs, per-batch key counts that differ between
+    neighbouring items (including 0 and 1), and rows whose maximum keeps rising (peaked logits), so that
+    the redo path also runs right before and after an item boundary."""
+    B, H, Nq, Nk, d = 24, 8, 300, 333, 64                   # 192 heads x 2 slabs = 384 items
+    rng = np.random.default_rng(1234)
+    Qb, Kb, Vb = rand_bits(rng, (B, H, Nq, d), 1.5), rand_bits(rng, (B, H, Nk, d), 1.5), rand_bits(rng, (B, H, Nk, d))
+    vl = rng.integers(1, Nk + 1, size=B).astype(np.int32)
+    vl[[0, 5, 11]] = [0, 1, Nk]
+    vl[7], vl[8], vl[9] = 128, 129, 256                      # tile edges
+    scale = 0.6                                              # logits of a few tens: the lazy maximum is overtaken often
+    ref = oracle.attention(Qb, Kb, Vb, scale, valid_len=vl)["O"]
+    got = run_fused_bf16(api, Qb, Kb, Vb, scale, vl=vl, variant=variant)
+    check_bf16(got, ref, "many items v%d" % variant)
+    assert np.all(got[0] == 0.0)
+
+
 @pytest.mark.parametrize("scale", [1.0, 0.05, -0.125, 3.0, 0.0])
 def test_fused_bf16_scales_tc(api, scale):
     B, H, Nq, Nk, d = 1, 2, 256, 512, 64
