@@ -5,21 +5,23 @@
 //     logits, exponentiated in place), so every scheduler of the SM holds four softmax warps whose
 //     waits (barrier, TMEM load, store completion) hide behind the exponentials of the others;
 //   * TMEM holds O_A, O_B (64 columns each) and THREE logit buffers X0..X2 of 128 columns that the
-//     tile-steps u = 0, 1, 2, ... (u even: tile A, u odd: tile B, key step u / 2) use in rotation;
-//     the weights P(u) overlay the logits S(u) they came from, and S(u + 3) is issued right behind
-//     the MMAs that read P(u) (same thread, so the tensor pipe keeps the order): the logits of a
-//     tile's next step are computed while the other tile's softmax runs.
+//     tile-steps g = 0, 1, 2, ... of the CTA (g even: tile A, g odd: tile B, key step g / 2, counted
+//     over all its work items) use in rotation; the weights P(g) overlay the logits S(g) they came
+//     from, and S(g + 3) is issued right behind the MMAs that read P(g) (same thread, so the tensor
+//     pipe keeps the order): the logits of a tile's next step are computed while the other tile's
+//     softmax runs.
 //
-// Paper mapping (Section 5, 5.1, 5.2): shared outer loops = (batch, head) on blockIdx.y and a slab
-// of 256 query rows on blockIdx.x (R-granularity); inner loops Logit and Attend interleaved over
-// 128-key tiles, the streaming softmax between them.
+// Paper mapping (Section 5, 5.1, 5.2): shared outer loops = work items (batch, head, slab of 256
+// query rows: R-granularity), walked by min(items, SMs) persistent CTAs -- CTA c takes items c,
+// c + gridDim.x, ... and its rings, buffers and barrier phases run on across item boundaries;
+// inner loops Logit and Attend interleaved over 128-key tiles, the streaming softmax between them.
 //
 // CTA = 640 threads, five warpgroups; registers move from the fifth to the first four:
 //   warps 0-15  softmax: warp w serves row group q = w % 4 (TMEM lanes 32q..32q+31) of tile
 //               t = w / 8, key half h = (w / 4) % 2 of every step
-//   warp  16    TMA producer (one lane): Q tiles once, then K and V tiles into separate rings
-//   warp  17/18 MMA issuers (one elected lane each): O_t += P(u) V for the tile-steps of tile A / B,
-//               each followed by the logits S(u + 3) of the other tile into the buffer just read
+//   warp  16    TMA producer (one lane): per item the Q tiles, then K and V tiles into separate rings
+//   warp  17/18 MMA issuers (one elected lane each): O_t += P(g) V for the tile-steps of tile A / B,
+//               each followed by the logits S(g + 3) of the other tile into the buffer just read
 //   warp  19    idle (it completes the warpgroup for the register hand-over)
 // The two warps that share a row keep the same reference maximum m_ref: the first step fixes it
 // from the exact maximum of both halves (exchanged through shared memory); later steps reuse it and
