@@ -698,12 +698,16 @@ int launch_tc3(const Problem& p, cudaStream_t st) {
         !make_map(&tmV, p.V, BH, p.Nk, D, BN))
         return FLAT_ERR_CUDA;
     if (!ensure_dynamic_smem<fused_tc3_kernel>(LY::SMEM_BYTES)) return FLAT_ERR_CUDA;
-    // One CTA per SM at most; each walks over its share of the (head, 256-row slab) items, slabs of
-    // a head next to each other so that CTAs running at the same time share K and V in L2.
+    // Work items = (head, 256-row slab), slabs of a head next to each other so that CTAs running at
+    // the same time share K and V in L2.  With many items per SM the grid is one persistent CTA per
+    // SM, each walking over its share (the fixed deal costs little then and the pipeline never
+    // drains); with few, one CTA per item, which the hardware hands out as SMs become free -- the
+    // better balance when the items differ in length (key-padding masks) and there are only a few
+    // rounds of them.
     const int slabs = (p.Nq + 2 * BM - 1) / (2 * BM);
     const int64_t items = static_cast<int64_t>(slabs) * BH;
     const int sms = device_sm_count();
-    const int grid = static_cast<int>(items < sms ? items : sms);
+    const int grid = static_cast<int>(items >= 8 * static_cast<int64_t>(sms) ? sms : items);
     fused_tc3_kernel<<<grid, LY::THREADS, LY::SMEM_BYTES, st>>>(tmQ, tmK, tmV, static_cast<__nv_bfloat16*>(p.O), p.H,
                                                                 p.Nq, p.Nk, static_cast<int>(items), slabs,
                                                                 p.scale * 1.4426950408889634f, p.k_valid_len, p.status);
