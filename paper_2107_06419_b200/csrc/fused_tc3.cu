@@ -488,9 +488,11 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             const uint32_t s_addr = tl + LY::X_COL(b) + h * HN;
             if (q == 0 && lane == 0) TRACE(trole, j, 0);
             const uint32_t xph = static_cast<uint32_t>(g / 6) & 1u;   // phase parity of this tile's use of the buffer
+            // A warp whose wait fails does not leave by itself: it goes on to the next vote with its
+            // partner (reading TMEM that may not be ready is harmless, nothing is stored), so that the
+            // two always pass the same sequence of named barriers and leave together.
             ok = bounded_wait_s(bars_s + 8 * (LY::S_FULL + t * 3 + b), xph, abort_s, status, 0x300 + t);
             ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
             tc_fence_after();
             if (q == 0 && lane == 0) TRACE(trole, j, 1);
             const int col0 = j * BN + h * HN;
@@ -503,11 +505,7 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             // two warps have voted, so the redo reads them again instead of holding them in registers.
             uint32_t pk[2][16];
             float ls[4] = {0.f, 0.f, 0.f, 0.f};
-#ifdef FLAT_TC3_ALWAYS_CAREFUL
-            bool careful = true;
-#else
             bool careful = (j == 0);
-#endif
             if (!careful) {
                 // (the logits come in two loads of 32 so that few registers are live at a time)
                 uint32_t r[32];
@@ -540,10 +538,11 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                     if (xmax > 126.f) lt = INFINITY;      // the polynomial was fed an argument beyond its range
                 }
                 if (q == 0 && lane == 0) TRACE(trole, j, 3);
-                careful = pair_any(pair_id, !(lt <= OVERFLOW_SUM));
+                careful = pair_any(pair_id, !(lt <= OVERFLOW_SUM) || !ok);
             }
             if (q == 0 && lane == 0) TRACE(trole, j, 4);
             if (careful) {
+                if (pair_any(pair_id, !ok)) { ok = false; break; }     // (both warps are here: j == 0 or the joint vote)
                 float mx = -INFINITY;
                 {
                     uint32_t s[HN];
