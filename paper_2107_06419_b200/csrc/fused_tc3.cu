@@ -75,6 +75,9 @@ constexpr float OVERFLOW_SUM = 1.0995116e12f;   // 2^40: a row sum beyond this m
 #ifndef FLAT_TC3_POLY
 #define FLAT_TC3_POLY true
 #endif
+#ifndef FLAT_TC3_PRODUCER_SLEEP
+#define FLAT_TC3_PRODUCER_SLEEP 400   // ns between the TMA producer's probes of a full ring (it runs far ahead: its reaction time is immaterial)
+#endif
 #ifndef FLAT_TC3_POLY_PAIRS
 #define FLAT_TC3_POLY_PAIRS 0x0202   // bit i: pair i of each 16 pairs (32 logits) takes the polynomial; two pairs = one element in eight
 #endif
@@ -348,7 +351,7 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             int q_loaded[2] = {0, 0}, k_issued = 0, v_issued = 0;    // (for the drain after a failed wait)
             auto load_q = [&](int t, int q, int row, int bh) {
                 // the logit MMAs of the previous item must have finished with this tile of shared memory
-                if (q > 0) ok = bounded_wait_s(bars_s + 8 * (LY::Q_EMPTY + t), (q - 1) & 1, abort_s, status, 0x120 + t);
+                if (q > 0) ok = bounded_wait_s<FLAT_TC3_PRODUCER_SLEEP>(bars_s + 8 * (LY::Q_EMPTY + t), (q - 1) & 1, abort_s, status, 0x120 + t);
                 if (!ok) return;
                 mbar_arrive_expect_tx(&bars[LY::Q_FULL + t], LY::Q_BYTES);
                 tma_load_3d(Qs + t * LY::Q_BYTES, &tmQ, &bars[LY::Q_FULL + t], 0, row, bh);
@@ -356,7 +359,7 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             };
             auto load_k = [&](int J, int j, int bh) {
                 const int s = J % LY::KS;
-                ok = bounded_wait_s(bars_s + 8 * (LY::K_EMPTY + s), ((J / LY::KS) & 1) ^ 1, abort_s, status, 0x100 + s);
+                ok = bounded_wait_s<FLAT_TC3_PRODUCER_SLEEP>(bars_s + 8 * (LY::K_EMPTY + s), ((J / LY::KS) & 1) ^ 1, abort_s, status, 0x100 + s);
                 if (!ok) return;
                 mbar_arrive_expect_tx(&bars[LY::K_FULL + s], LY::KV_BYTES);
                 tma_load_3d(Ks + s * LY::KV_BYTES, &tmK, &bars[LY::K_FULL + s], 0, j * BN, bh);
@@ -364,7 +367,7 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             };
             auto load_v = [&](int J, int j, int bh) {
                 const int s = J % LY::VS;
-                ok = bounded_wait_s(bars_s + 8 * (LY::V_EMPTY + s), ((J / LY::VS) & 1) ^ 1, abort_s, status, 0x110 + s);
+                ok = bounded_wait_s<FLAT_TC3_PRODUCER_SLEEP>(bars_s + 8 * (LY::V_EMPTY + s), ((J / LY::VS) & 1) ^ 1, abort_s, status, 0x110 + s);
                 if (!ok) return;
                 mbar_arrive_expect_tx(&bars[LY::V_FULL + s], LY::KV_BYTES);
                 tma_load_3d(Vs + s * LY::KV_BYTES, &tmV, &bars[LY::V_FULL + s], 0, j * BN, bh);

@@ -37,14 +37,20 @@ __device__ __forceinline__ bool bounded_wait(uint64_t* bar, uint32_t parity, vol
 }
 
 // The same wait with the barrier and the abort flag given as 32-bit shared-window addresses.
+// SLEEP_NS > 0: the thread sleeps that long between probes -- for a role whose reaction time does
+// not matter (a producer that runs ahead of its ring) and that should leave the issue slots and
+// the shared-memory pipe to the working warps while it waits.
+template <unsigned SLEEP_NS = 0>
 __device__ __forceinline__ bool bounded_wait_s(uint32_t bar_addr, uint32_t parity, uint32_t abort_addr,
                                                int32_t* status, int code, long long limit = WAIT_CYCLES) {
     if (ptx::mbar_try_wait_s(bar_addr, parity)) return true;
     const long long t0 = clock64();
     for (;;) {
 #pragma unroll 1
-        for (int i = 0; i < 32; ++i)
+        for (int i = 0; i < 32; ++i) {
+            if (SLEEP_NS) __nanosleep(SLEEP_NS);
             if (ptx::mbar_try_wait_s(bar_addr, parity)) return true;
+        }
         int aborted;
         asm volatile("ld.volatile.shared::cta.s32 %0, [%1];" : "=r"(aborted) : "r"(abort_addr) : "memory");
         if (aborted) return false;
