@@ -311,6 +311,12 @@ def main():
                          "traffic": load_traffic(w.name, kernel_name(args.variant, w)),
                          "algorithmic_bytes": w.qkvo_bytes()},
         }
+        if vl is not None:
+            # Masked workload: `value` counts the masked keys too (the stated metric, 4 B H Nq Nk d);
+            # this is the same rate counted over the valid keys only.
+            useful = 4.0 * w.H * w.Nq * w.d * float(np.sum(vl))
+            out["useful_work"] = {"value": value * useful / float(w.flops), "unit": UNIT,
+                                  "valid_key_fraction": useful / float(w.flops)}
         if args.with_naive and world == 1:
             # The paper's unfused baseline on the same inputs: L (fp32) and A (bf16) go through HBM.
             elems = w.B * w.H * w.Nq * w.Nk
