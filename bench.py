@@ -307,7 +307,8 @@ def main():
                          "peak": peaks["bf16_tflops"], "unit": UNIT, "frac": achieved / peaks["bf16_tflops"],
                          "peak_kind": "burst bf16 matmul, of " + peaks["source"],
                          "frac_of_sustained": achieved / peaks["bf16_tflops_sustained"],
-                         "kernel_ms": kernel_ms, "flops_per_launch": w.flops,
+                         "kernel_ms": kernel_ms, "kernel_ms_min": float(np.min(per_launch)),
+                         "kernel_ms_median": float(np.median(per_launch)), "flops_per_launch": w.flops,
                          "traffic": load_traffic(w.name, kernel_name(args.variant, w)),
                          "algorithmic_bytes": w.qkvo_bytes()},
         }
