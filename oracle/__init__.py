@@ -37,7 +37,7 @@ def _load():
         lib.oracle_attn_rows.argtypes = [
             ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int,
             ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, ctypes.c_float,
-            ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64,
+            ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p, ctypes.c_int64,
             ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.POINTER(ctypes.c_int)]
         lib.oracle_hardware_threads.restype = ctypes.c_int
         _lib = lib
@@ -49,11 +49,12 @@ def hardware_threads() -> int:
 
 
 def attention(Q, K, V, scale, valid_len=None, rows=None, want_logits=False, want_weights=False,
-              nthreads: int = 0):
+              nthreads: int = 0, causal: bool = False):
     """Exact attention in double precision.
 
     Q: [B,H,Nq,d], K/V: [B,H,Nk,d]; dtype uint16 (bf16 bit patterns) or float32.
     rows: optional int64 array of flat row ids ((b*H+h)*Nq + i); default all rows.
+    causal: query i attends keys j <= i + (Nk - Nq) only (intersected with valid_len).
     Returns dict with 'O' ([B,H,Nq,d] or [nrows,d] float64), optionally 'L' and
     'A' ([..., Nk]), and 'threads' (threads used).
     """
@@ -88,7 +89,7 @@ def attention(Q, K, V, scale, valid_len=None, rows=None, want_logits=False, want
     used = ctypes.c_int(0)
     ptr = lambda a: None if a is None else a.ctypes.data_as(ctypes.c_void_p)
     rc = _load().oracle_attn_rows(ptr(Q), ptr(K), ptr(V), dtype, B, H, Nq, Nk, d, float(np.float32(scale)),
-                                  ptr(vl), ptr(rows), n, ptr(O), ptr(L), ptr(A), int(nthreads),
+                                  ptr(vl), 1 if causal else 0, ptr(rows), n, ptr(O), ptr(L), ptr(A), int(nthreads),
                                   ctypes.byref(used))
     if rc != 0:
         raise ValueError("oracle_attn_rows rejected its arguments (code %d)" % rc)

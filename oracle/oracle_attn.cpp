@@ -22,6 +22,9 @@
 //   * key-padding mask: key j of batch b takes part iff j < valid_len[b]; masked
 //     keys are left out before the maximum.  A row with no valid key gives O = 0.
 //   * Nq may differ from Nk (cross attention): softmax still runs along keys.
+//   * causal mask (decoder workloads; the paper does not spell masks out): query i takes
+//     part with key j iff j <= i + (Nk - Nq), i.e. the last query sees every key and each
+//     earlier query one key fewer; combined with the key-padding mask by intersection.
 //
 // Parity pins (tests/test_oracle_pins.py): closed-form worked example, row sums,
 // Q = 0 -> mean of V, identical keys -> uniform weights, key permutation, key
@@ -49,6 +52,7 @@ struct Problem {
     int64_t B, H, Nq, Nk, d;
     double scale;
     const int32_t* valid_len;        // [B] or null
+    int causal;                      // 0 / 1
     const int64_t* rows;             // flat row ids (b*H + h)*Nq + i, or null = all rows
     int64_t nrows;
     double* O;                       // [nrows, d]
@@ -67,7 +71,12 @@ void attend_row(const Problem& p, int64_t r, std::vector<double>& s) {
     const int64_t i = row % p.Nq;
     const int64_t bh = row / p.Nq;
     const int64_t b = bh / p.H;
-    const int64_t n = p.valid_len ? p.valid_len[b] : p.Nk;
+    int64_t n = p.valid_len ? p.valid_len[b] : p.Nk;
+    if (p.causal) {                  // keys 0 .. i + (Nk - Nq) only
+        const int64_t lim = i + 1 + (p.Nk - p.Nq);
+        if (lim < n) n = lim;
+        if (n < 0) n = 0;
+    }
     const int64_t qoff = (bh * p.Nq + i) * p.d;
     const int64_t koff = bh * p.Nk * p.d;
     double* o = p.O + r * p.d;
@@ -118,7 +127,7 @@ extern "C" {
 // threads"; the count actually used is written to *threads_used if non-null.
 int oracle_attn_rows(const void* Q, const void* K, const void* V, int dtype,
                      int64_t B, int64_t H, int64_t Nq, int64_t Nk, int64_t d, float scale,
-                     const int32_t* valid_len, const int64_t* rows, int64_t nrows,
+                     const int32_t* valid_len, int causal, const int64_t* rows, int64_t nrows,
                      double* O, double* L, double* A, int nthreads, int* threads_used) {
     if (!Q || !K || !V || !O) return 1;
     if (B < 1 || H < 1 || Nq < 1 || Nk < 1 || d < 1) return 1;
@@ -129,7 +138,7 @@ int oracle_attn_rows(const void* Q, const void* K, const void* V, int dtype,
     if (rows) for (int64_t r = 0; r < nrows; ++r) if (rows[r] < 0 || rows[r] >= total) return 1;
     if (valid_len) for (int64_t b = 0; b < B; ++b) if (valid_len[b] < 0 || valid_len[b] > Nk) return 1;
 
-    Problem p{Q, K, V, dtype, B, H, Nq, Nk, d, static_cast<double>(scale), valid_len, rows, nrows, O, L, A};
+    Problem p{Q, K, V, dtype, B, H, Nq, Nk, d, static_cast<double>(scale), valid_len, causal ? 1 : 0, rows, nrows, O, L, A};
     int nt = nthreads > 0 ? nthreads : static_cast<int>(std::thread::hardware_concurrency());
     if (nt < 1) nt = 1;
     if (nt > nrows) nt = nrows > 0 ? static_cast<int>(nrows) : 1;

@@ -247,6 +247,50 @@ def test_brute_force_tiny(Nq, Nk, d, B, H, dtype):
 
 
 # Row selection returns exactly the rows of the full result, and bf16 bits == widened float32.
+@pytest.mark.parametrize("Nq,Nk", [(5, 5), (3, 9), (9, 3), (1, 7), (17, 130)])
+def test_causal_mask_pins(Nq, Nk):
+    """Causal reading: query i sees keys j <= i + (Nk - Nq).  Pinned against an explicit mask matrix
+    (independent numpy softmax over the kept logits), against per-row truncation through the unmasked
+    oracle, and by two closed cases: the last query row equals the unmasked row, and with Nq = Nk the
+    first row is V[0]."""
+    rng = np.random.default_rng(100 * Nq + Nk)
+    B, H, d = 2, 2, 4
+    Q = rng.standard_normal((B, H, Nq, d)).astype(np.float32)
+    K = rng.standard_normal((B, H, Nk, d)).astype(np.float32)
+    V = rng.standard_normal((B, H, Nk, d)).astype(np.float32)
+    vl = np.array([Nk, max(1, Nk - 2)], dtype=np.int32)
+    scale = 0.7
+    got = oracle.attention(Q, K, V, scale, valid_len=vl, causal=True, want_weights=True)
+    O, A = got["O"], got["A"]
+    # explicit mask matrix
+    sc = np.float64(np.float32(scale))
+    L = sc * np.einsum("bhid,bhjd->bhij", Q.astype(np.float64), K.astype(np.float64))
+    i = np.arange(Nq)[:, None]; j = np.arange(Nk)[None, :]
+    for b in range(B):
+        keep = (j <= i + (Nk - Nq)) & (j < vl[b])
+        for h in range(H):
+            W = np.where(keep, np.exp(L[b, h] - L[b, h].max()), 0.0)
+            den = W.sum(-1, keepdims=True)
+            Wn = np.divide(W, den, out=np.zeros_like(W), where=den > 0)
+            np.testing.assert_allclose(A[b, h], Wn, rtol=0, atol=1e-14)
+            np.testing.assert_allclose(O[b, h], Wn @ V[b, h].astype(np.float64), rtol=0, atol=1e-13)
+            assert np.all(A[b, h][~keep] == 0.0)
+    # per-row truncation through the unmasked oracle
+    for b in range(B):
+        for ii in range(Nq):
+            n = min(int(vl[b]), ii + 1 + Nk - Nq)
+            if n <= 0:
+                assert np.all(O[b, :, ii] == 0.0)
+                continue
+            ref = oracle.attention(Q[b:b + 1, :, ii:ii + 1], K[b:b + 1, :, :n], V[b:b + 1, :, :n], scale)["O"]
+            np.testing.assert_allclose(O[b, :, ii], ref[0, :, 0], rtol=0, atol=1e-14)
+    # the last query row is unaffected by the causal mask; with Nq == Nk the first row is V[0]
+    plain = oracle.attention(Q, K, V, scale, valid_len=vl)["O"]
+    np.testing.assert_allclose(O[:, :, -1], plain[:, :, -1], rtol=0, atol=1e-15)
+    if Nq == Nk:
+        np.testing.assert_allclose(O[:, :, 0], V[:, :, 0].astype(np.float64), rtol=0, atol=1e-15)
+
+
 def test_row_sampling_and_dtype_paths_agree():
     rng = np.random.default_rng(11)
     B, H, Nq, Nk, d = 2, 3, 10, 21, 8
