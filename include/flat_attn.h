@@ -86,6 +86,12 @@ typedef struct flat_attn_params {
     int32_t* status;           /* optional device word; a kernel that gives up on a bounded
                                   wait stores a non-zero code here (never traps or hangs)      */
     int variant;               /* FLAT_VARIANT_*                                               */
+    int causal;                /* 0, or 1 = causal mask: query i takes part with key j iff
+                                  j <= i + (Nk - Nq) (the last query sees every key), intersected
+                                  with k_valid_len.  The paper names masking only in passing
+                                  (Section 2, footnote); its decoder workloads need it.  Kernels
+                                  without support return FLAT_ERR_UNSUPPORTED when picked by
+                                  `variant`; AUTO picks one that has it.                        */
 } flat_attn_params_t;
 
 /*

@@ -36,7 +36,8 @@ class flat_attn_params_t(ctypes.Structure):
     _fields_ = [("Q", ctypes.c_void_p), ("K", ctypes.c_void_p), ("V", ctypes.c_void_p), ("O", ctypes.c_void_p),
                 ("B", ctypes.c_int), ("H", ctypes.c_int), ("Nq", ctypes.c_int), ("Nk", ctypes.c_int),
                 ("d", ctypes.c_int), ("scale", ctypes.c_float), ("dtype", ctypes.c_int),
-                ("k_valid_len", ctypes.c_void_p), ("status", ctypes.c_void_p), ("variant", ctypes.c_int)]
+                ("k_valid_len", ctypes.c_void_p), ("status", ctypes.c_void_p), ("variant", ctypes.c_int),
+                ("causal", ctypes.c_int)]
 
 
 _vp, _i, _f = ctypes.c_void_p, ctypes.c_int, ctypes.c_float
@@ -100,7 +101,7 @@ def _dtype_code(t) -> int:
     raise TypeError("Q/K/V/O must be bfloat16 or float32")
 
 
-def _params(Q, K, V, O, scale, k_valid_len, status, variant, host=False):
+def _params(Q, K, V, O, scale, k_valid_len, status, variant, host=False, causal=False):
     B, H, Nq, d = Q.shape
     Nk = K.shape[2]
     if tuple(K.shape) != (B, H, Nk, d) or tuple(V.shape) != (B, H, Nk, d) or tuple(O.shape) != (B, H, Nq, d):
@@ -123,6 +124,7 @@ def _params(Q, K, V, O, scale, k_valid_len, status, variant, host=False):
     p.k_valid_len = None if k_valid_len is None else k_valid_len.data_ptr()
     p.status = None if status is None else status.data_ptr()
     p.variant = int(variant)
+    p.causal = 1 if causal else 0
     return p
 
 
@@ -140,8 +142,11 @@ def flat_attn_fwd(Q, K, V, O, scale, stream=None):
     return O
 
 
-def flat_attn_fwd_ex(Q, K, V, O, scale, k_valid_len=None, status=None, variant=FLAT_VARIANT_AUTO, stream=None):
-    p = _params(Q, K, V, O, scale, k_valid_len, status, variant)
+def flat_attn_fwd_ex(Q, K, V, O, scale, k_valid_len=None, status=None, variant=FLAT_VARIANT_AUTO, stream=None,
+                     causal=False):
+    """Fused attention with dtype choice (from the tensors), key-padding mask, kernel choice and
+    causal mask (query i sees keys j <= i + (Nk - Nq))."""
+    p = _params(Q, K, V, O, scale, k_valid_len, status, variant, causal=causal)
     _check(_lib.flat_attn_fwd_ex(ctypes.byref(p), _stream_ptr(stream)))
     return O
 
@@ -155,8 +160,8 @@ def flat_attn_naive_fwd(Q, K, V, O, L, A, scale, stream=None):
     return O
 
 
-def flat_attn_naive_fwd_ex(Q, K, V, O, L, A, scale, k_valid_len=None, stream=None):
-    p = _params(Q, K, V, O, scale, k_valid_len, None, FLAT_VARIANT_AUTO)
+def flat_attn_naive_fwd_ex(Q, K, V, O, L, A, scale, k_valid_len=None, stream=None, causal=False):
+    p = _params(Q, K, V, O, scale, k_valid_len, None, FLAT_VARIANT_AUTO, causal=causal)
     _check_la(p, L, A)
     _check(_lib.flat_attn_naive_fwd_ex(ctypes.byref(p), _ptr(L), _ptr(A), _stream_ptr(stream)))
     return O
@@ -216,10 +221,10 @@ def flat_attn_host_workspace_bytes(B, H, Nq, Nk, d, dtype=FLAT_DTYPE_BF16) -> in
 
 
 def flat_attn_fwd_host(Q, K, V, O, scale, workspace, k_valid_len=None, status=None,
-                       variant=FLAT_VARIANT_AUTO, stream=None):
+                       variant=FLAT_VARIANT_AUTO, stream=None, causal=False):
     """Q, K, V, O (and k_valid_len) are HOST tensors (pinned for asynchrony); `workspace` is a CUDA
     uint8 tensor of at least flat_attn_host_workspace_bytes(...) bytes.  Asynchronous on `stream`."""
-    p = _params(Q, K, V, O, scale, k_valid_len, status, variant, host=True)
+    p = _params(Q, K, V, O, scale, k_valid_len, status, variant, host=True, causal=causal)
     if not workspace.is_cuda:
         raise ValueError("workspace must be a CUDA tensor")
     _check(_lib.flat_attn_fwd_host(ctypes.byref(p), _ptr(workspace), workspace.numel() * workspace.element_size(),

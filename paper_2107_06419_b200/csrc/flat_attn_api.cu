@@ -28,8 +28,9 @@ int validate(const flat_attn_params_t* p, flat::Problem* out) {
     if (!aligned16(p->Q) || !aligned16(p->K) || !aligned16(p->V) || !aligned16(p->O)) return FLAT_ERR_ALIGN;
     if (p->k_valid_len && (reinterpret_cast<uintptr_t>(p->k_valid_len) & 3u)) return FLAT_ERR_ALIGN;
     if (p->status && (reinterpret_cast<uintptr_t>(p->status) & 3u)) return FLAT_ERR_ALIGN;
+    if (p->causal != 0 && p->causal != 1) return FLAT_ERR_UNSUPPORTED;
     *out = flat::Problem{p->Q, p->K, p->V, p->O, p->B, p->H, p->Nq, p->Nk, p->d,
-                         p->scale, p->dtype, p->k_valid_len, p->status};
+                         p->scale, p->dtype, p->k_valid_len, p->status, p->causal};
     return FLAT_OK;
 }
 
@@ -51,8 +52,11 @@ int run_fused(const flat::Problem& q, int variant, cudaStream_t st) {
             const int sms = flat::device_sm_count();
             if (q.d == 64) v = 2 * ctas2 >= sms ? FLAT_VARIANT_TC3 : FLAT_VARIANT_TC2_SINGLE;
             else           v = ctas2 >= sms ? FLAT_VARIANT_TC2 : FLAT_VARIANT_TC;
+            // The causal mask lives in the FFMA kernel only so far.
+            if (q.causal) v = FLAT_VARIANT_SIMT;
         }
     }
+    if (q.causal && v != FLAT_VARIANT_SIMT) return FLAT_ERR_UNSUPPORTED;
     if (v == FLAT_VARIANT_TC2_SINGLE) {
         if (!tc_applies(q) || q.d != 64) return FLAT_ERR_UNSUPPORTED;
         return flat::launch_fused_tc2_single(q, st);
@@ -109,7 +113,7 @@ int flat_attn_fwd_ex(const flat_attn_params_t* p, void* stream) {
 
 int flat_attn_fwd(const void* Q, const void* K, const void* V, void* O, int B, int H, int Nq, int Nk, int d,
                   float scale, void* stream) {
-    flat_attn_params_t p{Q, K, V, O, B, H, Nq, Nk, d, scale, FLAT_DTYPE_BF16, nullptr, nullptr, FLAT_VARIANT_AUTO};
+    flat_attn_params_t p{Q, K, V, O, B, H, Nq, Nk, d, scale, FLAT_DTYPE_BF16, nullptr, nullptr, FLAT_VARIANT_AUTO, 0};
     return flat_attn_fwd_ex(&p, stream);
 }
 
@@ -126,7 +130,7 @@ int flat_attn_naive_fwd_ex(const flat_attn_params_t* p, void* L, void* A, void* 
 
 int flat_attn_naive_fwd(const void* Q, const void* K, const void* V, void* O, void* L, void* A, int B, int H,
                         int Nq, int Nk, int d, float scale, void* stream) {
-    flat_attn_params_t p{Q, K, V, O, B, H, Nq, Nk, d, scale, FLAT_DTYPE_BF16, nullptr, nullptr, FLAT_VARIANT_AUTO};
+    flat_attn_params_t p{Q, K, V, O, B, H, Nq, Nk, d, scale, FLAT_DTYPE_BF16, nullptr, nullptr, FLAT_VARIANT_AUTO, 0};
     return flat_attn_naive_fwd_ex(&p, L, A, stream);
 }
 

@@ -17,6 +17,7 @@ struct Problem {
     int dtype;
     const int32_t* k_valid_len;
     int32_t* status;
+    int causal;                      // 0 / 1: query i sees keys j <= i + (Nk - Nq)
 };
 
 // Each launcher enqueues its kernels on `st` and returns a FLAT_* code; *launches (if

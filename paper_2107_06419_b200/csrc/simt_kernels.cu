@@ -128,7 +128,7 @@ template <typename T, int D>
 __global__ void __launch_bounds__(NTHREADS) fused_simt_kernel(const T* __restrict__ Q, const T* __restrict__ K,
                                                               const T* __restrict__ V, T* __restrict__ O, int H,
                                                               int Nq, int Nk, float scale_log2e,
-                                                              const int32_t* __restrict__ valid_len) {
+                                                              const int32_t* __restrict__ valid_len, int causal) {
     extern __shared__ __align__(16) float smem[];
     float* Qs = smem;
     float* Ks = Qs + 64 * (D + 4);
@@ -137,7 +137,15 @@ __global__ void __launch_bounds__(NTHREADS) fused_simt_kernel(const T* __restric
     const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
     const int64_t bh = blockIdx.y;
     const int64_t row0 = static_cast<int64_t>(blockIdx.x) * TM;
-    const int n = valid_len ? min(max(valid_len[bh / H], 0), Nk) : Nk;
+    int n = valid_len ? min(max(valid_len[bh / H], 0), Nk) : Nk;
+    // Causal mask: row r sees keys j < r + 1 + (Nk - Nq); the tile stops at its last row's limit.
+    int nrow[4];
+#pragma unroll
+    for (int a = 0; a < 4; ++a) {
+        const int64_t lim = row0 + ty + 16 * a + 1 + (Nk - Nq);
+        nrow[a] = causal ? static_cast<int>(max(static_cast<int64_t>(0), min(static_cast<int64_t>(n), lim))) : n;
+    }
+    if (causal) n = static_cast<int>(max(static_cast<int64_t>(0), min(static_cast<int64_t>(n), row0 + TM + (Nk - Nq))));
     const T* Qg = Q + bh * Nq * D;
     const T* Kg = K + bh * Nk * D;
     const T* Vg = V + bh * Nk * D;
@@ -164,16 +172,19 @@ __global__ void __launch_bounds__(NTHREADS) fused_simt_kernel(const T* __restric
             float mx = -INFINITY;
 #pragma unroll
             for (int b = 0; b < 4; ++b) {
-                s[a][b] = (k0 + tx + 16 * b < n) ? s[a][b] * scale_log2e : -INFINITY;
+                s[a][b] = (k0 + tx + 16 * b < nrow[a]) ? s[a][b] * scale_log2e : -INFINITY;
                 mx = fmaxf(mx, s[a][b]);
             }
             mx = halfwarp_max(mx);
-            const float m_new = fmaxf(m[a], mx);       // finite: every tile has >= 1 valid key
-            const float alpha = exp2f(m[a] - m_new);   // exp2(-inf) = 0 on the first tile
+            const float m_new = fmaxf(m[a], mx);
+            // (a row that has seen no valid key yet -- possible under the causal mask -- keeps m = -inf;
+            // the reference below is then 0, so that its weights and alpha come out as 0 and not NaN)
+            const float m_use = m_new == -INFINITY ? 0.f : m_new;
+            const float alpha = exp2f(m[a] - m_use);   // exp2(-inf) = 0 on the first tile
             float sum = 0.f;
 #pragma unroll
             for (int b = 0; b < 4; ++b) {
-                const float p = exp2f(s[a][b] - m_new);
+                const float p = exp2f(s[a][b] - m_use);
                 sum += p;
                 Ps[(ty + 16 * a) * PSTRIDE + tx + 16 * b] = p;
             }
@@ -227,10 +238,11 @@ __global__ void __launch_bounds__(NTHREADS) naive_logit_kernel(const T* __restri
 template <typename TA>
 __global__ void __launch_bounds__(NTHREADS) naive_softmax_kernel(const float* __restrict__ L, TA* __restrict__ A,
                                                                  int H, int Nq, int Nk,
-                                                                 const int32_t* __restrict__ valid_len) {
+                                                                 const int32_t* __restrict__ valid_len, int causal) {
     __shared__ float red_m[NTHREADS / 32], red_l[NTHREADS / 32];
     const int64_t row = blockIdx.x;
-    const int n = valid_len ? min(max(valid_len[(row / Nq) / H], 0), Nk) : Nk;
+    int n = valid_len ? min(max(valid_len[(row / Nq) / H], 0), Nk) : Nk;
+    if (causal) n = static_cast<int>(max(static_cast<int64_t>(0), min(static_cast<int64_t>(n), row % Nq + 1 + (Nk - Nq))));
     const float* Lr = L + row * Nk;
     TA* Ar = A + row * Nk;
     constexpr float LOG2E = 1.4426950408889634f;
@@ -307,7 +319,7 @@ static int launch_fused_simt_td(const Problem& p, cudaStream_t st) {
     dim3 grid((p.Nq + TM - 1) / TM, p.B * p.H);
     kern<<<grid, NTHREADS, smem, st>>>(static_cast<const T*>(p.Q), static_cast<const T*>(p.K),
                                        static_cast<const T*>(p.V), static_cast<T*>(p.O), p.H, p.Nq, p.Nk,
-                                       p.scale * 1.4426950408889634f, p.k_valid_len);
+                                       p.scale * 1.4426950408889634f, p.k_valid_len, p.causal);
     return cudaGetLastError() == cudaSuccess ? FLAT_OK : FLAT_ERR_CUDA;
 }
 
@@ -325,7 +337,7 @@ static int launch_naive_td(const Problem& p, float* L, void* A, cudaStream_t st)
     {
         const int64_t rows = static_cast<int64_t>(p.B) * p.H * p.Nq;
         naive_softmax_kernel<TA><<<static_cast<unsigned>(rows), NTHREADS, 0, st>>>(L, static_cast<TA*>(A), p.H, p.Nq,
-                                                                                   p.Nk, p.k_valid_len);
+                                                                                   p.Nk, p.k_valid_len, p.causal);
         if (cudaGetLastError() != cudaSuccess) return FLAT_ERR_CUDA;
     }
     {
@@ -363,7 +375,7 @@ int launch_naive(const Problem& p, void* L, void* A, cudaStream_t st) {
         if (rc != FLAT_OK) return rc;
         const int64_t rows = static_cast<int64_t>(p.B) * p.H * p.Nq;
         naive_softmax_kernel<__nv_bfloat16><<<static_cast<unsigned>(rows), NTHREADS, 0, st>>>(
-            Lf, static_cast<__nv_bfloat16*>(A), p.H, p.Nq, p.Nk, p.k_valid_len);
+            Lf, static_cast<__nv_bfloat16*>(A), p.H, p.Nq, p.Nk, p.k_valid_len, p.causal);
         if (cudaGetLastError() != cudaSuccess) return FLAT_ERR_CUDA;
         return launch_naive_attend_tc(p, A, st);
     }

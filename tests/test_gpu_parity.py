@@ -18,12 +18,12 @@ def api():
     return _api
 
 
-def run_fused_bf16(api, Qb, Kb, Vb, scale, vl=None, variant=0):
+def run_fused_bf16(api, Qb, Kb, Vb, scale, vl=None, variant=0, causal=False):
     Q, K, V = bf16_tensor(Qb), bf16_tensor(Kb), bf16_tensor(Vb)
     O = torch.full(Q.shape, float("nan"), dtype=torch.bfloat16, device="cuda")
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     vlt = None if vl is None else torch.from_numpy(vl).cuda()
-    api.flat_attn_fwd_ex(Q, K, V, O, scale, k_valid_len=vlt, status=status, variant=variant)
+    api.flat_attn_fwd_ex(Q, K, V, O, scale, k_valid_len=vlt, status=status, variant=variant, causal=causal)
     torch.cuda.synchronize()
     assert int(status.item()) == 0, "device status 0x%x" % int(status.item())
     return bf16_to_f64(O)
@@ -113,6 +113,61 @@ def test_many_items_per_cta(api, variant):
     got = run_fused_bf16(api, Qb, Kb, Vb, scale, vl=vl, variant=variant)
     check_bf16(got, ref, "many items v%d" % variant)
     assert np.all(got[0] == 0.0)
+
+
+CAUSAL_SHAPES = [
+    # B, H, Nq, Nk, d, masked
+    (1, 2, 256, 256, 64, False),        # square: row i sees keys 0..i
+    (2, 2, 300, 300, 64, True),         # ragged tiles, key-padding on top
+    (1, 2, 130, 517, 64, False),        # Nk > Nq: the last query sees every key
+    (1, 1, 200, 70, 64, False),         # Nk < Nq: the first 130 queries see no key (O = 0)
+    (2, 1, 384, 640, 128, True),
+    (1, 2, 100, 100, 32, False),
+]
+
+
+@pytest.mark.parametrize("shape", CAUSAL_SHAPES)
+@pytest.mark.parametrize("variant", [0, 1], ids=["auto", "simt"])
+def test_fused_bf16_causal(api, shape, variant):
+    """Causal mask (query i sees keys j <= i + Nk - Nq), alone and on top of a key-padding mask."""
+    B, H, Nq, Nk, d, masked = shape
+    rng = np.random.default_rng(abs(hash(shape)) % (2 ** 31))
+    Qb, Kb, Vb = rand_bits(rng, (B, H, Nq, d)), rand_bits(rng, (B, H, Nk, d)), rand_bits(rng, (B, H, Nk, d))
+    vl = None
+    if masked:
+        vl = rng.integers(1, Nk + 1, size=B).astype(np.int32)
+        vl[0] = Nk // 2 + 1
+    scale = 1 / math.sqrt(d)
+    ref = oracle.attention(Qb, Kb, Vb, scale, valid_len=vl, causal=True)["O"]
+    got = run_fused_bf16(api, Qb, Kb, Vb, scale, vl=vl, variant=variant, causal=True)
+    check_bf16(got, ref, "causal %s v%d" % (shape, variant))
+    if Nk < Nq:
+        assert np.all(got[:, :, :Nq - Nk] == 0.0)
+
+
+def test_causal_f32_and_naive(api):
+    B, H, Nq, Nk, d = 1, 2, 150, 333, 64
+    rng = np.random.default_rng(99)
+    Qf = rng.standard_normal((B, H, Nq, d)).astype(np.float32)
+    Kf = rng.standard_normal((B, H, Nk, d)).astype(np.float32)
+    Vf = rng.standard_normal((B, H, Nk, d)).astype(np.float32)
+    ref = oracle.attention(Qf, Kf, Vf, 0.125, causal=True)["O"]
+    Q, K, V = (torch.from_numpy(x).cuda() for x in (Qf, Kf, Vf))
+    O = torch.full(Q.shape, float("nan"), dtype=torch.float32, device="cuda")
+    api.flat_attn_fwd_ex(Q, K, V, O, 0.125, causal=True)
+    check_f32(O.double().cpu().numpy(), ref, "causal f32")
+    # the unfused baseline with the same mask (bf16: tensor-core logits, masked softmax, attend)
+    Qb, Kb, Vb = (inputs.f32_to_bf16_bits(x).reshape(x.shape) for x in (Qf, Kf, Vf))
+    refb = oracle.attention(Qb, Kb, Vb, 0.125, causal=True)
+    Qt, Kt, Vt = bf16_tensor(Qb), bf16_tensor(Kb), bf16_tensor(Vb)
+    Ot = torch.full(Qt.shape, float("nan"), dtype=torch.bfloat16, device="cuda")
+    L = torch.empty((B, H, Nq, Nk), dtype=torch.float32, device="cuda")
+    A = torch.empty((B, H, Nq, Nk), dtype=torch.bfloat16, device="cuda")
+    api.flat_attn_naive_fwd_ex(Qt, Kt, Vt, Ot, L, A, 0.125, causal=True)
+    torch.cuda.synchronize()
+    check_bf16(bf16_to_f64(Ot), refb["O"], "causal naive")
+    iu = np.triu_indices(Nq, k=Nk - Nq + 1, m=Nk)
+    assert np.all(A.float().cpu().numpy()[0, 0][iu] == 0.0)
 
 
 @pytest.mark.parametrize("scale", [1.0, 0.05, -0.125, 3.0, 0.0])
