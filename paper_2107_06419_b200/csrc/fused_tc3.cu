@@ -243,14 +243,23 @@ __device__ __forceinline__ void exp_pack32(const uint32_t (&r)[32], float scale_
 // One work item = (batch, head, slab of 256 query rows).  A CTA takes the items blockIdx.x,
 // blockIdx.x + gridDim.x, ... one after the other without draining its pipeline in between.
 struct Item {
-    int bh, row0, n, ntiles;                             // n = number of valid keys, ntiles = key steps
+    int bh, row0, n, ntiles;                             // n = number of keys that any row of the slab sees, ntiles = key steps
 };
-__device__ __forceinline__ Item get_item(int idx, int slabs, int H, int Nk, const int32_t* __restrict__ valid_len) {
+// What every role needs to enumerate the items.
+struct Sched {
+    int items, slabs, H, Nk;
+    const int32_t* valid_len;
+    int coff;                                            // causal mask: row r sees keys j < r + 1 + coff (coff = Nk - Nq); none: 2^30
+};
+__device__ __forceinline__ Item get_item(int idx, const Sched& sc) {
     Item it;
-    it.bh = idx / slabs;
-    it.row0 = (idx - it.bh * slabs) * (2 * BM);
-    int n = Nk;
-    if (valid_len) { n = valid_len[it.bh / H]; n = n < 0 ? 0 : (n > Nk ? Nk : n); }
+    it.bh = idx / sc.slabs;
+    it.row0 = (idx - it.bh * sc.slabs) * (2 * BM);
+    int n = sc.Nk;
+    if (sc.valid_len) { n = sc.valid_len[it.bh / sc.H]; n = n < 0 ? 0 : (n > sc.Nk ? sc.Nk : n); }
+    // under the causal mask the slab's last row bounds the keys of the item
+    const long long lim = static_cast<long long>(it.row0) + 2 * BM + sc.coff;
+    n = lim < n ? (lim < 0 ? 0 : static_cast<int>(lim)) : n;
     it.n = n;
     it.ntiles = (n + BN - 1) / BN;
     return it;
@@ -264,35 +273,34 @@ struct Cursor {
     Item it;
     bool valid;
 };
-__device__ __forceinline__ void cursor_seek(Cursor& c, int items, int slabs, int H, int Nk,
-                                            const int32_t* __restrict__ valid_len) {
+__device__ __forceinline__ void cursor_seek(Cursor& c, const Sched& sc) {
     c.valid = false;
-    while (c.idx < items) {
-        c.it = get_item(c.idx, slabs, H, Nk, valid_len);
+    while (c.idx < sc.items) {
+        c.it = get_item(c.idx, sc);
         if (c.it.ntiles > 0) { c.valid = true; return; }
         c.idx += gridDim.x;
     }
 }
-__device__ __forceinline__ void cursor_init(Cursor& c, int items, int slabs, int H, int Nk,
-                                            const int32_t* __restrict__ valid_len) {
+__device__ __forceinline__ void cursor_init(Cursor& c, const Sched& sc) {
     c.idx = blockIdx.x; c.j = 0; c.J = 0; c.q = 0;
-    cursor_seek(c, items, slabs, H, Nk, valid_len);
+    cursor_seek(c, sc);
 }
-__device__ __forceinline__ void cursor_next(Cursor& c, int items, int slabs, int H, int Nk,
-                                            const int32_t* __restrict__ valid_len) {
+__device__ __forceinline__ void cursor_next(Cursor& c, const Sched& sc) {
     ++c.j; ++c.J;
     if (c.j == c.it.ntiles) {
         c.j = 0; ++c.q;
         c.idx += gridDim.x;
-        cursor_seek(c, items, slabs, H, Nk, valid_len);
+        cursor_seek(c, sc);
     }
 }
 
 __global__ void __launch_bounds__(L3::THREADS, 1)
 fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                  const __grid_constant__ CUtensorMap tmV, __nv_bfloat16* __restrict__ O, int H, int Nq, int Nk,
-                 int items, int slabs, float scale_log2e, const int32_t* __restrict__ valid_len, int32_t* status) {
+                 int items, int slabs, float scale_log2e, const int32_t* __restrict__ valid_len, int coff,
+                 int32_t* status) {
     using LY = L3;
+    const Sched sc{items, slabs, H, Nk, valid_len, coff};
     extern __shared__ uint8_t smem_raw[];
     uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* Qs = base;                                  // 2 tiles
@@ -365,7 +373,7 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             };
             int J0 = 0, q = 0;
             for (int idx = blockIdx.x; idx < items && ok; idx += gridDim.x) {
-                const Item it = get_item(idx, slabs, H, Nk, valid_len);
+                const Item it = get_item(idx, sc);
                 if (it.ntiles == 0) continue;
                 load_q(0, q, it.row0, it.bh);
                 if (ok) load_k(J0, 0, it.bh);
@@ -405,8 +413,8 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             if (ok) tc_fence_after();
         };
         Cursor cs, cp;                                   // where the logits / the O += P V of this warp stand
-        cursor_init(cs, items, slabs, H, Nk, valid_len);
-        cursor_init(cp, items, slabs, H, Nk, valid_len);
+        cursor_init(cs, sc);
+        cursor_init(cp, sc);
         auto issue_s = [&]() {                           // S of tile ts at cursor cs, then advance it
             if (!cs.valid || !ok) return;
             const int g = 2 * cs.J + ts, bs = g % 3, ks = cs.J % LY::KS;
@@ -425,7 +433,7 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                 TRACE(4, g, 1);
             }
             __syncwarp();
-            cursor_next(cs, items, slabs, H, Nk, valid_len);
+            cursor_next(cs, sc);
         };
         // the first three logit tiles need no buffer to be freed: S(0), S(2) (tile A, key steps 0 and 1)
         // come from tile B's issuer, S(1) (tile B, key step 0) from tile A's
@@ -450,7 +458,7 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                 TRACE(4, g, 3);
             }
             __syncwarp();
-            cursor_next(cp, items, slabs, H, Nk, valid_len);
+            cursor_next(cp, sc);
             issue_s();                                   // into buffer b: 2 J_s + ts = g + 3
         }
       }
@@ -473,8 +481,13 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         int b = t;                                       // buffer of tile-step g = 2 J + t: g % 3
         int g = t;                                       // this tile's next tile-step (J: key steps of all items so far)
         for (int idx = blockIdx.x; idx < items; idx += gridDim.x) {
-        const Item it = get_item(idx, slabs, H, Nk, valid_len);
-        const int n = it.n, ntiles = it.ntiles;
+        const Item it = get_item(idx, sc);
+        const int ntiles = it.ntiles;
+        // keys this thread's row sees (all the item's keys unless the causal mask cuts the row short);
+        // lane 0 has the shortest row of the warp, so its count tells whether a step needs the masked routine
+        const long long rlim = static_cast<long long>(it.row0) + t * BM + q * 32 + lane + 1 + sc.coff;
+        const int nrow = rlim < it.n ? (rlim < 0 ? 0 : static_cast<int>(rlim)) : it.n;
+        const int nrow_min = __shfl_sync(0xffffffffu, nrow, 0);
         float m_ref = -INFINITY, l = 0.f;
         for (int j = 0; j < ntiles; ++j, g += 2, b = (b == 0 ? 2 : b - 1)) {      // g += 2  <=>  b -= 1 (mod 3)
             // this warp's 64 logits of S(g); its 32 packed columns of P(g) go over the first half of them
@@ -489,8 +502,8 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             tc_fence_after();
             if (q == 0 && lane == 0) TRACE(trole, j, 1);
             const int col0 = j * BN + h * HN;
-            const bool tail = col0 + HN > n;
-            const int nvalid = tail ? (n > col0 ? n - col0 : 0) : HN;
+            const bool tail = col0 + HN > nrow_min;      // (warp-uniform) some row has masked keys in this step
+            const int nvalid = nrow > col0 ? (nrow - col0 < HN ? nrow - col0 : HN) : 0;   // per row
             // p = 2^(scale*s - m_ref); row sum in fp32 from the unrounded p; P rounded to bf16.  Any
             // reference m_ref gives the exact softmax, so the common case takes no row maximum; a sum
             // beyond 2^40 (or inf/NaN) in either half shows that the reference fell too far behind,
@@ -554,7 +567,8 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                 mx = fmaxf(mx, ld_shared_f32(xm_own ^ (BM * 4)));
                 if (__any_sync(0xffffffffu, mx > m_ref + RESCALE_THRESHOLD)) {
                     const float m_new = fmaxf(m_ref, mx);
-                    const float alpha = ex2_approx(m_ref - m_new);     // 0 on the first step
+                    // 0 on the first step; a row that has not seen a valid key yet (causal mask) keeps l = 0
+                    const float alpha = m_new == -INFINITY ? 1.f : ex2_approx(m_ref - m_new);
                     l *= alpha;
                     if (j > 0) {
                         // each half rescales its half of the columns of O_t
@@ -702,7 +716,8 @@ int launch_tc3(const Problem& p, cudaStream_t st) {
     const int grid = static_cast<int>(items >= 8 * static_cast<int64_t>(sms) ? sms : items);
     fused_tc3_kernel<<<grid, LY::THREADS, LY::SMEM_BYTES, st>>>(tmQ, tmK, tmV, static_cast<__nv_bfloat16*>(p.O), p.H,
                                                                 p.Nq, p.Nk, static_cast<int>(items), slabs,
-                                                                p.scale * 1.4426950408889634f, p.k_valid_len, p.status);
+                                                                p.scale * 1.4426950408889634f, p.k_valid_len,
+                                                                p.causal ? p.Nk - p.Nq : (1 << 30), p.status);
     return cudaGetLastError() == cudaSuccess ? FLAT_OK : FLAT_ERR_CUDA;
 }
 

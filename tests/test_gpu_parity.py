@@ -123,14 +123,18 @@ CAUSAL_SHAPES = [
     (1, 1, 200, 70, 64, False),         # Nk < Nq: the first 130 queries see no key (O = 0)
     (2, 1, 384, 640, 128, True),
     (1, 2, 100, 100, 32, False),
+    (3, 2, 1000, 1000, 64, False),      # several slabs and key steps per head
+    (2, 2, 640, 1664, 64, True),
 ]
 
 
 @pytest.mark.parametrize("shape", CAUSAL_SHAPES)
-@pytest.mark.parametrize("variant", [0, 1], ids=["auto", "simt"])
+@pytest.mark.parametrize("variant", [0, 1, 5], ids=["auto", "simt", "tc3"])
 def test_fused_bf16_causal(api, shape, variant):
     """Causal mask (query i sees keys j <= i + Nk - Nq), alone and on top of a key-padding mask."""
     B, H, Nq, Nk, d, masked = shape
+    if variant == 5 and d != 64:
+        pytest.skip("d = 64 only")
     rng = np.random.default_rng(abs(hash(shape)) % (2 ** 31))
     Qb, Kb, Vb = rand_bits(rng, (B, H, Nq, d)), rand_bits(rng, (B, H, Nk, d)), rand_bits(rng, (B, H, Nk, d))
     vl = None
