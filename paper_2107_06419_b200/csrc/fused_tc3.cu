@@ -254,7 +254,12 @@ struct Sched {
 __device__ __forceinline__ Item get_item(int idx, const Sched& sc) {
     Item it;
     it.bh = idx / sc.slabs;
-    it.row0 = (idx - it.bh * sc.slabs) * (2 * BM);
+    int slab = idx - it.bh * sc.slabs;
+    // Under the causal mask a slab's work grows with its position, and a CTA's stride through the
+    // items (gridDim.x) may share a factor with the slabs per head, so that it would keep meeting
+    // the same few positions: rotate the order of the slabs from head to head.
+    if (sc.coff < (1 << 29)) slab = (slab + 7 * it.bh) % sc.slabs;
+    it.row0 = slab * (2 * BM);
     int n = sc.Nk;
     if (sc.valid_len) { n = sc.valid_len[it.bh / sc.H]; n = n < 0 ? 0 : (n > sc.Nk ? sc.Nk : n); }
     // under the causal mask the slab's last row bounds the keys of the item
