@@ -52,11 +52,11 @@ int run_fused(const flat::Problem& q, int variant, cudaStream_t st) {
             const int sms = flat::device_sm_count();
             if (q.d == 64) v = 2 * ctas2 >= sms ? FLAT_VARIANT_TC3 : FLAT_VARIANT_TC2_SINGLE;
             else           v = ctas2 >= sms ? FLAT_VARIANT_TC2 : FLAT_VARIANT_TC;
-            // The causal mask lives in the d = 64 two-threads-per-row kernel and in the FFMA kernel.
-            if (q.causal) v = q.d == 64 ? FLAT_VARIANT_TC3 : FLAT_VARIANT_SIMT;
+            // (the single-tile predecessor kernel has no causal mask)
+            if (q.causal && v == FLAT_VARIANT_TC) v = FLAT_VARIANT_TC2;
         }
     }
-    if (q.causal && v != FLAT_VARIANT_SIMT && v != FLAT_VARIANT_TC3) return FLAT_ERR_UNSUPPORTED;
+    if (q.causal && v == FLAT_VARIANT_TC) return FLAT_ERR_UNSUPPORTED;
     if (v == FLAT_VARIANT_TC2_SINGLE) {
         if (!tc_applies(q) || q.d != 64) return FLAT_ERR_UNSUPPORTED;
         return flat::launch_fused_tc2_single(q, st);

@@ -192,7 +192,7 @@ template <int D, int NT>
 __global__ void __launch_bounds__(128 * NT + 128, NT == 1 ? 2 : 1)
 fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                  const __grid_constant__ CUtensorMap tmV, __nv_bfloat16* __restrict__ O, int H, int Nq, int Nk,
-                 float scale_log2e, const int32_t* __restrict__ valid_len, int32_t* status) {
+                 float scale_log2e, const int32_t* __restrict__ valid_len, int coff, int32_t* status) {
     using LY = L2<D, NT>;
 #ifdef FLAT_TRACE
     constexpr int THREADS = LY::THREADS;
@@ -218,6 +218,12 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     const int row0 = blockIdx.x * (NT * BM);
     int n = Nk;
     if (valid_len) { n = valid_len[bh / H]; n = n < 0 ? 0 : (n > Nk ? Nk : n); }
+    {
+        // Causal mask (coff = Nk - Nq; 2^30 = none): row r sees keys j < r + 1 + coff, so the CTA's
+        // last row bounds the keys of all its rows.
+        const long long lim = static_cast<long long>(row0) + NT * BM + coff;
+        if (lim < n) n = lim < 0 ? 0 : static_cast<int>(lim);
+    }
     const int ntiles = (n + BN - 1) / BN;
 
     if (threadIdx.x == LY::SOFT_WARPS * 32) {
@@ -375,6 +381,10 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         const bool neg_scale = scale_log2e < 0.f;
         float m_ref = -INFINITY, l = 0.f;
         bool ok = true;
+        // keys this thread's row sees; lane 0 has the shortest row of the warp
+        const long long rlim = static_cast<long long>(row) + 1 + coff;
+        const int nrow = rlim < n ? (rlim < 0 ? 0 : static_cast<int>(rlim)) : n;
+        const int nrow_min = __shfl_sync(0xffffffffu, nrow, 0);
         if (LY::TURNS && t == 1 && lane == 0) mbar_arrive(&bars[LY::TURN + (warp & 3)]);   // tile A goes first
         for (int j = 0; j < ntiles; ++j) {
             if ((warp & 3) == 0 && lane == 0) TRACE(t, j, 0);
@@ -393,11 +403,12 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             if ((warp & 3) == 0 && lane == 0) TRACE(t, j, 2);
 
             const int col0 = j * BN;
-            const bool tail = col0 + BN > n;
+            const bool tail = col0 + BN > nrow_min;      // (warp-uniform) some row has masked keys in this step
+            const int nvalid = nrow > col0 ? (nrow - col0 < BN ? nrow - col0 : BN) : 0;   // per row
             if (tail) {
                 const uint32_t excl = __float_as_uint(neg_scale ? INFINITY : -INFINITY);
 #pragma unroll
-                for (int i = 0; i < 128; ++i) if (col0 + i >= n) s[i] = excl;
+                for (int i = 0; i < 128; ++i) if (i >= nvalid) s[i] = excl;
             }
             // At d = 64 P_t is a single buffer: O_t += P_t(j-1) V must have consumed it before the
             // first store of P_t(j).  The wait sits inside the exponential pipeline (see exp_store).
@@ -442,10 +453,12 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                 careful = __any_sync(0xffffffffu, !(lt <= OVERFLOW_SUM));
             }
             if (careful) {
-                const float mx = (neg_scale ? row_min(s) : row_max(s)) * scale_log2e;
+                // (a row with no valid key in this step -- causal mask -- contributes no maximum)
+                const float mx = nvalid > 0 ? (neg_scale ? row_min(s) : row_max(s)) * scale_log2e : -INFINITY;
                 if (__any_sync(0xffffffffu, mx > m_ref + RESCALE_THRESHOLD)) {
                     const float m_new = fmaxf(m_ref, mx);
-                    const float alpha = ex2_approx(m_ref - m_new);     // 0 on the first tile
+                    // 0 on the first tile; a row that has not seen a valid key yet keeps l = 0
+                    const float alpha = m_new == -INFINITY ? 1.f : ex2_approx(m_ref - m_new);
                     l *= alpha;
                     if (j > 0) {
                         ok = __all_sync(0xffffffffu, bounded_wait(&bars[LY::PV_DONE + t], (j - 1) & 1, abort_flag,
@@ -465,8 +478,7 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                     }
                     m_ref = m_new;
                 }
-                lt = exp_store<true, false>(s, scale_log2e, -m_ref, tl + LY::P_COL(t), tail ? n - col0 : BN, wait_p_free,
-                                     pass_turn);
+                lt = exp_store<true, false>(s, scale_log2e, -m_ref, tl + LY::P_COL(t), nvalid, wait_p_free, pass_turn);
                 if (!ok) break;
             }
             l += lt;
@@ -536,7 +548,8 @@ int launch_tc2_d(const Problem& p, cudaStream_t st) {
     if (!ensure_dynamic_smem<fused_tc2_kernel<D, NT>>(LY::SMEM_BYTES)) return FLAT_ERR_CUDA;
     dim3 grid((p.Nq + NT * BM - 1) / (NT * BM), BH);
     kern<<<grid, LY::THREADS, LY::SMEM_BYTES, st>>>(tmQ, tmK, tmV, static_cast<__nv_bfloat16*>(p.O), p.H, p.Nq,
-                                                    p.Nk, p.scale * 1.4426950408889634f, p.k_valid_len, p.status);
+                                                    p.Nk, p.scale * 1.4426950408889634f, p.k_valid_len,
+                                                    p.causal ? p.Nk - p.Nq : (1 << 30), p.status);
     return cudaGetLastError() == cudaSuccess ? FLAT_OK : FLAT_ERR_CUDA;
 }
 

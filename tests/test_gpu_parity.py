@@ -129,12 +129,14 @@ CAUSAL_SHAPES = [
 
 
 @pytest.mark.parametrize("shape", CAUSAL_SHAPES)
-@pytest.mark.parametrize("variant", [0, 1, 5], ids=["auto", "simt", "tc3"])
+@pytest.mark.parametrize("variant", [0, 1, 3, 4, 5], ids=["auto", "simt", "tc2", "tc2single", "tc3"])
 def test_fused_bf16_causal(api, shape, variant):
     """Causal mask (query i sees keys j <= i + Nk - Nq), alone and on top of a key-padding mask."""
     B, H, Nq, Nk, d, masked = shape
-    if variant == 5 and d != 64:
+    if variant in (4, 5) and d != 64:
         pytest.skip("d = 64 only")
+    if variant in (3, 4, 5) and d not in (64, 128):
+        pytest.skip("tensor-core kernels: d in {64, 128}")
     rng = np.random.default_rng(abs(hash(shape)) % (2 ** 31))
     Qb, Kb, Vb = rand_bits(rng, (B, H, Nq, d)), rand_bits(rng, (B, H, Nk, d)), rand_bits(rng, (B, H, Nk, d))
     vl = None
