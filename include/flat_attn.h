@@ -89,9 +89,8 @@ typedef struct flat_attn_params {
     int causal;                /* 0, or 1 = causal mask: query i takes part with key j iff
                                   j <= i + (Nk - Nq) (the last query sees every key), intersected
                                   with k_valid_len.  The paper names masking only in passing
-                                  (Section 2, footnote); its decoder workloads need it.  Kernels
-                                  without support return FLAT_ERR_UNSUPPORTED when picked by
-                                  `variant`; AUTO picks one that has it.                        */
+                                  (Section 2, footnote); its decoder workloads need it.  The
+                                  unfused baseline honours it too (A is 0 beyond the limit).    */
 } flat_attn_params_t;
 
 /*
@@ -103,8 +102,10 @@ typedef struct flat_attn_params {
 int flat_attn_fwd(const void* Q, const void* K, const void* V, void* O,
                   int B, int H, int Nq, int Nk, int d, float scale, void* stream);
 
-/* Fused attention with dtype choice, optional key-padding mask and kernel choice (same
- * operation as flat_attn_fwd).  `p` is a HOST pointer, read before the call returns. */
+/* Fused attention with dtype choice, optional key-padding mask, optional causal mask and
+ * kernel choice (same operation as flat_attn_fwd; a masked key takes no part in the softmax of
+ * the row, a row without any key gives O = 0).  `p` is a HOST pointer, read before the call
+ * returns.  FLAT_VARIANT_TC does not implement the causal mask (FLAT_ERR_UNSUPPORTED). */
 int flat_attn_fwd_ex(const flat_attn_params_t* p, void* stream);
 
 /*

@@ -18,11 +18,11 @@ def api():
     return _api
 
 
-def fused(api, Q, K, V, scale, vl=None, variant=0):
+def fused(api, Q, K, V, scale, vl=None, variant=0, causal=False):
     O = torch.full(Q.shape, float("nan"), dtype=Q.dtype, device="cuda")
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     api.flat_attn_fwd_ex(Q, K, V, O, scale, k_valid_len=None if vl is None else torch.from_numpy(vl).cuda(),
-                         status=status, variant=variant)
+                         status=status, variant=variant, causal=causal)
     torch.cuda.synchronize()
     assert int(status.item()) == 0
     return O
@@ -62,6 +62,21 @@ def test_full_size_sampled_rows(api, name, per_head):
         Of = fused(api, Qf, Kf, Vf, w.scale, None)
         check_f32(rows_of(Of, rows, w.d), ref, name + " fp32 path")
         assert bool(torch.isfinite(Of).all())
+
+
+@pytest.mark.parametrize("name,per_head", [("c2_bert_large_4k", 8), ("p_16k_d128_small", 64), ("c5_cross_masked", 16)])
+def test_full_size_causal_sampled_rows(api, name, per_head):
+    """The same shapes under the causal mask (decoder use of the path): persistent CTAs whose items end at
+    the diagonal (d = 64), per-row key limits inside the diagonal tiles, and for the cross-attention shape
+    the offset Nk - Nq together with the key-padding mask."""
+    w = inputs.WORKLOADS[name]
+    Qb, Kb, Vb = inputs.make_qkv_bf16(w)
+    vl = inputs.make_valid_len(w) if w.masked else None
+    rows = inputs.sample_rows(w, per_head)
+    ref = oracle.attention(Qb, Kb, Vb, w.scale, valid_len=vl, rows=rows, causal=True)["O"]
+    O = fused(api, bf16_tensor(Qb), bf16_tensor(Kb), bf16_tensor(Vb), w.scale, vl, causal=True)
+    check_bf16(rows_of(O, rows, w.d), ref, name + " causal")
+    assert bool(torch.isfinite(O.float()).all())
 
 
 @pytest.mark.parametrize("name,per_head", [("c4_64k_d128", 64), ("c5_cross_masked", 32)])
