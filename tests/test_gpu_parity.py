@@ -176,6 +176,43 @@ def test_causal_f32_and_naive(api):
     assert np.all(A.float().cpu().numpy()[0, 0][iu] == 0.0)
 
 
+@pytest.mark.parametrize("seed", [20240607, 7, 424242])
+def test_randomised_shapes_against_the_ffma_kernel(api, seed):
+    """Forty random problems (shape, key-padding, causal, scale, logit spread) through the dispatcher and
+    through every tensor-core variant that applies, each compared element by element with the FFMA kernel
+    (an independent implementation: different tiling, exact running maximum, no polynomial) under the
+    bf16 tolerance, and the smaller ones with the oracle as well.  Some have more than eight work
+    items per SM (the persistent grid of the d = 64 kernel), some a single key step."""
+    rng = np.random.default_rng(seed)
+    for case in range(40):
+        d = int(rng.choice([64, 64, 64, 128]))
+        big = case % 5 == 0
+        if big:
+            B, H = int(rng.integers(20, 40)), 16
+            Nq, Nk = int(rng.integers(260, 520)), int(rng.integers(1, 400))
+        else:
+            B, H = int(rng.integers(1, 4)), int(rng.integers(1, 5))
+            Nq, Nk = int(rng.integers(1, 900)), int(rng.integers(1, 1400))
+        causal = bool(rng.integers(0, 2))
+        sigma = float(rng.choice([0.5, 1.0, 2.0]))
+        scale = float(rng.choice([1 / math.sqrt(d), 0.3, -0.2]))
+        Qb, Kb = rand_bits(rng, (B, H, Nq, d), sigma), rand_bits(rng, (B, H, Nk, d), sigma)
+        Vb = rand_bits(rng, (B, H, Nk, d), 0.25)
+        vl = None
+        if rng.integers(0, 2):
+            vl = rng.integers(0, Nk + 1, size=B).astype(np.int32)
+        what = "case %d: B%d H%d Nq%d Nk%d d%d causal=%s scale=%.3g sigma=%g vl=%s" % (
+            case, B, H, Nq, Nk, d, causal, scale, sigma, None if vl is None else vl.tolist()[:6])
+        ref = run_fused_bf16(api, Qb, Kb, Vb, scale, vl=vl, variant=1, causal=causal)
+        if B * H * Nq * Nk < 3e6:
+            check_bf16(ref, oracle.attention(Qb, Kb, Vb, scale, valid_len=vl, causal=causal)["O"], what + " (ffma vs oracle)")
+        variants = [0, 3] + ([4, 5] if d == 64 else [])
+        for variant in variants:
+            got = run_fused_bf16(api, Qb, Kb, Vb, scale, vl=vl, variant=variant, causal=causal)
+            # two bf16 results, each within half the tolerance of the exact one
+            check_bf16(got, ref, what + " v%d" % variant)
+
+
 @pytest.mark.parametrize("scale", [1.0, 0.05, -0.125, 3.0, 0.0])
 def test_fused_bf16_scales_tc(api, scale):
     B, H, Nq, Nk, d = 1, 2, 256, 512, 64
