@@ -50,7 +50,9 @@ int run_fused(const flat::Problem& q, int variant, cudaStream_t st) {
             // workload), and it is taken as soon as half the SMs get a CTA.
             const int64_t ctas2 = static_cast<int64_t>((q.Nq + 255) / 256) * q.B * q.H;
             const int sms = flat::device_sm_count();
-            if (q.d == 64) v = 2 * ctas2 >= sms ? FLAT_VARIANT_TC3 : FLAT_VARIANT_TC2_SINGLE;
+            // (with eight key steps or fewer a CTA is mostly fill and drain: two single-tile CTAs per SM
+            // overlap each other's, measured 3-14 % ahead of the two-tile kernel there)
+            if (q.d == 64) v = (2 * ctas2 >= sms && q.Nk > 1024) ? FLAT_VARIANT_TC3 : FLAT_VARIANT_TC2_SINGLE;
             else           v = ctas2 >= sms ? FLAT_VARIANT_TC2 : FLAT_VARIANT_TC;
             // (the single-tile predecessor kernel has no causal mask)
             if (q.causal && v == FLAT_VARIANT_TC) v = FLAT_VARIANT_TC2;
