@@ -321,6 +321,31 @@ def test_host_entry_point(api):
     assert e.value.code == 5
 
 
+def test_cuda_graph_capture_and_replay(api):
+    """The entry points only enqueue work on the caller's stream (no allocation, no synchronisation), so a
+    launch can be captured in a CUDA graph and replayed; the replays must reproduce the direct launch bit
+    for bit.  Both default kernels: d = 64 (persistent two-threads-per-row kernel) and d = 128."""
+    for (B, H, N, d) in [(8, 16, 2304, 64), (1, 8, 4736, 128)]:
+        rng = np.random.default_rng(N)
+        Q, K, V = (bf16_tensor(rand_bits(rng, (B, H, N, d))) for _ in range(3))
+        O_direct = torch.empty_like(Q)
+        api.flat_attn_fwd(Q, K, V, O_direct, d ** -0.5)           # also warms the per-device launch set-up
+        torch.cuda.synchronize()
+        O = torch.zeros_like(Q)
+        g = torch.cuda.CUDAGraph()
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(g, stream=side):
+                api.flat_attn_fwd(Q, K, V, O, d ** -0.5, stream=side)
+        torch.cuda.current_stream().wait_stream(side)
+        for _ in range(3):
+            O.zero_()
+            g.replay()
+            torch.cuda.synchronize()
+            assert torch.equal(O.view(torch.int16), O_direct.view(torch.int16)), (B, H, N, d)
+
+
 def test_output_padding_untouched(api):
     """Canary rows around O: the kernels write exactly B*H*Nq*d elements."""
     B, H, Nq, Nk, d = 1, 3, 130, 140, 64
