@@ -51,6 +51,11 @@ extern "C" int flat_debug_set_trace3(unsigned* p) {
     return cudaMemcpyToSymbol(g_trace3, &p, sizeof(p)) == cudaSuccess ? 0 : 6;
 }
 #define TRACE3_WORDS (6 * 64 * 16)
+#ifdef FLAT_TRACE3_LIGHT
+#define TRACE_Q0 false                                 // only the arrival stamps of every warp
+#else
+#define TRACE_Q0 true
+#endif
 #define TRACE(role, iter, point)                                                              \
     do {                                                                                      \
         if (blockIdx.x == 0 && blockIdx.y == 0 && (iter) < 64)                                \
@@ -58,6 +63,7 @@ extern "C" int flat_debug_set_trace3(unsigned* p) {
     } while (0)
 #else
 #define TRACE3_WORDS 0
+#define TRACE_Q0 false
 #define TRACE(role, iter, point) do { } while (0)
 #endif
 
@@ -497,7 +503,7 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         for (int j = 0; j < ntiles; ++j, g += 2, b = (b == 0 ? 2 : b - 1)) {      // g += 2  <=>  b -= 1 (mod 3)
             // this warp's 64 logits of S(g); its 32 packed columns of P(g) go over the first half of them
             const uint32_t s_addr = tl + LY::X_COL(b) + h * HN;
-            if (q == 0 && lane == 0) TRACE(trole, j, 0);
+            if (TRACE_Q0 && q == 0 && lane == 0) TRACE(trole, j, 0);
             const uint32_t xph = static_cast<uint32_t>(g / 6) & 1u;   // phase parity of this tile's use of the buffer
             // A warp whose wait fails does not leave by itself: it goes on to the next vote with its
             // partner (reading TMEM that may not be ready is harmless, nothing is stored), so that the
@@ -505,7 +511,7 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             ok = bounded_wait_s(bars_s + 8 * (LY::S_FULL + t * 3 + b), xph, abort_s, status, 0x300 + t);
             ok = __all_sync(0xffffffffu, ok);
             tc_fence_after();
-            if (q == 0 && lane == 0) TRACE(trole, j, 1);
+            if (TRACE_Q0 && q == 0 && lane == 0) TRACE(trole, j, 1);
             const int col0 = j * BN + h * HN;
             const bool tail = col0 + HN > nrow_min;      // (warp-uniform) some row has masked keys in this step
             const int nvalid = nrow > col0 ? (nrow - col0 < HN ? nrow - col0 : HN) : 0;   // per row
@@ -523,7 +529,7 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                 float lt;
                 tmem_ld_x32(s_addr, r);
                 tc_wait_ld();
-                if (q == 0 && lane == 0) TRACE(trole, j, 2);
+                if (TRACE_Q0 && q == 0 && lane == 0) TRACE(trole, j, 2);
                 if (tail) {
                     exp_pack32<true, false>(r, scale_log2e, -m_ref, nvalid, ls, pk[0]);
                     tmem_ld_x32(s_addr + 32, r);
@@ -548,10 +554,10 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                     ls[0] = lt;
                     if (xmax > 126.f) lt = INFINITY;      // the polynomial was fed an argument beyond its range
                 }
-                if (q == 0 && lane == 0) TRACE(trole, j, 3);
+                if (TRACE_Q0 && q == 0 && lane == 0) TRACE(trole, j, 3);
                 careful = pair_any(pair_id, !(lt <= OVERFLOW_SUM) || !ok);
             }
-            if (q == 0 && lane == 0) TRACE(trole, j, 4);
+            if (TRACE_Q0 && q == 0 && lane == 0) TRACE(trole, j, 4);
             if (careful) {
                 if (pair_any(pair_id, !ok)) { ok = false; break; }     // (both warps are here: j == 0 or the joint vote)
                 float mx = -INFINITY;
@@ -632,7 +638,7 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             // careful path waits for anything)
             if (careful && pair_any(pair_id, !ok)) ok = false;
             if (!ok) break;
-            if (q == 0 && lane == 0) TRACE(trole, j, 5);
+            if (TRACE_Q0 && q == 0 && lane == 0) TRACE(trole, j, 5);
             tmem_st_x16(s_addr, pk[0]);
             tmem_st_x16(s_addr + 16, pk[1]);
             l += (ls[0] + ls[1]) + (ls[2] + ls[3]);
@@ -640,7 +646,7 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive_s(bars_s + 8 * (LY::P_FULL + t * 3 + b));
-            if (q == 0 && lane == 0) TRACE(trole, j, 7);
+            if (TRACE_Q0 && q == 0 && lane == 0) TRACE(trole, j, 7);
             if (lane == 0) TRACE(trole, j, 8 + q);
         }
         if (ok && ntiles > 0) {
