@@ -7,9 +7,8 @@
 //   * TMEM holds O_A, O_B (64 columns each) and THREE logit buffers X0..X2 of 128 columns that the
 //     tile-steps g = 0, 1, 2, ... of the CTA (g even: tile A, g odd: tile B, key step g / 2, counted
 //     over all its work items) use in rotation; the weights P(g) overlay the logits S(g) they came
-//     from, and S(g + 3) is issued right behind the MMAs that read P(g) (same thread, so the tensor
-//     pipe keeps the order): the logits of a tile's next step are computed while the other tile's
-//     softmax runs.
+//     from, and S(g + 3) is issued as soon as the MMAs that read P(g) have completed: the logits
+//     of a tile's next step are computed while the other tile's softmax runs.
 //
 // Paper mapping (Section 5, 5.1, 5.2): shared outer loops = work items (batch, head, slab of 256
 // query rows: R-granularity), walked by min(items, SMs) persistent CTAs -- CTA c takes items c,
@@ -20,9 +19,8 @@
 //   warps 0-15  softmax: warp w serves row group q = w % 4 (TMEM lanes 32q..32q+31) of tile
 //               t = w / 8, key half h = (w / 4) % 2 of every step
 //   warp  16    TMA producer (one lane): per item the Q tiles, then K and V tiles into separate rings
-//   warp  17/18 MMA issuers (one elected lane each): O_t += P(g) V for the tile-steps of tile A / B,
-//               each followed by the logits S(g + 3) of the other tile into the buffer just read
-//   warp  19    idle (it completes the warpgroup for the register hand-over)
+//   warp  17/18 MMA issuers (one elected lane each) of O_t += P(g) V for the tile-steps of tile A / B
+//   warp  19    MMA issuer of the logits S(g) of both tiles
 // The two warps that share a row keep the same reference maximum m_ref: the first step fixes it
 // from the exact maximum of both halves (exchanged through shared memory); later steps reuse it and
 // vote, with one reducing named barrier per step, on whether either half's row sum overflowed 2^40,
@@ -334,7 +332,7 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     if (threadIdx.x == LY::SOFT_WARPS * 32) {
         for (int i = 0; i < LY::NUM_BARS; ++i)
             mbar_init(&bars[i], (i >= LY::P_FULL && i < LY::PV_DONE) ? 8               // one arrival per softmax warp of the tile
-                                : (i >= LY::K_EMPTY && i < LY::V_FULL) || (i >= LY::V_EMPTY && i < LY::S_FULL) ? 2 : 1);   // K/V_EMPTY: both issuers
+                                : (i >= LY::V_EMPTY && i < LY::S_FULL) ? 2 : 1);   // V_EMPTY: both O += P V issuers
         *abort_flag = 0;
         fence_mbar_init();
     }
@@ -406,71 +404,78 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                     drain_wait(&bars[LY::V_FULL + J % LY::VS], (J / LY::VS) & 1);
             }
         }
-      } else if (warp <= LY::SOFT_WARPS + 2) {
+      } else {
         // ------------------------------------------------------------ MMA issuers
-        // Warp 17 / 18 serves the tile-steps of tile A / B: O_t += P(g) V, then, into the buffer that
-        // these MMAs have just read (same thread: the tensor pipe keeps the order), the logits S(g + 3)
-        // of the OTHER tile.  A whole warp runs the loop (uniform control flow); one elected lane
-        // issues.  Tile-step g = 2 J + tile (J: global key step), buffer g % 3, barrier phase g / 6.
+        // Warp 17 / 18 issues O_t += P(g) V for the tile-steps of tile A / B; warp 19 issues every
+        // logit tile S(g), into buffer g % 3, once the O += P V of tile-step g - 3 (same buffer, the
+        // other tile) has read its weights.  Three warps, so that none of the three streams of MMAs
+        // queues behind a wait that belongs to another.  A whole warp runs the loop (uniform
+        // control flow); one elected lane issues.  Tile-step g = 2 J + tile
+        // (J: global key step), buffer g % 3, barrier phase g / 6.
         constexpr uint32_t IDESC_S = make_idesc_bf16(BM, BN, 0, 0);
         constexpr uint32_t IDESC_PV = make_idesc_bf16(BM, D, 0, 1);
-        const int t = warp - LY::SOFT_WARPS - 1, ts = t ^ 1;     // ts: the tile whose logits this warp issues
-        const uint64_t q_desc = make_smem_desc_sw128(smem_u32(Qs) + ts * LY::Q_BYTES, 16, 1024);
-        const uint64_t k_desc = make_smem_desc_sw128(smem_u32(Ks), 16, 1024);
-        const uint64_t v_desc = make_smem_desc_sw128(smem_u32(Vs), BN * 128, 1024);
         bool ok = true;
         auto wait = [&](int bar, uint32_t parity, int code) {
             if (ok) ok = __all_sync(0xffffffffu, bounded_wait_s(bars_s + 8 * bar, parity, abort_s, status, code));
             if (ok) tc_fence_after();
         };
-        Cursor cs, cp;                                   // where the logits / the O += P V of this warp stand
-        cursor_init(cs, sc);
-        cursor_init(cp, sc);
-        auto issue_s = [&]() {                           // S of tile ts at cursor cs, then advance it
-            if (!cs.valid || !ok) return;
-            const int g = 2 * cs.J + ts, bs = g % 3, ks = cs.J % LY::KS;
-            if (cs.j == 0) wait(LY::Q_FULL + ts, cs.q & 1, 0x200 + t);
-            wait(LY::K_FULL + ks, (cs.J / LY::KS) & 1, 0x210);
-            if (!ok) return;
-            if (elect_one()) {
-                const uint64_t kd = k_desc + static_cast<uint64_t>((ks * LY::KV_BYTES) >> 4);
+        Cursor c;
+        cursor_init(c, sc);
+        if (warp == LY::SOFT_WARPS + 3) {
+            const uint64_t q_desc = make_smem_desc_sw128(smem_u32(Qs), 16, 1024);
+            const uint64_t k_desc = make_smem_desc_sw128(smem_u32(Ks), 16, 1024);
+            while (c.valid && ok) {
+                const int ks = c.J % LY::KS;
+                wait(LY::K_FULL + ks, (c.J / LY::KS) & 1, 0x210);
 #pragma unroll
-                for (int k = 0; k < D / 16; ++k)
-                    mma_ss(tmem + LY::X_COL(bs), q_desc + static_cast<uint64_t>((k * 32) >> 4),
-                           kd + static_cast<uint64_t>((k * 32) >> 4), IDESC_S, k > 0);
-                tc_commit(&bars[LY::S_FULL + ts * 3 + bs]);
-                tc_commit(&bars[LY::K_EMPTY + ks]);       // (counts 2: both tiles' logits have used K_j)
-                if (cs.j == cs.it.ntiles - 1) tc_commit(&bars[LY::Q_EMPTY + ts]);   // the item's last use of Q_ts
-                TRACE(4, g, 1);
-            }
-            __syncwarp();
-            cursor_next(cs, sc);
-        };
-        // the first three logit tiles need no buffer to be freed: S(0), S(2) (tile A, key steps 0 and 1)
-        // come from tile B's issuer, S(1) (tile B, key step 0) from tile A's
-        issue_s();
-        if (t == 1) issue_s();
-        while (cp.valid && ok) {
-            const int g = 2 * cp.J + t, b = g % 3, vs = cp.J % LY::VS;
-            if (lane == 0) TRACE(4, g, 0);
-            wait(LY::V_FULL + vs, (cp.J / LY::VS) & 1, 0x220);
-            wait(LY::P_FULL + t * 3 + b, (g / 6) & 1, 0x221);
-            if (lane == 0) TRACE(4, g, 2);
-            if (!ok) break;
-            if (elect_one()) {
-                const uint64_t vd = v_desc + static_cast<uint64_t>((vs * LY::KV_BYTES) >> 4);
-                // the two halves of P(g) overlay the first 32 columns of each half of S(g)
+                for (int ts = 0; ts < 2; ++ts) {
+                    const int g = 2 * c.J + ts, bs = g % 3;
+                    if (c.j == 0) wait(LY::Q_FULL + ts, c.q & 1, 0x200 + ts);
+                    if (lane == 0) TRACE(4, g, 4);
+                    // buffer bs was last used by tile-step g - 3, of the other tile
+                    if (g >= 3) wait(LY::PV_DONE + (ts ^ 1) * 3 + bs, ((g - 3) / 6) & 1, 0x230 + ts);
+                    if (lane == 0) TRACE(4, g, 5);
+                    if (!ok) break;
+                    if (elect_one()) {
+                        const uint64_t qd = q_desc + static_cast<uint64_t>((ts * LY::Q_BYTES) >> 4);
+                        const uint64_t kd = k_desc + static_cast<uint64_t>((ks * LY::KV_BYTES) >> 4);
 #pragma unroll
-                for (int k = 0; k < BN / 16; ++k)
-                    mma_ts(tmem + LY::O_COL(t), tmem + LY::X_COL(b) + (k / 4) * HN + (k % 4) * 8,
-                           vd + static_cast<uint64_t>((k * 2048) >> 4), IDESC_PV, (cp.j > 0 || k > 0));
-                tc_commit(&bars[LY::PV_DONE + t * 3 + b]);
-                tc_commit(&bars[LY::V_EMPTY + vs]);
-                TRACE(4, g, 3);
+                        for (int k = 0; k < D / 16; ++k)
+                            mma_ss(tmem + LY::X_COL(bs), qd + static_cast<uint64_t>((k * 32) >> 4),
+                                   kd + static_cast<uint64_t>((k * 32) >> 4), IDESC_S, k > 0);
+                        tc_commit(&bars[LY::S_FULL + ts * 3 + bs]);
+                        if (ts == 1) tc_commit(&bars[LY::K_EMPTY + ks]);          // both tiles' logits have used K_j
+                        if (c.j == c.it.ntiles - 1) tc_commit(&bars[LY::Q_EMPTY + ts]);   // the item's last use of Q_ts
+                        TRACE(4, g, 1);
+                    }
+                    __syncwarp();
+                }
+                cursor_next(c, sc);
             }
-            __syncwarp();
-            cursor_next(cp, sc);
-            issue_s();                                   // into buffer b: 2 J_s + ts = g + 3
+        } else {
+            const int t = warp - LY::SOFT_WARPS - 1;
+            const uint64_t v_desc = make_smem_desc_sw128(smem_u32(Vs), BN * 128, 1024);
+            while (c.valid && ok) {
+                const int g = 2 * c.J + t, b = g % 3, vs = c.J % LY::VS;
+                if (lane == 0) TRACE(4, g, 0);
+                wait(LY::V_FULL + vs, (c.J / LY::VS) & 1, 0x220);
+                wait(LY::P_FULL + t * 3 + b, (g / 6) & 1, 0x221);
+                if (lane == 0) TRACE(4, g, 2);
+                if (!ok) break;
+                if (elect_one()) {
+                    const uint64_t vd = v_desc + static_cast<uint64_t>((vs * LY::KV_BYTES) >> 4);
+                    // the two halves of P(g) overlay the first 32 columns of each half of S(g)
+#pragma unroll
+                    for (int k = 0; k < BN / 16; ++k)
+                        mma_ts(tmem + LY::O_COL(t), tmem + LY::X_COL(b) + (k / 4) * HN + (k % 4) * 8,
+                               vd + static_cast<uint64_t>((k * 2048) >> 4), IDESC_PV, (c.j > 0 || k > 0));
+                    tc_commit(&bars[LY::PV_DONE + t * 3 + b]);
+                    tc_commit(&bars[LY::V_EMPTY + vs]);
+                    TRACE(4, g, 3);
+                }
+                __syncwarp();
+                cursor_next(c, sc);
+            }
         }
       }
     } else {
@@ -508,9 +513,17 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             // A warp whose wait fails does not leave by itself: it goes on to the next vote with its
             // partner (reading TMEM that may not be ready is harmless, nothing is stored), so that the
             // two always pass the same sequence of named barriers and leave together.
+#ifdef FLAT_TRACE3
+            const long long t_wait0 = clock64();
+#endif
             ok = bounded_wait_s(bars_s + 8 * (LY::S_FULL + t * 3 + b), xph, abort_s, status, 0x300 + t);
             ok = __all_sync(0xffffffffu, ok);
             tc_fence_after();
+#ifdef FLAT_TRACE3
+            if (lane == 0 && blockIdx.x == 0 && j < 64)                       // how long this warp waited for its logits
+                trace_buf[(trole * 64 + j) * 16 + 12 + q] = static_cast<unsigned>(clock64() - t_wait0);
+            if (!TRACE_Q0 && lane == 0) TRACE(trole, j, q);                   // light mode: when the logits were seen
+#endif
             if (TRACE_Q0 && q == 0 && lane == 0) TRACE(trole, j, 1);
             const int col0 = j * BN + h * HN;
             const bool tail = col0 + HN > nrow_min;      // (warp-uniform) some row has masked keys in this step
