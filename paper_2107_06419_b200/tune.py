@@ -15,6 +15,7 @@ from __future__ import annotations
 
 import argparse
 import json
+import time
 
 import torch
 
@@ -46,6 +47,11 @@ def time_variant(w, variant, steps, warmup=2):
         return None, str(e)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     torch.cuda.synchronize()
+    # let the power state of the previous variant decay (the long ones reach the power cap), then
+    # bring the clocks back up with two launches before timing
+    time.sleep(1.0)
+    for _ in range(2):
+        api.flat_attn_fwd_ex(Q, K, V, O, w.scale, k_valid_len=vl, variant=variant)
     e0.record()
     for _ in range(steps):
         api.flat_attn_fwd_ex(Q, K, V, O, w.scale, k_valid_len=vl, variant=variant)
