@@ -122,6 +122,39 @@ int flat_attn_naive_fwd(const void* Q, const void* K, const void* V, void* O, vo
 int flat_attn_naive_fwd_ex(const flat_attn_params_t* p, void* L, void* A, void* stream);
 
 /*
+ * The activation-weight operators of an attention layer (paper Section 2, "Computation
+ * operators": step 1, the Query / Key / Value projections of the input; step 5, the Output
+ * projection of the concatenated heads).  bf16 operands, fp32 accumulation, bf16 results; the
+ * paper names no bias and none is applied.  All pointers are DEVICE pointers owned by the
+ * caller, 16-byte aligned; `status` is an optional device word as in flat_attn_params_t.
+ *
+ * flat_qkv_proj_fwd:  X [B,N,Dm] row-major (Dm contiguous); Wqkv [3*H*d, Dm] row-major, its
+ *   rows being the H*d output features of Query, then Key, then Value, head by head;
+ *   Q, K, V [B,H,N,d]:   Q[b,h,n,c] = sum_k X[b,n,k] * Wqkv[h*d + c, k]   (K, V: rows offset by
+ *   H*d and 2*H*d).  One contraction; the results are written head-major, the layout the fused
+ *   attention reads.  Needs d in {64,128}, H*d a multiple of 256, Dm a multiple of 64.
+ * flat_out_proj_fwd:  O [B,H,N,d]; Wo [Dm, H*d] row-major; Y [B,N,Dm]:
+ *   Y[b,n,j] = sum_{h,c} O[b,h,n,c] * Wo[j, h*d + c].  Needs d in {64,128}, N a multiple of
+ *   128, Dm a multiple of 256.
+ * flat_attn_layer_fwd:  steps 1-5 of Section 2 for self-attention: the Q/K/V projection, the
+ *   fused Logit-softmax-Attend (flat_attn_fwd_ex with dtype BF16, no key-padding mask, `causal`
+ *   as given) and the Output projection, enqueued on `stream` in this order.  Q, K, V, O are
+ *   caller-owned device buffers of B*H*N*d bf16 elements each that hold the intermediates (the
+ *   library allocates nothing); their contents after the call are those intermediates.
+ *   Needs every condition of the two projections.
+ * Errors: FLAT_ERR_NULL / SHAPE / UNSUPPORTED / ALIGN as above; nothing is launched on an
+ * argument error.
+ */
+int flat_qkv_proj_fwd(const void* X, const void* Wqkv, void* Q, void* K, void* V,
+                      int B, int N, int H, int d, int Dm, int32_t* status, void* stream);
+int flat_out_proj_fwd(const void* O, const void* Wo, void* Y,
+                      int B, int N, int H, int d, int Dm, int32_t* status, void* stream);
+int flat_attn_layer_fwd(const void* X, const void* Wqkv, const void* Wo, void* Y,
+                        void* Q, void* K, void* V, void* O,
+                        int B, int N, int H, int d, int Dm, float scale, int causal,
+                        int32_t* status, void* stream);
+
+/*
  * End-to-end convenience call with HOST tensors: copies Q, K, V (and k_valid_len if
  * non-NULL) from host memory into `workspace`, runs the fused kernel, copies O back
  * to `O_host`, and returns without synchronising (use pinned host memory for true

@@ -99,3 +99,58 @@ def attention(Q, K, V, scale, valid_len=None, rows=None, want_logits=False, want
     if A is not None:
         out["A"] = A
     return out
+
+
+# ------------------------------------------------------------------------------------------------
+# The attention layer: Section 2, "Computation operators", steps 1-5 (Q/K/V projections, Logit,
+# softmax, Attend, Output projection).  The paper states the operators, not a number format; the
+# tensors between operators are stored as bf16 here (the storage type of the whole path), so the
+# oracle rounds Q, K, V and O to bf16 where they are stored and does everything else in double.
+
+def bf16_bits_to_f64(bits):
+    """uint16 bf16 bit patterns -> float64 (exact)."""
+    bits = np.ascontiguousarray(bits, dtype=np.uint16)
+    return (bits.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+
+
+def round_to_bf16_bits(x):
+    """float64 -> nearest bf16 (ties to even), returned as uint16 bit patterns.
+
+    Goes through float32 first (also round-to-nearest-even); a value can land one bf16 step away
+    from the directly rounded one only if it lies within 2^-29 (relative) of a bf16 tie.
+    """
+    b = np.ascontiguousarray(x, dtype=np.float64).astype(np.float32).view(np.uint32)
+    return ((b + np.uint32(0x7FFF) + ((b >> np.uint32(16)) & np.uint32(1))) >> np.uint32(16)).astype(np.uint16)
+
+
+def qkv_projection(X, Wqkv, H, d):
+    """Step 1: X [B,N,Dm], Wqkv [3*H*d, Dm] (uint16 bf16 bits; rows: Query, Key, Value features, head
+    by head) -> Q, K, V [B,H,N,d] as float64, before any rounding:  Q[b,h,n,c] = sum_k X[b,n,k] W[h*d+c, k]."""
+    B, N, Dm = X.shape
+    if Wqkv.shape != (3 * H * d, Dm):
+        raise ValueError("Wqkv must be [3*H*d, Dm]")
+    x = bf16_bits_to_f64(X).reshape(B * N, Dm)
+    w = bf16_bits_to_f64(Wqkv)
+    y = x @ w.T                                                    # [B*N, 3*H*d], double
+    y = y.reshape(B, N, 3, H, d).transpose(2, 0, 3, 1, 4)           # [3, B, H, N, d]
+    return np.ascontiguousarray(y[0]), np.ascontiguousarray(y[1]), np.ascontiguousarray(y[2])
+
+
+def out_projection(O, Wo):
+    """Step 5: O [B,H,N,d] float64, Wo [Dm, H*d] bf16 bits -> Y [B,N,Dm] float64:
+    Y[b,n,j] = sum_{h,c} O[b,h,n,c] Wo[j, h*d+c] (the heads are concatenated along the feature index)."""
+    B, H, N, d = O.shape
+    if Wo.shape[1] != H * d:
+        raise ValueError("Wo must be [Dm, H*d]")
+    o = np.ascontiguousarray(O.transpose(0, 2, 1, 3)).reshape(B * N, H * d)
+    return (o @ bf16_bits_to_f64(Wo).T).reshape(B, N, Wo.shape[0])
+
+
+def attention_layer(X, Wqkv, Wo, H, d, scale, causal=False, nthreads: int = 0):
+    """Steps 1-5 for self-attention.  Returns dict: 'Q','K','V','O' (uint16 bf16 bits, as stored
+    between the operators) and 'Y' [B,N,Dm] float64 (not rounded)."""
+    q, k, v = qkv_projection(X, Wqkv, H, d)
+    Qb, Kb, Vb = round_to_bf16_bits(q), round_to_bf16_bits(k), round_to_bf16_bits(v)
+    o = attention(Qb, Kb, Vb, scale, causal=causal, nthreads=nthreads)["O"]
+    Ob = round_to_bf16_bits(o)
+    return {"Q": Qb, "K": Kb, "V": Vb, "O": Ob, "Y": out_projection(bf16_bits_to_f64(Ob), Wo)}

@@ -29,7 +29,8 @@ FLAT_VARIANT_TC3 = 5
 EXPORTS = ["flat_attn_fwd", "flat_attn_fwd_ex", "flat_attn_naive_fwd", "flat_attn_naive_fwd_ex",
            "flat_attn_naive_fwd_static", "flat_attn_selftest_wait_timeout", "flat_attn_selftest_exp2_poly",
            "flat_attn_fwd_host", "flat_attn_host_workspace_bytes", "flat_attn_last_launch_count",
-           "flat_attn_status_string", "flat_attn_version"]
+           "flat_attn_status_string", "flat_attn_version",
+           "flat_qkv_proj_fwd", "flat_out_proj_fwd", "flat_attn_layer_fwd"]
 
 
 class flat_attn_params_t(ctypes.Structure):
@@ -57,6 +58,12 @@ _lib.flat_attn_selftest_wait_timeout.argtypes = [_vp, _vp]
 _lib.flat_attn_selftest_wait_timeout.restype = _i
 _lib.flat_attn_fwd_host.argtypes = [ctypes.POINTER(flat_attn_params_t), _vp, ctypes.c_size_t, _vp]
 _lib.flat_attn_fwd_host.restype = _i
+_lib.flat_qkv_proj_fwd.argtypes = [_vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _vp, _vp]
+_lib.flat_qkv_proj_fwd.restype = _i
+_lib.flat_out_proj_fwd.argtypes = [_vp, _vp, _vp, _i, _i, _i, _i, _i, _vp, _vp]
+_lib.flat_out_proj_fwd.restype = _i
+_lib.flat_attn_layer_fwd.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _f, _i, _vp, _vp]
+_lib.flat_attn_layer_fwd.restype = _i
 _lib.flat_attn_host_workspace_bytes.argtypes = [_i, _i, _i, _i, _i, _i]
 _lib.flat_attn_host_workspace_bytes.restype = ctypes.c_size_t
 _lib.flat_attn_last_launch_count.restype = _i
@@ -201,6 +208,47 @@ def flat_attn_selftest_wait_timeout(status, stream=None):
     if not status.is_cuda or status.dtype != torch.int32:
         raise ValueError("status must be a CUDA int32 tensor")
     _check(_lib.flat_attn_selftest_wait_timeout(_ptr(status), _stream_ptr(stream)))
+
+
+def _bf16_cuda(name, t, shape):
+    if t.dtype != torch.bfloat16 or not t.is_cuda or not t.is_contiguous() or tuple(t.shape) != tuple(shape):
+        raise ValueError("%s must be a contiguous CUDA bfloat16 tensor of shape %s" % (name, tuple(shape)))
+
+
+def flat_qkv_proj_fwd(X, Wqkv, Q, K, V, status=None, stream=None):
+    """Q/K/V projection: X [B,N,Dm], Wqkv [3*H*d, Dm] (Query, Key, Value rows, head by head) -> Q, K, V [B,H,N,d]."""
+    B, H, N, d = Q.shape
+    Dm = X.shape[2]
+    _bf16_cuda("X", X, (B, N, Dm)); _bf16_cuda("Wqkv", Wqkv, (3 * H * d, Dm))
+    for name, t in (("Q", Q), ("K", K), ("V", V)):
+        _bf16_cuda(name, t, (B, H, N, d))
+    _check(_lib.flat_qkv_proj_fwd(_ptr(X), _ptr(Wqkv), _ptr(Q), _ptr(K), _ptr(V), B, N, H, d, Dm, _ptr(status),
+                                  _stream_ptr(stream)))
+    return Q, K, V
+
+
+def flat_out_proj_fwd(O, Wo, Y, status=None, stream=None):
+    """Output projection: O [B,H,N,d], Wo [Dm, H*d] -> Y [B,N,Dm]."""
+    B, H, N, d = O.shape
+    Dm = Y.shape[2]
+    _bf16_cuda("O", O, (B, H, N, d)); _bf16_cuda("Wo", Wo, (Dm, H * d)); _bf16_cuda("Y", Y, (B, N, Dm))
+    _check(_lib.flat_out_proj_fwd(_ptr(O), _ptr(Wo), _ptr(Y), B, N, H, d, Dm, _ptr(status), _stream_ptr(stream)))
+    return Y
+
+
+def flat_attn_layer_fwd(X, Wqkv, Wo, Y, Q, K, V, O, scale, causal=False, status=None, stream=None):
+    """A self-attention layer: Q/K/V projection, fused attention, Output projection.  Q, K, V, O
+    [B,H,N,d] are caller-owned buffers for the intermediates."""
+    B, H, N, d = Q.shape
+    Dm = X.shape[2]
+    _bf16_cuda("X", X, (B, N, Dm)); _bf16_cuda("Wqkv", Wqkv, (3 * H * d, Dm)); _bf16_cuda("Wo", Wo, (Dm, H * d))
+    _bf16_cuda("Y", Y, (B, N, Dm))
+    for name, t in (("Q", Q), ("K", K), ("V", V), ("O", O)):
+        _bf16_cuda(name, t, (B, H, N, d))
+    _check(_lib.flat_attn_layer_fwd(_ptr(X), _ptr(Wqkv), _ptr(Wo), _ptr(Y), _ptr(Q), _ptr(K), _ptr(V), _ptr(O),
+                                    B, N, H, d, Dm, float(scale), 1 if causal else 0, _ptr(status),
+                                    _stream_ptr(stream)))
+    return Y
 
 
 def _check_la(p, L, A):

@@ -238,6 +238,40 @@ int flat_attn_selftest_wait_timeout(int32_t* status, void* stream) {
     return r;
 }
 
+int flat_qkv_proj_fwd(const void* X, const void* Wqkv, void* Q, void* K, void* V, int B, int N, int H, int d,
+                      int Dm, int32_t* status, void* stream) {
+    const int r = flat::launch_qkv_proj(X, Wqkv, Q, K, V, B, N, H, d, Dm, status, static_cast<cudaStream_t>(stream));
+    if (r == FLAT_OK) g_last_launches = 1;
+    return r;
+}
+
+int flat_out_proj_fwd(const void* O, const void* Wo, void* Y, int B, int N, int H, int d, int Dm, int32_t* status,
+                      void* stream) {
+    const int r = flat::launch_out_proj(O, Wo, Y, B, N, H, d, Dm, status, static_cast<cudaStream_t>(stream));
+    if (r == FLAT_OK) g_last_launches = 1;
+    return r;
+}
+
+int flat_attn_layer_fwd(const void* X, const void* Wqkv, const void* Wo, void* Y, void* Q, void* K, void* V, void* O,
+                        int B, int N, int H, int d, int Dm, float scale, int causal, int32_t* status, void* stream) {
+    if (!X || !Wqkv || !Wo || !Y || !Q || !K || !V || !O) return FLAT_ERR_NULL;
+    // validate all three steps before anything is launched
+    flat_attn_params_t p{Q, K, V, O, B, H, N, N, d, scale, FLAT_DTYPE_BF16, nullptr, status, FLAT_VARIANT_AUTO, causal};
+    flat::Problem q;
+    int rc = validate(&p, &q);
+    if (rc != FLAT_OK) return rc;
+    if ((d != 64 && d != 128) || (H * d) % 256 != 0 || Dm % 256 != 0 || N % 128 != 0) return FLAT_ERR_UNSUPPORTED;
+    if (!aligned16(X) || !aligned16(Wqkv) || !aligned16(Wo) || !aligned16(Y)) return FLAT_ERR_ALIGN;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    rc = flat::launch_qkv_proj(X, Wqkv, Q, K, V, B, N, H, d, Dm, status, st);
+    if (rc != FLAT_OK) return rc;
+    rc = run_fused(q, FLAT_VARIANT_AUTO, st);
+    if (rc != FLAT_OK) return rc;
+    rc = flat::launch_out_proj(O, Wo, Y, B, N, H, d, Dm, status, st);
+    if (rc == FLAT_OK) g_last_launches = 3;
+    return rc;
+}
+
 int flat_attn_last_launch_count(void) { return g_last_launches; }
 
 const char* flat_attn_status_string(int code) {

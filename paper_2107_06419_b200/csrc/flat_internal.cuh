@@ -28,6 +28,12 @@ int launch_fused_tc(const Problem& p, cudaStream_t st);
 int launch_fused_tc2(const Problem& p, cudaStream_t st);
 int launch_fused_tc2_single(const Problem& p, cudaStream_t st);
 int launch_fused_tc3(const Problem& p, cudaStream_t st);
+// The activation-weight operators around the fused path (proj_gemm.cu): Q/K/V projection into
+// head-major tensors and Output projection out of one.
+int launch_qkv_proj(const void* X, const void* Wqkv, void* Q, void* K, void* V, int B, int N, int H, int d, int Dm,
+                    int32_t* status, cudaStream_t st);
+int launch_out_proj(const void* O, const void* Wo, void* Y, int B, int N, int H, int d, int Dm, int32_t* status,
+                    cudaStream_t st);
 int launch_wait_timeout_selftest(int32_t* status, cudaStream_t st);
 int launch_exp2_poly_selftest(const float* x, float* y, int n, cudaStream_t st);
 // Tensor-core versions of the baseline's two contractions (bf16, d in {64,128}, Nk % 8 == 0).

@@ -25,7 +25,7 @@ def api(lib):
 def declared_functions():
     src = open(HEADER).read()
     src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
-    return sorted(set(re.findall(r"\b(flat_attn_\w+)\s*\(", src)))
+    return sorted(set(re.findall(r"\b(flat_(?:attn|qkv_proj|out_proj)_\w+)\s*\(", src)))
 
 
 def test_header_declares_and_library_exports(lib, api):
@@ -53,6 +53,36 @@ def _params(api, **kw):
     for k, v in kw.items():
         setattr(p, k, v)
     return p
+
+
+def test_projection_argument_errors(api):
+    # (no GPU needed: every case is rejected before a launch)
+    f = api._lib.flat_qkv_proj_fwd
+    ok = dict(X=0x10000, W=0x20000, Q=0x30000, K=0x40000, V=0x50000, B=2, N=256, H=4, d=64, Dm=256)
+    def qkv(**kw):
+        a = dict(ok, **kw)
+        return f(a["X"], a["W"], a["Q"], a["K"], a["V"], a["B"], a["N"], a["H"], a["d"], a["Dm"], None, None)
+    assert qkv(X=None) == 1 and qkv(V=None) == 1
+    assert qkv(B=0) == 2 and qkv(N=-1) == 2 and qkv(B=2 ** 20, N=2 ** 20) == 2
+    assert qkv(d=32) == 3 and qkv(H=3) == 3 and qkv(Dm=200) == 3        # H*d must be a multiple of 256, Dm of 64
+    assert qkv(X=0x10008) == 4
+    g = api._lib.flat_out_proj_fwd
+    def outp(**kw):
+        a = dict(dict(O=0x10000, W=0x20000, Y=0x30000, B=2, N=256, H=4, d=64, Dm=256), **kw)
+        return g(a["O"], a["W"], a["Y"], a["B"], a["N"], a["H"], a["d"], a["Dm"], None, None)
+    assert outp(Y=None) == 1 and outp(H=0) == 2
+    assert outp(N=200) == 3 and outp(Dm=320) == 3 and outp(d=16) == 3   # N multiple of 128, Dm of 256
+    assert outp(W=0x20004) == 4
+    h = api._lib.flat_attn_layer_fwd
+    def layer(**kw):
+        a = dict(dict(X=0x10000, Wqkv=0x20000, Wo=0x30000, Y=0x40000, Q=0x50000, K=0x60000, V=0x70000, O=0x80000,
+                      B=2, N=256, H=4, d=64, Dm=256, scale=0.125, causal=0), **kw)
+        return h(a["X"], a["Wqkv"], a["Wo"], a["Y"], a["Q"], a["K"], a["V"], a["O"], a["B"], a["N"], a["H"], a["d"],
+                 a["Dm"], a["scale"], a["causal"], None, None)
+    assert layer(O=None) == 1 and layer(Wo=None) == 1
+    assert layer(scale=float("nan")) == 2 and layer(B=0) == 2
+    assert layer(N=200) == 3 and layer(causal=2) == 3 and layer(H=2) == 3
+    assert layer(Y=0x40002) == 4
 
 
 @pytest.mark.parametrize("kw,code", [
