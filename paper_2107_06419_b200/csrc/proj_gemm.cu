@@ -3,17 +3,20 @@
 // Output projection of the concatenated heads back to [B,N,D].  Both are Y = A W^T with bf16
 // operands, fp32 accumulation in TMEM and bf16 results, as one persistent tcgen05 kernel:
 //   * the Q/K/V projection is ONE contraction against the stacked weights [3 H d, D]; its epilogue
-//     writes each 128 x 256 tile straight into the head-major tensors Q, K, V [B,H,N,d] that the
+//     writes each output tile straight into the head-major tensors Q, K, V [B,H,N,d] that the
 //     fused attention kernel reads (no transposition pass);
 //   * the Output projection reads its A operand straight from the head-major attention output
 //     O [B,H,N,d]: a 64-wide slice of the contraction index h * d + c is a (head, column) box of
 //     that tensor for TMA.
-// CTA = 192 threads: warps 0-3 epilogue (TMEM -> bf16 -> global), warp 4 TMA producer (one lane),
-// warp 5 MMA issuer (one elected lane).  Tiles of 128 x 256 outputs, contraction in slices of 64
-// through a four-stage ring; two accumulators of 256 TMEM columns, so the epilogue of a tile runs
-// under the MMAs of the next.  A CTA walks tiles blockIdx.x, blockIdx.x + gridDim.x, ...; tiles
-// that share their 128 rows of A are neighbours, so CTAs running together share A in L2 (the
-// weights fit L2 whole).  Every wait is bounded (tc_common.cuh).
+// CTA = 320 threads: warps 0-7 epilogue (TMEM -> bf16 -> global), warp 8 TMA producer (one lane),
+// warp 9 MMA issuer (one elected lane).  Tiles of 256 x 256 outputs as two row blocks of 128 that
+// share every 256-row tile of W (each W byte fetched feeds twice the MMAs); contraction in slices
+// of 64 through a three-stage ring (64 KB per stage); the two accumulators fill TMEM (2 x 256
+// columns), so a tile's epilogue is not overlapped with the next tile's MMAs (about a tenth of a
+// tile's time at a contraction length of 1024; tiles of 128 x 256 with two alternating
+// accumulators, which do overlap it, measured 1.6 % slower).  A CTA walks tiles blockIdx.x,
+// blockIdx.x + gridDim.x, ...; tiles that share their rows of A are neighbours, so CTAs running
+// together share A in L2 (the weights fit L2 whole).  Every wait is bounded (tc_common.cuh).
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -30,21 +33,21 @@ using namespace tc;
 
 namespace {
 
-constexpr int GM = 128;              // output rows per tile
+constexpr int GM = 256;              // output rows per tile: two MMA row blocks of 128 that share the W tile
 constexpr int GN = 256;              // output columns per tile
 constexpr int GK = 64;               // contraction slice (one 128-byte swizzle atom of bf16)
-constexpr int STAGES = 4;
-constexpr int GTHREADS = 192;
+constexpr int STAGES = 3;
+constexpr int GTHREADS = 320;        // 8 epilogue warps, TMA producer, MMA issuer
 
 struct GL {
     static constexpr int A_BYTES = GM * GK * 2;
     static constexpr int B_BYTES = GN * GK * 2;
     static constexpr int TILE_BYTES = STAGES * (A_BYTES + B_BYTES);
     static constexpr int SMEM_BYTES = TILE_BYTES + 256 + 1024;
-    static constexpr uint32_t TMEM_COLS = 512;           // two accumulators of GN columns
-    // barriers: FULL[STAGES], EMPTY[STAGES], ACC_FULL[2], ACC_EMPTY[2]
-    static constexpr int FULL = 0, EMPTY = STAGES, ACC_FULL = 2 * STAGES, ACC_EMPTY = ACC_FULL + 2;
-    static constexpr int NUM_BARS = ACC_EMPTY + 2;
+    static constexpr uint32_t TMEM_COLS = 512;           // the accumulators of the two row blocks, GN columns each
+    // barriers: FULL[STAGES], EMPTY[STAGES], ACC_FULL, ACC_EMPTY
+    static constexpr int FULL = 0, EMPTY = STAGES, ACC_FULL = 2 * STAGES, ACC_EMPTY = ACC_FULL + 1;
+    static constexpr int NUM_BARS = ACC_EMPTY + 1;
 };
 
 struct GemmArgs {
@@ -72,8 +75,8 @@ proj_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
-    if (threadIdx.x == 4 * 32) {
-        for (int i = 0; i < LY::NUM_BARS; ++i) mbar_init(&bars[i], i >= LY::ACC_EMPTY ? 4 : 1);   // four epilogue warps free an accumulator
+    if (threadIdx.x == 8 * 32) {
+        for (int i = 0; i < LY::NUM_BARS; ++i) mbar_init(&bars[i], i >= LY::ACC_EMPTY ? 8 : 1);   // eight epilogue warps free the accumulators
         *abort_flag = 0;
         fence_mbar_init();
     }
@@ -86,7 +89,7 @@ proj_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const int tiles_n = g.Nout / GN, tiles_m = (g.M + GM - 1) / GM;
     const int tiles = tiles_m * tiles_n, ksteps = g.Kdim / GK;
 
-    if (warp == 4) {
+    if (warp == 8) {
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
             prefetch_tensormap(&tmA); prefetch_tensormap(&tmW);
@@ -100,13 +103,21 @@ proj_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     if (!ok) break;
                     mbar_arrive_expect_tx(&bars[LY::FULL + s], LY::A_BYTES + LY::B_BYTES);
                     if (A_HEADS) {
-                        // rows m0.. are tokens of ONE sequence (N is a multiple of 128); slice kc of the
-                        // contraction index h * d + c lies in one head
-                        const int b = m0 / g.N, tok0 = m0 - b * g.N, k0 = kc * GK;
-                        const int h = k0 / g.d, c0 = k0 - h * g.d;
-                        tma_load_3d(As + s * LY::A_BYTES, &tmA, &bars[LY::FULL + s], c0, tok0, b * g.H + h);
+                        // each block of 128 rows holds tokens of ONE sequence (N is a multiple of 128); slice
+                        // kc of the contraction index h * d + c lies in one head.  (A block past the last
+                        // sequence has an out-of-range coordinate and reads zeros.)
+                        const int k0 = kc * GK, h = k0 / g.d, c0 = k0 - h * g.d;
+#pragma unroll
+                        for (int r = 0; r < GM / 128; ++r) {
+                            const int mr = m0 + r * 128, b = mr / g.N, tok0 = mr - b * g.N;
+                            tma_load_3d(As + s * LY::A_BYTES + r * 128 * GK * 2, &tmA, &bars[LY::FULL + s], c0, tok0,
+                                        b * g.H + h);
+                        }
                     } else {
-                        tma_load_3d(As + s * LY::A_BYTES, &tmA, &bars[LY::FULL + s], kc * GK, m0, 0);
+#pragma unroll
+                        for (int r = 0; r < GM / 128; ++r)
+                            tma_load_3d(As + s * LY::A_BYTES + r * 128 * GK * 2, &tmA, &bars[LY::FULL + s], kc * GK,
+                                        m0 + r * 128, 0);
                     }
                     tma_load_3d(Bs + s * LY::B_BYTES, &tmW, &bars[LY::FULL + s], kc * GK, n0, 0);
                     issued = it + 1;
@@ -116,18 +127,17 @@ proj_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 for (int j = issued > STAGES ? issued - STAGES : 0; j < issued; ++j)
                     drain_wait(&bars[LY::FULL + j % STAGES], (j / STAGES) & 1);
         }
-    } else if (warp == 5) {
+    } else if (warp == 9) {
         // ------------------------------------------------------------ MMA issuer
-        constexpr uint32_t IDESC = make_idesc_bf16(GM, GN, 0, 0);
+        constexpr uint32_t IDESC = make_idesc_bf16(128, GN, 0, 0);
         const uint64_t ad = make_smem_desc_sw128(smem_u32(As), 16, 1024);
         const uint64_t bd = make_smem_desc_sw128(smem_u32(Bs), 16, 1024);
         bool ok = true;
         int it = 0, tcount = 0;
         for (int tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x, ++tcount) {
-            const int ab = tcount & 1;                   // accumulator of this tile
-            // the epilogue must have read the accumulator's previous tile (two tiles ago)
-            if (tcount >= 2)
-                ok = __all_sync(0xffffffffu, bounded_wait(&bars[LY::ACC_EMPTY + ab], ((tcount >> 1) - 1) & 1, abort_flag,
+            // the epilogue must have read the accumulators of the previous tile
+            if (tcount >= 1)
+                ok = __all_sync(0xffffffffu, bounded_wait(&bars[LY::ACC_EMPTY], (tcount - 1) & 1, abort_flag,
                                                           status, 0x510));
             if (!ok) break;
             tc_fence_after();
@@ -142,26 +152,28 @@ proj_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     const uint64_t b = bd + static_cast<uint64_t>((s * LY::B_BYTES) >> 4);
 #pragma unroll
                     for (int k = 0; k < GK / 16; ++k)
-                        mma_ss(tmem + ab * GN, a + static_cast<uint64_t>((k * 32) >> 4),
-                               b + static_cast<uint64_t>((k * 32) >> 4), IDESC, (kc > 0 || k > 0));
+#pragma unroll
+                        for (int r = 0; r < GM / 128; ++r)
+                            mma_ss(tmem + r * GN, a + static_cast<uint64_t>((r * 128 * GK * 2 + k * 32) >> 4),
+                                   b + static_cast<uint64_t>((k * 32) >> 4), IDESC, (kc > 0 || k > 0));
                     tc_commit(&bars[LY::EMPTY + s]);
-                    if (kc == ksteps - 1) tc_commit(&bars[LY::ACC_FULL + ab]);
+                    if (kc == ksteps - 1) tc_commit(&bars[LY::ACC_FULL]);
                 }
                 __syncwarp();
             }
         }
     } else {
-        // ------------------------------------------------------------ epilogue (warps 0-3)
+        // ------------------------------------------------------------ epilogue (warps 0-7)
+        // warp w reads TMEM lanes 32 (w % 4) .. of row block w / 4
         bool ok = true;
         int tcount = 0;
-        const uint32_t tl = tmem + (static_cast<uint32_t>(warp * 32) << 16);
+        const int rb = warp >> 2;
+        const uint32_t tl = tmem + (static_cast<uint32_t>((warp & 3) * 32) << 16) + rb * GN;
         const int HD = g.H * g.d;
         for (int tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x, ++tcount) {
-            const int ab = tcount & 1;
             const int m0 = (tile / tiles_n) * GM, n0 = (tile % tiles_n) * GN;
             const int m = m0 + warp * 32 + lane;
-            ok = __all_sync(0xffffffffu,
-                            bounded_wait(&bars[LY::ACC_FULL + ab], (tcount >> 1) & 1, abort_flag, status, 0x530));
+            ok = __all_sync(0xffffffffu, bounded_wait(&bars[LY::ACC_FULL], tcount & 1, abort_flag, status, 0x530));
             if (!ok) break;
             tc_fence_after();
             int64_t row_off = 0;                         // element offset of this thread's row in its destination
@@ -171,13 +183,13 @@ proj_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 #pragma unroll 2
             for (int c = 0; c < GN / 32; ++c) {
                 uint32_t r[32];
-                tmem_ld_x32(tl + ab * GN + c * 32, r);
+                tmem_ld_x32(tl + c * 32, r);
                 tc_wait_ld();
                 if (c == GN / 32 - 1) {
-                    // the accumulator is in registers: the MMAs of the tile after next may overwrite it
+                    // the accumulator is in registers: the MMAs of the next tile may overwrite it
                     tc_fence_before();
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(&bars[LY::ACC_EMPTY + ab]);
+                    if (lane == 0) mbar_arrive(&bars[LY::ACC_EMPTY]);
                 }
                 __nv_bfloat16* dst;
                 if (OUT_HEADS) {
@@ -236,7 +248,7 @@ int launch_qkv_proj(const void* X, const void* Wqkv, void* Q, void* K, void* V, 
     GemmArgs g{B * N, 3 * H * d, Dm, N, H, d, static_cast<__nv_bfloat16*>(Q), static_cast<__nv_bfloat16*>(K),
                static_cast<__nv_bfloat16*>(V)};
     CUtensorMap tmA, tmW;
-    if (!make_map_2d(&tmA, X, g.M, Dm, GM) || !make_map_2d(&tmW, Wqkv, g.Nout, Dm, GN)) return FLAT_ERR_CUDA;
+    if (!make_map_2d(&tmA, X, g.M, Dm, 128) || !make_map_2d(&tmW, Wqkv, g.Nout, Dm, GN)) return FLAT_ERR_CUDA;
     return launch_gemm<false, true>(tmA, tmW, g, status, st);
 }
 
@@ -245,11 +257,11 @@ int launch_out_proj(const void* O, const void* Wo, void* Y, int B, int N, int H,
     if (!O || !Wo || !Y) return FLAT_ERR_NULL;
     if (B < 1 || N < 1 || H < 1 || Dm < 1) return FLAT_ERR_SHAPE;
     if (static_cast<int64_t>(B) * N > 0x7fffffff || static_cast<int64_t>(B) * H > 0x7fffffff) return FLAT_ERR_SHAPE;
-    if ((d != 64 && d != 128) || N % GM != 0 || Dm % GN != 0) return FLAT_ERR_UNSUPPORTED;
+    if ((d != 64 && d != 128) || N % 128 != 0 || Dm % GN != 0) return FLAT_ERR_UNSUPPORTED;
     if (!aligned16(O) || !aligned16(Wo) || !aligned16(Y)) return FLAT_ERR_ALIGN;
     GemmArgs g{B * N, Dm, H * d, N, H, d, static_cast<__nv_bfloat16*>(Y), nullptr, nullptr};
     CUtensorMap tmA, tmW;
-    if (!make_map(&tmA, O, B * H, N, d, GM) || !make_map_2d(&tmW, Wo, Dm, H * d, GN)) return FLAT_ERR_CUDA;
+    if (!make_map(&tmA, O, B * H, N, d, 128) || !make_map_2d(&tmW, Wo, Dm, H * d, GN)) return FLAT_ERR_CUDA;
     return launch_gemm<true, false>(tmA, tmW, g, status, st);
 }
 

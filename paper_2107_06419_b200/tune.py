@@ -7,6 +7,7 @@ variants: 64-row FFMA tiles, 128-row tensor-core CTAs (one or two per SM) and 25
 (with one or two softmax threads per row).
 
     python -m paper_2107_06419_b200.tune [--workloads c1_bert_base_512,c2_bert_large_4k,...] [--steps 10]
+    python -m paper_2107_06419_b200.tune --layer      (the attention layer around the fused path, step by step)
 
 Prints one JSON line per (workload, variant) and the winner per workload; inputs are random bf16
 (timing only -- parity is the tests' business).
@@ -80,15 +81,60 @@ def time_variant(w, variant, steps, warmup=2):
     return ms, None, e0.elapsed_time(e1) / (20 * steps)
 
 
+def time_layer(w, steps):
+    """The whole attention layer (Section 2 steps 1-5) of a self-attention workload with model width
+    H * d: times the Q/K/V projection, the fused attention, the Output projection and the layer call."""
+    dev = torch.device("cuda")
+    B, H, N, d = w.B, w.H, w.Nq, w.d
+    Dm = H * d
+    X = torch.randn(B, N, Dm, device=dev, dtype=torch.bfloat16)
+    Wqkv = (torch.randn(3 * H * d, Dm, device=dev) * Dm ** -0.5).to(torch.bfloat16)
+    Wo = (torch.randn(Dm, H * d, device=dev) * Dm ** -0.5).to(torch.bfloat16)
+    Q = torch.empty(B, H, N, d, device=dev, dtype=torch.bfloat16)
+    K, V, O = torch.empty_like(Q), torch.empty_like(Q), torch.empty_like(Q)
+    Y = torch.empty(B, N, Dm, device=dev, dtype=torch.bfloat16)
+    proj = 2.0 * B * N * Dm * H * d
+    parts = [("qkv_projection", lambda: api.flat_qkv_proj_fwd(X, Wqkv, Q, K, V), 3 * proj),
+             ("fused_attention", lambda: api.flat_attn_fwd(Q, K, V, O, w.scale), float(w.flops)),
+             ("out_projection", lambda: api.flat_out_proj_fwd(O, Wo, Y), proj),
+             ("layer", lambda: api.flat_attn_layer_fwd(X, Wqkv, Wo, Y, Q, K, V, O, w.scale), 4 * proj + w.flops)]
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for name, fn, flops in parts:
+        try:
+            for _ in range(2):
+                fn()
+        except api.FlatAttnError as e:
+            print(json.dumps({"workload": w.name, "step": name, "unsupported": str(e)}), flush=True)
+            return
+        torch.cuda.synchronize()
+        time.sleep(1.0)
+        for _ in range(2):
+            fn()
+        e0.record()
+        for _ in range(steps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / steps
+        print(json.dumps({"workload": w.name, "model_width": Dm, "step": name, "ms": round(ms, 4),
+                          "tflops": round(flops / ms / 1e9, 1)}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--workloads", default="c1_bert_base_512,c2_bert_large_4k,c3_16k,c4_64k_d128,c5_cross_masked")
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--skip-simt-above", type=float, default=2e12,
                     help="skip the FFMA variant for workloads above this many FLOP (it takes long)")
+    ap.add_argument("--layer", action="store_true",
+                    help="time the whole attention layer (projections + fused attention) instead of the variants")
     args = ap.parse_args()
     for name in args.workloads.split(","):
         w = inputs.WORKLOADS[name]
+        if args.layer:
+            if w.Nq == w.Nk and not w.masked:
+                time_layer(w, args.steps)
+            continue
         best = None
         for variant, label in VARIANTS.items():
             if variant == api.FLAT_VARIANT_SIMT and w.flops > args.skip_simt_above:
