@@ -155,6 +155,15 @@ int flat_attn_layer_fwd(const void* X, const void* Wqkv, const void* Wo, void* Y
                         int32_t* status, void* stream);
 
 /*
+ * A fully connected operator of the attention block (paper Section 2: "an attention layer, a
+ * normalization layer, followed by multiple (typically two) fully connected layers"; the FF1 / FF2
+ * of Table 2):  Y [M, Nout] = X [M, K] * W[Nout, K]^T, all row-major bf16, fp32 accumulation, no
+ * bias and no activation (the paper names none).  The same kernel as the projections.  Needs K a
+ * multiple of 64 and Nout a multiple of 256.  DEVICE pointers, 16-byte aligned; errors as above.
+ */
+int flat_fc_fwd(const void* X, const void* W, void* Y, int M, int K, int Nout, int32_t* status, void* stream);
+
+/*
  * End-to-end convenience call with HOST tensors: copies Q, K, V (and k_valid_len if
  * non-NULL) from host memory into `workspace`, runs the fused kernel, copies O back
  * to `O_host`, and returns without synchronising (use pinned host memory for true

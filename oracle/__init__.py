@@ -146,6 +146,13 @@ def out_projection(O, Wo):
     return (o @ bf16_bits_to_f64(Wo).T).reshape(B, N, Wo.shape[0])
 
 
+def fully_connected(X, W):
+    """A fully connected operator of the block (Section 2): X [..., K], W [Nout, K] bf16 bits ->
+    Y [..., Nout] float64, Y[..., j] = sum_k X[..., k] W[j, k]; no bias, no activation."""
+    x = bf16_bits_to_f64(X)
+    return (x.reshape(-1, x.shape[-1]) @ bf16_bits_to_f64(W).T).reshape(x.shape[:-1] + (W.shape[0],))
+
+
 def attention_layer(X, Wqkv, Wo, H, d, scale, causal=False, nthreads: int = 0):
     """Steps 1-5 for self-attention.  Returns dict: 'Q','K','V','O' (uint16 bf16 bits, as stored
     between the operators) and 'Y' [B,N,Dm] float64 (not rounded)."""

@@ -30,7 +30,7 @@ EXPORTS = ["flat_attn_fwd", "flat_attn_fwd_ex", "flat_attn_naive_fwd", "flat_att
            "flat_attn_naive_fwd_static", "flat_attn_selftest_wait_timeout", "flat_attn_selftest_exp2_poly",
            "flat_attn_fwd_host", "flat_attn_host_workspace_bytes", "flat_attn_last_launch_count",
            "flat_attn_status_string", "flat_attn_version",
-           "flat_qkv_proj_fwd", "flat_out_proj_fwd", "flat_attn_layer_fwd"]
+           "flat_qkv_proj_fwd", "flat_out_proj_fwd", "flat_attn_layer_fwd", "flat_fc_fwd"]
 
 
 class flat_attn_params_t(ctypes.Structure):
@@ -64,6 +64,8 @@ _lib.flat_out_proj_fwd.argtypes = [_vp, _vp, _vp, _i, _i, _i, _i, _i, _vp, _vp]
 _lib.flat_out_proj_fwd.restype = _i
 _lib.flat_attn_layer_fwd.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _f, _i, _vp, _vp]
 _lib.flat_attn_layer_fwd.restype = _i
+_lib.flat_fc_fwd.argtypes = [_vp, _vp, _vp, _i, _i, _i, _vp, _vp]
+_lib.flat_fc_fwd.restype = _i
 _lib.flat_attn_host_workspace_bytes.argtypes = [_i, _i, _i, _i, _i, _i]
 _lib.flat_attn_host_workspace_bytes.restype = ctypes.c_size_t
 _lib.flat_attn_last_launch_count.restype = _i
@@ -248,6 +250,15 @@ def flat_attn_layer_fwd(X, Wqkv, Wo, Y, Q, K, V, O, scale, causal=False, status=
     _check(_lib.flat_attn_layer_fwd(_ptr(X), _ptr(Wqkv), _ptr(Wo), _ptr(Y), _ptr(Q), _ptr(K), _ptr(V), _ptr(O),
                                     B, N, H, d, Dm, float(scale), 1 if causal else 0, _ptr(status),
                                     _stream_ptr(stream)))
+    return Y
+
+
+def flat_fc_fwd(X, W, Y, status=None, stream=None):
+    """Fully connected operator: X [..., K], W [Nout, K] -> Y [..., Nout] (bf16, no bias)."""
+    K, Nout = X.shape[-1], W.shape[0]
+    M = X.numel() // K
+    _bf16_cuda("X", X, X.shape); _bf16_cuda("W", W, (Nout, K)); _bf16_cuda("Y", Y, tuple(X.shape[:-1]) + (Nout,))
+    _check(_lib.flat_fc_fwd(_ptr(X), _ptr(W), _ptr(Y), M, K, Nout, _ptr(status), _stream_ptr(stream)))
     return Y
 
 

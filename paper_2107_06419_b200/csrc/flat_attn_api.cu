@@ -252,6 +252,12 @@ int flat_out_proj_fwd(const void* O, const void* Wo, void* Y, int B, int N, int 
     return r;
 }
 
+int flat_fc_fwd(const void* X, const void* W, void* Y, int M, int K, int Nout, int32_t* status, void* stream) {
+    const int r = flat::launch_fc(X, W, Y, M, K, Nout, status, static_cast<cudaStream_t>(stream));
+    if (r == FLAT_OK) g_last_launches = 1;
+    return r;
+}
+
 int flat_attn_layer_fwd(const void* X, const void* Wqkv, const void* Wo, void* Y, void* Q, void* K, void* V, void* O,
                         int B, int N, int H, int d, int Dm, float scale, int causal, int32_t* status, void* stream) {
     if (!X || !Wqkv || !Wo || !Y || !Q || !K || !V || !O) return FLAT_ERR_NULL;

@@ -307,7 +307,7 @@ __global__ void __launch_bounds__(L3::THREADS, 1)
 fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                  const __grid_constant__ CUtensorMap tmV, __nv_bfloat16* __restrict__ O, int H, int Nq, int Nk,
                  int items, int slabs, float scale_log2e, const int32_t* __restrict__ valid_len, int coff,
-                 int32_t* status) {
+                 int32_t* status, int wide_stores) {
     using LY = L3;
     const Sched sc{items, slabs, H, Nk, valid_len, coff};
     extern __shared__ uint8_t smem_raw[];
@@ -690,14 +690,18 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                     for (int i = 0; i < 32; ++i) r[i] = 0u;      // no valid key: O = 0
                 }
                 if (row < Nq) {
+                    uint32_t w[16];
 #pragma unroll
-                    for (int v = 0; v < 4; ++v) {
-                        uint4 w;
-                        w.x = pack_bf16x2(__uint_as_float(r[8 * v + 0]) * inv, __uint_as_float(r[8 * v + 1]) * inv);
-                        w.y = pack_bf16x2(__uint_as_float(r[8 * v + 2]) * inv, __uint_as_float(r[8 * v + 3]) * inv);
-                        w.z = pack_bf16x2(__uint_as_float(r[8 * v + 4]) * inv, __uint_as_float(r[8 * v + 5]) * inv);
-                        w.w = pack_bf16x2(__uint_as_float(r[8 * v + 6]) * inv, __uint_as_float(r[8 * v + 7]) * inv);
-                        *reinterpret_cast<uint4*>(orow + c * 32 + v * 8) = w;
+                    for (int i = 0; i < 16; ++i)
+                        w[i] = pack_bf16x2(__uint_as_float(r[2 * i]) * inv, __uint_as_float(r[2 * i + 1]) * inv);
+                    if (wide_stores) {                   // (O is 32-byte aligned)
+                        st_global_32B(orow + c * 32, *reinterpret_cast<uint32_t(*)[8]>(&w[0]));
+                        st_global_32B(orow + c * 32 + 16, *reinterpret_cast<uint32_t(*)[8]>(&w[8]));
+                    } else {
+#pragma unroll
+                        for (int v = 0; v < 4; ++v)
+                            *reinterpret_cast<uint4*>(orow + c * 32 + v * 8) =
+                                make_uint4(w[4 * v], w[4 * v + 1], w[4 * v + 2], w[4 * v + 3]);
                     }
                 }
             }
@@ -741,7 +745,8 @@ int launch_tc3(const Problem& p, cudaStream_t st) {
     fused_tc3_kernel<<<grid, LY::THREADS, LY::SMEM_BYTES, st>>>(tmQ, tmK, tmV, static_cast<__nv_bfloat16*>(p.O), p.H,
                                                                 p.Nq, p.Nk, static_cast<int>(items), slabs,
                                                                 p.scale * 1.4426950408889634f, p.k_valid_len,
-                                                                p.causal ? p.Nk - p.Nq : (1 << 30), p.status);
+                                                                p.causal ? p.Nk - p.Nq : (1 << 30), p.status,
+                                                                (reinterpret_cast<uintptr_t>(p.O) & 31) == 0 ? 1 : 0);
     return cudaGetLastError() == cudaSuccess ? FLAT_OK : FLAT_ERR_CUDA;
 }
 

@@ -56,6 +56,7 @@ struct GemmArgs {
     __nv_bfloat16* out0;             // token-major Y, or head-major Q
     __nv_bfloat16* out1;             // head-major K
     __nv_bfloat16* out2;             // head-major V
+    int wide_stores;                 // every output pointer is 32-byte aligned: 32-byte stores
 };
 
 // A_HEADS: A is the head-major tensor [B,H,N,d] (Output projection); else token-major [M, Kdim].
@@ -180,35 +181,41 @@ proj_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             int b = 0, tok = 0;
             if (OUT_HEADS) { b = m / g.N; tok = m - b * g.N; }
             else row_off = static_cast<int64_t>(m) * g.Nout + n0;
-#pragma unroll 2
+            // First the whole accumulator row goes to registers as packed bf16 (128 words), so that the
+            // accumulator is released for the next tile's MMAs before any store is issued.
+            uint32_t w[GN / 2];
+#pragma unroll
             for (int c = 0; c < GN / 32; ++c) {
                 uint32_t r[32];
                 tmem_ld_x32(tl + c * 32, r);
                 tc_wait_ld();
-                if (c == GN / 32 - 1) {
-                    // the accumulator is in registers: the MMAs of the next tile may overwrite it
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&bars[LY::ACC_EMPTY]);
-                }
-                __nv_bfloat16* dst;
-                if (OUT_HEADS) {
-                    // 32 consecutive output columns lie in one head of one of Q, K, V (32 divides d)
-                    const int n = n0 + c * 32, which = n / HD, rem = n - which * HD, h = rem / g.d, cc = rem - h * g.d;
-                    __nv_bfloat16* o = which == 0 ? g.out0 : (which == 1 ? g.out1 : g.out2);
-                    dst = o + ((static_cast<int64_t>(b) * g.H + h) * g.N + tok) * g.d + cc;
-                } else {
-                    dst = g.out0 + row_off + c * 32;
-                }
-                if (m < g.M) {
 #pragma unroll
-                    for (int v = 0; v < 4; ++v) {
-                        uint4 w;
-                        w.x = pack_bf16x2(__uint_as_float(r[8 * v + 0]), __uint_as_float(r[8 * v + 1]));
-                        w.y = pack_bf16x2(__uint_as_float(r[8 * v + 2]), __uint_as_float(r[8 * v + 3]));
-                        w.z = pack_bf16x2(__uint_as_float(r[8 * v + 4]), __uint_as_float(r[8 * v + 5]));
-                        w.w = pack_bf16x2(__uint_as_float(r[8 * v + 6]), __uint_as_float(r[8 * v + 7]));
-                        *reinterpret_cast<uint4*>(dst + v * 8) = w;
+                for (int i = 0; i < 16; ++i)
+                    w[c * 16 + i] = pack_bf16x2(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1]));
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&bars[LY::ACC_EMPTY]);
+            if (m < g.M) {
+#pragma unroll
+                for (int c = 0; c < GN / 32; ++c) {
+                    __nv_bfloat16* dst;
+                    if (OUT_HEADS) {
+                        // 32 consecutive output columns lie in one head of one of Q, K, V (32 divides d)
+                        const int n = n0 + c * 32, which = n / HD, rem = n - which * HD, h = rem / g.d, cc = rem - h * g.d;
+                        __nv_bfloat16* o = which == 0 ? g.out0 : (which == 1 ? g.out1 : g.out2);
+                        dst = o + ((static_cast<int64_t>(b) * g.H + h) * g.N + tok) * g.d + cc;
+                    } else {
+                        dst = g.out0 + row_off + c * 32;
+                    }
+                    if (g.wide_stores) {
+                        st_global_32B(dst, *reinterpret_cast<uint32_t(*)[8]>(&w[c * 16]));
+                        st_global_32B(dst + 16, *reinterpret_cast<uint32_t(*)[8]>(&w[c * 16 + 8]));
+                    } else {
+#pragma unroll
+                        for (int v = 0; v < 4; ++v)
+                            *reinterpret_cast<uint4*>(dst + v * 8) =
+                                make_uint4(w[c * 16 + 4 * v], w[c * 16 + 4 * v + 1], w[c * 16 + 4 * v + 2], w[c * 16 + 4 * v + 3]);
                     }
                 }
             }
@@ -235,6 +242,7 @@ int launch_gemm(const CUtensorMap& tmA, const CUtensorMap& tmW, const GemmArgs& 
 }
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+bool aligned32(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 31) == 0; }
 
 }  // namespace
 
@@ -246,7 +254,7 @@ int launch_qkv_proj(const void* X, const void* Wqkv, void* Q, void* K, void* V, 
     if ((d != 64 && d != 128) || (H * d) % GN != 0 || Dm % GK != 0) return FLAT_ERR_UNSUPPORTED;
     if (!aligned16(X) || !aligned16(Wqkv) || !aligned16(Q) || !aligned16(K) || !aligned16(V)) return FLAT_ERR_ALIGN;
     GemmArgs g{B * N, 3 * H * d, Dm, N, H, d, static_cast<__nv_bfloat16*>(Q), static_cast<__nv_bfloat16*>(K),
-               static_cast<__nv_bfloat16*>(V)};
+               static_cast<__nv_bfloat16*>(V), aligned32(Q) && aligned32(K) && aligned32(V)};
     CUtensorMap tmA, tmW;
     if (!make_map_2d(&tmA, X, g.M, Dm, 128) || !make_map_2d(&tmW, Wqkv, g.Nout, Dm, GN)) return FLAT_ERR_CUDA;
     return launch_gemm<false, true>(tmA, tmW, g, status, st);
@@ -259,10 +267,21 @@ int launch_out_proj(const void* O, const void* Wo, void* Y, int B, int N, int H,
     if (static_cast<int64_t>(B) * N > 0x7fffffff || static_cast<int64_t>(B) * H > 0x7fffffff) return FLAT_ERR_SHAPE;
     if ((d != 64 && d != 128) || N % 128 != 0 || Dm % GN != 0) return FLAT_ERR_UNSUPPORTED;
     if (!aligned16(O) || !aligned16(Wo) || !aligned16(Y)) return FLAT_ERR_ALIGN;
-    GemmArgs g{B * N, Dm, H * d, N, H, d, static_cast<__nv_bfloat16*>(Y), nullptr, nullptr};
+    GemmArgs g{B * N, Dm, H * d, N, H, d, static_cast<__nv_bfloat16*>(Y), nullptr, nullptr, aligned32(Y)};
     CUtensorMap tmA, tmW;
     if (!make_map(&tmA, O, B * H, N, d, 128) || !make_map_2d(&tmW, Wo, Dm, H * d, GN)) return FLAT_ERR_CUDA;
     return launch_gemm<true, false>(tmA, tmW, g, status, st);
+}
+
+int launch_fc(const void* X, const void* W, void* Y, int M, int Kdim, int Nout, int32_t* status, cudaStream_t st) {
+    if (!X || !W || !Y) return FLAT_ERR_NULL;
+    if (M < 1 || Kdim < 1 || Nout < 1) return FLAT_ERR_SHAPE;
+    if (Kdim % GK != 0 || Nout % GN != 0) return FLAT_ERR_UNSUPPORTED;
+    if (!aligned16(X) || !aligned16(W) || !aligned16(Y)) return FLAT_ERR_ALIGN;
+    GemmArgs g{M, Nout, Kdim, M, 1, 64, static_cast<__nv_bfloat16*>(Y), nullptr, nullptr, aligned32(Y)};
+    CUtensorMap tmA, tmW;
+    if (!make_map_2d(&tmA, X, M, Kdim, 128) || !make_map_2d(&tmW, W, Nout, Kdim, GN)) return FLAT_ERR_CUDA;
+    return launch_gemm<false, false>(tmA, tmW, g, status, st);
 }
 
 }  // namespace flat

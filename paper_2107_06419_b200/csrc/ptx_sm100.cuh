@@ -188,6 +188,14 @@ __device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
     asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
     return d;
 }
+// One 32-byte store (sixteen bf16) per lane: a warp whose lanes hold different rows then touches
+// every 32-byte sector once, where 16-byte stores touch each twice.  `p` must be 32-byte aligned.
+__device__ __forceinline__ void st_global_32B(void* p, const uint32_t (&w)[8]) {
+    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(p), "r"(w[0]), "r"(w[1]), "r"(w[2]),
+                 "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7])
+                 : "memory");
+}
+
 // ---------------------------------------------------------------- TMEM <-> registers (warp-collective)
 // 32x32b shape: thread t of the warp addresses TMEM lane (lane base of taddr) + t; .xN moves N
 // consecutive 32-bit columns.  A warp may only touch lanes 32*(warp_id % 4) .. +31.

@@ -94,10 +94,25 @@ def time_layer(w, steps):
     K, V, O = torch.empty_like(Q), torch.empty_like(Q), torch.empty_like(Q)
     Y = torch.empty(B, N, Dm, device=dev, dtype=torch.bfloat16)
     proj = 2.0 * B * N * Dm * H * d
+    # the two fully connected operators that follow the attention layer in a block, with the usual
+    # four-fold expansion of the model width
+    W1 = (torch.randn(4 * Dm, Dm, device=dev) * Dm ** -0.5).to(torch.bfloat16)
+    W2 = (torch.randn(Dm, 4 * Dm, device=dev) * (4 * Dm) ** -0.5).to(torch.bfloat16)
+    F1 = torch.empty(B, N, 4 * Dm, device=dev, dtype=torch.bfloat16)
+    Y2 = torch.empty_like(Y)
+
+    def block():
+        api.flat_attn_layer_fwd(X, Wqkv, Wo, Y, Q, K, V, O, w.scale)
+        api.flat_fc_fwd(Y, W1, F1)
+        api.flat_fc_fwd(F1, W2, Y2)
+
     parts = [("qkv_projection", lambda: api.flat_qkv_proj_fwd(X, Wqkv, Q, K, V), 3 * proj),
              ("fused_attention", lambda: api.flat_attn_fwd(Q, K, V, O, w.scale), float(w.flops)),
              ("out_projection", lambda: api.flat_out_proj_fwd(O, Wo, Y), proj),
-             ("layer", lambda: api.flat_attn_layer_fwd(X, Wqkv, Wo, Y, Q, K, V, O, w.scale), 4 * proj + w.flops)]
+             ("layer", lambda: api.flat_attn_layer_fwd(X, Wqkv, Wo, Y, Q, K, V, O, w.scale), 4 * proj + w.flops),
+             ("fc1", lambda: api.flat_fc_fwd(Y, W1, F1), 2.0 * B * N * Dm * 4 * Dm),
+             ("fc2", lambda: api.flat_fc_fwd(F1, W2, Y2), 2.0 * B * N * Dm * 4 * Dm),
+             ("block_gemm_operators", block, 4 * proj + w.flops + 4.0 * B * N * Dm * 4 * Dm)]
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     for name, fn, flops in parts:
         try:

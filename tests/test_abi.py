@@ -25,7 +25,7 @@ def api(lib):
 def declared_functions():
     src = open(HEADER).read()
     src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
-    return sorted(set(re.findall(r"\b(flat_(?:attn|qkv_proj|out_proj)_\w+)\s*\(", src)))
+    return sorted(set(re.findall(r"\b(flat_(?:attn|qkv_proj|out_proj|fc)_\w+)\s*\(", src)))
 
 
 def test_header_declares_and_library_exports(lib, api):
@@ -73,6 +73,11 @@ def test_projection_argument_errors(api):
     assert outp(Y=None) == 1 and outp(H=0) == 2
     assert outp(N=200) == 3 and outp(Dm=320) == 3 and outp(d=16) == 3   # N multiple of 128, Dm of 256
     assert outp(W=0x20004) == 4
+    fc = api._lib.flat_fc_fwd
+    assert fc(None, 0x20000, 0x30000, 128, 64, 256, None, None) == 1
+    assert fc(0x10000, 0x20000, 0x30000, 0, 64, 256, None, None) == 2
+    assert fc(0x10000, 0x20000, 0x30000, 128, 100, 256, None, None) == 3 and fc(0x10000, 0x20000, 0x30000, 128, 64, 128, None, None) == 3
+    assert fc(0x10000, 0x20000, 0x30008, 128, 64, 256, None, None) == 4
     h = api._lib.flat_attn_layer_fwd
     def layer(**kw):
         a = dict(dict(X=0x10000, Wqkv=0x20000, Wo=0x30000, Y=0x40000, Q=0x50000, K=0x60000, V=0x70000, O=0x80000,

@@ -143,3 +143,19 @@ def test_full_size_layer_sampled_rows(api):
     err = np.abs(gy - y)
     assert err.max() <= BF16_MAX and err.mean() <= BF16_MEAN
     assert err.max() / np.abs(y).max() <= 2 * BF16_REL_MAX
+
+
+@pytest.mark.parametrize("shape", [(300, 64, 256), (1024, 256, 1024), (77, 192, 512)])
+def test_fully_connected(api, shape):
+    M, K, Nout = shape
+    rng = np.random.default_rng(M + K)
+    X = rand_bits(rng, (M, K)); W = rand_bits(rng, (Nout, K), sigma=K ** -0.5)
+    Y = torch.full((M, Nout), 5.0, device="cuda", dtype=torch.bfloat16)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    api.flat_fc_fwd(bf16_tensor(X), bf16_tensor(W), Y, status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    ref = oracle.fully_connected(X, W)
+    g = bf16_to_f64(Y)
+    assert np.abs(g - ref).max() <= np.abs(ref).max() * 2.0 ** -7
+    assert np.mean(g == oracle.bf16_bits_to_f64(oracle.round_to_bf16_bits(ref))) > 0.98

@@ -108,3 +108,12 @@ def test_output_projection_is_linear_in_its_weights():
     assert np.array_equal(f64(Ws), f64(W1) + f64(W2))
     y = oracle.out_projection(O, W1) + oracle.out_projection(O, W2)
     assert np.allclose(oracle.out_projection(O, Ws), y, rtol=0, atol=1e-12)
+
+
+def test_fully_connected_by_hand():
+    X = bits([[1.0, 2.0, 3.0], [0.5, -1.0, 0.0]])
+    W = bits([[1, 0, 0], [0, 1, 1], [2, 2, 2], [-1, 0, 1]])              # [Nout = 4, K = 3]
+    Y = oracle.fully_connected(X, W)
+    assert np.array_equal(Y, [[1.0, 5.0, 12.0, 2.0], [0.5, -1.0, -1.0, -0.5]])
+    # leading dimensions are kept
+    assert oracle.fully_connected(X.reshape(1, 2, 3), W).shape == (1, 2, 4)
