@@ -248,27 +248,51 @@ __device__ __forceinline__ void exp_pack32(const uint32_t (&r)[32], float scale_
 // blockIdx.x + gridDim.x, ... one after the other without draining its pipeline in between.
 struct Item {
     int bh, row0, n, ntiles;                             // n = number of keys that any row of the slab sees, ntiles = key steps
+    bool skip;                                           // an empty slot of the paired order: no rows to write either
 };
 // What every role needs to enumerate the items.
 struct Sched {
     int items, slabs, H, Nk;
     const int32_t* valid_len;
     int coff;                                            // causal mask: row r sees keys j < r + 1 + coff (coff = Nk - Nq); none: 2^30
+    int paired;                                          // items come in pairs of complementary slabs (see get_item)
 };
+// The sequence of item indices of this CTA: blockIdx.x, blockIdx.x + gridDim.x, ...; in paired mode the
+// CTA takes PAIRS of consecutive indices (2 c, 2 c + 1), (2 (c + gridDim.x), ...), ...
+__device__ __forceinline__ int first_item(const Sched& sc) { return sc.paired ? 2 * blockIdx.x : blockIdx.x; }
+__device__ __forceinline__ int next_item(int idx, const Sched& sc) {
+    return sc.paired ? ((idx & 1) ? idx - 1 + 2 * static_cast<int>(gridDim.x) : idx + 1) : idx + static_cast<int>(gridDim.x);
+}
 __device__ __forceinline__ Item get_item(int idx, const Sched& sc) {
     Item it;
-    it.bh = idx / sc.slabs;
-    int slab = idx - it.bh * sc.slabs;
-    // Under the causal mask a slab's work grows with its position, and a CTA's stride through the
-    // items (gridDim.x) may share a factor with the slabs per head, so that it would keep meeting
-    // the same few positions: rotate the order of the slabs from head to head.
-    if (sc.coff < (1 << 29)) slab = (slab + 7 * it.bh) % sc.slabs;
+    int slab;
+    bool empty = false;
+    if (sc.paired) {
+        // Under the causal mask a slab's work grows with its position.  A persistent CTA walks a fixed
+        // share of the items, so the shares must weigh the same: the slabs of a head are taken in
+        // pairs (p, slabs - 1 - p), whose key counts add up to the same total for every p, and a CTA
+        // always takes both members.  Index = head * slots + 2 p + member; with an odd number of
+        // slabs the middle one is its own partner and its second slot stays empty.
+        const int slots = (sc.slabs + 1) & ~1;
+        it.bh = idx / slots;
+        const int i = idx - it.bh * slots, p = i >> 1;
+        slab = (i & 1) ? sc.slabs - 1 - p : p;
+        empty = (i & 1) && slab == p;
+    } else {
+        it.bh = idx / sc.slabs;
+        slab = idx - it.bh * sc.slabs;
+        // (one CTA per item under the causal mask: rotate the order of the slabs from head to head, so
+        // that CTAs launched together do not all hold slabs of the same length)
+        if (sc.coff < (1 << 29)) slab = (slab + 7 * it.bh) % sc.slabs;
+    }
     it.row0 = slab * (2 * BM);
     int n = sc.Nk;
     if (sc.valid_len) { n = sc.valid_len[it.bh / sc.H]; n = n < 0 ? 0 : (n > sc.Nk ? sc.Nk : n); }
     // under the causal mask the slab's last row bounds the keys of the item
     const long long lim = static_cast<long long>(it.row0) + 2 * BM + sc.coff;
     n = lim < n ? (lim < 0 ? 0 : static_cast<int>(lim)) : n;
+    if (empty) n = 0;
+    it.skip = empty;
     it.n = n;
     it.ntiles = (n + BN - 1) / BN;
     return it;
@@ -287,18 +311,18 @@ __device__ __forceinline__ void cursor_seek(Cursor& c, const Sched& sc) {
     while (c.idx < sc.items) {
         c.it = get_item(c.idx, sc);
         if (c.it.ntiles > 0) { c.valid = true; return; }
-        c.idx += gridDim.x;
+        c.idx = next_item(c.idx, sc);
     }
 }
 __device__ __forceinline__ void cursor_init(Cursor& c, const Sched& sc) {
-    c.idx = blockIdx.x; c.j = 0; c.J = 0; c.q = 0;
+    c.idx = first_item(sc); c.j = 0; c.J = 0; c.q = 0;
     cursor_seek(c, sc);
 }
 __device__ __forceinline__ void cursor_next(Cursor& c, const Sched& sc) {
     ++c.j; ++c.J;
     if (c.j == c.it.ntiles) {
         c.j = 0; ++c.q;
-        c.idx += gridDim.x;
+        c.idx = next_item(c.idx, sc);
         cursor_seek(c, sc);
     }
 }
@@ -307,9 +331,9 @@ __global__ void __launch_bounds__(L3::THREADS, 1)
 fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                  const __grid_constant__ CUtensorMap tmV, __nv_bfloat16* __restrict__ O, int H, int Nq, int Nk,
                  int items, int slabs, float scale_log2e, const int32_t* __restrict__ valid_len, int coff,
-                 int32_t* status, int wide_stores) {
+                 int32_t* status, int wide_stores, int paired) {
     using LY = L3;
-    const Sched sc{items, slabs, H, Nk, valid_len, coff};
+    const Sched sc{items, slabs, H, Nk, valid_len, coff, paired};
     extern __shared__ uint8_t smem_raw[];
     uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* Qs = base;                                  // 2 tiles
@@ -381,7 +405,7 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                 v_issued = J + 1;
             };
             int J0 = 0, q = 0;
-            for (int idx = blockIdx.x; idx < items && ok; idx += gridDim.x) {
+            for (int idx = first_item(sc); idx < items && ok; idx = next_item(idx, sc)) {
                 const Item it = get_item(idx, sc);
                 if (it.ntiles == 0) continue;
                 load_q(0, q, it.row0, it.bh);
@@ -496,8 +520,9 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         (void)trole;
         int b = t;                                       // buffer of tile-step g = 2 J + t: g % 3
         int g = t;                                       // this tile's next tile-step (J: key steps of all items so far)
-        for (int idx = blockIdx.x; idx < items; idx += gridDim.x) {
+        for (int idx = first_item(sc); idx < items; idx = next_item(idx, sc)) {
         const Item it = get_item(idx, sc);
+        if (it.skip) continue;
         const int ntiles = it.ntiles;
         // keys this thread's row sees (all the item's keys unless the causal mask cuts the row short);
         // lane 0 has the shortest row of the warp, so its count tells whether a step needs the masked routine
@@ -741,12 +766,18 @@ int launch_tc3(const Problem& p, cudaStream_t st) {
     const int slabs = (p.Nq + 2 * BM - 1) / (2 * BM);
     const int64_t items = static_cast<int64_t>(slabs) * BH;
     const int sms = device_sm_count();
-    const int grid = static_cast<int>(items >= 8 * static_cast<int64_t>(sms) ? sms : items);
+    const bool persistent = items >= 8 * static_cast<int64_t>(sms);
+    // Persistent CTAs under the causal mask take the slabs of a head in complementary pairs, so that
+    // every CTA's share weighs the same (get_item); the item index then runs over slots, two per pair.
+    const int paired = persistent && p.causal ? 1 : 0;
+    const int64_t slots = paired ? static_cast<int64_t>((slabs + 1) & ~1) * BH : items;
+    if (slots > 0x7fffffff) return FLAT_ERR_SHAPE;
+    const int grid = static_cast<int>(persistent ? sms : items);
     fused_tc3_kernel<<<grid, LY::THREADS, LY::SMEM_BYTES, st>>>(tmQ, tmK, tmV, static_cast<__nv_bfloat16*>(p.O), p.H,
-                                                                p.Nq, p.Nk, static_cast<int>(items), slabs,
+                                                                p.Nq, p.Nk, static_cast<int>(slots), slabs,
                                                                 p.scale * 1.4426950408889634f, p.k_valid_len,
                                                                 p.causal ? p.Nk - p.Nq : (1 << 30), p.status,
-                                                                (reinterpret_cast<uintptr_t>(p.O) & 31) == 0 ? 1 : 0);
+                                                                (reinterpret_cast<uintptr_t>(p.O) & 31) == 0 ? 1 : 0, paired);
     return cudaGetLastError() == cudaSuccess ? FLAT_OK : FLAT_ERR_CUDA;
 }
 

@@ -115,6 +115,25 @@ def test_many_items_per_cta(api, variant):
     assert np.all(got[0] == 0.0)
 
 
+@pytest.mark.parametrize("shape", [(40, 16, 700, 700), (40, 16, 520, 900), (80, 16, 256, 256)],
+                         ids=["three_slabs", "three_slabs_more_keys", "one_slab"])
+def test_causal_many_items_per_cta(api, shape):
+    """The causal mask on the persistent grid of the d = 64 kernel: the slabs of a head are dealt in
+    complementary pairs; with an odd number of slabs the middle one has no partner (an empty slot that must
+    neither compute nor store), and with one slab per head every second slot is empty.  O is preset to NaN,
+    so a row that no item wrote, or that an empty slot overwrote with zeros, fails the comparison."""
+    B, H, Nq, Nk = shape
+    d = 64
+    rng = np.random.default_rng(B * Nq + Nk)
+    Qb, Kb, Vb = rand_bits(rng, (B, H, Nq, d)), rand_bits(rng, (B, H, Nk, d)), rand_bits(rng, (B, H, Nk, d))
+    vl = rng.integers(Nk // 2, Nk + 1, size=B).astype(np.int32)
+    scale = d ** -0.5
+    ref = oracle.attention(Qb, Kb, Vb, scale, valid_len=vl, causal=True)["O"]
+    for variant in (0, 5):
+        got = run_fused_bf16(api, Qb, Kb, Vb, scale, vl=vl, variant=variant, causal=True)
+        check_bf16(got, ref, "causal many items v%d" % variant)
+
+
 CAUSAL_SHAPES = [
     # B, H, Nq, Nk, d, masked
     (1, 2, 256, 256, 64, False),        # square: row i sees keys 0..i
