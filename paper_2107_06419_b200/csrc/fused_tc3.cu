@@ -71,6 +71,10 @@ constexpr int BM = 128;              // rows per query tile (two tiles per CTA)
 constexpr int BN = 128;              // keys per step
 constexpr int HN = 64;               // keys per step and softmax thread
 constexpr float OVERFLOW_SUM = 1.0995116e12f;   // 2^40: a row sum beyond this means m_ref is stale
+constexpr float UNDERFLOW_SUM = 8.6736174e-19f; // 2^-60: a first-step sum below this means a carried m_ref is far too high
+#ifndef FLAT_TC3_CARRY_REF
+#define FLAT_TC3_CARRY_REF 1
+#endif
 // Registers per thread after the hand-over: 640 threads start with 96 each; 512 * 104 + 128 * 64 uses them all.
 #ifndef FLAT_TC3_SOFT_REGS
 #define FLAT_TC3_SOFT_REGS 104
@@ -520,6 +524,12 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         (void)trole;
         int b = t;                                       // buffer of tile-step g = 2 J + t: g % 3
         int g = t;                                       // this tile's next tile-step (J: key steps of all items so far)
+        // The reference maximum is carried from item to item: any reference gives the exact softmax
+        // as long as the sums neither overflow nor vanish, and the rows of the next item mostly have
+        // logits of the same size, so its first step can skip the exact maximum too.  The first item
+        // of the CTA and items whose first step is partly masked start from an exact maximum.
+        float m_ref = -INFINITY;
+        bool first_item_done = false;
         for (int idx = first_item(sc); idx < items; idx = next_item(idx, sc)) {
         const Item it = get_item(idx, sc);
         if (it.skip) continue;
@@ -529,7 +539,9 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         const long long rlim = static_cast<long long>(it.row0) + t * BM + q * 32 + lane + 1 + sc.coff;
         const int nrow = rlim < it.n ? (rlim < 0 ? 0 : static_cast<int>(rlim)) : it.n;
         const int nrow_min = __shfl_sync(0xffffffffu, nrow, 0);
-        float m_ref = -INFINITY, l = 0.f;
+        float l = 0.f;
+        const bool exact_first = !FLAT_TC3_CARRY_REF || !first_item_done || sc.coff < (1 << 29) || it.n < BN;   // (the same for all warps)
+        first_item_done = true;
         for (int j = 0; j < ntiles; ++j, g += 2, b = (b == 0 ? 2 : b - 1)) {      // g += 2  <=>  b -= 1 (mod 3)
             // this warp's 64 logits of S(g); its 32 packed columns of P(g) go over the first half of them
             const uint32_t s_addr = tl + LY::X_COL(b) + h * HN;
@@ -560,7 +572,7 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             // two warps have voted, so the redo reads them again instead of holding them in registers.
             uint32_t pk[2][16];
             float ls[4] = {0.f, 0.f, 0.f, 0.f};
-            bool careful = (j == 0);
+            bool careful = (j == 0) && exact_first;
             if (!careful) {
                 // (the logits come in two loads of 32 so that few registers are live at a time)
                 uint32_t r[32];
@@ -593,11 +605,14 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                     if (xmax > 126.f) lt = INFINITY;      // the polynomial was fed an argument beyond its range
                 }
                 if (TRACE_Q0 && q == 0 && lane == 0) TRACE(trole, j, 3);
-                careful = pair_any(pair_id, !(lt <= OVERFLOW_SUM) || !ok);
+                // (a first step on a carried reference must also show that the reference is not far
+                // ABOVE the row's logits: its sum must not have vanished)
+                careful = pair_any(pair_id, !(lt <= OVERFLOW_SUM) || (j == 0 && !(lt >= UNDERFLOW_SUM)) || !ok);
             }
             if (TRACE_Q0 && q == 0 && lane == 0) TRACE(trole, j, 4);
             if (careful) {
                 if (pair_any(pair_id, !ok)) { ok = false; break; }     // (both warps are here: j == 0 or the joint vote)
+                if (j == 0) m_ref = -INFINITY;           // nothing accumulated yet: the item starts from its own maximum
                 float mx = -INFINITY;
                 {
                     uint32_t s[HN];

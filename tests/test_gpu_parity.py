@@ -115,6 +115,26 @@ def test_many_items_per_cta(api, variant):
     assert np.all(got[0] == 0.0)
 
 
+@pytest.mark.parametrize("variant", [0, 5], ids=["auto", "tc3"])
+def test_reference_maximum_carried_from_item_to_item(api, variant):
+    """The persistent CTAs of the d = 64 kernel start an item on the reference maximum of the item before.
+    Heads whose logits differ by orders of magnitude follow each other here, in both directions: a reference
+    far too high (the first step's sums vanish), far too low (they overflow), and moderately off (kept: the
+    weights are then tiny or large but the quotient is the same)."""
+    B, H, Nq, Nk, d = 40, 16, 512, 384, 64                  # 640 heads x 2 slabs: the persistent grid
+    rng = np.random.default_rng(77)
+    q = rng.standard_normal((B, H, Nq, d)).astype(np.float32)
+    factor = np.array([1.0, 30.0, 0.02, 6.0, 100.0, 0.3, 12.0, 0.001], dtype=np.float32)
+    q *= factor[rng.integers(0, len(factor), size=(B, H))][:, :, None, None]
+    from paper_2107_06419_b200 import inputs
+    Qb = inputs.f32_to_bf16_bits(q).reshape(q.shape)
+    Kb, Vb = rand_bits(rng, (B, H, Nk, d)), rand_bits(rng, (B, H, Nk, d), 0.25)
+    scale = 0.5
+    ref = oracle.attention(Qb, Kb, Vb, scale)["O"]
+    got = run_fused_bf16(api, Qb, Kb, Vb, scale, variant=variant)
+    check_bf16(got, ref, "carried reference v%d" % variant)
+
+
 @pytest.mark.parametrize("shape", [(40, 16, 700, 700), (40, 16, 520, 900), (80, 16, 256, 256)],
                          ids=["three_slabs", "three_slabs_more_keys", "one_slab"])
 def test_causal_many_items_per_cta(api, shape):
