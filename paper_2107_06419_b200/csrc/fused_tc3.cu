@@ -21,11 +21,14 @@
 //   warp  16    TMA producer (one lane): per item the Q tiles, then K and V tiles into separate rings
 //   warp  17/18 MMA issuers (one elected lane each) of O_t += P(g) V for the tile-steps of tile A / B
 //   warp  19    MMA issuer of the logits S(g) of both tiles
-// The two warps that share a row keep the same reference maximum m_ref: the first step fixes it
-// from the exact maximum of both halves (exchanged through shared memory); later steps reuse it and
-// vote, with one reducing named barrier per step, on whether either half's row sum overflowed 2^40,
-// in which case both redo the step with a fresh common maximum (the logits are still in TMEM: the
-// vote comes before the weights are stored over them) and O_t, l are rescaled.
+// The two warps that share a row keep the same reference maximum m_ref: the first step of the CTA's
+// first item (and of an item whose first step is partly masked) fixes it from the exact maximum of
+// both halves (exchanged through shared memory); every other step reuses the reference it has -- the
+// first step of a later item the one carried over from the item before -- and the two warps vote,
+// with one reducing named barrier per step, on whether either half's row sum overflowed 2^40 (or,
+// on a carried reference, vanished), in which case both redo the step with a fresh common maximum
+// (the logits are still in TMEM: the vote comes before the weights are stored over them) and O_t, l
+// are rescaled.
 // Every wait is bounded (see tc_common.cuh); on expiry the CTA aborts cleanly and reports a code.
 #include <cuda.h>
 #include <cuda_bf16.h>
