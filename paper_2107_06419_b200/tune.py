@@ -32,7 +32,7 @@ VARIANTS = {
 }
 
 
-def time_variant(w, variant, steps, warmup=2):
+def time_variant(w, variant, steps, warmup=2, causal=False):
     dev = torch.device("cuda")
     Q = torch.randn(w.B, w.H, w.Nq, w.d, device=dev, dtype=torch.bfloat16)
     K = torch.randn(w.B, w.H, w.Nk, w.d, device=dev, dtype=torch.bfloat16)
@@ -43,7 +43,7 @@ def time_variant(w, variant, steps, warmup=2):
         vl = torch.from_numpy(inputs.make_valid_len(w)).to(dev)
     try:
         for _ in range(warmup):
-            api.flat_attn_fwd_ex(Q, K, V, O, w.scale, k_valid_len=vl, variant=variant)
+            api.flat_attn_fwd_ex(Q, K, V, O, w.scale, k_valid_len=vl, variant=variant, causal=causal)
     except api.FlatAttnError as e:
         return None, str(e), None
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -52,10 +52,10 @@ def time_variant(w, variant, steps, warmup=2):
     # bring the clocks back up with two launches before timing
     time.sleep(1.0)
     for _ in range(2):
-        api.flat_attn_fwd_ex(Q, K, V, O, w.scale, k_valid_len=vl, variant=variant)
+        api.flat_attn_fwd_ex(Q, K, V, O, w.scale, k_valid_len=vl, variant=variant, causal=causal)
     e0.record()
     for _ in range(steps):
-        api.flat_attn_fwd_ex(Q, K, V, O, w.scale, k_valid_len=vl, variant=variant)
+        api.flat_attn_fwd_ex(Q, K, V, O, w.scale, k_valid_len=vl, variant=variant, causal=causal)
     e1.record()
     torch.cuda.synchronize()
     ms = e0.elapsed_time(e1) / steps
@@ -65,12 +65,12 @@ def time_variant(w, variant, steps, warmup=2):
     # of twenty launches gives the time the GPU itself needs
     s = torch.cuda.Stream()
     with torch.cuda.stream(s):
-        api.flat_attn_fwd_ex(Q, K, V, O, w.scale, k_valid_len=vl, variant=variant)
+        api.flat_attn_fwd_ex(Q, K, V, O, w.scale, k_valid_len=vl, variant=variant, causal=causal)
         s.synchronize()
         graph = torch.cuda.CUDAGraph()
         with torch.cuda.graph(graph, stream=s):
             for _ in range(20):
-                api.flat_attn_fwd_ex(Q, K, V, O, w.scale, k_valid_len=vl, variant=variant)
+                api.flat_attn_fwd_ex(Q, K, V, O, w.scale, k_valid_len=vl, variant=variant, causal=causal)
         graph.replay()
         s.synchronize()
         e0.record(s)
@@ -141,6 +141,8 @@ def main():
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--skip-simt-above", type=float, default=2e12,
                     help="skip the FFMA variant for workloads above this many FLOP (it takes long)")
+    ap.add_argument("--causal", action="store_true",
+                    help="time the variants under the causal mask (TFLOP/s then count the nominal, unmasked FLOP)")
     ap.add_argument("--layer", action="store_true",
                     help="time the whole attention layer (projections + fused attention) instead of the variants")
     args = ap.parse_args()
@@ -154,8 +156,10 @@ def main():
         for variant, label in VARIANTS.items():
             if variant == api.FLAT_VARIANT_SIMT and w.flops > args.skip_simt_above:
                 continue
-            ms, err, ms_graph = time_variant(w, variant, args.steps if variant != api.FLAT_VARIANT_SIMT else 2)
+            ms, err, ms_graph = time_variant(w, variant, args.steps if variant != api.FLAT_VARIANT_SIMT else 2, causal=args.causal)
             row = {"workload": name, "variant": variant, "kernel": label}
+            if args.causal:
+                row["causal"] = True
             if ms is None:
                 row["unsupported"] = err
             else:
