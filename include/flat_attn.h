@@ -122,6 +122,26 @@ int flat_attn_naive_fwd(const void* Q, const void* K, const void* V, void* O, vo
 int flat_attn_naive_fwd_ex(const flat_attn_params_t* p, void* L, void* A, void* stream);
 
 /*
+ * Fused attention over a PACKED batch of sequences of different lengths (no padding): the same
+ * operation as flat_attn_fwd_ex (paper Section 5 applied to Section 2 steps 2-4), sequence by
+ * sequence.  Q, O are [total_q, H, d] and K, V [total_k, H, d], bf16, row-major (d contiguous, then
+ * the head, then the token); sequence s owns the query tokens cu_seqlens_q[s] .. cu_seqlens_q[s+1]-1
+ * and the key tokens cu_seqlens_k[s] .. cu_seqlens_k[s+1]-1.  cu_seqlens_q / _k are DEVICE arrays
+ * of num_seqs + 1 non-decreasing int32 offsets, the first 0, the last total_q / total_k; they are
+ * read by the kernel, not by the host.  max_seqlen_q >= the longest query sequence (it sizes the
+ * grid; a larger value only adds empty work items).  causal = 1: query i of a sequence sees key j
+ * of the same sequence iff j <= i + (its key count - its query count).  A query row without any
+ * visible key gives O = 0.  The paper works on dense [B,H,N,d] batches; packing is this library's
+ * way of running its workloads' real length mixes without padding.
+ * Needs d = 64 (FLAT_ERR_UNSUPPORTED otherwise: no fallback).  All pointers are device pointers,
+ * 16-byte aligned (the offset arrays 4-byte); `status` as in flat_attn_params_t.
+ */
+int flat_attn_varlen_fwd(const void* Q, const void* K, const void* V, void* O,
+                         const int32_t* cu_seqlens_q, const int32_t* cu_seqlens_k,
+                         int num_seqs, int H, int d, long long total_q, long long total_k,
+                         int max_seqlen_q, float scale, int causal, int32_t* status, void* stream);
+
+/*
  * The activation-weight operators of an attention layer (paper Section 2, "Computation
  * operators": step 1, the Query / Key / Value projections of the input; step 5, the Output
  * projection of the concatenated heads).  bf16 operands, fp32 accumulation, bf16 results; the

@@ -161,3 +161,23 @@ def attention_layer(X, Wqkv, Wo, H, d, scale, causal=False, nthreads: int = 0):
     o = attention(Qb, Kb, Vb, scale, causal=causal, nthreads=nthreads)["O"]
     Ob = round_to_bf16_bits(o)
     return {"Q": Qb, "K": Kb, "V": Vb, "O": Ob, "Y": out_projection(bf16_bits_to_f64(Ob), Wo)}
+
+
+def attention_varlen(Q, K, V, cu_seqlens_q, cu_seqlens_k, scale, causal=False, nthreads: int = 0):
+    """Exact attention over a packed batch: Q [total_q, H, d], K, V [total_k, H, d] (uint16 bf16 bits
+    or float32); sequence s owns query tokens cu_seqlens_q[s] .. cu_seqlens_q[s+1]-1 and key tokens
+    cu_seqlens_k[s] .. cu_seqlens_k[s+1]-1.  Each sequence is the plain definition (steps 2-4 of
+    Section 2) on its own tokens; a sequence without keys gives O = 0.  Returns O [total_q, H, d] float64."""
+    cq = np.asarray(cu_seqlens_q, dtype=np.int64); ck = np.asarray(cu_seqlens_k, dtype=np.int64)
+    total_q, H, d = Q.shape
+    O = np.zeros((total_q, H, d), dtype=np.float64)
+    for s in range(len(cq) - 1):
+        q0, q1, k0, k1 = int(cq[s]), int(cq[s + 1]), int(ck[s]), int(ck[s + 1])
+        if q1 <= q0 or k1 <= k0:
+            continue
+        q = np.ascontiguousarray(Q[q0:q1].transpose(1, 0, 2))[None]      # [1, H, nq, d]
+        k = np.ascontiguousarray(K[k0:k1].transpose(1, 0, 2))[None]
+        v = np.ascontiguousarray(V[k0:k1].transpose(1, 0, 2))[None]
+        o = attention(q, k, v, scale, causal=causal, nthreads=nthreads)["O"][0]   # [H, nq, d]
+        O[q0:q1] = o.transpose(1, 0, 2)
+    return O

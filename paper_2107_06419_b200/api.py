@@ -30,7 +30,8 @@ EXPORTS = ["flat_attn_fwd", "flat_attn_fwd_ex", "flat_attn_naive_fwd", "flat_att
            "flat_attn_naive_fwd_static", "flat_attn_selftest_wait_timeout", "flat_attn_selftest_exp2_poly",
            "flat_attn_fwd_host", "flat_attn_host_workspace_bytes", "flat_attn_last_launch_count",
            "flat_attn_status_string", "flat_attn_version",
-           "flat_qkv_proj_fwd", "flat_out_proj_fwd", "flat_attn_layer_fwd", "flat_fc_fwd"]
+           "flat_qkv_proj_fwd", "flat_out_proj_fwd", "flat_attn_layer_fwd", "flat_fc_fwd",
+           "flat_attn_varlen_fwd"]
 
 
 class flat_attn_params_t(ctypes.Structure):
@@ -66,6 +67,9 @@ _lib.flat_attn_layer_fwd.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i,
 _lib.flat_attn_layer_fwd.restype = _i
 _lib.flat_fc_fwd.argtypes = [_vp, _vp, _vp, _i, _i, _i, _vp, _vp]
 _lib.flat_fc_fwd.restype = _i
+_lib.flat_attn_varlen_fwd.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, ctypes.c_longlong, ctypes.c_longlong,
+                                      _i, _f, _i, _vp, _vp]
+_lib.flat_attn_varlen_fwd.restype = _i
 _lib.flat_attn_host_workspace_bytes.argtypes = [_i, _i, _i, _i, _i, _i]
 _lib.flat_attn_host_workspace_bytes.restype = ctypes.c_size_t
 _lib.flat_attn_last_launch_count.restype = _i
@@ -260,6 +264,25 @@ def flat_fc_fwd(X, W, Y, status=None, stream=None):
     _bf16_cuda("X", X, X.shape); _bf16_cuda("W", W, (Nout, K)); _bf16_cuda("Y", Y, tuple(X.shape[:-1]) + (Nout,))
     _check(_lib.flat_fc_fwd(_ptr(X), _ptr(W), _ptr(Y), M, K, Nout, _ptr(status), _stream_ptr(stream)))
     return Y
+
+
+def flat_attn_varlen_fwd(Q, K, V, O, cu_seqlens_q, cu_seqlens_k, max_seqlen_q, scale, causal=False, status=None,
+                         stream=None):
+    """Fused attention over a packed batch: Q, O [total_q, H, d], K, V [total_k, H, d] (bf16 CUDA);
+    cu_seqlens_q / _k int32 CUDA tensors of num_seqs + 1 offsets."""
+    total_q, H, d = Q.shape
+    total_k = K.shape[0]
+    _bf16_cuda("Q", Q, (total_q, H, d)); _bf16_cuda("O", O, (total_q, H, d))
+    _bf16_cuda("K", K, (total_k, H, d)); _bf16_cuda("V", V, (total_k, H, d))
+    for name, t in (("cu_seqlens_q", cu_seqlens_q), ("cu_seqlens_k", cu_seqlens_k)):
+        if t.dtype != torch.int32 or not t.is_cuda or t.dim() != 1 or not t.is_contiguous():
+            raise ValueError(name + " must be a contiguous int32 CUDA vector")
+    if cu_seqlens_q.numel() != cu_seqlens_k.numel() or cu_seqlens_q.numel() < 2:
+        raise ValueError("cu_seqlens_q and cu_seqlens_k must have num_seqs + 1 entries each")
+    _check(_lib.flat_attn_varlen_fwd(_ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(cu_seqlens_q), _ptr(cu_seqlens_k),
+                                     cu_seqlens_q.numel() - 1, H, d, total_q, total_k, int(max_seqlen_q), float(scale),
+                                     1 if causal else 0, _ptr(status), _stream_ptr(stream)))
+    return O
 
 
 def _check_la(p, L, A):

@@ -252,6 +252,26 @@ int flat_out_proj_fwd(const void* O, const void* Wo, void* Y, int B, int N, int 
     return r;
 }
 
+int flat_attn_varlen_fwd(const void* Q, const void* K, const void* V, void* O, const int32_t* cu_seqlens_q,
+                         const int32_t* cu_seqlens_k, int num_seqs, int H, int d, long long total_q, long long total_k,
+                         int max_seqlen_q, float scale, int causal, int32_t* status, void* stream) {
+    if (!Q || !K || !V || !O || !cu_seqlens_q || !cu_seqlens_k) return FLAT_ERR_NULL;
+    if (num_seqs < 1 || H < 1 || d < 1 || total_q < 1 || total_k < 1 || max_seqlen_q < 1 || !isfinite(scale))
+        return FLAT_ERR_SHAPE;
+    if (total_q > 0x7fffffffLL || total_k > 0x7fffffffLL || max_seqlen_q > total_q ||
+        static_cast<int64_t>(num_seqs) * H > 0x7fffffffLL)
+        return FLAT_ERR_SHAPE;
+    if (d != 64 || (causal != 0 && causal != 1)) return FLAT_ERR_UNSUPPORTED;
+    if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O)) return FLAT_ERR_ALIGN;
+    if ((reinterpret_cast<uintptr_t>(cu_seqlens_q) & 3u) || (reinterpret_cast<uintptr_t>(cu_seqlens_k) & 3u) ||
+        (status && (reinterpret_cast<uintptr_t>(status) & 3u)))
+        return FLAT_ERR_ALIGN;
+    const int r = flat::launch_fused_tc3_varlen(Q, K, V, O, cu_seqlens_q, cu_seqlens_k, num_seqs, H, total_q, total_k,
+                                                max_seqlen_q, scale, causal, status, static_cast<cudaStream_t>(stream));
+    if (r == FLAT_OK) g_last_launches = 1;
+    return r;
+}
+
 int flat_fc_fwd(const void* X, const void* W, void* Y, int M, int K, int Nout, int32_t* status, void* stream) {
     const int r = flat::launch_fc(X, W, Y, M, K, Nout, status, static_cast<cudaStream_t>(stream));
     if (r == FLAT_OK) g_last_launches = 1;

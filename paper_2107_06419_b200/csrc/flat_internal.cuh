@@ -28,6 +28,10 @@ int launch_fused_tc(const Problem& p, cudaStream_t st);
 int launch_fused_tc2(const Problem& p, cudaStream_t st);
 int launch_fused_tc2_single(const Problem& p, cudaStream_t st);
 int launch_fused_tc3(const Problem& p, cudaStream_t st);
+// Packed variable-length batches (bf16, d = 64): Q, O [total_q, H, d], K, V [total_k, H, d].
+int launch_fused_tc3_varlen(const void* Q, const void* K, const void* V, void* O, const int32_t* cu_q,
+                            const int32_t* cu_k, int num_seqs, int H, int64_t total_q, int64_t total_k,
+                            int max_seqlen_q, float scale, int causal, int32_t* status, cudaStream_t st);
 // The activation-weight operators around the fused path (proj_gemm.cu): Q/K/V projection into
 // head-major tensors and Output projection out of one.
 int launch_qkv_proj(const void* X, const void* Wqkv, void* Q, void* K, void* V, int B, int N, int H, int d, int Dm,

@@ -8,6 +8,8 @@ variants: 64-row FFMA tiles, 128-row tensor-core CTAs (one or two per SM) and 25
 
     python -m paper_2107_06419_b200.tune [--workloads c1_bert_base_512,c2_bert_large_4k,...] [--steps 10]
     python -m paper_2107_06419_b200.tune --layer      (the attention layer around the fused path, step by step)
+    python -m paper_2107_06419_b200.tune --causal     (the variants under the causal mask)
+    python -m paper_2107_06419_b200.tune --varlen     (packed variable-length batches; with --causal too)
 
 Prints one JSON line per (workload, variant) and the winner per workload; inputs are random bf16
 (timing only -- parity is the tests' business).
@@ -135,6 +137,48 @@ def time_layer(w, steps):
                           "tflops": round(flops / ms / 1e9, 1)}), flush=True)
 
 
+def time_varlen(w, steps, causal):
+    """The packed variable-length entry point on the tokens of a self-attention workload: once with
+    B equal sequences (the workload itself, packed) and once with a seeded mix of lengths that adds
+    up to the same number of tokens (lengths between 1/8 and 15/8 of the workload's)."""
+    import numpy as np
+    dev = torch.device("cuda")
+    B, H, N, d = w.B, w.H, w.Nq, w.d
+    total = B * N
+    rng = np.random.default_rng(2107)
+    S = max(2 * B, 8)                                    # the mix has more, shorter and longer sequences
+    mean = total // S
+    mix = rng.integers(mean // 8, mean * 15 // 8 + 1, size=S)
+    mix = np.maximum(1, (mix * (total / mix.sum())).astype(np.int64))
+    mix[-1] += total - mix.sum()
+    Q = torch.randn(total, H, d, device=dev, dtype=torch.bfloat16)
+    K, V, O = torch.randn_like(Q), torch.randn_like(Q), torch.empty_like(Q)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for label, lens in (("equal", np.full(B, N, dtype=np.int64)), ("mixed", mix)):
+        cu = torch.from_numpy(np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)).to(dev)
+        flops = 4.0 * H * d * float((lens.astype(np.float64) ** 2).sum())
+        fn = lambda: api.flat_attn_varlen_fwd(Q, K, V, O, cu, cu, int(lens.max()), w.scale, causal=causal)
+        try:
+            for _ in range(2):
+                fn()
+        except api.FlatAttnError as e:
+            print(json.dumps({"workload": w.name, "varlen": label, "unsupported": str(e)}), flush=True)
+            return
+        torch.cuda.synchronize()
+        time.sleep(1.0)
+        for _ in range(2):
+            fn()
+        e0.record()
+        for _ in range(steps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / steps
+        print(json.dumps({"workload": w.name, "varlen": label, "sequences": int(len(lens)), "longest": int(lens.max()),
+                          "shortest": int(lens.min()), "causal": causal, "ms": round(ms, 4),
+                          "tflops_nominal": round(flops / ms / 1e9, 1)}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--workloads", default="c1_bert_base_512,c2_bert_large_4k,c3_16k,c4_64k_d128,c5_cross_masked")
@@ -143,11 +187,17 @@ def main():
                     help="skip the FFMA variant for workloads above this many FLOP (it takes long)")
     ap.add_argument("--causal", action="store_true",
                     help="time the variants under the causal mask (TFLOP/s then count the nominal, unmasked FLOP)")
+    ap.add_argument("--varlen", action="store_true",
+                    help="time the packed variable-length entry point (equal lengths and a seeded mix)")
     ap.add_argument("--layer", action="store_true",
                     help="time the whole attention layer (projections + fused attention) instead of the variants")
     args = ap.parse_args()
     for name in args.workloads.split(","):
         w = inputs.WORKLOADS[name]
+        if args.varlen:
+            if w.Nq == w.Nk and not w.masked:
+                time_varlen(w, args.steps, args.causal)
+            continue
         if args.layer:
             if w.Nq == w.Nk and not w.masked:
                 time_layer(w, args.steps)
