@@ -133,8 +133,9 @@ int flat_attn_naive_fwd_ex(const flat_attn_params_t* p, void* L, void* A, void* 
  * of the same sequence iff j <= i + (its key count - its query count).  A query row without any
  * visible key gives O = 0.  The paper works on dense [B,H,N,d] batches; packing is this library's
  * way of running its workloads' real length mixes without padding.
- * Needs d = 64 (FLAT_ERR_UNSUPPORTED otherwise: no fallback).  All pointers are device pointers,
- * 16-byte aligned (the offset arrays 4-byte); `status` as in flat_attn_params_t.
+ * Needs d in {64, 128} (FLAT_ERR_UNSUPPORTED otherwise: no fallback) and, at d = 128,
+ * num_seqs * H <= 65535.  All pointers are device pointers, 16-byte aligned (the offset arrays
+ * 4-byte); `status` as in flat_attn_params_t.
  */
 int flat_attn_varlen_fwd(const void* Q, const void* K, const void* V, void* O,
                          const int32_t* cu_seqlens_q, const int32_t* cu_seqlens_k,

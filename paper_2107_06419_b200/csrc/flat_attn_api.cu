@@ -261,13 +261,14 @@ int flat_attn_varlen_fwd(const void* Q, const void* K, const void* V, void* O, c
     if (total_q > 0x7fffffffLL || total_k > 0x7fffffffLL || max_seqlen_q > total_q ||
         static_cast<int64_t>(num_seqs) * H > 0x7fffffffLL)
         return FLAT_ERR_SHAPE;
-    if (d != 64 || (causal != 0 && causal != 1)) return FLAT_ERR_UNSUPPORTED;
+    if ((d != 64 && d != 128) || (causal != 0 && causal != 1)) return FLAT_ERR_UNSUPPORTED;
     if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O)) return FLAT_ERR_ALIGN;
     if ((reinterpret_cast<uintptr_t>(cu_seqlens_q) & 3u) || (reinterpret_cast<uintptr_t>(cu_seqlens_k) & 3u) ||
         (status && (reinterpret_cast<uintptr_t>(status) & 3u)))
         return FLAT_ERR_ALIGN;
-    const int r = flat::launch_fused_tc3_varlen(Q, K, V, O, cu_seqlens_q, cu_seqlens_k, num_seqs, H, total_q, total_k,
-                                                max_seqlen_q, scale, causal, status, static_cast<cudaStream_t>(stream));
+    const int r = (d == 64 ? flat::launch_fused_tc3_varlen : flat::launch_fused_tc2_varlen)(
+        Q, K, V, O, cu_seqlens_q, cu_seqlens_k, num_seqs, H, total_q, total_k, max_seqlen_q, scale, causal, status,
+        static_cast<cudaStream_t>(stream));
     if (r == FLAT_OK) g_last_launches = 1;
     return r;
 }

@@ -188,11 +188,17 @@ __device__ __forceinline__ float exp_store(const uint32_t (&s)[128], float scale
     return (l0 + l1) + (l2 + l3);
 }
 
-template <int D, int NT>
+// VL: packed variable-length batches.  Q, O are [total_q, H, d], K, V [total_k, H, d]; sequence s owns
+// tokens cu_q[s] .. cu_q[s+1] - 1 of Q and cu_k[s] .. cu_k[s+1] - 1 of K, V; the tensor maps view the
+// packed tensors as {d, H, tokens}; blockIdx.y = sequence * H + head, blockIdx.x = slab of the
+// sequence's rows (a CTA past the end of its sequence leaves at once); the causal offset is that of
+// the sequence; valid_len is unused.
+template <int D, int NT, bool VL = false>
 __global__ void __launch_bounds__(128 * NT + 128, NT == 1 ? 2 : 1)
 fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                  const __grid_constant__ CUtensorMap tmV, __nv_bfloat16* __restrict__ O, int H, int Nq, int Nk,
-                 float scale_log2e, const int32_t* __restrict__ valid_len, int coff, int32_t* status) {
+                 float scale_log2e, const int32_t* __restrict__ valid_len, int coff, int32_t* status,
+                 const int32_t* __restrict__ cu_q = nullptr, const int32_t* __restrict__ cu_k = nullptr) {
     using LY = L2<D, NT>;
 #ifdef FLAT_TRACE
     constexpr int THREADS = LY::THREADS;
@@ -217,7 +223,16 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     const int bh = blockIdx.y;
     const int row0 = blockIdx.x * (NT * BM);
     int n = Nk;
-    if (valid_len) { n = valid_len[bh / H]; n = n < 0 ? 0 : (n > Nk ? Nk : n); }
+    int head = 0, q_tok0 = 0, k_tok0 = 0, q_rows = 0;    // (packed batches only)
+    if (VL) {
+        const int s = bh / H;
+        head = bh - s * H;
+        const int q0 = cu_q[s], ql = cu_q[s + 1] - q0, k0 = cu_k[s], kl = cu_k[s + 1] - k0;
+        if (row0 >= ql) return;                          // (the whole CTA: nothing is set up yet)
+        q_tok0 = q0 + row0; k_tok0 = k0; q_rows = ql - row0;
+        n = kl < 0 ? 0 : kl;
+        if (coff < (1 << 29)) coff = kl - ql;
+    } else if (valid_len) { n = valid_len[bh / H]; n = n < 0 ? 0 : (n > Nk ? Nk : n); }
     {
         // Causal mask (coff = Nk - Nq; 2^30 = none): row r sees keys j < r + 1 + coff, so the CTA's
         // last row bounds the keys of all its rows.
@@ -260,7 +275,8 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                 mbar_arrive_expect_tx(&bars[LY::K_FULL + s], LY::KV_BYTES);
 #pragma unroll
                 for (int c = 0; c < D / 64; ++c)
-                    tma_load_3d(Ks + s * LY::KV_BYTES + c * BN * 128, &tmK, &bars[LY::K_FULL + s], c * 64, j * BN, bh);
+                    tma_load_3d(Ks + s * LY::KV_BYTES + c * BN * 128, &tmK, &bars[LY::K_FULL + s], c * 64, VL ? head : j * BN,
+                                VL ? k_tok0 + j * BN : bh);
                 k_issued = j + 1;
             };
             auto load_v = [&](int j) {
@@ -270,20 +286,21 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                 mbar_arrive_expect_tx(&bars[LY::V_FULL + s], LY::KV_BYTES);
 #pragma unroll
                 for (int c = 0; c < D / 64; ++c)
-                    tma_load_3d(Vs + s * LY::KV_BYTES + c * BN * 128, &tmV, &bars[LY::V_FULL + s], c * 64, j * BN, bh);
+                    tma_load_3d(Vs + s * LY::KV_BYTES + c * BN * 128, &tmV, &bars[LY::V_FULL + s], c * 64, VL ? head : j * BN,
+                                VL ? k_tok0 + j * BN : bh);
                 v_issued = j + 1;
             };
             mbar_arrive_expect_tx(&bars[LY::Q_FULL + 0], LY::Q_BYTES);
 #pragma unroll
             for (int c = 0; c < D / 64; ++c)
-                tma_load_3d(Qs + c * BM * 128, &tmQ, &bars[LY::Q_FULL + 0], c * 64, row0, bh);
+                tma_load_3d(Qs + c * BM * 128, &tmQ, &bars[LY::Q_FULL + 0], c * 64, VL ? head : row0, VL ? q_tok0 : bh);
             load_k(0);
             if (NT == 2) {
                 mbar_arrive_expect_tx(&bars[LY::Q_FULL + NT - 1], LY::Q_BYTES);
 #pragma unroll
                 for (int c = 0; c < D / 64; ++c)
                     tma_load_3d(Qs + (NT - 1) * LY::Q_BYTES + c * BM * 128, &tmQ, &bars[LY::Q_FULL + NT - 1], c * 64,
-                                row0 + BM, bh);
+                                VL ? head : row0 + BM, VL ? q_tok0 + BM : bh);
             }
             for (int j = 0; j < ntiles && ok; ++j) {
                 if (j + 1 < ntiles) load_k(j + 1);
@@ -496,7 +513,8 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         if (ok) {
             const float inv = l > 0.f ? 1.f / l : 0.f;
             tc_fence_after();
-            __nv_bfloat16* orow = O + (static_cast<int64_t>(bh) * Nq + row) * D;
+            __nv_bfloat16* orow = VL ? O + ((static_cast<int64_t>(q_tok0) + (row - row0)) * H + head) * D
+                                     : O + (static_cast<int64_t>(bh) * Nq + row) * D;
 #pragma unroll
             for (int c = 0; c < D / 32; ++c) {
                 uint32_t r[32];
@@ -507,7 +525,7 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
 #pragma unroll
                     for (int i = 0; i < 32; ++i) r[i] = 0u;      // no valid key: O = 0
                 }
-                if (row < Nq) {
+                if (VL ? row - row0 < q_rows : row < Nq) {
 #pragma unroll
                     for (int v = 0; v < 4; ++v) {
                         uint4 w;
@@ -549,9 +567,45 @@ int launch_tc2_d(const Problem& p, cudaStream_t st) {
     dim3 grid((p.Nq + NT * BM - 1) / (NT * BM), BH);
     kern<<<grid, LY::THREADS, LY::SMEM_BYTES, st>>>(tmQ, tmK, tmV, static_cast<__nv_bfloat16*>(p.O), p.H, p.Nq,
                                                     p.Nk, p.scale * 1.4426950408889634f, p.k_valid_len,
-                                                    p.causal ? p.Nk - p.Nq : (1 << 30), p.status);
+                                                    p.causal ? p.Nk - p.Nq : (1 << 30), p.status, nullptr, nullptr);
     return cudaGetLastError() == cudaSuccess ? FLAT_OK : FLAT_ERR_CUDA;
 }
+
+}  // namespace
+
+// A packed tensor [tokens, H, d] bf16 as a TMA tensor {d, H, tokens} with boxes of 64 features x one
+// head x box_rows tokens.
+static bool make_map_packed2(CUtensorMap* m, const void* ptr, int64_t tokens, int H, int d, int box_rows) {
+    tc::EncodeTiledFn enc = tc::get_encode_fn();
+    if (!enc) return false;
+    cuuint64_t dims[3] = {static_cast<cuuint64_t>(d), static_cast<cuuint64_t>(H), static_cast<cuuint64_t>(tokens)};
+    cuuint64_t strides[2] = {static_cast<cuuint64_t>(d) * 2, static_cast<cuuint64_t>(H) * d * 2};
+    cuuint32_t box[3] = {64, 1, static_cast<cuuint32_t>(box_rows)};
+    cuuint32_t estr[3] = {1, 1, 1};
+    return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+int launch_fused_tc2_varlen(const void* Q, const void* K, const void* V, void* O, const int32_t* cu_q,
+                            const int32_t* cu_k, int num_seqs, int H, int64_t total_q, int64_t total_k,
+                            int max_seqlen_q, float scale, int causal, int32_t* status, cudaStream_t st) {
+    constexpr int D = 128, NT = 2;
+    using LY = L2<D, NT>;
+    if (static_cast<int64_t>(num_seqs) * H > 65535) return FLAT_ERR_SHAPE;      // (grid y)
+    CUtensorMap tmQ, tmK, tmV;
+    if (!make_map_packed2(&tmQ, Q, total_q, H, D, BM) || !make_map_packed2(&tmK, K, total_k, H, D, BN) ||
+        !make_map_packed2(&tmV, V, total_k, H, D, BN))
+        return FLAT_ERR_CUDA;
+    if (!ensure_dynamic_smem<fused_tc2_kernel<D, NT, true>>(LY::SMEM_BYTES)) return FLAT_ERR_CUDA;
+    dim3 grid((max_seqlen_q + NT * BM - 1) / (NT * BM), num_seqs * H);
+    fused_tc2_kernel<D, NT, true><<<grid, LY::THREADS, LY::SMEM_BYTES, st>>>(
+        tmQ, tmK, tmV, static_cast<__nv_bfloat16*>(O), H, max_seqlen_q, 0, scale * 1.4426950408889634f, nullptr,
+        causal ? 0 : (1 << 30), status, cu_q, cu_k);
+    return cudaGetLastError() == cudaSuccess ? FLAT_OK : FLAT_ERR_CUDA;
+}
+
+namespace {
 
 // Self-test of the give-up path: one warp waits on a barrier that nothing will ever complete, with
 // a limit of about a tenth of a second.  The wait must run out, record its code and let the kernel

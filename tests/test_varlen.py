@@ -67,6 +67,9 @@ VARLEN_CASES = [
     ([100, 0, 50], [100, 30, 0], 1, False),                                # a sequence without queries, one without keys
     ([40] * 700, None, 2, False),                                          # many short sequences: the persistent grid
     ([1000, 30, 513] * 40, None, 4, True),                                 # uneven slabs, empty slots, persistent, causal
+    ([300, 1, 128, 129, 517, 256, 77], None, 2, False, 128),               # head size 128: the two-tile kernel
+    ([300, 1, 128, 129, 517, 256, 77], [300, 5, 700, 129, 517, 300, 77], 2, True, 128),
+    ([100, 0, 50, 1000], [100, 30, 0, 900], 3, True, 128),
 ]
 
 
@@ -76,9 +79,9 @@ def test_varlen_against_oracle(case):
     import torch
     from helpers import bf16_tensor, bf16_to_f64, check_bf16
     from paper_2107_06419_b200 import api
-    lq, lk, H, causal = case
+    lq, lk, H, causal = case[:4]
     lk = lq if lk is None else lk
-    d = 64
+    d = case[4] if len(case) > 4 else 64
     rng = np.random.default_rng(sum(lq) + 7 * sum(lk) + H)
     Qb, Kb, Vb = rand_bits(rng, (sum(lq), H, d)), rand_bits(rng, (sum(lk), H, d)), rand_bits(rng, (sum(lk), H, d))
     cq, ck = cu(lq), cu(lk)
@@ -105,5 +108,5 @@ def test_varlen_argument_errors():
                  a["scale"], a["causal"], None, None)
     assert call(Q=None) == 1 and call(ck=None) == 1
     assert call(S=0) == 2 and call(tq=0) == 2 and call(mq=101) == 2 and call(scale=float("inf")) == 2
-    assert call(d=128) == 3 and call(causal=3) == 3
+    assert call(d=32) == 3 and call(causal=3) == 3
     assert call(V=0x30008) == 4 and call(cq=0x50002) == 4
