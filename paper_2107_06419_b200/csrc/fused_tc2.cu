@@ -573,19 +573,6 @@ int launch_tc2_d(const Problem& p, cudaStream_t st) {
 
 }  // namespace
 
-// A packed tensor [tokens, H, d] bf16 as a TMA tensor {d, H, tokens} with boxes of 64 features x one
-// head x box_rows tokens.
-static bool make_map_packed2(CUtensorMap* m, const void* ptr, int64_t tokens, int H, int d, int box_rows) {
-    tc::EncodeTiledFn enc = tc::get_encode_fn();
-    if (!enc) return false;
-    cuuint64_t dims[3] = {static_cast<cuuint64_t>(d), static_cast<cuuint64_t>(H), static_cast<cuuint64_t>(tokens)};
-    cuuint64_t strides[2] = {static_cast<cuuint64_t>(d) * 2, static_cast<cuuint64_t>(H) * d * 2};
-    cuuint32_t box[3] = {64, 1, static_cast<cuuint32_t>(box_rows)};
-    cuuint32_t estr[3] = {1, 1, 1};
-    return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
-               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
 
 int launch_fused_tc2_varlen(const void* Q, const void* K, const void* V, void* O, const int32_t* cu_q,
                             const int32_t* cu_k, int num_seqs, int H, int64_t total_q, int64_t total_k,
@@ -594,8 +581,8 @@ int launch_fused_tc2_varlen(const void* Q, const void* K, const void* V, void* O
     using LY = L2<D, NT>;
     if (static_cast<int64_t>(num_seqs) * H > 65535) return FLAT_ERR_SHAPE;      // (grid y)
     CUtensorMap tmQ, tmK, tmV;
-    if (!make_map_packed2(&tmQ, Q, total_q, H, D, BM) || !make_map_packed2(&tmK, K, total_k, H, D, BN) ||
-        !make_map_packed2(&tmV, V, total_k, H, D, BN))
+    if (!make_map_packed(&tmQ, Q, total_q, H, D, BM) || !make_map_packed(&tmK, K, total_k, H, D, BN) ||
+        !make_map_packed(&tmV, V, total_k, H, D, BN))
         return FLAT_ERR_CUDA;
     if (!ensure_dynamic_smem<fused_tc2_kernel<D, NT, true>>(LY::SMEM_BYTES)) return FLAT_ERR_CUDA;
     dim3 grid((max_seqlen_q + NT * BM - 1) / (NT * BM), num_seqs * H);
