@@ -29,6 +29,9 @@
 // on a carried reference, vanished), in which case both redo the step with a fresh common maximum
 // (the logits are still in TMEM: the vote comes before the weights are stored over them) and O_t, l
 // are rescaled.
+// A second instantiation (VL) runs packed batches of sequences of different lengths: the tensor maps
+// then view [tokens, H, d] tensors, an item is (sequence, head, slab) and reads its sequence's
+// offsets from device arrays (see get_item).
 // Every wait is bounded (see tc_common.cuh); on expiry the CTA aborts cleanly and reports a code.
 #include <cuda.h>
 #include <cuda_bf16.h>
@@ -377,6 +380,10 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                  const int32_t* __restrict__ cu_k) {
     using LY = L3;
     const Sched sc{items, slabs, H, Nk, valid_len, coff, paired, cu_q, cu_k};
+    if (VL && static_cast<int>(gridDim.x) == items) {
+        // one CTA per slot: a slot past the end of its sequence leaves before anything is set up
+        if (get_item<VL>(blockIdx.x, sc).skip) return;
+    }
     extern __shared__ uint8_t smem_raw[];
     uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* Qs = base;                                  // 2 tiles
