@@ -68,9 +68,12 @@ enum {
                                   pipe (the default for problems that fill the GPU)            */
     FLAT_VARIANT_TC2_SINGLE = 4, /* the TC2 pipeline with one 128-row tile per CTA and two CTAs
                                   per SM: bf16, d = 64 only                                    */
-    FLAT_VARIANT_TC3 = 5       /* two tiles per CTA, the softmax of every row split over two
+    FLAT_VARIANT_TC3 = 5,      /* two tiles per CTA, the softmax of every row split over two
                                   threads (sixteen softmax warps), logit tiles computed three
                                   tile-steps ahead in rotating TMEM buffers: bf16, d = 64 only */
+    FLAT_VARIANT_RGRAN = 6     /* the paper's row-granularity dataflow taken literally: the whole
+                                  row of logits of a 128-row tile stays on chip (TMEM), two-pass
+                                  softmax over complete rows: bf16, d = 64, Nk <= 512 only      */
 };
 
 typedef struct flat_attn_params {

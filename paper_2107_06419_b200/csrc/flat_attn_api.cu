@@ -24,7 +24,7 @@ int validate(const flat_attn_params_t* p, flat::Problem* out) {
     if (bh * static_cast<int64_t>(p->Nq > p->Nk ? p->Nq : p->Nk) > lim / p->d) return FLAT_ERR_SHAPE;
     if (p->dtype != FLAT_DTYPE_BF16 && p->dtype != FLAT_DTYPE_F32) return FLAT_ERR_UNSUPPORTED;
     if (p->d != 16 && p->d != 32 && p->d != 64 && p->d != 128) return FLAT_ERR_UNSUPPORTED;
-    if (p->variant < FLAT_VARIANT_AUTO || p->variant > FLAT_VARIANT_TC3) return FLAT_ERR_UNSUPPORTED;
+    if (p->variant < FLAT_VARIANT_AUTO || p->variant > FLAT_VARIANT_RGRAN) return FLAT_ERR_UNSUPPORTED;
     if (!aligned16(p->Q) || !aligned16(p->K) || !aligned16(p->V) || !aligned16(p->O)) return FLAT_ERR_ALIGN;
     if (p->k_valid_len && (reinterpret_cast<uintptr_t>(p->k_valid_len) & 3u)) return FLAT_ERR_ALIGN;
     if (p->status && (reinterpret_cast<uintptr_t>(p->status) & 3u)) return FLAT_ERR_ALIGN;
@@ -67,6 +67,7 @@ int run_fused(const flat::Problem& q, int variant, cudaStream_t st) {
         if (!tc_applies(q) || q.d != 64) return FLAT_ERR_UNSUPPORTED;
         return flat::launch_fused_tc3(q, st);
     }
+    if (v == FLAT_VARIANT_RGRAN) return flat::launch_fused_rgran(q, st);   // (checks its own conditions)
     if (v == FLAT_VARIANT_TC || v == FLAT_VARIANT_TC2) {
         if (!tc_applies(q)) return FLAT_ERR_UNSUPPORTED;
         return v == FLAT_VARIANT_TC ? flat::launch_fused_tc(q, st) : flat::launch_fused_tc2(q, st);

@@ -28,6 +28,8 @@ int launch_fused_tc(const Problem& p, cudaStream_t st);
 int launch_fused_tc2(const Problem& p, cudaStream_t st);
 int launch_fused_tc2_single(const Problem& p, cudaStream_t st);
 int launch_fused_tc3(const Problem& p, cudaStream_t st);
+bool rgran_applies(const Problem& p);              // bf16, d = 64, Nk <= 512
+int launch_fused_rgran(const Problem& p, cudaStream_t st);
 // Packed variable-length batches (bf16; fused_tc3: d = 64, fused_tc2: d = 128): Q, O [total_q, H, d], K, V [total_k, H, d].
 int launch_fused_tc2_varlen(const void* Q, const void* K, const void* V, void* O, const int32_t* cu_q,
                             const int32_t* cu_k, int num_seqs, int H, int64_t total_q, int64_t total_k,

@@ -30,6 +30,7 @@ VARIANTS = {
     api.FLAT_VARIANT_TC2_SINGLE: "tc2_single: 128-row CTA, two per SM (d = 64)",
     api.FLAT_VARIANT_TC2: "tc2: 256-row CTA (two tiles ping-pong)",
     api.FLAT_VARIANT_TC3: "tc3: 256-row CTA, half-row softmax threads, logits three tile-steps ahead (d = 64)",
+    api.FLAT_VARIANT_RGRAN: "rgran: whole logit rows on chip, two-pass softmax (d = 64, Nk <= 512)",
     api.FLAT_VARIANT_AUTO: "auto (the dispatcher's choice)",
 }
 
