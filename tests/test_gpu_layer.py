@@ -159,3 +159,40 @@ def test_fully_connected(api, shape):
     g = bf16_to_f64(Y)
     assert np.abs(g - ref).max() <= np.abs(ref).max() * 2.0 ** -7
     assert np.mean(g == oracle.bf16_bits_to_f64(oracle.round_to_bf16_bits(ref))) > 0.98
+
+
+def test_layer_and_packed_calls_in_a_cuda_graph_on_two_streams(api):
+    """The widened entry points also only enqueue work: a layer call and a packed variable-length call are
+    captured on two streams of one graph (they run concurrently) and the replays reproduce the direct launches
+    bit for bit."""
+    rng = np.random.default_rng(404)
+    B, N, H, d, Dm = 2, 512, 8, 64, 512
+    X, Wqkv, Wo = (bf16_tensor(t) for t in make_layer(rng, B, N, H, d, Dm))
+    mk = lambda: torch.empty((B, H, N, d), device="cuda", dtype=torch.bfloat16)
+    Q, K, V, O = mk(), mk(), mk(), mk()
+    Y_direct = torch.empty((B, N, Dm), device="cuda", dtype=torch.bfloat16)
+    api.flat_attn_layer_fwd(X, Wqkv, Wo, Y_direct, Q, K, V, O, d ** -0.5, causal=True)
+    lens = np.array([300, 1, 700, 129, 64], dtype=np.int64)
+    cu = torch.from_numpy(np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)).cuda()
+    Qp, Kp, Vp = (bf16_tensor(rand_bits(rng, (int(lens.sum()), H, d))) for _ in range(3))
+    Op_direct = torch.empty_like(Qp)
+    api.flat_attn_varlen_fwd(Qp, Kp, Vp, Op_direct, cu, cu, int(lens.max()), d ** -0.5)
+    torch.cuda.synchronize()
+    Y, Op = torch.zeros_like(Y_direct), torch.zeros_like(Op_direct)
+    g = torch.cuda.CUDAGraph()
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    s1.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(s1):
+        with torch.cuda.graph(g, stream=s1):
+            s2.wait_stream(s1)
+            api.flat_attn_layer_fwd(X, Wqkv, Wo, Y, Q, K, V, O, d ** -0.5, causal=True, stream=s1)
+            with torch.cuda.stream(s2):
+                api.flat_attn_varlen_fwd(Qp, Kp, Vp, Op, cu, cu, int(lens.max()), d ** -0.5, stream=s2)
+            s1.wait_stream(s2)
+    torch.cuda.current_stream().wait_stream(s1)
+    for _ in range(3):
+        Y.zero_(); Op.zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(Y.view(torch.int16), Y_direct.view(torch.int16))
+        assert torch.equal(Op.view(torch.int16), Op_direct.view(torch.int16))
