@@ -38,7 +38,9 @@ def kernel_name(variant, w):
         return KERNEL_NAMES[variant]
     ctas = ((w.Nq + 255) // 256) * w.B * w.H            # 256-row CTAs; the dispatcher's rule with 148 SMs
     if w.d == 64:
-        return "fused_tc3_kernel" if (2 * ctas >= 148 and w.Nk > 1024) else "fused_tc2_kernel"
+        slabs_fill = 3 * 256 * ((w.Nq + 255) // 256) <= 4 * w.Nq
+        tc3 = (2 * ctas >= 148 and w.Nk > 1024) or (ctas >= 2 * 148 and not w.masked and slabs_fill)
+        return "fused_tc3_kernel" if tc3 else "fused_tc2_kernel"
     return "fused_tc2_kernel" if ctas >= 148 else "fused_tc_kernel"
 
 

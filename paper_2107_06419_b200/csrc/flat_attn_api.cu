@@ -52,7 +52,15 @@ int run_fused(const flat::Problem& q, int variant, cudaStream_t st) {
             const int sms = flat::device_sm_count();
             // (with eight key steps or fewer a CTA is mostly fill and drain: two single-tile CTAs per SM
             // overlap each other's, measured 3-14 % ahead of the two-tile kernel there)
-            if (q.d == 64) v = (2 * ctas2 >= sms && q.Nk > 1024) ? FLAT_VARIANT_TC3 : FLAT_VARIANT_TC2_SINGLE;
+            // ... unless the two-tile kernel gets at least two items per SM: it then runs its persistent
+            // grid, where fill and drain are paid once per CTA instead of once per item (measured 11-26 %
+            // ahead of the single-tile CTAs at 512 and 1024 keys).
+            // (not when the 256-row slabs would be more than a quarter padding, e.g. 128 query rows)
+            if (q.d == 64) {
+                const bool slabs_fill = 3 * 256 * static_cast<int64_t>((q.Nq + 255) / 256) <= 4 * static_cast<int64_t>(q.Nq);
+                v = ((2 * ctas2 >= sms && q.Nk > 1024) || (ctas2 >= 2 * sms && !q.k_valid_len && slabs_fill))
+                        ? FLAT_VARIANT_TC3 : FLAT_VARIANT_TC2_SINGLE;
+            }
             else           v = ctas2 >= sms ? FLAT_VARIANT_TC2 : FLAT_VARIANT_TC;
             // (the single-tile predecessor kernel has no causal mask)
             if (q.causal && v == FLAT_VARIANT_TC) v = FLAT_VARIANT_TC2;

@@ -836,7 +836,9 @@ int launch_tc3(const Problem& p, cudaStream_t st) {
     const int slabs = (p.Nq + 2 * BM - 1) / (2 * BM);
     const int64_t items = static_cast<int64_t>(slabs) * BH;
     const int sms = device_sm_count();
-    const bool persistent = items >= 8 * static_cast<int64_t>(sms);
+    // (items of equal length: two per CTA are enough for the fixed deal to pay; under a key-padding
+    // mask the items differ in length and the hardware's hand-out balances better until there are many)
+    const bool persistent = items >= (p.k_valid_len ? 8 : 2) * static_cast<int64_t>(sms);
     // Persistent CTAs under the causal mask take the slabs of a head in complementary pairs, so that
     // every CTA's share weighs the same (get_item); the item index then runs over slots, two per pair.
     const int paired = persistent && p.causal ? 1 : 0;

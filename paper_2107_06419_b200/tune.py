@@ -192,9 +192,16 @@ def main():
                     help="time the packed variable-length entry point (equal lengths and a seeded mix)")
     ap.add_argument("--layer", action="store_true",
                     help="time the whole attention layer (projections + fused attention) instead of the variants")
+    ap.add_argument("--shapes", default="",
+                    help="extra self-attention shapes B:H:N:d, comma separated (e.g. 16:16:512:64), timed after the workloads")
     args = ap.parse_args()
-    for name in args.workloads.split(","):
-        w = inputs.WORKLOADS[name]
+    todo = [inputs.WORKLOADS[name] for name in args.workloads.split(",") if name]
+    for spec in args.shapes.split(","):
+        if spec:
+            B, H, N, d = (int(x) for x in spec.split(":"))
+            todo.append(inputs.Workload("B%d_H%d_N%d_d%d" % (B, H, N, d), B, H, N, N, d))
+    for w in todo:
+        name = w.name
         if args.varlen:
             if w.Nq == w.Nk and not w.masked:
                 time_varlen(w, args.steps, args.causal)
