@@ -41,7 +41,7 @@ def kernel_name(variant, w):
         slabs_fill = 3 * 256 * ((w.Nq + 255) // 256) <= 4 * w.Nq
         tc3 = (2 * ctas >= 148 and w.Nk > 1024) or (ctas >= 2 * 148 and not w.masked and slabs_fill)
         return "fused_tc3_kernel" if tc3 else "fused_tc2_kernel"
-    return "fused_tc2_kernel" if ctas >= 148 else "fused_tc_kernel"
+    return "fused_tc2_kernel" if (ctas >= 148 or w.Nk > 256) else "fused_tc_kernel"
 
 
 def load_peaks():

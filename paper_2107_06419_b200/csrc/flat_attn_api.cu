@@ -61,7 +61,11 @@ int run_fused(const flat::Problem& q, int variant, cudaStream_t st) {
                 v = ((2 * ctas2 >= sms && q.Nk > 1024) || (ctas2 >= 2 * sms && !q.k_valid_len && slabs_fill))
                         ? FLAT_VARIANT_TC3 : FLAT_VARIANT_TC2_SINGLE;
             }
-            else           v = ctas2 >= sms ? FLAT_VARIANT_TC2 : FLAT_VARIANT_TC;
+            // d = 128: the two-tile kernel (lazy reference maximum, polynomial exp2, packed arithmetic)
+            // is ahead of its single-tile predecessor even when it leaves SMs empty (B2 H8 2048 keys:
+            // 0.037 against 0.096 ms); only tiny problems (256 keys or fewer, less than one CTA per SM)
+            // are at par or a few per cent better on the 128-row CTAs.
+            else           v = (ctas2 >= sms || q.Nk > 256) ? FLAT_VARIANT_TC2 : FLAT_VARIANT_TC;
             // (the single-tile predecessor kernel has no causal mask)
             if (q.causal && v == FLAT_VARIANT_TC) v = FLAT_VARIANT_TC2;
         }
