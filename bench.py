@@ -5,14 +5,18 @@
 
 A step is one pass of the whole hot path (TMA loads of Q/K/V tiles, both tcgen05 contractions,
 the streaming softmax, the store of O) over one batch of synthetic input -- one kernel launch.
-Prints ONE JSON line: the metric is fused-attention TFLOP/s, 4*B*H*Nq*Nk*d FLOP per call.
-With N > 1 ranks (torchrun), every rank runs the same workload on its own batch: the (batch, head)
-pairs are independent units, so there is no data-path collective (weak scaling).
+Prints ONE JSON line: the metric is fused-attention TFLOP/s, 4*B*H*Nq*Nk*d FLOP per call, on the
+headline workload; the line's `workloads` list carries the other benchmark configurations (fewer
+steps each, with a parity check on a seeded row sample) and `naive` the unfused baseline.
+With N > 1 ranks every rank runs the same workload on its own batch: the (batch, head) pairs are
+independent units, so there is no data-path collective (weak scaling).  Ranks come from the
+launcher's environment (torchrun); without one, `--gpus N` starts N ranks itself.
 `--impl reference` times the CPU oracle, as it stands, on a bounded row sample (rank 0 only).
 """
 import argparse
 import json
 import os
+import socket
 import subprocess
 import sys
 import threading
@@ -27,21 +31,21 @@ import numpy as np
 METRIC = "fused attention TFLOP/s"
 UNIT = "TFLOP/s"
 DEFAULT_WORKLOAD = "c2_bert_large_4k"
+OTHER_WORKLOADS = ["c1_bert_base_512", "c3_16k", "c4_64k_d128", "c5_cross_masked"]
 L2_FLUSH_BELOW = 256 << 20          # workloads smaller than this get an L2 flush before every timed launch
-KERNEL_NAMES = {1: "fused_simt_kernel", 2: "fused_tc_kernel", 3: "fused_tc2_kernel", 4: "fused_tc2_kernel",
-                5: "fused_tc3_kernel"}
+# FLAT_VARIANT_* (as reported by the library after a call) -> the kernel that variant launches
+KERNEL_OF_VARIANT = {1: "fused_simt_kernel", 2: "fused_tc_kernel", 3: "fused_tc2_kernel<2 tiles>",
+                     4: "fused_tc2_kernel<1 tile>", 5: "fused_tc3_kernel", 6: "fused_rgran_kernel"}
 
-
-def kernel_name(variant, w):
-    """The kernel a launch of this workload runs (variant 0: the dispatcher's choice for problems that fill the GPU)."""
-    if variant in KERNEL_NAMES:
-        return KERNEL_NAMES[variant]
-    ctas = ((w.Nq + 255) // 256) * w.B * w.H            # 256-row CTAs; the dispatcher's rule with 148 SMs
-    if w.d == 64:
-        slabs_fill = 3 * 256 * ((w.Nq + 255) // 256) <= 4 * w.Nq
-        tc3 = (2 * ctas >= 148 and w.Nk > 1024) or (ctas >= 2 * 148 and not w.masked and slabs_fill)
-        return "fused_tc3_kernel" if tc3 else "fused_tc2_kernel"
-    return "fused_tc2_kernel" if (ctas >= 148 or w.Nk > 256) else "fused_tc_kernel"
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel from ncu
+# captures, with the capture they come from; a (kernel, workload) pair without a capture reports null.
+MEASURED_DRAM_TRAFFIC = {
+    ("fused_tc3_kernel", "c2_bert_large_4k"): (514_200_000, "profiles/fused_tc3_kernel_dram_and_pipes.md"),
+    ("fused_tc3_kernel", "p_4k_small"): (116_900_000, "profiles/fused_tc3_kernel_dram_and_pipes.md"),
+    ("fused_tc2_kernel<2 tiles>", "c2_bert_large_4k"): (516_000_000, "profiles/fused_tc2_kernel_dram_and_pipes.md"),
+    ("fused_tc2_kernel<2 tiles>", "p_4k_small"): (117_600_000, "profiles/fused_tc2_kernel_dram_and_pipes.md"),
+    ("fused_tc2_kernel<2 tiles>", "p_16k_d128_small"): (51_900_000, "profiles/fused_tc2_kernel_dram_and_pipes.md"),
+}
 
 
 def load_peaks():
@@ -54,20 +58,11 @@ def load_peaks():
     return {"bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "hbm_gbs": 6650.0, "source": "fallback"}
 
 
-# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel, copied from
-# the ncu captures summarised in profiles/fused_tc3_kernel_dram_and_pipes.md and
-# profiles/fused_tc2_kernel_dram_and_pipes.md (None where nothing was captured).
-MEASURED_DRAM_TRAFFIC = {
-    ("fused_tc3_kernel", "c2_bert_large_4k"): 514_200_000,
-    ("fused_tc3_kernel", "p_4k_small"): 116_900_000,
-    ("fused_tc2_kernel", "c2_bert_large_4k"): 516_000_000,
-    ("fused_tc2_kernel", "p_4k_small"): 117_600_000,
-    ("fused_tc2_kernel", "p_16k_d128_small"): 51_900_000,
-}
-
-
-def load_traffic(workload, kernel="fused_tc2_kernel"):
-    return MEASURED_DRAM_TRAFFIC.get((kernel, workload))
+def traffic_fields(kernel, workload):
+    hit = MEASURED_DRAM_TRAFFIC.get((kernel, workload))
+    if hit:
+        return {"traffic": hit[0], "traffic_source": "ncu dram__bytes_read.sum + dram__bytes_write.sum, " + hit[1]}
+    return {"traffic": None, "traffic_note": "no ncu capture of %s on %s" % (kernel, workload)}
 
 
 class ClockSampler:
@@ -89,6 +84,7 @@ class ClockSampler:
             self.thread.start()
         except OSError:
             self.proc = None
+        return self
 
     def _read(self):
         for ln in self.proc.stdout:
@@ -120,18 +116,20 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
-def cpu_baseline(w, Qb, Kb, Vb, vl, target_seconds=15.0):
-    """The oracle, as it stands, on a bounded seeded row sample of the same workload."""
+def oracle_on_sample(w, Qb, Kb, Vb, vl, per_head=None, target_seconds=15.0):
+    """The oracle, as it stands, on a seeded row sample of the workload: (timing dict, rows, O rows).
+    per_head = None sizes the sample for about `target_seconds` of wall time."""
     import oracle
     from paper_2107_06419_b200 import inputs
     threads = oracle.hardware_threads()
-    rows = inputs.sample_rows(w, 1)[:threads]                       # calibration: one row per thread
-    t0 = time.perf_counter()
-    oracle.attention(Qb, Kb, Vb, w.scale, valid_len=vl, rows=rows)
-    per_row = (time.perf_counter() - t0) / max(1, len(rows)) * threads    # thread-seconds per row
-    total_rows = w.B * w.H * w.Nq
-    nrows = int(min(total_rows, max(threads, target_seconds * threads / max(per_row, 1e-9))))
-    per_head = max(1, nrows // (w.B * w.H))
+    if per_head is None:
+        rows = inputs.sample_rows(w, 1)[:threads]                       # calibration: one row per thread
+        t0 = time.perf_counter()
+        oracle.attention(Qb, Kb, Vb, w.scale, valid_len=vl, rows=rows)
+        per_row = (time.perf_counter() - t0) / max(1, len(rows)) * threads    # thread-seconds per row
+        total_rows = w.B * w.H * w.Nq
+        nrows = int(min(total_rows, max(threads, target_seconds * threads / max(per_row, 1e-9))))
+        per_head = max(1, nrows // (w.B * w.H))
     rows = inputs.sample_rows(w, per_head)
     t0 = time.perf_counter()
     r = oracle.attention(Qb, Kb, Vb, w.scale, valid_len=vl, rows=rows)
@@ -192,17 +190,138 @@ def workload_config(w, extra=None):
     return c
 
 
+def free_port():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def spawn_ranks(n):
+    """No launcher gave this process a rank: start `n` ranks of this script (one per GPU) under
+    torch.distributed.run on this node and pass their exit code on."""
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(n),
+           "--master-addr", "127.0.0.1", "--master-port", str(free_port()), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
+
+
+def dry_run(args, w):
+    """The rank plumbing without a GPU (CPU tests): every rank draws its seed, 'times' a fake step and
+    joins the max-reduction over the chosen backend; rank 0 prints the line."""
+    import torch
+    import torch.distributed as dist
+    from paper_2107_06419_b200 import inputs, shard
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if world > 1:
+        dist.init_process_group(args.backend)
+    seed = shard.rank_seed(inputs.DEFAULT_SEED, rank)
+    ms = 1.0 + rank                                                   # the slowest rank decides
+    (ms_max,) = shard.max_over_ranks([ms], torch.device("cpu"))
+    if rank == 0:
+        print(json.dumps({"metric": METRIC, "value": shard.whole_job_rate(float(w.flops), world, ms_max) / 1e12,
+                          "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+                          "ms_per_step": ms_max, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+                          "dtype": "bf16", "data": "synthetic", "dry_run": True, "seed_rank0": seed,
+                          "config": workload_config(w, {"parallelism": "dp%d over independent batches, no collective" % world})}))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+class Bench:
+    """One GPU's view of the benchmark: device buffers of a workload, timed launches."""
+
+    def __init__(self, torch, api, dev, world, variant):
+        self.torch, self.api, self.dev, self.world, self.variant = torch, api, dev, world, variant
+        self.flush = None
+
+    def barrier(self):
+        if self.world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        self.torch.cuda.synchronize()
+
+    def timed(self, fn, steps, flush):
+        """K launches bracketed by barrier + synchronize; returns (total ms, per-launch ms list).
+        With an L2 flush between launches the total is the sum of the per-launch times."""
+        torch = self.torch
+        if flush and self.flush is None:
+            self.flush = torch.empty(256 << 20, dtype=torch.uint8, device=self.dev)
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        self.barrier()
+        t_begin.record()
+        for a, b in evs:
+            if flush:
+                self.flush.fill_(1)
+            a.record(); fn(); b.record()
+        t_end.record()
+        self.barrier()
+        per = [a.elapsed_time(b) for a, b in evs]
+        return (sum(per) if flush else t_begin.elapsed_time(t_end)), per
+
+    def load(self, w, seed):
+        """Generates the workload on the host (pinned) and uploads it."""
+        from paper_2107_06419_b200 import inputs
+        torch = self.torch
+        Qb, Kb, Vb = inputs.make_qkv_bf16(w, seed)
+        vl = inputs.make_valid_len(w, seed) if w.masked else None
+        as_t = lambda bits: torch.from_numpy(bits.view(np.int16)).view(torch.bfloat16)
+        host = {"Q": as_t(Qb).pin_memory(), "K": as_t(Kb).pin_memory(), "V": as_t(Vb).pin_memory(),
+                "vl": None if vl is None else torch.from_numpy(vl).pin_memory()}
+        devt = {k: (None if v is None else v.to(self.dev)) for k, v in host.items()}
+        devt["O"] = torch.empty_like(devt["Q"])
+        devt["status"] = torch.zeros(1, dtype=torch.int32, device=self.dev)
+        return (Qb, Kb, Vb, vl), host, devt
+
+    def measure(self, w, d, steps, warmup, sample_clocks):
+        """Warm-up, then `steps` timed launches of the fused call on resident inputs."""
+        api = self.api
+        step = lambda: api.flat_attn_fwd_ex(d["Q"], d["K"], d["V"], d["O"], w.scale, k_valid_len=d["vl"],
+                                            status=d["status"], variant=self.variant)
+        for _ in range(warmup):
+            step()
+        kernel = KERNEL_OF_VARIANT.get(api.flat_attn_last_variant(), "?")
+        sampler = ClockSampler(self.dev.index).start() if sample_clocks else None
+        total_ms, per = self.timed(step, steps, flush=w.qkvo_bytes() <= L2_FLUSH_BELOW)
+        clocks = sampler.stop() if sampler else None
+        code = int(d["status"].item())
+        assert code == 0, "device status 0x%x" % code
+        return total_ms, per, kernel, clocks
+
+
+def roofline_entry(w, per_launch, kernel, peaks):
+    kernel_ms = float(np.mean(per_launch))
+    achieved = float(w.flops) / (kernel_ms * 1e-3) / 1e12
+    r = {"bound": "tensor", "kernel": kernel, "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": UNIT,
+         "frac": achieved / peaks["bf16_tflops"], "peak_kind": "burst bf16 matmul, of " + peaks["source"],
+         "frac_of_sustained": achieved / peaks["bf16_tflops_sustained"], "kernel_ms": kernel_ms,
+         "kernel_ms_min": float(np.min(per_launch)), "kernel_ms_median": float(np.median(per_launch)),
+         "flops_per_launch": w.flops, "algorithmic_bytes": w.qkvo_bytes()}
+    r.update(traffic_fields(kernel, w.name))
+    return r
+
+
+def parity_on_sample(torch, w, data, O, dev, per_head):
+    Qb, Kb, Vb, vl = data
+    cb, rows, Oref = oracle_on_sample(w, Qb, Kb, Vb, vl, per_head=per_head)
+    got = O.view(-1, w.d)[torch.from_numpy(rows).to(dev)].float().cpu().numpy().astype(np.float64)
+    err = np.abs(got - Oref)
+    return cb, {"rows": int(len(rows)), "max_abs": float(err.max()), "mean_abs": float(err.mean())}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
-    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--variant", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--with-naive", action="store_true",
-                    help="also time the unfused baseline (L and A materialised in device memory)")
+    ap.add_argument("--headline-only", action="store_true",
+                    help="skip the other workloads and the unfused baseline (they run at N = 1 only anyway)")
+    ap.add_argument("--backend", default="nccl", choices=["nccl", "gloo"])
+    ap.add_argument("--dry-run", action="store_true", help="rank plumbing only, no CUDA call (CPU tests)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -210,6 +329,11 @@ def main():
     w = inputs.WORKLOADS[args.workload]
     if args.impl == "reference":
         run_reference(args, w)
+        return
+    if "WORLD_SIZE" not in os.environ and args.gpus > 1:
+        sys.exit(spawn_ranks(args.gpus))
+    if args.dry_run:
+        dry_run(args, w)
         return
 
     import torch
@@ -223,67 +347,24 @@ def main():
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
     if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
+        dist.init_process_group(args.backend, device_id=dev)
+    bench = Bench(torch, api, dev, world, args.variant)
 
     # Each rank owns one full batch of the workload (its own seed): units are independent.
     seed = shard.rank_seed(inputs.DEFAULT_SEED, rank)
-    Qb, Kb, Vb = inputs.make_qkv_bf16(w, seed)
-    vl = inputs.make_valid_len(w, seed) if w.masked else None
-    as_t = lambda bits: torch.from_numpy(bits.view(np.int16)).view(torch.bfloat16)
-    Qh, Kh, Vh = (as_t(x).pin_memory() for x in (Qb, Kb, Vb))
-    Oh = torch.empty(Qh.shape, dtype=torch.bfloat16).pin_memory()
-    vlh = None if vl is None else torch.from_numpy(vl).pin_memory()
-    Q, K, V = Qh.to(dev), Kh.to(dev), Vh.to(dev)
-    O = torch.empty_like(Q)
-    vld = None if vl is None else vlh.to(dev)
-    status = torch.zeros(1, dtype=torch.int32, device=dev)
-    ws = torch.empty(api.flat_attn_host_workspace_bytes(w.B, w.H, w.Nq, w.Nk, w.d), dtype=torch.uint8, device=dev)
-
-    def step():
-        api.flat_attn_fwd_ex(Q, K, V, O, w.scale, k_valid_len=vld, status=status, variant=args.variant)
-
-    def step_e2e():
-        api.flat_attn_fwd_host(Qh, Kh, Vh, Oh, w.scale, ws, k_valid_len=vlh, status=status, variant=args.variant)
-
-    def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
-
-    flush = None
-    if w.qkvo_bytes() <= L2_FLUSH_BELOW:
-        flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
-
-    def timed(fn, steps):
-        """K launches bracketed by barrier + synchronize; returns (total ms, per-launch ms list).
-        With an L2 flush between launches the total is the sum of the per-launch times."""
-        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
-        t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        barrier()
-        t_begin.record()
-        for a, b in evs:
-            if flush is not None:
-                flush.fill_(1)
-            a.record(); fn(); b.record()
-        t_end.record()
-        barrier()
-        per = [a.elapsed_time(b) for a, b in evs]
-        return (sum(per) if flush is not None else t_begin.elapsed_time(t_end)), per
-
-    for _ in range(args.warmup):
-        step()
-    sampler = ClockSampler(local)
-    if rank == 0:
-        sampler.start()
-    total_ms, per_launch = timed(step, args.steps)
+    data, host, d = bench.load(w, seed)
+    total_ms, per_launch, kernel, clocks = bench.measure(w, d, args.steps, args.warmup, sample_clocks=rank == 0)
     launches = api.flat_attn_last_launch_count() * args.steps
-    clocks = sampler.stop() if rank == 0 else None
-    assert int(status.item()) == 0, "device status 0x%x" % int(status.item())
 
+    Oh = torch.empty(host["Q"].shape, dtype=torch.bfloat16).pin_memory()
+    ws = torch.empty(api.flat_attn_host_workspace_bytes(w.B, w.H, w.Nq, w.Nk, w.d), dtype=torch.uint8, device=dev)
+    step_e2e = lambda: api.flat_attn_fwd_host(host["Q"], host["K"], host["V"], Oh, w.scale, ws, k_valid_len=host["vl"],
+                                              status=d["status"], variant=args.variant)
     for _ in range(2):
         step_e2e()
-    e2e_ms, _ = timed(step_e2e, max(3, min(args.steps, 5)))
-    e2e_ms /= max(3, min(args.steps, 5))
+    e2e_steps = max(3, min(args.steps, 5))
+    e2e_ms, _ = bench.timed(step_e2e, e2e_steps, flush=False)
+    e2e_ms /= e2e_steps
 
     total_ms, e2e_ms = shard.max_over_ranks([total_ms, e2e_ms], dev)
     ms_per_step = total_ms / args.steps
@@ -292,58 +373,80 @@ def main():
 
     if rank == 0:
         peaks = load_peaks()
-        kernel_ms = float(np.mean(per_launch))
-        achieved = float(w.flops) / (kernel_ms * 1e-3) / 1e12
         out = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": workload_config(w, {"parallelism": "dp%d over independent batches, no collective" % world}),
             "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": e2e_ms,
-                    "h2d_bytes_per_step": int(2 * (Qh.numel() + Kh.numel() + Vh.numel()) + (0 if vl is None else 4 * w.B)),
+                    "h2d_bytes_per_step": int(2 * (host["Q"].numel() + host["K"].numel() + host["V"].numel())
+                                              + (0 if data[3] is None else 4 * w.B)),
                     "d2h_bytes_per_step": int(2 * Oh.numel())},
             "gpu_launches": launches,
             "clocks": clocks,
-            "roofline": {"bound": "tensor", "kernel": kernel_name(args.variant, w),
-                         "achieved": achieved,
-                         "peak": peaks["bf16_tflops"], "unit": UNIT, "frac": achieved / peaks["bf16_tflops"],
-                         "peak_kind": "burst bf16 matmul, of " + peaks["source"],
-                         "frac_of_sustained": achieved / peaks["bf16_tflops_sustained"],
-                         "kernel_ms": kernel_ms, "kernel_ms_min": float(np.min(per_launch)),
-                         "kernel_ms_median": float(np.median(per_launch)), "flops_per_launch": w.flops,
-                         "traffic": load_traffic(w.name, kernel_name(args.variant, w)),
-                         "algorithmic_bytes": w.qkvo_bytes()},
+            "roofline": roofline_entry(w, per_launch, kernel, peaks),
         }
-        if vl is not None:
+        if data[3] is not None:
             # Masked workload: `value` counts the masked keys too (the stated metric, 4 B H Nq Nk d);
             # this is the same rate counted over the valid keys only.
-            useful = 4.0 * w.H * w.Nq * w.d * float(np.sum(vl))
+            useful = 4.0 * w.H * w.Nq * w.d * float(np.sum(data[3]))
             out["useful_work"] = {"value": value * useful / float(w.flops), "unit": UNIT,
                                   "valid_key_fraction": useful / float(w.flops)}
-        if args.with_naive and world == 1:
-            # The paper's unfused baseline on the same inputs: L (fp32) and A (bf16) go through HBM.
-            elems = w.B * w.H * w.Nq * w.Nk
-            L = torch.empty((w.B, w.H, w.Nq, w.Nk), dtype=torch.float32, device=dev)
-            A = torch.empty((w.B, w.H, w.Nq, w.Nk), dtype=torch.bfloat16, device=dev)
-            O2 = torch.empty_like(Q)
-            naive = lambda: api.flat_attn_naive_fwd_ex(Q, K, V, O2, L, A, w.scale, k_valid_len=vld)
-            naive()
-            n_ms, _ = timed(naive, 3)
-            n_ms /= 3
-            out["naive"] = {"ms_per_step": n_ms, "value": float(w.flops) / (n_ms * 1e-3) / 1e12, "unit": UNIT,
-                            "kernels_per_step": 3, "materialised_bytes": 6 * elems,
-                            "algorithmic_bytes": 12 * elems + w.qkvo_bytes(),
-                            "max_abs_diff_vs_fused": float((O2.float() - O.float()).abs().max())}
-            del L, A, O2
         if not args.no_cpu_baseline and world == 1:
-            cb, rows, Oref = cpu_baseline(w, Qb, Kb, Vb, vl)
-            got = O.view(-1, w.d)[torch.from_numpy(rows).to(dev)].float().cpu().numpy().astype(np.float64)
-            err = np.abs(got - Oref)
-            cb["parity_on_sample"] = {"max_abs": float(err.max()), "mean_abs": float(err.mean())}
+            cb, par = parity_on_sample(torch, w, data, d["O"], dev, per_head=None)
+            cb["parity_on_sample"] = par
             out["cpu_baseline"] = cb
+        if not args.headline_only and world == 1:
+            del ws, Oh
+            out["naive"] = run_naive(bench, torch, api, w, d) if w.name == DEFAULT_WORKLOAD else None
+            host = d = data = None
+            torch.cuda.empty_cache()
+            out["workloads"] = [run_other(bench, torch, api, inputs.WORKLOADS[n], seed, args, peaks, dev)
+                                for n in OTHER_WORKLOADS if n != w.name]
         print(json.dumps(out))
     if world > 1:
         dist.destroy_process_group()
+
+
+def run_naive(bench, torch, api, w, d):
+    """The paper's unfused baseline on the same inputs: L (fp32) and A (bf16) go through HBM."""
+    elems = w.B * w.H * w.Nq * w.Nk
+    L = torch.empty((w.B, w.H, w.Nq, w.Nk), dtype=torch.float32, device=bench.dev)
+    A = torch.empty((w.B, w.H, w.Nq, w.Nk), dtype=torch.bfloat16, device=bench.dev)
+    O2 = torch.empty_like(d["Q"])
+    naive = lambda: api.flat_attn_naive_fwd_ex(d["Q"], d["K"], d["V"], O2, L, A, w.scale, k_valid_len=d["vl"])
+    naive()
+    n_ms, _ = bench.timed(naive, 3, flush=False)
+    n_ms /= 3
+    return {"ms_per_step": n_ms, "value": float(w.flops) / (n_ms * 1e-3) / 1e12, "unit": UNIT,
+            "kernels_per_step": 3, "materialised_bytes": 6 * elems,
+            "bytes_model": 12 * elems + w.qkvo_bytes(),
+            "hbm_gbs_on_model": (12 * elems + w.qkvo_bytes()) / (n_ms * 1e-3) / 1e9,
+            "max_abs_diff_vs_fused": float((O2.float() - d["O"].float()).abs().max())}
+
+
+def run_other(bench, torch, api, w, seed, args, peaks, dev):
+    """One more benchmark configuration: fewer steps, a parity check on 64 seeded rows per (b,h)."""
+    time.sleep(1.0)                                      # let the power window of the previous workload pass
+    data, host, d = bench.load(w, seed)
+    ms1 = float(w.flops) / 0.9e15 * 1e3                  # a rough guess of one launch, to bound the timed region
+    steps = int(max(3, min(args.steps, 20, 60.0 / ms1)))
+    total_ms, per, kernel, clocks = bench.measure(w, d, steps, max(3, min(args.warmup, 5)), sample_clocks=True)
+    ms = float(np.mean(per))
+    val = float(w.flops) / (ms * 1e-3) / 1e12
+    e = {"workload": w.name, "config": workload_config(w), "kernel": kernel, "steps": steps, "ms": ms,
+         "ms_min": float(np.min(per)), "value": val, "unit": UNIT, "frac": val / peaks["bf16_tflops"],
+         "frac_of_sustained": val / peaks["bf16_tflops_sustained"], "clocks": clocks}
+    if data[3] is not None:
+        useful = 4.0 * w.H * w.Nq * w.d * float(np.sum(data[3])) / float(w.flops)
+        e["useful_work"] = {"value": val * useful, "unit": UNIT, "valid_key_fraction": useful,
+                            "frac": val * useful / peaks["bf16_tflops"]}
+    e.update(traffic_fields(kernel, w.name))
+    if not args.no_cpu_baseline:
+        _, e["parity_on_sample"] = parity_on_sample(torch, w, data, d["O"], dev, per_head=64)
+    del data, host, d
+    torch.cuda.empty_cache()
+    return e
 
 
 if __name__ == "__main__":

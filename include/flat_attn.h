@@ -87,7 +87,9 @@ typedef struct flat_attn_params {
                                   accumulation is always fp32                                 */
     const int32_t* k_valid_len;/* device, [B], or NULL = all keys valid                        */
     int32_t* status;           /* optional device word; a kernel that gives up on a bounded
-                                  wait stores a non-zero code here (never traps or hangs)      */
+                                  wait stores a non-zero code here (never traps or hangs).
+                                  NULL: the code goes to the library's own device word instead,
+                                  see flat_attn_last_device_error                              */
     int variant;               /* FLAT_VARIANT_*                                               */
     int causal;                /* 0, or 1 = causal mask: query i takes part with key j iff
                                   j <= i + (Nk - Nq) (the last query sees every key), intersected
@@ -118,7 +120,8 @@ int flat_attn_fwd_ex(const flat_attn_params_t* p, void* stream);
  *   O = A V.
  * L and A are caller-allocated device buffers; their contents after the call are
  * the logits (all columns, masked ones included, unmasked values) and the weights
- * (masked columns 0).
+ * (masked columns 0).  The row softmax runs one thread block per row of L, so B*H*Nq must not
+ * exceed 2^31 - 1 (FLAT_ERR_SHAPE, nothing launched).
  */
 int flat_attn_naive_fwd(const void* Q, const void* K, const void* V, void* O, void* L, void* A,
                         int B, int H, int Nq, int Nk, int d, float scale, void* stream);
@@ -179,9 +182,8 @@ int flat_attn_layer_fwd(const void* X, const void* Wqkv, const void* Wo, void* Y
                         int32_t* status, void* stream);
 
 /*
- * A fully connected operator of the attention block (paper Section 2: "an attention layer, a
- * normalization layer, followed by multiple (typically two) fully connected layers"; the FF1 / FF2
- * of Table 2):  Y [M, Nout] = X [M, K] * W[Nout, K]^T, all row-major bf16, fp32 accumulation, no
+ * A fully connected operator of the attention block (the layers that follow the attention and
+ * normalisation layers of a block, paper Section 2; FF1 / FF2 of Table 2):  Y [M, Nout] = X [M, K] * W[Nout, K]^T, all row-major bf16, fp32 accumulation, no
  * bias and no activation (the paper names none).  The same kernel as the projections.  Needs K a
  * multiple of 64 and Nout a multiple of 256.  DEVICE pointers, 16-byte aligned; errors as above.
  */
@@ -226,9 +228,13 @@ size_t flat_attn_host_workspace_bytes(int B, int H, int Nq, int Nk, int d, int d
  *   - Limit: B*H*Nq*Nk <= FLAT_STATIC_MAX_ELEMS, otherwise FLAT_ERR_WORKSPACE is
  *     returned before anything touches the device.  Other argument rules and error
  *     codes are those of flat_attn_naive_fwd; Q, K, V, O stay caller-owned.
- *   - The first call on each device looks up the array's device address (with that
- *     device current, which is the caller's job as for every entry point).  Make that
- *     first call outside any stream capture.
+ *   - Arguments are checked first (size gate, then pointers, d, alignment), before the
+ *     device is looked at.  The first valid call on each device then looks up the array's
+ *     device address (with that device current, which is the caller's job as for every
+ *     entry point); this is also the latest moment at which the CUDA runtime makes the
+ *     array resident on that device, so it is the one call that can fail for lack of
+ *     device memory (FLAT_ERR_CUDA).  Make one small warm-up call per device at start-up,
+ *     outside any stream capture; later calls only enqueue the three kernels.
  *   - All calls on a device share the one array, and it keeps whatever the last call
  *     left in it.  The three kernels overwrite every element they later read, so
  *     nothing has to be cleared, but two calls whose kernels overlap on the GPU
@@ -243,7 +249,9 @@ int flat_attn_naive_fwd_static(const void* Q, const void* K, const void* V, void
  * tensor-core kernels is bounded; when one runs out, the kernel stores a non-zero code in the
  * caller's `status` word and returns normally.  This call launches a one-warp kernel that waits,
  * for about 0.1 s, on a barrier nothing completes, and must leave FLAT_SELFTEST_TIMEOUT_CODE in
- * *status (a device int32, zeroed by the caller) with the context still usable afterwards.
+ * *status (a device int32, zeroed by the caller) with the context still usable afterwards.  With
+ * status == NULL the code goes where every kernel's goes in that case: to the library's own word
+ * (flat_attn_last_device_error).
  */
 #define FLAT_SELFTEST_TIMEOUT_CODE 0x7e57
 int flat_attn_selftest_wait_timeout(int32_t* status, void* stream);
@@ -257,6 +265,25 @@ int flat_attn_selftest_exp2_poly(const float* x, float* y, int n, void* stream);
 
 /* Number of kernels the most recent successful call on this thread launched. */
 int flat_attn_last_launch_count(void);
+
+/* The FLAT_VARIANT_* that the most recent fused call on this host thread ran (what
+ * FLAT_VARIANT_AUTO resolved to for that problem on the current device); 0 before any call. */
+int flat_attn_last_variant(void);
+
+/*
+ * Device-side give-up codes when the caller passed no `status` word (the paper has no
+ * counterpart).  Every wait inside the tensor-core kernels is bounded (about a second of SM
+ * clock, which also runs while a context is time-sliced out on a GPU shared with other
+ * processes); a kernel whose wait runs out stores a code and returns, leaving O partly written,
+ * after the host call has long returned FLAT_OK.  With status == NULL that code goes to one
+ * sticky word per device inside the library.  flat_attn_last_device_error copies the word of
+ * the current device to *code (HOST pointer; 0 = no kernel has given up since the last clear).
+ * It is a blocking copy: synchronise the streams whose work you ask about first.
+ * flat_attn_clear_device_error zeroes the word.  The first fused call on a device looks the
+ * word's address up; make it outside any stream capture.
+ */
+int flat_attn_last_device_error(int32_t* code);
+int flat_attn_clear_device_error(void);
 
 const char* flat_attn_status_string(int code);
 int flat_attn_version(void);

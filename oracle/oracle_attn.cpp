@@ -10,7 +10,7 @@
 // operators", steps 2-4; Q, K, V are [B, H, N, d] with d = D / H):
 //   step 2, Logit  L[b,h,i,j] = sum_t Q[b,h,i,t] * K[b,h,j,t]   (a d-dim dot product)
 //   step 3, Softmax over each row of logits, i.e. along the key index j
-//           (Section 5.2: "the reduction is along the key dimension")
+//           (the softmax reduces over the key index, Section 5.2)
 //   step 4, Attend O[b,h,i,t] = sum_j A[b,h,i,j] * V[b,h,j,t]
 // The fused dataflow (Section 5) claims the same function as the unfused
 // chain, so the oracle is the definition written out.

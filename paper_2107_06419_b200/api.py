@@ -32,7 +32,8 @@ EXPORTS = ["flat_attn_fwd", "flat_attn_fwd_ex", "flat_attn_naive_fwd", "flat_att
            "flat_attn_fwd_host", "flat_attn_host_workspace_bytes", "flat_attn_last_launch_count",
            "flat_attn_status_string", "flat_attn_version",
            "flat_qkv_proj_fwd", "flat_out_proj_fwd", "flat_attn_layer_fwd", "flat_fc_fwd",
-           "flat_attn_varlen_fwd"]
+           "flat_attn_varlen_fwd", "flat_attn_last_variant", "flat_attn_last_device_error",
+           "flat_attn_clear_device_error"]
 
 
 class flat_attn_params_t(ctypes.Structure):
@@ -74,6 +75,10 @@ _lib.flat_attn_varlen_fwd.restype = _i
 _lib.flat_attn_host_workspace_bytes.argtypes = [_i, _i, _i, _i, _i, _i]
 _lib.flat_attn_host_workspace_bytes.restype = ctypes.c_size_t
 _lib.flat_attn_last_launch_count.restype = _i
+_lib.flat_attn_last_variant.restype = _i
+_lib.flat_attn_last_device_error.argtypes = [ctypes.POINTER(ctypes.c_int32)]
+_lib.flat_attn_last_device_error.restype = _i
+_lib.flat_attn_clear_device_error.restype = _i
 _lib.flat_attn_status_string.argtypes = [_i]
 _lib.flat_attn_status_string.restype = ctypes.c_char_p
 _lib.flat_attn_version.restype = _i
@@ -95,6 +100,22 @@ def flat_attn_version() -> int:
 
 def flat_attn_last_launch_count() -> int:
     return int(_lib.flat_attn_last_launch_count())
+
+
+def flat_attn_last_variant() -> int:
+    """The FLAT_VARIANT_* the most recent fused call on this thread ran (what AUTO resolved to)."""
+    return int(_lib.flat_attn_last_variant())
+
+
+def flat_attn_last_device_error() -> int:
+    """The library's sticky per-device give-up code (0 = none); synchronise your streams first."""
+    code = ctypes.c_int32(0)
+    _check(_lib.flat_attn_last_device_error(ctypes.byref(code)))
+    return int(code.value)
+
+
+def flat_attn_clear_device_error() -> None:
+    _check(_lib.flat_attn_clear_device_error())
 
 
 def _stream_ptr(stream):
@@ -211,9 +232,9 @@ def flat_attn_selftest_exp2_poly(x, y, stream=None):
 
 
 def flat_attn_selftest_wait_timeout(status, stream=None):
-    """Runs the bounded-wait self-test; `status` is a zeroed CUDA int32 tensor of one element."""
-    if not status.is_cuda or status.dtype != torch.int32:
-        raise ValueError("status must be a CUDA int32 tensor")
+    """Runs the bounded-wait self-test; `status` is a zeroed CUDA int32 tensor of one element, or None."""
+    if status is not None and (not status.is_cuda or status.dtype != torch.int32):
+        raise ValueError("status must be a CUDA int32 tensor (or None: the library's own word)")
     _check(_lib.flat_attn_selftest_wait_timeout(_ptr(status), _stream_ptr(stream)))
 
 

@@ -3,11 +3,41 @@
 #include <math.h>
 #include <stdint.h>
 
+#include <mutex>
+
 #include "flat_internal.cuh"
 
 namespace {
 
 thread_local int g_last_launches = 0;
+thread_local int g_last_variant = 0;
+
+// The library's own device status word: kernels that give up on a bounded wait store their code
+// here when the caller passed no `status` word, so that a timeout always leaves a trace.  In host
+// code the name is a handle for the runtime's symbol table; its device address is looked up once
+// per device.
+__device__ int32_t g_device_error = 0;
+constexpr int kMaxDevices = 64;
+std::mutex g_err_mu;
+int32_t* g_err_addr[kMaxDevices];
+bool g_err_ready[kMaxDevices];
+
+int32_t* library_status_word() {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+    std::lock_guard<std::mutex> lock(g_err_mu);
+    if (!g_err_ready[dev]) {
+        void* a = nullptr;
+        if (cudaGetSymbolAddress(&a, g_device_error) != cudaSuccess || a == nullptr) {
+            cudaGetLastError();                          // (no device, or no image for it: the caller's launch will say so)
+            return nullptr;
+        }
+        g_err_addr[dev] = static_cast<int32_t*>(a);
+        g_err_ready[dev] = true;
+    }
+    return g_err_addr[dev];
+}
+inline int32_t* status_or_library_word(int32_t* s) { return s ? s : library_status_word(); }
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -30,9 +60,20 @@ int validate(const flat_attn_params_t* p, flat::Problem* out) {
     if (p->status && (reinterpret_cast<uintptr_t>(p->status) & 3u)) return FLAT_ERR_ALIGN;
     if (p->causal != 0 && p->causal != 1) return FLAT_ERR_UNSUPPORTED;
     *out = flat::Problem{p->Q, p->K, p->V, p->O, p->B, p->H, p->Nq, p->Nk, p->d,
-                         p->scale, p->dtype, p->k_valid_len, p->status, p->causal};
+                         p->scale, p->dtype, p->k_valid_len, status_or_library_word(p->status), p->causal};
     return FLAT_OK;
 }
+
+}  // namespace
+
+namespace flat {
+int check_params(const flat_attn_params_t* p) {
+    Problem q;
+    return validate(p, &q);
+}
+}  // namespace flat
+
+namespace {
 
 bool tc_applies(const flat::Problem& q) {
     return q.dtype == FLAT_DTYPE_BF16 && (q.d == 64 || q.d == 128);
@@ -71,6 +112,7 @@ int run_fused(const flat::Problem& q, int variant, cudaStream_t st) {
         }
     }
     if (q.causal && v == FLAT_VARIANT_TC) return FLAT_ERR_UNSUPPORTED;
+    g_last_variant = v;
     if (v == FLAT_VARIANT_TC2_SINGLE) {
         if (!tc_applies(q) || q.d != 64) return FLAT_ERR_UNSUPPORTED;
         return flat::launch_fused_tc2_single(q, st);
@@ -138,6 +180,8 @@ int flat_attn_naive_fwd_ex(const flat_attn_params_t* p, void* L, void* A, void* 
     if (rc != FLAT_OK) return rc;
     if (!L || !A) return FLAT_ERR_NULL;
     if (!aligned16(L) || !aligned16(A)) return FLAT_ERR_ALIGN;
+    // (the row softmax runs one CTA per row of L: the row count is a grid dimension)
+    if (static_cast<int64_t>(q.B) * q.H * q.Nq > 0x7fffffffLL) return FLAT_ERR_SHAPE;
     const int r = flat::launch_naive(q, L, A, static_cast<cudaStream_t>(stream));
     if (r == FLAT_OK) g_last_launches = 3;
     return r;
@@ -244,8 +288,9 @@ int flat_attn_selftest_exp2_poly(const float* x, float* y, int n, void* stream) 
 }
 
 int flat_attn_selftest_wait_timeout(int32_t* status, void* stream) {
-    if (!status) return FLAT_ERR_NULL;
-    if (reinterpret_cast<uintptr_t>(status) & 3u) return FLAT_ERR_ALIGN;
+    if (status && (reinterpret_cast<uintptr_t>(status) & 3u)) return FLAT_ERR_ALIGN;
+    status = status_or_library_word(status);             // NULL: the code goes to the library's own word
+    if (!status) return FLAT_ERR_CUDA;
     const int r = flat::launch_wait_timeout_selftest(status, static_cast<cudaStream_t>(stream));
     if (r == FLAT_OK) g_last_launches = 1;
     return r;
@@ -253,14 +298,14 @@ int flat_attn_selftest_wait_timeout(int32_t* status, void* stream) {
 
 int flat_qkv_proj_fwd(const void* X, const void* Wqkv, void* Q, void* K, void* V, int B, int N, int H, int d,
                       int Dm, int32_t* status, void* stream) {
-    const int r = flat::launch_qkv_proj(X, Wqkv, Q, K, V, B, N, H, d, Dm, status, static_cast<cudaStream_t>(stream));
+    const int r = flat::launch_qkv_proj(X, Wqkv, Q, K, V, B, N, H, d, Dm, status_or_library_word(status), static_cast<cudaStream_t>(stream));
     if (r == FLAT_OK) g_last_launches = 1;
     return r;
 }
 
 int flat_out_proj_fwd(const void* O, const void* Wo, void* Y, int B, int N, int H, int d, int Dm, int32_t* status,
                       void* stream) {
-    const int r = flat::launch_out_proj(O, Wo, Y, B, N, H, d, Dm, status, static_cast<cudaStream_t>(stream));
+    const int r = flat::launch_out_proj(O, Wo, Y, B, N, H, d, Dm, status_or_library_word(status), static_cast<cudaStream_t>(stream));
     if (r == FLAT_OK) g_last_launches = 1;
     return r;
 }
@@ -280,14 +325,15 @@ int flat_attn_varlen_fwd(const void* Q, const void* K, const void* V, void* O, c
         (status && (reinterpret_cast<uintptr_t>(status) & 3u)))
         return FLAT_ERR_ALIGN;
     const int r = (d == 64 ? flat::launch_fused_tc3_varlen : flat::launch_fused_tc2_varlen)(
-        Q, K, V, O, cu_seqlens_q, cu_seqlens_k, num_seqs, H, total_q, total_k, max_seqlen_q, scale, causal, status,
+        Q, K, V, O, cu_seqlens_q, cu_seqlens_k, num_seqs, H, total_q, total_k, max_seqlen_q, scale, causal,
+        status_or_library_word(status),
         static_cast<cudaStream_t>(stream));
     if (r == FLAT_OK) g_last_launches = 1;
     return r;
 }
 
 int flat_fc_fwd(const void* X, const void* W, void* Y, int M, int K, int Nout, int32_t* status, void* stream) {
-    const int r = flat::launch_fc(X, W, Y, M, K, Nout, status, static_cast<cudaStream_t>(stream));
+    const int r = flat::launch_fc(X, W, Y, M, K, Nout, status_or_library_word(status), static_cast<cudaStream_t>(stream));
     if (r == FLAT_OK) g_last_launches = 1;
     return r;
 }
@@ -303,16 +349,31 @@ int flat_attn_layer_fwd(const void* X, const void* Wqkv, const void* Wo, void* Y
     if ((d != 64 && d != 128) || (H * d) % 256 != 0 || Dm % 256 != 0 || N % 128 != 0) return FLAT_ERR_UNSUPPORTED;
     if (!aligned16(X) || !aligned16(Wqkv) || !aligned16(Wo) || !aligned16(Y)) return FLAT_ERR_ALIGN;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    rc = flat::launch_qkv_proj(X, Wqkv, Q, K, V, B, N, H, d, Dm, status, st);
+    rc = flat::launch_qkv_proj(X, Wqkv, Q, K, V, B, N, H, d, Dm, status_or_library_word(status), st);
     if (rc != FLAT_OK) return rc;
     rc = run_fused(q, FLAT_VARIANT_AUTO, st);
     if (rc != FLAT_OK) return rc;
-    rc = flat::launch_out_proj(O, Wo, Y, B, N, H, d, Dm, status, st);
+    rc = flat::launch_out_proj(O, Wo, Y, B, N, H, d, Dm, status_or_library_word(status), st);
     if (rc == FLAT_OK) g_last_launches = 3;
     return rc;
 }
 
 int flat_attn_last_launch_count(void) { return g_last_launches; }
+
+int flat_attn_last_variant(void) { return g_last_variant; }
+
+int flat_attn_last_device_error(int32_t* code) {
+    if (!code) return FLAT_ERR_NULL;
+    int32_t* w = library_status_word();
+    if (!w) return FLAT_ERR_CUDA;
+    return cudaMemcpy(code, w, sizeof(int32_t), cudaMemcpyDeviceToHost) == cudaSuccess ? FLAT_OK : FLAT_ERR_CUDA;
+}
+
+int flat_attn_clear_device_error(void) {
+    int32_t* w = library_status_word();
+    if (!w) return FLAT_ERR_CUDA;
+    return cudaMemset(w, 0, sizeof(int32_t)) == cudaSuccess ? FLAT_OK : FLAT_ERR_CUDA;
+}
 
 const char* flat_attn_status_string(int code) {
     switch (code) {

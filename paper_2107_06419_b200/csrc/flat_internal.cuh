@@ -20,6 +20,10 @@ struct Problem {
     int causal;                      // 0 / 1: query i sees keys j <= i + (Nk - Nq)
 };
 
+// Argument check of the public parameter block (what every fused / baseline entry point applies
+// before it launches anything): FLAT_OK or the error code.
+int check_params(const flat_attn_params_t* p);
+
 // Each launcher enqueues its kernels on `st` and returns a FLAT_* code; *launches (if
 // non-null) receives the number of kernels enqueued.
 int launch_fused_simt(const Problem& p, cudaStream_t st);

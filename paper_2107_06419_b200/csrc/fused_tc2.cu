@@ -38,39 +38,13 @@ namespace flat {
 using namespace ptx;
 using namespace tc;
 
-#ifdef FLAT_TRACE
-// Developer tracing (off in the product build): CTA (0,0) keeps SM-clock stamps in shared memory
-// and copies them to a global buffer when it ends.
-__device__ unsigned* g_trace = nullptr;
-extern "C" int flat_debug_set_trace(unsigned* p) {
-    return cudaMemcpyToSymbol(g_trace, &p, sizeof(p)) == cudaSuccess ? 0 : 6;
-}
-#define TRACE_WORDS (3 * 64 * 16)
-#define TRACE(role, iter, point)                                                              \
-    do {                                                                                      \
-        if (blockIdx.x == 0 && blockIdx.y == 0 && (iter) < 64)                                \
-            trace_buf[((role) * 64 + (iter)) * 16 + (point)] = static_cast<unsigned>(clock64()); \
-    } while (0)
-#else
-#define TRACE_WORDS 0
-#define TRACE(role, iter, point) do { } while (0)
-#endif
 
 namespace {
 
 constexpr int BM = 128;              // rows per query tile (two tiles per CTA)
 constexpr int BN = 128;              // keys per step
-#ifndef FLAT_TURNS_EXPR
-#define FLAT_TURNS_EXPR (D == 128)
-#endif
-#ifndef FLAT_PASS_AT
-#define FLAT_PASS_AT 3
-#endif
-constexpr int PASS_AT_CHUNK = FLAT_PASS_AT;     // the other tile gets its turn once this chunk's ex2 are issued
-#ifndef FLAT_POLY_LANE
-#define FLAT_POLY_LANE 3
-#endif
-constexpr int POLY_LANE = FLAT_POLY_LANE;       // element index mod 4 that uses ex2_poly; -1 = none
+constexpr int PASS_AT_CHUNK = 3;                // the other tile gets its turn once this chunk's ex2 are issued
+constexpr int POLY_LANE = 3;                    // element index mod 4 that uses ex2_poly; -1 = none
 constexpr float OVERFLOW_SUM = 1.0995116e12f;   // 2^40: a tile row sum beyond this means m_ref is stale
 
 template <int D, int NT> struct L2 {
@@ -83,7 +57,7 @@ template <int D, int NT> struct L2 {
     static constexpr int Q_BYTES = BM * D * 2;           // one query tile
     static constexpr int KV_BYTES = BN * D * 2;
     static constexpr int TILE_BYTES = NT * Q_BYTES + (KS + VS) * KV_BYTES;
-    static constexpr int SMEM_BYTES = TILE_BYTES + 512 + 1024 + 4 * TRACE_WORDS;
+    static constexpr int SMEM_BYTES = TILE_BYTES + 512 + 1024;
     __host__ __device__ static constexpr uint32_t S_COL(int t) { return 128u * t; }
     __host__ __device__ static constexpr uint32_t O_COL(int t) { return 128u * NT + D * t; }
     __host__ __device__ static constexpr uint32_t P_COL(int t) { return ALIAS ? 128u * t : 128u * NT + D * NT + 64u * t; }
@@ -99,7 +73,7 @@ template <int D, int NT> struct L2 {
     // softmax -> (O += P V, next S) -> softmax with nothing to overlap inside the tile, so the tiles
     // must interleave: one computes exponentials while the other's MMAs run.  Left to themselves
     // they fall into lockstep and the phases add up instead.
-    static constexpr bool TURNS = (NT == 2) && FLAT_TURNS_EXPR;
+    static constexpr bool TURNS = (NT == 2) && (D == 128);
 };
 
 __device__ __forceinline__ float row_max(const uint32_t (&s)[128]) {
@@ -135,7 +109,7 @@ __device__ __forceinline__ float row_min(const uint32_t (&s)[128]) {
 template <bool TAIL, bool POLY, typename BeforeFirstStore, typename AfterLastExp>
 __device__ __forceinline__ float exp_store(const uint32_t (&s)[128], float scale_log2e, float neg_m, uint32_t p_addr,
                                            int nvalid, BeforeFirstStore&& before_first_store,
-                                           AfterLastExp&& after_last_exp, volatile unsigned* trace_row = nullptr) {
+                                           AfterLastExp&& after_last_exp) {
     // Four chunks of 32 logits.  Within a chunk all FFMAs come first, then all exponentials, then
     // the sums and the bf16 packing, so that consecutive ex2 never wait on a neighbour.  The
     // logits s[] are left intact (a stale reference maximum may force a second pass over them).
@@ -178,9 +152,6 @@ __device__ __forceinline__ float exp_store(const uint32_t (&s)[128], float scale
             if (c == 1) { before_first_store(); tmem_st_x16(p_addr, pk0); }
             tmem_st_x16(p_addr + c * 16, pk);
         }
-#ifdef FLAT_TRACE
-        if (trace_row != nullptr && (threadIdx.x & 127) == 0) trace_row[8 + c] = static_cast<unsigned>(clock64());
-#endif
     }
     float l0, l1, l2, l3;
     unpack2(lsum0, l0, l1);
@@ -200,9 +171,6 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                  float scale_log2e, const int32_t* __restrict__ valid_len, int coff, int32_t* status,
                  const int32_t* __restrict__ cu_q = nullptr, const int32_t* __restrict__ cu_k = nullptr) {
     using LY = L2<D, NT>;
-#ifdef FLAT_TRACE
-    constexpr int THREADS = LY::THREADS;
-#endif
     extern __shared__ uint8_t smem_raw[];
     uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* Qs = base;                                  // NT tiles
@@ -211,15 +179,8 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     uint64_t* bars = reinterpret_cast<uint64_t*>(base + LY::TILE_BYTES);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + LY::NUM_BARS);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-#ifdef FLAT_TRACE
-    volatile unsigned* trace_buf = reinterpret_cast<volatile unsigned*>(base + LY::TILE_BYTES + 512);
-    for (int i = threadIdx.x; i < TRACE_WORDS; i += THREADS) trace_buf[i] = 0;
-#endif
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-#ifdef FLAT_TRACE
-    const unsigned t_entry = static_cast<unsigned>(clock64());
-#endif
     const int bh = blockIdx.y;
     const int row0 = blockIdx.x * (NT * BM);
     int n = Nk;
@@ -255,9 +216,6 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
-#ifdef FLAT_TRACE
-    if (threadIdx.x == 0) { TRACE(2, 63, 0); trace_buf[(2 * 64 + 63) * 16 + 1] = t_entry; }
-#endif
 
     if (warp >= LY::SOFT_WARPS) {
       if (NT == 2) asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
@@ -342,23 +300,19 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                     }
                     tc_commit(&bars[LY::S_FULL + t]);
                     tc_commit(&bars[LY::K_EMPTY + ks]);
-                    TRACE(2, j, t);
                 }
                 __syncwarp();
             };
             auto issue_pv = [&](int j) {                 // O_t += P_t V_j, then release the V stage
                 const int vs = j % LY::VS;
                 if (elect_one()) {
-                    if (t == 0) TRACE(2, j, 4);
                     const uint64_t vd = v_desc + static_cast<uint64_t>((vs * LY::KV_BYTES) >> 4);
 #pragma unroll
                     for (int k = 0; k < BN / 16; ++k)
                         mma_ts(o_tmem, p_tmem + k * 8, vd + static_cast<uint64_t>((k * 2048) >> 4), IDESC_PV,
                                (j > 0 || k > 0));
-                    if (t == 0) TRACE(2, j, 5);
                     tc_commit(&bars[LY::PV_DONE + t]);
                     tc_commit(&bars[LY::V_EMPTY + vs]);
-                    TRACE(2, j, 2 + t);
                 }
                 __syncwarp();
             };
@@ -376,9 +330,7 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                     if (ok) issue_s(j + 1);
                 }
                 wait(LY::V_FULL + vs, vph, 0x220);
-                if (t == 0 && lane == 0) TRACE(2, j, 6);
                 wait(LY::P_FULL + t, j & 1, 0x221);
-                if (t == 0 && lane == 0) TRACE(2, j, 7);
                 if (ok) issue_pv(j);
                 if (LY::ALIAS && more) {
                     // P overlays S: the next S_t goes behind the MMA that reads P_t(j)
@@ -404,12 +356,10 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         const int nrow_min = __shfl_sync(0xffffffffu, nrow, 0);
         if (LY::TURNS && t == 1 && lane == 0) mbar_arrive(&bars[LY::TURN + (warp & 3)]);   // tile A goes first
         for (int j = 0; j < ntiles; ++j) {
-            if ((warp & 3) == 0 && lane == 0) TRACE(t, j, 0);
             ok = bounded_wait(&bars[LY::S_FULL + t], j & 1, abort_flag, status, 0x300 + t);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
-            if ((warp & 3) == 0 && lane == 0) TRACE(t, j, 1);
             uint32_t s[128];
 #pragma unroll
             for (int c = 0; c < 4; ++c) tmem_ld_x32(tl + LY::S_COL(t) + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
@@ -417,7 +367,6 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&bars[LY::S_FREE + t]);   // S_t may be overwritten (d = 64: by the next S_t)
-            if ((warp & 3) == 0 && lane == 0) TRACE(t, j, 2);
 
             const int col0 = j * BN;
             const bool tail = col0 + BN > nrow_min;      // (warp-uniform) some row has masked keys in this step
@@ -432,11 +381,9 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             bool pv_waited = LY::ALIAS || j == 0;
             auto wait_p_free = [&]() {
                 if (!pv_waited) {
-                    if ((warp & 3) == 0 && lane == 0) TRACE(t, j, 7);
                     ok = __all_sync(0xffffffffu, bounded_wait(&bars[LY::PV_DONE + t], (j - 1) & 1, abort_flag,
                                                              status, 0x320 + t));
                     pv_waited = true;
-                    if ((warp & 3) == 0 && lane == 0) TRACE(t, j, 3);
                 }
             };
             bool turn_passed = !LY::TURNS;
@@ -452,7 +399,6 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                                                          status, 0x340 + t));
                 if (!ok) break;
             }
-            if ((warp & 3) == 0 && lane == 0) TRACE(t, j, 4);
             // p = 2^(scale*s - m_ref); row sum in fp32 from the unrounded p; P rounded to bf16.
             // Any reference m_ref gives the exact softmax, so the common case reuses the one in
             // hand and takes no row maximum at all; a row sum beyond 2^40 (or inf/NaN) shows that
@@ -460,12 +406,7 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             bool careful = (j == 0) || tail;
             float lt = 0.f;
             if (!careful) {
-#ifdef FLAT_TRACE
-                lt = exp_store<false, !LY::TURNS>(s, scale_log2e, -m_ref, tl + LY::P_COL(t), BN, wait_p_free, pass_turn,
-                                      (blockIdx.x == 0 && blockIdx.y == 0 && j < 64) ? trace_buf + (t * 64 + j) * 16 : nullptr);
-#else
                 lt = exp_store<false, !LY::TURNS>(s, scale_log2e, -m_ref, tl + LY::P_COL(t), BN, wait_p_free, pass_turn);
-#endif
                 if (!ok) break;                           // (a failed wait means the stores went nowhere useful)
                 careful = __any_sync(0xffffffffu, !(lt <= OVERFLOW_SUM));
             }
@@ -499,12 +440,10 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                 if (!ok) break;
             }
             l += lt;
-            if ((warp & 3) == 0 && lane == 0) TRACE(t, j, 5);
             tc_wait_st();
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&bars[LY::P_FULL + t]);
-            if ((warp & 3) == 0 && lane == 0) TRACE(t, j, 6);
         }
         if (ok && ntiles > 0) {
             ok = bounded_wait(&bars[LY::PV_DONE + t], (ntiles - 1) & 1, abort_flag, status, 0x330 + t);
@@ -539,19 +478,9 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             }
         }
     }
-#ifdef FLAT_TRACE
-    if (threadIdx.x == 0) TRACE(2, 63, 2);               // softmax warp 0 done with its epilogue
-#endif
     tc_fence_before();
     __syncthreads();
-#ifdef FLAT_TRACE
-    if (threadIdx.x == 0) TRACE(2, 63, 3);
-#endif
     if (warp == 0) tmem_dealloc(tmem, LY::TMEM_COLS);
-#ifdef FLAT_TRACE
-    if (g_trace && blockIdx.x == 0 && blockIdx.y == 0)
-        for (int i = threadIdx.x; i < TRACE_WORDS; i += THREADS) g_trace[i] = trace_buf[i];
-#endif
 }
 
 template <int D, int NT>

@@ -47,29 +47,6 @@ namespace flat {
 using namespace ptx;
 using namespace tc;
 
-#ifdef FLAT_TRACE3
-// Developer tracing (off in the product build): CTA (0,0) keeps SM-clock stamps in shared memory
-// and copies them to a global buffer when it ends.
-__device__ unsigned* g_trace3 = nullptr;
-extern "C" int flat_debug_set_trace3(unsigned* p) {
-    return cudaMemcpyToSymbol(g_trace3, &p, sizeof(p)) == cudaSuccess ? 0 : 6;
-}
-#define TRACE3_WORDS (6 * 64 * 16)
-#ifdef FLAT_TRACE3_LIGHT
-#define TRACE_Q0 false                                 // only the arrival stamps of every warp
-#else
-#define TRACE_Q0 true
-#endif
-#define TRACE(role, iter, point)                                                              \
-    do {                                                                                      \
-        if (blockIdx.x == 0 && blockIdx.y == 0 && (iter) < 64)                                \
-            trace_buf[((role) * 64 + (iter)) * 16 + (point)] = static_cast<unsigned>(clock64()); \
-    } while (0)
-#else
-#define TRACE3_WORDS 0
-#define TRACE_Q0 false
-#define TRACE(role, iter, point) do { } while (0)
-#endif
 
 namespace {
 
@@ -78,25 +55,12 @@ constexpr int BN = 128;              // keys per step
 constexpr int HN = 64;               // keys per step and softmax thread
 constexpr float OVERFLOW_SUM = 1.0995116e12f;   // 2^40: a row sum beyond this means m_ref is stale
 constexpr float UNDERFLOW_SUM = 8.6736174e-19f; // 2^-60: a first-step sum below this means a carried m_ref is far too high
-#ifndef FLAT_TC3_CARRY_REF
-#define FLAT_TC3_CARRY_REF 1
-#endif
 // Registers per thread after the hand-over: 640 threads start with 96 each; 512 * 104 + 128 * 64 uses them all.
-#ifndef FLAT_TC3_SOFT_REGS
-#define FLAT_TC3_SOFT_REGS 104
-#define FLAT_TC3_OTHER_REGS 64
-#endif
-#ifndef FLAT_TC3_POLY
-#define FLAT_TC3_POLY true
-#endif
-#ifndef FLAT_TC3_PRODUCER_SLEEP
-#define FLAT_TC3_PRODUCER_SLEEP 400   // ns between the TMA producer's probes of a full ring (it runs far ahead: its reaction time is immaterial)
-#endif
-#ifndef FLAT_TC3_POLY_PAIRS
-#define FLAT_TC3_POLY_PAIRS 0x0202   // bit i: pair i of each 16 pairs (32 logits) takes the polynomial; two pairs = one element in eight
-#endif
-constexpr int SOFT_REGS = FLAT_TC3_SOFT_REGS, OTHER_REGS = FLAT_TC3_OTHER_REGS;
+constexpr int SOFT_REGS = 104, OTHER_REGS = 64;
 static_assert(512 * SOFT_REGS + 128 * OTHER_REGS <= 640 * 96, "register hand-over exceeds the CTA's allocation");
+constexpr bool USE_POLY = true;          // part of the exponentials on the FMA pipe (see exp_pack_x2)
+constexpr unsigned POLY_PAIRS = 0x0202;  // bit i: pair i of each 16 pairs (32 logits) takes the polynomial; two pairs = one element in eight
+constexpr unsigned PRODUCER_SLEEP = 400; // ns between the TMA producer's probes of a full ring (it runs far ahead: its reaction time is immaterial)
 
 constexpr int D = 64;                // head size of this kernel
 
@@ -110,7 +74,7 @@ struct L3 {
     static constexpr int KV_BYTES = BN * D * 2;
     static constexpr int TILE_BYTES = 2 * Q_BYTES + (KS + VS) * KV_BYTES;
     static constexpr int XCH_BYTES = 2 * 2 * 2 * BM * 4; // [maximum | row sum][tile][half][row] floats
-    static constexpr int SMEM_BYTES = TILE_BYTES + XCH_BYTES + 512 + 1024 + 4 * TRACE3_WORDS;
+    static constexpr int SMEM_BYTES = TILE_BYTES + XCH_BYTES + 512 + 1024;
     __host__ __device__ static constexpr uint32_t O_COL(int t) { return 64u * t; }
     __host__ __device__ static constexpr uint32_t X_COL(int b) { return 128u + 128u * b; }   // logit / weight buffer b
     // barrier indices
@@ -212,7 +176,7 @@ __device__ __forceinline__ void exp_pack_x2(const uint64_t (&x2)[16], uint64_t (
     for (int i = 0; i < 16; ++i) {
         float a, b;
         unpack2(x2[i], a, b);
-        if (POLY && ((FLAT_TC3_POLY_PAIRS >> i) & 1)) {
+        if (POLY && ((POLY_PAIRS >> i) & 1)) {
             xmax = max3(xmax, a, b);
             p[2 * i] = ex2_poly_lo(a);
             p[2 * i + 1] = ex2_poly_lo(b);
@@ -393,15 +357,8 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     uint64_t* bars = reinterpret_cast<uint64_t*>(base + LY::TILE_BYTES + LY::XCH_BYTES);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + LY::NUM_BARS);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-#ifdef FLAT_TRACE3
-    volatile unsigned* trace_buf = reinterpret_cast<volatile unsigned*>(base + LY::TILE_BYTES + LY::XCH_BYTES + 512);
-    for (int i = threadIdx.x; i < TRACE3_WORDS; i += LY::THREADS) trace_buf[i] = 0;
-#endif
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-#ifdef FLAT_TRACE3
-    const unsigned t_entry = static_cast<unsigned>(clock64());
-#endif
 
     if (threadIdx.x == LY::SOFT_WARPS * 32) {
         for (int i = 0; i < LY::NUM_BARS; ++i)
@@ -415,9 +372,6 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
-#ifdef FLAT_TRACE3
-    if (threadIdx.x == 0) { trace_buf[(5 * 64) * 16 + 0] = t_entry; TRACE(5, 0, 1); }
-#endif
 
     if (warp >= LY::SOFT_WARPS) {
       asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(OTHER_REGS));
@@ -434,7 +388,7 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             // the batch), or (head, token) for packed batches
             auto load_q = [&](int t, int q, int y, int z) {
                 // the logit MMAs of the previous item must have finished with this tile of shared memory
-                if (q > 0) ok = bounded_wait_s<FLAT_TC3_PRODUCER_SLEEP>(bars_s + 8 * (LY::Q_EMPTY + t), (q - 1) & 1, abort_s, status, 0x120 + t);
+                if (q > 0) ok = bounded_wait_s<PRODUCER_SLEEP>(bars_s + 8 * (LY::Q_EMPTY + t), (q - 1) & 1, abort_s, status, 0x120 + t);
                 if (!ok) return;
                 mbar_arrive_expect_tx(&bars[LY::Q_FULL + t], LY::Q_BYTES);
                 tma_load_3d(Qs + t * LY::Q_BYTES, &tmQ, &bars[LY::Q_FULL + t], 0, y, z);
@@ -442,7 +396,7 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             };
             auto load_k = [&](int J, int y, int z) {
                 const int s = J % LY::KS;
-                ok = bounded_wait_s<FLAT_TC3_PRODUCER_SLEEP>(bars_s + 8 * (LY::K_EMPTY + s), ((J / LY::KS) & 1) ^ 1, abort_s, status, 0x100 + s);
+                ok = bounded_wait_s<PRODUCER_SLEEP>(bars_s + 8 * (LY::K_EMPTY + s), ((J / LY::KS) & 1) ^ 1, abort_s, status, 0x100 + s);
                 if (!ok) return;
                 mbar_arrive_expect_tx(&bars[LY::K_FULL + s], LY::KV_BYTES);
                 tma_load_3d(Ks + s * LY::KV_BYTES, &tmK, &bars[LY::K_FULL + s], 0, y, z);
@@ -450,7 +404,7 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             };
             auto load_v = [&](int J, int y, int z) {
                 const int s = J % LY::VS;
-                ok = bounded_wait_s<FLAT_TC3_PRODUCER_SLEEP>(bars_s + 8 * (LY::V_EMPTY + s), ((J / LY::VS) & 1) ^ 1, abort_s, status, 0x110 + s);
+                ok = bounded_wait_s<PRODUCER_SLEEP>(bars_s + 8 * (LY::V_EMPTY + s), ((J / LY::VS) & 1) ^ 1, abort_s, status, 0x110 + s);
                 if (!ok) return;
                 mbar_arrive_expect_tx(&bars[LY::V_FULL + s], LY::KV_BYTES);
                 tma_load_3d(Vs + s * LY::KV_BYTES, &tmV, &bars[LY::V_FULL + s], 0, y, z);
@@ -512,10 +466,8 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                 for (int ts = 0; ts < 2; ++ts) {
                     const int g = 2 * c.J + ts, bs = g % 3;
                     if (c.j == 0) wait(LY::Q_FULL + ts, c.q & 1, 0x200 + ts);
-                    if (lane == 0) TRACE(4, g, 4);
                     // buffer bs was last used by tile-step g - 3, of the other tile
                     if (g >= 3) wait(LY::PV_DONE + (ts ^ 1) * 3 + bs, ((g - 3) / 6) & 1, 0x230 + ts);
-                    if (lane == 0) TRACE(4, g, 5);
                     if (!ok) break;
                     if (elect_one()) {
                         const uint64_t qd = q_desc + static_cast<uint64_t>((ts * LY::Q_BYTES) >> 4);
@@ -527,7 +479,6 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                         tc_commit(&bars[LY::S_FULL + ts * 3 + bs]);
                         if (ts == 1) tc_commit(&bars[LY::K_EMPTY + ks]);          // both tiles' logits have used K_j
                         if (c.j == c.it.ntiles - 1) tc_commit(&bars[LY::Q_EMPTY + ts]);   // the item's last use of Q_ts
-                        TRACE(4, g, 1);
                     }
                     __syncwarp();
                 }
@@ -538,10 +489,8 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             const uint64_t v_desc = make_smem_desc_sw128(smem_u32(Vs), BN * 128, 1024);
             while (c.valid && ok) {
                 const int g = 2 * c.J + t, b = g % 3, vs = c.J % LY::VS;
-                if (lane == 0) TRACE(4, g, 0);
                 wait(LY::V_FULL + vs, (c.J / LY::VS) & 1, 0x220);
                 wait(LY::P_FULL + t * 3 + b, (g / 6) & 1, 0x221);
-                if (lane == 0) TRACE(4, g, 2);
                 if (!ok) break;
                 if (elect_one()) {
                     const uint64_t vd = v_desc + static_cast<uint64_t>((vs * LY::KV_BYTES) >> 4);
@@ -552,7 +501,6 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                                vd + static_cast<uint64_t>((k * 2048) >> 4), IDESC_PV, (c.j > 0 || k > 0));
                     tc_commit(&bars[LY::PV_DONE + t * 3 + b]);
                     tc_commit(&bars[LY::V_EMPTY + vs]);
-                    TRACE(4, g, 3);
                 }
                 __syncwarp();
                 cursor_next<VL>(c, sc);
@@ -573,8 +521,6 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         const uint32_t xm_own = smem_u32(xch + ((t * 2 + h) * BM + q * 32 + lane));
         const bool neg_scale = scale_log2e < 0.f;
         bool ok = true;
-        const int trole = t * 2 + h;
-        (void)trole;
         int b = t;                                       // buffer of tile-step g = 2 J + t: g % 3
         int g = t;                                       // this tile's next tile-step (J: key steps of all items so far)
         // The reference maximum is carried from item to item: any reference gives the exact softmax
@@ -593,28 +539,18 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         const int nrow = rlim < it.n ? (rlim < 0 ? 0 : static_cast<int>(rlim)) : it.n;
         const int nrow_min = __shfl_sync(0xffffffffu, nrow, 0);
         float l = 0.f;
-        const bool exact_first = !FLAT_TC3_CARRY_REF || !first_item_done || sc.coff < (1 << 29) || it.n < BN;   // (the same for all warps)
+        const bool exact_first = !first_item_done || sc.coff < (1 << 29) || it.n < BN;   // (the same for all warps)
         first_item_done = true;
         for (int j = 0; j < ntiles; ++j, g += 2, b = (b == 0 ? 2 : b - 1)) {      // g += 2  <=>  b -= 1 (mod 3)
             // this warp's 64 logits of S(g); its 32 packed columns of P(g) go over the first half of them
             const uint32_t s_addr = tl + LY::X_COL(b) + h * HN;
-            if (TRACE_Q0 && q == 0 && lane == 0) TRACE(trole, j, 0);
             const uint32_t xph = static_cast<uint32_t>(g / 6) & 1u;   // phase parity of this tile's use of the buffer
             // A warp whose wait fails does not leave by itself: it goes on to the next vote with its
             // partner (reading TMEM that may not be ready is harmless, nothing is stored), so that the
             // two always pass the same sequence of named barriers and leave together.
-#ifdef FLAT_TRACE3
-            const long long t_wait0 = clock64();
-#endif
             ok = bounded_wait_s(bars_s + 8 * (LY::S_FULL + t * 3 + b), xph, abort_s, status, 0x300 + t);
             ok = __all_sync(0xffffffffu, ok);
             tc_fence_after();
-#ifdef FLAT_TRACE3
-            if (lane == 0 && blockIdx.x == 0 && j < 64)                       // how long this warp waited for its logits
-                trace_buf[(trole * 64 + j) * 16 + 12 + q] = static_cast<unsigned>(clock64() - t_wait0);
-            if (!TRACE_Q0 && lane == 0) TRACE(trole, j, q);                   // light mode: when the logits were seen
-#endif
-            if (TRACE_Q0 && q == 0 && lane == 0) TRACE(trole, j, 1);
             const int col0 = j * BN + h * HN;
             const bool tail = col0 + HN > nrow_min;      // (warp-uniform) some row has masked keys in this step
             const int nvalid = nrow > col0 ? (nrow - col0 < HN ? nrow - col0 : HN) : 0;   // per row
@@ -632,7 +568,6 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                 float lt;
                 tmem_ld_x32(s_addr, r);
                 tc_wait_ld();
-                if (TRACE_Q0 && q == 0 && lane == 0) TRACE(trole, j, 2);
                 if (tail) {
                     exp_pack32<true, false>(r, scale_log2e, -m_ref, nvalid, ls, pk[0]);
                     tmem_ld_x32(s_addr + 32, r);
@@ -646,10 +581,10 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                     float xmax = 0.f;
                     scale32(r, scale2, neg_m2, x2);
                     tmem_ld_x32(s_addr + 32, r);         // the second 32 logits arrive during the first 32 exponentials
-                    exp_pack_x2<FLAT_TC3_POLY>(x2, l2, xmax, pk[0]);
+                    exp_pack_x2<USE_POLY>(x2, l2, xmax, pk[0]);
                     tc_wait_ld();
                     scale32(r, scale2, neg_m2, x2);
-                    exp_pack_x2<FLAT_TC3_POLY>(x2, l2, xmax, pk[1]);
+                    exp_pack_x2<USE_POLY>(x2, l2, xmax, pk[1]);
                     float a, b2, c, d2;
                     unpack2(l2[0], a, b2);
                     unpack2(l2[1], c, d2);
@@ -657,12 +592,10 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                     ls[0] = lt;
                     if (xmax > 126.f) lt = INFINITY;      // the polynomial was fed an argument beyond its range
                 }
-                if (TRACE_Q0 && q == 0 && lane == 0) TRACE(trole, j, 3);
                 // (a first step on a carried reference must also show that the reference is not far
                 // ABOVE the row's logits: its sum must not have vanished)
                 careful = pair_any(pair_id, !(lt <= OVERFLOW_SUM) || (j == 0 && !(lt >= UNDERFLOW_SUM)) || !ok);
             }
-            if (TRACE_Q0 && q == 0 && lane == 0) TRACE(trole, j, 4);
             if (careful) {
                 if (pair_any(pair_id, !ok)) { ok = false; break; }     // (both warps are here: j == 0 or the joint vote)
                 if (j == 0) m_ref = -INFINITY;           // nothing accumulated yet: the item starts from its own maximum
@@ -732,7 +665,7 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                         tmem_ld_x32(s_addr + c * 32, r);
                         tc_wait_ld();
                         scale32(r, scale2, neg_m2, x2);
-                        exp_pack_x2<FLAT_TC3_POLY>(x2, l2, xmax, pk[c]);
+                        exp_pack_x2<USE_POLY>(x2, l2, xmax, pk[c]);
                     }
                     float a, b2, c2, d2;
                     unpack2(l2[0], a, b2);
@@ -744,7 +677,6 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             // careful path waits for anything)
             if (careful && pair_any(pair_id, !ok)) ok = false;
             if (!ok) break;
-            if (TRACE_Q0 && q == 0 && lane == 0) TRACE(trole, j, 5);
             tmem_st_x16(s_addr, pk[0]);
             tmem_st_x16(s_addr + 16, pk[1]);
             l += (ls[0] + ls[1]) + (ls[2] + ls[3]);
@@ -752,8 +684,6 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive_s(bars_s + 8 * (LY::P_FULL + t * 3 + b));
-            if (TRACE_Q0 && q == 0 && lane == 0) TRACE(trole, j, 7);
-            if (lane == 0) TRACE(trole, j, 8 + q);
         }
         if (ok && ntiles > 0) {
             // the last O_t += P V of the item (the issuer's MMAs complete in order)
@@ -806,17 +736,9 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         }
         }
     }
-#ifdef FLAT_TRACE3
-    if (threadIdx.x == 0) TRACE(5, 0, 2);
-#endif
     tc_fence_before();
     __syncthreads();
     if (warp == 0) tmem_dealloc(tmem, LY::TMEM_COLS);
-#ifdef FLAT_TRACE3
-    if (threadIdx.x == 0) TRACE(5, 0, 3);
-    if (g_trace3 && blockIdx.x == 0 && blockIdx.y == 0)
-        for (int i = threadIdx.x; i < TRACE3_WORDS; i += LY::THREADS) g_trace3[i] = trace_buf[i];
-#endif
 }
 
 int launch_tc3(const Problem& p, cudaStream_t st) {

@@ -1,7 +1,9 @@
 // flat_attn_naive_fwd_static: the unfused baseline for callers that cannot allocate device
 // memory.  The logit and weight tensors live in one file-scope device array that is part of
 // the library image, so the call path contains no cudaMalloc/cudaFree and no allocating
-// library routine.
+// library routine.  (The array becomes resident when the runtime loads this part of the
+// library on a device -- at the latest during the first call's address lookup -- which is the
+// one moment at which a device short of memory can make the call fail.)
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -52,6 +54,13 @@ extern "C" int flat_attn_naive_fwd_static(const void* Q, const void* K, const vo
     if (elems > kMaxElems) return FLAT_ERR_WORKSPACE;
     elems *= Nk;
     if (elems > kMaxElems) return FLAT_ERR_WORKSPACE;
+    // Then the remaining argument rules (pointers, d, alignment, scale), with stand-ins for L and A,
+    // so that a bad argument is reported as such before the device is looked at.
+    {
+        flat_attn_params_t chk{Q, K, V, O, B, H, Nq, Nk, d, scale, FLAT_DTYPE_BF16, nullptr, nullptr, FLAT_VARIANT_AUTO, 0};
+        const int rc = flat::check_params(&chk);
+        if (rc != FLAT_OK) return rc;
+    }
     void* base = nullptr;
     const int rc = scratch_for_current_device(&base);
     if (rc != FLAT_OK) return rc;

@@ -110,6 +110,10 @@ def test_naive_and_host_argument_errors(api):
     assert api._lib.flat_attn_naive_fwd_ex(ctypes.byref(p), None, 0x60000, None) == 1
     assert api._lib.flat_attn_naive_fwd_ex(ctypes.byref(p), 0x60004, 0x70000, None) == 4
     assert api._lib.flat_attn_naive_fwd(0x10000, 0x20000, 0x30000, 0x40000, 0x50000, 0x60000, 1, 1, 0, 5, 64, 1.0, None) == 2
+    # the baseline's row softmax uses one thread block per row: more than 2^31 - 1 rows are refused up front
+    rows = _params(api, B=4, H=1, Nq=2 ** 29, Nk=8)
+    assert api._lib.flat_attn_naive_fwd_ex(ctypes.byref(rows), 0x60000, 0x70000, None) == 2
+    assert api._lib.flat_attn_naive_fwd_ex(ctypes.byref(_params(api, B=2, H=1, Nq=2 ** 30, Nk=8)), 0x60000, 0x70000, None) == 2
     need = api.flat_attn_host_workspace_bytes(1, 2, 128, 128, 64)
     assert need == 4 * 2 * 128 * 64 * 2 + 256
     assert api.flat_attn_host_workspace_bytes(1, 2, 128, 128, 64, 1) == 4 * 2 * 128 * 64 * 4 + 256
@@ -117,6 +121,17 @@ def test_naive_and_host_argument_errors(api):
     assert api._lib.flat_attn_fwd_host(ctypes.byref(p), None, need, None) == 1
     assert api._lib.flat_attn_fwd_host(ctypes.byref(p), 0x100010, need, None) == 4
     assert api._lib.flat_attn_fwd_host(ctypes.byref(p), 0x100000, need - 1, None) == 5
+
+
+def test_device_error_word_and_last_variant_calls(api):
+    # host-side behaviour only: a NULL output pointer is refused, and before any fused call the last variant is 0
+    assert api._lib.flat_attn_last_device_error(None) == 1
+    import subprocess
+    import sys
+    r = subprocess.run([sys.executable, "-c",
+                        "import paper_2107_06419_b200.api as a; print(a.flat_attn_last_variant())"],
+                       cwd=ROOT, capture_output=True, text=True)
+    assert r.returncode == 0 and r.stdout.strip() == "0", r.stderr
 
 
 def test_binding_rejects_bad_tensors(api):

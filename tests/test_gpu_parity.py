@@ -414,6 +414,31 @@ def test_bounded_wait_gives_up_cleanly(api):
     check_bf16(got, oracle.attention(Qb, Kb, Vb, 0.125)["O"], "after timeout self-test")
 
 
+def test_give_up_without_a_status_word_leaves_a_trace(api):
+    """Callers that pass no status word (flat_attn_fwd) can still learn of a device-side give-up: the
+    code goes to the library's sticky word.  The wait that runs out is the self-test's (a barrier that
+    nothing completes); nothing faults."""
+    api.flat_attn_clear_device_error()
+    rng = np.random.default_rng(98)
+    Qb, Kb, Vb = rand_bits(rng, (2, 8, 2048, 64)), rand_bits(rng, (2, 8, 2048, 64)), rand_bits(rng, (2, 8, 2048, 64))
+    Q, K, V = bf16_tensor(Qb), bf16_tensor(Kb), bf16_tensor(Vb)
+    O = torch.empty_like(Q)
+    api.flat_attn_fwd(Q, K, V, O, 0.125)
+    torch.cuda.synchronize()
+    assert api.flat_attn_last_device_error() == 0          # a healthy call leaves the word alone
+    assert api.flat_attn_last_variant() == api.FLAT_VARIANT_TC3
+    api.flat_attn_selftest_wait_timeout(None)
+    torch.cuda.synchronize()
+    assert api.flat_attn_last_device_error() == api.FLAT_SELFTEST_TIMEOUT_CODE
+    O2 = torch.empty_like(Q)
+    api.flat_attn_fwd(Q, K, V, O2, 0.125)
+    torch.cuda.synchronize()
+    assert api.flat_attn_last_device_error() == api.FLAT_SELFTEST_TIMEOUT_CODE   # sticky until cleared
+    assert torch.equal(O.view(torch.int16), O2.view(torch.int16))
+    api.flat_attn_clear_device_error()
+    assert api.flat_attn_last_device_error() == 0
+
+
 @pytest.mark.parametrize("sigma,scale", [(3.0, 1.0), (1.0, 20.0), (6.0, 0.5)])
 def test_wide_dynamic_range(api, sigma, scale):
     """Logits with a standard deviation of dozens to hundreds: row maxima jump by far more than the

@@ -70,3 +70,23 @@ def test_whole_job_rate_and_single_process_identity():
     assert shard.whole_job_rate(1e12, 8, 2.0) == 8e12 / 2e-3
     assert shard.max_over_ranks([1.5, 2.5], torch.device("cpu")) == [1.5, 2.5]
     assert shard.rank_seed(7, 0) == 7 and shard.rank_seed(7, 3) != shard.rank_seed(7, 2)
+
+
+def test_bench_gpus_flag_starts_the_ranks_itself():
+    """`bench.py --gpus 2` without a launcher must create two ranks (here: gloo, no CUDA call) and
+    report them; run the way the driver runs the single-command form."""
+    import json
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    r = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--gpus", "2", "--steps", "2", "--warmup", "3",
+                        "--dry-run", "--backend", "gloo", "--workload", "c1_bert_base_512"],
+                       capture_output=True, text=True, env=env, timeout=300)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [ln for ln in r.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1, r.stdout
+    out = json.loads(lines[0])
+    assert out["n_gpus"] == 2 and out["dry_run"] is True
+    assert out["ms_per_step"] == 2.0                    # the slower rank's fake step time
+    assert out["value"] == 2 * inputs.WORKLOADS["c1_bert_base_512"].flops / 2e-3 / 1e12
