@@ -15,16 +15,16 @@ import subprocess
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-_SRC = os.path.join(_HERE, "oracle_attn.cpp")
+_SRCS = [os.path.join(_HERE, "oracle_attn.cpp"), os.path.join(_HERE, "oracle_attn_bwd.cpp")]
 _LIB = os.path.join(_HERE, "liboracle_attn.so")
 _lib = None
 
 
 def build(force: bool = False) -> str:
     """Compile the oracle with g++ (-O2, no fast-math) if missing or stale."""
-    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < max(os.path.getmtime(f) for f in _SRCS):
         tmp = _LIB + ".%d.tmp" % os.getpid()
-        subprocess.check_call(["g++", "-O2", "-std=c++17", "-fPIC", "-shared", "-pthread", _SRC, "-o", tmp])
+        subprocess.check_call(["g++", "-O2", "-std=c++17", "-fPIC", "-shared", "-pthread"] + _SRCS + ["-o", tmp])
         os.replace(tmp, _LIB)
     return _LIB
 
@@ -33,12 +33,20 @@ def _load():
     global _lib
     if _lib is None:
         lib = ctypes.CDLL(build())
-        lib.oracle_attn_rows.restype = ctypes.c_int
-        lib.oracle_attn_rows.argtypes = [
+        lib.oracle_attn_rows_lse.restype = ctypes.c_int
+        lib.oracle_attn_rows_lse.argtypes = [
             ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int,
             ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, ctypes.c_float,
             ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p, ctypes.c_int64,
-            ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.POINTER(ctypes.c_int)]
+            ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int,
+            ctypes.POINTER(ctypes.c_int)]
+        lib.oracle_attn_bwd_heads.restype = ctypes.c_int
+        lib.oracle_attn_bwd_heads.argtypes = [
+            ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int,
+            ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, ctypes.c_float,
+            ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p, ctypes.c_int64,
+            ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int,
+            ctypes.POINTER(ctypes.c_int)]
         lib.oracle_hardware_threads.restype = ctypes.c_int
         _lib = lib
     return _lib
@@ -49,14 +57,15 @@ def hardware_threads() -> int:
 
 
 def attention(Q, K, V, scale, valid_len=None, rows=None, want_logits=False, want_weights=False,
-              nthreads: int = 0, causal: bool = False):
+              nthreads: int = 0, causal: bool = False, want_lse=False):
     """Exact attention in double precision.
 
     Q: [B,H,Nq,d], K/V: [B,H,Nk,d]; dtype uint16 (bf16 bit patterns) or float32.
     rows: optional int64 array of flat row ids ((b*H+h)*Nq + i); default all rows.
     causal: query i attends keys j <= i + (Nk - Nq) only (intersected with valid_len).
     Returns dict with 'O' ([B,H,Nq,d] or [nrows,d] float64), optionally 'L' and
-    'A' ([..., Nk]), and 'threads' (threads used).
+    'A' ([..., Nk]), 'LSE' ([B,H,Nq] or [nrows]: log of the row's sum of exp(scaled logit) over its
+    valid keys, -inf for a row without any), and 'threads' (threads used).
     """
     Q = np.ascontiguousarray(Q); K = np.ascontiguousarray(K); V = np.ascontiguousarray(V)
     if Q.dtype == np.uint16:
@@ -86,11 +95,12 @@ def attention(Q, K, V, scale, valid_len=None, rows=None, want_logits=False, want
     O = np.empty(oshape, dtype=np.float64)
     L = np.empty(lshape, dtype=np.float64) if want_logits else None
     A = np.empty(lshape, dtype=np.float64) if want_weights else None
+    LSE = np.empty(oshape[:-1], dtype=np.float64) if want_lse else None
     used = ctypes.c_int(0)
     ptr = lambda a: None if a is None else a.ctypes.data_as(ctypes.c_void_p)
-    rc = _load().oracle_attn_rows(ptr(Q), ptr(K), ptr(V), dtype, B, H, Nq, Nk, d, float(np.float32(scale)),
-                                  ptr(vl), 1 if causal else 0, ptr(rows), n, ptr(O), ptr(L), ptr(A), int(nthreads),
-                                  ctypes.byref(used))
+    rc = _load().oracle_attn_rows_lse(ptr(Q), ptr(K), ptr(V), dtype, B, H, Nq, Nk, d, float(np.float32(scale)),
+                                      ptr(vl), 1 if causal else 0, ptr(rows), n, ptr(O), ptr(L), ptr(A), ptr(LSE),
+                                      int(nthreads), ctypes.byref(used))
     if rc != 0:
         raise ValueError("oracle_attn_rows rejected its arguments (code %d)" % rc)
     out = {"O": O, "threads": used.value}
@@ -98,7 +108,54 @@ def attention(Q, K, V, scale, valid_len=None, rows=None, want_logits=False, want
         out["L"] = L
     if A is not None:
         out["A"] = A
+    if LSE is not None:
+        out["LSE"] = LSE
     return out
+
+
+def attention_bwd(Q, K, V, dO, scale, valid_len=None, causal: bool = False, heads=None, nthreads: int = 0):
+    """Gradient of exact attention (the chain rule on Section 2's steps 2-4) in double precision.
+
+    Q, dO: [B,H,Nq,d], K, V: [B,H,Nk,d]; uint16 (bf16 bit patterns) or float32, one dtype for all.
+    heads: optional int64 array of flat head ids b*H + h to compute (each complete); default all.
+    Returns dict: 'dQ' [B,H,Nq,d] (or [nheads,Nq,d]), 'dK', 'dV' [B,H,Nk,d] (or [nheads,Nk,d]),
+    'LSE' [B,H,Nq] (or [nheads,Nq]), all float64, and 'threads'.
+    """
+    Q, K, V, dO = (np.ascontiguousarray(x) for x in (Q, K, V, dO))
+    if Q.dtype == np.uint16:
+        dtype = 0
+    elif Q.dtype == np.float32:
+        dtype = 1
+    else:
+        raise TypeError("Q/K/V/dO must be uint16 (bf16 bits) or float32")
+    if any(x.dtype != Q.dtype for x in (K, V, dO)):
+        raise TypeError("Q, K, V, dO must share a dtype")
+    B, H, Nq, d = Q.shape
+    Nk = K.shape[2]
+    if K.shape != (B, H, Nk, d) or V.shape != (B, H, Nk, d) or dO.shape != Q.shape:
+        raise ValueError("shape mismatch")
+    vl = None
+    if valid_len is not None:
+        vl = np.ascontiguousarray(valid_len, dtype=np.int32)
+        if vl.shape != (B,):
+            raise ValueError("valid_len must have shape [B]")
+    if heads is not None:
+        heads = np.ascontiguousarray(heads, dtype=np.int64)
+        lead = (heads.shape[0],)
+    else:
+        lead = (B, H)
+    dQ = np.empty(lead + (Nq, d), dtype=np.float64)
+    dK = np.empty(lead + (Nk, d), dtype=np.float64)
+    dV = np.empty(lead + (Nk, d), dtype=np.float64)
+    LSE = np.empty(lead + (Nq,), dtype=np.float64)
+    used = ctypes.c_int(0)
+    ptr = lambda a: None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+    rc = _load().oracle_attn_bwd_heads(ptr(Q), ptr(K), ptr(V), ptr(dO), dtype, B, H, Nq, Nk, d, float(np.float32(scale)),
+                                       ptr(vl), 1 if causal else 0, ptr(heads), 0 if heads is None else heads.shape[0],
+                                       ptr(dQ), ptr(dK), ptr(dV), ptr(LSE), int(nthreads), ctypes.byref(used))
+    if rc != 0:
+        raise ValueError("oracle_attn_bwd_heads rejected its arguments (code %d)" % rc)
+    return {"dQ": dQ, "dK": dK, "dV": dV, "LSE": LSE, "threads": used.value}
 
 
 # ------------------------------------------------------------------------------------------------

@@ -58,6 +58,7 @@ struct Problem {
     double* O;                       // [nrows, d]
     double* L;                       // [nrows, Nk] scaled logits, or null
     double* A;                       // [nrows, Nk] softmax weights, or null
+    double* LSE;                     // [nrows] log of the row's sum of exponentials of the scaled logits, or null
 };
 
 inline double elem(const void* base, int dtype, int64_t idx) {
@@ -96,6 +97,7 @@ void attend_row(const Problem& p, int64_t r, std::vector<double>& s) {
 
     for (int64_t t = 0; t < p.d; ++t) o[t] = 0.0;
     if (arow) for (int64_t j = 0; j < p.Nk; ++j) arow[j] = 0.0;
+    if (p.LSE) p.LSE[r] = -INFINITY; // (the empty sum)
     if (n <= 0) return;              // no valid key: O = 0 by convention
 
     // Step 3: softmax along the key index.
@@ -103,6 +105,7 @@ void attend_row(const Problem& p, int64_t r, std::vector<double>& s) {
     for (int64_t j = 1; j < n; ++j) if (s[j] > m) m = s[j];
     double l = 0.0;
     for (int64_t j = 0; j < n; ++j) { s[j] = std::exp(s[j] - m); l += s[j]; }
+    if (p.LSE) p.LSE[r] = m + std::log(l);
     for (int64_t j = 0; j < n; ++j) s[j] /= l;
     if (arow) for (int64_t j = 0; j < n; ++j) arow[j] = s[j];
 
@@ -125,10 +128,10 @@ extern "C" {
 
 // Returns 0 on success, 1 on a bad argument.  `nthreads` <= 0 means "all hardware
 // threads"; the count actually used is written to *threads_used if non-null.
-int oracle_attn_rows(const void* Q, const void* K, const void* V, int dtype,
-                     int64_t B, int64_t H, int64_t Nq, int64_t Nk, int64_t d, float scale,
-                     const int32_t* valid_len, int causal, const int64_t* rows, int64_t nrows,
-                     double* O, double* L, double* A, int nthreads, int* threads_used) {
+int oracle_attn_rows_lse(const void* Q, const void* K, const void* V, int dtype,
+                         int64_t B, int64_t H, int64_t Nq, int64_t Nk, int64_t d, float scale,
+                         const int32_t* valid_len, int causal, const int64_t* rows, int64_t nrows,
+                         double* O, double* L, double* A, double* LSE, int nthreads, int* threads_used) {
     if (!Q || !K || !V || !O) return 1;
     if (B < 1 || H < 1 || Nq < 1 || Nk < 1 || d < 1) return 1;
     if (dtype != 0 && dtype != 1) return 1;
@@ -138,7 +141,7 @@ int oracle_attn_rows(const void* Q, const void* K, const void* V, int dtype,
     if (rows) for (int64_t r = 0; r < nrows; ++r) if (rows[r] < 0 || rows[r] >= total) return 1;
     if (valid_len) for (int64_t b = 0; b < B; ++b) if (valid_len[b] < 0 || valid_len[b] > Nk) return 1;
 
-    Problem p{Q, K, V, dtype, B, H, Nq, Nk, d, static_cast<double>(scale), valid_len, causal ? 1 : 0, rows, nrows, O, L, A};
+    Problem p{Q, K, V, dtype, B, H, Nq, Nk, d, static_cast<double>(scale), valid_len, causal ? 1 : 0, rows, nrows, O, L, A, LSE};
     int nt = nthreads > 0 ? nthreads : static_cast<int>(std::thread::hardware_concurrency());
     if (nt < 1) nt = 1;
     if (nt > nrows) nt = nrows > 0 ? static_cast<int>(nrows) : 1;
@@ -153,6 +156,14 @@ int oracle_attn_rows(const void* Q, const void* K, const void* V, int dtype,
     }
     for (auto& th : pool) th.join();
     return 0;
+}
+
+int oracle_attn_rows(const void* Q, const void* K, const void* V, int dtype,
+                     int64_t B, int64_t H, int64_t Nq, int64_t Nk, int64_t d, float scale,
+                     const int32_t* valid_len, int causal, const int64_t* rows, int64_t nrows,
+                     double* O, double* L, double* A, int nthreads, int* threads_used) {
+    return oracle_attn_rows_lse(Q, K, V, dtype, B, H, Nq, Nk, d, scale, valid_len, causal, rows, nrows, O, L, A,
+                                nullptr, nthreads, threads_used);
 }
 
 int oracle_hardware_threads(void) {
