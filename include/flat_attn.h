@@ -96,6 +96,13 @@ typedef struct flat_attn_params {
                                   with k_valid_len.  The paper names masking only in passing
                                   (Section 2, footnote); its decoder workloads need it.  The
                                   unfused baseline honours it too (A is 0 beyond the limit).    */
+    float* lse;                /* optional device output [B,H,Nq] fp32 (4-byte aligned), fused
+                                  path only: lse[b,h,i] = log sum_j exp(scale * q_i . k_j) over the
+                                  keys that row i sees (natural logarithm; -inf for a row without
+                                  any).  It is what flat_attn_bwd needs from the forward pass.
+                                  Written by the SIMT, TC2, TC2_SINGLE and TC3 kernels (AUTO picks
+                                  among these when it is set); FLAT_ERR_UNSUPPORTED for the others.
+                                  The paper has no counterpart (it stops at inference).           */
 } flat_attn_params_t;
 
 /*
@@ -126,6 +133,39 @@ int flat_attn_fwd_ex(const flat_attn_params_t* p, void* stream);
 int flat_attn_naive_fwd(const void* Q, const void* K, const void* V, void* O, void* L, void* A,
                         int B, int H, int Nq, int Nk, int d, float scale, void* stream);
 int flat_attn_naive_fwd_ex(const flat_attn_params_t* p, void* L, void* A, void* stream);
+
+/*
+ * Backward pass of the fused attention: gradients dQ, dK, dV of a scalar loss, given dO = dLoss/dO.
+ * The paper describes the forward operators only; this is the chain rule on its Section 2 steps 2-4,
+ * run with the idea of its Section 5: the [B,H,Nq,Nk] intermediates (the weights, their gradient and
+ * the logit gradient) are rebuilt tile by tile on chip from Q, K, V and the forward's `lse`, and never
+ * reach device memory.  With S = scale Q K^T, P = exp(S - lse) and delta_i = sum_t dO[i,t] O[i,t]:
+ *     dV = P^T dO      dP = dO V^T      dS = P o (dP - delta)      dQ = scale dS K      dK = scale dS^T Q
+ * Masks as in the forward (k_valid_len, causal): masked (query, key) pairs carry no gradient, masked
+ * keys get dK = dV = 0, a query row without any visible key gets dQ = 0.
+ *   Q, O, dO, dQ : [B,H,Nq,d] bf16      K, V, dK, dV : [B,H,Nk,d] bf16      (16-byte aligned)
+ *   lse          : [B,H,Nq] fp32, as written by flat_attn_fwd_ex (params.lse) for the same inputs
+ *   delta        : [B,H,Nq] fp32 scratch owned by the caller (4-byte aligned); overwritten
+ * Two kernels are enqueued on `stream` (dQ and delta; then dK and dV), no atomics, results are
+ * bit-reproducible.  bf16 only, d in {64, 128} (FLAT_ERR_UNSUPPORTED otherwise: no fallback); other
+ * argument rules and error codes as for flat_attn_fwd_ex; nothing is launched on an argument error.
+ * `p` is a HOST pointer, read before the call returns.
+ */
+typedef struct flat_attn_bwd_params {
+    const void *Q, *K, *V, *O, *dO;
+    const float* lse;
+    void *dQ, *dK, *dV;
+    float* delta;
+    int B, H, Nq, Nk, d;
+    float scale;
+    const int32_t* k_valid_len;/* device, [B], or NULL                                          */
+    int32_t* status;           /* optional device word, as in flat_attn_params_t                */
+    int causal;                /* 0 / 1, as in flat_attn_params_t                                */
+} flat_attn_bwd_params_t;
+int flat_attn_bwd_ex(const flat_attn_bwd_params_t* p, void* stream);
+int flat_attn_bwd(const void* Q, const void* K, const void* V, const void* O, const void* dO, const float* lse,
+                  void* dQ, void* dK, void* dV, float* delta,
+                  int B, int H, int Nq, int Nk, int d, float scale, void* stream);
 
 /*
  * Fused attention over a PACKED batch of sequences of different lengths (no padding): the same
@@ -200,8 +240,8 @@ int flat_fc_fwd(const void* X, const void* W, void* Y, int M, int K, int Nout, i
  * neighbours; to the caller it behaves like work enqueued on `stream`.  The side
  * streams and events are created once per device and host thread and never freed
  * (no device memory is allocated).
- * p->Q, p->K, p->V, p->O and p->k_valid_len are HOST pointers here; p->status is
- * still a device pointer or NULL.  `workspace` is a caller-owned DEVICE buffer of at
+ * p->Q, p->K, p->V, p->O and p->k_valid_len are HOST pointers here; p->status and
+ * p->lse are still device pointers or NULL.  `workspace` is a caller-owned DEVICE buffer of at
  * least flat_attn_host_workspace_bytes(...) bytes, 256-byte aligned.
  * The operation is that of flat_attn_fwd_ex; the paper has no counterpart for the copies.
  */

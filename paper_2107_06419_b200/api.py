@@ -33,7 +33,7 @@ EXPORTS = ["flat_attn_fwd", "flat_attn_fwd_ex", "flat_attn_naive_fwd", "flat_att
            "flat_attn_status_string", "flat_attn_version",
            "flat_qkv_proj_fwd", "flat_out_proj_fwd", "flat_attn_layer_fwd", "flat_fc_fwd",
            "flat_attn_varlen_fwd", "flat_attn_last_variant", "flat_attn_last_device_error",
-           "flat_attn_clear_device_error"]
+           "flat_attn_clear_device_error", "flat_attn_bwd", "flat_attn_bwd_ex"]
 
 
 class flat_attn_params_t(ctypes.Structure):
@@ -41,10 +41,23 @@ class flat_attn_params_t(ctypes.Structure):
                 ("B", ctypes.c_int), ("H", ctypes.c_int), ("Nq", ctypes.c_int), ("Nk", ctypes.c_int),
                 ("d", ctypes.c_int), ("scale", ctypes.c_float), ("dtype", ctypes.c_int),
                 ("k_valid_len", ctypes.c_void_p), ("status", ctypes.c_void_p), ("variant", ctypes.c_int),
-                ("causal", ctypes.c_int)]
+                ("causal", ctypes.c_int), ("lse", ctypes.c_void_p)]
+
+
+class flat_attn_bwd_params_t(ctypes.Structure):
+    _fields_ = [("Q", ctypes.c_void_p), ("K", ctypes.c_void_p), ("V", ctypes.c_void_p), ("O", ctypes.c_void_p),
+                ("dO", ctypes.c_void_p), ("lse", ctypes.c_void_p), ("dQ", ctypes.c_void_p), ("dK", ctypes.c_void_p),
+                ("dV", ctypes.c_void_p), ("delta", ctypes.c_void_p),
+                ("B", ctypes.c_int), ("H", ctypes.c_int), ("Nq", ctypes.c_int), ("Nk", ctypes.c_int),
+                ("d", ctypes.c_int), ("scale", ctypes.c_float), ("k_valid_len", ctypes.c_void_p),
+                ("status", ctypes.c_void_p), ("causal", ctypes.c_int)]
 
 
 _vp, _i, _f = ctypes.c_void_p, ctypes.c_int, ctypes.c_float
+_lib.flat_attn_bwd_ex.argtypes = [ctypes.POINTER(flat_attn_bwd_params_t), _vp]
+_lib.flat_attn_bwd_ex.restype = _i
+_lib.flat_attn_bwd.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _f, _vp]
+_lib.flat_attn_bwd.restype = _i
 _lib.flat_attn_fwd.argtypes = [_vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _f, _vp]
 _lib.flat_attn_fwd.restype = _i
 _lib.flat_attn_fwd_ex.argtypes = [ctypes.POINTER(flat_attn_params_t), _vp]
@@ -136,7 +149,7 @@ def _dtype_code(t) -> int:
     raise TypeError("Q/K/V/O must be bfloat16 or float32")
 
 
-def _params(Q, K, V, O, scale, k_valid_len, status, variant, host=False, causal=False):
+def _params(Q, K, V, O, scale, k_valid_len, status, variant, host=False, causal=False, lse=None):
     B, H, Nq, d = Q.shape
     Nk = K.shape[2]
     if tuple(K.shape) != (B, H, Nk, d) or tuple(V.shape) != (B, H, Nk, d) or tuple(O.shape) != (B, H, Nq, d):
@@ -160,6 +173,12 @@ def _params(Q, K, V, O, scale, k_valid_len, status, variant, host=False, causal=
     p.status = None if status is None else status.data_ptr()
     p.variant = int(variant)
     p.causal = 1 if causal else 0
+    if lse is not None:
+        if lse.dtype != torch.float32 or tuple(lse.shape) != (B, H, Nq) or not lse.is_cuda or not lse.is_contiguous():
+            raise ValueError("lse must be a contiguous CUDA float32 tensor [B,H,Nq]")
+        p.lse = lse.data_ptr()
+    else:
+        p.lse = None
     return p
 
 
@@ -178,12 +197,54 @@ def flat_attn_fwd(Q, K, V, O, scale, stream=None):
 
 
 def flat_attn_fwd_ex(Q, K, V, O, scale, k_valid_len=None, status=None, variant=FLAT_VARIANT_AUTO, stream=None,
-                     causal=False):
+                     causal=False, lse=None):
     """Fused attention with dtype choice (from the tensors), key-padding mask, kernel choice and
-    causal mask (query i sees keys j <= i + (Nk - Nq))."""
-    p = _params(Q, K, V, O, scale, k_valid_len, status, variant, causal=causal)
+    causal mask (query i sees keys j <= i + (Nk - Nq)); `lse` [B,H,Nq] float32 receives each row's
+    log-sum-exp of the scaled logits (what the backward pass needs)."""
+    p = _params(Q, K, V, O, scale, k_valid_len, status, variant, causal=causal, lse=lse)
     _check(_lib.flat_attn_fwd_ex(ctypes.byref(p), _stream_ptr(stream)))
     return O
+
+
+def _bwd_params(Q, K, V, O, dO, lse, dQ, dK, dV, delta, scale, k_valid_len, status, causal):
+    B, H, Nq, d = Q.shape
+    Nk = K.shape[2]
+    for name, t, shape in (("Q", Q, (B, H, Nq, d)), ("O", O, (B, H, Nq, d)), ("dO", dO, (B, H, Nq, d)),
+                           ("dQ", dQ, (B, H, Nq, d)), ("K", K, (B, H, Nk, d)), ("V", V, (B, H, Nk, d)),
+                           ("dK", dK, (B, H, Nk, d)), ("dV", dV, (B, H, Nk, d))):
+        _bf16_cuda(name, t, shape)
+    for name, t in (("lse", lse), ("delta", delta)):
+        if t.dtype != torch.float32 or tuple(t.shape) != (B, H, Nq) or not t.is_cuda or not t.is_contiguous():
+            raise ValueError(name + " must be a contiguous CUDA float32 tensor [B,H,Nq]")
+    if k_valid_len is not None and (k_valid_len.dtype != torch.int32 or tuple(k_valid_len.shape) != (B,)
+                                    or not k_valid_len.is_cuda):
+        raise ValueError("k_valid_len must be a CUDA int32 tensor [B]")
+    p = flat_attn_bwd_params_t()
+    p.Q, p.K, p.V, p.O, p.dO = Q.data_ptr(), K.data_ptr(), V.data_ptr(), O.data_ptr(), dO.data_ptr()
+    p.lse, p.dQ, p.dK, p.dV, p.delta = lse.data_ptr(), dQ.data_ptr(), dK.data_ptr(), dV.data_ptr(), delta.data_ptr()
+    p.B, p.H, p.Nq, p.Nk, p.d = B, H, Nq, Nk, d
+    p.scale = float(scale)
+    p.k_valid_len = None if k_valid_len is None else k_valid_len.data_ptr()
+    p.status = None if status is None else status.data_ptr()
+    p.causal = 1 if causal else 0
+    return p
+
+
+def flat_attn_bwd_ex(Q, K, V, O, dO, lse, dQ, dK, dV, delta, scale, k_valid_len=None, status=None, causal=False,
+                     stream=None):
+    """Backward pass: writes dQ [B,H,Nq,d], dK, dV [B,H,Nk,d] (bf16 CUDA tensors) from Q, K, V, the
+    forward's O and lse [B,H,Nq] (float32), and dO; `delta` [B,H,Nq] float32 is scratch."""
+    p = _bwd_params(Q, K, V, O, dO, lse, dQ, dK, dV, delta, scale, k_valid_len, status, causal)
+    _check(_lib.flat_attn_bwd_ex(ctypes.byref(p), _stream_ptr(stream)))
+    return dQ, dK, dV
+
+
+def flat_attn_bwd(Q, K, V, O, dO, lse, dQ, dK, dV, delta, scale, stream=None):
+    """flat_attn_bwd_ex without masks and without a status word."""
+    p = _bwd_params(Q, K, V, O, dO, lse, dQ, dK, dV, delta, scale, None, None, False)
+    _check(_lib.flat_attn_bwd(p.Q, p.K, p.V, p.O, p.dO, p.lse, p.dQ, p.dK, p.dV, p.delta, p.B, p.H, p.Nq, p.Nk, p.d,
+                              p.scale, _stream_ptr(stream)))
+    return dQ, dK, dV
 
 
 def flat_attn_naive_fwd(Q, K, V, O, L, A, scale, stream=None):

@@ -1,0 +1,375 @@
+// Backward pass of the fused Logit-softmax-Attend on the sm_100a tensor cores (tcgen05 + TMEM + TMA):
+// bf16 in, fp32 accumulate, bf16 gradients out.
+//
+// The paper stops at inference; this is the chain rule on its Section 2 steps 2-4, computed with the
+// same idea as its Section 5 dataflow: the [Nq, Nk] intermediates (weights P, their gradient dP and the
+// logit gradient dS) are rebuilt tile by tile on chip and never reach device memory.  With S = scale Q K^T,
+// lse the row-wise log-sum-exp that the forward pass saved, P = exp(S - lse) and delta_i = sum_t dO[i,t] O[i,t]:
+//     dV = P^T dO        dP = dO V^T        dS = P o (dP - delta)        dQ = scale dS K        dK = scale dS^T Q
+// Two launches of one kernel template, no atomics and no workspace beyond delta [B,H,Nq]:
+//   MODE_DQ : one CTA per 128 query rows, streaming key tiles:   S = Q K^T, dP = dO V^T, dQ += dS K.
+//             Also computes delta for its rows and writes it for the second launch.
+//   MODE_DKV: one CTA per 128 keys, streaming query tiles:       S^T = K Q^T, dP^T = V dO^T,
+//             dV += P^T dO, dK += dS^T Q.
+// Both are the same program: a stationary pair of tiles (X1, X2) whose rows are the TMEM lanes, a streamed
+// pair (Y1, Y2) whose rows are the columns:  T1 = X1 Y1^T,  T2 = X2 Y2^T  (both operands K-major in shared
+// memory), then element-wise p = 2^(c T1 - lse2), ds = p (T2 - delta) with lse2 / delta taken per lane
+// (MODE_DQ) or per column (MODE_DKV), P and dS rounded to bf16 and written over T1 / T2, and
+// acc_a += dS Y1, acc_b += P Y2 with the bf16 tile as the TMEM A-operand and Y as an MN-major B-operand.
+//
+// CTA = 320 threads: warps 0-7 element-wise (warp w: TMEM lane quarter w % 4, column half w / 4),
+// warp 8 TMA producer, warp 9 MMA issuer.  TMEM: T1 | T2 | acc_a | acc_b (128 + 128 + D + D columns).
+// Every wait is bounded (tc_common.cuh); on expiry the CTA aborts cleanly and reports a code.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "flat_internal.cuh"
+#include "ptx_sm100.cuh"
+#include "tc_common.cuh"
+
+namespace flat {
+
+using namespace ptx;
+using namespace tc;
+
+namespace {
+
+constexpr int BT = 128;              // rows of every tile (queries or keys)
+constexpr int STAGES = 2;            // ring of streamed tile pairs
+constexpr int EW_WARPS = 8;
+constexpr int BWD_THREADS = 32 * EW_WARPS + 64;
+constexpr int MODE_DQ = 0, MODE_DKV = 1;
+constexpr float LOG2E = 1.4426950408889634f;
+
+template <int D> struct BL {
+    static constexpr int TILE_BYTES = BT * D * 2;
+    static constexpr int OPERAND_BYTES = (2 + 2 * STAGES) * TILE_BYTES;      // X1, X2, STAGES x (Y1, Y2)
+    static constexpr int VEC_BYTES = 2 * 2 * BT * 4;                         // [buffer][lse2 | delta][column]
+    static constexpr int XCH_BYTES = 2 * BT * 4;                             // delta halves of MODE_DQ
+    static constexpr int SMEM_BYTES = OPERAND_BYTES + VEC_BYTES + XCH_BYTES + 256 + 1024;
+    static constexpr uint32_t T1_COL = 0, T2_COL = 128, ACC_A_COL = 256, ACC_B_COL = 256 + D;
+    static constexpr uint32_t TMEM_COLS = 512;
+};
+
+enum { BAR_X_FULL = 0, BAR_Y_FULL = 1, BAR_Y_EMPTY = 1 + STAGES, BAR_T_FULL = 1 + 2 * STAGES, BAR_PD_FULL,
+       BAR_ACC_DONE, NUM_BARS };
+
+__device__ __forceinline__ void ew_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+
+// X1, X2 / Y1, Y2 by mode:  MODE_DQ: (Q, dO) / (K, V);  MODE_DKV: (K, V) / (Q, dO).
+template <int D, int MODE>
+__global__ void __launch_bounds__(BWD_THREADS, 1)
+bwd_tc_kernel(const __grid_constant__ CUtensorMap tmX1, const __grid_constant__ CUtensorMap tmX2,
+              const __grid_constant__ CUtensorMap tmY1, const __grid_constant__ CUtensorMap tmY2,
+              const __nv_bfloat16* __restrict__ dOg, const __nv_bfloat16* __restrict__ Og,
+              const float* __restrict__ lse, float* __restrict__ delta,
+              __nv_bfloat16* __restrict__ outA, __nv_bfloat16* __restrict__ outB,
+              int H, int Nq, int Nk, float scale, const int32_t* __restrict__ valid_len, int coff, int32_t* status) {
+    using LY = BL<D>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t* X1s = base;
+    uint8_t* X2s = X1s + LY::TILE_BYTES;
+    uint8_t* Ys = X2s + LY::TILE_BYTES;                  // stage s: Y1 at 2 s, Y2 at 2 s + 1 (tiles)
+    float* vec = reinterpret_cast<float*>(base + LY::OPERAND_BYTES);
+    float* xch = vec + 2 * 2 * BT;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(xch + 2 * BT);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + NUM_BARS);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int bh = blockIdx.y;
+    const int x0 = blockIdx.x * BT;                      // first row of the stationary tile (query or key)
+    const int NX = MODE == MODE_DQ ? Nq : Nk;            // rows of the stationary / streamed tensors
+    const int NY = MODE == MODE_DQ ? Nk : Nq;
+    int nkeys = Nk;                                      // keys of this batch that take part at all
+    if (valid_len) { nkeys = valid_len[bh / H]; nkeys = nkeys < 0 ? 0 : (nkeys > Nk ? Nk : nkeys); }
+    // Range of streamed tiles [y_begin, y_end) that hold at least one visible (query, key) pair.
+    // Causal mask (coff = Nk - Nq; 2^30 = none): query i sees key j iff j <= i + coff.
+    int y_begin = 0, y_end;
+    if (MODE == MODE_DQ) {
+        const long long lim = static_cast<long long>(x0) + BT + coff;          // keys below this for the tile's last row
+        const int n = lim < nkeys ? (lim < 0 ? 0 : static_cast<int>(lim)) : nkeys;
+        y_end = (n + BT - 1) / BT;
+    } else {
+        y_end = x0 < nkeys ? (Nq + BT - 1) / BT : 0;
+        const long long first = static_cast<long long>(x0) - coff;             // first query that sees key x0
+        if (first > 0) y_begin = static_cast<int>(first / BT < y_end ? first / BT : y_end);
+    }
+    const int nsteps = y_end - y_begin;
+
+    if (threadIdx.x == EW_WARPS * 32) {
+        for (int i = 0; i < NUM_BARS; ++i) mbar_init(&bars[i], i == BAR_PD_FULL ? EW_WARPS : 1);
+        *abort_flag = 0;
+        fence_mbar_init();
+    }
+    if (warp == 0) { tmem_alloc(tmem_slot, LY::TMEM_COLS); tmem_relinquish(); }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    if (warp == EW_WARPS) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0 && nsteps > 0) {
+            prefetch_tensormap(&tmX1); prefetch_tensormap(&tmX2); prefetch_tensormap(&tmY1); prefetch_tensormap(&tmY2);
+            mbar_arrive_expect_tx(&bars[BAR_X_FULL], 2 * LY::TILE_BYTES);
+#pragma unroll
+            for (int c = 0; c < D / 64; ++c) {
+                tma_load_3d(X1s + c * BT * 128, &tmX1, &bars[BAR_X_FULL], c * 64, x0, bh);
+                tma_load_3d(X2s + c * BT * 128, &tmX2, &bars[BAR_X_FULL], c * 64, x0, bh);
+            }
+            int issued = 0;
+            bool ok = true;
+            for (int j = 0; j < nsteps && ok; ++j) {
+                const int s = j % STAGES;
+                ok = bounded_wait(&bars[BAR_Y_EMPTY + s], ((j / STAGES) & 1) ^ 1, abort_flag, status, 0x500 + s);
+                if (!ok) break;
+                mbar_arrive_expect_tx(&bars[BAR_Y_FULL + s], 2 * LY::TILE_BYTES);
+#pragma unroll
+                for (int c = 0; c < D / 64; ++c) {
+                    tma_load_3d(Ys + (2 * s) * LY::TILE_BYTES + c * BT * 128, &tmY1, &bars[BAR_Y_FULL + s], c * 64,
+                                (y_begin + j) * BT, bh);
+                    tma_load_3d(Ys + (2 * s + 1) * LY::TILE_BYTES + c * BT * 128, &tmY2, &bars[BAR_Y_FULL + s], c * 64,
+                                (y_begin + j) * BT, bh);
+                }
+                issued = j + 1;
+            }
+            if (!ok) {
+                drain_wait(&bars[BAR_X_FULL], 0);
+                for (int j = issued > STAGES ? issued - STAGES : 0; j < issued; ++j)
+                    drain_wait(&bars[BAR_Y_FULL + j % STAGES], (j / STAGES) & 1);
+            }
+        }
+    } else if (warp == EW_WARPS + 1) {
+        // ------------------------------------------------------------ MMA issuer
+        // Per step: T1 = X1 Y1^T and T2 = X2 Y2^T; once the element-wise warps have put P over T1 and dS
+        // over T2: acc_a += dS Y1 (and acc_b += P Y2).  The MMAs of one thread execute in issue order, so
+        // the next step's T1 / T2 (which overwrite P / dS) need no wait of their own.
+        if (lane == 0 && nsteps > 0) {
+            constexpr uint32_t IDESC_T = make_idesc_bf16(BT, BT, 0, 0);
+            constexpr uint32_t IDESC_ACC = make_idesc_bf16(BT, D, 0, 1);
+            bool ok = bounded_wait(&bars[BAR_X_FULL], 0, abort_flag, status, 0x510);
+            const uint32_t x1 = smem_u32(X1s), x2 = smem_u32(X2s);
+            for (int j = 0; j < nsteps && ok; ++j) {
+                const int s = j % STAGES;
+                ok = bounded_wait(&bars[BAR_Y_FULL + s], (j / STAGES) & 1, abort_flag, status, 0x520 + s);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t y1 = smem_u32(Ys + (2 * s) * LY::TILE_BYTES), y2 = y1 + LY::TILE_BYTES;
+#pragma unroll
+                for (int k = 0; k < D / 16; ++k) {
+                    const uint32_t off = (k / 4) * (BT * 128) + (k % 4) * 32;
+                    mma_ss(tmem + LY::T1_COL, make_smem_desc_sw128(x1 + off, 16, 1024),
+                           make_smem_desc_sw128(y1 + off, 16, 1024), IDESC_T, k > 0);
+                }
+#pragma unroll
+                for (int k = 0; k < D / 16; ++k) {
+                    const uint32_t off = (k / 4) * (BT * 128) + (k % 4) * 32;
+                    mma_ss(tmem + LY::T2_COL, make_smem_desc_sw128(x2 + off, 16, 1024),
+                           make_smem_desc_sw128(y2 + off, 16, 1024), IDESC_T, k > 0);
+                }
+                tc_commit(&bars[BAR_T_FULL]);
+                ok = bounded_wait(&bars[BAR_PD_FULL], j & 1, abort_flag, status, 0x530);
+                if (!ok) break;
+                tc_fence_after();
+                // the bf16 tiles: slice k (16 contraction indices) of column half k / 4 sits at columns
+                // 64 (k / 4) + 8 (k % 4) of its T buffer (each half over the columns it was computed from)
+#pragma unroll
+                for (int k = 0; k < BT / 16; ++k)
+                    mma_ts(tmem + LY::ACC_A_COL, tmem + LY::T2_COL + (k / 4) * 64 + (k % 4) * 8,
+                           make_smem_desc_sw128(y1 + k * 2048, BT * 128, 1024), IDESC_ACC, (j > 0 || k > 0));
+                if (MODE == MODE_DKV) {
+#pragma unroll
+                    for (int k = 0; k < BT / 16; ++k)
+                        mma_ts(tmem + LY::ACC_B_COL, tmem + LY::T1_COL + (k / 4) * 64 + (k % 4) * 8,
+                               make_smem_desc_sw128(y2 + k * 2048, BT * 128, 1024), IDESC_ACC, (j > 0 || k > 0));
+                }
+                tc_commit(&bars[BAR_Y_EMPTY + s]);
+                if (j == nsteps - 1) tc_commit(&bars[BAR_ACC_DONE]);
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ element-wise + epilogue (warps 0-7)
+        const int q = warp & 3, h = warp >> 2;
+        const int r = q * 32 + lane;                     // lane of the TMEM = row of the stationary tile
+        const int xr = x0 + r;                           // that row's index (query in MODE_DQ, key in MODE_DKV)
+        const uint32_t tl = tmem + (static_cast<uint32_t>(q * 32) << 16);
+        const float c2 = scale * LOG2E;
+        bool ok = true;
+        // Per-lane terms (MODE_DQ): lse of the row in base-2 units (+inf switches a row off: no key, or
+        // past the end) and delta = sum_t dO O, each column half summing its half of the features.
+        float lse2_r = INFINITY, delta_r = 0.f;
+        if (MODE == MODE_DQ) {
+            float part = 0.f;
+            if (xr < Nq) {
+                const uint4* a = reinterpret_cast<const uint4*>(dOg + (static_cast<int64_t>(bh) * Nq + xr) * D + h * (D / 2));
+                const uint4* b = reinterpret_cast<const uint4*>(Og + (static_cast<int64_t>(bh) * Nq + xr) * D + h * (D / 2));
+#pragma unroll
+                for (int v = 0; v < D / 16; ++v) {
+                    const uint4 av = a[v], bv = b[v];
+                    const uint32_t aw[4] = {av.x, av.y, av.z, av.w}, bw[4] = {bv.x, bv.y, bv.z, bv.w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        part = fmaf(__uint_as_float(aw[e] << 16), __uint_as_float(bw[e] << 16), part);
+                        part = fmaf(__uint_as_float(aw[e] & 0xffff0000u), __uint_as_float(bw[e] & 0xffff0000u), part);
+                    }
+                }
+                const float l = lse[static_cast<int64_t>(bh) * Nq + xr];
+                lse2_r = l == -INFINITY ? INFINITY : l * LOG2E;
+            }
+            xch[h * BT + r] = part;
+            ew_sync();
+            delta_r = xch[r] + xch[BT + r];
+            if (h == 0 && xr < Nq) delta[static_cast<int64_t>(bh) * Nq + xr] = delta_r;
+        }
+        // Per-column terms (MODE_DKV): lse2 and delta of the streamed tile's queries, two buffers in
+        // shared memory; thread t < 128 fetches lse of column t, thread 128 + t its delta, one step ahead.
+        const int vt = threadIdx.x & (BT - 1);
+        const bool v_is_delta = threadIdx.x >= BT;
+        auto fetch_vec = [&](int step) -> float {
+            const int i = (y_begin + step) * BT + vt;
+            if (step >= nsteps || i >= Nq) return v_is_delta ? 0.f : INFINITY;
+            if (v_is_delta) return delta[static_cast<int64_t>(bh) * Nq + i];
+            const float l = lse[static_cast<int64_t>(bh) * Nq + i];
+            return l == -INFINITY ? INFINITY : l * LOG2E;
+        };
+        if (MODE == MODE_DKV && nsteps > 0) {
+            vec[(v_is_delta ? BT : 0) + vt] = fetch_vec(0);
+            ew_sync();
+        }
+        // keys the row takes part with (MODE_DQ: per query row; MODE_DKV: the row IS a key)
+        const long long rlim = static_cast<long long>(xr) + 1 + coff;
+        const int nrow = rlim < nkeys ? (rlim < 0 ? 0 : static_cast<int>(rlim)) : nkeys;
+        const bool key_live = xr < nkeys;
+        for (int j = 0; j < nsteps; ++j) {
+            float v_next = 0.f;
+            if (MODE == MODE_DKV) v_next = fetch_vec(j + 1);
+            // (a warp whose wait failed keeps walking the loop without working, so that all eight warps
+            // pass the same sequence of named barriers; the issuer's wait for its arrival then runs out)
+            if (ok) ok = __all_sync(0xffffffffu, bounded_wait(&bars[BAR_T_FULL], j & 1, abort_flag, status, 0x540));
+            if (ok) {
+            tc_fence_after();
+            const int y0 = (y_begin + j) * BT + h * 64;  // index of this half's first column (key or query)
+            const float* lv = vec + (j & 1) * 2 * BT + h * 64;
+#pragma unroll
+            for (int c = 0; c < 2; ++c) {
+                uint32_t t1[32], t2[32], pk[16], dk[16];
+                tmem_ld_x32(tl + LY::T1_COL + h * 64 + c * 32, t1);
+                tmem_ld_x32(tl + LY::T2_COL + h * 64 + c * 32, t2);
+                tc_wait_ld();
+#pragma unroll
+                for (int i = 0; i < 32; i += 2) {
+                    float p[2], ds[2];
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        const int col = y0 + c * 32 + i + e;
+                        float lse2, dl;
+                        bool live;
+                        if (MODE == MODE_DQ) { lse2 = lse2_r; dl = delta_r; live = col < nrow; }
+                        else {
+                            lse2 = lv[c * 32 + i + e]; dl = lv[BT + c * 32 + i + e];
+                            live = key_live && static_cast<long long>(col) + coff >= xr;      // query col sees key xr
+                        }
+                        const float pe = live ? ex2_approx(fmaf(__uint_as_float(t1[i + e]), c2, -lse2)) : 0.f;
+                        p[e] = pe;
+                        ds[e] = pe * (__uint_as_float(t2[i + e]) - dl);
+                    }
+                    pk[i / 2] = pack_bf16x2(p[0], p[1]);
+                    dk[i / 2] = pack_bf16x2(ds[0], ds[1]);
+                }
+                if (MODE == MODE_DKV) tmem_st_x16(tl + LY::T1_COL + h * 64 + c * 16, pk);
+                tmem_st_x16(tl + LY::T2_COL + h * 64 + c * 16, dk);
+            }
+            tc_wait_st();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&bars[BAR_PD_FULL]);
+            }
+            if (MODE == MODE_DKV) {
+                vec[((j + 1) & 1) * 2 * BT + (v_is_delta ? BT : 0) + vt] = v_next;
+                ew_sync();
+            }
+        }
+        if (ok && nsteps > 0) ok = __all_sync(0xffffffffu, bounded_wait(&bars[BAR_ACC_DONE], 0, abort_flag, status, 0x550));
+        if (ok) {
+            tc_fence_after();
+            // this thread's half of the features of its row: acc_a -> outA (dQ, or dK), acc_b -> outB (dV)
+#pragma unroll
+            for (int o = 0; o < (MODE == MODE_DKV ? 2 : 1); ++o) {
+                __nv_bfloat16* out = o == 0 ? outA : outB;
+                const float f = o == 0 ? scale : 1.f;
+                const uint32_t col = (o == 0 ? LY::ACC_A_COL : LY::ACC_B_COL) + h * (D / 2);
+                __nv_bfloat16* orow = out + (static_cast<int64_t>(bh) * NX + xr) * D + h * (D / 2);
+#pragma unroll
+                for (int c = 0; c < D / 64; ++c) {
+                    uint32_t a[32];
+                    if (nsteps > 0) {
+                        tmem_ld_x32(tl + col + c * 32, a);
+                        tc_wait_ld();
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) a[i] = 0u;  // nothing sees this tile: zero gradient
+                    }
+                    if (xr < NX) {
+#pragma unroll
+                        for (int v = 0; v < 4; ++v) {
+                            uint4 w;
+                            w.x = pack_bf16x2(__uint_as_float(a[8 * v + 0]) * f, __uint_as_float(a[8 * v + 1]) * f);
+                            w.y = pack_bf16x2(__uint_as_float(a[8 * v + 2]) * f, __uint_as_float(a[8 * v + 3]) * f);
+                            w.z = pack_bf16x2(__uint_as_float(a[8 * v + 4]) * f, __uint_as_float(a[8 * v + 5]) * f);
+                            w.w = pack_bf16x2(__uint_as_float(a[8 * v + 6]) * f, __uint_as_float(a[8 * v + 7]) * f);
+                            *reinterpret_cast<uint4*>(orow + c * 32 + v * 8) = w;
+                        }
+                    }
+                }
+            }
+        }
+        (void)NY;
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem, LY::TMEM_COLS);
+}
+
+template <int D>
+int launch_bwd_d(const BwdProblem& p, cudaStream_t st) {
+    using LY = BL<D>;
+    CUtensorMap tmQ, tmK, tmV, tmdO;
+    const int BH = p.B * p.H;
+    if (!make_map(&tmQ, p.Q, BH, p.Nq, D, BT) || !make_map(&tmK, p.K, BH, p.Nk, D, BT) ||
+        !make_map(&tmV, p.V, BH, p.Nk, D, BT) || !make_map(&tmdO, p.dO, BH, p.Nq, D, BT))
+        return FLAT_ERR_CUDA;
+    if (!ensure_dynamic_smem<bwd_tc_kernel<D, MODE_DQ>>(LY::SMEM_BYTES)) return FLAT_ERR_CUDA;
+    if (!ensure_dynamic_smem<bwd_tc_kernel<D, MODE_DKV>>(LY::SMEM_BYTES)) return FLAT_ERR_CUDA;
+    const int coff = p.causal ? p.Nk - p.Nq : (1 << 30);
+    const __nv_bfloat16* dO = static_cast<const __nv_bfloat16*>(p.dO);
+    const __nv_bfloat16* O = static_cast<const __nv_bfloat16*>(p.O);
+    {
+        dim3 grid((p.Nq + BT - 1) / BT, BH);
+        bwd_tc_kernel<D, MODE_DQ><<<grid, BWD_THREADS, LY::SMEM_BYTES, st>>>(
+            tmQ, tmdO, tmK, tmV, dO, O, p.lse, p.delta, static_cast<__nv_bfloat16*>(p.dQ), nullptr, p.H, p.Nq, p.Nk,
+            p.scale, p.k_valid_len, coff, p.status);
+        if (cudaGetLastError() != cudaSuccess) return FLAT_ERR_CUDA;
+    }
+    {
+        dim3 grid((p.Nk + BT - 1) / BT, BH);
+        bwd_tc_kernel<D, MODE_DKV><<<grid, BWD_THREADS, LY::SMEM_BYTES, st>>>(
+            tmK, tmV, tmQ, tmdO, dO, O, p.lse, p.delta, static_cast<__nv_bfloat16*>(p.dK),
+            static_cast<__nv_bfloat16*>(p.dV), p.H, p.Nq, p.Nk, p.scale, p.k_valid_len, coff, p.status);
+        if (cudaGetLastError() != cudaSuccess) return FLAT_ERR_CUDA;
+    }
+    return FLAT_OK;
+}
+
+}  // namespace
+
+int launch_bwd_tc(const BwdProblem& p, cudaStream_t st) {
+    if (p.d == 64) return launch_bwd_d<64>(p, st);
+    if (p.d == 128) return launch_bwd_d<128>(p, st);
+    return FLAT_ERR_UNSUPPORTED;
+}
+
+}  // namespace flat

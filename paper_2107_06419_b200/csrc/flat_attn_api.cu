@@ -59,8 +59,9 @@ int validate(const flat_attn_params_t* p, flat::Problem* out) {
     if (p->k_valid_len && (reinterpret_cast<uintptr_t>(p->k_valid_len) & 3u)) return FLAT_ERR_ALIGN;
     if (p->status && (reinterpret_cast<uintptr_t>(p->status) & 3u)) return FLAT_ERR_ALIGN;
     if (p->causal != 0 && p->causal != 1) return FLAT_ERR_UNSUPPORTED;
+    if (p->lse && (reinterpret_cast<uintptr_t>(p->lse) & 3u)) return FLAT_ERR_ALIGN;
     *out = flat::Problem{p->Q, p->K, p->V, p->O, p->B, p->H, p->Nq, p->Nk, p->d,
-                         p->scale, p->dtype, p->k_valid_len, status_or_library_word(p->status), p->causal};
+                         p->scale, p->dtype, p->k_valid_len, status_or_library_word(p->status), p->causal, p->lse};
     return FLAT_OK;
 }
 
@@ -107,11 +108,12 @@ int run_fused(const flat::Problem& q, int variant, cudaStream_t st) {
             // 0.037 against 0.096 ms); only tiny problems (256 keys or fewer, less than one CTA per SM)
             // are at par or a few per cent better on the 128-row CTAs.
             else           v = (ctas2 >= sms || q.Nk > 256) ? FLAT_VARIANT_TC2 : FLAT_VARIANT_TC;
-            // (the single-tile predecessor kernel has no causal mask)
-            if (q.causal && v == FLAT_VARIANT_TC) v = FLAT_VARIANT_TC2;
+            // (the single-tile predecessor kernel has no causal mask and does not write lse)
+            if ((q.causal || q.lse) && v == FLAT_VARIANT_TC) v = FLAT_VARIANT_TC2;
         }
     }
     if (q.causal && v == FLAT_VARIANT_TC) return FLAT_ERR_UNSUPPORTED;
+    if (q.lse && (v == FLAT_VARIANT_TC || v == FLAT_VARIANT_RGRAN)) return FLAT_ERR_UNSUPPORTED;
     g_last_variant = v;
     if (v == FLAT_VARIANT_TC2_SINGLE) {
         if (!tc_applies(q) || q.d != 64) return FLAT_ERR_UNSUPPORTED;
@@ -170,7 +172,7 @@ int flat_attn_fwd_ex(const flat_attn_params_t* p, void* stream) {
 
 int flat_attn_fwd(const void* Q, const void* K, const void* V, void* O, int B, int H, int Nq, int Nk, int d,
                   float scale, void* stream) {
-    flat_attn_params_t p{Q, K, V, O, B, H, Nq, Nk, d, scale, FLAT_DTYPE_BF16, nullptr, nullptr, FLAT_VARIANT_AUTO, 0};
+    flat_attn_params_t p{Q, K, V, O, B, H, Nq, Nk, d, scale, FLAT_DTYPE_BF16, nullptr, nullptr, FLAT_VARIANT_AUTO, 0, nullptr};
     return flat_attn_fwd_ex(&p, stream);
 }
 
@@ -189,8 +191,35 @@ int flat_attn_naive_fwd_ex(const flat_attn_params_t* p, void* L, void* A, void* 
 
 int flat_attn_naive_fwd(const void* Q, const void* K, const void* V, void* O, void* L, void* A, int B, int H,
                         int Nq, int Nk, int d, float scale, void* stream) {
-    flat_attn_params_t p{Q, K, V, O, B, H, Nq, Nk, d, scale, FLAT_DTYPE_BF16, nullptr, nullptr, FLAT_VARIANT_AUTO, 0};
+    flat_attn_params_t p{Q, K, V, O, B, H, Nq, Nk, d, scale, FLAT_DTYPE_BF16, nullptr, nullptr, FLAT_VARIANT_AUTO, 0, nullptr};
     return flat_attn_naive_fwd_ex(&p, L, A, stream);
+}
+
+int flat_attn_bwd_ex(const flat_attn_bwd_params_t* p, void* stream) {
+    if (!p) return FLAT_ERR_NULL;
+    if (!p->Q || !p->K || !p->V || !p->O || !p->dO || !p->lse || !p->dQ || !p->dK || !p->dV || !p->delta)
+        return FLAT_ERR_NULL;
+    // sizes, scale, masks and the alignment of Q, K, V, O: the forward's rules
+    flat_attn_params_t f{p->Q, p->K, p->V, const_cast<void*>(p->O), p->B, p->H, p->Nq, p->Nk, p->d, p->scale,
+                         FLAT_DTYPE_BF16, p->k_valid_len, p->status, FLAT_VARIANT_AUTO, p->causal, nullptr};
+    flat::Problem q;
+    const int rc = validate(&f, &q);
+    if (rc != FLAT_OK) return rc;
+    if (p->d != 64 && p->d != 128) return FLAT_ERR_UNSUPPORTED;
+    if (!aligned16(p->dO) || !aligned16(p->dQ) || !aligned16(p->dK) || !aligned16(p->dV)) return FLAT_ERR_ALIGN;
+    if ((reinterpret_cast<uintptr_t>(p->lse) & 3u) || (reinterpret_cast<uintptr_t>(p->delta) & 3u)) return FLAT_ERR_ALIGN;
+    const flat::BwdProblem b{p->Q, p->K, p->V, p->O, p->dO, p->lse, p->dQ, p->dK, p->dV, p->delta, p->B, p->H, p->Nq,
+                             p->Nk, p->d, p->scale, p->k_valid_len, q.status, p->causal};
+    const int r = flat::launch_bwd_tc(b, static_cast<cudaStream_t>(stream));
+    if (r == FLAT_OK) g_last_launches = 2;
+    return r;
+}
+
+int flat_attn_bwd(const void* Q, const void* K, const void* V, const void* O, const void* dO, const float* lse,
+                  void* dQ, void* dK, void* dV, float* delta, int B, int H, int Nq, int Nk, int d, float scale,
+                  void* stream) {
+    flat_attn_bwd_params_t p{Q, K, V, O, dO, lse, dQ, dK, dV, delta, B, H, Nq, Nk, d, scale, nullptr, nullptr, 0};
+    return flat_attn_bwd_ex(&p, stream);
 }
 
 size_t flat_attn_host_workspace_bytes(int B, int H, int Nq, int Nk, int d, int dtype) {
@@ -265,6 +294,7 @@ int flat_attn_fwd_host(const flat_attn_params_t* p, void* workspace, size_t work
         sub.Q = dQ + qo; sub.K = dK + ko; sub.V = dV + ko; sub.O = dO + qo;
         if (p->B > 1) { sub.B = u1 - u0; if (sub.k_valid_len) sub.k_valid_len += u0; }
         else          { sub.H = u1 - u0; }
+        if (sub.lse) sub.lse += static_cast<size_t>(u0) * (p->B > 1 ? static_cast<size_t>(p->H) * p->Nq : static_cast<size_t>(p->Nq));
         const int r = run_fused(sub, p->variant, ss);
         if (r != FLAT_OK) return r;
         ++launches;
@@ -342,7 +372,7 @@ int flat_attn_layer_fwd(const void* X, const void* Wqkv, const void* Wo, void* Y
                         int B, int N, int H, int d, int Dm, float scale, int causal, int32_t* status, void* stream) {
     if (!X || !Wqkv || !Wo || !Y || !Q || !K || !V || !O) return FLAT_ERR_NULL;
     // validate all three steps before anything is launched
-    flat_attn_params_t p{Q, K, V, O, B, H, N, N, d, scale, FLAT_DTYPE_BF16, nullptr, status, FLAT_VARIANT_AUTO, causal};
+    flat_attn_params_t p{Q, K, V, O, B, H, N, N, d, scale, FLAT_DTYPE_BF16, nullptr, status, FLAT_VARIANT_AUTO, causal, nullptr};
     flat::Problem q;
     int rc = validate(&p, &q);
     if (rc != FLAT_OK) return rc;

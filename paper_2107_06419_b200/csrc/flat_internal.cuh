@@ -18,7 +18,22 @@ struct Problem {
     const int32_t* k_valid_len;
     int32_t* status;
     int causal;                      // 0 / 1: query i sees keys j <= i + (Nk - Nq)
+    float* lse;                      // optional [B,H,Nq] fp32 output of the fused kernels: log-sum-exp of each row's scaled logits
 };
+
+// A validated backward problem (device pointers; bf16 tensors, fp32 lse / delta).
+struct BwdProblem {
+    const void *Q, *K, *V, *O, *dO;
+    const float* lse;
+    void *dQ, *dK, *dV;
+    float* delta;
+    int B, H, Nq, Nk, d;
+    float scale;
+    const int32_t* k_valid_len;
+    int32_t* status;
+    int causal;
+};
+int launch_bwd_tc(const BwdProblem& p, cudaStream_t st);   // bf16, d in {64, 128}: two kernels (dQ; dK and dV)
 
 // Argument check of the public parameter block (what every fused / baseline entry point applies
 // before it launches anything): FLAT_OK or the error code.

@@ -169,7 +169,8 @@ __global__ void __launch_bounds__(128 * NT + 128, NT == 1 ? 2 : 1)
 fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                  const __grid_constant__ CUtensorMap tmV, __nv_bfloat16* __restrict__ O, int H, int Nq, int Nk,
                  float scale_log2e, const int32_t* __restrict__ valid_len, int coff, int32_t* status,
-                 const int32_t* __restrict__ cu_q = nullptr, const int32_t* __restrict__ cu_k = nullptr) {
+                 const int32_t* __restrict__ cu_q = nullptr, const int32_t* __restrict__ cu_k = nullptr,
+                 float* __restrict__ lse = nullptr) {
     using LY = L2<D, NT>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -451,6 +452,9 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         }
         if (ok) {
             const float inv = l > 0.f ? 1.f / l : 0.f;
+            // (dense batches only) log of the row's sum of exponentials; m_ref and the exponents are in base-2 units
+            if (!VL && lse && row < Nq)
+                lse[static_cast<int64_t>(bh) * Nq + row] = l > 0.f ? (m_ref + log2f(l)) * 0.6931471805599453f : -INFINITY;
             tc_fence_after();
             __nv_bfloat16* orow = VL ? O + ((static_cast<int64_t>(q_tok0) + (row - row0)) * H + head) * D
                                      : O + (static_cast<int64_t>(bh) * Nq + row) * D;
@@ -496,7 +500,7 @@ int launch_tc2_d(const Problem& p, cudaStream_t st) {
     dim3 grid((p.Nq + NT * BM - 1) / (NT * BM), BH);
     kern<<<grid, LY::THREADS, LY::SMEM_BYTES, st>>>(tmQ, tmK, tmV, static_cast<__nv_bfloat16*>(p.O), p.H, p.Nq,
                                                     p.Nk, p.scale * 1.4426950408889634f, p.k_valid_len,
-                                                    p.causal ? p.Nk - p.Nq : (1 << 30), p.status, nullptr, nullptr);
+                                                    p.causal ? p.Nk - p.Nq : (1 << 30), p.status, nullptr, nullptr, p.lse);
     return cudaGetLastError() == cudaSuccess ? FLAT_OK : FLAT_ERR_CUDA;
 }
 

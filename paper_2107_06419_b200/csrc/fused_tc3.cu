@@ -335,13 +335,16 @@ __device__ __forceinline__ void cursor_next(Cursor& c, const Sched& sc) {
 
 // VL: packed variable-length batches (see get_item); the tensor maps then view the packed tensors as
 // {d, H, tokens} and valid_len is unused (cu_k gives the key counts).
-template <bool VL>
+// WLSE: also writes lse[b,h,i] = log of row i's sum of exponentials (dense batches; what the
+// backward pass takes from the forward one).  A separate instantiation, so that the plain forward
+// kernel is compiled exactly as it is without the output.
+template <bool VL, bool WLSE = false>
 __global__ void __launch_bounds__(L3::THREADS, 1)
 fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                  const __grid_constant__ CUtensorMap tmV, __nv_bfloat16* __restrict__ O, int H, int Nq, int Nk,
                  int items, int slabs, float scale_log2e, const int32_t* __restrict__ valid_len, int coff,
                  int32_t* status, int wide_stores, int paired, const int32_t* __restrict__ cu_q,
-                 const int32_t* __restrict__ cu_k) {
+                 const int32_t* __restrict__ cu_k, float* __restrict__ lse) {
     using LY = L3;
     const Sched sc{items, slabs, H, Nk, valid_len, coff, paired, cu_q, cu_k};
     if (VL && static_cast<int>(gridDim.x) == items) {
@@ -700,6 +703,9 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         {
             const int row = it.row0 + t * BM + q * 32 + lane;
             const float inv = l > 0.f ? 1.f / l : 0.f;
+            // (m_ref, common to the row's two warps, and the exponents are in base-2 units)
+            if (WLSE && h == 0 && row < Nq)
+                lse[static_cast<int64_t>(it.bh) * Nq + row] = l > 0.f ? (m_ref + log2f(l)) * 0.6931471805599453f : -INFINITY;
             tc_fence_after();
             // (packed batches: token-major [tokens, H, d])
             __nv_bfloat16* orow = VL ? O + ((static_cast<int64_t>(it.q_tok0) + (row - it.row0)) * H + it.head) * D + h * (D / 2)
@@ -748,7 +754,9 @@ int launch_tc3(const Problem& p, cudaStream_t st) {
     if (!make_map(&tmQ, p.Q, BH, p.Nq, D, BM) || !make_map(&tmK, p.K, BH, p.Nk, D, BN) ||
         !make_map(&tmV, p.V, BH, p.Nk, D, BN))
         return FLAT_ERR_CUDA;
-    if (!ensure_dynamic_smem<fused_tc3_kernel<false>>(LY::SMEM_BYTES)) return FLAT_ERR_CUDA;
+    if (!(p.lse ? ensure_dynamic_smem<fused_tc3_kernel<false, true>>(LY::SMEM_BYTES)
+                : ensure_dynamic_smem<fused_tc3_kernel<false, false>>(LY::SMEM_BYTES)))
+        return FLAT_ERR_CUDA;
     // Work items = (head, 256-row slab), slabs of a head next to each other so that CTAs running at
     // the same time share K and V in L2.  With many items per SM the grid is one persistent CTA per
     // SM, each walking over its share (the fixed deal costs little then and the pipeline never
@@ -767,12 +775,12 @@ int launch_tc3(const Problem& p, cudaStream_t st) {
     const int64_t slots = paired ? static_cast<int64_t>((slabs + 1) & ~1) * BH : items;
     if (slots > 0x7fffffff) return FLAT_ERR_SHAPE;
     const int grid = static_cast<int>(persistent ? sms : items);
-    fused_tc3_kernel<false><<<grid, LY::THREADS, LY::SMEM_BYTES, st>>>(tmQ, tmK, tmV, static_cast<__nv_bfloat16*>(p.O), p.H,
-                                                                p.Nq, p.Nk, static_cast<int>(slots), slabs,
-                                                                p.scale * 1.4426950408889634f, p.k_valid_len,
-                                                                p.causal ? p.Nk - p.Nq : (1 << 30), p.status,
-                                                                (reinterpret_cast<uintptr_t>(p.O) & 31) == 0 ? 1 : 0, paired,
-                                                                nullptr, nullptr);
+    auto kern = p.lse ? fused_tc3_kernel<false, true> : fused_tc3_kernel<false, false>;
+    kern<<<grid, LY::THREADS, LY::SMEM_BYTES, st>>>(tmQ, tmK, tmV, static_cast<__nv_bfloat16*>(p.O), p.H, p.Nq, p.Nk,
+                                                    static_cast<int>(slots), slabs, p.scale * 1.4426950408889634f,
+                                                    p.k_valid_len, p.causal ? p.Nk - p.Nq : (1 << 30), p.status,
+                                                    (reinterpret_cast<uintptr_t>(p.O) & 31) == 0 ? 1 : 0, paired, nullptr,
+                                                    nullptr, p.lse);
     return cudaGetLastError() == cudaSuccess ? FLAT_OK : FLAT_ERR_CUDA;
 }
 
@@ -802,7 +810,7 @@ int launch_fused_tc3_varlen(const void* Q, const void* K, const void* V, void* O
     fused_tc3_kernel<true><<<grid, LY::THREADS, LY::SMEM_BYTES, st>>>(
         tmQ, tmK, tmV, static_cast<__nv_bfloat16*>(O), H, max_seqlen_q, 0, static_cast<int>(items), slabs,
         scale * 1.4426950408889634f, nullptr, causal ? 0 : (1 << 30), status,
-        (reinterpret_cast<uintptr_t>(O) & 31) == 0 ? 1 : 0, 0, cu_q, cu_k);
+        (reinterpret_cast<uintptr_t>(O) & 31) == 0 ? 1 : 0, 0, cu_q, cu_k, nullptr);
     return cudaGetLastError() == cudaSuccess ? FLAT_OK : FLAT_ERR_CUDA;
 }
 

@@ -128,7 +128,8 @@ template <typename T, int D>
 __global__ void __launch_bounds__(NTHREADS) fused_simt_kernel(const T* __restrict__ Q, const T* __restrict__ K,
                                                               const T* __restrict__ V, T* __restrict__ O, int H,
                                                               int Nq, int Nk, float scale_log2e,
-                                                              const int32_t* __restrict__ valid_len, int causal) {
+                                                              const int32_t* __restrict__ valid_len, int causal,
+                                                              float* __restrict__ lse) {
     extern __shared__ __align__(16) float smem[];
     float* Qs = smem;
     float* Ks = Qs + 64 * (D + 4);
@@ -203,6 +204,8 @@ __global__ void __launch_bounds__(NTHREADS) fused_simt_kernel(const T* __restric
         const float inv = l[a] > 0.f ? 1.f / l[a] : 0.f;   // no valid key: O = 0
 #pragma unroll
         for (int b = 0; b < D / 16; ++b) store_out(O + (bh * Nq + r) * D + tx + 16 * b, o[a][b] * inv);
+        // log of the row's sum of exponentials (m and the exponents are in base-2 units here)
+        if (lse && tx == 0) lse[bh * Nq + r] = l[a] > 0.f ? (m[a] + log2f(l[a])) * 0.6931471805599453f : -INFINITY;
     }
 }
 
@@ -319,7 +322,7 @@ static int launch_fused_simt_td(const Problem& p, cudaStream_t st) {
     dim3 grid((p.Nq + TM - 1) / TM, p.B * p.H);
     kern<<<grid, NTHREADS, smem, st>>>(static_cast<const T*>(p.Q), static_cast<const T*>(p.K),
                                        static_cast<const T*>(p.V), static_cast<T*>(p.O), p.H, p.Nq, p.Nk,
-                                       p.scale * 1.4426950408889634f, p.k_valid_len, p.causal);
+                                       p.scale * 1.4426950408889634f, p.k_valid_len, p.causal, p.lse);
     return cudaGetLastError() == cudaSuccess ? FLAT_OK : FLAT_ERR_CUDA;
 }
 
