@@ -17,8 +17,8 @@
 // (MODE_DQ) or per column (MODE_DKV), P and dS rounded to bf16 and written over T1 / T2, and
 // acc_a += dS Y1, acc_b += P Y2 with the bf16 tile as the TMEM A-operand and Y as an MN-major B-operand.
 //
-// CTA = 320 threads: warps 0-7 element-wise (warp w: TMEM lane quarter w % 4, column half w / 4),
-// warp 8 TMA producer, warp 9 MMA issuer.  TMEM: T1 | T2 | acc_a | acc_b (128 + 128 + D + D columns).
+// CTA = 320 threads: warps 0-7 element-wise (warp w: TMEM lane quarter w % 4, 32 of the 64 columns of
+// every half step: w / 4), warp 8 TMA producer, warp 9 MMA issuer.  TMEM: T1 | T2 | acc_a | acc_b (128 + 128 + D + D columns).
 // Every wait is bounded (tc_common.cuh); on expiry the CTA aborts cleanly and reports a code.
 #include <cuda.h>
 #include <cuda_bf16.h>
@@ -37,6 +37,7 @@ using namespace tc;
 namespace {
 
 constexpr int BT = 128;              // rows of every tile (queries or keys)
+constexpr int HC = 64;               // columns (rows of the streamed tile) per half step
 constexpr int STAGES = 2;            // ring of streamed tile pairs
 constexpr int EW_WARPS = 8;
 constexpr int BWD_THREADS = 32 * EW_WARPS + 64;
@@ -53,8 +54,9 @@ template <int D> struct BL {
     static constexpr uint32_t TMEM_COLS = 512;
 };
 
-enum { BAR_X_FULL = 0, BAR_Y_FULL = 1, BAR_Y_EMPTY = 1 + STAGES, BAR_T_FULL = 1 + 2 * STAGES, BAR_PD_FULL,
-       BAR_ACC_DONE, NUM_BARS };
+// T_FULL / PD_FULL [half]: the half's T1, T2 are computed / its dS (and P) are written, once per step
+enum { BAR_X_FULL = 0, BAR_Y_FULL = 1, BAR_Y_EMPTY = 1 + STAGES, BAR_T_FULL = 1 + 2 * STAGES,
+       BAR_PD_FULL = BAR_T_FULL + 2, BAR_ACC_DONE = BAR_PD_FULL + 2, NUM_BARS };
 
 __device__ __forceinline__ void ew_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 
@@ -101,7 +103,7 @@ bwd_tc_kernel(const __grid_constant__ CUtensorMap tmX1, const __grid_constant__ 
     const int nsteps = y_end - y_begin;
 
     if (threadIdx.x == EW_WARPS * 32) {
-        for (int i = 0; i < NUM_BARS; ++i) mbar_init(&bars[i], i == BAR_PD_FULL ? EW_WARPS : 1);
+        for (int i = 0; i < NUM_BARS; ++i) mbar_init(&bars[i], (i >= BAR_PD_FULL && i < BAR_ACC_DONE) ? EW_WARPS : 1);
         *abort_flag = 0;
         fence_mbar_init();
     }
@@ -145,50 +147,90 @@ bwd_tc_kernel(const __grid_constant__ CUtensorMap tmX1, const __grid_constant__ 
         }
     } else if (warp == EW_WARPS + 1) {
         // ------------------------------------------------------------ MMA issuer
-        // Per step: T1 = X1 Y1^T and T2 = X2 Y2^T; once the element-wise warps have put P over T1 and dS
-        // over T2: acc_a += dS Y1 (and acc_b += P Y2).  The MMAs of one thread execute in issue order, so
-        // the next step's T1 / T2 (which overwrite P / dS) need no wait of their own.
-        if (lane == 0 && nsteps > 0) {
-            constexpr uint32_t IDESC_T = make_idesc_bf16(BT, BT, 0, 0);
+        // The streamed tile is worked on in two halves of 64 columns (a: rows 0-63 of Y, b: rows 64-127), so
+        // that the MMAs of one half run while the element-wise warps are busy with the other:
+        //   T(j, half):   T1 = X1 Y1[half]^T and T2 = X2 Y2[half]^T into the half's 64 columns of T1 / T2;
+        //   ACC(j, half): once the element-wise warps have put dS over T2 (and P over T1):
+        //                 acc_a += dS Y1[half] (and acc_b += P Y2[half]).
+        // Issue order: T(0,a) T(0,b) | ACC(j,a) T(j+1,a) ACC(j,b) T(j+1,b) | ...  The MMAs of one thread
+        // execute in issue order, so T(j+1, half), which overwrites the half's P / dS, needs no wait of its
+        // own behind ACC(j, half).
+        // The whole warp walks the loop (uniform control flow) and one elected lane issues: the MMA and
+        // commit instructions take their operands from uniform registers, which the compiler can only
+        // use when it knows that a single thread runs the code.
+        if (nsteps > 0) {
+            constexpr uint32_t IDESC_T = make_idesc_bf16(BT, HC, 0, 0);
             constexpr uint32_t IDESC_ACC = make_idesc_bf16(BT, D, 0, 1);
-            bool ok = bounded_wait(&bars[BAR_X_FULL], 0, abort_flag, status, 0x510);
-            const uint32_t x1 = smem_u32(X1s), x2 = smem_u32(X2s);
-            for (int j = 0; j < nsteps && ok; ++j) {
-                const int s = j % STAGES;
-                ok = bounded_wait(&bars[BAR_Y_FULL + s], (j / STAGES) & 1, abort_flag, status, 0x520 + s);
-                if (!ok) break;
-                tc_fence_after();
-                const uint32_t y1 = smem_u32(Ys + (2 * s) * LY::TILE_BYTES), y2 = y1 + LY::TILE_BYTES;
+            auto wait = [&](int bar, uint32_t parity, int code) {
+                return __all_sync(0xffffffffu, bounded_wait(&bars[bar], parity, abort_flag, status, code));
+            };
+            bool ok = wait(BAR_X_FULL, 0, 0x510);
+            // descriptors of the first feature slice of each operand (the others are constant offsets away)
+            const uint64_t x1d = make_smem_desc_sw128(smem_u32(X1s), 16, 1024);            // K-major
+            const uint64_t x2d = make_smem_desc_sw128(smem_u32(X2s), 16, 1024);
+            const uint64_t ykd = make_smem_desc_sw128(smem_u32(Ys), 16, 1024);             // Y1 of stage 0, K-major
+            const uint64_t ymd = make_smem_desc_sw128(smem_u32(Ys), BT * 128, 1024);       // Y1 of stage 0, MN-major
+            constexpr uint64_t TILE16 = LY::TILE_BYTES >> 4;                                // descriptor units of 16 bytes
+            auto issue_t = [&](int j, int half) {
+                // (K-major operands: rows 64.. of a tile start 64 * 128 bytes into each 64-feature panel)
+                const uint64_t y1 = ykd + static_cast<uint64_t>(2 * (j % STAGES)) * TILE16 + static_cast<uint64_t>((half * HC * 128) >> 4);
+                const uint64_t y2 = y1 + TILE16;
 #pragma unroll
                 for (int k = 0; k < D / 16; ++k) {
-                    const uint32_t off = (k / 4) * (BT * 128) + (k % 4) * 32;
-                    mma_ss(tmem + LY::T1_COL, make_smem_desc_sw128(x1 + off, 16, 1024),
-                           make_smem_desc_sw128(y1 + off, 16, 1024), IDESC_T, k > 0);
+                    const uint64_t off = static_cast<uint64_t>(((k / 4) * (BT * 128) + (k % 4) * 32) >> 4);
+                    mma_ss(tmem + LY::T1_COL + half * HC, x1d + off, y1 + off, IDESC_T, k > 0);
                 }
 #pragma unroll
                 for (int k = 0; k < D / 16; ++k) {
-                    const uint32_t off = (k / 4) * (BT * 128) + (k % 4) * 32;
-                    mma_ss(tmem + LY::T2_COL, make_smem_desc_sw128(x2 + off, 16, 1024),
-                           make_smem_desc_sw128(y2 + off, 16, 1024), IDESC_T, k > 0);
+                    const uint64_t off = static_cast<uint64_t>(((k / 4) * (BT * 128) + (k % 4) * 32) >> 4);
+                    mma_ss(tmem + LY::T2_COL + half * HC, x2d + off, y2 + off, IDESC_T, k > 0);
                 }
-                tc_commit(&bars[BAR_T_FULL]);
-                ok = bounded_wait(&bars[BAR_PD_FULL], j & 1, abort_flag, status, 0x530);
-                if (!ok) break;
-                tc_fence_after();
-                // the bf16 tiles: slice k (16 contraction indices) of column half k / 4 sits at columns
-                // 64 (k / 4) + 8 (k % 4) of its T buffer (each half over the columns it was computed from)
+                tc_commit(&bars[BAR_T_FULL + half]);
+            };
+            auto issue_acc = [&](int j, int half) {
+                // the bf16 tiles of a half: slice k (16 contraction indices) was written by the warps of
+                // column quarter k / 2 at columns 32 (k / 2) + 8 (k % 2) of the half (over what they had read)
+                const uint64_t y1 = ymd + static_cast<uint64_t>(2 * (j % STAGES)) * TILE16 + static_cast<uint64_t>((half * 4 * 2048) >> 4);
+                const uint64_t y2 = y1 + TILE16;
+                const uint32_t acc = (j > 0 || half > 0) ? 1u : 0u;
 #pragma unroll
-                for (int k = 0; k < BT / 16; ++k)
-                    mma_ts(tmem + LY::ACC_A_COL, tmem + LY::T2_COL + (k / 4) * 64 + (k % 4) * 8,
-                           make_smem_desc_sw128(y1 + k * 2048, BT * 128, 1024), IDESC_ACC, (j > 0 || k > 0));
+                for (int k = 0; k < HC / 16; ++k)
+                    mma_ts(tmem + LY::ACC_A_COL, tmem + LY::T2_COL + half * HC + (k / 2) * 32 + (k % 2) * 8,
+                           y1 + static_cast<uint64_t>((k * 2048) >> 4), IDESC_ACC, k > 0 ? 1u : acc);
                 if (MODE == MODE_DKV) {
 #pragma unroll
-                    for (int k = 0; k < BT / 16; ++k)
-                        mma_ts(tmem + LY::ACC_B_COL, tmem + LY::T1_COL + (k / 4) * 64 + (k % 4) * 8,
-                               make_smem_desc_sw128(y2 + k * 2048, BT * 128, 1024), IDESC_ACC, (j > 0 || k > 0));
+                    for (int k = 0; k < HC / 16; ++k)
+                        mma_ts(tmem + LY::ACC_B_COL, tmem + LY::T1_COL + half * HC + (k / 2) * 32 + (k % 2) * 8,
+                               y2 + static_cast<uint64_t>((k * 2048) >> 4), IDESC_ACC, k > 0 ? 1u : acc);
                 }
-                tc_commit(&bars[BAR_Y_EMPTY + s]);
-                if (j == nsteps - 1) tc_commit(&bars[BAR_ACC_DONE]);
+            };
+            if (ok) ok = wait(BAR_Y_FULL, 0, 0x520);
+            if (ok) {
+                tc_fence_after();
+                if (elect_one()) { issue_t(0, 0); issue_t(0, 1); }
+                __syncwarp();
+            }
+            for (int j = 0; j < nsteps && ok; ++j) {
+                const bool more = j + 1 < nsteps;
+                ok = wait(BAR_PD_FULL + 0, j & 1, 0x530);
+                if (ok && more) ok = wait(BAR_Y_FULL + (j + 1) % STAGES, ((j + 1) / STAGES) & 1, 0x521);
+                if (!ok) break;
+                tc_fence_after();
+                if (elect_one()) {
+                    issue_acc(j, 0);
+                    if (more) issue_t(j + 1, 0);
+                }
+                __syncwarp();
+                ok = wait(BAR_PD_FULL + 1, j & 1, 0x531);
+                if (!ok) break;
+                tc_fence_after();
+                if (elect_one()) {
+                    issue_acc(j, 1);
+                    tc_commit(&bars[BAR_Y_EMPTY + j % STAGES]);
+                    if (more) issue_t(j + 1, 1);
+                    else tc_commit(&bars[BAR_ACC_DONE]);
+                }
+                __syncwarp();
             }
         }
     } else {
@@ -247,46 +289,73 @@ bwd_tc_kernel(const __grid_constant__ CUtensorMap tmX1, const __grid_constant__ 
         for (int j = 0; j < nsteps; ++j) {
             float v_next = 0.f;
             if (MODE == MODE_DKV) v_next = fetch_vec(j + 1);
-            // (a warp whose wait failed keeps walking the loop without working, so that all eight warps
-            // pass the same sequence of named barriers; the issuer's wait for its arrival then runs out)
-            if (ok) ok = __all_sync(0xffffffffu, bounded_wait(&bars[BAR_T_FULL], j & 1, abort_flag, status, 0x540));
-            if (ok) {
-            tc_fence_after();
-            const int y0 = (y_begin + j) * BT + h * 64;  // index of this half's first column (key or query)
-            const float* lv = vec + (j & 1) * 2 * BT + h * 64;
-#pragma unroll
-            for (int c = 0; c < 2; ++c) {
+#pragma unroll 1
+            for (int half = 0; half < 2; ++half) {
+                // (a warp whose wait failed keeps walking the loops without working, so that all eight warps
+                // pass the same sequence of named barriers; the issuer's wait for its arrival then runs out)
+                if (ok) ok = __all_sync(0xffffffffu, bounded_wait(&bars[BAR_T_FULL + half], j & 1, abort_flag, status, 0x540 + half));
+                if (!ok) continue;
+                tc_fence_after();
+                const int cq = half * HC + h * 32;       // this warp's 32 columns of the step
+                const int y0 = (y_begin + j) * BT + cq;  // index of the first of them (key or query)
+                // all 32 x 32 (row, column) pairs of this warp visible?  (then no per-element selection)
+                const bool fast = __all_sync(0xffffffffu, MODE == MODE_DQ ? y0 + 32 <= nrow
+                                                                          : key_live && static_cast<long long>(y0) + coff >= xr);
                 uint32_t t1[32], t2[32], pk[16], dk[16];
-                tmem_ld_x32(tl + LY::T1_COL + h * 64 + c * 32, t1);
-                tmem_ld_x32(tl + LY::T2_COL + h * 64 + c * 32, t2);
+                tmem_ld_x32(tl + LY::T1_COL + cq, t1);
+                tmem_ld_x32(tl + LY::T2_COL + cq, t2);
+                const float4* lv4 = reinterpret_cast<const float4*>(vec + (j & 1) * 2 * BT + cq);
+                const uint64_t c22 = pack2(c2, c2);
                 tc_wait_ld();
+                // p = 2^(c T1 - lse2), ds = p (T2 - delta), on packed pairs (two results per issue slot)
+                if (fast) {
 #pragma unroll
-                for (int i = 0; i < 32; i += 2) {
-                    float p[2], ds[2];
-#pragma unroll
-                    for (int e = 0; e < 2; ++e) {
-                        const int col = y0 + c * 32 + i + e;
-                        float lse2, dl;
-                        bool live;
-                        if (MODE == MODE_DQ) { lse2 = lse2_r; dl = delta_r; live = col < nrow; }
-                        else {
-                            lse2 = lv[c * 32 + i + e]; dl = lv[BT + c * 32 + i + e];
-                            live = key_live && static_cast<long long>(col) + coff >= xr;      // query col sees key xr
+                    for (int i = 0; i < 32; i += 4) {
+                        uint64_t nl[2], dl[2];           // -lse2 and delta of columns i..i+1, i+2..i+3
+                        if (MODE == MODE_DQ) {
+                            nl[0] = nl[1] = pack2(-lse2_r, -lse2_r);
+                            dl[0] = dl[1] = pack2(delta_r, delta_r);
+                        } else {
+                            const float4 a4 = lv4[i / 4], b4 = lv4[(BT + i) / 4];
+                            nl[0] = pack2(-a4.x, -a4.y); nl[1] = pack2(-a4.z, -a4.w);
+                            dl[0] = pack2(b4.x, b4.y); dl[1] = pack2(b4.z, b4.w);
                         }
-                        const float pe = live ? ex2_approx(fmaf(__uint_as_float(t1[i + e]), c2, -lse2)) : 0.f;
-                        p[e] = pe;
-                        ds[e] = pe * (__uint_as_float(t2[i + e]) - dl);
+#pragma unroll
+                        for (int e = 0; e < 2; ++e) {
+                            const int x = i + 2 * e;
+                            float a0, a1;
+                            unpack2(fma2(pack2(__uint_as_float(t1[x]), __uint_as_float(t1[x + 1])), c22, nl[e]), a0, a1);
+                            const float p0 = ex2_approx(a0), p1 = ex2_approx(a1);
+                            const uint64_t pp = pack2(p0, p1);
+                            float d0, d1;
+                            unpack2(mul2(pp, sub2(pack2(__uint_as_float(t2[x]), __uint_as_float(t2[x + 1])), dl[e])), d0, d1);
+                            if (MODE == MODE_DKV) pk[x / 2] = pack_bf16x2(p0, p1);
+                            dk[x / 2] = pack_bf16x2(d0, d1);
+                        }
                     }
-                    pk[i / 2] = pack_bf16x2(p[0], p[1]);
-                    dk[i / 2] = pack_bf16x2(ds[0], ds[1]);
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 32; i += 2) {
+                        float p[2], ds[2];
+#pragma unroll
+                        for (int e = 0; e < 2; ++e) {
+                            const int col = y0 + i + e;
+                            const float lse2 = MODE == MODE_DQ ? lse2_r : vec[(j & 1) * 2 * BT + cq + i + e];
+                            const float dl = MODE == MODE_DQ ? delta_r : vec[(j & 1) * 2 * BT + BT + cq + i + e];
+                            const bool live = MODE == MODE_DQ ? col < nrow : key_live && static_cast<long long>(col) + coff >= xr;
+                            p[e] = live ? ex2_approx(fmaf(__uint_as_float(t1[i + e]), c2, -lse2)) : 0.f;
+                            ds[e] = p[e] * (__uint_as_float(t2[i + e]) - dl);
+                        }
+                        pk[i / 2] = pack_bf16x2(p[0], p[1]);
+                        dk[i / 2] = pack_bf16x2(ds[0], ds[1]);
+                    }
                 }
-                if (MODE == MODE_DKV) tmem_st_x16(tl + LY::T1_COL + h * 64 + c * 16, pk);
-                tmem_st_x16(tl + LY::T2_COL + h * 64 + c * 16, dk);
-            }
-            tc_wait_st();
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&bars[BAR_PD_FULL]);
+                if (MODE == MODE_DKV) tmem_st_x16(tl + LY::T1_COL + cq, pk);
+                tmem_st_x16(tl + LY::T2_COL + cq, dk);
+                tc_wait_st();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&bars[BAR_PD_FULL + half]);
             }
             if (MODE == MODE_DKV) {
                 vec[((j + 1) & 1) * 2 * BT + (v_is_delta ? BT : 0) + vt] = v_next;

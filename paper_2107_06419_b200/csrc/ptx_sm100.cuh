@@ -188,6 +188,16 @@ __device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
     asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
     return d;
 }
+__device__ __forceinline__ uint64_t sub2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
 // One 32-byte store (sixteen bf16) per lane: a warp whose lanes hold different rows then touches
 // every 32-byte sector once, where 16-byte stores touch each twice.  `p` must be 32-byte aligned.
 __device__ __forceinline__ void st_global_32B(void* p, const uint32_t (&w)[8]) {
