@@ -55,13 +55,16 @@ constexpr float LOG2E = 1.4426950408889634f;
 
 template <int D, int MODE> struct BL {
     static constexpr int TILE_BYTES = BT * D * 2;
-    // ring of streamed tile pairs: deep enough that a copy (about two microseconds from device memory) is
-    // under way for every step the element-wise warps and the MMAs are working on
-    static constexpr int STAGES = D == 64 ? 4 : 2;
-    static constexpr int OPERAND_BYTES = (2 + 2 * STAGES) * TILE_BYTES;      // X1, X2, STAGES x (Y1, Y2)
-    static constexpr int VEC_BYTES = STAGES * 2 * BT * 4;                    // [stage][lse2 | delta][column]
+    // Ring of streamed HALF tile pairs (64 rows of Y1 and of Y2 per stage, one stage per half step): deep
+    // enough that a copy (about two microseconds from device memory) is under way for every half step the
+    // element-wise warps and the MMAs are working on, and released half by half.
+    static constexpr int HTILE_BYTES = HC * D * 2;
+    static constexpr int HSTAGES = D == 64 ? 8 : 4;
+    static constexpr int VSTAGES = HSTAGES / 2;                              // ring of per-column vectors (whole steps)
+    static constexpr int OPERAND_BYTES = 2 * TILE_BYTES + 2 * HSTAGES * HTILE_BYTES;   // X1, X2, HSTAGES x (Y1, Y2 halves)
+    static constexpr int VEC_BYTES = VSTAGES * 2 * BT * 4;                   // [stage][lse2 | delta][column]
     static constexpr int XCH_BYTES = 4 * BT * 4;                             // delta quarters of MODE_DQ
-    static constexpr int SMEM_BYTES = OPERAND_BYTES + VEC_BYTES + XCH_BYTES + 256 + 1024;
+    static constexpr int SMEM_BYTES = OPERAND_BYTES + VEC_BYTES + XCH_BYTES + 512 + 1024;
     static constexpr uint32_t T1_COL = 0, T2_COL = 128, ACC_A_COL = 256, ACC_B_COL = 256 + D;
     static constexpr uint32_t ACC_END = 256 + (MODE == MODE_DKV ? 2 : 1) * D;
     static constexpr bool SEP = ACC_END + 128 <= 512;                        // room for the bf16 tiles beside T1 / T2
@@ -76,9 +79,9 @@ template <int D, int MODE> struct BL {
     // barriers.  T_FULL / PD_FULL / ACC_HALF [half]: the half's T1, T2 are computed / its dS (and P) are
     // written / the MMAs that read them have completed -- once per step each; VEC_FULL [stage]: the step's
     // lse2 / delta vectors are in shared memory (MODE_DKV)
-    static constexpr int BAR_X_FULL = 0, BAR_Y_FULL = 1, BAR_Y_EMPTY = 1 + STAGES, BAR_T_FULL = 1 + 2 * STAGES,
+    static constexpr int BAR_X_FULL = 0, BAR_Y_FULL = 1, BAR_Y_EMPTY = 1 + HSTAGES, BAR_T_FULL = 1 + 2 * HSTAGES,
                          BAR_PD_FULL = BAR_T_FULL + 2, BAR_ACC_HALF = BAR_PD_FULL + 2, BAR_VEC_FULL = BAR_ACC_HALF + 2,
-                         BAR_ACC_DONE = BAR_VEC_FULL + STAGES, NUM_BARS = BAR_ACC_DONE + 1;
+                         BAR_ACC_DONE = BAR_VEC_FULL + VSTAGES, NUM_BARS = BAR_ACC_DONE + 1;
 };
 
 __device__ __forceinline__ void ew_sync() { asm volatile("bar.sync 1, 512;" ::: "memory"); }
@@ -97,9 +100,9 @@ bwd_tc_kernel(const __grid_constant__ CUtensorMap tmX1, const __grid_constant__ 
     uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* X1s = base;
     uint8_t* X2s = X1s + LY::TILE_BYTES;
-    uint8_t* Ys = X2s + LY::TILE_BYTES;                  // stage s: Y1 at 2 s, Y2 at 2 s + 1 (tiles)
+    uint8_t* Ys = X2s + LY::TILE_BYTES;                  // half stage s: Y1 rows at 2 s, Y2 rows at 2 s + 1 (half tiles)
     float* vec = reinterpret_cast<float*>(base + LY::OPERAND_BYTES);
-    float* xch = vec + LY::STAGES * 2 * BT;
+    float* xch = vec + LY::VSTAGES * 2 * BT;
     uint64_t* bars = reinterpret_cast<uint64_t*>(xch + 4 * BT);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + LY::NUM_BARS);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
@@ -155,22 +158,25 @@ bwd_tc_kernel(const __grid_constant__ CUtensorMap tmX1, const __grid_constant__ 
             }
             int issued = 0;
             bool ok = true;
-            for (int j = 0; j < nsteps && ok; ++j) {
-                const int s = j % LY::STAGES;
-                ok = wait_warp(LY::BAR_Y_EMPTY + s, ((j / LY::STAGES) & 1) ^ 1, 0x500 + s);
+            for (int g = 0; g < 2 * nsteps && ok; ++g) {     // half steps: g = 2 j + half
+                const int s = g % LY::HSTAGES, j = g >> 1, half = g & 1;
+                ok = wait_warp(LY::BAR_Y_EMPTY + s, ((g / LY::HSTAGES) & 1) ^ 1, 0x500 + s);
                 if (!ok) break;
                 if (lane == 0) {
-                    mbar_arrive_expect_tx(&bars[LY::BAR_Y_FULL + s], 2 * LY::TILE_BYTES);
+                    mbar_arrive_expect_tx(&bars[LY::BAR_Y_FULL + s], 2 * LY::HTILE_BYTES);
 #pragma unroll
                     for (int c = 0; c < D / 64; ++c) {
-                        tma_load_3d(Ys + (2 * s) * LY::TILE_BYTES + c * BT * 128, &tmY1, &bars[LY::BAR_Y_FULL + s], c * 64,
-                                    (y_begin + j) * BT, bh);
-                        tma_load_3d(Ys + (2 * s + 1) * LY::TILE_BYTES + c * BT * 128, &tmY2, &bars[LY::BAR_Y_FULL + s], c * 64,
-                                    (y_begin + j) * BT, bh);
+                        tma_load_3d(Ys + (2 * s) * LY::HTILE_BYTES + c * HC * 128, &tmY1, &bars[LY::BAR_Y_FULL + s], c * 64,
+                                    (y_begin + j) * BT + half * HC, bh);
+                        tma_load_3d(Ys + (2 * s + 1) * LY::HTILE_BYTES + c * HC * 128, &tmY2, &bars[LY::BAR_Y_FULL + s], c * 64,
+                                    (y_begin + j) * BT + half * HC, bh);
                     }
                 }
-                issued = j + 1;
-                if (MODE == MODE_DKV) {
+                issued = g + 1;
+                if (MODE == MODE_DKV && half == 1) {
+                    // The step's vectors go into ring slot j % VSTAGES, last read in step j - VSTAGES.  The
+                    // stage just granted (the SECOND half's) was released behind the second half of that
+                    // step, i.e. after all of its element-wise work.
                     float l2[4], dl[4];
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
@@ -182,19 +188,17 @@ bwd_tc_kernel(const __grid_constant__ CUtensorMap tmX1, const __grid_constant__ 
                             dl[e] = delta[static_cast<int64_t>(bh) * Nq + i];
                         }
                     }
-                    // (the vectors share the ring's stage: it was last read in step j - STAGES, whose element-wise
-                    // work was over before the stage that this iteration has just been granted was released)
-                    float* vb = vec + s * 2 * BT + lane * 4;
+                    float* vb = vec + (j % LY::VSTAGES) * 2 * BT + lane * 4;
                     *reinterpret_cast<float4*>(vb) = make_float4(l2[0], l2[1], l2[2], l2[3]);
                     *reinterpret_cast<float4*>(vb + BT) = make_float4(dl[0], dl[1], dl[2], dl[3]);
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(&bars[LY::BAR_VEC_FULL + s]);
+                    if (lane == 0) mbar_arrive(&bars[LY::BAR_VEC_FULL + j % LY::VSTAGES]);
                 }
             }
             if (!ok && lane == 0) {
                 drain_wait(&bars[LY::BAR_X_FULL], 0);
-                for (int j = issued > LY::STAGES ? issued - LY::STAGES : 0; j < issued; ++j)
-                    drain_wait(&bars[LY::BAR_Y_FULL + j % LY::STAGES], (j / LY::STAGES) & 1);
+                for (int g = issued > LY::HSTAGES ? issued - LY::HSTAGES : 0; g < issued; ++g)
+                    drain_wait(&bars[LY::BAR_Y_FULL + g % LY::HSTAGES], (g / LY::HSTAGES) & 1);
             }
         }
     } else if (warp == EW_WARPS + 1) {
@@ -215,26 +219,28 @@ bwd_tc_kernel(const __grid_constant__ CUtensorMap tmX1, const __grid_constant__ 
             // descriptors of the first feature slice of each operand (the others are constant offsets away)
             const uint64_t x1d = make_smem_desc_sw128(smem_u32(X1s), 16, 1024);            // K-major
             const uint64_t x2d = make_smem_desc_sw128(smem_u32(X2s), 16, 1024);
-            const uint64_t ykd = make_smem_desc_sw128(smem_u32(Ys), 16, 1024);             // Y1 of stage 0, K-major
-            const uint64_t ymd = make_smem_desc_sw128(smem_u32(Ys), BT * 128, 1024);       // Y1 of stage 0, MN-major
-            constexpr uint64_t TILE16 = LY::TILE_BYTES >> 4;                                // descriptor units of 16 bytes
+            const uint64_t ykd = make_smem_desc_sw128(smem_u32(Ys), 16, 1024);             // Y1 half of stage 0, K-major
+            const uint64_t ymd = make_smem_desc_sw128(smem_u32(Ys), HC * 128, 1024);       // Y1 half of stage 0, MN-major
+            constexpr uint64_t HTILE16 = LY::HTILE_BYTES >> 4;                              // descriptor units of 16 bytes
             // Consecutive MMAs into ONE accumulator wait for each other, so the slices of independent
             // products are issued in turn: T1 and T2 of a half, and the accumulations acc_a and acc_b.
             auto issue_t = [&](int j, int half) {
-                // (K-major operands: rows 64.. of a tile start 64 * 128 bytes into each 64-feature panel)
-                const uint64_t y1 = ykd + static_cast<uint64_t>(2 * (j % LY::STAGES)) * TILE16 + static_cast<uint64_t>((half * HC * 128) >> 4);
-                const uint64_t y2 = y1 + TILE16;
+                // (feature slice k of a K-major operand: panel k / 4 of 64 features, 32 bytes per slice; a panel
+                // is 128 rows of 128 bytes for the stationary tiles, 64 rows for the streamed half tiles)
+                const uint64_t y1 = ykd + static_cast<uint64_t>(2 * ((2 * j + half) % LY::HSTAGES)) * HTILE16;
+                const uint64_t y2 = y1 + HTILE16;
 #pragma unroll
                 for (int k = 0; k < D / 16; ++k) {
-                    const uint64_t off = static_cast<uint64_t>(((k / 4) * (BT * 128) + (k % 4) * 32) >> 4);
-                    mma_ss(tmem + LY::T1_COL + half * HC, x1d + off, y1 + off, IDESC_T, k > 0);
-                    mma_ss(tmem + LY::T2_COL + half * HC, x2d + off, y2 + off, IDESC_T, k > 0);
+                    const uint64_t xoff = static_cast<uint64_t>(((k / 4) * (BT * 128) + (k % 4) * 32) >> 4);
+                    const uint64_t yoff = static_cast<uint64_t>(((k / 4) * (HC * 128) + (k % 4) * 32) >> 4);
+                    mma_ss(tmem + LY::T1_COL + half * HC, x1d + xoff, y1 + yoff, IDESC_T, k > 0);
+                    mma_ss(tmem + LY::T2_COL + half * HC, x2d + xoff, y2 + yoff, IDESC_T, k > 0);
                 }
                 tc_commit(&bars[LY::BAR_T_FULL + half]);
             };
             auto issue_acc = [&](int j, int half) {
-                const uint64_t y1 = ymd + static_cast<uint64_t>(2 * (j % LY::STAGES)) * TILE16 + static_cast<uint64_t>((half * 4 * 2048) >> 4);
-                const uint64_t y2 = y1 + TILE16;
+                const uint64_t y1 = ymd + static_cast<uint64_t>(2 * ((2 * j + half) % LY::HSTAGES)) * HTILE16;
+                const uint64_t y2 = y1 + HTILE16;
                 const uint32_t acc = (j > 0 || half > 0) ? 1u : 0u;
 #pragma unroll
                 for (int k = 0; k < HC / 16; ++k) {
@@ -246,7 +252,10 @@ bwd_tc_kernel(const __grid_constant__ CUtensorMap tmX1, const __grid_constant__ 
                 }
                 if (LY::SEP) tc_commit(&bars[LY::BAR_ACC_HALF + half]);
             };
-            if (ok) ok = wait_warp(LY::BAR_Y_FULL, 0, 0x520);
+            auto y_full = [&](int g, int code) {         // the copy of half step g has landed
+                return wait_warp(LY::BAR_Y_FULL + g % LY::HSTAGES, (g / LY::HSTAGES) & 1, code);
+            };
+            if (ok) ok = y_full(0, 0x520) && y_full(1, 0x520);
             if (ok) {
                 tc_fence_after();
                 if (elect_one()) { issue_t(0, 0); issue_t(0, 1); }
@@ -257,17 +266,15 @@ bwd_tc_kernel(const __grid_constant__ CUtensorMap tmX1, const __grid_constant__ 
 #pragma unroll
                 for (int half = 0; half < 2; ++half) {
                     ok = wait_warp(LY::BAR_PD_FULL + half, j & 1, 0x530 + half);
-                    if (ok && more && half == 0) ok = wait_warp(LY::BAR_Y_FULL + (j + 1) % LY::STAGES, ((j + 1) / LY::STAGES) & 1, 0x521);
+                    if (ok && more) ok = y_full(2 * (j + 1) + half, 0x521);
                     if (!ok) break;
                     tc_fence_after();
                     if (elect_one()) {
                         if (LY::SEP && more) issue_t(j + 1, half);
                         issue_acc(j, half);
                         if (!LY::SEP && more) issue_t(j + 1, half);
-                        if (half == 1) {
-                            tc_commit(&bars[LY::BAR_Y_EMPTY + j % LY::STAGES]);
-                            if (!more) tc_commit(&bars[LY::BAR_ACC_DONE]);
-                        }
+                        tc_commit(&bars[LY::BAR_Y_EMPTY + (2 * j + half) % LY::HSTAGES]);
+                        if (half == 1 && !more) tc_commit(&bars[LY::BAR_ACC_DONE]);
                     }
                     __syncwarp();
                 }
@@ -316,7 +323,7 @@ bwd_tc_kernel(const __grid_constant__ CUtensorMap tmX1, const __grid_constant__ 
         const uint32_t ds_addr = tl + (half == 0 ? LY::ds_store(0, 0) : LY::ds_store(1, 0)) + h * (LY::ds_store(0, 1) - LY::ds_store(0, 0));
         const uint32_t p_addr = tl + (half == 0 ? LY::p_store(0, 0) : LY::p_store(1, 0)) + h * (LY::p_store(0, 1) - LY::p_store(0, 0));
         for (int j = 0; j < nsteps && ok; ++j) {
-            if (MODE == MODE_DKV) ok = wait_warp(LY::BAR_VEC_FULL + j % LY::STAGES, static_cast<uint32_t>(j / LY::STAGES) & 1u, 0x548);
+            if (MODE == MODE_DKV) ok = wait_warp(LY::BAR_VEC_FULL + j % LY::VSTAGES, static_cast<uint32_t>(j / LY::VSTAGES) & 1u, 0x548);
             if (ok) ok = wait_warp(LY::BAR_T_FULL + half, j & 1, 0x540 + half);
             if (!ok) break;
             tc_fence_after();
@@ -324,7 +331,7 @@ bwd_tc_kernel(const __grid_constant__ CUtensorMap tmX1, const __grid_constant__ 
             // all 32 x 32 (row, column) pairs of this warp visible?  (then no per-element selection)
             const bool fast = __all_sync(0xffffffffu, MODE == MODE_DQ ? y0 + 32 <= nrow
                                                                       : key_live && static_cast<long long>(y0) + coff >= xr);
-            const float* lv = vec + (j % LY::STAGES) * 2 * BT + cq;
+            const float* lv = vec + (j % LY::VSTAGES) * 2 * BT + cq;
             uint32_t pk[16], dk[16];
             // two loads of 16 columns each from T1 and T2 (few registers live at a time)
 #pragma unroll
@@ -431,10 +438,13 @@ bwd_tc_kernel(const __grid_constant__ CUtensorMap tmX1, const __grid_constant__ 
 
 template <int D>
 int launch_bwd_d(const BwdProblem& p, cudaStream_t st) {
-    CUtensorMap tmQ, tmK, tmV, tmdO;
+    // every tensor is stationary (boxes of 128 rows) in one launch and streamed (boxes of 64 rows) in the other
+    CUtensorMap tmQ, tmK, tmV, tmdO, tmQh, tmKh, tmVh, tmdOh;
     const int BH = p.B * p.H;
     if (!make_map(&tmQ, p.Q, BH, p.Nq, D, BT) || !make_map(&tmK, p.K, BH, p.Nk, D, BT) ||
-        !make_map(&tmV, p.V, BH, p.Nk, D, BT) || !make_map(&tmdO, p.dO, BH, p.Nq, D, BT))
+        !make_map(&tmV, p.V, BH, p.Nk, D, BT) || !make_map(&tmdO, p.dO, BH, p.Nq, D, BT) ||
+        !make_map(&tmQh, p.Q, BH, p.Nq, D, HC) || !make_map(&tmKh, p.K, BH, p.Nk, D, HC) ||
+        !make_map(&tmVh, p.V, BH, p.Nk, D, HC) || !make_map(&tmdOh, p.dO, BH, p.Nq, D, HC))
         return FLAT_ERR_CUDA;
     if (!ensure_dynamic_smem<bwd_tc_kernel<D, MODE_DQ>>(BL<D, MODE_DQ>::SMEM_BYTES)) return FLAT_ERR_CUDA;
     if (!ensure_dynamic_smem<bwd_tc_kernel<D, MODE_DKV>>(BL<D, MODE_DKV>::SMEM_BYTES)) return FLAT_ERR_CUDA;
@@ -444,14 +454,14 @@ int launch_bwd_d(const BwdProblem& p, cudaStream_t st) {
     {
         dim3 grid((p.Nq + BT - 1) / BT, BH);
         bwd_tc_kernel<D, MODE_DQ><<<grid, BWD_THREADS, BL<D, MODE_DQ>::SMEM_BYTES, st>>>(
-            tmQ, tmdO, tmK, tmV, dO, O, p.lse, p.delta, static_cast<__nv_bfloat16*>(p.dQ), nullptr, p.H, p.Nq, p.Nk,
+            tmQ, tmdO, tmKh, tmVh, dO, O, p.lse, p.delta, static_cast<__nv_bfloat16*>(p.dQ), nullptr, p.H, p.Nq, p.Nk,
             p.scale, p.k_valid_len, coff, p.status);
         if (cudaGetLastError() != cudaSuccess) return FLAT_ERR_CUDA;
     }
     {
         dim3 grid((p.Nk + BT - 1) / BT, BH);
         bwd_tc_kernel<D, MODE_DKV><<<grid, BWD_THREADS, BL<D, MODE_DKV>::SMEM_BYTES, st>>>(
-            tmK, tmV, tmQ, tmdO, dO, O, p.lse, p.delta, static_cast<__nv_bfloat16*>(p.dK),
+            tmK, tmV, tmQh, tmdOh, dO, O, p.lse, p.delta, static_cast<__nv_bfloat16*>(p.dK),
             static_cast<__nv_bfloat16*>(p.dV), p.H, p.Nq, p.Nk, p.scale, p.k_valid_len, coff, p.status);
         if (cudaGetLastError() != cudaSuccess) return FLAT_ERR_CUDA;
     }
