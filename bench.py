@@ -399,6 +399,7 @@ def main():
         if not args.headline_only and world == 1:
             del ws, Oh
             out["naive"] = run_naive(bench, torch, api, w, d) if w.name == DEFAULT_WORKLOAD else None
+            out["backward"] = run_backward(bench, torch, api, w, d, data, seed, args, peaks)
             host = d = data = None
             torch.cuda.empty_cache()
             out["workloads"] = [run_other(bench, torch, api, inputs.WORKLOADS[n], seed, args, peaks, dev)
@@ -423,6 +424,52 @@ def run_naive(bench, torch, api, w, d):
             "bytes_model": 12 * elems + w.qkvo_bytes(),
             "hbm_gbs_on_model": (12 * elems + w.qkvo_bytes()) / (n_ms * 1e-3) / 1e9,
             "max_abs_diff_vs_fused": float((O2.float() - d["O"].float()).abs().max())}
+
+
+def run_backward(bench, torch, api, w, d, data, seed, args, peaks):
+    """The backward pass (dQ, dK, dV from dO, recomputing the weights from the forward's lse) on the same
+    workload: 10 B H Nq Nk d FLOP per call (five contractions), two kernels per step."""
+    from paper_2107_06419_b200 import inputs
+    if w.d not in (64, 128):
+        return None
+    time.sleep(1.0)
+    dev = bench.dev
+    n = w.B * w.H * w.Nq * w.d
+    dOb = inputs.f32_to_bf16_bits(inputs.normal_f32(seed, 5, 0, n)).reshape(w.B, w.H, w.Nq, w.d)
+    dO = torch.from_numpy(dOb.view(np.int16)).view(torch.bfloat16).to(dev)
+    lse = torch.empty((w.B, w.H, w.Nq), dtype=torch.float32, device=dev)
+    delta = torch.empty_like(lse)
+    dQ, dK, dV = torch.empty_like(d["Q"]), torch.empty_like(d["K"]), torch.empty_like(d["K"])
+    api.flat_attn_fwd_ex(d["Q"], d["K"], d["V"], d["O"], w.scale, k_valid_len=d["vl"], status=d["status"], lse=lse)
+    step = lambda: api.flat_attn_bwd_ex(d["Q"], d["K"], d["V"], d["O"], dO, lse, dQ, dK, dV, delta, w.scale,
+                                        k_valid_len=d["vl"], status=d["status"])
+    for _ in range(3):
+        step()
+    steps = int(max(3, min(args.steps, 10)))
+    sampler = ClockSampler(dev.index).start()
+    total_ms, per = bench.timed(step, steps, flush=False)
+    clocks = sampler.stop()
+    assert int(d["status"].item()) == 0
+    ms = float(np.mean(per))
+    flops = 2.5 * float(w.flops)
+    val = flops / (ms * 1e-3) / 1e12
+    e = {"workload": w.name, "kernel": "bwd_tc_kernel<dQ> + bwd_tc_kernel<dK,dV>", "kernels_per_step": 2, "steps": steps,
+         "ms": ms, "ms_min": float(np.min(per)), "flops_per_step": flops, "value": val, "unit": UNIT,
+         "frac": val / peaks["bf16_tflops"], "frac_of_sustained": val / peaks["bf16_tflops_sustained"],
+         "flops_executed_per_step": 3.5 * float(w.flops), "clocks": clocks}
+    if not args.no_cpu_baseline:
+        import oracle
+        Qb, Kb, Vb, vl = data
+        heads = np.array([0, (w.B * w.H) // 2 + 1], dtype=np.int64)
+        ref = oracle.attention_bwd(Qb, Kb, Vb, dOb, w.scale, valid_len=vl, heads=heads)
+        par = {}
+        for name, got in (("dQ", dQ), ("dK", dK), ("dV", dV)):
+            g = got.view(w.B * w.H, -1, w.d)[torch.from_numpy(heads).to(dev)].float().cpu().numpy().astype(np.float64)
+            err = np.abs(g - ref[name])
+            par[name] = {"max_rel_to_max": float(err.max() / np.abs(ref[name]).max()),
+                         "mean_rel_to_mean": float(err.mean() / np.abs(ref[name]).mean())}
+        e["parity_on_sample"] = {"heads": [int(h) for h in heads], **par}
+    return e
 
 
 def run_other(bench, torch, api, w, seed, args, peaks, dev):

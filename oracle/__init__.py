@@ -33,12 +33,13 @@ def _load():
     global _lib
     if _lib is None:
         lib = ctypes.CDLL(build())
-        lib.oracle_attn_rows_lse.restype = ctypes.c_int
-        lib.oracle_attn_rows_lse.argtypes = [
+        lib.oracle_attn_rows_bias.restype = ctypes.c_int
+        lib.oracle_attn_rows_bias.argtypes = [
             ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int,
             ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, ctypes.c_float,
             ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p, ctypes.c_int64,
-            ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int,
+            ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+            ctypes.c_void_p, ctypes.c_int, ctypes.c_int64, ctypes.c_int64, ctypes.c_int,
             ctypes.POINTER(ctypes.c_int)]
         lib.oracle_attn_bwd_heads.restype = ctypes.c_int
         lib.oracle_attn_bwd_heads.argtypes = [
@@ -57,7 +58,7 @@ def hardware_threads() -> int:
 
 
 def attention(Q, K, V, scale, valid_len=None, rows=None, want_logits=False, want_weights=False,
-              nthreads: int = 0, causal: bool = False, want_lse=False):
+              nthreads: int = 0, causal: bool = False, want_lse=False, bias=None):
     """Exact attention in double precision.
 
     Q: [B,H,Nq,d], K/V: [B,H,Nk,d]; dtype uint16 (bf16 bit patterns) or float32.
@@ -66,6 +67,8 @@ def attention(Q, K, V, scale, valid_len=None, rows=None, want_logits=False, want
     Returns dict with 'O' ([B,H,Nq,d] or [nrows,d] float64), optionally 'L' and
     'A' ([..., Nk]), 'LSE' ([B,H,Nq] or [nrows]: log of the row's sum of exp(scaled logit) over its
     valid keys, -inf for a row without any), and 'threads' (threads used).
+    bias: optional additive term of the scaled logits, [B or 1, H or 1, Nq, Nk], uint16 (bf16 bits) or
+    float32; size-1 batch / head axes are repeated; -inf switches a (query, key) pair off.
     """
     Q = np.ascontiguousarray(Q); K = np.ascontiguousarray(K); V = np.ascontiguousarray(V)
     if Q.dtype == np.uint16:
@@ -96,11 +99,24 @@ def attention(Q, K, V, scale, valid_len=None, rows=None, want_logits=False, want
     L = np.empty(lshape, dtype=np.float64) if want_logits else None
     A = np.empty(lshape, dtype=np.float64) if want_weights else None
     LSE = np.empty(oshape[:-1], dtype=np.float64) if want_lse else None
+    bias_dtype = bias_sb = bias_sh = 0
+    if bias is not None:
+        bias = np.ascontiguousarray(bias)
+        if bias.dtype == np.uint16:
+            bias_dtype = 0
+        elif bias.dtype == np.float32:
+            bias_dtype = 1
+        else:
+            raise TypeError("bias must be uint16 (bf16 bits) or float32")
+        if bias.ndim != 4 or bias.shape[2:] != (Nq, Nk) or bias.shape[0] not in (1, B) or bias.shape[1] not in (1, H):
+            raise ValueError("bias must be [B or 1, H or 1, Nq, Nk]")
+        bias_sh = 0 if bias.shape[1] == 1 else Nq * Nk
+        bias_sb = 0 if bias.shape[0] == 1 else bias.shape[1] * Nq * Nk
     used = ctypes.c_int(0)
     ptr = lambda a: None if a is None else a.ctypes.data_as(ctypes.c_void_p)
-    rc = _load().oracle_attn_rows_lse(ptr(Q), ptr(K), ptr(V), dtype, B, H, Nq, Nk, d, float(np.float32(scale)),
-                                      ptr(vl), 1 if causal else 0, ptr(rows), n, ptr(O), ptr(L), ptr(A), ptr(LSE),
-                                      int(nthreads), ctypes.byref(used))
+    rc = _load().oracle_attn_rows_bias(ptr(Q), ptr(K), ptr(V), dtype, B, H, Nq, Nk, d, float(np.float32(scale)),
+                                       ptr(vl), 1 if causal else 0, ptr(rows), n, ptr(O), ptr(L), ptr(A), ptr(LSE),
+                                       ptr(bias), bias_dtype, bias_sb, bias_sh, int(nthreads), ctypes.byref(used))
     if rc != 0:
         raise ValueError("oracle_attn_rows rejected its arguments (code %d)" % rc)
     out = {"O": O, "threads": used.value}

@@ -22,6 +22,9 @@
 //   * key-padding mask: key j of batch b takes part iff j < valid_len[b]; masked
 //     keys are left out before the maximum.  A row with no valid key gives O = 0.
 //   * Nq may differ from Nk (cross attention): softmax still runs along keys.
+//   * additive bias (the relative-position terms of the paper's T5 / TrXL workloads, Section 6.1;
+//     the paper does not model them): a tensor [B or 1, H or 1, Nq, Nk] added to the SCALED logit
+//     before the maximum; -inf switches a pair off, a row with every pair off gives O = 0.
 //   * causal mask (decoder workloads; the paper does not spell masks out): query i takes
 //     part with key j iff j <= i + (Nk - Nq), i.e. the last query sees every key and each
 //     earlier query one key fewer; combined with the key-padding mask by intersection.
@@ -59,6 +62,9 @@ struct Problem {
     double* L;                       // [nrows, Nk] scaled logits, or null
     double* A;                       // [nrows, Nk] softmax weights, or null
     double* LSE;                     // [nrows] log of the row's sum of exponentials of the scaled logits, or null
+    const void* bias;                // additive term of the logits, or null: element (b,h,i,j) at
+    int bias_dtype;                  //   b * bias_sb + h * bias_sh + i * Nk + j  (0: bf16 bits, 1: float32);
+    int64_t bias_sb, bias_sh;        //   a stride of 0 repeats the same values for every batch / head
 };
 
 inline double elem(const void* base, int dtype, int64_t idx) {
@@ -90,6 +96,9 @@ void attend_row(const Problem& p, int64_t r, std::vector<double>& s) {
         for (int64_t t = 0; t < p.d; ++t)
             acc += elem(p.Q, p.dtype, qoff + t) * elem(p.K, p.dtype, koff + j * p.d + t);
         s[j] = p.scale * acc;
+        // The bias joins the SCALED logit (it is not multiplied by scale) and takes part in the
+        // maximum and the softmax like any logit; -inf switches the pair off.
+        if (p.bias) s[j] += elem(p.bias, p.bias_dtype, b * p.bias_sb + (bh % p.H) * p.bias_sh + i * p.Nk + j);
     }
     if (lrow) {
         for (int64_t j = 0; j < p.Nk; ++j) lrow[j] = (j < n) ? s[j] : -INFINITY;
@@ -103,6 +112,7 @@ void attend_row(const Problem& p, int64_t r, std::vector<double>& s) {
     // Step 3: softmax along the key index.
     double m = s[0];
     for (int64_t j = 1; j < n; ++j) if (s[j] > m) m = s[j];
+    if (m == -INFINITY) return;      // every pair switched off by the bias: as for a row without keys
     double l = 0.0;
     for (int64_t j = 0; j < n; ++j) { s[j] = std::exp(s[j] - m); l += s[j]; }
     if (p.LSE) p.LSE[r] = m + std::log(l);
@@ -128,20 +138,24 @@ extern "C" {
 
 // Returns 0 on success, 1 on a bad argument.  `nthreads` <= 0 means "all hardware
 // threads"; the count actually used is written to *threads_used if non-null.
-int oracle_attn_rows_lse(const void* Q, const void* K, const void* V, int dtype,
-                         int64_t B, int64_t H, int64_t Nq, int64_t Nk, int64_t d, float scale,
-                         const int32_t* valid_len, int causal, const int64_t* rows, int64_t nrows,
-                         double* O, double* L, double* A, double* LSE, int nthreads, int* threads_used) {
+int oracle_attn_rows_bias(const void* Q, const void* K, const void* V, int dtype,
+                          int64_t B, int64_t H, int64_t Nq, int64_t Nk, int64_t d, float scale,
+                          const int32_t* valid_len, int causal, const int64_t* rows, int64_t nrows,
+                          double* O, double* L, double* A, double* LSE,
+                          const void* bias, int bias_dtype, int64_t bias_sb, int64_t bias_sh,
+                          int nthreads, int* threads_used) {
     if (!Q || !K || !V || !O) return 1;
     if (B < 1 || H < 1 || Nq < 1 || Nk < 1 || d < 1) return 1;
     if (dtype != 0 && dtype != 1) return 1;
+    if (bias && ((bias_dtype != 0 && bias_dtype != 1) || bias_sb < 0 || bias_sh < 0)) return 1;
     const int64_t total = B * H * Nq;
     if (!rows) nrows = total;
     if (nrows < 0) return 1;
     if (rows) for (int64_t r = 0; r < nrows; ++r) if (rows[r] < 0 || rows[r] >= total) return 1;
     if (valid_len) for (int64_t b = 0; b < B; ++b) if (valid_len[b] < 0 || valid_len[b] > Nk) return 1;
 
-    Problem p{Q, K, V, dtype, B, H, Nq, Nk, d, static_cast<double>(scale), valid_len, causal ? 1 : 0, rows, nrows, O, L, A, LSE};
+    Problem p{Q, K, V, dtype, B, H, Nq, Nk, d, static_cast<double>(scale), valid_len, causal ? 1 : 0, rows, nrows, O, L, A, LSE,
+              bias, bias_dtype, bias_sb, bias_sh};
     int nt = nthreads > 0 ? nthreads : static_cast<int>(std::thread::hardware_concurrency());
     if (nt < 1) nt = 1;
     if (nt > nrows) nt = nrows > 0 ? static_cast<int>(nrows) : 1;
@@ -156,6 +170,14 @@ int oracle_attn_rows_lse(const void* Q, const void* K, const void* V, int dtype,
     }
     for (auto& th : pool) th.join();
     return 0;
+}
+
+int oracle_attn_rows_lse(const void* Q, const void* K, const void* V, int dtype,
+                         int64_t B, int64_t H, int64_t Nq, int64_t Nk, int64_t d, float scale,
+                         const int32_t* valid_len, int causal, const int64_t* rows, int64_t nrows,
+                         double* O, double* L, double* A, double* LSE, int nthreads, int* threads_used) {
+    return oracle_attn_rows_bias(Q, K, V, dtype, B, H, Nq, Nk, d, scale, valid_len, causal, rows, nrows, O, L, A, LSE,
+                                 nullptr, 0, 0, 0, nthreads, threads_used);
 }
 
 int oracle_attn_rows(const void* Q, const void* K, const void* V, int dtype,

@@ -327,3 +327,84 @@ def test_bad_arguments_rejected():
         oracle.attention(Q, Q, Q, 1.0, valid_len=np.array([3], np.int32))
     with pytest.raises(ValueError):
         oracle.attention(Q, Q, Q, 1.0, rows=np.array([2], np.int64))
+
+
+# ------------------------------------------------------------------------------------------------
+# Additive bias of the logits (reading: added to the SCALED logit before the maximum; [B or 1, H or 1,
+# Nq, Nk]; -inf switches a pair off).  Pinned by closed forms, invariances, mask equivalences and an
+# independent numpy softmax.
+
+def _rand_f32(rng, *shape):
+    return rng.standard_normal(shape).astype(np.float32)
+
+
+def test_bias_closed_form_and_not_scaled():
+    # Q = 0: the weights are softmax(bias) whatever the scale; bias = log(1, 2, 3), V = (6, 12, 18) -> 14
+    Q = np.zeros((1, 1, 2, 1), dtype=np.float32)
+    K = np.array([0.3, -1.0, 2.0], dtype=np.float32).reshape(1, 1, 3, 1)
+    V = np.array([6.0, 12.0, 18.0], dtype=np.float32).reshape(1, 1, 3, 1)
+    bias = np.log(np.array([[1.0, 2.0, 3.0], [3.0, 2.0, 1.0]])).astype(np.float32).reshape(1, 1, 2, 3)
+    r = oracle.attention(Q, K, V, 7.0, bias=bias, want_weights=True)
+    assert np.abs(r["A"][0, 0, 0] - np.array([1, 2, 3]) / 6.0).max() < 1e-7       # (float32 logs)
+    assert abs(r["O"][0, 0, 0, 0] - 14.0) < 1e-5 and abs(r["O"][0, 0, 1, 0] - 10.0) < 1e-5
+    # scale = 0 with arbitrary Q: again softmax(bias) -- the bias is not multiplied by the scale
+    Q2 = _rand_f32(np.random.default_rng(1), 1, 1, 2, 1)
+    r0 = oracle.attention(Q2, K, V, 0.0, bias=bias, want_weights=True)
+    assert np.abs(r0["A"] - r["A"]).max() < 1e-15
+    # ... and with scale != 0 it differs from scaling the bias too
+    r1 = oracle.attention(Q2, K, V, 2.0, bias=bias)["O"]
+    r2 = oracle.attention(Q2, K, V, 2.0, bias=(2.0 * bias).astype(np.float32))["O"]
+    assert np.abs(r1 - r2).max() > 1e-3
+
+
+def test_bias_invariances_and_independent_softmax():
+    rng = np.random.default_rng(12)
+    B, H, Nq, Nk, d = 2, 3, 5, 9, 4
+    Q, K, V = _rand_f32(rng, B, H, Nq, d), _rand_f32(rng, B, H, Nk, d), _rand_f32(rng, B, H, Nk, d)
+    bias = _rand_f32(rng, B, H, Nq, Nk)
+    s = np.float64(np.float32(0.6))
+    got = oracle.attention(Q, K, V, 0.6, bias=bias, want_lse=True)
+    S = s * np.einsum("bhid,bhjd->bhij", Q.astype(np.float64), K.astype(np.float64)) + bias
+    A = np.exp(S - S.max(-1, keepdims=True)); A /= A.sum(-1, keepdims=True)
+    assert np.abs(got["O"] - A @ V.astype(np.float64)).max() < 1e-13
+    from scipy.special import logsumexp
+    assert np.abs(got["LSE"] - logsumexp(S, axis=-1)).max() < 1e-12
+    # a per-row constant added to the bias changes nothing (exactly representable shifts)
+    shift = (np.round(rng.standard_normal((B, H, Nq, 1)) * 4) / 4).astype(np.float32)
+    b16 = (np.round(bias * 16) / 16).astype(np.float32)
+    o1 = oracle.attention(Q, K, V, 0.6, bias=b16)["O"]
+    o2 = oracle.attention(Q, K, V, 0.6, bias=(b16 + shift).astype(np.float32))["O"]
+    assert np.abs(o1 - o2).max() < 1e-13
+    # zero bias = no bias, bit for bit
+    assert np.array_equal(oracle.attention(Q, K, V, 0.6, bias=np.zeros_like(bias))["O"], oracle.attention(Q, K, V, 0.6)["O"])
+    # broadcast over batch and / or head = the explicitly repeated tensor
+    for shape in ((1, H), (B, 1), (1, 1)):
+        small = _rand_f32(rng, shape[0], shape[1], Nq, Nk)
+        full = np.ascontiguousarray(np.broadcast_to(small, (B, H, Nq, Nk)))
+        assert np.array_equal(oracle.attention(Q, K, V, 0.6, bias=small)["O"], oracle.attention(Q, K, V, 0.6, bias=full)["O"])
+    # bf16 bias bits = the widened values
+    bits = inputs.f32_to_bf16_bits(bias).reshape(bias.shape)
+    wide = inputs.bf16_bits_to_f32(bits).reshape(bias.shape)
+    assert np.array_equal(oracle.attention(Q, K, V, 0.6, bias=bits)["O"], oracle.attention(Q, K, V, 0.6, bias=wide)["O"])
+
+
+def test_bias_minus_infinity_is_a_mask():
+    rng = np.random.default_rng(13)
+    B, H, Nq, Nk, d = 2, 2, 6, 8, 4
+    Q, K, V = _rand_f32(rng, B, H, Nq, d), _rand_f32(rng, B, H, Nk, d), _rand_f32(rng, B, H, Nk, d)
+    # key padding: -inf on keys j >= valid_len[b]
+    vl = np.array([5, 8], dtype=np.int32)
+    bias = np.zeros((B, 1, Nq, Nk), dtype=np.float32)
+    bias[0, :, :, 5:] = -np.inf
+    a = oracle.attention(Q, K, V, 0.7, bias=bias, want_weights=True)
+    b = oracle.attention(Q, K, V, 0.7, valid_len=vl, want_weights=True)
+    assert np.abs(a["O"] - b["O"]).max() < 1e-15 and np.array_equal(a["A"] == 0, b["A"] == 0)
+    # causal: -inf above the diagonal (offset Nk - Nq)
+    cb = np.where(np.arange(Nk)[None, :] <= np.arange(Nq)[:, None] + (Nk - Nq), 0.0, -np.inf).astype(np.float32)
+    a = oracle.attention(Q, K, V, 0.7, bias=cb.reshape(1, 1, Nq, Nk))["O"]
+    assert np.abs(a - oracle.attention(Q, K, V, 0.7, causal=True)["O"]).max() < 1e-15
+    # a row with every pair switched off: O = 0, lse = -inf, no NaN
+    bias = np.zeros((1, 1, Nq, Nk), dtype=np.float32)
+    bias[0, 0, 2, :] = -np.inf
+    r = oracle.attention(Q, K, V, 0.7, bias=bias, want_lse=True)
+    assert np.all(r["O"][:, :, 2] == 0) and np.all(np.isneginf(r["LSE"][:, :, 2])) and np.all(np.isfinite(r["O"]))
