@@ -103,6 +103,20 @@ typedef struct flat_attn_params {
                                   Written by the SIMT, TC2, TC2_SINGLE and TC3 kernels (AUTO picks
                                   among these when it is set); FLAT_ERR_UNSUPPORTED for the others.
                                   The paper has no counterpart (it stops at inference).           */
+    const void* bias;          /* optional device tensor added to the SCALED logits before the
+                                  softmax (it is not multiplied by `scale`): the relative-position
+                                  terms of the paper's T5 / TrXL workloads (Section 6.1), which the
+                                  paper itself does not model.  Element (b,h,i,j) is read at
+                                  b * bias_stride_b + h * bias_stride_h + i * Nk + j (rows dense);
+                                  a stride of 0 repeats the values for every batch / head.  -inf
+                                  switches a (query, key) pair off; a row with every pair off gives
+                                  O = 0.  Aligned to its element size (16-byte alignment of the
+                                  base, the strides and Nk lets the kernel use vector loads).
+                                  Fused path only; run by the SIMT and TC2 kernels (AUTO picks TC2
+                                  for bf16 with d in {64,128}); FLAT_ERR_UNSUPPORTED for the other
+                                  variants.  NULL = none.                                         */
+    int bias_dtype;            /* FLAT_DTYPE_BF16 or FLAT_DTYPE_F32 (storage of `bias`)            */
+    long long bias_stride_b, bias_stride_h;   /* in elements, >= 0                               */
 } flat_attn_params_t;
 
 /*

@@ -41,7 +41,8 @@ class flat_attn_params_t(ctypes.Structure):
                 ("B", ctypes.c_int), ("H", ctypes.c_int), ("Nq", ctypes.c_int), ("Nk", ctypes.c_int),
                 ("d", ctypes.c_int), ("scale", ctypes.c_float), ("dtype", ctypes.c_int),
                 ("k_valid_len", ctypes.c_void_p), ("status", ctypes.c_void_p), ("variant", ctypes.c_int),
-                ("causal", ctypes.c_int), ("lse", ctypes.c_void_p)]
+                ("causal", ctypes.c_int), ("lse", ctypes.c_void_p), ("bias", ctypes.c_void_p),
+                ("bias_dtype", ctypes.c_int), ("bias_stride_b", ctypes.c_longlong), ("bias_stride_h", ctypes.c_longlong)]
 
 
 class flat_attn_bwd_params_t(ctypes.Structure):
@@ -149,7 +150,7 @@ def _dtype_code(t) -> int:
     raise TypeError("Q/K/V/O must be bfloat16 or float32")
 
 
-def _params(Q, K, V, O, scale, k_valid_len, status, variant, host=False, causal=False, lse=None):
+def _params(Q, K, V, O, scale, k_valid_len, status, variant, host=False, causal=False, lse=None, bias=None):
     B, H, Nq, d = Q.shape
     Nk = K.shape[2]
     if tuple(K.shape) != (B, H, Nk, d) or tuple(V.shape) != (B, H, Nk, d) or tuple(O.shape) != (B, H, Nq, d):
@@ -179,6 +180,16 @@ def _params(Q, K, V, O, scale, k_valid_len, status, variant, host=False, causal=
         p.lse = lse.data_ptr()
     else:
         p.lse = None
+    if bias is not None:
+        if (bias.dim() != 4 or tuple(bias.shape[2:]) != (Nq, Nk) or bias.shape[0] not in (1, B) or bias.shape[1] not in (1, H)
+                or not bias.is_cuda or not bias.is_contiguous() or bias.dtype not in (torch.bfloat16, torch.float32)):
+            raise ValueError("bias must be a contiguous CUDA bfloat16 / float32 tensor [B or 1, H or 1, Nq, Nk]")
+        p.bias = bias.data_ptr()
+        p.bias_dtype = _dtype_code(bias)
+        p.bias_stride_h = 0 if bias.shape[1] == 1 else Nq * Nk
+        p.bias_stride_b = 0 if bias.shape[0] == 1 else bias.shape[1] * Nq * Nk
+    else:
+        p.bias = None
     return p
 
 
@@ -197,11 +208,12 @@ def flat_attn_fwd(Q, K, V, O, scale, stream=None):
 
 
 def flat_attn_fwd_ex(Q, K, V, O, scale, k_valid_len=None, status=None, variant=FLAT_VARIANT_AUTO, stream=None,
-                     causal=False, lse=None):
+                     causal=False, lse=None, bias=None):
     """Fused attention with dtype choice (from the tensors), key-padding mask, kernel choice and
     causal mask (query i sees keys j <= i + (Nk - Nq)); `lse` [B,H,Nq] float32 receives each row's
-    log-sum-exp of the scaled logits (what the backward pass needs)."""
-    p = _params(Q, K, V, O, scale, k_valid_len, status, variant, causal=causal, lse=lse)
+    log-sum-exp of the scaled logits (what the backward pass needs); `bias` [B or 1, H or 1, Nq, Nk]
+    (bfloat16 or float32) is added to the scaled logits before the softmax (-inf switches a pair off)."""
+    p = _params(Q, K, V, O, scale, k_valid_len, status, variant, causal=causal, lse=lse, bias=bias)
     _check(_lib.flat_attn_fwd_ex(ctypes.byref(p), _stream_ptr(stream)))
     return O
 

@@ -19,7 +19,25 @@ struct Problem {
     int32_t* status;
     int causal;                      // 0 / 1: query i sees keys j <= i + (Nk - Nq)
     float* lse;                      // optional [B,H,Nq] fp32 output of the fused kernels: log-sum-exp of each row's scaled logits
+    // optional additive term of the scaled logits: element (b,h,i,j) at b * bias_sb + h * bias_sh + i * Nk + j
+    const void* bias;
+    int bias_dtype;                  // FLAT_DTYPE_*
+    long long bias_sb, bias_sh;      // strides in elements; 0 = the same values for every batch / head
 };
+
+// What a kernel needs to read the bias (passed by value).
+struct BiasArg {
+    const void* p;
+    int f32;                         // 1: float32, 0: bf16
+    long long sb, sh;
+    int vec;                         // 16-byte loads allowed (base, strides and Nk all multiples of 16 bytes)
+};
+inline BiasArg bias_arg(const Problem& q) {
+    const long long es = q.bias_dtype == FLAT_DTYPE_F32 ? 4 : 2, per16 = 16 / es;
+    const bool vec = q.bias && (reinterpret_cast<uintptr_t>(q.bias) & 15u) == 0 && q.Nk % per16 == 0 &&
+                     q.bias_sb % per16 == 0 && q.bias_sh % per16 == 0;
+    return BiasArg{q.bias, q.bias_dtype == FLAT_DTYPE_F32 ? 1 : 0, q.bias_sb, q.bias_sh, vec ? 1 : 0};
+}
 
 // A validated backward problem (device pointers; bf16 tensors, fp32 lse / delta).
 struct BwdProblem {
@@ -44,7 +62,7 @@ int check_params(const flat_attn_params_t* p);
 int launch_fused_simt(const Problem& p, cudaStream_t st);
 int launch_naive(const Problem& p, void* L, void* A, cudaStream_t st);
 int launch_fused_tc(const Problem& p, cudaStream_t st);
-int launch_fused_tc2(const Problem& p, cudaStream_t st);
+int launch_fused_tc2(const Problem& p, cudaStream_t st);      // (also the tensor-core kernel for calls with a bias)
 int launch_fused_tc2_single(const Problem& p, cudaStream_t st);
 int launch_fused_tc3(const Problem& p, cudaStream_t st);
 bool rgran_applies(const Problem& p);              // bf16, d = 64, Nk <= 512

@@ -164,13 +164,16 @@ __device__ __forceinline__ float exp_store(const uint32_t (&s)[128], float scale
 // packed tensors as {d, H, tokens}; blockIdx.y = sequence * H + head, blockIdx.x = slab of the
 // sequence's rows (a CTA past the end of its sequence leaves at once); the causal offset is that of
 // the sequence; valid_len is unused.
-template <int D, int NT, bool VL = false>
+// BIAS: a separate instantiation that adds a bias tensor to the scaled logits (dense batches): the softmax
+// thread fetches its row's 128 values of the step straight from device memory -- a bf16 bias adds
+// 2 B H Nq Nk bytes of traffic, four times |Q|+|K|+|V|+|O| on a 4096 x 4096, d = 64 problem.
+template <int D, int NT, bool VL = false, bool BIAS = false>
 __global__ void __launch_bounds__(128 * NT + 128, NT == 1 ? 2 : 1)
 fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                  const __grid_constant__ CUtensorMap tmV, __nv_bfloat16* __restrict__ O, int H, int Nq, int Nk,
                  float scale_log2e, const int32_t* __restrict__ valid_len, int coff, int32_t* status,
                  const int32_t* __restrict__ cu_q = nullptr, const int32_t* __restrict__ cu_k = nullptr,
-                 float* __restrict__ lse = nullptr) {
+                 float* __restrict__ lse = nullptr, BiasArg bias = BiasArg{nullptr, 0, 0, 0, 0}) {
     using LY = L2<D, NT>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -348,7 +351,9 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         const int t = warp >> 2;                         // query tile of this warpgroup
         const int row = row0 + t * BM + (warp & 3) * 32 + lane;
         const uint32_t tl = tmem + (static_cast<uint32_t>((warp & 3) * 32) << 16);
-        const bool neg_scale = scale_log2e < 0.f;
+        // (with a bias the logits are rescaled and shifted as they arrive, and the step goes on with scale 1)
+        const float sc = BIAS ? 1.f : scale_log2e;
+        const bool neg_scale = BIAS ? false : scale_log2e < 0.f;
         float m_ref = -INFINITY, l = 0.f;
         bool ok = true;
         // keys this thread's row sees; lane 0 has the shortest row of the warp
@@ -357,6 +362,23 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         const int nrow_min = __shfl_sync(0xffffffffu, nrow, 0);
         if (LY::TURNS && t == 1 && lane == 0) mbar_arrive(&bars[LY::TURN + (warp & 3)]);   // tile A goes first
         for (int j = 0; j < ntiles; ++j) {
+            // (bias, the common case of an aligned bf16 tensor: the row's 128 values of this step are fetched
+            // before the wait for the logits, so that the two latencies overlap)
+            uint32_t bpk[BIAS ? 64 : 1];
+            bool bias_ready = false;
+            if (BIAS) {
+                if (bias.vec && !bias.f32 && row < Nq && (j + 1) * BN <= Nk) {
+                    const uint4* g = reinterpret_cast<const uint4*>(
+                        static_cast<const __nv_bfloat16*>(bias.p) + static_cast<long long>(bh / H) * bias.sb +
+                        static_cast<long long>(bh % H) * bias.sh + static_cast<long long>(row) * Nk + j * BN);
+#pragma unroll
+                    for (int v = 0; v < 16; ++v) {
+                        const uint4 w = g[v];
+                        bpk[4 * v] = w.x; bpk[4 * v + 1] = w.y; bpk[4 * v + 2] = w.z; bpk[4 * v + 3] = w.w;
+                    }
+                    bias_ready = true;
+                }
+            }
             ok = bounded_wait(&bars[LY::S_FULL + t], j & 1, abort_flag, status, 0x300 + t);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
@@ -370,6 +392,58 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             if (lane == 0) mbar_arrive(&bars[LY::S_FREE + t]);   // S_t may be overwritten (d = 64: by the next S_t)
 
             const int col0 = j * BN;
+            if (BIAS) {
+                // x = s * scale * log2(e) + bias * log2(e); a row past the end and columns past Nk read nothing
+                const long long at = static_cast<long long>(bh / H) * bias.sb + static_cast<long long>(bh % H) * bias.sh +
+                                     static_cast<long long>(row) * Nk + col0;
+                const bool in_rows = row < Nq;
+                if (bias_ready) {
+#pragma unroll
+                    for (int i = 0; i < 64; ++i) {
+                        s[2 * i] = __float_as_uint(fmaf(__uint_as_float(s[2 * i]), scale_log2e,
+                                                        __uint_as_float(bpk[i] << 16) * 1.4426950408889634f));
+                        s[2 * i + 1] = __float_as_uint(fmaf(__uint_as_float(s[2 * i + 1]), scale_log2e,
+                                                            __uint_as_float(bpk[i] & 0xffff0000u) * 1.4426950408889634f));
+                    }
+                } else if (bias.vec && in_rows && col0 + BN <= Nk) {
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) {        // sixteen columns at a time (few registers live)
+                        float bv[16];
+                        if (bias.f32) {
+                            const float4* g = reinterpret_cast<const float4*>(static_cast<const float*>(bias.p) + at + c * 16);
+#pragma unroll
+                            for (int v = 0; v < 4; ++v) {
+                                const float4 w = g[v];
+                                bv[4 * v] = w.x; bv[4 * v + 1] = w.y; bv[4 * v + 2] = w.z; bv[4 * v + 3] = w.w;
+                            }
+                        } else {
+                            const uint4* g = reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(bias.p) + at + c * 16);
+#pragma unroll
+                            for (int v = 0; v < 2; ++v) {
+                                const uint4 w = g[v];
+                                const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+                                for (int e = 0; e < 4; ++e) {
+                                    bv[8 * v + 2 * e] = __uint_as_float(ww[e] << 16);
+                                    bv[8 * v + 2 * e + 1] = __uint_as_float(ww[e] & 0xffff0000u);
+                                }
+                            }
+                        }
+#pragma unroll
+                        for (int i = 0; i < 16; ++i)
+                            s[c * 16 + i] = __float_as_uint(fmaf(__uint_as_float(s[c * 16 + i]), scale_log2e, bv[i] * 1.4426950408889634f));
+                    }
+                } else {
+#pragma unroll                                           // (fully: the logits must stay in registers)
+                    for (int i = 0; i < 128; ++i) {
+                        float bvi = 0.f;
+                        if (in_rows && col0 + i < Nk)
+                            bvi = bias.f32 ? static_cast<const float*>(bias.p)[at + i]
+                                           : __bfloat162float(static_cast<const __nv_bfloat16*>(bias.p)[at + i]);
+                        s[i] = __float_as_uint(fmaf(__uint_as_float(s[i]), scale_log2e, bvi * 1.4426950408889634f));
+                    }
+                }
+            }
             const bool tail = col0 + BN > nrow_min;      // (warp-uniform) some row has masked keys in this step
             const int nvalid = nrow > col0 ? (nrow - col0 < BN ? nrow - col0 : BN) : 0;   // per row
             if (tail) {
@@ -407,13 +481,13 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             bool careful = (j == 0) || tail;
             float lt = 0.f;
             if (!careful) {
-                lt = exp_store<false, !LY::TURNS>(s, scale_log2e, -m_ref, tl + LY::P_COL(t), BN, wait_p_free, pass_turn);
+                lt = exp_store<false, !LY::TURNS>(s, sc, -m_ref, tl + LY::P_COL(t), BN, wait_p_free, pass_turn);
                 if (!ok) break;                           // (a failed wait means the stores went nowhere useful)
                 careful = __any_sync(0xffffffffu, !(lt <= OVERFLOW_SUM));
             }
             if (careful) {
                 // (a row with no valid key in this step -- causal mask -- contributes no maximum)
-                const float mx = nvalid > 0 ? (neg_scale ? row_min(s) : row_max(s)) * scale_log2e : -INFINITY;
+                const float mx = nvalid > 0 ? (neg_scale ? row_min(s) : row_max(s)) * sc : -INFINITY;
                 if (__any_sync(0xffffffffu, mx > m_ref + RESCALE_THRESHOLD)) {
                     const float m_new = fmaxf(m_ref, mx);
                     // 0 on the first tile; a row that has not seen a valid key yet keeps l = 0
@@ -437,7 +511,10 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                     }
                     m_ref = m_new;
                 }
-                lt = exp_store<true, false>(s, scale_log2e, -m_ref, tl + LY::P_COL(t), nvalid, wait_p_free, pass_turn);
+                // (a row whose every pair so far was switched off by a -inf bias still has no reference:
+                // 0 then stands in, so that its weights come out as 2^-inf = 0 and not as NaN)
+                lt = exp_store<true, false>(s, sc, (BIAS && m_ref == -INFINITY) ? 0.f : -m_ref, tl + LY::P_COL(t), nvalid,
+                                            wait_p_free, pass_turn);
                 if (!ok) break;
             }
             l += lt;
@@ -495,12 +572,24 @@ int launch_tc2_d(const Problem& p, cudaStream_t st) {
     if (!make_map(&tmQ, p.Q, BH, p.Nq, D, BM) || !make_map(&tmK, p.K, BH, p.Nk, D, BN) ||
         !make_map(&tmV, p.V, BH, p.Nk, D, BN))
         return FLAT_ERR_CUDA;
+    dim3 grid((p.Nq + NT * BM - 1) / (NT * BM), BH);
+    if (p.bias) {
+        if constexpr (NT == 2) {
+            if (!ensure_dynamic_smem<fused_tc2_kernel<D, NT, false, true>>(LY::SMEM_BYTES)) return FLAT_ERR_CUDA;
+            fused_tc2_kernel<D, NT, false, true><<<grid, LY::THREADS, LY::SMEM_BYTES, st>>>(
+                tmQ, tmK, tmV, static_cast<__nv_bfloat16*>(p.O), p.H, p.Nq, p.Nk, p.scale * 1.4426950408889634f,
+                p.k_valid_len, p.causal ? p.Nk - p.Nq : (1 << 30), p.status, nullptr, nullptr, p.lse, bias_arg(p));
+            return cudaGetLastError() == cudaSuccess ? FLAT_OK : FLAT_ERR_CUDA;
+        } else {
+            return FLAT_ERR_UNSUPPORTED;
+        }
+    }
     auto kern = fused_tc2_kernel<D, NT>;
     if (!ensure_dynamic_smem<fused_tc2_kernel<D, NT>>(LY::SMEM_BYTES)) return FLAT_ERR_CUDA;
-    dim3 grid((p.Nq + NT * BM - 1) / (NT * BM), BH);
     kern<<<grid, LY::THREADS, LY::SMEM_BYTES, st>>>(tmQ, tmK, tmV, static_cast<__nv_bfloat16*>(p.O), p.H, p.Nq,
                                                     p.Nk, p.scale * 1.4426950408889634f, p.k_valid_len,
-                                                    p.causal ? p.Nk - p.Nq : (1 << 30), p.status, nullptr, nullptr, p.lse);
+                                                    p.causal ? p.Nk - p.Nq : (1 << 30), p.status, nullptr, nullptr, p.lse,
+                                                    BiasArg{nullptr, 0, 0, 0, 0});
     return cudaGetLastError() == cudaSuccess ? FLAT_OK : FLAT_ERR_CUDA;
 }
 

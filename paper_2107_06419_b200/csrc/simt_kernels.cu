@@ -129,7 +129,7 @@ __global__ void __launch_bounds__(NTHREADS) fused_simt_kernel(const T* __restric
                                                               const T* __restrict__ V, T* __restrict__ O, int H,
                                                               int Nq, int Nk, float scale_log2e,
                                                               const int32_t* __restrict__ valid_len, int causal,
-                                                              float* __restrict__ lse) {
+                                                              float* __restrict__ lse, BiasArg bias) {
     extern __shared__ __align__(16) float smem[];
     float* Qs = smem;
     float* Ks = Qs + 64 * (D + 4);
@@ -174,6 +174,13 @@ __global__ void __launch_bounds__(NTHREADS) fused_simt_kernel(const T* __restric
 #pragma unroll
             for (int b = 0; b < 4; ++b) {
                 s[a][b] = (k0 + tx + 16 * b < nrow[a]) ? s[a][b] * scale_log2e : -INFINITY;
+                // additive bias of the scaled logit (natural units -> base 2); -inf switches the pair off
+                if (bias.p && k0 + tx + 16 * b < nrow[a] && row0 + ty + 16 * a < Nq) {
+                    const long long at = (bh / H) * bias.sb + (bh % H) * bias.sh + (row0 + ty + 16 * a) * Nk + k0 + tx + 16 * b;
+                    const float bv = bias.f32 ? static_cast<const float*>(bias.p)[at]
+                                              : __bfloat162float(static_cast<const __nv_bfloat16*>(bias.p)[at]);
+                    s[a][b] = fmaf(bv, 1.4426950408889634f, s[a][b]);
+                }
                 mx = fmaxf(mx, s[a][b]);
             }
             mx = halfwarp_max(mx);
@@ -322,7 +329,7 @@ static int launch_fused_simt_td(const Problem& p, cudaStream_t st) {
     dim3 grid((p.Nq + TM - 1) / TM, p.B * p.H);
     kern<<<grid, NTHREADS, smem, st>>>(static_cast<const T*>(p.Q), static_cast<const T*>(p.K),
                                        static_cast<const T*>(p.V), static_cast<T*>(p.O), p.H, p.Nq, p.Nk,
-                                       p.scale * 1.4426950408889634f, p.k_valid_len, p.causal, p.lse);
+                                       p.scale * 1.4426950408889634f, p.k_valid_len, p.causal, p.lse, bias_arg(p));
     return cudaGetLastError() == cudaSuccess ? FLAT_OK : FLAT_ERR_CUDA;
 }
 
