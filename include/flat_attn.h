@@ -244,6 +244,19 @@ int flat_attn_layer_fwd(const void* X, const void* Wqkv, const void* Wo, void* Y
 int flat_fc_fwd(const void* X, const void* W, void* Y, int M, int K, int Nout, int32_t* status, void* stream);
 
 /*
+ * The normalisation layer of an attention block (paper Section 2 lists it between the attention layer
+ * and the fully connected layers and says no more).  Reading taken: layer normalisation of every token
+ * over its D features, after the residual add:
+ *     z = X + R  (R may be NULL: z = X),    Y = gamma * (z - mean(z)) / sqrt(var(z) + eps) + beta
+ * with the biased variance (divided by D).  X, R, Y: [M, D] row-major bf16; gamma, beta: [D] bf16;
+ * statistics in fp32.  Y may alias X or R.  Needs D a multiple of 8 and at most 8192
+ * (FLAT_ERR_UNSUPPORTED otherwise), eps >= 0; DEVICE pointers, 16-byte aligned.  One kernel, bound by
+ * device-memory bandwidth (each element read once, written once).
+ */
+int flat_layernorm_fwd(const void* X, const void* R, const void* gamma, const void* beta, void* Y,
+                       long long M, int D, float eps, void* stream);
+
+/*
  * End-to-end convenience call with HOST tensors: copies Q, K, V (and k_valid_len if
  * non-NULL) from host memory into `workspace`, runs the fused kernel, copies O back
  * to `O_host`, and returns without synchronising (use pinned host memory for true

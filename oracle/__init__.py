@@ -226,6 +226,28 @@ def fully_connected(X, W):
     return (x.reshape(-1, x.shape[-1]) @ bf16_bits_to_f64(W).T).reshape(x.shape[:-1] + (W.shape[0],))
 
 
+def layer_norm(X, gamma, beta, eps, residual=None):
+    """The block's normalisation layer (Section 2 names it without defining it; reading: layer
+    normalisation over the features of each token, after the residual add, biased variance):
+    z = X + residual, Y = gamma * (z - mean z) / sqrt(var z + eps) + beta.  X, residual [..., D] and
+    gamma, beta [D] are uint16 bf16 bits; returns Y float64 (not rounded).  Written as plain loops over
+    the rows so that it can be read against the formula."""
+    x = bf16_bits_to_f64(X)
+    if residual is not None:
+        x = x + bf16_bits_to_f64(residual)
+    g, b = bf16_bits_to_f64(gamma), bf16_bits_to_f64(beta)
+    D = x.shape[-1]
+    rows = x.reshape(-1, D)
+    out = np.empty_like(rows)
+    e = float(np.float32(eps))
+    for i in range(rows.shape[0]):
+        z = rows[i]
+        mean = z.sum() / D
+        var = ((z - mean) ** 2).sum() / D
+        out[i] = g * (z - mean) / np.sqrt(var + e) + b
+    return out.reshape(x.shape)
+
+
 def attention_layer(X, Wqkv, Wo, H, d, scale, causal=False, nthreads: int = 0):
     """Steps 1-5 for self-attention.  Returns dict: 'Q','K','V','O' (uint16 bf16 bits, as stored
     between the operators) and 'Y' [B,N,Dm] float64 (not rounded)."""

@@ -33,7 +33,7 @@ EXPORTS = ["flat_attn_fwd", "flat_attn_fwd_ex", "flat_attn_naive_fwd", "flat_att
            "flat_attn_status_string", "flat_attn_version",
            "flat_qkv_proj_fwd", "flat_out_proj_fwd", "flat_attn_layer_fwd", "flat_fc_fwd",
            "flat_attn_varlen_fwd", "flat_attn_last_variant", "flat_attn_last_device_error",
-           "flat_attn_clear_device_error", "flat_attn_bwd", "flat_attn_bwd_ex"]
+           "flat_attn_clear_device_error", "flat_attn_bwd", "flat_attn_bwd_ex", "flat_layernorm_fwd"]
 
 
 class flat_attn_params_t(ctypes.Structure):
@@ -83,6 +83,8 @@ _lib.flat_attn_layer_fwd.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i,
 _lib.flat_attn_layer_fwd.restype = _i
 _lib.flat_fc_fwd.argtypes = [_vp, _vp, _vp, _i, _i, _i, _vp, _vp]
 _lib.flat_fc_fwd.restype = _i
+_lib.flat_layernorm_fwd.argtypes = [_vp, _vp, _vp, _vp, _vp, ctypes.c_longlong, _i, _f, _vp]
+_lib.flat_layernorm_fwd.restype = _i
 _lib.flat_attn_varlen_fwd.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, ctypes.c_longlong, ctypes.c_longlong,
                                       _i, _f, _i, _vp, _vp]
 _lib.flat_attn_varlen_fwd.restype = _i
@@ -358,6 +360,18 @@ def flat_fc_fwd(X, W, Y, status=None, stream=None):
     M = X.numel() // K
     _bf16_cuda("X", X, X.shape); _bf16_cuda("W", W, (Nout, K)); _bf16_cuda("Y", Y, tuple(X.shape[:-1]) + (Nout,))
     _check(_lib.flat_fc_fwd(_ptr(X), _ptr(W), _ptr(Y), M, K, Nout, _ptr(status), _stream_ptr(stream)))
+    return Y
+
+
+def flat_layernorm_fwd(X, gamma, beta, Y, eps=1e-5, residual=None, stream=None):
+    """Y = gamma * layer_norm(X + residual) + beta over the last axis (bf16 CUDA tensors; gamma, beta [D])."""
+    D = X.shape[-1]
+    M = X.numel() // D
+    _bf16_cuda("X", X, X.shape); _bf16_cuda("Y", Y, X.shape); _bf16_cuda("gamma", gamma, (D,)); _bf16_cuda("beta", beta, (D,))
+    if residual is not None:
+        _bf16_cuda("residual", residual, X.shape)
+    _check(_lib.flat_layernorm_fwd(_ptr(X), _ptr(residual), _ptr(gamma), _ptr(beta), _ptr(Y), M, D, float(eps),
+                                   _stream_ptr(stream)))
     return Y
 
 

@@ -378,6 +378,18 @@ int flat_fc_fwd(const void* X, const void* W, void* Y, int M, int K, int Nout, i
     return r;
 }
 
+int flat_layernorm_fwd(const void* X, const void* R, const void* gamma, const void* beta, void* Y, long long M, int D,
+                       float eps, void* stream) {
+    if (!X || !gamma || !beta || !Y) return FLAT_ERR_NULL;
+    if (M < 1 || D < 1 || !(eps >= 0.f) || !isfinite(eps)) return FLAT_ERR_SHAPE;
+    if (M > INT64_MAX / 16 / D) return FLAT_ERR_SHAPE;
+    if (D % 8 != 0 || D > 8192) return FLAT_ERR_UNSUPPORTED;
+    if (!aligned16(X) || !aligned16(gamma) || !aligned16(beta) || !aligned16(Y) || (R && !aligned16(R))) return FLAT_ERR_ALIGN;
+    const int r = flat::launch_layernorm(X, R, gamma, beta, Y, M, D, eps, static_cast<cudaStream_t>(stream));
+    if (r == FLAT_OK) g_last_launches = 1;
+    return r;
+}
+
 int flat_attn_layer_fwd(const void* X, const void* Wqkv, const void* Wo, void* Y, void* Q, void* K, void* V, void* O,
                         int B, int N, int H, int d, int Dm, float scale, int causal, int32_t* status, void* stream) {
     if (!X || !Wqkv || !Wo || !Y || !Q || !K || !V || !O) return FLAT_ERR_NULL;

@@ -81,6 +81,9 @@ int launch_qkv_proj(const void* X, const void* Wqkv, void* Q, void* K, void* V, 
 int launch_out_proj(const void* O, const void* Wo, void* Y, int B, int N, int H, int d, int Dm, int32_t* status,
                     cudaStream_t st);
 int launch_fc(const void* X, const void* W, void* Y, int M, int Kdim, int Nout, int32_t* status, cudaStream_t st);
+// The block's normalisation layer (layernorm.cu): Y = gamma * normalise(X + R) + beta over rows of D features.
+int launch_layernorm(const void* X, const void* R, const void* gamma, const void* beta, void* Y, long long M, int D,
+                     float eps, cudaStream_t st);
 int launch_wait_timeout_selftest(int32_t* status, cudaStream_t st);
 int launch_exp2_poly_selftest(const float* x, float* y, int n, cudaStream_t st);
 // Tensor-core versions of the baseline's two contractions (bf16, d in {64,128}, Nk % 8 == 0).

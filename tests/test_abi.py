@@ -25,7 +25,7 @@ def api(lib):
 def declared_functions():
     src = open(HEADER).read()
     src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
-    return sorted(set(re.findall(r"\b(flat_(?:attn|qkv_proj|out_proj|fc)_\w+)\s*\(", src)))
+    return sorted(set(re.findall(r"\b(flat_(?:attn|qkv_proj|out_proj|fc|layernorm)_\w+)\s*\(", src)))
 
 
 def test_header_declares_and_library_exports(lib, api):
@@ -78,6 +78,13 @@ def test_projection_argument_errors(api):
     assert fc(0x10000, 0x20000, 0x30000, 0, 64, 256, None, None) == 2
     assert fc(0x10000, 0x20000, 0x30000, 128, 100, 256, None, None) == 3 and fc(0x10000, 0x20000, 0x30000, 128, 64, 128, None, None) == 3
     assert fc(0x10000, 0x20000, 0x30008, 128, 64, 256, None, None) == 4
+    ln = api._lib.flat_layernorm_fwd
+    assert ln(None, None, 0x20000, 0x30000, 0x40000, 16, 256, 1e-5, None) == 1
+    assert ln(0x10000, None, 0x20000, 0x30000, 0x40000, 0, 256, 1e-5, None) == 2
+    assert ln(0x10000, None, 0x20000, 0x30000, 0x40000, 16, 256, -1.0, None) == 2
+    assert ln(0x10000, None, 0x20000, 0x30000, 0x40000, 16, 100, 1e-5, None) == 3      # D a multiple of 8
+    assert ln(0x10000, None, 0x20000, 0x30000, 0x40000, 16, 16384, 1e-5, None) == 3    # D at most 8192
+    assert ln(0x10000, 0x50008, 0x20000, 0x30000, 0x40000, 16, 256, 1e-5, None) == 4
     h = api._lib.flat_attn_layer_fwd
     def layer(**kw):
         a = dict(dict(X=0x10000, Wqkv=0x20000, Wo=0x30000, Y=0x40000, Q=0x50000, K=0x60000, V=0x70000, O=0x80000,

@@ -117,3 +117,59 @@ def test_fully_connected_by_hand():
     assert np.array_equal(Y, [[1.0, 5.0, 12.0, 2.0], [0.5, -1.0, -1.0, -0.5]])
     # leading dimensions are kept
     assert oracle.fully_connected(X.reshape(1, 2, 3), W).shape == (1, 2, 4)
+
+
+# ------------------------------------------------------------------------------------------------
+# The block's normalisation layer (reading: layer normalisation over the features, after the residual add)
+
+def _bits(a):
+    return inputs.f32_to_bf16_bits(np.asarray(a, dtype=np.float32)).reshape(np.shape(a))
+
+
+def test_layer_norm_hand_example_and_moments():
+    # z = (1, 2, 3, 4): mean 2.5, biased variance 1.25 -> (z - 2.5) / sqrt(1.25); eps = 0
+    X = _bits([[1.0, 2.0, 3.0, 4.0]])
+    one, zero = _bits(np.ones(4)), _bits(np.zeros(4))
+    y = oracle.layer_norm(X, one, zero, 0.0)
+    assert np.abs(y[0] - np.array([-1.5, -0.5, 0.5, 1.5]) / np.sqrt(1.25)).max() < 1e-15
+    # gamma scales and beta shifts feature by feature
+    y2 = oracle.layer_norm(X, _bits([2.0, 1.0, 0.5, -1.0]), _bits([0.0, 1.0, 2.0, 3.0]), 0.0)
+    assert np.abs(y2[0] - (np.array([2.0, 1.0, 0.5, -1.0]) * y[0] + np.array([0.0, 1.0, 2.0, 3.0]))).max() < 1e-15
+    # random rows: zero mean and unit (biased) variance of the output when gamma = 1, beta = 0, eps = 0
+    rng = np.random.default_rng(3)
+    X = _bits(rng.standard_normal((5, 7, 64)) * 3 + 1)
+    y = oracle.layer_norm(X, _bits(np.ones(64)), _bits(np.zeros(64)), 0.0)
+    assert np.abs(y.mean(-1)).max() < 1e-14 and np.abs((y ** 2).mean(-1) - 1).max() < 1e-13
+
+
+def test_layer_norm_invariances_residual_and_eps():
+    rng = np.random.default_rng(4)
+    x = np.round(rng.standard_normal((6, 32)) * 8) / 8           # exactly representable, also after the maps below
+    g, b = _bits(rng.standard_normal(32)), _bits(rng.standard_normal(32))
+    y = oracle.layer_norm(_bits(x), g, b, 0.0)
+    # shifting a row by a constant and scaling it by a positive constant change nothing (eps = 0)
+    assert np.abs(oracle.layer_norm(_bits(4 * x + 2), g, b, 0.0) - y).max() < 1e-13
+    # a negative scale flips the normalised row: y -> 2 beta - y
+    assert np.abs(oracle.layer_norm(_bits(-x), g, b, 0.0) - (2 * oracle.bf16_bits_to_f64(b) - y)).max() < 1e-13
+    # the residual is added before the statistics: LN(x, residual = r) = LN(x + r)
+    r = np.round(rng.standard_normal((6, 32)) * 8) / 8
+    assert np.array_equal(oracle.layer_norm(_bits(x), g, b, 1e-5, residual=_bits(r)), oracle.layer_norm(_bits(x + r), g, b, 1e-5))
+    # eps enters under the root, next to the variance: a constant row gives exactly beta, and a row of
+    # variance v is scaled by sqrt(v / (v + eps))
+    c = oracle.layer_norm(_bits(np.full((1, 32), 3.0)), g, b, 1e-5)
+    assert np.array_equal(c[0], oracle.bf16_bits_to_f64(b))
+    v = x[0].var()
+    e = np.float64(np.float32(0.5))
+    lhs = oracle.layer_norm(_bits(x[:1]), _bits(np.ones(32)), _bits(np.zeros(32)), 0.5)
+    rhs = oracle.layer_norm(_bits(x[:1]), _bits(np.ones(32)), _bits(np.zeros(32)), 0.0) * np.sqrt(v / (v + e))
+    assert np.abs(lhs - rhs).max() < 1e-14
+
+
+def test_layer_norm_against_an_independent_library_routine():
+    import torch
+    rng = np.random.default_rng(5)
+    X, R = _bits(rng.standard_normal((3, 9, 128))), _bits(rng.standard_normal((3, 9, 128)))
+    g, b = _bits(rng.standard_normal(128)), _bits(rng.standard_normal(128))
+    f = lambda bits: torch.from_numpy(oracle.bf16_bits_to_f64(bits))
+    want = torch.nn.functional.layer_norm(f(X) + f(R), (128,), f(g), f(b), eps=float(np.float32(1e-5))).numpy()
+    assert np.abs(oracle.layer_norm(X, g, b, 1e-5, residual=R) - want).max() < 1e-12
