@@ -79,8 +79,11 @@ def test_full_size_causal_sampled_rows(api, name, per_head):
     assert bool(torch.isfinite(O.float()).all())
 
 
-@pytest.mark.parametrize("name,per_head", [("c4_64k_d128", 64), ("c5_cross_masked", 32)])
+@pytest.mark.parametrize("name,per_head", [("c2_bert_large_4k", 16), ("c3_16k", 16), ("c4_64k_d128", 64),
+                                           ("c5_cross_masked", 32)])
 def test_full_size_planted_keys(api, name, per_head):
+    """(c2 and c3 run on the persistent grid, 27-28 work items per CTA: a key tile lost or repeated at an
+    item boundary would move these outputs by O(1), where iid rows would hide it inside the tolerance)"""
     w = inputs.WORKLOADS[name]
     Qb, Kb, Vb, planted = inputs.make_planted_qkv_bf16(w)
     vl = inputs.make_valid_len(w) if w.masked else None
