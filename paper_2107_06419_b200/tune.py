@@ -11,7 +11,8 @@ variants: 64-row FFMA tiles, 128-row tensor-core CTAs (one or two per SM) and 25
     python -m paper_2107_06419_b200.tune --causal     (the variants under the causal mask)
     python -m paper_2107_06419_b200.tune --varlen     (packed variable-length batches; with --causal too)
 
-Prints one JSON line per (workload, variant) and the winner per workload; inputs are random bf16
+Prints one JSON line per (workload, variant) and the winner per workload; the batched sweeps run on
+the seeded generator's inputs (the bytes bench.py times), the layer and packed sweeps on random bf16
 (timing only -- parity is the tests' business).
 """
 from __future__ import annotations
@@ -20,6 +21,7 @@ import argparse
 import json
 import time
 
+import numpy as np
 import torch
 
 from . import api, inputs
@@ -35,11 +37,22 @@ VARIANTS = {
 }
 
 
+_QKV_CACHE = {}
+
+
+def _seeded_qkv(w, dev):
+    """The workload's inputs from the seeded generator (the bytes that bench.py and the tests use),
+    generated once per workload."""
+    if w.name not in _QKV_CACHE:
+        _QKV_CACHE.clear()
+        as_t = lambda bits: torch.from_numpy(bits.view(np.int16)).view(torch.bfloat16).to(dev)
+        _QKV_CACHE[w.name] = tuple(as_t(x) for x in inputs.make_qkv_bf16(w))
+    return _QKV_CACHE[w.name]
+
+
 def time_variant(w, variant, steps, warmup=2, causal=False):
     dev = torch.device("cuda")
-    Q = torch.randn(w.B, w.H, w.Nq, w.d, device=dev, dtype=torch.bfloat16)
-    K = torch.randn(w.B, w.H, w.Nk, w.d, device=dev, dtype=torch.bfloat16)
-    V = torch.randn_like(K)
+    Q, K, V = _seeded_qkv(w, dev)
     O = torch.empty_like(Q)
     vl = None
     if w.masked:
