@@ -33,13 +33,14 @@ def _load():
     global _lib
     if _lib is None:
         lib = ctypes.CDLL(build())
-        lib.oracle_attn_rows_bias.restype = ctypes.c_int
-        lib.oracle_attn_rows_bias.argtypes = [
+        lib.oracle_attn_rows_sparse.restype = ctypes.c_int
+        lib.oracle_attn_rows_sparse.argtypes = [
             ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int,
             ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, ctypes.c_float,
             ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p, ctypes.c_int64,
             ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
-            ctypes.c_void_p, ctypes.c_int, ctypes.c_int64, ctypes.c_int64, ctypes.c_int,
+            ctypes.c_void_p, ctypes.c_int, ctypes.c_int64, ctypes.c_int64,
+            ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, ctypes.c_int,
             ctypes.POINTER(ctypes.c_int)]
         lib.oracle_attn_bwd_heads.restype = ctypes.c_int
         lib.oracle_attn_bwd_heads.argtypes = [
@@ -58,7 +59,7 @@ def hardware_threads() -> int:
 
 
 def attention(Q, K, V, scale, valid_len=None, rows=None, want_logits=False, want_weights=False,
-              nthreads: int = 0, causal: bool = False, want_lse=False, bias=None):
+              nthreads: int = 0, causal: bool = False, want_lse=False, bias=None, block_mask=None, block: int = 128):
     """Exact attention in double precision.
 
     Q: [B,H,Nq,d], K/V: [B,H,Nk,d]; dtype uint16 (bf16 bit patterns) or float32.
@@ -69,6 +70,8 @@ def attention(Q, K, V, scale, valid_len=None, rows=None, want_logits=False, want
     valid keys, -inf for a row without any), and 'threads' (threads used).
     bias: optional additive term of the scaled logits, [B or 1, H or 1, Nq, Nk], uint16 (bf16 bits) or
     float32; size-1 batch / head axes are repeated; -inf switches a (query, key) pair off.
+    block_mask: optional uint8 map [B or 1, H or 1, ceil(Nq / block), ceil(Nk / block)] of the blocks of the
+    logit matrix that are kept (non-zero) or pruned (0): pruned pairs take no part.
     """
     Q = np.ascontiguousarray(Q); K = np.ascontiguousarray(K); V = np.ascontiguousarray(V)
     if Q.dtype == np.uint16:
@@ -112,11 +115,20 @@ def attention(Q, K, V, scale, valid_len=None, rows=None, want_logits=False, want
             raise ValueError("bias must be [B or 1, H or 1, Nq, Nk]")
         bias_sh = 0 if bias.shape[1] == 1 else Nq * Nk
         bias_sb = 0 if bias.shape[0] == 1 else bias.shape[1] * Nq * Nk
+    bm_sb = bm_sh = 0
+    if block_mask is not None:
+        block_mask = np.ascontiguousarray(block_mask, dtype=np.uint8)
+        tq, tk = -(-Nq // block), -(-Nk // block)
+        if block_mask.ndim != 4 or block_mask.shape[2:] != (tq, tk) or block_mask.shape[0] not in (1, B) or block_mask.shape[1] not in (1, H):
+            raise ValueError("block_mask must be [B or 1, H or 1, ceil(Nq/block), ceil(Nk/block)]")
+        bm_sh = 0 if block_mask.shape[1] == 1 else tq * tk
+        bm_sb = 0 if block_mask.shape[0] == 1 else block_mask.shape[1] * tq * tk
     used = ctypes.c_int(0)
     ptr = lambda a: None if a is None else a.ctypes.data_as(ctypes.c_void_p)
-    rc = _load().oracle_attn_rows_bias(ptr(Q), ptr(K), ptr(V), dtype, B, H, Nq, Nk, d, float(np.float32(scale)),
+    rc = _load().oracle_attn_rows_sparse(ptr(Q), ptr(K), ptr(V), dtype, B, H, Nq, Nk, d, float(np.float32(scale)),
                                        ptr(vl), 1 if causal else 0, ptr(rows), n, ptr(O), ptr(L), ptr(A), ptr(LSE),
-                                       ptr(bias), bias_dtype, bias_sb, bias_sh, int(nthreads), ctypes.byref(used))
+                                       ptr(bias), bias_dtype, bias_sb, bias_sh, ptr(block_mask), bm_sb, bm_sh, int(block),
+                                       int(nthreads), ctypes.byref(used))
     if rc != 0:
         raise ValueError("oracle_attn_rows rejected its arguments (code %d)" % rc)
     out = {"O": O, "threads": used.value}

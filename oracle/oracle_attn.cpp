@@ -25,6 +25,9 @@
 //   * additive bias (the relative-position terms of the paper's T5 / TrXL workloads, Section 6.1;
 //     the paper does not model them): a tensor [B or 1, H or 1, Nq, Nk] added to the SCALED logit
 //     before the maximum; -inf switches a pair off, a row with every pair off gives O = 0.
+//   * pruned (sparse) Logit-Attend (Section 8.2 studies randomly pruned attention): a byte map over
+//     tile x tile blocks of the logit matrix; a pruned block's pairs take no part (their logits count
+//     as -inf), a row whose every block is pruned gives O = 0.
 //   * causal mask (decoder workloads; the paper does not spell masks out): query i takes
 //     part with key j iff j <= i + (Nk - Nq), i.e. the last query sees every key and each
 //     earlier query one key fewer; combined with the key-padding mask by intersection.
@@ -65,6 +68,9 @@ struct Problem {
     const void* bias;                // additive term of the logits, or null: element (b,h,i,j) at
     int bias_dtype;                  //   b * bias_sb + h * bias_sh + i * Nk + j  (0: bf16 bits, 1: float32);
     int64_t bias_sb, bias_sh;        //   a stride of 0 repeats the same values for every batch / head
+    const uint8_t* bmask;            // pruned attention, or null: the pair (i, j) takes part iff byte
+    int64_t bmask_sb, bmask_sh;      //   b * bmask_sb + h * bmask_sh + (i / tile) * ceil(Nk / tile) + j / tile is non-zero
+    int64_t bmask_tile;              //   (tile x tile blocks of the logit matrix; strides of 0 repeat)
 };
 
 inline double elem(const void* base, int dtype, int64_t idx) {
@@ -99,6 +105,11 @@ void attend_row(const Problem& p, int64_t r, std::vector<double>& s) {
         // The bias joins the SCALED logit (it is not multiplied by scale) and takes part in the
         // maximum and the softmax like any logit; -inf switches the pair off.
         if (p.bias) s[j] += elem(p.bias, p.bias_dtype, b * p.bias_sb + (bh % p.H) * p.bias_sh + i * p.Nk + j);
+        // A pruned block takes no part: its logits count as -inf.
+        if (p.bmask) {
+            const int64_t tk = (p.Nk + p.bmask_tile - 1) / p.bmask_tile;
+            if (!p.bmask[b * p.bmask_sb + (bh % p.H) * p.bmask_sh + (i / p.bmask_tile) * tk + j / p.bmask_tile]) s[j] = -INFINITY;
+        }
     }
     if (lrow) {
         for (int64_t j = 0; j < p.Nk; ++j) lrow[j] = (j < n) ? s[j] : -INFINITY;
@@ -138,16 +149,18 @@ extern "C" {
 
 // Returns 0 on success, 1 on a bad argument.  `nthreads` <= 0 means "all hardware
 // threads"; the count actually used is written to *threads_used if non-null.
-int oracle_attn_rows_bias(const void* Q, const void* K, const void* V, int dtype,
-                          int64_t B, int64_t H, int64_t Nq, int64_t Nk, int64_t d, float scale,
-                          const int32_t* valid_len, int causal, const int64_t* rows, int64_t nrows,
-                          double* O, double* L, double* A, double* LSE,
-                          const void* bias, int bias_dtype, int64_t bias_sb, int64_t bias_sh,
-                          int nthreads, int* threads_used) {
+int oracle_attn_rows_sparse(const void* Q, const void* K, const void* V, int dtype,
+                            int64_t B, int64_t H, int64_t Nq, int64_t Nk, int64_t d, float scale,
+                            const int32_t* valid_len, int causal, const int64_t* rows, int64_t nrows,
+                            double* O, double* L, double* A, double* LSE,
+                            const void* bias, int bias_dtype, int64_t bias_sb, int64_t bias_sh,
+                            const uint8_t* bmask, int64_t bmask_sb, int64_t bmask_sh, int64_t bmask_tile,
+                            int nthreads, int* threads_used) {
     if (!Q || !K || !V || !O) return 1;
     if (B < 1 || H < 1 || Nq < 1 || Nk < 1 || d < 1) return 1;
     if (dtype != 0 && dtype != 1) return 1;
     if (bias && ((bias_dtype != 0 && bias_dtype != 1) || bias_sb < 0 || bias_sh < 0)) return 1;
+    if (bmask && (bmask_tile < 1 || bmask_sb < 0 || bmask_sh < 0)) return 1;
     const int64_t total = B * H * Nq;
     if (!rows) nrows = total;
     if (nrows < 0) return 1;
@@ -155,7 +168,7 @@ int oracle_attn_rows_bias(const void* Q, const void* K, const void* V, int dtype
     if (valid_len) for (int64_t b = 0; b < B; ++b) if (valid_len[b] < 0 || valid_len[b] > Nk) return 1;
 
     Problem p{Q, K, V, dtype, B, H, Nq, Nk, d, static_cast<double>(scale), valid_len, causal ? 1 : 0, rows, nrows, O, L, A, LSE,
-              bias, bias_dtype, bias_sb, bias_sh};
+              bias, bias_dtype, bias_sb, bias_sh, bmask, bmask_sb, bmask_sh, bmask_tile};
     int nt = nthreads > 0 ? nthreads : static_cast<int>(std::thread::hardware_concurrency());
     if (nt < 1) nt = 1;
     if (nt > nrows) nt = nrows > 0 ? static_cast<int>(nrows) : 1;
@@ -170,6 +183,16 @@ int oracle_attn_rows_bias(const void* Q, const void* K, const void* V, int dtype
     }
     for (auto& th : pool) th.join();
     return 0;
+}
+
+int oracle_attn_rows_bias(const void* Q, const void* K, const void* V, int dtype,
+                          int64_t B, int64_t H, int64_t Nq, int64_t Nk, int64_t d, float scale,
+                          const int32_t* valid_len, int causal, const int64_t* rows, int64_t nrows,
+                          double* O, double* L, double* A, double* LSE,
+                          const void* bias, int bias_dtype, int64_t bias_sb, int64_t bias_sh,
+                          int nthreads, int* threads_used) {
+    return oracle_attn_rows_sparse(Q, K, V, dtype, B, H, Nq, Nk, d, scale, valid_len, causal, rows, nrows, O, L, A, LSE,
+                                   bias, bias_dtype, bias_sb, bias_sh, nullptr, 0, 0, 1, nthreads, threads_used);
 }
 
 int oracle_attn_rows_lse(const void* Q, const void* K, const void* V, int dtype,

@@ -408,3 +408,60 @@ def test_bias_minus_infinity_is_a_mask():
     bias[0, 0, 2, :] = -np.inf
     r = oracle.attention(Q, K, V, 0.7, bias=bias, want_lse=True)
     assert np.all(r["O"][:, :, 2] == 0) and np.all(np.isneginf(r["LSE"][:, :, 2])) and np.all(np.isfinite(r["O"]))
+
+
+# ------------------------------------------------------------------------------------------------
+# Pruned (block-sparse) attention: a byte map over blocks of the logit matrix; pruned pairs take no part.
+
+def test_block_mask_is_a_minus_infinity_bias_on_the_pruned_blocks():
+    rng = np.random.default_rng(21)
+    B, H, Nq, Nk, d, blk = 2, 2, 10, 14, 4, 4
+    Q, K, V = _rand_f32(rng, B, H, Nq, d), _rand_f32(rng, B, H, Nk, d), _rand_f32(rng, B, H, Nk, d)
+    tq, tk = 3, 4
+    for shape in ((B, H), (1, H), (B, 1), (1, 1)):
+        m = (rng.random(shape + (tq, tk)) < 0.5).astype(np.uint8)
+        m[..., 1, :] = 0                                   # a block row with nothing kept
+        m[..., 0, 0] = 1
+        # the same thing as an explicit bias tensor (the bias path has its own pins)
+        full = np.repeat(np.repeat(m, blk, axis=2), blk, axis=3)[:, :, :Nq, :Nk]
+        bias = np.where(full != 0, 0.0, -np.inf).astype(np.float32)
+        a = oracle.attention(Q, K, V, 0.6, block_mask=m, block=blk, want_weights=True, want_lse=True)
+        b = oracle.attention(Q, K, V, 0.6, bias=bias, want_weights=True, want_lse=True)
+        assert np.array_equal(a["O"], b["O"]) and np.array_equal(a["A"], b["A"])
+        assert np.array_equal(a["LSE"], b["LSE"])
+        assert np.all(a["O"][:, :, 4:8] == 0) and np.all(np.isneginf(a["LSE"][:, :, 4:8]))   # rows of block row 1
+        # an independent softmax over the kept columns only
+        S = np.float64(np.float32(0.6)) * np.einsum("bhid,bhjd->bhij", Q.astype(np.float64), K.astype(np.float64))
+        S = np.where(np.broadcast_to(full, S.shape) != 0, S, -np.inf)
+        with np.errstate(invalid="ignore"):
+            W = np.exp(S - S.max(-1, keepdims=True))
+        W = np.nan_to_num(W)
+        den = W.sum(-1, keepdims=True)
+        ref = np.where(den > 0, W / np.where(den > 0, den, 1), 0) @ V.astype(np.float64)
+        assert np.abs(a["O"] - ref).max() < 1e-13
+
+
+def test_block_mask_special_cases():
+    rng = np.random.default_rng(22)
+    B, H, Nq, Nk, d, blk = 1, 2, 9, 12, 3, 4
+    Q, K, V = _rand_f32(rng, B, H, Nq, d), _rand_f32(rng, B, H, Nk, d), _rand_f32(rng, B, H, Nk, d)
+    ones = np.ones((1, 1, 3, 3), dtype=np.uint8)
+    assert np.array_equal(oracle.attention(Q, K, V, 0.5, block_mask=ones, block=blk)["O"], oracle.attention(Q, K, V, 0.5)["O"])
+    # pruning the trailing block column of every row = a key-padding mask at 8 keys = truncation
+    m = ones.copy(); m[..., 2] = 0
+    assert np.array_equal(oracle.attention(Q, K, V, 0.5, block_mask=m, block=blk)["O"],
+                          oracle.attention(Q, K, V, 0.5, valid_len=np.array([8], dtype=np.int32))["O"])
+    # the lower block triangle kept + the causal mask = the causal mask alone (Nq = Nk, blocks on the diagonal)
+    Q2 = _rand_f32(rng, B, H, 12, d)
+    tri = np.tril(np.ones((3, 3), dtype=np.uint8)).reshape(1, 1, 3, 3)
+    assert np.array_equal(oracle.attention(Q2, K, V, 0.5, block_mask=tri, block=blk, causal=True)["O"],
+                          oracle.attention(Q2, K, V, 0.5, causal=True)["O"])
+    # one kept block: the row attends exactly those keys
+    one = np.zeros((1, 1, 3, 3), dtype=np.uint8); one[0, 0, :, 1] = 1
+    got = oracle.attention(Q, K, V, 0.5, block_mask=one, block=blk)["O"]
+    assert np.abs(got - oracle.attention(Q, K[:, :, 4:8], V[:, :, 4:8], 0.5)["O"]).max() < 1e-15
+    # sampled rows see the same map
+    rows = np.array([0, 5, 13], dtype=np.int64)
+    m = (rng.random((1, 2, 3, 3)) < 0.6).astype(np.uint8); m[..., 0] = 1
+    allr = oracle.attention(Q, K, V, 0.5, block_mask=m, block=blk)["O"].reshape(-1, d)
+    assert np.array_equal(oracle.attention(Q, K, V, 0.5, block_mask=m, block=blk, rows=rows)["O"], allr[rows])
