@@ -117,6 +117,19 @@ typedef struct flat_attn_params {
                                   variants.  NULL = none.                                         */
     int bias_dtype;            /* FLAT_DTYPE_BF16 or FLAT_DTYPE_F32 (storage of `bias`)            */
     long long bias_stride_b, bias_stride_h;   /* in elements, >= 0                               */
+    const uint8_t* block_mask; /* optional device byte map for PRUNED (sparse) Logit-Attend (paper
+                                  Section 8.2 studies randomly pruned attention): one byte per
+                                  128 x 128 block of the logit matrix, [B or 1, H or 1,
+                                  ceil(Nq/128), ceil(Nk/128)], read at b * block_mask_stride_b +
+                                  h * block_mask_stride_h + tq * ceil(Nk/128) + tk.  A block whose
+                                  byte is 0 takes no part: its key tile is neither loaded nor
+                                  multiplied for that query tile (the work and the K/V traffic
+                                  shrink with the density); a query row whose every block is pruned
+                                  gives O = 0.  Combines with k_valid_len, causal and lse, not with
+                                  bias.  bf16, d in {64, 128}, Nk <= 131072; run by the one-tile
+                                  tensor-core kernel (AUTO picks it); FLAT_ERR_UNSUPPORTED otherwise.
+                                  NULL = dense.                                                   */
+    long long block_mask_stride_b, block_mask_stride_h;   /* in bytes (= elements), >= 0         */
 } flat_attn_params_t;
 
 /*

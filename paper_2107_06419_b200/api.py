@@ -42,7 +42,9 @@ class flat_attn_params_t(ctypes.Structure):
                 ("d", ctypes.c_int), ("scale", ctypes.c_float), ("dtype", ctypes.c_int),
                 ("k_valid_len", ctypes.c_void_p), ("status", ctypes.c_void_p), ("variant", ctypes.c_int),
                 ("causal", ctypes.c_int), ("lse", ctypes.c_void_p), ("bias", ctypes.c_void_p),
-                ("bias_dtype", ctypes.c_int), ("bias_stride_b", ctypes.c_longlong), ("bias_stride_h", ctypes.c_longlong)]
+                ("bias_dtype", ctypes.c_int), ("bias_stride_b", ctypes.c_longlong), ("bias_stride_h", ctypes.c_longlong),
+                ("block_mask", ctypes.c_void_p), ("block_mask_stride_b", ctypes.c_longlong),
+                ("block_mask_stride_h", ctypes.c_longlong)]
 
 
 class flat_attn_bwd_params_t(ctypes.Structure):
@@ -152,7 +154,8 @@ def _dtype_code(t) -> int:
     raise TypeError("Q/K/V/O must be bfloat16 or float32")
 
 
-def _params(Q, K, V, O, scale, k_valid_len, status, variant, host=False, causal=False, lse=None, bias=None):
+def _params(Q, K, V, O, scale, k_valid_len, status, variant, host=False, causal=False, lse=None, bias=None,
+            block_mask=None):
     B, H, Nq, d = Q.shape
     Nk = K.shape[2]
     if tuple(K.shape) != (B, H, Nk, d) or tuple(V.shape) != (B, H, Nk, d) or tuple(O.shape) != (B, H, Nq, d):
@@ -192,6 +195,17 @@ def _params(Q, K, V, O, scale, k_valid_len, status, variant, host=False, causal=
         p.bias_stride_b = 0 if bias.shape[0] == 1 else bias.shape[1] * Nq * Nk
     else:
         p.bias = None
+    if block_mask is not None:
+        tq, tk = -(-Nq // 128), -(-Nk // 128)
+        if (block_mask.dim() != 4 or tuple(block_mask.shape[2:]) != (tq, tk) or block_mask.shape[0] not in (1, B)
+                or block_mask.shape[1] not in (1, H) or not block_mask.is_cuda or not block_mask.is_contiguous()
+                or block_mask.dtype != torch.uint8):
+            raise ValueError("block_mask must be a contiguous CUDA uint8 tensor [B or 1, H or 1, ceil(Nq/128), ceil(Nk/128)]")
+        p.block_mask = block_mask.data_ptr()
+        p.block_mask_stride_h = 0 if block_mask.shape[1] == 1 else tq * tk
+        p.block_mask_stride_b = 0 if block_mask.shape[0] == 1 else block_mask.shape[1] * tq * tk
+    else:
+        p.block_mask = None
     return p
 
 
@@ -210,12 +224,15 @@ def flat_attn_fwd(Q, K, V, O, scale, stream=None):
 
 
 def flat_attn_fwd_ex(Q, K, V, O, scale, k_valid_len=None, status=None, variant=FLAT_VARIANT_AUTO, stream=None,
-                     causal=False, lse=None, bias=None):
+                     causal=False, lse=None, bias=None, block_mask=None):
     """Fused attention with dtype choice (from the tensors), key-padding mask, kernel choice and
     causal mask (query i sees keys j <= i + (Nk - Nq)); `lse` [B,H,Nq] float32 receives each row's
     log-sum-exp of the scaled logits (what the backward pass needs); `bias` [B or 1, H or 1, Nq, Nk]
-    (bfloat16 or float32) is added to the scaled logits before the softmax (-inf switches a pair off)."""
-    p = _params(Q, K, V, O, scale, k_valid_len, status, variant, causal=causal, lse=lse, bias=bias)
+    (bfloat16 or float32) is added to the scaled logits before the softmax (-inf switches a pair off);
+    `block_mask` (uint8 [B or 1, H or 1, ceil(Nq/128), ceil(Nk/128)]) prunes 128 x 128 blocks of the logit
+    matrix (0 = the block takes no part)."""
+    p = _params(Q, K, V, O, scale, k_valid_len, status, variant, causal=causal, lse=lse, bias=bias,
+                block_mask=block_mask)
     _check(_lib.flat_attn_fwd_ex(ctypes.byref(p), _stream_ptr(stream)))
     return O
 

@@ -65,9 +65,11 @@ int validate(const flat_attn_params_t* p, flat::Problem* out) {
         if (p->bias_stride_b < 0 || p->bias_stride_h < 0) return FLAT_ERR_SHAPE;
         if (reinterpret_cast<uintptr_t>(p->bias) & (p->bias_dtype == FLAT_DTYPE_F32 ? 3u : 1u)) return FLAT_ERR_ALIGN;
     }
+    if (p->block_mask && (p->block_mask_stride_b < 0 || p->block_mask_stride_h < 0)) return FLAT_ERR_SHAPE;
     *out = flat::Problem{p->Q, p->K, p->V, p->O, p->B, p->H, p->Nq, p->Nk, p->d,
                          p->scale, p->dtype, p->k_valid_len, status_or_library_word(p->status), p->causal, p->lse,
-                         p->bias, p->bias_dtype, p->bias_stride_b, p->bias_stride_h};
+                         p->bias, p->bias_dtype, p->bias_stride_b, p->bias_stride_h,
+                         p->block_mask, p->block_mask_stride_b, p->block_mask_stride_h};
     return FLAT_OK;
 }
 
@@ -118,14 +120,17 @@ int run_fused(const flat::Problem& q, int variant, cudaStream_t st) {
             if ((q.causal || q.lse) && v == FLAT_VARIANT_TC) v = FLAT_VARIANT_TC2;
             // (the bias is read by the two-tile kernel with one thread per row)
             if (q.bias) v = FLAT_VARIANT_TC2;
+            // (pruned attention runs on the one-tile kernel: a CTA walks the list of its query tile's kept key tiles)
+            if (q.block_mask) v = FLAT_VARIANT_TC2_SINGLE;
         }
     }
     if (q.causal && v == FLAT_VARIANT_TC) return FLAT_ERR_UNSUPPORTED;
     if (q.lse && (v == FLAT_VARIANT_TC || v == FLAT_VARIANT_RGRAN)) return FLAT_ERR_UNSUPPORTED;
     if (q.bias && v != FLAT_VARIANT_TC2 && v != FLAT_VARIANT_SIMT) return FLAT_ERR_UNSUPPORTED;
+    if (q.block_mask && (v != FLAT_VARIANT_TC2_SINGLE || q.bias || !tc_applies(q) || q.Nk > 131072)) return FLAT_ERR_UNSUPPORTED;
     g_last_variant = v;
     if (v == FLAT_VARIANT_TC2_SINGLE) {
-        if (!tc_applies(q) || q.d != 64) return FLAT_ERR_UNSUPPORTED;
+        if (!tc_applies(q) || (q.d != 64 && !q.block_mask)) return FLAT_ERR_UNSUPPORTED;
         return flat::launch_fused_tc2_single(q, st);
     }
     if (v == FLAT_VARIANT_TC3) {
@@ -181,7 +186,7 @@ int flat_attn_fwd_ex(const flat_attn_params_t* p, void* stream) {
 
 int flat_attn_fwd(const void* Q, const void* K, const void* V, void* O, int B, int H, int Nq, int Nk, int d,
                   float scale, void* stream) {
-    flat_attn_params_t p{Q, K, V, O, B, H, Nq, Nk, d, scale, FLAT_DTYPE_BF16, nullptr, nullptr, FLAT_VARIANT_AUTO, 0, nullptr, nullptr, 0, 0, 0};
+    flat_attn_params_t p{Q, K, V, O, B, H, Nq, Nk, d, scale, FLAT_DTYPE_BF16, nullptr, nullptr, FLAT_VARIANT_AUTO, 0, nullptr, nullptr, 0, 0, 0, nullptr, 0, 0};
     return flat_attn_fwd_ex(&p, stream);
 }
 
@@ -190,7 +195,7 @@ int flat_attn_naive_fwd_ex(const flat_attn_params_t* p, void* L, void* A, void* 
     const int rc = validate(p, &q);
     if (rc != FLAT_OK) return rc;
     if (!L || !A) return FLAT_ERR_NULL;
-    if (q.bias) return FLAT_ERR_UNSUPPORTED;                 // (the baseline has no bias operand)
+    if (q.bias || q.block_mask) return FLAT_ERR_UNSUPPORTED; // (the baseline has no bias operand and no pruning map)
     if (!aligned16(L) || !aligned16(A)) return FLAT_ERR_ALIGN;
     // (the row softmax runs one CTA per row of L: the row count is a grid dimension)
     if (static_cast<int64_t>(q.B) * q.H * q.Nq > 0x7fffffffLL) return FLAT_ERR_SHAPE;
@@ -201,7 +206,7 @@ int flat_attn_naive_fwd_ex(const flat_attn_params_t* p, void* L, void* A, void* 
 
 int flat_attn_naive_fwd(const void* Q, const void* K, const void* V, void* O, void* L, void* A, int B, int H,
                         int Nq, int Nk, int d, float scale, void* stream) {
-    flat_attn_params_t p{Q, K, V, O, B, H, Nq, Nk, d, scale, FLAT_DTYPE_BF16, nullptr, nullptr, FLAT_VARIANT_AUTO, 0, nullptr, nullptr, 0, 0, 0};
+    flat_attn_params_t p{Q, K, V, O, B, H, Nq, Nk, d, scale, FLAT_DTYPE_BF16, nullptr, nullptr, FLAT_VARIANT_AUTO, 0, nullptr, nullptr, 0, 0, 0, nullptr, 0, 0};
     return flat_attn_naive_fwd_ex(&p, L, A, stream);
 }
 
@@ -211,7 +216,7 @@ int flat_attn_bwd_ex(const flat_attn_bwd_params_t* p, void* stream) {
         return FLAT_ERR_NULL;
     // sizes, scale, masks and the alignment of Q, K, V, O: the forward's rules
     flat_attn_params_t f{p->Q, p->K, p->V, const_cast<void*>(p->O), p->B, p->H, p->Nq, p->Nk, p->d, p->scale,
-                         FLAT_DTYPE_BF16, p->k_valid_len, p->status, FLAT_VARIANT_AUTO, p->causal, nullptr, nullptr, 0, 0, 0};
+                         FLAT_DTYPE_BF16, p->k_valid_len, p->status, FLAT_VARIANT_AUTO, p->causal, nullptr, nullptr, 0, 0, 0, nullptr, 0, 0};
     flat::Problem q;
     const int rc = validate(&f, &q);
     if (rc != FLAT_OK) return rc;
@@ -394,7 +399,7 @@ int flat_attn_layer_fwd(const void* X, const void* Wqkv, const void* Wo, void* Y
                         int B, int N, int H, int d, int Dm, float scale, int causal, int32_t* status, void* stream) {
     if (!X || !Wqkv || !Wo || !Y || !Q || !K || !V || !O) return FLAT_ERR_NULL;
     // validate all three steps before anything is launched
-    flat_attn_params_t p{Q, K, V, O, B, H, N, N, d, scale, FLAT_DTYPE_BF16, nullptr, status, FLAT_VARIANT_AUTO, causal, nullptr, nullptr, 0, 0, 0};
+    flat_attn_params_t p{Q, K, V, O, B, H, N, N, d, scale, FLAT_DTYPE_BF16, nullptr, status, FLAT_VARIANT_AUTO, causal, nullptr, nullptr, 0, 0, 0, nullptr, 0, 0};
     flat::Problem q;
     int rc = validate(&p, &q);
     if (rc != FLAT_OK) return rc;

@@ -23,6 +23,10 @@ struct Problem {
     const void* bias;
     int bias_dtype;                  // FLAT_DTYPE_*
     long long bias_sb, bias_sh;      // strides in elements; 0 = the same values for every batch / head
+    // optional pruning map over 128 x 128 blocks of the logit matrix: byte (b,h,tq,tk) at
+    // b * bmask_sb + h * bmask_sh + tq * ceil(Nk / 128) + tk; 0 = the block takes no part
+    const uint8_t* block_mask;
+    long long bmask_sb, bmask_sh;
 };
 
 // What a kernel needs to read the bias (passed by value).
@@ -63,7 +67,7 @@ int launch_fused_simt(const Problem& p, cudaStream_t st);
 int launch_naive(const Problem& p, void* L, void* A, cudaStream_t st);
 int launch_fused_tc(const Problem& p, cudaStream_t st);
 int launch_fused_tc2(const Problem& p, cudaStream_t st);      // (also the tensor-core kernel for calls with a bias)
-int launch_fused_tc2_single(const Problem& p, cudaStream_t st);
+int launch_fused_tc2_single(const Problem& p, cudaStream_t st);   // (d = 64; with a block mask also d = 128)
 int launch_fused_tc3(const Problem& p, cudaStream_t st);
 bool rgran_applies(const Problem& p);              // bf16, d = 64, Nk <= 512
 int launch_fused_rgran(const Problem& p, cudaStream_t st);

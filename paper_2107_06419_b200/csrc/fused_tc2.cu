@@ -167,14 +167,22 @@ __device__ __forceinline__ float exp_store(const uint32_t (&s)[128], float scale
 // BIAS: a separate instantiation that adds a bias tensor to the scaled logits (dense batches): the softmax
 // thread fetches its row's 128 values of the step straight from device memory -- a bf16 bias adds
 // 2 B H Nq Nk bytes of traffic, four times |Q|+|K|+|V|+|O| on a 4096 x 4096, d = 64 problem.
-template <int D, int NT, bool VL = false, bool BIAS = false>
+// SPARSE (one tile per CTA): pruned attention.  A byte map over 128 x 128 blocks of the logit matrix says
+// which key tiles the CTA's query tile attends; the CTA compacts its row of the map into a list in shared
+// memory and every role walks that list instead of 0, 1, 2, ...: pruned key tiles are neither loaded nor
+// multiplied.
+template <int D, int NT, bool VL = false, bool BIAS = false, bool SPARSE = false>
 __global__ void __launch_bounds__(128 * NT + 128, NT == 1 ? 2 : 1)
 fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                  const __grid_constant__ CUtensorMap tmV, __nv_bfloat16* __restrict__ O, int H, int Nq, int Nk,
                  float scale_log2e, const int32_t* __restrict__ valid_len, int coff, int32_t* status,
                  const int32_t* __restrict__ cu_q = nullptr, const int32_t* __restrict__ cu_k = nullptr,
-                 float* __restrict__ lse = nullptr, BiasArg bias = BiasArg{nullptr, 0, 0, 0, 0}) {
+                 float* __restrict__ lse = nullptr, BiasArg bias = BiasArg{nullptr, 0, 0, 0, 0},
+                 const uint8_t* __restrict__ block_mask = nullptr, long long bmask_sb = 0, long long bmask_sh = 0) {
     using LY = L2<D, NT>;
+    static_assert(!SPARSE || (NT == 1 && !VL && !BIAS), "the pruning map is read by the one-tile dense kernel");
+    __shared__ uint16_t tile_list[SPARSE ? 1024 : 1];    // the kept key tiles of this query tile, ascending
+    __shared__ int tile_count;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* Qs = base;                                  // NT tiles
@@ -204,7 +212,22 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         const long long lim = static_cast<long long>(row0) + NT * BM + coff;
         if (lim < n) n = lim < 0 ? 0 : static_cast<int>(lim);
     }
-    const int ntiles = (n + BN - 1) / BN;
+    int ntiles = (n + BN - 1) / BN;
+    if (SPARSE && (threadIdx.x >> 5) == 1) {
+        // warp 1 compacts the map's row (tiles below the key limit n only) into the list
+        const uint8_t* mrow = block_mask + static_cast<long long>(bh / H) * bmask_sb + static_cast<long long>(bh % H) * bmask_sh +
+                              static_cast<long long>(blockIdx.x) * ((Nk + BN - 1) / BN);
+        const int ln = threadIdx.x & 31;
+        int count = 0;
+        for (int base = 0; base < ntiles; base += 32) {
+            const int jj = base + ln;
+            const bool keep = jj < ntiles && mrow[jj] != 0;
+            const unsigned m = __ballot_sync(0xffffffffu, keep);
+            if (keep) tile_list[count + __popc(m & ((1u << ln) - 1u))] = static_cast<uint16_t>(jj);
+            count += __popc(m);
+        }
+        if (ln == 0) tile_count = count;
+    }
 
     if (threadIdx.x == LY::SOFT_WARPS * 32) {
         for (int i = 0; i < LY::NUM_BARS; ++i) {
@@ -220,6 +243,9 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
+    if (SPARSE) ntiles = tile_count;
+    // key tile of step j: the j-th kept one under a pruning map, else j itself
+    auto tile_of = [&](int j) -> int { return SPARSE ? static_cast<int>(tile_list[j]) : j; };
 
     if (warp >= LY::SOFT_WARPS) {
       if (NT == 2) asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
@@ -237,7 +263,7 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                 mbar_arrive_expect_tx(&bars[LY::K_FULL + s], LY::KV_BYTES);
 #pragma unroll
                 for (int c = 0; c < D / 64; ++c)
-                    tma_load_3d(Ks + s * LY::KV_BYTES + c * BN * 128, &tmK, &bars[LY::K_FULL + s], c * 64, VL ? head : j * BN,
+                    tma_load_3d(Ks + s * LY::KV_BYTES + c * BN * 128, &tmK, &bars[LY::K_FULL + s], c * 64, VL ? head : tile_of(j) * BN,
                                 VL ? k_tok0 + j * BN : bh);
                 k_issued = j + 1;
             };
@@ -248,7 +274,7 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                 mbar_arrive_expect_tx(&bars[LY::V_FULL + s], LY::KV_BYTES);
 #pragma unroll
                 for (int c = 0; c < D / 64; ++c)
-                    tma_load_3d(Vs + s * LY::KV_BYTES + c * BN * 128, &tmV, &bars[LY::V_FULL + s], c * 64, VL ? head : j * BN,
+                    tma_load_3d(Vs + s * LY::KV_BYTES + c * BN * 128, &tmV, &bars[LY::V_FULL + s], c * 64, VL ? head : tile_of(j) * BN,
                                 VL ? k_tok0 + j * BN : bh);
                 v_issued = j + 1;
             };
@@ -391,7 +417,7 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             __syncwarp();
             if (lane == 0) mbar_arrive(&bars[LY::S_FREE + t]);   // S_t may be overwritten (d = 64: by the next S_t)
 
-            const int col0 = j * BN;
+            const int col0 = tile_of(j) * BN;
             if (BIAS) {
                 // x = s * scale * log2(e) + bias * log2(e); a row past the end and columns past Nk read nothing
                 const long long at = static_cast<long long>(bh / H) * bias.sb + static_cast<long long>(bh % H) * bias.sh +
@@ -573,6 +599,18 @@ int launch_tc2_d(const Problem& p, cudaStream_t st) {
         !make_map(&tmV, p.V, BH, p.Nk, D, BN))
         return FLAT_ERR_CUDA;
     dim3 grid((p.Nq + NT * BM - 1) / (NT * BM), BH);
+    if (p.block_mask) {
+        if constexpr (NT == 1) {
+            if (!ensure_dynamic_smem<fused_tc2_kernel<D, NT, false, false, true>>(LY::SMEM_BYTES)) return FLAT_ERR_CUDA;
+            fused_tc2_kernel<D, NT, false, false, true><<<grid, LY::THREADS, LY::SMEM_BYTES, st>>>(
+                tmQ, tmK, tmV, static_cast<__nv_bfloat16*>(p.O), p.H, p.Nq, p.Nk, p.scale * 1.4426950408889634f,
+                p.k_valid_len, p.causal ? p.Nk - p.Nq : (1 << 30), p.status, nullptr, nullptr, p.lse,
+                BiasArg{nullptr, 0, 0, 0, 0}, p.block_mask, p.bmask_sb, p.bmask_sh);
+            return cudaGetLastError() == cudaSuccess ? FLAT_OK : FLAT_ERR_CUDA;
+        } else {
+            return FLAT_ERR_UNSUPPORTED;
+        }
+    }
     if (p.bias) {
         if constexpr (NT == 2) {
             if (!ensure_dynamic_smem<fused_tc2_kernel<D, NT, false, true>>(LY::SMEM_BYTES)) return FLAT_ERR_CUDA;
@@ -589,7 +627,7 @@ int launch_tc2_d(const Problem& p, cudaStream_t st) {
     kern<<<grid, LY::THREADS, LY::SMEM_BYTES, st>>>(tmQ, tmK, tmV, static_cast<__nv_bfloat16*>(p.O), p.H, p.Nq,
                                                     p.Nk, p.scale * 1.4426950408889634f, p.k_valid_len,
                                                     p.causal ? p.Nk - p.Nq : (1 << 30), p.status, nullptr, nullptr, p.lse,
-                                                    BiasArg{nullptr, 0, 0, 0, 0});
+                                                    BiasArg{nullptr, 0, 0, 0, 0}, nullptr, 0, 0);
     return cudaGetLastError() == cudaSuccess ? FLAT_OK : FLAT_ERR_CUDA;
 }
 
@@ -657,6 +695,7 @@ int launch_fused_tc2(const Problem& p, cudaStream_t st) {
 int launch_fused_tc2_single(const Problem& p, cudaStream_t st) {
     if (p.dtype != FLAT_DTYPE_BF16) return FLAT_ERR_UNSUPPORTED;
     if (p.d == 64) return launch_tc2_d<64, 1>(p, st);
+    if (p.d == 128 && p.block_mask) return launch_tc2_d<128, 1>(p, st);   // (one CTA per SM: the pruned path only)
     return FLAT_ERR_UNSUPPORTED;
 }
 

@@ -57,7 +57,7 @@ extern "C" int flat_attn_naive_fwd_static(const void* Q, const void* K, const vo
     // Then the remaining argument rules (pointers, d, alignment, scale), with stand-ins for L and A,
     // so that a bad argument is reported as such before the device is looked at.
     {
-        flat_attn_params_t chk{Q, K, V, O, B, H, Nq, Nk, d, scale, FLAT_DTYPE_BF16, nullptr, nullptr, FLAT_VARIANT_AUTO, 0, nullptr, nullptr, 0, 0, 0};
+        flat_attn_params_t chk{Q, K, V, O, B, H, Nq, Nk, d, scale, FLAT_DTYPE_BF16, nullptr, nullptr, FLAT_VARIANT_AUTO, 0, nullptr, nullptr, 0, 0, 0, nullptr, 0, 0};
         const int rc = flat::check_params(&chk);
         if (rc != FLAT_OK) return rc;
     }
