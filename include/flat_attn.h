@@ -71,9 +71,13 @@ enum {
     FLAT_VARIANT_TC3 = 5,      /* two tiles per CTA, the softmax of every row split over two
                                   threads (sixteen softmax warps), logit tiles computed three
                                   tile-steps ahead in rotating TMEM buffers: bf16, d = 64 only */
-    FLAT_VARIANT_RGRAN = 6     /* the paper's row-granularity dataflow taken literally: the whole
+    FLAT_VARIANT_RGRAN = 6,    /* the paper's row-granularity dataflow taken literally: the whole
                                   row of logits of a 128-row tile stays on chip (TMEM), two-pass
                                   softmax over complete rows: bf16, d = 64, Nk <= 512 only      */
+    FLAT_VARIANT_TF32 = 7      /* fp32 tensors on the tensor cores: every operand split into a tf32
+                                  head and an fp32 remainder, each contraction three tf32 products,
+                                  running sums in fp32 registers: fp32, d = 64, no bias, no
+                                  pruning map (what AUTO picks there)                            */
 };
 
 typedef struct flat_attn_params {

@@ -9,7 +9,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libflat_attn.so")
-SOURCES = ["flat_attn_api.cu", "simt_kernels.cu", "fused_tc.cu", "fused_tc2.cu", "fused_tc3.cu", "fused_rgran.cu", "proj_gemm.cu", "naive_tc.cu", "naive_static.cu", "bwd_tc.cu", "layernorm.cu"]
+SOURCES = ["flat_attn_api.cu", "simt_kernels.cu", "fused_tc.cu", "fused_tc2.cu", "fused_tc3.cu", "fused_rgran.cu", "proj_gemm.cu", "naive_tc.cu", "naive_static.cu", "bwd_tc.cu", "layernorm.cu", "fused_tf32.cu"]
 HEADERS = ["flat_internal.cuh", "ptx_sm100.cuh", "tc_common.cuh", os.path.join("..", "..", "include", "flat_attn.h")]
 
 

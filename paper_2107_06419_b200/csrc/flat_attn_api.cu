@@ -54,7 +54,7 @@ int validate(const flat_attn_params_t* p, flat::Problem* out) {
     if (bh * static_cast<int64_t>(p->Nq > p->Nk ? p->Nq : p->Nk) > lim / p->d) return FLAT_ERR_SHAPE;
     if (p->dtype != FLAT_DTYPE_BF16 && p->dtype != FLAT_DTYPE_F32) return FLAT_ERR_UNSUPPORTED;
     if (p->d != 16 && p->d != 32 && p->d != 64 && p->d != 128) return FLAT_ERR_UNSUPPORTED;
-    if (p->variant < FLAT_VARIANT_AUTO || p->variant > FLAT_VARIANT_RGRAN) return FLAT_ERR_UNSUPPORTED;
+    if (p->variant < FLAT_VARIANT_AUTO || p->variant > FLAT_VARIANT_TF32) return FLAT_ERR_UNSUPPORTED;
     if (!aligned16(p->Q) || !aligned16(p->K) || !aligned16(p->V) || !aligned16(p->O)) return FLAT_ERR_ALIGN;
     if (p->k_valid_len && (reinterpret_cast<uintptr_t>(p->k_valid_len) & 3u)) return FLAT_ERR_ALIGN;
     if (p->status && (reinterpret_cast<uintptr_t>(p->status) & 3u)) return FLAT_ERR_ALIGN;
@@ -92,7 +92,8 @@ int run_fused(const flat::Problem& q, int variant, cudaStream_t st) {
     int v = variant;
     if (v == FLAT_VARIANT_AUTO) {
         if (!tc_applies(q)) {
-            v = FLAT_VARIANT_SIMT;
+            // fp32 tensors: the split-tf32 tensor-core kernel where it applies, else the FFMA kernel
+            v = flat::tf32_applies(q) ? FLAT_VARIANT_TF32 : FLAT_VARIANT_SIMT;
         } else {
             // Two-tile CTAs (256 query rows) once they fill the SMs; otherwise 128-row CTAs, which
             // give twice as many CTAs for small problems.  At d = 64 the two-tile kernel is the one
@@ -127,6 +128,7 @@ int run_fused(const flat::Problem& q, int variant, cudaStream_t st) {
     if (q.causal && v == FLAT_VARIANT_TC) return FLAT_ERR_UNSUPPORTED;
     if (q.lse && (v == FLAT_VARIANT_TC || v == FLAT_VARIANT_RGRAN)) return FLAT_ERR_UNSUPPORTED;
     if (q.bias && v != FLAT_VARIANT_TC2 && v != FLAT_VARIANT_SIMT) return FLAT_ERR_UNSUPPORTED;
+    if (v == FLAT_VARIANT_TF32 && !flat::tf32_applies(q)) return FLAT_ERR_UNSUPPORTED;
     if (q.block_mask && (v != FLAT_VARIANT_TC2_SINGLE || q.bias || !tc_applies(q) || q.Nk > 131072)) return FLAT_ERR_UNSUPPORTED;
     g_last_variant = v;
     if (v == FLAT_VARIANT_TC2_SINGLE) {
@@ -137,6 +139,7 @@ int run_fused(const flat::Problem& q, int variant, cudaStream_t st) {
         if (!tc_applies(q) || q.d != 64) return FLAT_ERR_UNSUPPORTED;
         return flat::launch_fused_tc3(q, st);
     }
+    if (v == FLAT_VARIANT_TF32) return flat::launch_fused_tf32(q, st);
     if (v == FLAT_VARIANT_RGRAN) return flat::launch_fused_rgran(q, st);   // (checks its own conditions)
     if (v == FLAT_VARIANT_TC || v == FLAT_VARIANT_TC2) {
         if (!tc_applies(q)) return FLAT_ERR_UNSUPPORTED;

@@ -69,6 +69,8 @@ int launch_fused_tc(const Problem& p, cudaStream_t st);
 int launch_fused_tc2(const Problem& p, cudaStream_t st);      // (also the tensor-core kernel for calls with a bias)
 int launch_fused_tc2_single(const Problem& p, cudaStream_t st);   // (d = 64; with a block mask also d = 128)
 int launch_fused_tc3(const Problem& p, cudaStream_t st);
+bool tf32_applies(const Problem& p);               // fp32, d = 64, no bias, no pruning map
+int launch_fused_tf32(const Problem& p, cudaStream_t st);     // fp32 tensors through split tf32 products
 bool rgran_applies(const Problem& p);              // bf16, d = 64, Nk <= 512
 int launch_fused_rgran(const Problem& p, cudaStream_t st);
 // Packed variable-length batches (bf16; fused_tc3: d = 64, fused_tc2: d = 128): Q, O [total_q, H, d], K, V [total_k, H, d].
