@@ -32,10 +32,12 @@ METRIC = "fused attention TFLOP/s"
 UNIT = "TFLOP/s"
 DEFAULT_WORKLOAD = "c2_bert_large_4k"
 OTHER_WORKLOADS = ["c1_bert_base_512", "c3_16k", "c4_64k_d128", "c5_cross_masked"]
+FP32_WORKLOAD = "c3_16k"             # the configuration the fp32 path is timed on (widened to fp32 tensors)
 L2_FLUSH_BELOW = 256 << 20          # workloads smaller than this get an L2 flush before every timed launch
 # FLAT_VARIANT_* (as reported by the library after a call) -> the kernel that variant launches
 KERNEL_OF_VARIANT = {1: "fused_simt_kernel", 2: "fused_tc_kernel", 3: "fused_tc2_kernel<2 tiles>",
-                     4: "fused_tc2_kernel<1 tile>", 5: "fused_tc3_kernel", 6: "fused_rgran_kernel"}
+                     4: "fused_tc2_kernel<1 tile>", 5: "fused_tc3_kernel", 6: "fused_rgran_kernel", 7: "fused_tf32_kernel"}
+TF32_OVER_BF16 = 1.1 / 2.25          # nominal dense tensor peaks: the tf32 roofline is the measured bf16 peak times this
 
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel from ncu
 # captures, with the capture they come from; a (kernel, workload) pair without a capture reports null.
@@ -404,6 +406,7 @@ def main():
             torch.cuda.empty_cache()
             out["workloads"] = [run_other(bench, torch, api, inputs.WORKLOADS[n], seed, args, peaks, dev)
                                 for n in OTHER_WORKLOADS if n != w.name]
+            out["fp32"] = run_fp32(bench, torch, api, inputs.WORKLOADS[FP32_WORKLOAD], seed, args, peaks, dev)
         print(json.dumps(out))
     if world > 1:
         dist.destroy_process_group()
@@ -469,6 +472,43 @@ def run_backward(bench, torch, api, w, d, data, seed, args, peaks):
             par[name] = {"max_rel_to_max": float(err.max() / np.abs(ref[name]).max()),
                          "mean_rel_to_mean": float(err.mean() / np.abs(ref[name]).mean())}
         e["parity_on_sample"] = {"heads": [int(h) for h in heads], **par}
+    return e
+
+
+def run_fp32(bench, torch, api, w, seed, args, peaks, dev):
+    """The fp32 path on one configuration widened to fp32 tensors (the same seeded values, exactly representable):
+    every contraction runs as three tf32 products, so the kernel executes 3 x the metric's FLOP on the tensor
+    cores; `frac` is the metric's FLOP rate over the tf32 peak, `frac_executed` counts the three products."""
+    time.sleep(1.0)
+    data, host, d = bench.load(w, seed)
+    Q, K, V = d["Q"].float(), d["K"].float(), d["V"].float()
+    O = torch.full(Q.shape, float("nan"), dtype=torch.float32, device=dev)
+    del host
+    d["Q"] = d["K"] = d["V"] = d["O"] = None
+    step = lambda: api.flat_attn_fwd_ex(Q, K, V, O, w.scale, k_valid_len=d["vl"], status=d["status"])
+    for _ in range(3):
+        step()
+    kernel = KERNEL_OF_VARIANT.get(api.flat_attn_last_variant(), "?")
+    steps = int(max(3, min(args.steps, 5)))
+    sampler = ClockSampler(dev.index).start()
+    total_ms, per = bench.timed(step, steps, flush=False)
+    clocks = sampler.stop()
+    assert int(d["status"].item()) == 0
+    ms = float(np.mean(per))
+    val = float(w.flops) / (ms * 1e-3) / 1e12
+    peak = peaks["bf16_tflops"] * TF32_OVER_BF16
+    cfg = workload_config(w)
+    cfg["inputs"] = "the workload's seeded bf16 values widened to fp32"
+    cfg["l2"] = "inputs (%d MiB) larger than the 126 MB L2; no flush between steps" % (2 * w.qkvo_bytes() >> 20)
+    e = {"workload": w.name + " as fp32", "config": cfg, "dtype": "f32 (3 x tf32 products, fp32 sums)",
+         "kernel": kernel, "steps": steps, "ms": ms, "ms_min": float(np.min(per)), "value": val, "unit": UNIT,
+         "peak": peak, "peak_source": "measured bf16 peak x nominal tf32/bf16 ratio", "frac": val / peak,
+         "frac_executed": 3.0 * val / peak, "clocks": clocks}
+    if not args.no_cpu_baseline:
+        _, e["parity_on_sample"] = parity_on_sample(torch, w, data, O, dev, per_head=8)
+        e["parity_on_sample"]["bar_max_abs"] = 1e-4
+    del data, d, Q, K, V, O
+    torch.cuda.empty_cache()
     return e
 
 

@@ -4,7 +4,8 @@
 
 CASE: fused | fused_lse | naive | backward | fp32 | bias | layernorm | layer.  The workload is one of
 `inputs.WORKLOADS` (default p_4k_small, a quarter of c2: inputs larger than L2, a few hundred MB on the
-device); inputs are the seeded generator's.  Prints the mean launch time from CUDA events.
+device); inputs are the seeded generator's.  Prints the mean launch time from CUDA events.  `fp32` runs the
+split-tf32 tensor-core kernel at d = 64 (`--variant 1`: the FFMA kernel).
 """
 from __future__ import annotations
 
@@ -52,7 +53,7 @@ def main():
     elif args.case == "fp32":
         Qf, Kf, Vf = Q.float(), K.float(), V.float()
         Of = torch.empty_like(Qf)
-        step = lambda: api.flat_attn_fwd_ex(Qf, Kf, Vf, Of, w.scale, k_valid_len=vl, status=status)
+        step = lambda: api.flat_attn_fwd_ex(Qf, Kf, Vf, Of, w.scale, k_valid_len=vl, status=status, variant=args.variant)
     elif args.case == "bias":
         bias = t(inputs.f32_to_bf16_bits(inputs.normal_f32(inputs.DEFAULT_SEED, 6, 0, w.H * w.Nq * w.Nk)).reshape(1, w.H, w.Nq, w.Nk))
         step = lambda: api.flat_attn_fwd_ex(Q, K, V, O, w.scale, k_valid_len=vl, status=status, bias=bias)
