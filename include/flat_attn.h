@@ -74,10 +74,16 @@ enum {
     FLAT_VARIANT_RGRAN = 6,    /* the paper's row-granularity dataflow taken literally: the whole
                                   row of logits of a 128-row tile stays on chip (TMEM), two-pass
                                   softmax over complete rows: bf16, d = 64, Nk <= 512 only      */
-    FLAT_VARIANT_TF32 = 7      /* fp32 tensors on the tensor cores: every operand split into a tf32
+    FLAT_VARIANT_TF32 = 7,     /* fp32 tensors on the tensor cores: every operand split into a tf32
                                   head and an fp32 remainder, each contraction three tf32 products,
                                   running sums in fp32 registers: fp32, d = 64, no bias, no
                                   pruning map (what AUTO picks there)                            */
+    FLAT_VARIANT_TC2_SPLIT2 = 8, /* TC2_SINGLE with the keys of every query tile split over a cluster
+                                  of two CTAs, whose partial softmaxes are merged through
+                                  distributed shared memory: bf16, d = 64, no bias, no pruning map;
+                                  what AUTO picks for launches that would leave most SMs empty   */
+    FLAT_VARIANT_TC2_SPLIT4 = 9, /* the same over a cluster of four CTAs                           */
+    FLAT_VARIANT_TC2_SPLIT8 = 10 /* the same over a cluster of eight CTAs                          */
 };
 
 typedef struct flat_attn_params {

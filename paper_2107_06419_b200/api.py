@@ -27,6 +27,7 @@ FLAT_VARIANT_AUTO, FLAT_VARIANT_SIMT, FLAT_VARIANT_TC, FLAT_VARIANT_TC2, FLAT_VA
 FLAT_VARIANT_TC3 = 5
 FLAT_VARIANT_RGRAN = 6
 FLAT_VARIANT_TF32 = 7
+FLAT_VARIANT_TC2_SPLIT2, FLAT_VARIANT_TC2_SPLIT4, FLAT_VARIANT_TC2_SPLIT8 = 8, 9, 10
 
 EXPORTS = ["flat_attn_fwd", "flat_attn_fwd_ex", "flat_attn_naive_fwd", "flat_attn_naive_fwd_ex",
            "flat_attn_naive_fwd_static", "flat_attn_selftest_wait_timeout", "flat_attn_selftest_exp2_poly",

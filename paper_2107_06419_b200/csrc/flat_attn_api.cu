@@ -54,7 +54,7 @@ int validate(const flat_attn_params_t* p, flat::Problem* out) {
     if (bh * static_cast<int64_t>(p->Nq > p->Nk ? p->Nq : p->Nk) > lim / p->d) return FLAT_ERR_SHAPE;
     if (p->dtype != FLAT_DTYPE_BF16 && p->dtype != FLAT_DTYPE_F32) return FLAT_ERR_UNSUPPORTED;
     if (p->d != 16 && p->d != 32 && p->d != 64 && p->d != 128) return FLAT_ERR_UNSUPPORTED;
-    if (p->variant < FLAT_VARIANT_AUTO || p->variant > FLAT_VARIANT_TF32) return FLAT_ERR_UNSUPPORTED;
+    if (p->variant < FLAT_VARIANT_AUTO || p->variant > FLAT_VARIANT_TC2_SPLIT8) return FLAT_ERR_UNSUPPORTED;
     if (!aligned16(p->Q) || !aligned16(p->K) || !aligned16(p->V) || !aligned16(p->O)) return FLAT_ERR_ALIGN;
     if (p->k_valid_len && (reinterpret_cast<uintptr_t>(p->k_valid_len) & 3u)) return FLAT_ERR_ALIGN;
     if (p->status && (reinterpret_cast<uintptr_t>(p->status) & 3u)) return FLAT_ERR_ALIGN;
@@ -123,11 +123,31 @@ int run_fused(const flat::Problem& q, int variant, cudaStream_t st) {
             if (q.bias) v = FLAT_VARIANT_TC2;
             // (pruned attention runs on the one-tile kernel: a CTA walks the list of its query tile's kept key tiles)
             if (q.block_mask) v = FLAT_VARIANT_TC2_SINGLE;
+            // A launch of single-tile CTAs that would leave most SMs empty splits the keys of every query tile
+            // over a cluster of 8, 4 or 2 CTAs: the per-CTA chain of key steps, which is what such a launch waits
+            // for, gets that much shorter at the price of one exchange through distributed shared memory (1-2 us).
+            // The largest split that still fits the GPU at two CTAs per SM and leaves every CTA two key steps
+            // (one is enough while every CTA gets an SM of its own).
+            if (v == FLAT_VARIANT_TC2_SINGLE && q.d == 64 && !q.block_mask && !q.bias) {
+                const int64_t ctas1 = static_cast<int64_t>((q.Nq + 127) / 128) * q.B * q.H;
+                const int key_tiles = (q.Nk + 127) / 128;
+                for (int cs = 8; cs >= 2; cs /= 2) {
+                    if (ctas1 * cs > 7 * sms / 4) continue;
+                    if (key_tiles < (ctas1 * cs <= sms ? cs : 2 * cs)) continue;
+                    v = cs == 8 ? FLAT_VARIANT_TC2_SPLIT8 : cs == 4 ? FLAT_VARIANT_TC2_SPLIT4 : FLAT_VARIANT_TC2_SPLIT2;
+                    break;
+                }
+            }
         }
     }
     if (q.causal && v == FLAT_VARIANT_TC) return FLAT_ERR_UNSUPPORTED;
     if (q.lse && (v == FLAT_VARIANT_TC || v == FLAT_VARIANT_RGRAN)) return FLAT_ERR_UNSUPPORTED;
     if (q.bias && v != FLAT_VARIANT_TC2 && v != FLAT_VARIANT_SIMT) return FLAT_ERR_UNSUPPORTED;
+    if (v == FLAT_VARIANT_TC2_SPLIT2 || v == FLAT_VARIANT_TC2_SPLIT4 || v == FLAT_VARIANT_TC2_SPLIT8) {
+        if (!tc_applies(q) || q.d != 64 || q.block_mask) return FLAT_ERR_UNSUPPORTED;
+        g_last_variant = v;
+        return flat::launch_fused_tc2_single(q, st, v == FLAT_VARIANT_TC2_SPLIT2 ? 2 : v == FLAT_VARIANT_TC2_SPLIT4 ? 4 : 8);
+    }
     if (v == FLAT_VARIANT_TF32 && !flat::tf32_applies(q)) return FLAT_ERR_UNSUPPORTED;
     if (q.block_mask && (v != FLAT_VARIANT_TC2_SINGLE || q.bias || !tc_applies(q) || q.Nk > 131072)) return FLAT_ERR_UNSUPPORTED;
     g_last_variant = v;

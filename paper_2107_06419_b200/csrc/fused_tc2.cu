@@ -29,6 +29,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <type_traits>
+
 #include "flat_internal.cuh"
 #include "ptx_sm100.cuh"
 #include "tc_common.cuh"
@@ -45,6 +47,7 @@ constexpr int BM = 128;              // rows per query tile (two tiles per CTA)
 constexpr int BN = 128;              // keys per step
 constexpr int PASS_AT_CHUNK = 3;                // the other tile gets its turn once this chunk's ex2 are issued
 constexpr int POLY_LANE = 3;                    // element index mod 4 that uses ex2_poly; -1 = none
+constexpr int MERGE_VECS = 17;                   // (key split) 16-byte vectors per row of a partial result: 64 outputs, then (m, l)
 constexpr float OVERFLOW_SUM = 1.0995116e12f;   // 2^40: a tile row sum beyond this means m_ref is stale
 
 template <int D, int NT> struct L2 {
@@ -68,7 +71,10 @@ template <int D, int NT> struct L2 {
     static constexpr int S_FULL = V_EMPTY + VS;          // [NT]
     static constexpr int S_FREE = S_FULL + NT, P_FULL = S_FREE + NT, PV_DONE = P_FULL + NT;
     static constexpr int TURN = PV_DONE + NT;            // [2][4]: per warp pair, "tile t may run its exponentials"
-    static constexpr int NUM_BARS = TURN + 8;
+    static constexpr int MERGE_BAR = TURN + 8;           // (key split over a cluster) partial results of the other CTAs have arrived
+    static constexpr int NUM_BARS = MERGE_BAR + 1;
+    // rows of partial results a CTA of a CS-way split receives: CS - 1 senders x 128 / CS rows it owns
+    __host__ __device__ static constexpr int merge_bytes(int cs) { return cs > 1 ? (cs - 1) * (128 / cs) * MERGE_VECS * 16 : 0; }
     // Strict alternation of the two tiles' exponential phases.  At d = 128 the chain of a tile is
     // softmax -> (O += P V, next S) -> softmax with nothing to overlap inside the tile, so the tiles
     // must interleave: one computes exponentials while the other's MMAs run.  Left to themselves
@@ -171,7 +177,13 @@ __device__ __forceinline__ float exp_store(const uint32_t (&s)[128], float scale
 // which key tiles the CTA's query tile attends; the CTA compacts its row of the map into a list in shared
 // memory and every role walks that list instead of 0, 1, 2, ...: pruned key tiles are neither loaded nor
 // multiplied.
-template <int D, int NT, bool VL = false, bool BIAS = false, bool SPARSE = false>
+// CS > 1 (one tile per CTA, dense, d = 64): the keys of a query tile are split over the CS CTAs of a thread-block
+// cluster (2, 4 or 8) -- for launches that would leave most SMs empty.  Each CTA runs the pipeline over its share of
+// the key tiles and ends with a partial (m, l, O) per row; rank r owns rows [128 r / CS, 128 (r + 1) / CS): the other
+// ranks store their partials for those rows into r's shared memory (st.shared::cluster, lanes of a warp writing
+// contiguous bytes) and arrive on r's mbarrier, and the owner merges them with the split-softmax identity and writes
+// the rows.  Plain remote stores only.
+template <int D, int NT, bool VL = false, bool BIAS = false, bool SPARSE = false, int CS = 1>
 __global__ void __launch_bounds__(128 * NT + 128, NT == 1 ? 2 : 1)
 fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                  const __grid_constant__ CUtensorMap tmV, __nv_bfloat16* __restrict__ O, int H, int Nq, int Nk,
@@ -181,6 +193,7 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                  const uint8_t* __restrict__ block_mask = nullptr, long long bmask_sb = 0, long long bmask_sh = 0) {
     using LY = L2<D, NT>;
     static_assert(!SPARSE || (NT == 1 && !VL && !BIAS), "the pruning map is read by the one-tile dense kernel");
+    static_assert(CS == 1 || (NT == 1 && D == 64 && !VL && !BIAS && !SPARSE && (CS == 2 || CS == 4 || CS == 8)), "key split: one-tile dense kernel, d = 64");
     __shared__ uint16_t tile_list[SPARSE ? 1024 : 1];    // the kept key tiles of this query tile, ascending
     __shared__ int tile_count;
     extern __shared__ uint8_t smem_raw[];
@@ -191,10 +204,12 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     uint64_t* bars = reinterpret_cast<uint64_t*>(base + LY::TILE_BYTES);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + LY::NUM_BARS);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    float4* merge_buf = reinterpret_cast<float4*>(base + LY::TILE_BYTES + 512);   // (CS > 1) [CS - 1][MERGE_VECS][128 / CS]: lanes of a warp touch contiguous bytes
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int bh = blockIdx.y;
-    const int row0 = blockIdx.x * (NT * BM);
+    const int crank = CS > 1 ? static_cast<int>(cluster_ctarank()) : 0;   // (cluster = CS consecutive CTAs along x)
+    const int row0 = (blockIdx.x / CS) * (NT * BM);
     int n = Nk;
     int head = 0, q_tok0 = 0, k_tok0 = 0, q_rows = 0;    // (packed batches only)
     if (VL) {
@@ -213,6 +228,12 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         if (lim < n) n = lim < 0 ? 0 : static_cast<int>(lim);
     }
     int ntiles = (n + BN - 1) / BN;
+    int tile0 = 0;                                       // first key tile of this CTA
+    if (CS > 1) {
+        const int per = (ntiles + CS - 1) / CS, left = ntiles - crank * per;
+        tile0 = crank * per;
+        ntiles = left < 0 ? 0 : (left > per ? per : left);
+    }
     if (SPARSE && (threadIdx.x >> 5) == 1) {
         // warp 1 compacts the map's row (tiles below the key limit n only) into the list
         const uint8_t* mrow = block_mask + static_cast<long long>(bh / H) * bmask_sb + static_cast<long long>(bh % H) * bmask_sh +
@@ -233,7 +254,7 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         for (int i = 0; i < LY::NUM_BARS; ++i) {
             const bool by_softmax = (i >= LY::S_FREE && i < LY::PV_DONE);      // one arrival per softmax warp
             const bool by_issuers = (i >= LY::K_EMPTY && i < LY::V_FULL) || (i >= LY::V_EMPTY && i < LY::S_FULL);
-            mbar_init(&bars[i], by_softmax ? 4 : by_issuers ? NT : 1);
+            mbar_init(&bars[i], i == LY::MERGE_BAR ? (CS > 1 ? (CS - 1) * (CS <= 4 ? 128 / CS / 32 : 1) : 1) : by_softmax ? 4 : by_issuers ? NT : 1);
         }
         *abort_flag = 0;
         fence_mbar_init();
@@ -243,9 +264,10 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
+    if (CS > 1) cluster_sync_all();                      // every CTA of the cluster has its barriers before anyone's first remote access
     if (SPARSE) ntiles = tile_count;
-    // key tile of step j: the j-th kept one under a pruning map, else j itself
-    auto tile_of = [&](int j) -> int { return SPARSE ? static_cast<int>(tile_list[j]) : j; };
+    // key tile of step j: the j-th kept one under a pruning map, else the j-th of this CTA's range
+    auto tile_of = [&](int j) -> int { return SPARSE ? static_cast<int>(tile_list[j]) : tile0 + j; };
 
     if (warp >= LY::SOFT_WARPS) {
       if (NT == 2) asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
@@ -553,6 +575,83 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             ok = bounded_wait(&bars[LY::PV_DONE + t], (ntiles - 1) & 1, abort_flag, status, 0x330 + t);
             ok = __all_sync(0xffffffffu, ok);
         }
+        if constexpr (CS > 1) {
+            // ---- key split: exchange of the partial (m, l, O) rows inside the cluster, then the owner's merge
+            constexpr int RP = 128 / CS;                  // rows owned per rank: whole warps, or half a warp at CS = 8
+            constexpr int GRP = RP < 32 ? RP : 32;        // lanes of a warp that share an owner
+            const int tr = (warp & 3) * 32 + lane, owner = tr / RP;
+            float o[D];
+            tc_fence_after();
+#pragma unroll
+            for (int c = 0; c < D / 32; ++c) {
+                uint32_t r[32];
+                if (ok && ntiles > 0) {
+                    tmem_ld_x32(tl + LY::O_COL(t) + c * 32, r);
+                    tc_wait_ld();
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) r[i] = 0u;      // no key tile in this CTA's share
+                }
+#pragma unroll
+                for (int i = 0; i < 32; ++i) o[c * 32 + i] = __uint_as_float(r[i]);
+            }
+            if (!ok) l = __int_as_float(0x7fc00000);     // (a CTA that gave up poisons the rows it took part in)
+            if (owner != crank) {
+                const int slot = (crank - owner - 1 + CS) % CS;
+                const uint32_t dst = mapa_shared(smem_u32(merge_buf + slot * MERGE_VECS * RP + tr % RP), owner);
+#pragma unroll
+                for (int v = 0; v < D / 4; ++v) st_cluster_v4(dst + 16 * RP * v, o[4 * v], o[4 * v + 1], o[4 * v + 2], o[4 * v + 3]);
+                st_cluster_v2(dst + 16 * RP * (D / 4), m_ref, l);
+            }
+            // one arrival per group of lanes with the same owner: the warp barrier orders the lanes' stores before
+            // the first lane's release
+            __syncwarp();
+            if (owner != crank && lane % GRP == 0) mbar_arrive_cluster(mapa_shared(smem_u32(&bars[LY::MERGE_BAR]), owner));
+            if (owner == crank) {
+                bool got = true;
+                {
+                    const long long t0 = clock64();
+                    while (!mbar_try_wait_cluster(&bars[LY::MERGE_BAR], 0)) {
+                        if (clock64() - t0 > WAIT_CYCLES) {
+                            got = false;
+                            if (status) atomicExch(status, 0x350);
+                            break;
+                        }
+                    }
+                }
+                if (got) {
+#pragma unroll
+                    for (int q = 0; q < CS - 1; ++q) {
+                        const float4* src = merge_buf + q * MERGE_VECS * RP + tr % RP;
+                        const float mq = src[RP * (D / 4)].x, lq = src[RP * (D / 4)].y;
+                        const float mt = fmaxf(m_ref, mq), mu = mt == -INFINITY ? 0.f : mt;
+                        const float a = ex2_approx(m_ref - mu), b = ex2_approx(mq - mu);
+                        l = l * a + lq * b;
+                        m_ref = mt;
+#pragma unroll
+                        for (int v = 0; v < D / 4; ++v) {
+                            const float4 w = src[RP * v];
+                            o[4 * v] = o[4 * v] * a + w.x * b;         o[4 * v + 1] = o[4 * v + 1] * a + w.y * b;
+                            o[4 * v + 2] = o[4 * v + 2] * a + w.z * b; o[4 * v + 3] = o[4 * v + 3] * a + w.w * b;
+                        }
+                    }
+                    if (row < Nq) {
+                        const float inv = l > 0.f ? 1.f / l : (l == l ? 0.f : l);
+                        if (lse) lse[static_cast<int64_t>(bh) * Nq + row] = l > 0.f ? (m_ref + log2f(l)) * 0.6931471805599453f : -INFINITY;
+                        __nv_bfloat16* orow = O + (static_cast<int64_t>(bh) * Nq + row) * D;
+#pragma unroll
+                        for (int v = 0; v < D / 8; ++v) {
+                            uint4 w;
+                            w.x = pack_bf16x2(o[8 * v + 0] * inv, o[8 * v + 1] * inv);
+                            w.y = pack_bf16x2(o[8 * v + 2] * inv, o[8 * v + 3] * inv);
+                            w.z = pack_bf16x2(o[8 * v + 4] * inv, o[8 * v + 5] * inv);
+                            w.w = pack_bf16x2(o[8 * v + 6] * inv, o[8 * v + 7] * inv);
+                            *reinterpret_cast<uint4*>(orow + v * 8) = w;
+                        }
+                    }
+                }
+            }
+        } else
         if (ok) {
             const float inv = l > 0.f ? 1.f / l : 0.f;
             // (dense batches only) log of the row's sum of exponentials; m_ref and the exponents are in base-2 units
@@ -591,7 +690,7 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
 }
 
 template <int D, int NT>
-int launch_tc2_d(const Problem& p, cudaStream_t st) {
+int launch_tc2_d(const Problem& p, cudaStream_t st, int key_split = 1) {
     using LY = L2<D, NT>;
     CUtensorMap tmQ, tmK, tmV;
     const int BH = p.B * p.H;
@@ -622,6 +721,35 @@ int launch_tc2_d(const Problem& p, cudaStream_t st) {
             return FLAT_ERR_UNSUPPORTED;
         }
     }
+    if constexpr (NT == 1 && D == 64) {
+        if (key_split == 2 || key_split == 4 || key_split == 8) {
+            // the keys of every query tile over a cluster of 2, 4 or 8 CTAs (consecutive along x)
+            auto launch = [&](auto cs_tag) -> int {
+                constexpr int CS = decltype(cs_tag)::value;
+                constexpr int BYTES = LY::SMEM_BYTES + LY::merge_bytes(CS);
+                if (!ensure_dynamic_smem<fused_tc2_kernel<D, NT, false, false, false, CS>>(BYTES)) return FLAT_ERR_CUDA;
+                cudaLaunchConfig_t cfg = {};
+                cfg.gridDim = dim3(grid.x * CS, grid.y);
+                cfg.blockDim = dim3(LY::THREADS);
+                cfg.dynamicSmemBytes = BYTES;
+                cfg.stream = st;
+                cudaLaunchAttribute attr[1];
+                attr[0].id = cudaLaunchAttributeClusterDimension;
+                attr[0].val.clusterDim.x = CS; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+                cfg.attrs = attr;
+                cfg.numAttrs = 1;
+                const cudaError_t e = cudaLaunchKernelEx(
+                    &cfg, fused_tc2_kernel<D, NT, false, false, false, CS>, tmQ, tmK, tmV, static_cast<__nv_bfloat16*>(p.O), p.H,
+                    p.Nq, p.Nk, p.scale * 1.4426950408889634f, p.k_valid_len, p.causal ? p.Nk - p.Nq : (1 << 30), p.status,
+                    static_cast<const int32_t*>(nullptr), static_cast<const int32_t*>(nullptr), p.lse,
+                    BiasArg{nullptr, 0, 0, 0, 0}, static_cast<const uint8_t*>(nullptr), 0ll, 0ll);
+                return e == cudaSuccess ? FLAT_OK : FLAT_ERR_CUDA;
+            };
+            return key_split == 2 ? launch(std::integral_constant<int, 2>{})
+                   : key_split == 4 ? launch(std::integral_constant<int, 4>{}) : launch(std::integral_constant<int, 8>{});
+        }
+    }
+    if (key_split != 1) return FLAT_ERR_UNSUPPORTED;
     auto kern = fused_tc2_kernel<D, NT>;
     if (!ensure_dynamic_smem<fused_tc2_kernel<D, NT>>(LY::SMEM_BYTES)) return FLAT_ERR_CUDA;
     kern<<<grid, LY::THREADS, LY::SMEM_BYTES, st>>>(tmQ, tmK, tmV, static_cast<__nv_bfloat16*>(p.O), p.H, p.Nq,
@@ -692,9 +820,10 @@ int launch_fused_tc2(const Problem& p, cudaStream_t st) {
 }
 
 // One 128-row tile per CTA, two CTAs per SM (d = 64 only: at d = 128 two CTAs do not fit in shared memory).
-int launch_fused_tc2_single(const Problem& p, cudaStream_t st) {
+int launch_fused_tc2_single(const Problem& p, cudaStream_t st, int key_split) {
     if (p.dtype != FLAT_DTYPE_BF16) return FLAT_ERR_UNSUPPORTED;
-    if (p.d == 64) return launch_tc2_d<64, 1>(p, st);
+    if (key_split != 1 && (p.d != 64 || p.bias || p.block_mask)) return FLAT_ERR_UNSUPPORTED;
+    if (p.d == 64) return launch_tc2_d<64, 1>(p, st, key_split);
     if (p.d == 128 && p.block_mask) return launch_tc2_d<128, 1>(p, st);   // (one CTA per SM: the pruned path only)
     return FLAT_ERR_UNSUPPORTED;
 }
