@@ -36,7 +36,9 @@ FP32_WORKLOAD = "c3_16k"             # the configuration the fp32 path is timed 
 L2_FLUSH_BELOW = 256 << 20          # workloads smaller than this get an L2 flush before every timed launch
 # FLAT_VARIANT_* (as reported by the library after a call) -> the kernel that variant launches
 KERNEL_OF_VARIANT = {1: "fused_simt_kernel", 2: "fused_tc_kernel", 3: "fused_tc2_kernel<2 tiles>",
-                     4: "fused_tc2_kernel<1 tile>", 5: "fused_tc3_kernel", 6: "fused_rgran_kernel", 7: "fused_tf32_kernel"}
+                     4: "fused_tc2_kernel<1 tile>", 5: "fused_tc3_kernel", 6: "fused_rgran_kernel", 7: "fused_tf32_kernel",
+                     8: "fused_tc2_kernel<1 tile, keys over a 2-CTA cluster>", 9: "fused_tc2_kernel<1 tile, keys over a 4-CTA cluster>",
+                     10: "fused_tc2_kernel<1 tile, keys over an 8-CTA cluster>"}
 TF32_OVER_BF16 = 1.1 / 2.25          # nominal dense tensor peaks: the tf32 roofline is the measured bf16 peak times this
 
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel from ncu

@@ -3,8 +3,9 @@
 The paper explores, per workload, how many query rows a fused tile should hold (its R-granularity
 trade-off, Section 5.3: fewer rows mean more K/V re-fetches and a worse-filled compute array) and
 picks the best mapping by search (Section 6.1).  On B200 the candidates are the compiled kernel
-variants: 64-row FFMA tiles, 128-row tensor-core CTAs (one or two per SM) and 256-row CTAs
-(with one or two softmax threads per row).
+variants: 64-row FFMA tiles, 128-row tensor-core CTAs (one or two per SM; with the keys of a tile split
+over a cluster of 2, 4 or 8 CTAs for launches that leave SMs empty) and 256-row CTAs (with one or two
+softmax threads per row).
 
     python -m paper_2107_06419_b200.tune [--workloads c1_bert_base_512,c2_bert_large_4k,...] [--steps 10]
     python -m paper_2107_06419_b200.tune --layer      (the attention layer around the fused path, step by step)
@@ -33,6 +34,9 @@ VARIANTS = {
     api.FLAT_VARIANT_TC2: "tc2: 256-row CTA (two tiles ping-pong)",
     api.FLAT_VARIANT_TC3: "tc3: 256-row CTA, half-row softmax threads, logits three tile-steps ahead (d = 64)",
     api.FLAT_VARIANT_RGRAN: "rgran: whole logit rows on chip, two-pass softmax (d = 64, Nk <= 512)",
+    api.FLAT_VARIANT_TC2_SPLIT2: "tc2_split2: 128-row CTA, keys split over a cluster of 2 CTAs (d = 64)",
+    api.FLAT_VARIANT_TC2_SPLIT4: "tc2_split4: ... over a cluster of 4 CTAs",
+    api.FLAT_VARIANT_TC2_SPLIT8: "tc2_split8: ... over a cluster of 8 CTAs",
     api.FLAT_VARIANT_AUTO: "auto (the dispatcher's choice)",
 }
 
@@ -206,13 +210,14 @@ def main():
     ap.add_argument("--layer", action="store_true",
                     help="time the whole attention layer (projections + fused attention) instead of the variants")
     ap.add_argument("--shapes", default="",
-                    help="extra self-attention shapes B:H:N:d, comma separated (e.g. 16:16:512:64), timed after the workloads")
+                    help="extra shapes B:H:N:d or B:H:Nq:Nk:d, comma separated (e.g. 16:16:512:64,1:1:128:16384:64), timed after the workloads")
     args = ap.parse_args()
     todo = [inputs.WORKLOADS[name] for name in args.workloads.split(",") if name]
     for spec in args.shapes.split(","):
         if spec:
-            B, H, N, d = (int(x) for x in spec.split(":"))
-            todo.append(inputs.Workload("B%d_H%d_N%d_d%d" % (B, H, N, d), B, H, N, N, d))
+            f = [int(x) for x in spec.split(":")]
+            B, H, Nq, Nk, d = f if len(f) == 5 else (f[0], f[1], f[2], f[2], f[3])
+            todo.append(inputs.Workload("B%d_H%d_Nq%d_Nk%d_d%d" % (B, H, Nq, Nk, d), B, H, Nq, Nk, d))
     for w in todo:
         name = w.name
         if args.varlen:
