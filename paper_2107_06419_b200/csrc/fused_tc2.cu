@@ -50,16 +50,20 @@ constexpr int POLY_LANE = 3;                    // element index mod 4 that uses
 constexpr int MERGE_VECS = 17;                   // (key split) 16-byte vectors per row of a partial result: 64 outputs, then (m, l)
 constexpr float OVERFLOW_SUM = 1.0995116e12f;   // 2^40: a tile row sum beyond this means m_ref is stale
 
-template <int D, int NT> struct L2 {
+// BT: the bias tile of every (tile, step) is staged through shared memory by TMA (two stages per query tile)
+template <int D, int NT, bool BT = false> struct L2 {
     static constexpr bool ALIAS = (D == 128);            // P overlays S
-    static constexpr int KS = (NT == 1) ? 2 : (D == 64) ? 3 : 2;   // K ring depth
+    static constexpr int KS = (NT == 1 || BT) ? 2 : (D == 64) ? 3 : 2;   // K ring depth
     static constexpr int VS = KS;                        // V ring depth
     static constexpr int THREADS = 128 * NT + 128;       // NT softmax warpgroups + {TMA, NT MMA issuers, idle}
     static constexpr int SOFT_WARPS = 4 * NT;
     static constexpr uint32_t TMEM_COLS = (NT == 2) ? 512 : 256;
     static constexpr int Q_BYTES = BM * D * 2;           // one query tile
     static constexpr int KV_BYTES = BN * D * 2;
-    static constexpr int TILE_BYTES = NT * Q_BYTES + (KS + VS) * KV_BYTES;
+    static constexpr int BS = 2;                         // bias ring depth per query tile
+    static constexpr int BIAS_BYTES = BM * BN * 2;       // one 128 x 128 bf16 tile: two panels of 128 rows x 128 bytes
+    static constexpr int BIAS_OFF = NT * Q_BYTES + (KS + VS) * KV_BYTES;
+    static constexpr int TILE_BYTES = BIAS_OFF + (BT ? NT * BS * BIAS_BYTES : 0);
     static constexpr int SMEM_BYTES = TILE_BYTES + 512 + 1024;
     __host__ __device__ static constexpr uint32_t S_COL(int t) { return 128u * t; }
     __host__ __device__ static constexpr uint32_t O_COL(int t) { return 128u * NT + D * t; }
@@ -72,7 +76,8 @@ template <int D, int NT> struct L2 {
     static constexpr int S_FREE = S_FULL + NT, P_FULL = S_FREE + NT, PV_DONE = P_FULL + NT;
     static constexpr int TURN = PV_DONE + NT;            // [2][4]: per warp pair, "tile t may run its exponentials"
     static constexpr int MERGE_BAR = TURN + 8;           // (key split over a cluster) partial results of the other CTAs have arrived
-    static constexpr int NUM_BARS = MERGE_BAR + 1;
+    static constexpr int B_FULL = MERGE_BAR + 1, B_EMPTY = B_FULL + NT * BS;   // (BT) [NT][BS]
+    static constexpr int NUM_BARS = BT ? B_EMPTY + NT * BS : MERGE_BAR + 1;
     // rows of partial results a CTA of a CS-way split receives: CS - 1 senders x 128 / CS rows it owns
     __host__ __device__ static constexpr int merge_bytes(int cs) { return cs > 1 ? (cs - 1) * (128 / cs) * MERGE_VECS * 16 : 0; }
     // Strict alternation of the two tiles' exponential phases.  At d = 128 the chain of a tile is
@@ -183,15 +188,20 @@ __device__ __forceinline__ float exp_store(const uint32_t (&s)[128], float scale
 // ranks store their partials for those rows into r's shared memory (st.shared::cluster, lanes of a warp writing
 // contiguous bytes) and arrive on r's mbarrier, and the owner merges them with the split-softmax identity and writes
 // the rows.  Plain remote stores only.
-template <int D, int NT, bool VL = false, bool BIAS = false, bool SPARSE = false, int CS = 1>
+// BIAS = 2: the same with the bias tile of each step staged through shared memory by TMA (bf16, 16-byte aligned
+// rows, d = 64): the rows then arrive coalesced and a softmax thread reads its 256 bytes from shared memory; with a
+// bias shared by all batches the grid runs the batches of a head next to each other, so that its slice stays in L2.
+template <int D, int NT, bool VL = false, int BIAS = 0, bool SPARSE = false, int CS = 1>
 __global__ void __launch_bounds__(128 * NT + 128, NT == 1 ? 2 : 1)
 fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                  const __grid_constant__ CUtensorMap tmV, __nv_bfloat16* __restrict__ O, int H, int Nq, int Nk,
                  float scale_log2e, const int32_t* __restrict__ valid_len, int coff, int32_t* status,
                  const int32_t* __restrict__ cu_q = nullptr, const int32_t* __restrict__ cu_k = nullptr,
                  float* __restrict__ lse = nullptr, BiasArg bias = BiasArg{nullptr, 0, 0, 0, 0},
-                 const uint8_t* __restrict__ block_mask = nullptr, long long bmask_sb = 0, long long bmask_sh = 0) {
-    using LY = L2<D, NT>;
+                 const uint8_t* __restrict__ block_mask = nullptr, long long bmask_sb = 0, long long bmask_sh = 0,
+                 const __grid_constant__ CUtensorMap tmBias = CUtensorMap{}) {
+    using LY = L2<D, NT, BIAS == 2>;
+    static_assert(BIAS != 2 || (NT == 2 && D == 64 && !VL && !SPARSE && CS == 1), "staged bias: the two-tile dense kernel, d = 64");
     static_assert(!SPARSE || (NT == 1 && !VL && !BIAS), "the pruning map is read by the one-tile dense kernel");
     static_assert(CS == 1 || (NT == 1 && D == 64 && !VL && !BIAS && !SPARSE && (CS == 2 || CS == 4 || CS == 8)), "key split: one-tile dense kernel, d = 64");
     __shared__ uint16_t tile_list[SPARSE ? 1024 : 1];    // the kept key tiles of this query tile, ascending
@@ -207,7 +217,12 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     float4* merge_buf = reinterpret_cast<float4*>(base + LY::TILE_BYTES + 512);   // (CS > 1) [CS - 1][MERGE_VECS][128 / CS]: lanes of a warp touch contiguous bytes
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int bh = blockIdx.y;
+    int bh = blockIdx.y;
+    if (BIAS == 2 && bias.sb == 0) {
+        // a bias shared by the batches: y runs over the batches first, so that CTAs in flight share a head's slice
+        const int nb = gridDim.y / H;
+        bh = (blockIdx.y % nb) * H + blockIdx.y / nb;
+    }
     const int crank = CS > 1 ? static_cast<int>(cluster_ctarank()) : 0;   // (cluster = CS consecutive CTAs along x)
     const int row0 = (blockIdx.x / CS) * (NT * BM);
     int n = Nk;
@@ -252,7 +267,8 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
 
     if (threadIdx.x == LY::SOFT_WARPS * 32) {
         for (int i = 0; i < LY::NUM_BARS; ++i) {
-            const bool by_softmax = (i >= LY::S_FREE && i < LY::PV_DONE);      // one arrival per softmax warp
+            const bool by_softmax = (i >= LY::S_FREE && i < LY::PV_DONE) ||    // one arrival per softmax warp
+                                    (BIAS == 2 && i >= LY::B_EMPTY);
             const bool by_issuers = (i >= LY::K_EMPTY && i < LY::V_FULL) || (i >= LY::V_EMPTY && i < LY::S_FULL);
             mbar_init(&bars[i], i == LY::MERGE_BAR ? (CS > 1 ? (CS - 1) * (CS <= 4 ? 128 / CS / 32 : 1) : 1) : by_softmax ? 4 : by_issuers ? NT : 1);
         }
@@ -300,11 +316,30 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                                 VL ? k_tok0 + j * BN : bh);
                 v_issued = j + 1;
             };
+            int b_issued = 0;
+            auto load_b = [&](int j) {                   // (BIAS == 2) the bias tiles of step j, one per query tile
+                const int s = j % LY::BS;
+#pragma unroll
+                for (int t = 0; t < NT; ++t) {
+                    if (!ok) return;
+                    ok = bounded_wait(&bars[LY::B_EMPTY + t * LY::BS + s], ((j / LY::BS) & 1) ^ 1, abort_flag, status, 0x120 + t);
+                    if (!ok) return;
+                    uint8_t* dst = base + LY::BIAS_OFF + (t * LY::BS + s) * LY::BIAS_BYTES;
+                    mbar_arrive_expect_tx(&bars[LY::B_FULL + t * LY::BS + s], LY::BIAS_BYTES);
+#pragma unroll
+                    for (int c = 0; c < 2; ++c)
+                        tma_load_4d(dst + c * BM * 128, &tmBias, &bars[LY::B_FULL + t * LY::BS + s], j * BN + c * 64, row0 + t * BM,
+                                    bias.sh ? bh % H : 0, bias.sb ? bh / H : 0);
+                }
+                b_issued = j + 1;
+            };
+            if (BIAS == 2) prefetch_tensormap(&tmBias);
             mbar_arrive_expect_tx(&bars[LY::Q_FULL + 0], LY::Q_BYTES);
 #pragma unroll
             for (int c = 0; c < D / 64; ++c)
                 tma_load_3d(Qs + c * BM * 128, &tmQ, &bars[LY::Q_FULL + 0], c * 64, VL ? head : row0, VL ? q_tok0 : bh);
             load_k(0);
+            if (BIAS == 2) load_b(0);
             if (NT == 2) {
                 mbar_arrive_expect_tx(&bars[LY::Q_FULL + NT - 1], LY::Q_BYTES);
 #pragma unroll
@@ -315,8 +350,12 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             for (int j = 0; j < ntiles && ok; ++j) {
                 if (j + 1 < ntiles) load_k(j + 1);
                 if (ok) load_v(j);
+                if (BIAS == 2 && ok && j + 1 < ntiles) load_b(j + 1);
             }
             if (!ok) {
+                if (BIAS == 2)
+                    for (int j = b_issued > LY::BS ? b_issued - LY::BS : 0; j < b_issued; ++j)
+                        for (int t = 0; t < NT; ++t) drain_wait(&bars[LY::B_FULL + t * LY::BS + j % LY::BS], (j / LY::BS) & 1);
                 drain_wait(&bars[LY::Q_FULL + 0], 0);
                 if (NT == 2) drain_wait(&bars[LY::Q_FULL + NT - 1], 0);
                 for (int j = k_issued > LY::KS ? k_issued - LY::KS : 0; j < k_issued; ++j)
@@ -412,9 +451,9 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         for (int j = 0; j < ntiles; ++j) {
             // (bias, the common case of an aligned bf16 tensor: the row's 128 values of this step are fetched
             // before the wait for the logits, so that the two latencies overlap)
-            uint32_t bpk[BIAS ? 64 : 1];
+            uint32_t bpk[BIAS == 1 ? 64 : 1];
             bool bias_ready = false;
-            if (BIAS) {
+            if (BIAS == 1) {
                 if (bias.vec && !bias.f32 && row < Nq && (j + 1) * BN <= Nk) {
                     const uint4* g = reinterpret_cast<const uint4*>(
                         static_cast<const __nv_bfloat16*>(bias.p) + static_cast<long long>(bh / H) * bias.sb +
@@ -440,7 +479,28 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             if (lane == 0) mbar_arrive(&bars[LY::S_FREE + t]);   // S_t may be overwritten (d = 64: by the next S_t)
 
             const int col0 = tile_of(j) * BN;
-            if (BIAS) {
+            if (BIAS == 2) {
+                // x = s * scale * log2(e) + bias * log2(e): the thread's row of the staged tile (two swizzled panels)
+                const int bs = j % LY::BS, rt = (warp & 3) * 32 + lane;
+                ok = __all_sync(0xffffffffu, bounded_wait(&bars[LY::B_FULL + t * LY::BS + bs], (j / LY::BS) & 1, abort_flag,
+                                                         status, 0x360 + t));
+                if (!ok) break;
+                const uint8_t* brow = base + LY::BIAS_OFF + (t * LY::BS + bs) * LY::BIAS_BYTES + rt * 128;
+#pragma unroll
+                for (int c = 0; c < 16; ++c) {
+                    const uint4 w = *reinterpret_cast<const uint4*>(brow + (c >> 3) * (BM * 128) + (((c & 7) ^ (rt & 7)) << 4));
+                    const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        s[c * 8 + 2 * e] = __float_as_uint(fmaf(__uint_as_float(s[c * 8 + 2 * e]), scale_log2e,
+                                                                __uint_as_float(ww[e] << 16) * 1.4426950408889634f));
+                        s[c * 8 + 2 * e + 1] = __float_as_uint(fmaf(__uint_as_float(s[c * 8 + 2 * e + 1]), scale_log2e,
+                                                                    __uint_as_float(ww[e] & 0xffff0000u) * 1.4426950408889634f));
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&bars[LY::B_EMPTY + t * LY::BS + bs]);
+            } else if (BIAS) {
                 // x = s * scale * log2(e) + bias * log2(e); a row past the end and columns past Nk read nothing
                 const long long at = static_cast<long long>(bh / H) * bias.sb + static_cast<long long>(bh % H) * bias.sh +
                                      static_cast<long long>(row) * Nk + col0;
@@ -689,6 +749,24 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     if (warp == 0) tmem_dealloc(tmem, LY::TMEM_COLS);
 }
 
+// The bias [B or 1, H or 1, Nq, Nk] bf16 as a 4-D tensor {Nk, Nq, heads, batches} with boxes of 64 columns x 128
+// rows (one 128-byte-swizzled panel); a broadcast axis has extent 1 and is always read at coordinate 0.
+bool make_bias_map(CUtensorMap* m, const Problem& p) {
+    EncodeTiledFn enc = get_encode_fn();
+    if (!enc) return false;
+    const cuuint64_t rowb = static_cast<cuuint64_t>(p.Nk) * 2, slice = static_cast<cuuint64_t>(p.Nq) * rowb;
+    const cuuint64_t sh = p.bias_sh ? static_cast<cuuint64_t>(p.bias_sh) * 2 : slice;
+    const cuuint64_t hb = p.bias_sh ? p.H : 1, bb = p.bias_sb ? p.B : 1;
+    const cuuint64_t sb = p.bias_sb ? static_cast<cuuint64_t>(p.bias_sb) * 2 : sh * hb;
+    cuuint64_t dims[4] = {static_cast<cuuint64_t>(p.Nk), static_cast<cuuint64_t>(p.Nq), hb, bb};
+    cuuint64_t strides[3] = {rowb, sh, sb};
+    cuuint32_t box[4] = {64, static_cast<cuuint32_t>(BM), 1, 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(p.bias), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 template <int D, int NT>
 int launch_tc2_d(const Problem& p, cudaStream_t st, int key_split = 1) {
     using LY = L2<D, NT>;
@@ -711,6 +789,19 @@ int launch_tc2_d(const Problem& p, cudaStream_t st, int key_split = 1) {
         }
     }
     if (p.bias) {
+        if constexpr (NT == 2 && D == 64) {
+            // bf16 bias with 16-byte aligned rows: tiles staged through shared memory by TMA
+            const BiasArg ba = bias_arg(p);
+            CUtensorMap tmB;
+            if (ba.vec && !ba.f32 && make_bias_map(&tmB, p)) {
+                using LB = L2<D, NT, true>;
+                if (!ensure_dynamic_smem<fused_tc2_kernel<D, NT, false, 2>>(LB::SMEM_BYTES)) return FLAT_ERR_CUDA;
+                fused_tc2_kernel<D, NT, false, 2><<<grid, LB::THREADS, LB::SMEM_BYTES, st>>>(
+                    tmQ, tmK, tmV, static_cast<__nv_bfloat16*>(p.O), p.H, p.Nq, p.Nk, p.scale * 1.4426950408889634f,
+                    p.k_valid_len, p.causal ? p.Nk - p.Nq : (1 << 30), p.status, nullptr, nullptr, p.lse, ba, nullptr, 0, 0, tmB);
+                return cudaGetLastError() == cudaSuccess ? FLAT_OK : FLAT_ERR_CUDA;
+            }
+        }
         if constexpr (NT == 2) {
             if (!ensure_dynamic_smem<fused_tc2_kernel<D, NT, false, true>>(LY::SMEM_BYTES)) return FLAT_ERR_CUDA;
             fused_tc2_kernel<D, NT, false, true><<<grid, LY::THREADS, LY::SMEM_BYTES, st>>>(
@@ -742,7 +833,7 @@ int launch_tc2_d(const Problem& p, cudaStream_t st, int key_split = 1) {
                     &cfg, fused_tc2_kernel<D, NT, false, false, false, CS>, tmQ, tmK, tmV, static_cast<__nv_bfloat16*>(p.O), p.H,
                     p.Nq, p.Nk, p.scale * 1.4426950408889634f, p.k_valid_len, p.causal ? p.Nk - p.Nq : (1 << 30), p.status,
                     static_cast<const int32_t*>(nullptr), static_cast<const int32_t*>(nullptr), p.lse,
-                    BiasArg{nullptr, 0, 0, 0, 0}, static_cast<const uint8_t*>(nullptr), 0ll, 0ll);
+                    BiasArg{nullptr, 0, 0, 0, 0}, static_cast<const uint8_t*>(nullptr), 0ll, 0ll, CUtensorMap{});
                 return e == cudaSuccess ? FLAT_OK : FLAT_ERR_CUDA;
             };
             return key_split == 2 ? launch(std::integral_constant<int, 2>{})
@@ -755,7 +846,7 @@ int launch_tc2_d(const Problem& p, cudaStream_t st, int key_split = 1) {
     kern<<<grid, LY::THREADS, LY::SMEM_BYTES, st>>>(tmQ, tmK, tmV, static_cast<__nv_bfloat16*>(p.O), p.H, p.Nq,
                                                     p.Nk, p.scale * 1.4426950408889634f, p.k_valid_len,
                                                     p.causal ? p.Nk - p.Nq : (1 << 30), p.status, nullptr, nullptr, p.lse,
-                                                    BiasArg{nullptr, 0, 0, 0, 0}, nullptr, 0, 0);
+                                                    BiasArg{nullptr, 0, 0, 0, 0}, nullptr, 0, 0, CUtensorMap{});
     return cudaGetLastError() == cudaSuccess ? FLAT_OK : FLAT_ERR_CUDA;
 }
 

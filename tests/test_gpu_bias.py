@@ -66,6 +66,29 @@ def test_bias_f32_storage_masks_and_minus_infinity(api):
         assert np.array_equal(np.isneginf(lse), dead) and np.abs(lse[~dead] - ref["LSE"][~dead]).max() <= 1e-3
 
 
+@pytest.mark.parametrize("bshape", ["full", "per_head", "per_batch", "one"])
+@pytest.mark.parametrize("causal", [False, True])
+def test_bias_bf16_tiles_staged_in_shared_memory(api, bshape, causal):
+    """d = 64 with a bf16 bias whose rows are 16-byte aligned: the tiles come through shared memory, the batches of a
+    head run next to each other when the bias is shared by the batches (a different order of the CTAs, the same
+    results), ragged last key tile, a key-padding mask, -inf entries."""
+    B, H, Nq, Nk, d = 3, 2, 300, 520, 64
+    rng = np.random.default_rng(11 + len(bshape) + causal)
+    Qb, Kb, Vb = (rand_bits(rng, s) for s in ((B, H, Nq, d), (B, H, Nk, d), (B, H, Nk, d)))
+    bs = {"full": (B, H), "per_head": (1, H), "per_batch": (B, 1), "one": (1, 1)}[bshape]
+    bf = (rng.standard_normal(bs + (Nq, Nk)) * 2.0).astype(np.float32)
+    bf[0, 0, :, 130:260] = -np.inf                       # a block of keys switched off
+    bf[0, -1, 9, :] = -np.inf                            # a whole row switched off
+    bias = inputs.f32_to_bf16_bits(bf).reshape(bf.shape)
+    vl = np.array([520, 391, 77], dtype=np.int32)
+    got, lse = run(api, Qb, Kb, Vb, 0.125, bias, vl=vl, causal=causal, want_lse=True)
+    assert api.flat_attn_last_variant() == api.FLAT_VARIANT_TC2
+    ref = oracle.attention(Qb, Kb, Vb, 0.125, bias=bias, valid_len=vl, causal=causal, want_lse=True)
+    check_bf16(got, ref["O"], "staged bias %s causal=%d" % (bshape, causal))
+    dead = np.isneginf(ref["LSE"])
+    assert np.array_equal(np.isneginf(lse), dead) and np.abs(lse[~dead] - ref["LSE"][~dead]).max() <= 1e-3
+
+
 def test_bias_unaligned_rows_take_the_scalar_loads(api):
     B, H, Nq, Nk, d = 1, 2, 130, 263, 64                 # Nk odd: no 16-byte loads
     rng = np.random.default_rng(4)
