@@ -225,6 +225,33 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     }
     const int crank = CS > 1 ? static_cast<int>(cluster_ctarank()) : 0;   // (cluster = CS consecutive CTAs along x)
     const int row0 = (blockIdx.x / CS) * (NT * BM);
+    // Barriers and TMEM columns.  The one-tile dense kernels (short launches, where the gap between two kernels of a
+    // stream is a good part of the time) do this before anything else and then let the next kernel of the stream
+    // start its own set-up (griddepcontrol.launch_dependents) and wait for the previous one to finish
+    // (griddepcontrol.wait) before the first access to device memory: launched with programmatic stream
+    // serialization, consecutive kernels overlap one's tail with the other's prologue.
+    constexpr bool PDL = (NT == 1 && !VL && !SPARSE && !BIAS);
+    auto setup = [&]() {
+        if (threadIdx.x == LY::SOFT_WARPS * 32) {
+            for (int i = 0; i < LY::NUM_BARS; ++i) {
+                const bool by_softmax = (i >= LY::S_FREE && i < LY::PV_DONE) ||    // one arrival per softmax warp
+                                        (BIAS == 2 && i >= LY::B_EMPTY);
+                const bool by_issuers = (i >= LY::K_EMPTY && i < LY::V_FULL) || (i >= LY::V_EMPTY && i < LY::S_FULL);
+                mbar_init(&bars[i], i == LY::MERGE_BAR ? (CS > 1 ? (CS - 1) * (CS <= 4 ? 128 / CS / 32 : 1) : 1) : by_softmax ? 4 : by_issuers ? NT : 1);
+            }
+            *abort_flag = 0;
+            fence_mbar_init();
+        }
+        if (warp == 0) { tmem_alloc(tmem_slot, LY::TMEM_COLS); tmem_relinquish(); }
+        tc_fence_before();
+        __syncthreads();
+        tc_fence_after();
+    };
+    if (PDL) {
+        setup();
+        asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+    }
     int n = Nk;
     int head = 0, q_tok0 = 0, k_tok0 = 0, q_rows = 0;    // (packed batches only)
     if (VL) {
@@ -265,20 +292,7 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         if (ln == 0) tile_count = count;
     }
 
-    if (threadIdx.x == LY::SOFT_WARPS * 32) {
-        for (int i = 0; i < LY::NUM_BARS; ++i) {
-            const bool by_softmax = (i >= LY::S_FREE && i < LY::PV_DONE) ||    // one arrival per softmax warp
-                                    (BIAS == 2 && i >= LY::B_EMPTY);
-            const bool by_issuers = (i >= LY::K_EMPTY && i < LY::V_FULL) || (i >= LY::V_EMPTY && i < LY::S_FULL);
-            mbar_init(&bars[i], i == LY::MERGE_BAR ? (CS > 1 ? (CS - 1) * (CS <= 4 ? 128 / CS / 32 : 1) : 1) : by_softmax ? 4 : by_issuers ? NT : 1);
-        }
-        *abort_flag = 0;
-        fence_mbar_init();
-    }
-    if (warp == 0) { tmem_alloc(tmem_slot, LY::TMEM_COLS); tmem_relinquish(); }
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
+    if (!PDL) setup();
     const uint32_t tmem = *tmem_slot;
     if (CS > 1) cluster_sync_all();                      // every CTA of the cluster has its barriers before anyone's first remote access
     if (SPARSE) ntiles = tile_count;
@@ -824,11 +838,13 @@ int launch_tc2_d(const Problem& p, cudaStream_t st, int key_split = 1) {
                 cfg.blockDim = dim3(LY::THREADS);
                 cfg.dynamicSmemBytes = BYTES;
                 cfg.stream = st;
-                cudaLaunchAttribute attr[1];
+                cudaLaunchAttribute attr[2];
                 attr[0].id = cudaLaunchAttributeClusterDimension;
                 attr[0].val.clusterDim.x = CS; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+                attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // (see the kernel's prologue)
+                attr[1].val.programmaticStreamSerializationAllowed = 1;
                 cfg.attrs = attr;
-                cfg.numAttrs = 1;
+                cfg.numAttrs = 2;
                 const cudaError_t e = cudaLaunchKernelEx(
                     &cfg, fused_tc2_kernel<D, NT, false, false, false, CS>, tmQ, tmK, tmV, static_cast<__nv_bfloat16*>(p.O), p.H,
                     p.Nq, p.Nk, p.scale * 1.4426950408889634f, p.k_valid_len, p.causal ? p.Nk - p.Nq : (1 << 30), p.status,
@@ -843,6 +859,25 @@ int launch_tc2_d(const Problem& p, cudaStream_t st, int key_split = 1) {
     if (key_split != 1) return FLAT_ERR_UNSUPPORTED;
     auto kern = fused_tc2_kernel<D, NT>;
     if (!ensure_dynamic_smem<fused_tc2_kernel<D, NT>>(LY::SMEM_BYTES)) return FLAT_ERR_CUDA;
+    if constexpr (NT == 1) {
+        // short launches: the kernel may start while its predecessor in the stream drains (see its prologue)
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = grid;
+        cfg.blockDim = dim3(LY::THREADS);
+        cfg.dynamicSmemBytes = LY::SMEM_BYTES;
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        const cudaError_t e = cudaLaunchKernelEx(
+            &cfg, kern, tmQ, tmK, tmV, static_cast<__nv_bfloat16*>(p.O), p.H, p.Nq, p.Nk, p.scale * 1.4426950408889634f,
+            p.k_valid_len, p.causal ? p.Nk - p.Nq : (1 << 30), p.status, static_cast<const int32_t*>(nullptr),
+            static_cast<const int32_t*>(nullptr), p.lse, BiasArg{nullptr, 0, 0, 0, 0}, static_cast<const uint8_t*>(nullptr), 0ll, 0ll,
+            CUtensorMap{});
+        return e == cudaSuccess ? FLAT_OK : FLAT_ERR_CUDA;
+    }
     kern<<<grid, LY::THREADS, LY::SMEM_BYTES, st>>>(tmQ, tmK, tmV, static_cast<__nv_bfloat16*>(p.O), p.H, p.Nq,
                                                     p.Nk, p.scale * 1.4426950408889634f, p.k_valid_len,
                                                     p.causal ? p.Nk - p.Nq : (1 << 30), p.status, nullptr, nullptr, p.lse,
