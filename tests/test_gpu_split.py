@@ -127,3 +127,40 @@ def test_cluster_launch_in_a_cuda_graph(api):
         g.replay()
         s.synchronize()
     check_bf16(bf16_to_f64(O), ref, "split in a graph")
+
+
+@pytest.mark.parametrize("variant", [4, 8, 9])
+def test_back_to_back_launches_that_depend_on_each_other(api, variant):
+    """The one-tile kernels let the next kernel of the stream start its set-up early (programmatic dependent launch)
+    and wait for their predecessor before the first access to device memory.  A chain in which every call reads
+    the previous call's output -- and the third call overwrites the first call's input -- must give the bits of the
+    same chain run with a device synchronisation after every call."""
+    rng = np.random.default_rng(77)
+    B, H, Nq, Nk = 1, 6, 512, 512
+    Qb, Kb, Vb = rand_bits(rng, (B, H, Nq, 64)), rand_bits(rng, (B, H, Nk, 64)), rand_bits(rng, (B, H, Nk, 64))
+    K, V = bf16_tensor(Kb), bf16_tensor(Vb)
+
+    def chain(sync):
+        X = bf16_tensor(Qb).clone()
+        Y = torch.zeros_like(X)
+        Z = torch.zeros_like(X)
+        for _ in range(4):
+            api.flat_attn_fwd_ex(X, K, V, Y, 0.125, variant=variant)      # Y = f(X)
+            if sync: torch.cuda.synchronize()
+            api.flat_attn_fwd_ex(Y, K, V, Z, 0.125, variant=variant)      # Z = f(Y)
+            if sync: torch.cuda.synchronize()
+            api.flat_attn_fwd_ex(Z, K, V, X, 0.125, variant=variant)      # X = f(Z): overwrites the first call's input
+            if sync: torch.cuda.synchronize()
+        torch.cuda.synchronize()
+        return X.view(torch.int16).clone(), Y.view(torch.int16).clone(), Z.view(torch.int16).clone()
+
+    ref = chain(True)
+    for _ in range(3):
+        got = chain(False)
+        for a, b in zip(ref, got):
+            assert torch.equal(a, b)
+    # and the first link against the oracle
+    O = torch.zeros(B, H, Nq, 64, dtype=torch.bfloat16, device="cuda")
+    api.flat_attn_fwd_ex(bf16_tensor(Qb), K, V, O, 0.125, variant=variant)
+    torch.cuda.synchronize()
+    check_bf16(bf16_to_f64(O), oracle.attention(Qb, Kb, Vb, 0.125)["O"], "chain link v%d" % variant)
