@@ -80,7 +80,7 @@ enum {
                                   pruning map (what AUTO picks there)                            */
     FLAT_VARIANT_TC2_SPLIT2 = 8, /* TC2_SINGLE with the keys of every query tile split over a cluster
                                   of two CTAs, whose partial softmaxes are merged through
-                                  distributed shared memory: bf16, d = 64, no bias, no pruning map;
+                                  distributed shared memory: bf16, d in {64,128}, no bias, no pruning map;
                                   what AUTO picks for launches that would leave most SMs empty   */
     FLAT_VARIANT_TC2_SPLIT4 = 9, /* the same over a cluster of four CTAs                           */
     FLAT_VARIANT_TC2_SPLIT8 = 10 /* the same over a cluster of eight CTAs                          */

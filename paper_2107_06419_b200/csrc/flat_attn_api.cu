@@ -138,13 +138,25 @@ int run_fused(const flat::Problem& q, int variant, cudaStream_t st) {
                     break;
                 }
             }
+            // d = 128: the same split (one CTA per SM there: 160 KB of tiles) while the two-tile CTAs would cover
+            // less than half the SMs and every CTA of the split keeps at least two key steps (128 queries x
+            // 16K keys, 8 heads: 247 -> 41 us).
+            if (q.d == 128 && !q.block_mask && !q.bias && 2 * ctas2 < sms) {
+                const int64_t ctas1 = static_cast<int64_t>((q.Nq + 127) / 128) * q.B * q.H;
+                const int key_tiles = (q.Nk + 127) / 128;
+                for (int cs = 8; cs >= 2; cs /= 2) {
+                    if (ctas1 * cs > sms || key_tiles < 2 * cs) continue;
+                    v = cs == 8 ? FLAT_VARIANT_TC2_SPLIT8 : cs == 4 ? FLAT_VARIANT_TC2_SPLIT4 : FLAT_VARIANT_TC2_SPLIT2;
+                    break;
+                }
+            }
         }
     }
     if (q.causal && v == FLAT_VARIANT_TC) return FLAT_ERR_UNSUPPORTED;
     if (q.lse && (v == FLAT_VARIANT_TC || v == FLAT_VARIANT_RGRAN)) return FLAT_ERR_UNSUPPORTED;
     if (q.bias && v != FLAT_VARIANT_TC2 && v != FLAT_VARIANT_SIMT) return FLAT_ERR_UNSUPPORTED;
     if (v == FLAT_VARIANT_TC2_SPLIT2 || v == FLAT_VARIANT_TC2_SPLIT4 || v == FLAT_VARIANT_TC2_SPLIT8) {
-        if (!tc_applies(q) || q.d != 64 || q.block_mask) return FLAT_ERR_UNSUPPORTED;
+        if (!tc_applies(q) || q.block_mask) return FLAT_ERR_UNSUPPORTED;
         g_last_variant = v;
         return flat::launch_fused_tc2_single(q, st, v == FLAT_VARIANT_TC2_SPLIT2 ? 2 : v == FLAT_VARIANT_TC2_SPLIT4 ? 4 : 8);
     }

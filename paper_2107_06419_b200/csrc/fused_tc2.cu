@@ -47,7 +47,7 @@ constexpr int BM = 128;              // rows per query tile (two tiles per CTA)
 constexpr int BN = 128;              // keys per step
 constexpr int PASS_AT_CHUNK = 3;                // the other tile gets its turn once this chunk's ex2 are issued
 constexpr int POLY_LANE = 3;                    // element index mod 4 that uses ex2_poly; -1 = none
-constexpr int MERGE_VECS = 17;                   // (key split) 16-byte vectors per row of a partial result: 64 outputs, then (m, l)
+__host__ __device__ constexpr int merge_vecs(int d) { return d / 4 + 1; }   // (key split) 16-byte vectors per row of a partial result: d outputs, then (m, l)
 constexpr float OVERFLOW_SUM = 1.0995116e12f;   // 2^40: a tile row sum beyond this means m_ref is stale
 
 // BT: the bias tile of every (tile, step) is staged through shared memory by TMA (two stages per query tile)
@@ -79,7 +79,7 @@ template <int D, int NT, bool BT = false> struct L2 {
     static constexpr int B_FULL = MERGE_BAR + 1, B_EMPTY = B_FULL + NT * BS;   // (BT) [NT][BS]
     static constexpr int NUM_BARS = BT ? B_EMPTY + NT * BS : MERGE_BAR + 1;
     // rows of partial results a CTA of a CS-way split receives: CS - 1 senders x 128 / CS rows it owns
-    __host__ __device__ static constexpr int merge_bytes(int cs) { return cs > 1 ? (cs - 1) * (128 / cs) * MERGE_VECS * 16 : 0; }
+    __host__ __device__ static constexpr int merge_bytes(int cs) { return cs > 1 ? (cs - 1) * (128 / cs) * merge_vecs(D) * 16 : 0; }
     // Strict alternation of the two tiles' exponential phases.  At d = 128 the chain of a tile is
     // softmax -> (O += P V, next S) -> softmax with nothing to overlap inside the tile, so the tiles
     // must interleave: one computes exponentials while the other's MMAs run.  Left to themselves
@@ -182,7 +182,7 @@ __device__ __forceinline__ float exp_store(const uint32_t (&s)[128], float scale
 // which key tiles the CTA's query tile attends; the CTA compacts its row of the map into a list in shared
 // memory and every role walks that list instead of 0, 1, 2, ...: pruned key tiles are neither loaded nor
 // multiplied.
-// CS > 1 (one tile per CTA, dense, d = 64): the keys of a query tile are split over the CS CTAs of a thread-block
+// CS > 1 (one tile per CTA, dense): the keys of a query tile are split over the CS CTAs of a thread-block
 // cluster (2, 4 or 8) -- for launches that would leave most SMs empty.  Each CTA runs the pipeline over its share of
 // the key tiles and ends with a partial (m, l, O) per row; rank r owns rows [128 r / CS, 128 (r + 1) / CS): the other
 // ranks store their partials for those rows into r's shared memory (st.shared::cluster, lanes of a warp writing
@@ -203,7 +203,7 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     using LY = L2<D, NT, BIAS == 2>;
     static_assert(BIAS != 2 || (NT == 2 && D == 64 && !VL && !SPARSE && CS == 1), "staged bias: the two-tile dense kernel, d = 64");
     static_assert(!SPARSE || (NT == 1 && !VL && !BIAS), "the pruning map is read by the one-tile dense kernel");
-    static_assert(CS == 1 || (NT == 1 && D == 64 && !VL && !BIAS && !SPARSE && (CS == 2 || CS == 4 || CS == 8)), "key split: one-tile dense kernel, d = 64");
+    static_assert(CS == 1 || (NT == 1 && !VL && !BIAS && !SPARSE && (CS == 2 || CS == 4 || CS == 8)), "key split: one-tile dense kernel");
     __shared__ uint16_t tile_list[SPARSE ? 1024 : 1];    // the kept key tiles of this query tile, ascending
     __shared__ int tile_count;
     extern __shared__ uint8_t smem_raw[];
@@ -214,7 +214,7 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     uint64_t* bars = reinterpret_cast<uint64_t*>(base + LY::TILE_BYTES);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + LY::NUM_BARS);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-    float4* merge_buf = reinterpret_cast<float4*>(base + LY::TILE_BYTES + 512);   // (CS > 1) [CS - 1][MERGE_VECS][128 / CS]: lanes of a warp touch contiguous bytes
+    float4* merge_buf = reinterpret_cast<float4*>(base + LY::TILE_BYTES + 512);   // (CS > 1) [CS - 1][d / 4 + 1][128 / CS]: lanes of a warp touch contiguous bytes
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     int bh = blockIdx.y;
@@ -672,7 +672,7 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             if (!ok) l = __int_as_float(0x7fc00000);     // (a CTA that gave up poisons the rows it took part in)
             if (owner != crank) {
                 const int slot = (crank - owner - 1 + CS) % CS;
-                const uint32_t dst = mapa_shared(smem_u32(merge_buf + slot * MERGE_VECS * RP + tr % RP), owner);
+                const uint32_t dst = mapa_shared(smem_u32(merge_buf + slot * merge_vecs(D) * RP + tr % RP), owner);
 #pragma unroll
                 for (int v = 0; v < D / 4; ++v) st_cluster_v4(dst + 16 * RP * v, o[4 * v], o[4 * v + 1], o[4 * v + 2], o[4 * v + 3]);
                 st_cluster_v2(dst + 16 * RP * (D / 4), m_ref, l);
@@ -696,7 +696,7 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                 if (got) {
 #pragma unroll
                     for (int q = 0; q < CS - 1; ++q) {
-                        const float4* src = merge_buf + q * MERGE_VECS * RP + tr % RP;
+                        const float4* src = merge_buf + q * merge_vecs(D) * RP + tr % RP;
                         const float mq = src[RP * (D / 4)].x, lq = src[RP * (D / 4)].y;
                         const float mt = fmaxf(m_ref, mq), mu = mt == -INFINITY ? 0.f : mt;
                         const float a = ex2_approx(m_ref - mu), b = ex2_approx(mq - mu);
@@ -826,7 +826,7 @@ int launch_tc2_d(const Problem& p, cudaStream_t st, int key_split = 1) {
             return FLAT_ERR_UNSUPPORTED;
         }
     }
-    if constexpr (NT == 1 && D == 64) {
+    if constexpr (NT == 1) {
         if (key_split == 2 || key_split == 4 || key_split == 8) {
             // the keys of every query tile over a cluster of 2, 4 or 8 CTAs (consecutive along x)
             auto launch = [&](auto cs_tag) -> int {
@@ -948,9 +948,9 @@ int launch_fused_tc2(const Problem& p, cudaStream_t st) {
 // One 128-row tile per CTA, two CTAs per SM (d = 64 only: at d = 128 two CTAs do not fit in shared memory).
 int launch_fused_tc2_single(const Problem& p, cudaStream_t st, int key_split) {
     if (p.dtype != FLAT_DTYPE_BF16) return FLAT_ERR_UNSUPPORTED;
-    if (key_split != 1 && (p.d != 64 || p.bias || p.block_mask)) return FLAT_ERR_UNSUPPORTED;
+    if (key_split != 1 && (p.bias || p.block_mask)) return FLAT_ERR_UNSUPPORTED;
     if (p.d == 64) return launch_tc2_d<64, 1>(p, st, key_split);
-    if (p.d == 128 && p.block_mask) return launch_tc2_d<128, 1>(p, st);   // (one CTA per SM: the pruned path only)
+    if (p.d == 128 && (p.block_mask || key_split != 1)) return launch_tc2_d<128, 1>(p, st, key_split);   // (one CTA per SM: the pruned path and the key split)
     return FLAT_ERR_UNSUPPORTED;
 }
 

@@ -34,7 +34,7 @@ VARIANTS = {
     api.FLAT_VARIANT_TC2: "tc2: 256-row CTA (two tiles ping-pong)",
     api.FLAT_VARIANT_TC3: "tc3: 256-row CTA, half-row softmax threads, logits three tile-steps ahead (d = 64)",
     api.FLAT_VARIANT_RGRAN: "rgran: whole logit rows on chip, two-pass softmax (d = 64, Nk <= 512)",
-    api.FLAT_VARIANT_TC2_SPLIT2: "tc2_split2: 128-row CTA, keys split over a cluster of 2 CTAs (d = 64)",
+    api.FLAT_VARIANT_TC2_SPLIT2: "tc2_split2: 128-row CTA, keys split over a cluster of 2 CTAs",
     api.FLAT_VARIANT_TC2_SPLIT4: "tc2_split4: ... over a cluster of 4 CTAs",
     api.FLAT_VARIANT_TC2_SPLIT8: "tc2_split8: ... over a cluster of 8 CTAs",
     api.FLAT_VARIANT_AUTO: "auto (the dispatcher's choice)",

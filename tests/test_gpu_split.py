@@ -99,9 +99,37 @@ def test_auto_takes_the_split_for_underfilled_launches(api):
         check_bf16(O, ref, "auto split %s" % ((B, H, Nq, Nk),))
 
 
+@pytest.mark.parametrize("variant", SPLITS)
+@pytest.mark.parametrize("shape", [(1, 2, 128, 128), (2, 2, 200, 333), (1, 3, 300, 2100), (1, 1, 77, 4096)])
+def test_head_size_128(api, shape, variant):
+    B, H, Nq, Nk = shape
+    rng = np.random.default_rng(Nq + Nk + variant + 128)
+    Qb, Kb, Vb = rand_bits(rng, (B, H, Nq, 128)), rand_bits(rng, (B, H, Nk, 128)), rand_bits(rng, (B, H, Nk, 128))
+    vl = np.array([Nk, Nk // 2], dtype=np.int32)[:B]
+    for causal in (False, True):
+        ref = oracle.attention(Qb, Kb, Vb, 128 ** -0.5, valid_len=vl, causal=causal, want_lse=True)
+        O, lse = run(api, Qb, Kb, Vb, 128 ** -0.5, variant, vl=vl, causal=causal)
+        assert api.flat_attn_last_variant() == variant
+        check_bf16(O, ref["O"], "split d128 v%d %s causal=%d" % (variant, shape, causal))
+        fin = np.isfinite(ref["LSE"])
+        assert np.array_equal(np.isneginf(lse), np.isneginf(ref["LSE"])) and np.max(np.abs(lse[fin] - ref["LSE"][fin])) < 1e-3
+
+
+def test_auto_takes_the_split_at_head_size_128(api):
+    rng = np.random.default_rng(19)
+    for (B, H, Nq, Nk, expect) in [(1, 8, 128, 16384, api.FLAT_VARIANT_TC2_SPLIT8), (1, 8, 512, 4096, api.FLAT_VARIANT_TC2_SPLIT4),
+                                   (4, 16, 2048, 2048, api.FLAT_VARIANT_TC2)]:
+        Qb, Kb, Vb = rand_bits(rng, (B, H, Nq, 128)), rand_bits(rng, (B, H, Nk, 128)), rand_bits(rng, (B, H, Nk, 128))
+        rows = inputs.sample_rows(inputs.Workload("x", B, H, Nq, Nk, 128), 4)
+        ref = oracle.attention(Qb, Kb, Vb, 0.1, rows=rows)["O"]
+        O, _ = run(api, Qb, Kb, Vb, 0.1, api.FLAT_VARIANT_AUTO)
+        assert api.flat_attn_last_variant() == expect, (B, H, Nq, Nk)
+        check_bf16(O.reshape(-1, 128)[rows], ref, "auto split d128 %s" % ((B, H, Nq, Nk),))
+
+
 def test_refusals(api):
-    Q = torch.zeros(1, 1, 128, 128, device="cuda", dtype=torch.bfloat16)
-    with pytest.raises(api.FlatAttnError):               # d = 128
+    Q = torch.zeros(1, 1, 128, 32, device="cuda", dtype=torch.bfloat16)
+    with pytest.raises(api.FlatAttnError):               # d = 32
         api.flat_attn_fwd_ex(Q, Q, Q, torch.empty_like(Q), 1.0, variant=api.FLAT_VARIANT_TC2_SPLIT2)
     Q64 = torch.zeros(1, 1, 128, 64, device="cuda", dtype=torch.bfloat16)
     bias = torch.zeros(1, 1, 128, 128, device="cuda", dtype=torch.bfloat16)
