@@ -32,6 +32,8 @@ METRIC = "fused attention TFLOP/s"
 UNIT = "TFLOP/s"
 DEFAULT_WORKLOAD = "c2_bert_large_4k"
 OTHER_WORKLOADS = ["c1_bert_base_512", "c3_16k", "c4_64k_d128", "c5_cross_masked"]
+# launches that leave most SMs empty (few query tiles, long key sequences): what the key split over a cluster is for
+UNDERFILLED = [("u1_128q_16k_d64", 1, 1, 128, 16384, 64), ("u2_128q_16k_h8_d128", 1, 8, 128, 16384, 128)]
 FP32_WORKLOAD = "c3_16k"             # the configuration the fp32 path is timed on (widened to fp32 tensors)
 L2_FLUSH_BELOW = 256 << 20          # workloads smaller than this get an L2 flush before every timed launch
 # FLAT_VARIANT_* (as reported by the library after a call) -> the kernel that variant launches
@@ -409,6 +411,7 @@ def main():
             out["workloads"] = [run_other(bench, torch, api, inputs.WORKLOADS[n], seed, args, peaks, dev)
                                 for n in OTHER_WORKLOADS if n != w.name]
             out["fp32"] = run_fp32(bench, torch, api, inputs.WORKLOADS[FP32_WORKLOAD], seed, args, peaks, dev)
+            out["underfilled"] = [run_underfilled(torch, api, inputs.Workload(*spec), seed, args, dev) for spec in UNDERFILLED]
         print(json.dumps(out))
     if world > 1:
         dist.destroy_process_group()
@@ -511,6 +514,53 @@ def run_fp32(bench, torch, api, w, seed, args, peaks, dev):
         e["parity_on_sample"]["bar_max_abs"] = 1e-4
     del data, d, Q, K, V, O
     torch.cuda.empty_cache()
+    return e
+
+
+def run_underfilled(torch, api, w, seed, args, dev):
+    """A launch with far fewer query tiles than SMs: GPU time per launch in a replay of a CUDA graph of 20 launches,
+    the dispatcher's choice (keys of a tile split over a thread-block cluster) beside the unsplit kernel, and parity
+    of the dispatcher's output on every row."""
+    from paper_2107_06419_b200 import inputs
+    Qb, Kb, Vb = inputs.make_qkv_bf16(w, seed)
+    as_t = lambda bits: torch.from_numpy(bits.view(np.int16)).view(torch.bfloat16).to(dev)
+    Q, K, V = as_t(Qb), as_t(Kb), as_t(Vb)
+    O = torch.empty_like(Q)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+
+    def replay_us(variant):
+        s = torch.cuda.Stream(device=dev)
+        with torch.cuda.stream(s):
+            for _ in range(3):
+                api.flat_attn_fwd_ex(Q, K, V, O, w.scale, status=status, variant=variant, stream=s.cuda_stream)
+            ran = api.flat_attn_last_variant()
+            s.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=s):
+                for _ in range(20):
+                    api.flat_attn_fwd_ex(Q, K, V, O, w.scale, status=status, variant=variant, stream=s.cuda_stream)
+            g.replay()
+            s.synchronize()
+            best = None
+            for _ in range(5):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(s); g.replay(); e1.record(s); s.synchronize()
+                t = e0.elapsed_time(e1) / 20 * 1e3
+                best = t if best is None or t < best else best
+        return best, ran
+
+    unsplit_us, unsplit_variant = replay_us(api.FLAT_VARIANT_TC2_SINGLE if w.d == 64 else api.FLAT_VARIANT_TC2)
+    auto_us, auto_variant = replay_us(api.FLAT_VARIANT_AUTO)           # (last: O holds the dispatcher's result)
+    assert int(status.item()) == 0
+    e = {"workload": w.name, "config": {"B": w.B, "H": w.H, "Nq": w.Nq, "Nk": w.Nk, "d": w.d},
+         "timing": "CUDA-graph replay of 20 launches, best of 5, microseconds per launch",
+         "kernel": KERNEL_OF_VARIANT.get(auto_variant, "?"), "us": auto_us, "value": float(w.flops) / auto_us / 1e6, "unit": UNIT,
+         "unsplit_kernel": KERNEL_OF_VARIANT.get(unsplit_variant, "?"), "unsplit_us": unsplit_us}
+    if not args.no_cpu_baseline:
+        import oracle
+        ref = oracle.attention(Qb, Kb, Vb, w.scale)["O"]
+        err = np.abs(O.float().cpu().numpy().astype(np.float64) - ref)
+        e["parity_all_rows"] = {"max_abs": float(err.max()), "mean_abs": float(err.mean())}
     return e
 
 
