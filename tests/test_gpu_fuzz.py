@@ -142,3 +142,60 @@ def test_backward(api, case):
         # the absolute floors stand for 'zero at the scale of the other gradients', which are of order 1 here)
         assert float(np.abs(g - r).max()) <= 2e-2 * top + 1e-4, (case[:7], name)
         assert float(np.abs(g - r).mean()) <= 1e-2 * float(np.abs(r).mean()) + 1e-5, (case[:7], name)
+
+
+@pytest.mark.parametrize("case", cases(777, 24), ids=lambda c: "B%dH%dq%dk%dd%d%s%s" % (c[0], c[1], c[2], c[3], c[4], "c" if c[5] else "", "m%d" % c[6]))
+def test_bias_and_pruning_map(api, case):
+    """The same random problems with an additive bias (bf16 or fp32, a random broadcast form, a few -inf entries;
+    row lengths that are multiples of 8 take the tiles staged in shared memory at d = 64, the others the per-thread
+    loads) and, separately, with a random pruning map over 128 x 128 blocks."""
+    B, H, Nq, Nk, d, causal, mask, seed = case
+    rng = np.random.default_rng(seed)
+    if rng.integers(0, 2):
+        Nk = (Nk + 7) // 8 * 8                           # 16-byte aligned bias rows
+    Qb, Kb, Vb = rand_bits(rng, (B, H, Nq, d)), rand_bits(rng, (B, H, Nk, d)), rand_bits(rng, (B, H, Nk, d))
+    vl = None
+    if mask == 1:
+        vl = rng.integers(1, Nk + 1, size=B).astype(np.int32)
+    elif mask == 2:
+        vl = np.array([0, Nk, Nk // 2][:B], dtype=np.int32)
+    vlt = None if vl is None else torch.from_numpy(vl).cuda()
+    Q, K, V = bf16_tensor(Qb), bf16_tensor(Kb), bf16_tensor(Vb)
+    lead = [(B, H), (1, H), (B, 1), (1, 1)][int(rng.integers(0, 4))]
+    bf = (rng.standard_normal(lead + (Nq, Nk)) * 1.5).astype(np.float32)
+    bf[..., rng.integers(0, Nq), :] = -np.inf            # a whole row switched off
+    bf[..., :, rng.integers(0, Nk)] = -np.inf            # and a whole key
+    if rng.integers(0, 2):
+        bias = inputs.f32_to_bf16_bits(bf).reshape(bf.shape)
+        bt = bf16_tensor(bias)
+    else:
+        bias = bf
+        bt = torch.from_numpy(bf).cuda()
+    ref = oracle.attention(Qb, Kb, Vb, 0.2, valid_len=vl, causal=causal, bias=bias, want_lse=True)
+    for variant in (0, 1):
+        O = torch.full(Q.shape, float("nan"), dtype=torch.bfloat16, device="cuda")
+        lse = torch.full(Q.shape[:3], float("nan"), dtype=torch.float32, device="cuda")
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        api.flat_attn_fwd_ex(Q, K, V, O, 0.2, k_valid_len=vlt, status=status, variant=variant, causal=causal, bias=bt, lse=lse)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        check_bf16(bf16_to_f64(O), ref["O"], "fuzz bias %s variant %d" % (case[:7], variant))
+        dead = np.isneginf(ref["LSE"])
+        got = lse.double().cpu().numpy()
+        assert np.array_equal(np.isneginf(got), dead), (case[:7], variant)
+        if (~dead).any():
+            assert np.max(np.abs(got[~dead] - ref["LSE"][~dead])) < 2e-3
+    # pruning map
+    tq, tk = -(-Nq // 128), -(-Nk // 128)
+    mlead = [(B, H), (1, H), (B, 1), (1, 1)][int(rng.integers(0, 4))]
+    bm = (rng.random(mlead + (tq, tk)) < 0.6).astype(np.uint8)
+    refm = oracle.attention(Qb, Kb, Vb, 0.2, valid_len=vl, causal=causal, block_mask=bm, want_lse=True)
+    O = torch.full(Q.shape, float("nan"), dtype=torch.bfloat16, device="cuda")
+    lse = torch.full(Q.shape[:3], float("nan"), dtype=torch.float32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    api.flat_attn_fwd_ex(Q, K, V, O, 0.2, k_valid_len=vlt, status=status, causal=causal, block_mask=torch.from_numpy(bm).cuda(), lse=lse)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    check_bf16(bf16_to_f64(O), refm["O"], "fuzz pruning map %s" % (case[:7],))
+    dead = np.isneginf(refm["LSE"])
+    assert np.array_equal(np.isneginf(lse.double().cpu().numpy()), dead)
