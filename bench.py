@@ -290,6 +290,17 @@ class Bench:
         sampler = ClockSampler(self.dev.index).start() if sample_clocks else None
         total_ms, per = self.timed(step, steps, flush=w.qkvo_bytes() <= L2_FLUSH_BELOW)
         clocks = sampler.stop() if sampler else None
+        # a run that saw a hardware or thermal slowdown is not a measurement: taken once more after a pause
+        # (a power cap is normal on a 1 kW part and is kept and noted); every rank takes the same decision
+        # because the region is bracketed by barriers, and with one rank sampling it is that rank's alone
+        throttled = {"hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown"}
+        if clocks and self.world == 1 and throttled & set(clocks.get("reasons", [])):
+            time.sleep(5.0)
+            first = clocks
+            sampler = ClockSampler(self.dev.index).start()
+            total_ms, per = self.timed(step, steps, flush=w.qkvo_bytes() <= L2_FLUSH_BELOW)
+            clocks = sampler.stop()
+            clocks["remeasured_after"] = first.get("reasons", [])
         code = int(d["status"].item())
         assert code == 0, "device status 0x%x" % code
         return total_ms, per, kernel, clocks
