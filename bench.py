@@ -78,6 +78,7 @@ class ClockSampler:
         self.gpu = gpu_index
         self.proc = None
         self.lines = []
+        self.first = 0
 
     def start(self):
         q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
@@ -96,6 +97,12 @@ class ClockSampler:
         for ln in self.proc.stdout:
             self.lines.append(ln.strip())
 
+    def mark(self):
+        """Only samples taken from now on count (the sampler is started ahead of the warm-up launches, so that the
+        start-up of nvidia-smi does not fall into the timed region)."""
+        self.first = len(self.lines)
+        return self
+
     def stop(self):
         if not self.proc:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
@@ -107,7 +114,7 @@ class ClockSampler:
             self.proc.kill()
         sm, mx, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for ln in self.lines:
+        for ln in self.lines[self.first:]:
             f = [x.strip() for x in ln.split(",")]
             if len(f) < 6:
                 continue
@@ -284,10 +291,14 @@ class Bench:
         api = self.api
         step = lambda: api.flat_attn_fwd_ex(d["Q"], d["K"], d["V"], d["O"], w.scale, k_valid_len=d["vl"],
                                             status=d["status"], variant=self.variant)
+        sampler = ClockSampler(self.dev.index).start() if sample_clocks else None
+        if sampler:
+            time.sleep(0.3)                              # nvidia-smi attaches to the GPU: not during the launches
         for _ in range(warmup):
             step()
         kernel = KERNEL_OF_VARIANT.get(api.flat_attn_last_variant(), "?")
-        sampler = ClockSampler(self.dev.index).start() if sample_clocks else None
+        if sampler:
+            sampler.mark()
         total_ms, per = self.timed(step, steps, flush=w.qkvo_bytes() <= L2_FLUSH_BELOW)
         clocks = sampler.stop() if sampler else None
         # a run that saw a hardware or thermal slowdown is not a measurement: taken once more after a pause
@@ -298,6 +309,10 @@ class Bench:
             time.sleep(5.0)
             first = clocks
             sampler = ClockSampler(self.dev.index).start()
+            time.sleep(0.3)
+            for _ in range(warmup):
+                step()
+            sampler.mark()
             total_ms, per = self.timed(step, steps, flush=w.qkvo_bytes() <= L2_FLUSH_BELOW)
             clocks = sampler.stop()
             clocks["remeasured_after"] = first.get("reasons", [])
@@ -462,10 +477,12 @@ def run_backward(bench, torch, api, w, d, data, seed, args, peaks):
     api.flat_attn_fwd_ex(d["Q"], d["K"], d["V"], d["O"], w.scale, k_valid_len=d["vl"], status=d["status"], lse=lse)
     step = lambda: api.flat_attn_bwd_ex(d["Q"], d["K"], d["V"], d["O"], dO, lse, dQ, dK, dV, delta, w.scale,
                                         k_valid_len=d["vl"], status=d["status"])
+    sampler = ClockSampler(dev.index).start()
+    time.sleep(0.3)
     for _ in range(3):
         step()
     steps = int(max(3, min(args.steps, 10)))
-    sampler = ClockSampler(dev.index).start()
+    sampler.mark()
     total_ms, per = bench.timed(step, steps, flush=False)
     clocks = sampler.stop()
     assert int(d["status"].item()) == 0
@@ -502,11 +519,13 @@ def run_fp32(bench, torch, api, w, seed, args, peaks, dev):
     del host
     d["Q"] = d["K"] = d["V"] = d["O"] = None
     step = lambda: api.flat_attn_fwd_ex(Q, K, V, O, w.scale, k_valid_len=d["vl"], status=d["status"])
+    sampler = ClockSampler(dev.index).start()
+    time.sleep(0.3)
     for _ in range(3):
         step()
     kernel = KERNEL_OF_VARIANT.get(api.flat_attn_last_variant(), "?")
     steps = int(max(3, min(args.steps, 5)))
-    sampler = ClockSampler(dev.index).start()
+    sampler.mark()
     total_ms, per = bench.timed(step, steps, flush=False)
     clocks = sampler.stop()
     assert int(d["status"].item()) == 0
