@@ -720,12 +720,28 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
 #pragma unroll
                     for (int i = 0; i < 32; ++i) r[i] = 0u;      // no valid key: O = 0
                 }
-                if (VL ? row - it.row0 < it.q_rows : row < Nq) {
-                    uint32_t w[16];
+                uint32_t w[16];
 #pragma unroll
-                    for (int i = 0; i < 16; ++i)
-                        w[i] = pack_bf16x2(__uint_as_float(r[2 * i]) * inv, __uint_as_float(r[2 * i + 1]) * inv);
-                    if (wide_stores) {                   // (O is 32-byte aligned)
+                for (int i = 0; i < 16; ++i)
+                    w[i] = pack_bf16x2(__uint_as_float(r[2 * i]) * inv, __uint_as_float(r[2 * i + 1]) * inv);
+                if (!VL && wide_stores) {                // (O is 32-byte aligned; dense layout: rows 128 bytes apart)
+                    // Lane pairs swap one 32-byte sector each, so that a store instruction of the warp covers 16 rows
+                    // x 64 contiguous bytes instead of 32 rows x 32 bytes: the load/store unit takes a store one line
+                    // at a time, and the sixteen warps' stores are what an item boundary waits for.
+                    const bool odd = lane & 1;
+                    uint32_t a[8], b[8];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const uint32_t got = __shfl_xor_sync(0xffffffffu, odd ? w[i] : w[8 + i], 1);   // odd lanes give their first sector, even lanes their second
+                        a[i] = odd ? got : w[i];         // first instruction: the even lane's row (own first sector / the partner's second)
+                        b[i] = odd ? w[8 + i] : got;     // second instruction: the odd lane's row
+                    }
+                    const int row_e = row - (odd ? 1 : 0);
+                    __nv_bfloat16* even_row = orow - (odd ? D : 0);
+                    if (row_e < Nq) st_global_32B(even_row + c * 32 + (odd ? 16 : 0), a);
+                    if (row_e + 1 < Nq) st_global_32B(even_row + D + c * 32 + (odd ? 16 : 0), b);
+                } else if (VL ? row - it.row0 < it.q_rows : row < Nq) {
+                    if (wide_stores) {
                         st_global_32B(orow + c * 32, *reinterpret_cast<uint32_t(*)[8]>(&w[0]));
                         st_global_32B(orow + c * 32 + 16, *reinterpret_cast<uint32_t(*)[8]>(&w[8]));
                     } else {
