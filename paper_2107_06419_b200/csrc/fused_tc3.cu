@@ -59,7 +59,9 @@ constexpr float UNDERFLOW_SUM = 8.6736174e-19f; // 2^-60: a first-step sum below
 constexpr int SOFT_REGS = 104, OTHER_REGS = 64;
 static_assert(512 * SOFT_REGS + 128 * OTHER_REGS <= 640 * 96, "register hand-over exceeds the CTA's allocation");
 constexpr bool USE_POLY = true;          // part of the exponentials on the FMA pipe (see exp_pack_x2)
-constexpr unsigned POLY_PAIRS = 0x0202;  // bit i: pair i of each 16 pairs (32 logits) takes the polynomial; two pairs = one element in eight
+// bit i: pair i of the 16 pairs (32 logits) of a half step takes the polynomial; two pairs = one element in eight.
+// Which pairs is a matter of the instruction schedule only: all 120 two-pair masks were timed on c2 (958-981 TFLOP/s).
+constexpr unsigned POLY_PAIRS_A = 0x0210, POLY_PAIRS_B = 0x0210;   // first / second 32 logits of a thread's 64
 constexpr unsigned PRODUCER_SLEEP = 400; // ns between the TMA producer's probes of a full ring (it runs far ahead: its reaction time is immaterial)
 
 constexpr int D = 64;                // head size of this kernel
@@ -169,7 +171,7 @@ __device__ __forceinline__ void scale32(const uint32_t (&r)[32], uint64_t scale2
 // Part 2: p = 2^x, packed row sums, bf16 packing.  With POLY, pairs 1, 5, 9, 13 (one element in
 // four) take the polynomial instead of the ex2 unit and `xmax` follows the largest argument given
 // to it.  l2[0] sums elements 0, 1 (mod 4), l2[1] elements 2, 3.
-template <bool POLY>
+template <bool POLY, unsigned POLY_PAIRS = POLY_PAIRS_A>
 __device__ __forceinline__ void exp_pack_x2(const uint64_t (&x2)[16], uint64_t (&l2)[2], float& xmax, uint32_t (&pk)[16]) {
     float p[32];
 #pragma unroll
@@ -587,7 +589,7 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                     exp_pack_x2<USE_POLY>(x2, l2, xmax, pk[0]);
                     tc_wait_ld();
                     scale32(r, scale2, neg_m2, x2);
-                    exp_pack_x2<USE_POLY>(x2, l2, xmax, pk[1]);
+                    exp_pack_x2<USE_POLY, POLY_PAIRS_B>(x2, l2, xmax, pk[1]);
                     float a, b2, c, d2;
                     unpack2(l2[0], a, b2);
                     unpack2(l2[1], c, d2);
