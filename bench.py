@@ -46,7 +46,7 @@ TF32_OVER_BF16 = 1.1 / 2.25          # nominal dense tensor peaks: the tf32 roof
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel from ncu
 # captures, with the capture they come from; a (kernel, workload) pair without a capture reports null.
 MEASURED_DRAM_TRAFFIC = {
-    ("fused_tc3_kernel", "c2_bert_large_4k"): (514_200_000, "profiles/fused_tc3_kernel_dram_and_pipes.md"),
+    ("fused_tc3_kernel", "c2_bert_large_4k"): (515_300_000, "profiles/fused_tc3_kernel_dram_and_pipes.md"),
     ("fused_tc3_kernel", "p_4k_small"): (116_900_000, "profiles/fused_tc3_kernel_dram_and_pipes.md"),
     ("fused_tc2_kernel<2 tiles>", "c2_bert_large_4k"): (516_000_000, "profiles/fused_tc2_kernel_dram_and_pipes.md"),
     ("fused_tc2_kernel<2 tiles>", "p_4k_small"): (117_600_000, "profiles/fused_tc2_kernel_dram_and_pipes.md"),

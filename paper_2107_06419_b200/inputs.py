@@ -104,6 +104,8 @@ WORKLOADS = {
     "c5_cross_masked": Workload("c5_cross_masked", 8, 12, 1024, 16384, 64, masked=True),
     # reduced copies of c2 / c4 for profiler captures (same tile shapes, a few hundred MB at most)
     "p_4k_small": Workload("p_4k_small", 4, 16, 4096, 4096, 64),
+    # half of c2: 2048 row slabs, enough for the persistent grid (14 items per CTA on 148 SMs)
+    "p_4k_half": Workload("p_4k_half", 8, 16, 4096, 4096, 64),
     "p_16k_d128_small": Workload("p_16k_d128_small", 1, 4, 16384, 16384, 128),
 }
 
