@@ -361,6 +361,21 @@ int flat_attn_last_launch_count(void);
 int flat_attn_last_variant(void);
 
 /*
+ * How the most recent FLAT_VARIANT_TC3 launch on this host thread handed the work items (batch, head, slab of
+ * 256 query rows) to the SMs -- the tile order of the paper's Section 5.1 / 5.3: FLAT_SCHEDULE_ITEMS one CTA per
+ * item, FLAT_SCHEDULE_PERSISTENT one CTA per SM walking a fixed share of the items, FLAT_SCHEDULE_EVEN_DEAL one
+ * CTA per SM taking an equal share of the key steps of all items, items cut where a share ends and their
+ * partial softmaxes merged through the library's own device workspace (chosen for few items of unequal
+ * length -- key-padding masks -- or a last round that would stay mostly empty; not under the causal mask, not
+ * with the lse output, not during stream capture, not while a launch from another stream may still use the
+ * workspace).  0 before any such launch.
+ */
+#define FLAT_SCHEDULE_ITEMS 1
+#define FLAT_SCHEDULE_PERSISTENT 2
+#define FLAT_SCHEDULE_EVEN_DEAL 3
+int flat_attn_last_schedule(void);
+
+/*
  * Device-side give-up codes when the caller passed no `status` word (the paper has no
  * counterpart).  Every wait inside the tensor-core kernels is bounded (about a second of SM
  * clock, which also runs while a context is time-sliced out on a GPU shared with other

@@ -35,7 +35,9 @@ EXPORTS = ["flat_attn_fwd", "flat_attn_fwd_ex", "flat_attn_naive_fwd", "flat_att
            "flat_attn_status_string", "flat_attn_version",
            "flat_qkv_proj_fwd", "flat_out_proj_fwd", "flat_attn_layer_fwd", "flat_fc_fwd",
            "flat_attn_varlen_fwd", "flat_attn_last_variant", "flat_attn_last_device_error",
-           "flat_attn_clear_device_error", "flat_attn_bwd", "flat_attn_bwd_ex", "flat_layernorm_fwd"]
+           "flat_attn_clear_device_error", "flat_attn_bwd", "flat_attn_bwd_ex", "flat_layernorm_fwd",
+           "flat_attn_last_schedule"]
+FLAT_SCHEDULE_ITEMS, FLAT_SCHEDULE_PERSISTENT, FLAT_SCHEDULE_EVEN_DEAL = 1, 2, 3
 
 
 class flat_attn_params_t(ctypes.Structure):
@@ -96,6 +98,7 @@ _lib.flat_attn_host_workspace_bytes.argtypes = [_i, _i, _i, _i, _i, _i]
 _lib.flat_attn_host_workspace_bytes.restype = ctypes.c_size_t
 _lib.flat_attn_last_launch_count.restype = _i
 _lib.flat_attn_last_variant.restype = _i
+_lib.flat_attn_last_schedule.restype = _i
 _lib.flat_attn_last_device_error.argtypes = [ctypes.POINTER(ctypes.c_int32)]
 _lib.flat_attn_last_device_error.restype = _i
 _lib.flat_attn_clear_device_error.restype = _i
@@ -125,6 +128,11 @@ def flat_attn_last_launch_count() -> int:
 def flat_attn_last_variant() -> int:
     """The FLAT_VARIANT_* the most recent fused call on this thread ran (what AUTO resolved to)."""
     return int(_lib.flat_attn_last_variant())
+
+
+def flat_attn_last_schedule() -> int:
+    """FLAT_SCHEDULE_* of the most recent FLAT_VARIANT_TC3 launch on this thread (how its items went to the SMs)."""
+    return int(_lib.flat_attn_last_schedule())
 
 
 def flat_attn_last_device_error() -> int:

@@ -454,6 +454,8 @@ int flat_attn_last_launch_count(void) { return g_last_launches; }
 
 int flat_attn_last_variant(void) { return g_last_variant; }
 
+int flat_attn_last_schedule(void) { return flat::g_last_schedule; }
+
 int flat_attn_last_device_error(int32_t* code) {
     if (!code) return FLAT_ERR_NULL;
     int32_t* w = library_status_word();

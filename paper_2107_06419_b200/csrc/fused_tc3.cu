@@ -38,6 +38,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <mutex>
+
 #include "flat_internal.cuh"
 #include "ptx_sm100.cuh"
 #include "tc_common.cuh"
@@ -63,6 +65,7 @@ constexpr bool USE_POLY = true;          // part of the exponentials on the FMA 
 // Which pairs is a matter of the instruction schedule only: all 120 two-pair masks were timed on c2 with the
 // descending sum loop of exp_pack_x2 (960-986 TFLOP/s), then the 20 mixed choices among the best five.
 constexpr unsigned POLY_PAIRS_A = 0x0900, POLY_PAIRS_B = 0x0900;   // first / second 32 logits of a thread's 64
+constexpr unsigned POLY_PAIRS_SA = 0x0900, POLY_PAIRS_SB = 0x0900; // the same for the even-deal instantiation (timed on c5)
 constexpr unsigned PRODUCER_SLEEP = 400; // ns between the TMA producer's probes of a full ring (it runs far ahead: its reaction time is immaterial)
 
 constexpr int D = 64;                // head size of this kernel
@@ -77,7 +80,7 @@ struct L3 {
     static constexpr int KV_BYTES = BN * D * 2;
     static constexpr int TILE_BYTES = 2 * Q_BYTES + (KS + VS) * KV_BYTES;
     static constexpr int XCH_BYTES = 2 * 2 * 2 * BM * 4; // [maximum | row sum][tile][half][row] floats
-    static constexpr int SMEM_BYTES = TILE_BYTES + XCH_BYTES + 512 + 1024;
+    static constexpr int SMEM_BYTES = TILE_BYTES + XCH_BYTES + 512 + 512 + 1024;   // (.. barriers, the even deal's table, alignment)
     __host__ __device__ static constexpr uint32_t O_COL(int t) { return 64u * t; }
     __host__ __device__ static constexpr uint32_t X_COL(int b) { return 128u + 128u * b; }   // logit / weight buffer b
     // barrier indices
@@ -228,9 +231,43 @@ __device__ __forceinline__ void exp_pack32(const uint32_t (&r)[32], float scale_
 struct Item {
     int bh, row0, n, ntiles;                             // n = number of keys that any row of the slab sees, ntiles = key steps
     bool skip;                                           // an empty slot of the paired order: no rows to write either
+    int tile0;                                           // first key step of the item that this CTA takes (even deal: see EvenDeal)
     // packed variable-length batches only:
     int head, q_tok0, k_tok0, q_rows, coff;              // head; first token of the slab's rows / of the sequence's keys; rows of the sequence from row0 on; Nk - Nq of the sequence
 };
+// The even deal (template parameter SPLIT), for launches whose items would fill the SMs badly when dealt whole:
+// few items of different length (key-padding masks: the hardware hands out whole items, and the last SM to get
+// a long one finishes long after the others), or a number of equal items that leaves the last round mostly empty.
+// Every item (b, h, slab) has L_b key steps (at least one, so that a batch without valid keys still gets its
+// zero rows written); the key steps of all items, T of them in item order, are cut into gridDim.x equal ranges
+// and CTA c takes steps c T / grid .. (c + 1) T / grid - 1: the end of one item, whole items, the beginning of
+// one more.  The CTA whose range holds an item's first key step writes the item's rows; every other part of the
+// item leaves its un-normalised (m_ref, l, O) in the workspace slot of its CTA -- a CTA has at most one such
+// part, its first -- and raises that slot's flags to the launch's epoch, and the writer merges them (the
+// split-merge identity of the streaming softmax).  A CTA works through its range in order, so the part it leaves
+// for somebody else comes first and the part it must wait for others on comes last; CTA c only ever waits for
+// CTAs of a higher number: no cycle, and every wait is bounded.
+// Teams: the slabs of a head read the same K and V, and CTAs that hold them at the same key step share those
+// tiles in L2.  Dealt item by item, neighbouring CTAs would sit at different key steps of the same head and every
+// tile would come from DRAM once per slab (measured: no gain at all on the masked workload).  So the unit that is
+// dealt is the head -- all its slabs -- and a team of `team` = slabs CTAs takes a range of head key steps, member
+// s of the team working on slab s; team = 1 deals single items.
+struct EvenDeal {
+    int team;
+    int epoch;
+    float* ws;                                           // [gridDim.x][WS_FLOATS]
+    int* flags;                                          // [gridDim.x][16 softmax warps]
+};
+// A slot of the workspace: O as [tile][key half][row group][32 columns][32 lanes] fp32, then per tile, key half
+// and row group 32 reference maxima and 32 row sums -- every thread reads back what the thread of the same role
+// wrote, so a warp waits for the flag of the other CTA's warp of the same number and for nothing else.
+constexpr int WS_O_FLOATS = 2 * 2 * 4 * 32 * 32, WS_FLOATS = WS_O_FLOATS + 2 * 2 * 4 * 64;
+constexpr int WS_MAX_CTAS = 160;
+// The deal's table in shared memory (filled by one warp before the roles start): this CTA's range lo, hi, its
+// first item and the one after its last, T, and from DEAL_PREFIX on the number of key steps before batch b's
+// items for b = 0 .. B (DEAL_MAX_B batches at most).
+constexpr int DEAL_LO = 0, DEAL_HI = 1, DEAL_FIRST = 2, DEAL_END = 3, DEAL_T = 4, DEAL_TEAM = 5, DEAL_TEAMS = 6, DEAL_PREFIX = 8, DEAL_MAX_B = 64;
+static_assert((DEAL_PREFIX + DEAL_MAX_B + 1) * 4 <= 512, "the deal's table has 512 bytes of shared memory");
 // What every role needs to enumerate the items.
 struct Sched {
     int items, slabs, H, Nk;
@@ -239,22 +276,141 @@ struct Sched {
     int paired;                                          // items come in pairs of complementary slabs (see get_item)
     const int32_t* cu_q;                                 // packed variable-length batches: first token of every sequence's
     const int32_t* cu_k;                                 // queries / keys in the packed tensors ([sequences + 1] entries)
+    const int* deal;                                     // even deal: its table in shared memory
+    EvenDeal ed;
 };
+// Even deal: first key step of team g's range, of `teams` (g T < 2^32: the launcher checks).
+__device__ __forceinline__ int deal_lo(int T, int g, int teams) {
+    return static_cast<int>(static_cast<unsigned>(g) * static_cast<unsigned>(T) / static_cast<unsigned>(teams));
+}
+// Even deal: where item idx (its unit: the item, or its head) sits in the sequence of all key steps.
+__device__ __forceinline__ void deal_item_range(const Sched& sc, int idx, int& start, int& end) {
+    const int team = sc.deal[DEAL_TEAM], u = idx / team;
+    const int per = sc.H * sc.slabs / team, b = u / per, k = u - b * per;
+    const int p0 = sc.deal[DEAL_PREFIX + b], Lb = (sc.deal[DEAL_PREFIX + b + 1] - p0) / per;
+    start = p0 + k * Lb;
+    end = start + Lb;
+}
+// Even deal: what the softmax warps do with the rows of item idx when this CTA's key steps of it are done:
+// 0 normalise and store them (the CTA had the whole item), 2 leave them in this CTA's slot, 1 merge the slots of
+// CTAs first, first + team, ... (count of them: the same member of the following teams, whose ranges cover the
+// rest of the item) and store.
+__device__ __forceinline__ void deal_role(const Sched& sc, int idx, int& part, int& first, int& count) {
+    int start, end;
+    deal_item_range(sc, idx, start, end);
+    const int team = sc.deal[DEAL_TEAM], teams = sc.deal[DEAL_TEAMS], g = static_cast<int>(blockIdx.x) / team;
+    part = 0; first = static_cast<int>(blockIdx.x) + team; count = 0;
+    if (sc.deal[DEAL_LO] > start) { part = 2; return; }
+    if (sc.deal[DEAL_HI] < end) {
+        const int T = sc.deal[DEAL_T];
+        while (g + 1 + count < teams && deal_lo(T, g + 1 + count, teams) < end) ++count;
+        part = count > 0 ? 1 : 0;
+    }
+}
+// A warp waits until `*flag` holds the launch's epoch (lane 0 polls; bounded like every other wait of the kernel).
+__device__ __forceinline__ bool wait_flag_warp(const int* flag, int epoch, uint32_t abort_addr, int32_t* status, int code) {
+    bool ok = true;
+    if ((threadIdx.x & 31) == 0) {
+        const long long t0 = clock64();
+        for (;;) {
+            int v, aborted;
+            asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
+            if (v == epoch) break;
+            asm volatile("ld.volatile.shared::cta.s32 %0, [%1];" : "=r"(aborted) : "r"(abort_addr) : "memory");
+            if (aborted) { ok = false; break; }
+            if (clock64() - t0 > WAIT_CYCLES) {
+                asm volatile("st.volatile.shared::cta.s32 [%0], %1;" ::"r"(abort_addr), "r"(1) : "memory");
+                if (status) atomicExch(status, code);
+                ok = false;
+                break;
+            }
+            __nanosleep(100);
+        }
+    }
+    ok = __all_sync(0xffffffffu, ok);
+    __syncwarp();
+    __threadfence();
+    return ok;
+}
+// A part that begins inside its item: the un-normalised rows (this thread: 32 columns of one row, from TMEM
+// address `o_addr`), their reference and their sums go to this CTA's slot for the CTA that holds the item's
+// beginning.  `role` = (tile * 2 + key half) * 4 + row group.
+__device__ __noinline__ void deal_write_partial(const EvenDeal ed, uint32_t o_addr, int role, float m_ref, float l) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    float* slot = ed.ws + static_cast<size_t>(blockIdx.x) * WS_FLOATS;
+    float* po = slot + role * 1024 + lane;
+    float* pm = slot + WS_O_FLOATS + role * 64 + lane;
+    uint32_t r[32];
+    tmem_ld_x32(o_addr, r);
+    tc_wait_ld();
+#pragma unroll
+    for (int i = 0; i < 32; ++i) po[i * 32] = __uint_as_float(r[i]);
+    pm[0] = m_ref;
+    pm[32] = l;
+    __threadfence();
+    __syncwarp();
+    if (lane == 0)
+        asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(ed.flags + blockIdx.x * 16 + warp), "r"(ed.epoch) : "memory");
+}
+// The part that begins its item: (m, l, O) of two parts merge as m = max, l = sum of l_i 2^(m_i - m), O likewise
+// (the row-wise softmax of Section 5.2, split along the keys); then 1/l and the store of this thread's 32 columns.
+// A part without a valid key carries m = -inf and l = 0 and drops out of the merge.
+__device__ __noinline__ void deal_finish_merged(const EvenDeal ed, uint32_t o_addr, int role, float m_ref, float l, int pfirst,
+                                                int pcount, __nv_bfloat16* orow, bool row_valid, uint32_t abort_s, int32_t* status) {
+    // (partner CTAs: pfirst, pfirst + team, ...)
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint32_t r[32];
+    tmem_ld_x32(o_addr, r);
+    tc_wait_ld();
+    float mm = m_ref;
+    for (int pi = 0; pi < pcount; ++pi) {
+        const int cp = pfirst + pi * ed.team;
+        if (!wait_flag_warp(ed.flags + cp * 16 + warp, ed.epoch, abort_s, status, 0x360)) break;
+        const float* slot = ed.ws + static_cast<size_t>(cp) * WS_FLOATS;
+        const float* po = slot + role * 1024 + lane;
+        const float* pm = slot + WS_O_FLOATS + role * 64 + lane;
+        const float m2 = __ldcg(pm), l2 = __ldcg(pm + 32);
+        const float mn = fmaxf(mm, m2);
+        const float fa = mm == -INFINITY ? 0.f : ex2_approx(mm - mn), fb = m2 == -INFINITY ? 0.f : ex2_approx(m2 - mn);
+        l = l * fa + l2 * fb;
+#pragma unroll
+        for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * fa + __ldcg(po + i * 32) * fb);
+        mm = mn;
+    }
+    const float inv = l > 0.f ? 1.f / l : 0.f;
+    if (row_valid) {
+#pragma unroll
+        for (int v = 0; v < 4; ++v) {
+            uint32_t w[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                w[i] = pack_bf16x2(__uint_as_float(r[8 * v + 2 * i]) * inv, __uint_as_float(r[8 * v + 2 * i + 1]) * inv);
+            *reinterpret_cast<uint4*>(orow + v * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+    }
+}
 // The sequence of item indices of this CTA: blockIdx.x, blockIdx.x + gridDim.x, ...; in paired mode the
 // CTA takes PAIRS of consecutive indices (2 c, 2 c + 1), (2 (c + gridDim.x), ...), ...
-__device__ __forceinline__ int first_item(const Sched& sc) { return sc.paired ? 2 * blockIdx.x : blockIdx.x; }
+template <bool SPLIT = false>
+__device__ __forceinline__ int first_item(const Sched& sc) {
+    if (SPLIT) return sc.deal[DEAL_FIRST];
+    return sc.paired ? 2 * blockIdx.x : blockIdx.x;
+}
+template <bool SPLIT = false>
 __device__ __forceinline__ int next_item(int idx, const Sched& sc) {
+    if (SPLIT) return idx + sc.deal[DEAL_TEAM];
     return sc.paired ? ((idx & 1) ? idx - 1 + 2 * static_cast<int>(gridDim.x) : idx + 1) : idx + static_cast<int>(gridDim.x);
 }
 // VL (packed variable-length batches): Q, O are [total_q, H, d], K, V [total_k, H, d]; sequence s owns
 // tokens cu_q[s] .. cu_q[s+1] - 1 of Q and cu_k[s] .. cu_k[s+1] - 1 of K, V.  Item index =
 // (sequence * H + head) * slabs + slab with `slabs` taken from the longest sequence; a slab past the
 // end of its sequence is an empty slot.  The causal offset is that of the sequence.
-template <bool VL>
+template <bool VL, bool SPLIT = false>
 __device__ __forceinline__ Item get_item(int idx, const Sched& sc) {
     Item it;
     int slab;
     bool empty = false;
+    it.tile0 = 0;
     if (VL) {
         it.bh = idx / sc.slabs;
         slab = idx - it.bh * sc.slabs;
@@ -303,6 +459,14 @@ __device__ __forceinline__ Item get_item(int idx, const Sched& sc) {
     it.skip = empty;
     it.n = n;
     it.ntiles = (n + BN - 1) / BN;
+    if (SPLIT) {
+        // this CTA's share of the item's key steps (an item without a valid key counts one step, fully masked)
+        int start, end;
+        deal_item_range(sc, idx, start, end);
+        const int lo = sc.deal[DEAL_LO] > start ? sc.deal[DEAL_LO] : start, hi = sc.deal[DEAL_HI] < end ? sc.deal[DEAL_HI] : end;
+        it.tile0 = lo - start;
+        it.ntiles = hi - lo;
+    }
     return it;
 }
 // Position of a role in the CTA's sequence of key steps.  Items without a valid key have no steps
@@ -314,27 +478,27 @@ struct Cursor {
     Item it;
     bool valid;
 };
-template <bool VL>
+template <bool VL, bool SPLIT = false>
 __device__ __forceinline__ void cursor_seek(Cursor& c, const Sched& sc) {
     c.valid = false;
     while (c.idx < sc.items) {
-        c.it = get_item<VL>(c.idx, sc);
+        c.it = get_item<VL, SPLIT>(c.idx, sc);
         if (c.it.ntiles > 0) { c.valid = true; return; }
-        c.idx = next_item(c.idx, sc);
+        c.idx = next_item<SPLIT>(c.idx, sc);
     }
 }
-template <bool VL>
+template <bool VL, bool SPLIT = false>
 __device__ __forceinline__ void cursor_init(Cursor& c, const Sched& sc) {
-    c.idx = first_item(sc); c.j = 0; c.J = 0; c.q = 0;
-    cursor_seek<VL>(c, sc);
+    c.idx = first_item<SPLIT>(sc); c.j = 0; c.J = 0; c.q = 0;
+    cursor_seek<VL, SPLIT>(c, sc);
 }
-template <bool VL>
+template <bool VL, bool SPLIT = false>
 __device__ __forceinline__ void cursor_next(Cursor& c, const Sched& sc) {
     ++c.j; ++c.J;
     if (c.j == c.it.ntiles) {
         c.j = 0; ++c.q;
-        c.idx = next_item(c.idx, sc);
-        cursor_seek<VL>(c, sc);
+        c.idx = next_item<SPLIT>(c.idx, sc);
+        cursor_seek<VL, SPLIT>(c, sc);
     }
 }
 
@@ -343,15 +507,18 @@ __device__ __forceinline__ void cursor_next(Cursor& c, const Sched& sc) {
 // WLSE: also writes lse[b,h,i] = log of row i's sum of exponentials (dense batches; what the
 // backward pass takes from the forward one).  A separate instantiation, so that the plain forward
 // kernel is compiled exactly as it is without the output.
-template <bool VL, bool WLSE = false>
+// SPLIT: the even deal by key steps (see EvenDeal; dense batches, no causal mask, B <= DEAL_MAX_B; `items` is the
+// number of items, B * H * slabs, and the grid must not exceed the SMs that can hold a CTA each).
+template <bool VL, bool WLSE = false, bool SPLIT = false>
 __global__ void __launch_bounds__(L3::THREADS, 1)
 fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                  const __grid_constant__ CUtensorMap tmV, __nv_bfloat16* __restrict__ O, int H, int Nq, int Nk,
                  int items, int slabs, float scale_log2e, const int32_t* __restrict__ valid_len, int coff,
                  int32_t* status, int wide_stores, int paired, const int32_t* __restrict__ cu_q,
-                 const int32_t* __restrict__ cu_k, float* __restrict__ lse) {
+                 const int32_t* __restrict__ cu_k, float* __restrict__ lse, const EvenDeal ed) {
     using LY = L3;
-    const Sched sc{items, slabs, H, Nk, valid_len, coff, paired, cu_q, cu_k};
+    static_assert(!SPLIT || (!VL && !WLSE), "the even deal is built for the plain dense forward kernel only");
+    Sched sc{items, slabs, H, Nk, valid_len, coff, paired, cu_q, cu_k, nullptr, ed};
     if (VL && static_cast<int>(gridDim.x) == items) {
         // one CTA per slot: a slot past the end of its sequence leaves before anything is set up
         if (get_item<VL>(blockIdx.x, sc).skip) return;
@@ -365,6 +532,7 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     uint64_t* bars = reinterpret_cast<uint64_t*>(base + LY::TILE_BYTES + LY::XCH_BYTES);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + LY::NUM_BARS);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    int* deal = reinterpret_cast<int*>(base + LY::TILE_BYTES + LY::XCH_BYTES + 512);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -376,10 +544,56 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         fence_mbar_init();
     }
     if (warp == 0) { tmem_alloc(tmem_slot, LY::TMEM_COLS); tmem_relinquish(); }
+    if (SPLIT && warp == 1) {
+        // The deal's table.  Batch b's items have L_b = max(1, key steps of its valid keys) steps each; two
+        // batches per lane, prefix sums by shuffles.
+        const int team = ed.team, teams = static_cast<int>(gridDim.x) / team;
+        const int B = items / (H * slabs), per = H * slabs / team;      // units (items or heads) per batch
+        int v[2];
+#pragma unroll
+        for (int k = 0; k < 2; ++k) {
+            const int b = lane + 32 * k;
+            int n = Nk;
+            if (valid_len && b < B) { n = valid_len[b]; n = n < 0 ? 0 : (n > Nk ? Nk : n); }
+            const int L = (n + BN - 1) / BN;
+            v[k] = b < B ? (L > 0 ? L : 1) * per : 0;
+        }
+        int carry = 0;
+#pragma unroll
+        for (int k = 0; k < 2; ++k) {
+            int x = v[k];
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int y = __shfl_up_sync(0xffffffffu, x, o);
+                if (lane >= o) x += y;
+            }
+            deal[DEAL_PREFIX + 1 + lane + 32 * k] = carry + x;          // steps before batch lane + 32 k + 1
+            carry += __shfl_sync(0xffffffffu, x, 31);
+        }
+        __syncwarp();
+        if (lane == 0) {
+            deal[DEAL_PREFIX] = 0;
+            const int T = deal[DEAL_PREFIX + B];
+            // (CTAs beyond the last whole team have nothing to do)
+            const int g = static_cast<int>(blockIdx.x) / team, member = static_cast<int>(blockIdx.x) - g * team;
+            const int lo = g < teams ? deal_lo(T, g, teams) : 0, hi = g < teams ? deal_lo(T, g + 1, teams) : 0;
+            // the unit that holds key step x: the batch by its prefix, the unit within the batch by division
+            auto unit_of = [&](int x) {
+                int b = 0;
+                while (b + 1 < B && deal[DEAL_PREFIX + b + 1] <= x) ++b;
+                const int p0 = deal[DEAL_PREFIX + b], Lb = (deal[DEAL_PREFIX + b + 1] - p0) / per;
+                return b * per + (x - p0) / Lb;
+            };
+            deal[DEAL_LO] = lo; deal[DEAL_HI] = hi; deal[DEAL_T] = T; deal[DEAL_TEAM] = team; deal[DEAL_TEAMS] = teams;
+            deal[DEAL_FIRST] = hi > lo ? unit_of(lo) * team + member : 0;
+            deal[DEAL_END] = hi > lo ? (unit_of(hi - 1) + 1) * team : 0;
+        }
+    }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
+    if (SPLIT) { sc.deal = deal; sc.items = deal[DEAL_END]; items = deal[DEAL_END]; }
 
     if (warp >= LY::SOFT_WARPS) {
       asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(OTHER_REGS));
@@ -419,13 +633,13 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                 v_issued = J + 1;
             };
             int J0 = 0, q = 0;
-            for (int idx = first_item(sc); idx < items && ok; idx = next_item(idx, sc)) {
-                const Item it = get_item<VL>(idx, sc);
+            for (int idx = first_item<SPLIT>(sc); idx < items && ok; idx = next_item<SPLIT>(idx, sc)) {
+                const Item it = get_item<VL, SPLIT>(idx, sc);
                 if (it.ntiles == 0) continue;
                 // tile of query rows r.. / of keys of step j
                 auto qy = [&](int r) { return VL ? it.head : r; };
                 auto qz = [&](int r) { return VL ? it.q_tok0 + (r - it.row0) : it.bh; };
-                auto ky = [&](int j) { return VL ? it.head : j * BN; };
+                auto ky = [&](int j) { return VL ? it.head : (it.tile0 + j) * BN; };
                 auto kz = [&](int j) { return VL ? it.k_tok0 + j * BN : it.bh; };
                 load_q(0, q, qy(it.row0), qz(it.row0));
                 if (ok) load_k(J0, ky(0), kz(0));
@@ -463,7 +677,7 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             if (ok) tc_fence_after();
         };
         Cursor c;
-        cursor_init<VL>(c, sc);
+        cursor_init<VL, SPLIT>(c, sc);
         if (warp == LY::SOFT_WARPS + 3) {
             const uint64_t q_desc = make_smem_desc_sw128(smem_u32(Qs), 16, 1024);
             const uint64_t k_desc = make_smem_desc_sw128(smem_u32(Ks), 16, 1024);
@@ -490,7 +704,7 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                     }
                     __syncwarp();
                 }
-                cursor_next<VL>(c, sc);
+                cursor_next<VL, SPLIT>(c, sc);
             }
         } else {
             const int t = warp - LY::SOFT_WARPS - 1;
@@ -511,7 +725,7 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                     tc_commit(&bars[LY::V_EMPTY + vs]);
                 }
                 __syncwarp();
-                cursor_next<VL>(c, sc);
+                cursor_next<VL, SPLIT>(c, sc);
             }
         }
       }
@@ -537,14 +751,16 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         // of the CTA and items whose first step is partly masked start from an exact maximum.
         float m_ref = -INFINITY;
         bool first_item_done = false;
-        for (int idx = first_item(sc); idx < items; idx = next_item(idx, sc)) {
-        const Item it = get_item<VL>(idx, sc);
+        for (int idx = first_item<SPLIT>(sc); idx < items; idx = next_item<SPLIT>(idx, sc)) {
+        const Item it = get_item<VL, SPLIT>(idx, sc);
         if (it.skip) continue;
         const int ntiles = it.ntiles;
         // keys this thread's row sees (all the item's keys unless the causal mask cuts the row short);
         // lane 0 has the shortest row of the warp, so its count tells whether a step needs the masked routine
         const long long rlim = static_cast<long long>(it.row0) + t * BM + q * 32 + lane + 1 + (VL ? it.coff : sc.coff);
-        const int nrow = rlim < it.n ? (rlim < 0 ? 0 : static_cast<int>(rlim)) : it.n;
+        // (a part of the even deal counts its keys from its own first step)
+        const int nrow_item = rlim < it.n ? (rlim < 0 ? 0 : static_cast<int>(rlim)) : it.n;
+        const int nrow = SPLIT ? (nrow_item > it.tile0 * BN ? nrow_item - it.tile0 * BN : 0) : nrow_item;
         const int nrow_min = __shfl_sync(0xffffffffu, nrow, 0);
         float l = 0.f;
         const bool exact_first = !first_item_done || sc.coff < (1 << 29) || it.n < BN;   // (the same for all warps)
@@ -589,10 +805,10 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                     float xmax = 0.f;
                     scale32(r, scale2, neg_m2, x2);
                     tmem_ld_x32(s_addr + 32, r);         // the second 32 logits arrive during the first 32 exponentials
-                    exp_pack_x2<USE_POLY>(x2, l2, xmax, pk[0]);
+                    exp_pack_x2<USE_POLY, SPLIT ? POLY_PAIRS_SA : POLY_PAIRS_A>(x2, l2, xmax, pk[0]);
                     tc_wait_ld();
                     scale32(r, scale2, neg_m2, x2);
-                    exp_pack_x2<USE_POLY, POLY_PAIRS_B>(x2, l2, xmax, pk[1]);
+                    exp_pack_x2<USE_POLY, SPLIT ? POLY_PAIRS_SB : POLY_PAIRS_B>(x2, l2, xmax, pk[1]);
                     float a, b2, c, d2;
                     unpack2(l2[0], a, b2);
                     unpack2(l2[1], c, d2);
@@ -705,6 +921,22 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         st_shared_f32(xm_own + 4 * BM * 4, l);
         pair_sync(pair_id);
         l += ld_shared_f32((xm_own ^ (BM * 4)) + 4 * BM * 4);
+        if (SPLIT) {
+            // an item shared with other CTAs: out of line, the code of whole items stays as it is
+            int part, pfirst, pcount;
+            deal_role(sc, idx, part, pfirst, pcount);
+            if (part != 0) {
+                tc_fence_after();
+                if (part == 2)
+                    deal_write_partial(sc.ed, tl + LY::O_COL(t) + h * (D / 2), (t * 2 + h) * 4 + q, m_ref, l);
+                else
+                    deal_finish_merged(sc.ed, tl + LY::O_COL(t) + h * (D / 2), (t * 2 + h) * 4 + q, m_ref, l, pfirst, pcount,
+                                       O + (static_cast<int64_t>(it.bh) * Nq + it.row0 + t * BM + q * 32 + lane) * D + h * (D / 2),
+                                       it.row0 + t * BM + q * 32 + lane < Nq, abort_s, status);
+                tc_fence_before();
+                continue;
+            }
+        }
         {
             const int row = it.row0 + t * BM + q * 32 + lane;
             const float inv = l > 0.f ? 1.f / l : 0.f;
@@ -768,6 +1000,64 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     if (warp == 0) tmem_dealloc(tmem, LY::TMEM_COLS);
 }
 
+// The even deal's workspace: one slot and sixteen flags per CTA, in the library's own device memory (nothing is
+// allocated at run time).  The flags hold the epoch of the launch that last wrote the slot; epochs only grow, so
+// nothing is ever reset.  One workspace per device: a launch may use it when no launch from another stream can
+// still be using it (an event recorded behind every user tells), and not during stream capture (a captured launch
+// could be replayed beside anything); otherwise the launch deals whole items as before.
+__device__ float g_deal_ws[static_cast<size_t>(WS_MAX_CTAS) * WS_FLOATS];
+__device__ int g_deal_flags[WS_MAX_CTAS * 16];
+struct DealOwner {
+    bool ready = false, used = false;
+    float* ws = nullptr;
+    int* flags = nullptr;
+    cudaEvent_t ev = nullptr;
+    cudaStream_t last = nullptr;
+};
+std::mutex g_deal_mu;
+DealOwner g_deal[64];
+int g_deal_epoch = 0;
+
+// Fills `ed` (workspace, flags, a fresh epoch) if a launch on `st` may use the current device's workspace; the
+// caller launches and calls deal_release() while `lock` is still held.
+bool deal_acquire(cudaStream_t st, EvenDeal& ed, std::unique_lock<std::mutex>& lock) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return false;
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(st, &cap) != cudaSuccess || cap != cudaStreamCaptureStatusNone) return false;
+    lock = std::unique_lock<std::mutex>(g_deal_mu);
+    DealOwner& o = g_deal[dev];
+    if (!o.ready) {
+        void *w = nullptr, *f = nullptr;
+        if (cudaGetSymbolAddress(&w, g_deal_ws) != cudaSuccess || cudaGetSymbolAddress(&f, g_deal_flags) != cudaSuccess ||
+            cudaEventCreateWithFlags(&o.ev, cudaEventDisableTiming) != cudaSuccess) {
+            cudaGetLastError();
+            lock.unlock();
+            return false;
+        }
+        o.ws = static_cast<float*>(w);
+        o.flags = static_cast<int*>(f);
+        o.ready = true;
+    }
+    if (o.used && o.last != st && cudaEventQuery(o.ev) != cudaSuccess) {
+        cudaGetLastError();                              // (not ready: another stream's launch may still be running)
+        lock.unlock();
+        return false;
+    }
+    ed.ws = o.ws;
+    ed.flags = o.flags;
+    if (g_deal_epoch == 0x7fffffff) g_deal_epoch = 0;
+    ed.epoch = ++g_deal_epoch;
+    return true;
+}
+void deal_release(cudaStream_t st) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return;
+    DealOwner& o = g_deal[dev];
+    o.used = cudaEventRecord(o.ev, st) == cudaSuccess;
+    o.last = st;
+}
+
 int launch_tc3(const Problem& p, cudaStream_t st) {
     using LY = L3;
     CUtensorMap tmQ, tmK, tmV;
@@ -796,17 +1086,44 @@ int launch_tc3(const Problem& p, cudaStream_t st) {
     const int64_t slots = paired ? static_cast<int64_t>((slabs + 1) & ~1) * BH : items;
     if (slots > 0x7fffffff) return FLAT_ERR_SHAPE;
     const int grid = static_cast<int>(persistent ? sms : items);
+    // Too few items for the fixed deal: whole items handed out by the hardware leave SMs idle when the items differ
+    // in length (key-padding masks) or when the last round is mostly empty; the key steps are dealt evenly instead
+    // (EvenDeal), if the average share is long enough to carry the two extra item boundaries.
+    if (!persistent && !p.causal && !p.lse && p.B <= DEAL_MAX_B && sms <= WS_MAX_CTAS && items > 0) {
+        const int64_t nt = (p.Nk + BN - 1) / BN, rounds = (items + sms - 1) / sms;
+        const bool ragged = p.k_valid_len != nullptr || 4 * items < 3 * rounds * sms;   // (unmasked: under three quarters of the rounds filled)
+        // teams of `slabs` CTAs if they fill nine SMs in ten; single items only where K and V of all heads stay in L2
+        EvenDeal ed{};
+        const bool teams_fit = slabs <= sms && 10 * ((sms / slabs) * slabs) >= 9 * sms;
+        const bool kv_in_l2 = 4 * static_cast<int64_t>(BH) * p.Nk * D <= (48ll << 20);
+        ed.team = teams_fit ? slabs : 1;
+        std::unique_lock<std::mutex> lock;
+        if (ragged && (teams_fit || kv_in_l2) && items * nt >= 16 * static_cast<int64_t>(sms) && items * nt * (sms + 1) < (1ll << 32) &&
+            ensure_dynamic_smem<fused_tc3_kernel<false, false, true>>(LY::SMEM_BYTES) && deal_acquire(st, ed, lock)) {
+            fused_tc3_kernel<false, false, true><<<sms, LY::THREADS, LY::SMEM_BYTES, st>>>(
+                tmQ, tmK, tmV, static_cast<__nv_bfloat16*>(p.O), p.H, p.Nq, p.Nk, static_cast<int>(items), slabs,
+                p.scale * 1.4426950408889634f, p.k_valid_len, 1 << 30, p.status,
+                (reinterpret_cast<uintptr_t>(p.O) & 31) == 0 ? 1 : 0, 0, nullptr, nullptr, nullptr, ed);
+            const bool launched = cudaGetLastError() == cudaSuccess;
+            deal_release(st);
+            g_last_schedule = FLAT_SCHEDULE_EVEN_DEAL;
+            return launched ? FLAT_OK : FLAT_ERR_CUDA;
+        }
+    }
+    g_last_schedule = persistent ? FLAT_SCHEDULE_PERSISTENT : FLAT_SCHEDULE_ITEMS;
     auto kern = p.lse ? fused_tc3_kernel<false, true> : fused_tc3_kernel<false, false>;
     kern<<<grid, LY::THREADS, LY::SMEM_BYTES, st>>>(tmQ, tmK, tmV, static_cast<__nv_bfloat16*>(p.O), p.H, p.Nq, p.Nk,
                                                     static_cast<int>(slots), slabs, p.scale * 1.4426950408889634f,
                                                     p.k_valid_len, p.causal ? p.Nk - p.Nq : (1 << 30), p.status,
                                                     (reinterpret_cast<uintptr_t>(p.O) & 31) == 0 ? 1 : 0, paired, nullptr,
-                                                    nullptr, p.lse);
+                                                    nullptr, p.lse, EvenDeal{});
     return cudaGetLastError() == cudaSuccess ? FLAT_OK : FLAT_ERR_CUDA;
 }
 
 
 }  // namespace
+
+thread_local int g_last_schedule = 0;
 
 int launch_fused_tc3_varlen(const void* Q, const void* K, const void* V, void* O, const int32_t* cu_q,
                             const int32_t* cu_k, int num_seqs, int H, int64_t total_q, int64_t total_k,
@@ -828,10 +1145,11 @@ int launch_fused_tc3_varlen(const void* Q, const void* K, const void* V, void* O
     // grid saves the per-CTA set-up.
     const bool persistent = items >= 8 * static_cast<int64_t>(sms) && slabs < 8;
     const int grid = static_cast<int>(persistent ? sms : items);
+    g_last_schedule = persistent ? FLAT_SCHEDULE_PERSISTENT : FLAT_SCHEDULE_ITEMS;
     fused_tc3_kernel<true><<<grid, LY::THREADS, LY::SMEM_BYTES, st>>>(
         tmQ, tmK, tmV, static_cast<__nv_bfloat16*>(O), H, max_seqlen_q, 0, static_cast<int>(items), slabs,
         scale * 1.4426950408889634f, nullptr, causal ? 0 : (1 << 30), status,
-        (reinterpret_cast<uintptr_t>(O) & 31) == 0 ? 1 : 0, 0, cu_q, cu_k, nullptr);
+        (reinterpret_cast<uintptr_t>(O) & 31) == 0 ? 1 : 0, 0, cu_q, cu_k, nullptr, EvenDeal{});
     return cudaGetLastError() == cudaSuccess ? FLAT_OK : FLAT_ERR_CUDA;
 }
 
