@@ -248,6 +248,7 @@ class Bench:
         # written before a timed launch whose inputs fit in L2, and once in front of every timed region; allocated
         # here, not between warm-up and timing, where the allocation would leave the GPU idle for milliseconds
         self.flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+        self.schedule = None
 
     def barrier(self):
         if self.world > 1:
@@ -302,6 +303,11 @@ class Bench:
         for _ in range(warmup):
             step()
         kernel = KERNEL_OF_VARIANT.get(api.flat_attn_last_variant(), "?")
+        # how fused_tc3_kernel handed the items to the SMs (as reported by the library for the last launch)
+        self.schedule = None
+        if api.flat_attn_last_variant() == api.FLAT_VARIANT_TC3:
+            self.schedule = {api.FLAT_SCHEDULE_ITEMS: "one CTA per item", api.FLAT_SCHEDULE_PERSISTENT: "persistent CTAs",
+                             api.FLAT_SCHEDULE_EVEN_DEAL: "key steps dealt evenly"}.get(api.flat_attn_last_schedule())
         if sampler:
             sampler.mark()
         total_ms, per = self.timed(step, steps, flush=w.qkvo_bytes() <= L2_FLUSH_BELOW)
@@ -391,6 +397,7 @@ def main():
     seed = shard.rank_seed(inputs.DEFAULT_SEED, rank)
     data, host, d = bench.load(w, seed)
     total_ms, per_launch, kernel, clocks = bench.measure(w, d, args.steps, args.warmup, sample_clocks=rank == 0)
+    headline_schedule = bench.schedule
     launches = api.flat_attn_last_launch_count() * args.steps
 
     Oh = torch.empty(host["Q"].shape, dtype=torch.bfloat16).pin_memory()
@@ -423,6 +430,8 @@ def main():
             "clocks": clocks,
             "roofline": roofline_entry(w, per_launch, kernel, peaks),
         }
+        if headline_schedule:
+            out["roofline"]["schedule"] = headline_schedule
         if data[3] is not None:
             # Masked workload: `value` counts the masked keys too (the stated metric, 4 B H Nq Nk d);
             # this is the same rate counted over the valid keys only.
@@ -617,6 +626,8 @@ def run_other(bench, torch, api, w, seed, args, peaks, dev):
         useful = 4.0 * w.H * w.Nq * w.d * float(np.sum(data[3])) / float(w.flops)
         e["useful_work"] = {"value": val * useful, "unit": UNIT, "valid_key_fraction": useful,
                             "frac": val * useful / peaks["bf16_tflops"]}
+    if bench.schedule:
+        e["schedule"] = bench.schedule
     e.update(traffic_fields(kernel, w.name))
     if not args.no_cpu_baseline:
         _, e["parity_on_sample"] = parity_on_sample(torch, w, data, d["O"], dev, per_head=64)
