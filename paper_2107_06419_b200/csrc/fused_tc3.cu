@@ -335,7 +335,7 @@ __device__ __forceinline__ bool wait_flag_warp(const int* flag, int epoch, uint3
 // A part that begins inside its item: the un-normalised rows (this thread: 32 columns of one row, from TMEM
 // address `o_addr`), their reference and their sums go to this CTA's slot for the CTA that holds the item's
 // beginning.  `role` = (tile * 2 + key half) * 4 + row group.
-__device__ __noinline__ void deal_write_partial(const EvenDeal ed, uint32_t o_addr, int role, float m_ref, float l) {
+__device__ __forceinline__ void deal_write_partial(const EvenDeal ed, uint32_t o_addr, int role, float m_ref, float l) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     float* slot = ed.ws + static_cast<size_t>(blockIdx.x) * WS_FLOATS;
     float* po = slot + role * 1024 + lane;
@@ -355,7 +355,7 @@ __device__ __noinline__ void deal_write_partial(const EvenDeal ed, uint32_t o_ad
 // The part that begins its item: (m, l, O) of two parts merge as m = max, l = sum of l_i 2^(m_i - m), O likewise
 // (the row-wise softmax of Section 5.2, split along the keys); then 1/l and the store of this thread's 32 columns.
 // A part without a valid key carries m = -inf and l = 0 and drops out of the merge.
-__device__ __noinline__ void deal_finish_merged(const EvenDeal ed, uint32_t o_addr, int role, float m_ref, float l, int pfirst,
+__device__ __forceinline__ void deal_finish_merged(const EvenDeal ed, uint32_t o_addr, int role, float m_ref, float l, int pfirst,
                                                 int pcount, __nv_bfloat16* orow, bool row_valid, uint32_t abort_s, int32_t* status) {
     // (partner CTAs: pfirst, pfirst + team, ...)
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -922,7 +922,8 @@ fused_tc3_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         pair_sync(pair_id);
         l += ld_shared_f32((xm_own ^ (BM * 4)) + 4 * BM * 4);
         if (SPLIT) {
-            // an item shared with other CTAs: out of line, the code of whole items stays as it is
+            // an item shared with other CTAs (inlined: with these paths as called functions c5 ran 2 % slower,
+            // with the deal's index arithmetic out of line as well 6 %)
             int part, pfirst, pcount;
             deal_role(sc, idx, part, pfirst, pcount);
             if (part != 0) {
