@@ -83,7 +83,14 @@ enum {
                                   distributed shared memory: bf16, d in {64,128}, no bias, no pruning map;
                                   what AUTO picks for launches that would leave most SMs empty   */
     FLAT_VARIANT_TC2_SPLIT4 = 9, /* the same over a cluster of four CTAs                           */
-    FLAT_VARIANT_TC2_SPLIT8 = 10 /* the same over a cluster of eight CTAs                          */
+    FLAT_VARIANT_TC2_SPLIT8 = 10, /* the same over a cluster of eight CTAs                          */
+    FLAT_VARIANT_TC2_HALVES = 11, /* one 128-row tile per CTA worked on by two softmax warpgroups, which take the
+                                  even and the odd key tiles and merge their partial softmaxes through shared
+                                  memory at the end (half the chain of key steps that a short launch waits for):
+                                  bf16, d = 64, no bias, no pruning map; one CTA per SM             */
+    FLAT_VARIANT_TC2_HALVES_SPLIT2 = 12, /* the same with the keys also split over a cluster of two CTAs     */
+    FLAT_VARIANT_TC2_HALVES_SPLIT4 = 13, /* ... of four CTAs                                             */
+    FLAT_VARIANT_TC2_HALVES_SPLIT8 = 14  /* ... of eight CTAs                                            */
 };
 
 typedef struct flat_attn_params {

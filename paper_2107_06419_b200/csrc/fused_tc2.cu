@@ -191,7 +191,13 @@ __device__ __forceinline__ float exp_store(const uint32_t (&s)[128], float scale
 // BIAS = 2: the same with the bias tile of each step staged through shared memory by TMA (bf16, 16-byte aligned
 // rows, d = 64): the rows then arrive coalesced and a softmax thread reads its 256 bytes from shared memory; with a
 // bias shared by all batches the grid runs the batches of a head next to each other, so that its slice stays in L2.
-template <int D, int NT, bool VL = false, int BIAS = 0, bool SPARSE = false, int CS = 1>
+// KH (two warpgroups, ONE query tile, d = 64, dense): a short launch waits for one CTA's chain of key steps, and a
+// step is one warp per scheduler working through 128 exponentials per row.  With KH the CTA's two softmax warpgroups
+// (and their two MMA issuers, logit / weight / output columns) take the even and the odd key tiles of the same 128
+// query rows, each with its own running (m_ref, l, O); at the end the second warpgroup leaves its rows in shared
+// memory and the first merges them (the split-softmax identity again) before the ordinary epilogue or the cluster
+// exchange.  The chain is half as long and two warps per scheduler share the exponent unit.
+template <int D, int NT, bool VL = false, int BIAS = 0, bool SPARSE = false, int CS = 1, bool KH = false>
 __global__ void __launch_bounds__(128 * NT + 128, NT == 1 ? 2 : 1)
 fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                  const __grid_constant__ CUtensorMap tmV, __nv_bfloat16* __restrict__ O, int H, int Nq, int Nk,
@@ -203,7 +209,9 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     using LY = L2<D, NT, BIAS == 2>;
     static_assert(BIAS != 2 || (NT == 2 && D == 64 && !VL && !SPARSE && CS == 1), "staged bias: the two-tile dense kernel, d = 64");
     static_assert(!SPARSE || (NT == 1 && !VL && !BIAS), "the pruning map is read by the one-tile dense kernel");
-    static_assert(CS == 1 || (NT == 1 && !VL && !BIAS && !SPARSE && (CS == 2 || CS == 4 || CS == 8)), "key split: one-tile dense kernel");
+    static_assert(CS == 1 || ((NT == 1 || KH) && !VL && !BIAS && !SPARSE && (CS == 2 || CS == 4 || CS == 8)), "key split: one-tile dense kernel");
+    static_assert(!KH || (NT == 2 && D == 64 && !VL && !BIAS && !SPARSE), "key halves: two warpgroups on one dense d = 64 tile");
+    constexpr int QT = KH ? 1 : NT;                      // query tiles of the CTA
     __shared__ uint16_t tile_list[SPARSE ? 1024 : 1];    // the kept key tiles of this query tile, ascending
     __shared__ int tile_count;
     extern __shared__ uint8_t smem_raw[];
@@ -215,6 +223,7 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + LY::NUM_BARS);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
     float4* merge_buf = reinterpret_cast<float4*>(base + LY::TILE_BYTES + 512);   // (CS > 1) [CS - 1][d / 4 + 1][128 / CS]: lanes of a warp touch contiguous bytes
+    float4* kh_buf = reinterpret_cast<float4*>(base + LY::TILE_BYTES + 512 + LY::merge_bytes(CS));   // (KH) [d / 4 + 1][128]: the second warpgroup's rows
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     int bh = blockIdx.y;
@@ -224,20 +233,20 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         bh = (blockIdx.y % nb) * H + blockIdx.y / nb;
     }
     const int crank = CS > 1 ? static_cast<int>(cluster_ctarank()) : 0;   // (cluster = CS consecutive CTAs along x)
-    const int row0 = (blockIdx.x / CS) * (NT * BM);
+    const int row0 = (blockIdx.x / CS) * (QT * BM);
     // Barriers and TMEM columns.  The one-tile dense kernels (short launches, where the gap between two kernels of a
     // stream is a good part of the time) do this before anything else and then let the next kernel of the stream
     // start its own set-up (griddepcontrol.launch_dependents) and wait for the previous one to finish
     // (griddepcontrol.wait) before the first access to device memory: launched with programmatic stream
     // serialization, consecutive kernels overlap one's tail with the other's prologue.
-    constexpr bool PDL = (NT == 1 && !VL && !SPARSE && !BIAS);
+    constexpr bool PDL = ((NT == 1 || KH) && !VL && !SPARSE && !BIAS);
     auto setup = [&]() {
         if (threadIdx.x == LY::SOFT_WARPS * 32) {
             for (int i = 0; i < LY::NUM_BARS; ++i) {
                 const bool by_softmax = (i >= LY::S_FREE && i < LY::PV_DONE) ||    // one arrival per softmax warp
                                         (BIAS == 2 && i >= LY::B_EMPTY);
                 const bool by_issuers = (i >= LY::K_EMPTY && i < LY::V_FULL) || (i >= LY::V_EMPTY && i < LY::S_FULL);
-                mbar_init(&bars[i], i == LY::MERGE_BAR ? (CS > 1 ? (CS - 1) * (CS <= 4 ? 128 / CS / 32 : 1) : 1) : by_softmax ? 4 : by_issuers ? NT : 1);
+                mbar_init(&bars[i], i == LY::MERGE_BAR ? (CS > 1 ? (CS - 1) * (CS <= 4 ? 128 / CS / 32 : 1) : 1) : by_softmax ? 4 : by_issuers ? (KH ? 1 : NT) : 1);   // (KH: a key tile is used by one warpgroup only)
             }
             *abort_flag = 0;
             fence_mbar_init();
@@ -266,7 +275,7 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     {
         // Causal mask (coff = Nk - Nq; 2^30 = none): row r sees keys j < r + 1 + coff, so the CTA's
         // last row bounds the keys of all its rows.
-        const long long lim = static_cast<long long>(row0) + NT * BM + coff;
+        const long long lim = static_cast<long long>(row0) + QT * BM + coff;
         if (lim < n) n = lim < 0 ? 0 : static_cast<int>(lim);
     }
     int ntiles = (n + BN - 1) / BN;
@@ -359,7 +368,7 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
 #pragma unroll
                 for (int c = 0; c < D / 64; ++c)
                     tma_load_3d(Qs + (NT - 1) * LY::Q_BYTES + c * BM * 128, &tmQ, &bars[LY::Q_FULL + NT - 1], c * 64,
-                                VL ? head : row0 + BM, VL ? q_tok0 + BM : bh);
+                                VL ? head : row0 + (KH ? 0 : BM), VL ? q_tok0 + BM : bh);   // (KH: the same rows again)
             }
             for (int j = 0; j < ntiles && ok; ++j) {
                 if (j + 1 < ntiles) load_k(j + 1);
@@ -382,7 +391,11 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         // ------------------------------------------------------------ MMA issuer of tile t
         // The whole warp runs this loop (uniform control flow); one elected lane issues.
         const int t = warp - LY::SOFT_WARPS - 1;
-        if (ntiles > 0) {
+        // (KH: this warpgroup's key tiles are every second one of the CTA's sequence; the rings are indexed with
+        // the position in that sequence, the tile's own barriers with the count of its own steps)
+        const int nt_t = KH ? (ntiles - t + 1) / 2 : ntiles;
+        auto gi = [&](int j) -> int { return KH ? 2 * j + t : j; };
+        if (nt_t > 0) {
             constexpr uint32_t IDESC_S = make_idesc_bf16(BM, BN, 0, 0);
             constexpr uint32_t IDESC_PV = make_idesc_bf16(BM, D, 0, 1);
             const uint64_t q_desc = make_smem_desc_sw128(smem_u32(Qs) + t * LY::Q_BYTES, 16, 1024);
@@ -395,7 +408,7 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                 if (ok) tc_fence_after();
             };
             auto issue_s = [&](int j) {                  // S_t = Q_t K_j^T, then release the K stage
-                const int ks = j % LY::KS;
+                const int ks = gi(j) % LY::KS;
                 if (elect_one()) {
                     const uint64_t kd = k_desc + static_cast<uint64_t>((ks * LY::KV_BYTES) >> 4);
 #pragma unroll
@@ -409,7 +422,7 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                 __syncwarp();
             };
             auto issue_pv = [&](int j) {                 // O_t += P_t V_j, then release the V stage
-                const int vs = j % LY::VS;
+                const int vs = gi(j) % LY::VS;
                 if (elect_one()) {
                     const uint64_t vd = v_desc + static_cast<uint64_t>((vs * LY::KV_BYTES) >> 4);
 #pragma unroll
@@ -422,12 +435,12 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                 __syncwarp();
             };
             wait(LY::Q_FULL + t, 0, 0x200 + t);
-            wait(LY::K_FULL + 0, 0, 0x202);
+            wait(LY::K_FULL + gi(0) % LY::KS, (gi(0) / LY::KS) & 1, 0x202);
             if (ok) issue_s(0);
-            for (int j = 0; j < ntiles && ok; ++j) {
-                const bool more = j + 1 < ntiles;
-                const int ks = (j + 1) % LY::KS, vs = j % LY::VS;
-                const uint32_t kph = ((j + 1) / LY::KS) & 1, vph = (j / LY::VS) & 1;
+            for (int j = 0; j < nt_t && ok; ++j) {
+                const bool more = j + 1 < nt_t;
+                const int ks = gi(j + 1) % LY::KS, vs = gi(j) % LY::VS;
+                const uint32_t kph = (gi(j + 1) / LY::KS) & 1, vph = (gi(j) / LY::VS) & 1;
                 if (!LY::ALIAS && more) {
                     // P has columns of its own: the next S_t only needs the softmax to have taken S_t(j)
                     wait(LY::K_FULL + ks, kph, 0x210);
@@ -449,8 +462,10 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         // ------------------------------------------------------------ softmax + epilogue (warps 0-7)
         if (NT == 2) asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
         else         asm volatile("setmaxnreg.inc.sync.aligned.u32 208;");
-        const int t = warp >> 2;                         // query tile of this warpgroup
-        const int row = row0 + t * BM + (warp & 3) * 32 + lane;
+        const int t = warp >> 2;                         // query tile of this warpgroup (KH: its half of the key tiles)
+        const int row = row0 + (KH ? 0 : t * BM) + (warp & 3) * 32 + lane;
+        const int nt_t = KH ? (ntiles - t + 1) / 2 : ntiles;
+        auto gi = [&](int j) -> int { return KH ? 2 * j + t : j; };
         const uint32_t tl = tmem + (static_cast<uint32_t>((warp & 3) * 32) << 16);
         // (with a bias the logits are rescaled and shifted as they arrive, and the step goes on with scale 1)
         const float sc = BIAS ? 1.f : scale_log2e;
@@ -462,7 +477,7 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         const int nrow = rlim < n ? (rlim < 0 ? 0 : static_cast<int>(rlim)) : n;
         const int nrow_min = __shfl_sync(0xffffffffu, nrow, 0);
         if (LY::TURNS && t == 1 && lane == 0) mbar_arrive(&bars[LY::TURN + (warp & 3)]);   // tile A goes first
-        for (int j = 0; j < ntiles; ++j) {
+        for (int j = 0; j < nt_t; ++j) {
             // (bias, the common case of an aligned bf16 tensor: the row's 128 values of this step are fetched
             // before the wait for the logits, so that the two latencies overlap)
             uint32_t bpk[BIAS == 1 ? 64 : 1];
@@ -492,7 +507,7 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             __syncwarp();
             if (lane == 0) mbar_arrive(&bars[LY::S_FREE + t]);   // S_t may be overwritten (d = 64: by the next S_t)
 
-            const int col0 = tile_of(j) * BN;
+            const int col0 = tile_of(gi(j)) * BN;
             if (BIAS == 2) {
                 // x = s * scale * log2(e) + bias * log2(e): the thread's row of the staged tile (two swizzled panels)
                 const int bs = j % LY::BS, rt = (warp & 3) * 32 + lane;
@@ -645,12 +660,12 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             __syncwarp();
             if (lane == 0) mbar_arrive(&bars[LY::P_FULL + t]);
         }
-        if (ok && ntiles > 0) {
-            ok = bounded_wait(&bars[LY::PV_DONE + t], (ntiles - 1) & 1, abort_flag, status, 0x330 + t);
+        if (ok && nt_t > 0) {
+            ok = bounded_wait(&bars[LY::PV_DONE + t], (nt_t - 1) & 1, abort_flag, status, 0x330 + t);
             ok = __all_sync(0xffffffffu, ok);
         }
-        if constexpr (CS > 1) {
-            // ---- key split: exchange of the partial (m, l, O) rows inside the cluster, then the owner's merge
+        if constexpr (CS > 1 || KH) {
+            // ---- partial (m, l, O) rows: merged inside the CTA (KH), exchanged inside the cluster (CS > 1), written
             constexpr int RP = 128 / CS;                  // rows owned per rank: whole warps, or half a warp at CS = 8
             constexpr int GRP = RP < 32 ? RP : 32;        // lanes of a warp that share an owner
             const int tr = (warp & 3) * 32 + lane, owner = tr / RP;
@@ -659,70 +674,86 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
 #pragma unroll
             for (int c = 0; c < D / 32; ++c) {
                 uint32_t r[32];
-                if (ok && ntiles > 0) {
+                if (ok && nt_t > 0) {
                     tmem_ld_x32(tl + LY::O_COL(t) + c * 32, r);
                     tc_wait_ld();
                 } else {
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) r[i] = 0u;      // no key tile in this CTA's share
+                    for (int i = 0; i < 32; ++i) r[i] = 0u;      // no key tile in this share
                 }
 #pragma unroll
                 for (int i = 0; i < 32; ++i) o[c * 32 + i] = __uint_as_float(r[i]);
             }
-            if (!ok) l = __int_as_float(0x7fc00000);     // (a CTA that gave up poisons the rows it took part in)
-            if (owner != crank) {
-                const int slot = (crank - owner - 1 + CS) % CS;
-                const uint32_t dst = mapa_shared(smem_u32(merge_buf + slot * merge_vecs(D) * RP + tr % RP), owner);
+            if (!ok) l = __int_as_float(0x7fc00000);     // (a share that gave up poisons the rows it took part in)
+            // (m, l, O) of two shares of a row's keys: m = max, l = sum of l_i 2^(m_i - m), O likewise
+            auto merge_row = [&](const float4* src, int stride) {
+                const float mq = src[stride * (D / 4)].x, lq = src[stride * (D / 4)].y;
+                const float mt = fmaxf(m_ref, mq), mu = mt == -INFINITY ? 0.f : mt;
+                const float a = ex2_approx(m_ref - mu), b = ex2_approx(mq - mu);
+                l = l * a + lq * b;
+                m_ref = mt;
 #pragma unroll
-                for (int v = 0; v < D / 4; ++v) st_cluster_v4(dst + 16 * RP * v, o[4 * v], o[4 * v + 1], o[4 * v + 2], o[4 * v + 3]);
-                st_cluster_v2(dst + 16 * RP * (D / 4), m_ref, l);
+                for (int v = 0; v < D / 4; ++v) {
+                    const float4 w = src[stride * v];
+                    o[4 * v] = o[4 * v] * a + w.x * b;         o[4 * v + 1] = o[4 * v + 1] * a + w.y * b;
+                    o[4 * v + 2] = o[4 * v + 2] * a + w.z * b; o[4 * v + 3] = o[4 * v + 3] * a + w.w * b;
+                }
+            };
+            bool writer = true;
+            if constexpr (KH) {
+                // the second warpgroup hands its rows to the first through shared memory (lanes of a warp write
+                // contiguous 16-byte vectors) and is done; a named barrier of the eight softmax warps in between
+                if (t == 1) {
+#pragma unroll
+                    for (int v = 0; v < D / 4; ++v) kh_buf[v * 128 + tr] = make_float4(o[4 * v], o[4 * v + 1], o[4 * v + 2], o[4 * v + 3]);
+                    kh_buf[(D / 4) * 128 + tr] = make_float4(m_ref, l, 0.f, 0.f);
+                }
+                asm volatile("bar.sync 2, 256;" ::: "memory");
+                if (t == 1) writer = false;
+                else merge_row(kh_buf + tr, 128);
             }
-            // one arrival per group of lanes with the same owner: the warp barrier orders the lanes' stores before
-            // the first lane's release
-            __syncwarp();
-            if (owner != crank && lane % GRP == 0) mbar_arrive_cluster(mapa_shared(smem_u32(&bars[LY::MERGE_BAR]), owner));
-            if (owner == crank) {
-                bool got = true;
-                {
-                    const long long t0 = clock64();
-                    while (!mbar_try_wait_cluster(&bars[LY::MERGE_BAR], 0)) {
-                        if (clock64() - t0 > WAIT_CYCLES) {
-                            got = false;
-                            if (status) atomicExch(status, 0x350);
-                            break;
+            if constexpr (CS > 1) {
+                if (writer) {                             // (warp-uniform)
+                    if (owner != crank) {
+                        const int slot = (crank - owner - 1 + CS) % CS;
+                        const uint32_t dst = mapa_shared(smem_u32(merge_buf + slot * merge_vecs(D) * RP + tr % RP), owner);
+#pragma unroll
+                        for (int v = 0; v < D / 4; ++v) st_cluster_v4(dst + 16 * RP * v, o[4 * v], o[4 * v + 1], o[4 * v + 2], o[4 * v + 3]);
+                        st_cluster_v2(dst + 16 * RP * (D / 4), m_ref, l);
+                    }
+                    // one arrival per group of lanes with the same owner: the warp barrier orders the lanes' stores
+                    // before the first lane's release
+                    __syncwarp();
+                    if (owner != crank && lane % GRP == 0) mbar_arrive_cluster(mapa_shared(smem_u32(&bars[LY::MERGE_BAR]), owner));
+                    writer = owner == crank;
+                    if (writer) {
+                        const long long t0 = clock64();
+                        while (!mbar_try_wait_cluster(&bars[LY::MERGE_BAR], 0)) {
+                            if (clock64() - t0 > WAIT_CYCLES) {
+                                writer = false;
+                                if (status) atomicExch(status, 0x350);
+                                break;
+                            }
                         }
+                    }
+                    if (writer) {
+#pragma unroll
+                        for (int q = 0; q < CS - 1; ++q) merge_row(merge_buf + q * merge_vecs(D) * RP + tr % RP, RP);
                     }
                 }
-                if (got) {
+            }
+            if (writer && row < Nq) {
+                const float inv = l > 0.f ? 1.f / l : (l == l ? 0.f : l);
+                if (lse) lse[static_cast<int64_t>(bh) * Nq + row] = l > 0.f ? (m_ref + log2f(l)) * 0.6931471805599453f : -INFINITY;
+                __nv_bfloat16* orow = O + (static_cast<int64_t>(bh) * Nq + row) * D;
 #pragma unroll
-                    for (int q = 0; q < CS - 1; ++q) {
-                        const float4* src = merge_buf + q * merge_vecs(D) * RP + tr % RP;
-                        const float mq = src[RP * (D / 4)].x, lq = src[RP * (D / 4)].y;
-                        const float mt = fmaxf(m_ref, mq), mu = mt == -INFINITY ? 0.f : mt;
-                        const float a = ex2_approx(m_ref - mu), b = ex2_approx(mq - mu);
-                        l = l * a + lq * b;
-                        m_ref = mt;
-#pragma unroll
-                        for (int v = 0; v < D / 4; ++v) {
-                            const float4 w = src[RP * v];
-                            o[4 * v] = o[4 * v] * a + w.x * b;         o[4 * v + 1] = o[4 * v + 1] * a + w.y * b;
-                            o[4 * v + 2] = o[4 * v + 2] * a + w.z * b; o[4 * v + 3] = o[4 * v + 3] * a + w.w * b;
-                        }
-                    }
-                    if (row < Nq) {
-                        const float inv = l > 0.f ? 1.f / l : (l == l ? 0.f : l);
-                        if (lse) lse[static_cast<int64_t>(bh) * Nq + row] = l > 0.f ? (m_ref + log2f(l)) * 0.6931471805599453f : -INFINITY;
-                        __nv_bfloat16* orow = O + (static_cast<int64_t>(bh) * Nq + row) * D;
-#pragma unroll
-                        for (int v = 0; v < D / 8; ++v) {
-                            uint4 w;
-                            w.x = pack_bf16x2(o[8 * v + 0] * inv, o[8 * v + 1] * inv);
-                            w.y = pack_bf16x2(o[8 * v + 2] * inv, o[8 * v + 3] * inv);
-                            w.z = pack_bf16x2(o[8 * v + 4] * inv, o[8 * v + 5] * inv);
-                            w.w = pack_bf16x2(o[8 * v + 6] * inv, o[8 * v + 7] * inv);
-                            *reinterpret_cast<uint4*>(orow + v * 8) = w;
-                        }
-                    }
+                for (int v = 0; v < D / 8; ++v) {
+                    uint4 w;
+                    w.x = pack_bf16x2(o[8 * v + 0] * inv, o[8 * v + 1] * inv);
+                    w.y = pack_bf16x2(o[8 * v + 2] * inv, o[8 * v + 3] * inv);
+                    w.z = pack_bf16x2(o[8 * v + 4] * inv, o[8 * v + 5] * inv);
+                    w.w = pack_bf16x2(o[8 * v + 6] * inv, o[8 * v + 7] * inv);
+                    *reinterpret_cast<uint4*>(orow + v * 8) = w;
                 }
             }
         } else
@@ -885,6 +916,47 @@ int launch_tc2_d(const Problem& p, cudaStream_t st, int key_split = 1) {
     return cudaGetLastError() == cudaSuccess ? FLAT_OK : FLAT_ERR_CUDA;
 }
 
+// Key halves (see the kernel's KH): d = 64, dense, one 128-row tile per CTA worked on by two warpgroups, optionally
+// with the keys over a cluster on top.  One CTA per SM (all 512 TMEM columns).
+int launch_tc2_kh(const Problem& p, cudaStream_t st, int key_split) {
+    constexpr int D = 64, NT = 2;
+    using LY = L2<D, NT>;
+    CUtensorMap tmQ, tmK, tmV;
+    const int BH = p.B * p.H;
+    if (!make_map(&tmQ, p.Q, BH, p.Nq, D, BM) || !make_map(&tmK, p.K, BH, p.Nk, D, BN) ||
+        !make_map(&tmV, p.V, BH, p.Nk, D, BN))
+        return FLAT_ERR_CUDA;
+    const dim3 grid((p.Nq + BM - 1) / BM, BH);
+    auto launch = [&](auto cs_tag) -> int {
+        constexpr int CS = decltype(cs_tag)::value;
+        constexpr int BYTES = LY::SMEM_BYTES + LY::merge_bytes(CS) + 128 * merge_vecs(D) * 16;
+        auto kern = fused_tc2_kernel<D, NT, false, 0, false, CS, true>;
+        if (!ensure_dynamic_smem<fused_tc2_kernel<D, NT, false, 0, false, CS, true>>(BYTES)) return FLAT_ERR_CUDA;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(grid.x * CS, grid.y);
+        cfg.blockDim = dim3(LY::THREADS);
+        cfg.dynamicSmemBytes = BYTES;
+        cfg.stream = st;
+        cudaLaunchAttribute attr[2];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // (see the kernel's prologue)
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        attr[1].id = cudaLaunchAttributeClusterDimension;
+        attr[1].val.clusterDim.x = CS; attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = CS > 1 ? 2 : 1;
+        const cudaError_t e = cudaLaunchKernelEx(
+            &cfg, kern, tmQ, tmK, tmV, static_cast<__nv_bfloat16*>(p.O), p.H, p.Nq, p.Nk, p.scale * 1.4426950408889634f,
+            p.k_valid_len, p.causal ? p.Nk - p.Nq : (1 << 30), p.status, static_cast<const int32_t*>(nullptr),
+            static_cast<const int32_t*>(nullptr), p.lse, BiasArg{nullptr, 0, 0, 0, 0}, static_cast<const uint8_t*>(nullptr), 0ll, 0ll,
+            CUtensorMap{});
+        return e == cudaSuccess ? FLAT_OK : FLAT_ERR_CUDA;
+    };
+    return key_split == 1   ? launch(std::integral_constant<int, 1>{})
+           : key_split == 2 ? launch(std::integral_constant<int, 2>{})
+           : key_split == 4 ? launch(std::integral_constant<int, 4>{})
+           : key_split == 8 ? launch(std::integral_constant<int, 8>{}) : FLAT_ERR_UNSUPPORTED;
+}
+
 }  // namespace
 
 
@@ -943,6 +1015,11 @@ int launch_fused_tc2(const Problem& p, cudaStream_t st) {
     if (p.d == 64) return launch_tc2_d<64, 2>(p, st);
     if (p.d == 128) return launch_tc2_d<128, 2>(p, st);
     return FLAT_ERR_UNSUPPORTED;
+}
+
+int launch_fused_tc2_halves(const Problem& p, cudaStream_t st, int key_split) {
+    if (p.dtype != FLAT_DTYPE_BF16 || p.d != 64 || p.bias || p.block_mask) return FLAT_ERR_UNSUPPORTED;
+    return launch_tc2_kh(p, st, key_split);
 }
 
 // One 128-row tile per CTA, two CTAs per SM (d = 64 only: at d = 128 two CTAs do not fit in shared memory).

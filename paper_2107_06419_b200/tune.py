@@ -37,6 +37,10 @@ VARIANTS = {
     api.FLAT_VARIANT_TC2_SPLIT2: "tc2_split2: 128-row CTA, keys split over a cluster of 2 CTAs",
     api.FLAT_VARIANT_TC2_SPLIT4: "tc2_split4: ... over a cluster of 4 CTAs",
     api.FLAT_VARIANT_TC2_SPLIT8: "tc2_split8: ... over a cluster of 8 CTAs",
+    api.FLAT_VARIANT_TC2_HALVES: "tc2_halves: 128-row CTA, two warpgroups on alternate key tiles (d = 64)",
+    api.FLAT_VARIANT_TC2_HALVES_SPLIT2: "tc2_halves_split2: ... and the keys over a cluster of 2 CTAs",
+    api.FLAT_VARIANT_TC2_HALVES_SPLIT4: "tc2_halves_split4: ... of 4 CTAs",
+    api.FLAT_VARIANT_TC2_HALVES_SPLIT8: "tc2_halves_split8: ... of 8 CTAs",
     api.FLAT_VARIANT_AUTO: "auto (the dispatcher's choice)",
 }
 

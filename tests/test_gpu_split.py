@@ -12,7 +12,9 @@ from helpers import bf16_tensor, bf16_to_f64, check_bf16, rand_bits
 
 pytestmark = pytest.mark.gpu
 
-SPLITS = [8, 9, 10]            # FLAT_VARIANT_TC2_SPLIT2 / 4 / 8
+# FLAT_VARIANT_TC2_SPLIT2 / 4 / 8, then FLAT_VARIANT_TC2_HALVES and HALVES_SPLIT2 / 4 / 8 (the tile's two warpgroups
+# on alternate key tiles, merged through shared memory, with the keys over a cluster on top)
+SPLITS = [8, 9, 10, 11, 12, 13, 14]
 
 
 @pytest.fixture(scope="module")
@@ -90,8 +92,14 @@ def test_planted_keys_and_rising_maximum(api, variant):
 
 def test_auto_takes_the_split_for_underfilled_launches(api):
     rng = np.random.default_rng(9)
-    for (B, H, Nq, Nk, expect) in [(1, 1, 128, 8192, api.FLAT_VARIANT_TC2_SPLIT8), (1, 12, 512, 512, api.FLAT_VARIANT_TC2_SPLIT2),
-                                   (1, 12, 512, 2048, api.FLAT_VARIANT_TC2_SPLIT4), (1, 2, 128, 128, api.FLAT_VARIANT_TC2_SINGLE)]:
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    if sms != 148:
+        pytest.skip("the expected choices are those of a 148-SM GPU")
+    # (more tiles than seven SMs in eight: two-per-SM CTAs, unsplit; one key tile: nothing to split)
+    for (B, H, Nq, Nk, expect) in [(1, 1, 128, 8192, api.FLAT_VARIANT_TC2_HALVES_SPLIT8), (1, 12, 512, 512, api.FLAT_VARIANT_TC2_HALVES_SPLIT2),
+                                   (1, 12, 512, 2048, api.FLAT_VARIANT_TC2_HALVES_SPLIT2), (1, 8, 256, 2048, api.FLAT_VARIANT_TC2_HALVES_SPLIT4),
+                                   (1, 24, 512, 1024, api.FLAT_VARIANT_TC2_HALVES), (1, 34, 512, 512, api.FLAT_VARIANT_TC2_SINGLE),
+                                   (1, 2, 128, 128, api.FLAT_VARIANT_TC2_SINGLE)]:
         Qb, Kb, Vb = rand_bits(rng, (B, H, Nq, 64)), rand_bits(rng, (B, H, Nk, 64)), rand_bits(rng, (B, H, Nk, 64))
         ref = oracle.attention(Qb, Kb, Vb, 0.125)["O"]
         O, _ = run(api, Qb, Kb, Vb, 0.125, api.FLAT_VARIANT_AUTO)
@@ -99,7 +107,7 @@ def test_auto_takes_the_split_for_underfilled_launches(api):
         check_bf16(O, ref, "auto split %s" % ((B, H, Nq, Nk),))
 
 
-@pytest.mark.parametrize("variant", SPLITS)
+@pytest.mark.parametrize("variant", [8, 9, 10])          # (the two-warpgroup form is built for d = 64)
 @pytest.mark.parametrize("shape", [(1, 2, 128, 128), (2, 2, 200, 333), (1, 3, 300, 2100), (1, 1, 77, 4096)])
 def test_head_size_128(api, shape, variant):
     B, H, Nq, Nk = shape
@@ -135,6 +143,11 @@ def test_refusals(api):
     bias = torch.zeros(1, 1, 128, 128, device="cuda", dtype=torch.bfloat16)
     with pytest.raises(api.FlatAttnError):               # no bias operand in the split kernel
         api.flat_attn_fwd_ex(Q64, Q64, Q64, torch.empty_like(Q64), 1.0, variant=api.FLAT_VARIANT_TC2_SPLIT4, bias=bias)
+    with pytest.raises(api.FlatAttnError):
+        api.flat_attn_fwd_ex(Q64, Q64, Q64, torch.empty_like(Q64), 1.0, variant=api.FLAT_VARIANT_TC2_HALVES, bias=bias)
+    Q128 = torch.zeros(1, 1, 128, 128, device="cuda", dtype=torch.bfloat16)
+    with pytest.raises(api.FlatAttnError):               # the two-warpgroup form: d = 64 only
+        api.flat_attn_fwd_ex(Q128, Q128, Q128, torch.empty_like(Q128), 1.0, variant=api.FLAT_VARIANT_TC2_HALVES_SPLIT2)
 
 
 def test_cluster_launch_in_a_cuda_graph(api):
@@ -157,7 +170,7 @@ def test_cluster_launch_in_a_cuda_graph(api):
     check_bf16(bf16_to_f64(O), ref, "split in a graph")
 
 
-@pytest.mark.parametrize("variant", [4, 8, 9])
+@pytest.mark.parametrize("variant", [4, 8, 9, 11, 12])
 def test_back_to_back_launches_that_depend_on_each_other(api, variant):
     """The one-tile kernels let the next kernel of the stream start its set-up early (programmatic dependent launch)
     and wait for their predecessor before the first access to device memory.  A chain in which every call reads
