@@ -448,13 +448,13 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                     if (ok) issue_s(j + 1);
                 }
                 wait(LY::V_FULL + vs, vph, 0x220);
+                // (P overlays S: the next key tile's barrier is checked here, while the softmax still runs, so that
+                // the next S_t can go straight behind the MMA that reads P_t(j): a barrier check costs about 150
+                // cycles of the tile's chain even when the tile has long arrived)
+                if (LY::ALIAS && more) wait(LY::K_FULL + ks, kph, 0x230);
                 wait(LY::P_FULL + t, j & 1, 0x221);
                 if (ok) issue_pv(j);
-                if (LY::ALIAS && more) {
-                    // P overlays S: the next S_t goes behind the MMA that reads P_t(j)
-                    wait(LY::K_FULL + ks, kph, 0x230);
-                    if (ok) issue_s(j + 1);
-                }
+                if (LY::ALIAS && more && ok) issue_s(j + 1);
             }
         }
       }
