@@ -45,7 +45,7 @@ namespace {
 
 constexpr int BM = 128;              // rows per query tile (two tiles per CTA)
 constexpr int BN = 128;              // keys per step
-constexpr int PASS_AT_CHUNK = 3;                // the other tile gets its turn once this chunk's ex2 are issued
+constexpr int PASS_AT_CHUNK = 2;                // the other tile gets its turn once this chunk's ex2 are issued (of chunks 0-3; measured on c4: 3 -> 1166, 2 -> 1187, 1 -> 995 TFLOP/s)
 constexpr int POLY_LANE = 3;                    // element index mod 4 that uses ex2_poly; -1 = none
 __host__ __device__ constexpr int merge_vecs(int d) { return d / 4 + 1; }   // (key split) 16-byte vectors per row of a partial result: d outputs, then (m, l)
 constexpr float OVERFLOW_SUM = 1.0995116e12f;   // 2^40: a tile row sum beyond this means m_ref is stale
@@ -148,7 +148,7 @@ __device__ __forceinline__ float exp_store(const uint32_t (&s)[128], float scale
             p[i] = (!TAIL && POLY && (i & 3) == POLY_LANE) ? ex2_poly(p[i]) : ex2_approx(p[i]);
             if (TAIL && c * 32 + i >= nvalid) p[i] = 0.f;
         }
-        if (c == PASS_AT_CHUNK) after_last_exp();       // (nearly) every ex2 of the row has been issued
+        if (c == PASS_AT_CHUNK) after_last_exp();       // most ex2 of the row have been issued
 #pragma unroll
         for (int i = 0; i < 32; i += 4) {
             lsum0 = add2(lsum0, pack2(p[i], p[i + 1]));
