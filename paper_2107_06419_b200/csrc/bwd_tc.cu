@@ -265,8 +265,10 @@ bwd_tc_kernel(const __grid_constant__ CUtensorMap tmX1, const __grid_constant__ 
                 const bool more = j + 1 < nsteps;
 #pragma unroll
                 for (int half = 0; half < 2; ++half) {
-                    ok = wait_warp(LY::BAR_PD_FULL + half, j & 1, 0x530 + half);
-                    if (ok && more) ok = y_full(2 * (j + 1) + half, 0x521);
+                    // (the next half step's copy landed long ago: its barrier is checked before the wait for the
+                    // element-wise warps, not behind it, where the check would sit in the chain of the half)
+                    if (more) ok = y_full(2 * (j + 1) + half, 0x521);
+                    if (ok) ok = wait_warp(LY::BAR_PD_FULL + half, j & 1, 0x530 + half);
                     if (!ok) break;
                     tc_fence_after();
                     if (elect_one()) {
