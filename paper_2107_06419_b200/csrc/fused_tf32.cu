@@ -230,13 +230,13 @@ fused_tf32_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 for (int j = g; j < ntiles && ok; j += 2) {
                     wait(VT_FULL + j % VS, (j / VS) & 1, 0x630);
                     wait(PV_FREE + (j & 1), ((j >> 1) & 1) ^ 1, 0x631);
+                    // (the converted keys of step j + 2 are checked here, ahead of the wait for the weights, so that
+                    // the check does not sit between the two batches of products)
+                    if (j + 2 < ntiles) wait(KC_FULL + (j + 2) % KS, ((j + 2) / KS) & 1, 0x633);
                     wait(P_FULL + (j & 1), (j >> 1) & 1, 0x632);
                     if (ok) issue_pv(j);
-                    if (j + 2 < ntiles) {
-                        // (S(j+2) overwrites P_hi(j): it goes behind the products that read it)
-                        wait(KC_FULL + (j + 2) % KS, ((j + 2) / KS) & 1, 0x633);
-                        if (ok) issue_s(j + 2);
-                    }
+                    // (S(j+2) overwrites P_hi(j): it goes behind the products that read it)
+                    if (j + 2 < ntiles && ok) issue_s(j + 2);
                 }
             }
         }
