@@ -1025,7 +1025,11 @@ bool deal_acquire(cudaStream_t st, EvenDeal& ed, std::unique_lock<std::mutex>& l
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return false;
     cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
-    if (cudaStreamIsCapturing(st, &cap) != cudaSuccess || cap != cudaStreamCaptureStatusNone) return false;
+    if (cudaStreamIsCapturing(st, &cap) != cudaSuccess) {
+        cudaGetLastError();                              // (e.g. the legacy stream while another stream captures: not our launch's error)
+        return false;
+    }
+    if (cap != cudaStreamCaptureStatusNone) return false;
     lock = std::unique_lock<std::mutex>(g_deal_mu);
     DealOwner& o = g_deal[dev];
     if (!o.ready) {
