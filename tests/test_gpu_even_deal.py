@@ -197,3 +197,49 @@ def test_many_launches_in_a_row(api):
         rows = sampled_rows(B, H, Nq, 6, i)
         ref = oracle.attention(Qb, Kb, Vb, 0.125, valid_len=vl, rows=rows)["O"]
         check_bf16(bf16_to_f64(O).reshape(-1, 64)[rows], ref, "launch %d of the chain" % i)
+
+
+def test_two_host_threads_on_two_streams(api):
+    """The workspace is one per device: launches from two host threads on two streams must never share it while
+    one of them may still be running (the second falls back to the plain deal), and every result must be right."""
+    import threading
+    rng = np.random.default_rng(37)
+    jobs = []
+    for (B, H, Nq, Nk) in [(4, 12, 1024, 4096), (2, 9, 1200, 5000)]:
+        Qb, Kb, Vb = rand_bits(rng, (B, H, Nq, 64)), rand_bits(rng, (B, H, Nk, 64)), rand_bits(rng, (B, H, Nk, 64))
+        vl = rng.integers(Nk // 2, Nk + 1, B).astype(np.int32)
+        rows = sampled_rows(B, H, Nq, 6, 41)
+        ref = oracle.attention(Qb, Kb, Vb, 0.125, valid_len=vl, rows=rows)["O"]
+        jobs.append((bf16_tensor(Qb), bf16_tensor(Kb), bf16_tensor(Vb), torch.from_numpy(vl).cuda(), rows, ref))
+    torch.cuda.synchronize()
+    results, errors, schedules = [[], []], [], [[], []]
+
+    def worker(k):
+        try:
+            Q, K, V, vlt, rows, ref = jobs[k]
+            s = torch.cuda.Stream()
+            for _ in range(12):
+                O = torch.full(Q.shape, float("nan"), dtype=torch.bfloat16, device="cuda")
+                status = torch.zeros(1, dtype=torch.int32, device="cuda")
+                s.wait_stream(torch.cuda.current_stream())
+                api.flat_attn_fwd_ex(Q, K, V, O, 0.125, k_valid_len=vlt, status=status, variant=api.FLAT_VARIANT_TC3,
+                                     stream=s.cuda_stream)
+                schedules[k].append(api.flat_attn_last_schedule())
+                results[k].append((O, status))
+            s.synchronize()
+        except Exception as e:                           # (surfaces in the main thread)
+            errors.append(e)
+
+    threads = [threading.Thread(target=worker, args=(k,)) for k in range(2)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    torch.cuda.synchronize()
+    assert not errors, errors
+    for k in range(2):
+        rows, ref = jobs[k][4], jobs[k][5]
+        assert all(x in (api.FLAT_SCHEDULE_ITEMS, api.FLAT_SCHEDULE_EVEN_DEAL) for x in schedules[k])
+        for O, status in results[k]:
+            assert int(status.item()) == 0
+            check_bf16(bf16_to_f64(O).reshape(-1, 64)[rows], ref, "thread %d" % k)
