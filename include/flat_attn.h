@@ -81,13 +81,15 @@ enum {
     FLAT_VARIANT_TC2_SPLIT2 = 8, /* TC2_SINGLE with the keys of every query tile split over a cluster
                                   of two CTAs, whose partial softmaxes are merged through
                                   distributed shared memory: bf16, d in {64,128}, no bias, no pruning map;
-                                  what AUTO picks for launches that would leave most SMs empty   */
+                                  what AUTO picks at d = 128 for launches that would leave most
+                                  SMs empty (at d = 64 it takes the HALVES forms below)          */
     FLAT_VARIANT_TC2_SPLIT4 = 9, /* the same over a cluster of four CTAs                           */
     FLAT_VARIANT_TC2_SPLIT8 = 10, /* the same over a cluster of eight CTAs                          */
     FLAT_VARIANT_TC2_HALVES = 11, /* one 128-row tile per CTA worked on by two softmax warpgroups, which take the
                                   even and the odd key tiles and merge their partial softmaxes through shared
                                   memory at the end (half the chain of key steps that a short launch waits for):
-                                  bf16, d = 64, no bias, no pruning map; one CTA per SM             */
+                                  bf16, d = 64, no bias, no pruning map; one CTA per SM; what AUTO picks,
+                                  with the largest cluster that fits, while every CTA gets an SM of its own */
     FLAT_VARIANT_TC2_HALVES_SPLIT2 = 12, /* the same with the keys also split over a cluster of two CTAs     */
     FLAT_VARIANT_TC2_HALVES_SPLIT4 = 13, /* ... of four CTAs                                             */
     FLAT_VARIANT_TC2_HALVES_SPLIT8 = 14  /* ... of eight CTAs                                            */
