@@ -53,6 +53,8 @@ MEASURED_DRAM_TRAFFIC = {
     ("fused_tc3_kernel", "c2_bert_large_4k"): (515_300_000, "profiles/fused_tc3_kernel_dram_and_pipes.md"),
     ("fused_tc3_kernel", "p_4k_small"): (116_900_000, "profiles/fused_tc3_kernel_dram_and_pipes.md"),
     ("fused_tc3_kernel", "c5_cross_masked"): (349_600_000, "profiles/fused_tc3_kernel_even_deal_cuda_events.md"),
+    ("fused_tc3_kernel", "c3_16k"): (520_600_000, "profiles/fused_tc3_kernel_dram_and_pipes.md"),
+    ("fused_tc2_kernel<2 tiles>", "c4_64k_d128"): (597_400_000, "profiles/fused_tc2_kernel_dram_and_pipes.md"),
     ("fused_tc2_kernel<2 tiles>", "c2_bert_large_4k"): (516_000_000, "profiles/fused_tc2_kernel_dram_and_pipes.md"),
     ("fused_tc2_kernel<2 tiles>", "p_4k_small"): (117_600_000, "profiles/fused_tc2_kernel_dram_and_pipes.md"),
     ("fused_tc2_kernel<2 tiles>", "p_16k_d128_small"): (51_900_000, "profiles/fused_tc2_kernel_dram_and_pipes.md"),
