@@ -54,7 +54,7 @@ int validate(const flat_attn_params_t* p, flat::Problem* out) {
     if (bh * static_cast<int64_t>(p->Nq > p->Nk ? p->Nq : p->Nk) > lim / p->d) return FLAT_ERR_SHAPE;
     if (p->dtype != FLAT_DTYPE_BF16 && p->dtype != FLAT_DTYPE_F32) return FLAT_ERR_UNSUPPORTED;
     if (p->d != 16 && p->d != 32 && p->d != 64 && p->d != 128) return FLAT_ERR_UNSUPPORTED;
-    if (p->variant < FLAT_VARIANT_AUTO || p->variant > FLAT_VARIANT_TC2_HALVES_SPLIT8) return FLAT_ERR_UNSUPPORTED;
+    if (p->variant < FLAT_VARIANT_AUTO || p->variant > FLAT_VARIANT_TC2_SPLIT16) return FLAT_ERR_UNSUPPORTED;
     if (!aligned16(p->Q) || !aligned16(p->K) || !aligned16(p->V) || !aligned16(p->O)) return FLAT_ERR_ALIGN;
     if (p->k_valid_len && (reinterpret_cast<uintptr_t>(p->k_valid_len) & 3u)) return FLAT_ERR_ALIGN;
     if (p->status && (reinterpret_cast<uintptr_t>(p->status) & 3u)) return FLAT_ERR_ALIGN;
@@ -156,9 +156,14 @@ int run_fused(const flat::Problem& q, int variant, cudaStream_t st) {
             if (q.d == 128 && !q.block_mask && !q.bias && 2 * ctas2 < sms) {
                 const int64_t ctas1 = static_cast<int64_t>((q.Nq + 127) / 128) * q.B * q.H;
                 const int key_tiles = (q.Nk + 127) / 128;
-                for (int cs = 8; cs >= 2; cs /= 2) {
+                for (int cs = 16; cs >= 2; cs /= 2) {
                     if (ctas1 * cs > sms || key_tiles < 2 * cs) continue;
-                    v = cs == 8 ? FLAT_VARIANT_TC2_SPLIT8 : cs == 4 ? FLAT_VARIANT_TC2_SPLIT4 : FLAT_VARIANT_TC2_SPLIT2;
+                    // (clusters of sixteen -- beyond the portable size -- pay for one or two query tiles only: 128
+                    // queries x 64K keys 123 -> 83 us, two heads x 32K keys 68 -> 55 us; with three or four clusters
+                    // they are at par with eight, with eight clusters twice as slow)
+                    if (cs == 16 && ctas1 > 2) continue;
+                    v = cs == 16 ? FLAT_VARIANT_TC2_SPLIT16 : cs == 8 ? FLAT_VARIANT_TC2_SPLIT8
+                        : cs == 4 ? FLAT_VARIANT_TC2_SPLIT4 : FLAT_VARIANT_TC2_SPLIT2;
                     break;
                 }
             }
@@ -172,10 +177,17 @@ int run_fused(const flat::Problem& q, int variant, cudaStream_t st) {
         g_last_variant = v;
         return flat::launch_fused_tc2_halves(q, st, 1 << (v - FLAT_VARIANT_TC2_HALVES));
     }
-    if (v == FLAT_VARIANT_TC2_SPLIT2 || v == FLAT_VARIANT_TC2_SPLIT4 || v == FLAT_VARIANT_TC2_SPLIT8) {
-        if (!tc_applies(q) || q.block_mask) return FLAT_ERR_UNSUPPORTED;
+    if (v == FLAT_VARIANT_TC2_SPLIT2 || v == FLAT_VARIANT_TC2_SPLIT4 || v == FLAT_VARIANT_TC2_SPLIT8 || v == FLAT_VARIANT_TC2_SPLIT16) {
+        if (!tc_applies(q) || q.block_mask || (v == FLAT_VARIANT_TC2_SPLIT16 && q.d != 128)) return FLAT_ERR_UNSUPPORTED;
+        const int cs = v == FLAT_VARIANT_TC2_SPLIT2 ? 2 : v == FLAT_VARIANT_TC2_SPLIT4 ? 4 : v == FLAT_VARIANT_TC2_SPLIT8 ? 8 : 16;
+        int rc = flat::launch_fused_tc2_single(q, st, cs, variant == FLAT_VARIANT_AUTO);
+        if (rc == FLAT_ERR_UNSUPPORTED && cs == 16 && variant == FLAT_VARIANT_AUTO) {
+            // (AUTO asked for sixteen and the device cannot hold all the launch's clusters at once: eight)
+            v = FLAT_VARIANT_TC2_SPLIT8;
+            rc = flat::launch_fused_tc2_single(q, st, 8);
+        }
         g_last_variant = v;
-        return flat::launch_fused_tc2_single(q, st, v == FLAT_VARIANT_TC2_SPLIT2 ? 2 : v == FLAT_VARIANT_TC2_SPLIT4 ? 4 : 8);
+        return rc;
     }
     if (v == FLAT_VARIANT_TF32 && !flat::tf32_applies(q)) return FLAT_ERR_UNSUPPORTED;
     if (q.block_mask && (v != FLAT_VARIANT_TC2_SINGLE || q.bias || !tc_applies(q) || q.Nk > 131072)) return FLAT_ERR_UNSUPPORTED;

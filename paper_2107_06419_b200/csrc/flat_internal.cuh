@@ -67,7 +67,9 @@ int launch_fused_simt(const Problem& p, cudaStream_t st);
 int launch_naive(const Problem& p, void* L, void* A, cudaStream_t st);
 int launch_fused_tc(const Problem& p, cudaStream_t st);
 int launch_fused_tc2(const Problem& p, cudaStream_t st);      // (also the tensor-core kernel for calls with a bias)
-int launch_fused_tc2_single(const Problem& p, cudaStream_t st, int key_split = 1);
+// (only_if_resident: sixteen-CTA clusters only when all clusters of the launch can run at the same time; else
+// FLAT_ERR_UNSUPPORTED)
+int launch_fused_tc2_single(const Problem& p, cudaStream_t st, int key_split = 1, bool only_if_resident = false);
 // The same tile worked on by two warpgroups that take alternate key tiles (bf16, d = 64, dense; key_split 1, 2, 4, 8).
 int launch_fused_tc2_halves(const Problem& p, cudaStream_t st, int key_split = 1);   // (d = 64; with a block mask also d = 128; key_split 2 / 4: the keys of a tile over a CTA cluster)
 int launch_fused_tc3(const Problem& p, cudaStream_t st);

@@ -29,6 +29,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include <type_traits>
 
 #include "flat_internal.cuh"
@@ -209,7 +211,7 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     using LY = L2<D, NT, BIAS == 2>;
     static_assert(BIAS != 2 || (NT == 2 && D == 64 && !VL && !SPARSE && CS == 1), "staged bias: the two-tile dense kernel, d = 64");
     static_assert(!SPARSE || (NT == 1 && !VL && !BIAS), "the pruning map is read by the one-tile dense kernel");
-    static_assert(CS == 1 || ((NT == 1 || KH) && !VL && !BIAS && !SPARSE && (CS == 2 || CS == 4 || CS == 8)), "key split: one-tile dense kernel");
+    static_assert(CS == 1 || ((NT == 1 || KH) && !VL && !BIAS && !SPARSE && (CS == 2 || CS == 4 || CS == 8 || CS == 16)), "key split: one-tile dense kernel");
     static_assert(!KH || (NT == 2 && D == 64 && !VL && !BIAS && !SPARSE), "key halves: two warpgroups on one dense d = 64 tile");
     constexpr int QT = KH ? 1 : NT;                      // query tiles of the CTA
     __shared__ uint16_t tile_list[SPARSE ? 1024 : 1];    // the kept key tiles of this query tile, ascending
@@ -813,7 +815,7 @@ bool make_bias_map(CUtensorMap* m, const Problem& p) {
 }
 
 template <int D, int NT>
-int launch_tc2_d(const Problem& p, cudaStream_t st, int key_split = 1) {
+int launch_tc2_d(const Problem& p, cudaStream_t st, int key_split = 1, bool only_if_resident = false) {
     using LY = L2<D, NT>;
     CUtensorMap tmQ, tmK, tmV;
     const int BH = p.B * p.H;
@@ -858,12 +860,45 @@ int launch_tc2_d(const Problem& p, cudaStream_t st, int key_split = 1) {
         }
     }
     if constexpr (NT == 1) {
-        if (key_split == 2 || key_split == 4 || key_split == 8) {
-            // the keys of every query tile over a cluster of 2, 4 or 8 CTAs (consecutive along x)
+        if (key_split == 2 || key_split == 4 || key_split == 8 || (key_split == 16 && D == 128)) {
+            // the keys of every query tile over a cluster of 2, 4, 8 or 16 CTAs (consecutive along x)
             auto launch = [&](auto cs_tag) -> int {
                 constexpr int CS = decltype(cs_tag)::value;
                 constexpr int BYTES = LY::SMEM_BYTES + LY::merge_bytes(CS);
                 if (!ensure_dynamic_smem<fused_tc2_kernel<D, NT, false, false, false, CS>>(BYTES)) return FLAT_ERR_CUDA;
+                if constexpr (CS > 8) {
+                    // sixteen CTAs are more than the portable cluster size: the kernel must opt in, and the device
+                    // must be able to hold such a cluster at all (sixteen free SMs in one GPC: asked once per device)
+                    static std::atomic<uint64_t> asked{0};
+                    static std::atomic<int> resident[64];       // clusters of sixteen the device holds at a time
+                    int dev = 0;
+                    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return FLAT_ERR_UNSUPPORTED;
+                    const uint64_t bit = 1ull << dev;
+                    if (!(asked.load(std::memory_order_acquire) & bit)) {
+                        int n = 0;
+                        bool good = cudaFuncSetAttribute(fused_tc2_kernel<D, NT, false, false, false, CS>,
+                                                         cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess;
+                        if (good) {
+                            cudaLaunchConfig_t q = {};
+                            q.gridDim = dim3(CS, 1);
+                            q.blockDim = dim3(LY::THREADS);
+                            q.dynamicSmemBytes = BYTES;
+                            cudaLaunchAttribute a[1];
+                            a[0].id = cudaLaunchAttributeClusterDimension;
+                            a[0].val.clusterDim.x = CS; a[0].val.clusterDim.y = 1; a[0].val.clusterDim.z = 1;
+                            q.attrs = a;
+                            q.numAttrs = 1;
+                            good = cudaOccupancyMaxActiveClusters(&n, fused_tc2_kernel<D, NT, false, false, false, CS>, &q) == cudaSuccess && n >= 1;
+                        }
+                        if (!good) { cudaGetLastError(); n = 0; }
+                        resident[dev].store(n, std::memory_order_release);
+                        asked.fetch_or(bit, std::memory_order_release);
+                    }
+                    const int fit = resident[dev].load(std::memory_order_acquire);
+                    // (the dispatcher only wants them when all clusters of the launch run at once: 8 clusters of sixteen
+                    // one-per-SM CTAs took 80 us where clusters of eight take 41)
+                    if (fit < 1 || (only_if_resident && static_cast<int64_t>(grid.x) * grid.y > fit)) return FLAT_ERR_UNSUPPORTED;
+                }
                 cudaLaunchConfig_t cfg = {};
                 cfg.gridDim = dim3(grid.x * CS, grid.y);
                 cfg.blockDim = dim3(LY::THREADS);
@@ -883,6 +918,9 @@ int launch_tc2_d(const Problem& p, cudaStream_t st, int key_split = 1) {
                     BiasArg{nullptr, 0, 0, 0, 0}, static_cast<const uint8_t*>(nullptr), 0ll, 0ll, CUtensorMap{});
                 return e == cudaSuccess ? FLAT_OK : FLAT_ERR_CUDA;
             };
+            if constexpr (D == 128) {
+                if (key_split == 16) return launch(std::integral_constant<int, 16>{});
+            }
             return key_split == 2 ? launch(std::integral_constant<int, 2>{})
                    : key_split == 4 ? launch(std::integral_constant<int, 4>{}) : launch(std::integral_constant<int, 8>{});
         }
@@ -1023,11 +1061,12 @@ int launch_fused_tc2_halves(const Problem& p, cudaStream_t st, int key_split) {
 }
 
 // One 128-row tile per CTA, two CTAs per SM (d = 64 only: at d = 128 two CTAs do not fit in shared memory).
-int launch_fused_tc2_single(const Problem& p, cudaStream_t st, int key_split) {
+int launch_fused_tc2_single(const Problem& p, cudaStream_t st, int key_split, bool only_if_resident) {
     if (p.dtype != FLAT_DTYPE_BF16) return FLAT_ERR_UNSUPPORTED;
     if (key_split != 1 && (p.bias || p.block_mask)) return FLAT_ERR_UNSUPPORTED;
     if (p.d == 64) return launch_tc2_d<64, 1>(p, st, key_split);
-    if (p.d == 128 && (p.block_mask || key_split != 1)) return launch_tc2_d<128, 1>(p, st, key_split);   // (one CTA per SM: the pruned path and the key split)
+    if (key_split == 16 && p.d != 128) return FLAT_ERR_UNSUPPORTED;      // (sixteen-CTA clusters: built for d = 128, one CTA per SM)
+    if (p.d == 128 && (p.block_mask || key_split != 1)) return launch_tc2_d<128, 1>(p, st, key_split, only_if_resident);   // (one CTA per SM: the pruned path and the key split)
     return FLAT_ERR_UNSUPPORTED;
 }
 

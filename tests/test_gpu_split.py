@@ -107,7 +107,7 @@ def test_auto_takes_the_split_for_underfilled_launches(api):
         check_bf16(O, ref, "auto split %s" % ((B, H, Nq, Nk),))
 
 
-@pytest.mark.parametrize("variant", [8, 9, 10])          # (the two-warpgroup form is built for d = 64)
+@pytest.mark.parametrize("variant", [8, 9, 10, 15])      # (the two-warpgroup form is built for d = 64; 15: clusters of sixteen)
 @pytest.mark.parametrize("shape", [(1, 2, 128, 128), (2, 2, 200, 333), (1, 3, 300, 2100), (1, 1, 77, 4096)])
 def test_head_size_128(api, shape, variant):
     B, H, Nq, Nk = shape
@@ -126,7 +126,7 @@ def test_head_size_128(api, shape, variant):
 def test_auto_takes_the_split_at_head_size_128(api):
     rng = np.random.default_rng(19)
     for (B, H, Nq, Nk, expect) in [(1, 8, 128, 16384, api.FLAT_VARIANT_TC2_SPLIT8), (1, 8, 512, 4096, api.FLAT_VARIANT_TC2_SPLIT4),
-                                   (4, 16, 2048, 2048, api.FLAT_VARIANT_TC2)]:
+                                   (1, 2, 128, 8192, api.FLAT_VARIANT_TC2_SPLIT16), (4, 16, 2048, 2048, api.FLAT_VARIANT_TC2)]:
         Qb, Kb, Vb = rand_bits(rng, (B, H, Nq, 128)), rand_bits(rng, (B, H, Nk, 128)), rand_bits(rng, (B, H, Nk, 128))
         rows = inputs.sample_rows(inputs.Workload("x", B, H, Nq, Nk, 128), 4)
         ref = oracle.attention(Qb, Kb, Vb, 0.1, rows=rows)["O"]
