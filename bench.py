@@ -45,7 +45,8 @@ KERNEL_OF_VARIANT = {1: "fused_simt_kernel", 2: "fused_tc_kernel", 3: "fused_tc2
                      12: "fused_tc2_kernel<1 tile, two warpgroups, keys over a 2-CTA cluster>",
                      13: "fused_tc2_kernel<1 tile, two warpgroups, keys over a 4-CTA cluster>",
                      14: "fused_tc2_kernel<1 tile, two warpgroups, keys over an 8-CTA cluster>",
-                     15: "fused_tc2_kernel<1 tile, keys over a 16-CTA cluster>"}
+                     15: "fused_tc2_kernel<1 tile, keys over a 16-CTA cluster>",
+                     16: "fused_tc2_kernel<1 tile, two warpgroups, keys over a 16-CTA cluster>"}
 TF32_OVER_BF16 = 1.1 / 2.25          # nominal dense tensor peaks: the tf32 roofline is the measured bf16 peak times this
 
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel from ncu

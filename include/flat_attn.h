@@ -93,8 +93,9 @@ enum {
     FLAT_VARIANT_TC2_HALVES_SPLIT2 = 12, /* the same with the keys also split over a cluster of two CTAs     */
     FLAT_VARIANT_TC2_HALVES_SPLIT4 = 13, /* ... of four CTAs                                             */
     FLAT_VARIANT_TC2_HALVES_SPLIT8 = 14, /* ... of eight CTAs                                            */
-    FLAT_VARIANT_TC2_SPLIT16 = 15 /* TC2_SPLIT2 over a cluster of sixteen CTAs (more than the portable cluster size:
+    FLAT_VARIANT_TC2_SPLIT16 = 15, /* TC2_SPLIT2 over a cluster of sixteen CTAs (more than the portable cluster size:
                                   taken only where the device can hold such a cluster): bf16, d = 128       */
+    FLAT_VARIANT_TC2_HALVES_SPLIT16 = 16 /* TC2_HALVES over a cluster of sixteen CTAs: bf16, d = 64               */
 };
 
 typedef struct flat_attn_params {

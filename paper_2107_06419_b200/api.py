@@ -29,7 +29,7 @@ FLAT_VARIANT_RGRAN = 6
 FLAT_VARIANT_TF32 = 7
 FLAT_VARIANT_TC2_SPLIT2, FLAT_VARIANT_TC2_SPLIT4, FLAT_VARIANT_TC2_SPLIT8 = 8, 9, 10
 FLAT_VARIANT_TC2_HALVES, FLAT_VARIANT_TC2_HALVES_SPLIT2, FLAT_VARIANT_TC2_HALVES_SPLIT4, FLAT_VARIANT_TC2_HALVES_SPLIT8 = 11, 12, 13, 14
-FLAT_VARIANT_TC2_SPLIT16 = 15
+FLAT_VARIANT_TC2_SPLIT16, FLAT_VARIANT_TC2_HALVES_SPLIT16 = 15, 16
 
 EXPORTS = ["flat_attn_fwd", "flat_attn_fwd_ex", "flat_attn_naive_fwd", "flat_attn_naive_fwd_ex",
            "flat_attn_naive_fwd_static", "flat_attn_selftest_wait_timeout", "flat_attn_selftest_exp2_poly",

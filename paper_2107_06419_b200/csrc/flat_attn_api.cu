@@ -54,7 +54,7 @@ int validate(const flat_attn_params_t* p, flat::Problem* out) {
     if (bh * static_cast<int64_t>(p->Nq > p->Nk ? p->Nq : p->Nk) > lim / p->d) return FLAT_ERR_SHAPE;
     if (p->dtype != FLAT_DTYPE_BF16 && p->dtype != FLAT_DTYPE_F32) return FLAT_ERR_UNSUPPORTED;
     if (p->d != 16 && p->d != 32 && p->d != 64 && p->d != 128) return FLAT_ERR_UNSUPPORTED;
-    if (p->variant < FLAT_VARIANT_AUTO || p->variant > FLAT_VARIANT_TC2_SPLIT16) return FLAT_ERR_UNSUPPORTED;
+    if (p->variant < FLAT_VARIANT_AUTO || p->variant > FLAT_VARIANT_TC2_HALVES_SPLIT16) return FLAT_ERR_UNSUPPORTED;
     if (!aligned16(p->Q) || !aligned16(p->K) || !aligned16(p->V) || !aligned16(p->O)) return FLAT_ERR_ALIGN;
     if (p->k_valid_len && (reinterpret_cast<uintptr_t>(p->k_valid_len) & 3u)) return FLAT_ERR_ALIGN;
     if (p->status && (reinterpret_cast<uintptr_t>(p->status) & 3u)) return FLAT_ERR_ALIGN;
@@ -142,10 +142,11 @@ int run_fused(const flat::Problem& q, int variant, cudaStream_t st) {
                 // cluster that leaves each warpgroup a key tile and fits -- eight-CTA clusters of one-per-SM CTAs
                 // only up to half the SMs, beyond that they no longer all start at once (measured on 16 tiles x
                 // 16 key tiles: 17.1 us against 9.6 with clusters of four).
-                for (int cs = 8; cs >= 1 && key_tiles >= 2; cs /= 2) {
-                    if (ctas1 * cs > (cs == 8 ? sms / 2 : 7 * sms / 8)) continue;
+                for (int cs = 16; cs >= 1 && key_tiles >= 2; cs /= 2) {
+                    if (ctas1 * cs > (cs >= 8 ? sms / 2 : 7 * sms / 8)) continue;
                     if (key_tiles < 2 * cs) continue;
-                    v = cs == 8 ? FLAT_VARIANT_TC2_HALVES_SPLIT8 : cs == 4 ? FLAT_VARIANT_TC2_HALVES_SPLIT4
+                    if (cs == 16 && ctas1 > 2) continue;     // (clusters of sixteen: for one or two query tiles, see d = 128 below)
+                    v = cs == 16 ? FLAT_VARIANT_TC2_HALVES_SPLIT16 : cs == 8 ? FLAT_VARIANT_TC2_HALVES_SPLIT8 : cs == 4 ? FLAT_VARIANT_TC2_HALVES_SPLIT4
                         : cs == 2 ? FLAT_VARIANT_TC2_HALVES_SPLIT2 : FLAT_VARIANT_TC2_HALVES;
                     break;
                 }
@@ -172,10 +173,17 @@ int run_fused(const flat::Problem& q, int variant, cudaStream_t st) {
     if (q.causal && v == FLAT_VARIANT_TC) return FLAT_ERR_UNSUPPORTED;
     if (q.lse && (v == FLAT_VARIANT_TC || v == FLAT_VARIANT_RGRAN)) return FLAT_ERR_UNSUPPORTED;
     if (q.bias && v != FLAT_VARIANT_TC2 && v != FLAT_VARIANT_SIMT) return FLAT_ERR_UNSUPPORTED;
-    if (v >= FLAT_VARIANT_TC2_HALVES && v <= FLAT_VARIANT_TC2_HALVES_SPLIT8) {
+    if ((v >= FLAT_VARIANT_TC2_HALVES && v <= FLAT_VARIANT_TC2_HALVES_SPLIT8) || v == FLAT_VARIANT_TC2_HALVES_SPLIT16) {
         if (!tc_applies(q) || q.d != 64 || q.block_mask || q.bias) return FLAT_ERR_UNSUPPORTED;
+        const int cs = v == FLAT_VARIANT_TC2_HALVES_SPLIT16 ? 16 : 1 << (v - FLAT_VARIANT_TC2_HALVES);
+        int rc = flat::launch_fused_tc2_halves(q, st, cs, variant == FLAT_VARIANT_AUTO);
+        if (rc == FLAT_ERR_UNSUPPORTED && cs == 16 && variant == FLAT_VARIANT_AUTO) {
+            // (AUTO asked for sixteen and the device cannot hold all the launch's clusters at once: eight)
+            v = FLAT_VARIANT_TC2_HALVES_SPLIT8;
+            rc = flat::launch_fused_tc2_halves(q, st, 8);
+        }
         g_last_variant = v;
-        return flat::launch_fused_tc2_halves(q, st, 1 << (v - FLAT_VARIANT_TC2_HALVES));
+        return rc;
     }
     if (v == FLAT_VARIANT_TC2_SPLIT2 || v == FLAT_VARIANT_TC2_SPLIT4 || v == FLAT_VARIANT_TC2_SPLIT8 || v == FLAT_VARIANT_TC2_SPLIT16) {
         if (!tc_applies(q) || q.block_mask || (v == FLAT_VARIANT_TC2_SPLIT16 && q.d != 128)) return FLAT_ERR_UNSUPPORTED;

@@ -71,7 +71,7 @@ int launch_fused_tc2(const Problem& p, cudaStream_t st);      // (also the tenso
 // FLAT_ERR_UNSUPPORTED)
 int launch_fused_tc2_single(const Problem& p, cudaStream_t st, int key_split = 1, bool only_if_resident = false);
 // The same tile worked on by two warpgroups that take alternate key tiles (bf16, d = 64, dense; key_split 1, 2, 4, 8).
-int launch_fused_tc2_halves(const Problem& p, cudaStream_t st, int key_split = 1);   // (d = 64; with a block mask also d = 128; key_split 2 / 4: the keys of a tile over a CTA cluster)
+int launch_fused_tc2_halves(const Problem& p, cudaStream_t st, int key_split = 1, bool only_if_resident = false);   // (key_split 1, 2, 4, 8, 16)   // (d = 64; with a block mask also d = 128; key_split 2 / 4: the keys of a tile over a CTA cluster)
 int launch_fused_tc3(const Problem& p, cudaStream_t st);
 // How the last launch_fused_tc3 of this host thread dealt its items (FLAT_SCHEDULE_*; 0 before any).
 extern thread_local int g_last_schedule;

@@ -814,6 +814,38 @@ bool make_bias_map(CUtensorMap* m, const Problem& p) {
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Clusters of sixteen CTAs are more than the portable cluster size: the kernel must opt in, and the device must be
+// able to hold such a cluster at all (sixteen free SMs in one GPC).  Asked once per kernel and device; returns the
+// number of such clusters the device holds at a time (0: none, or the query failed).
+template <auto kern>                                     // (one set of flags per kernel, not per kernel type)
+int clusters_of_sixteen(int threads, int bytes) {
+    static std::atomic<uint64_t> asked{0};
+    static std::atomic<int> resident[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
+    const uint64_t bit = 1ull << dev;
+    if (!(asked.load(std::memory_order_acquire) & bit)) {
+        int n = 0;
+        bool good = cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess;
+        if (good) {
+            cudaLaunchConfig_t q = {};
+            q.gridDim = dim3(16, 1);
+            q.blockDim = dim3(threads);
+            q.dynamicSmemBytes = bytes;
+            cudaLaunchAttribute a[1];
+            a[0].id = cudaLaunchAttributeClusterDimension;
+            a[0].val.clusterDim.x = 16; a[0].val.clusterDim.y = 1; a[0].val.clusterDim.z = 1;
+            q.attrs = a;
+            q.numAttrs = 1;
+            good = cudaOccupancyMaxActiveClusters(&n, kern, &q) == cudaSuccess && n >= 1;
+        }
+        if (!good) { cudaGetLastError(); n = 0; }
+        resident[dev].store(n, std::memory_order_release);
+        asked.fetch_or(bit, std::memory_order_release);
+    }
+    return resident[dev].load(std::memory_order_acquire);
+}
+
 template <int D, int NT>
 int launch_tc2_d(const Problem& p, cudaStream_t st, int key_split = 1, bool only_if_resident = false) {
     using LY = L2<D, NT>;
@@ -867,36 +899,9 @@ int launch_tc2_d(const Problem& p, cudaStream_t st, int key_split = 1, bool only
                 constexpr int BYTES = LY::SMEM_BYTES + LY::merge_bytes(CS);
                 if (!ensure_dynamic_smem<fused_tc2_kernel<D, NT, false, false, false, CS>>(BYTES)) return FLAT_ERR_CUDA;
                 if constexpr (CS > 8) {
-                    // sixteen CTAs are more than the portable cluster size: the kernel must opt in, and the device
-                    // must be able to hold such a cluster at all (sixteen free SMs in one GPC: asked once per device)
-                    static std::atomic<uint64_t> asked{0};
-                    static std::atomic<int> resident[64];       // clusters of sixteen the device holds at a time
-                    int dev = 0;
-                    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return FLAT_ERR_UNSUPPORTED;
-                    const uint64_t bit = 1ull << dev;
-                    if (!(asked.load(std::memory_order_acquire) & bit)) {
-                        int n = 0;
-                        bool good = cudaFuncSetAttribute(fused_tc2_kernel<D, NT, false, false, false, CS>,
-                                                         cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess;
-                        if (good) {
-                            cudaLaunchConfig_t q = {};
-                            q.gridDim = dim3(CS, 1);
-                            q.blockDim = dim3(LY::THREADS);
-                            q.dynamicSmemBytes = BYTES;
-                            cudaLaunchAttribute a[1];
-                            a[0].id = cudaLaunchAttributeClusterDimension;
-                            a[0].val.clusterDim.x = CS; a[0].val.clusterDim.y = 1; a[0].val.clusterDim.z = 1;
-                            q.attrs = a;
-                            q.numAttrs = 1;
-                            good = cudaOccupancyMaxActiveClusters(&n, fused_tc2_kernel<D, NT, false, false, false, CS>, &q) == cudaSuccess && n >= 1;
-                        }
-                        if (!good) { cudaGetLastError(); n = 0; }
-                        resident[dev].store(n, std::memory_order_release);
-                        asked.fetch_or(bit, std::memory_order_release);
-                    }
-                    const int fit = resident[dev].load(std::memory_order_acquire);
                     // (the dispatcher only wants them when all clusters of the launch run at once: 8 clusters of sixteen
                     // one-per-SM CTAs took 80 us where clusters of eight take 41)
+                    const int fit = clusters_of_sixteen<fused_tc2_kernel<D, NT, false, false, false, CS>>(LY::THREADS, BYTES);
                     if (fit < 1 || (only_if_resident && static_cast<int64_t>(grid.x) * grid.y > fit)) return FLAT_ERR_UNSUPPORTED;
                 }
                 cudaLaunchConfig_t cfg = {};
@@ -956,7 +961,7 @@ int launch_tc2_d(const Problem& p, cudaStream_t st, int key_split = 1, bool only
 
 // Key halves (see the kernel's KH): d = 64, dense, one 128-row tile per CTA worked on by two warpgroups, optionally
 // with the keys over a cluster on top.  One CTA per SM (all 512 TMEM columns).
-int launch_tc2_kh(const Problem& p, cudaStream_t st, int key_split) {
+int launch_tc2_kh(const Problem& p, cudaStream_t st, int key_split, bool only_if_resident) {
     constexpr int D = 64, NT = 2;
     using LY = L2<D, NT>;
     CUtensorMap tmQ, tmK, tmV;
@@ -970,6 +975,10 @@ int launch_tc2_kh(const Problem& p, cudaStream_t st, int key_split) {
         constexpr int BYTES = LY::SMEM_BYTES + LY::merge_bytes(CS) + 128 * merge_vecs(D) * 16;
         auto kern = fused_tc2_kernel<D, NT, false, 0, false, CS, true>;
         if (!ensure_dynamic_smem<fused_tc2_kernel<D, NT, false, 0, false, CS, true>>(BYTES)) return FLAT_ERR_CUDA;
+        if constexpr (CS > 8) {
+            const int fit = clusters_of_sixteen<fused_tc2_kernel<D, NT, false, 0, false, CS, true>>(LY::THREADS, BYTES);
+            if (fit < 1 || (only_if_resident && static_cast<int64_t>(grid.x) * grid.y > fit)) return FLAT_ERR_UNSUPPORTED;
+        }
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(grid.x * CS, grid.y);
         cfg.blockDim = dim3(LY::THREADS);
@@ -992,7 +1001,8 @@ int launch_tc2_kh(const Problem& p, cudaStream_t st, int key_split) {
     return key_split == 1   ? launch(std::integral_constant<int, 1>{})
            : key_split == 2 ? launch(std::integral_constant<int, 2>{})
            : key_split == 4 ? launch(std::integral_constant<int, 4>{})
-           : key_split == 8 ? launch(std::integral_constant<int, 8>{}) : FLAT_ERR_UNSUPPORTED;
+           : key_split == 8 ? launch(std::integral_constant<int, 8>{})
+           : key_split == 16 ? launch(std::integral_constant<int, 16>{}) : FLAT_ERR_UNSUPPORTED;
 }
 
 }  // namespace
@@ -1055,9 +1065,9 @@ int launch_fused_tc2(const Problem& p, cudaStream_t st) {
     return FLAT_ERR_UNSUPPORTED;
 }
 
-int launch_fused_tc2_halves(const Problem& p, cudaStream_t st, int key_split) {
+int launch_fused_tc2_halves(const Problem& p, cudaStream_t st, int key_split, bool only_if_resident) {
     if (p.dtype != FLAT_DTYPE_BF16 || p.d != 64 || p.bias || p.block_mask) return FLAT_ERR_UNSUPPORTED;
-    return launch_tc2_kh(p, st, key_split);
+    return launch_tc2_kh(p, st, key_split, only_if_resident);
 }
 
 // One 128-row tile per CTA, two CTAs per SM (d = 64 only: at d = 128 two CTAs do not fit in shared memory).

@@ -42,6 +42,7 @@ VARIANTS = {
     api.FLAT_VARIANT_TC2_HALVES_SPLIT4: "tc2_halves_split4: ... of 4 CTAs",
     api.FLAT_VARIANT_TC2_HALVES_SPLIT8: "tc2_halves_split8: ... of 8 CTAs",
     api.FLAT_VARIANT_TC2_SPLIT16: "tc2_split16: keys over a cluster of 16 CTAs (d = 128)",
+    api.FLAT_VARIANT_TC2_HALVES_SPLIT16: "tc2_halves_split16: two warpgroups per tile, keys over a cluster of 16 CTAs (d = 64)",
     api.FLAT_VARIANT_AUTO: "auto (the dispatcher's choice)",
 }
 

@@ -102,7 +102,7 @@ def test_projection_argument_errors(api):
     (dict(B=0), 2), (dict(Nk=-3), 2), (dict(scale=float("inf")), 2), (dict(scale=float("nan")), 2),
     (dict(B=70000), 2), (dict(B=60000, Nq=2 ** 31 - 1, Nk=2 ** 31 - 1), 2),
     (dict(d=48), 3), (dict(d=256), 3), (dict(dtype=2), 3), (dict(variant=9, dtype=1), 3),
-    (dict(dtype=1, variant=2), 3), (dict(dtype=1, variant=3), 3), (dict(d=16, variant=3), 3), (dict(d=128, variant=4), 3), (dict(variant=7), 3), (dict(variant=16), 3), (dict(variant=15, d=32), 3), (dict(variant=11, d=128), 3), (dict(variant=14, dtype=1), 3), (dict(variant=8, d=32), 3), (dict(variant=10, dtype=1), 3), (dict(dtype=1, variant=7, d=128), 3), (dict(dtype=1, variant=7, d=32), 3), (dict(variant=6, Nk=513), 3), (dict(variant=6, d=128), 3), (dict(variant=6, dtype=1), 3), (dict(dtype=1, variant=5), 3), (dict(d=32, variant=5), 3), (dict(d=128, variant=5), 3), (dict(causal=2), 3), (dict(causal=-1), 3), (dict(causal=1, variant=2), 3), (dict(causal=1, variant=2, d=128), 3),                               # tensor-core kernel is bf16 only
+    (dict(dtype=1, variant=2), 3), (dict(dtype=1, variant=3), 3), (dict(d=16, variant=3), 3), (dict(d=128, variant=4), 3), (dict(variant=7), 3), (dict(variant=17), 3), (dict(variant=15, d=32), 3), (dict(variant=16, d=128), 3), (dict(variant=11, d=128), 3), (dict(variant=14, dtype=1), 3), (dict(variant=8, d=32), 3), (dict(variant=10, dtype=1), 3), (dict(dtype=1, variant=7, d=128), 3), (dict(dtype=1, variant=7, d=32), 3), (dict(variant=6, Nk=513), 3), (dict(variant=6, d=128), 3), (dict(variant=6, dtype=1), 3), (dict(dtype=1, variant=5), 3), (dict(d=32, variant=5), 3), (dict(d=128, variant=5), 3), (dict(causal=2), 3), (dict(causal=-1), 3), (dict(causal=1, variant=2), 3), (dict(causal=1, variant=2, d=128), 3),                               # tensor-core kernel is bf16 only
     (dict(d=32, variant=2), 3),
     (dict(K=0x20008), 4), (dict(k_valid_len=0x50002), 4),
 ])

@@ -33,7 +33,7 @@ def cases(seed, count):
     return out
 
 
-BF16_VARIANTS = [0, 1, 2, 3, 4, 5, 8, 9, 10, 11, 12, 13, 14]
+BF16_VARIANTS = [0, 1, 2, 3, 4, 5, 8, 9, 10, 11, 12, 13, 14, 15, 16]
 
 
 @pytest.mark.parametrize("case", cases(20210706, 96), ids=lambda c: "B%dH%dq%dk%dd%d%s%s" % (c[0], c[1], c[2], c[3], c[4], "c" if c[5] else "", "m%d" % c[6]))

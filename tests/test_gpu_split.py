@@ -14,7 +14,7 @@ pytestmark = pytest.mark.gpu
 
 # FLAT_VARIANT_TC2_SPLIT2 / 4 / 8, then FLAT_VARIANT_TC2_HALVES and HALVES_SPLIT2 / 4 / 8 (the tile's two warpgroups
 # on alternate key tiles, merged through shared memory, with the keys over a cluster on top)
-SPLITS = [8, 9, 10, 11, 12, 13, 14]
+SPLITS = [8, 9, 10, 11, 12, 13, 14, 16]           # (16: the two-warpgroup form over clusters of sixteen)
 
 
 @pytest.fixture(scope="module")
@@ -96,7 +96,7 @@ def test_auto_takes_the_split_for_underfilled_launches(api):
     if sms != 148:
         pytest.skip("the expected choices are those of a 148-SM GPU")
     # (more tiles than seven SMs in eight: two-per-SM CTAs, unsplit; one key tile: nothing to split)
-    for (B, H, Nq, Nk, expect) in [(1, 1, 128, 8192, api.FLAT_VARIANT_TC2_HALVES_SPLIT8), (1, 12, 512, 512, api.FLAT_VARIANT_TC2_HALVES_SPLIT2),
+    for (B, H, Nq, Nk, expect) in [(1, 1, 128, 8192, api.FLAT_VARIANT_TC2_HALVES_SPLIT16), (1, 4, 128, 4096, api.FLAT_VARIANT_TC2_HALVES_SPLIT8), (1, 12, 512, 512, api.FLAT_VARIANT_TC2_HALVES_SPLIT2),
                                    (1, 12, 512, 2048, api.FLAT_VARIANT_TC2_HALVES_SPLIT2), (1, 8, 256, 2048, api.FLAT_VARIANT_TC2_HALVES_SPLIT4),
                                    (1, 24, 512, 1024, api.FLAT_VARIANT_TC2_HALVES), (1, 34, 512, 512, api.FLAT_VARIANT_TC2_SINGLE),
                                    (1, 2, 128, 128, api.FLAT_VARIANT_TC2_SINGLE)]:
