@@ -53,10 +53,17 @@ __host__ __device__ constexpr int merge_vecs(int d) { return d / 4 + 1; }   // (
 constexpr float OVERFLOW_SUM = 1.0995116e12f;   // 2^40: a tile row sum beyond this means m_ref is stale
 
 // BT: the bias tile of every (tile, step) is staged through shared memory by TMA (two stages per query tile)
-template <int D, int NT, bool BT = false> struct L2 {
+// KHL (the two warpgroups of a CTA on alternate key tiles of ONE query tile, see the kernel's KH): every key tile has one
+// consumer, the warpgroup of its parity, so the ring depths must be even -- stage g % depth then always belongs to
+// the same warpgroup and a parity wait on its barrier is unambiguous.  (With three stages a stage alternates between
+// the two consumers, each of which always waits for the SAME parity of its barrier, and a warpgroup that had run
+// ahead could take the completion of its previous fill for that of the next one: wrong keys, then a stuck ring.
+// Seen as rare wrong rows and time-outs on masked batches.)  1: four K and four V stages; 2: four and two (the
+// sixteen-CTA cluster's receive buffer leaves no room for more).
+template <int D, int NT, bool BT = false, int KHL = 0> struct L2 {
     static constexpr bool ALIAS = (D == 128);            // P overlays S
-    static constexpr int KS = (NT == 1 || BT) ? 2 : (D == 64) ? 3 : 2;   // K ring depth
-    static constexpr int VS = KS;                        // V ring depth
+    static constexpr int KS = KHL ? 4 : (NT == 1 || BT) ? 2 : (D == 64) ? 3 : 2;   // K ring depth
+    static constexpr int VS = KHL == 2 ? 2 : KS;         // V ring depth
     static constexpr int THREADS = 128 * NT + 128;       // NT softmax warpgroups + {TMA, NT MMA issuers, idle}
     static constexpr int SOFT_WARPS = 4 * NT;
     static constexpr uint32_t TMEM_COLS = (NT == 2) ? 512 : 256;
@@ -208,7 +215,7 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                  float* __restrict__ lse = nullptr, BiasArg bias = BiasArg{nullptr, 0, 0, 0, 0},
                  const uint8_t* __restrict__ block_mask = nullptr, long long bmask_sb = 0, long long bmask_sh = 0,
                  const __grid_constant__ CUtensorMap tmBias = CUtensorMap{}) {
-    using LY = L2<D, NT, BIAS == 2>;
+    using LY = L2<D, NT, BIAS == 2, KH ? (CS == 16 ? 2 : 1) : 0>;
     static_assert(BIAS != 2 || (NT == 2 && D == 64 && !VL && !SPARSE && CS == 1), "staged bias: the two-tile dense kernel, d = 64");
     static_assert(!SPARSE || (NT == 1 && !VL && !BIAS), "the pruning map is read by the one-tile dense kernel");
     static_assert(CS == 1 || ((NT == 1 || KH) && !VL && !BIAS && !SPARSE && (CS == 2 || CS == 4 || CS == 8 || CS == 16)), "key split: one-tile dense kernel");
@@ -729,9 +736,14 @@ fused_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                     if (owner != crank && lane % GRP == 0) mbar_arrive_cluster(mapa_shared(smem_u32(&bars[LY::MERGE_BAR]), owner));
                     writer = owner == crank;
                     if (writer) {
+                        // An owner must not leave before its senders have stored (a remote store into the shared
+                        // memory of a CTA that has left is a fault).  Every sender stores and arrives whatever
+                        // happened to it: its roles give up at their first wait that runs out (WAIT_CYCLES) and go
+                        // straight to the exchange, and the CTAs of a cluster start together -- so the owner waits
+                        // four times as long as any sender can take before it gives up itself.
                         const long long t0 = clock64();
                         while (!mbar_try_wait_cluster(&bars[LY::MERGE_BAR], 0)) {
-                            if (clock64() - t0 > WAIT_CYCLES) {
+                            if (clock64() - t0 > 4 * WAIT_CYCLES) {
                                 writer = false;
                                 if (status) atomicExch(status, 0x350);
                                 break;
@@ -963,7 +975,6 @@ int launch_tc2_d(const Problem& p, cudaStream_t st, int key_split = 1, bool only
 // with the keys over a cluster on top.  One CTA per SM (all 512 TMEM columns).
 int launch_tc2_kh(const Problem& p, cudaStream_t st, int key_split, bool only_if_resident) {
     constexpr int D = 64, NT = 2;
-    using LY = L2<D, NT>;
     CUtensorMap tmQ, tmK, tmV;
     const int BH = p.B * p.H;
     if (!make_map(&tmQ, p.Q, BH, p.Nq, D, BM) || !make_map(&tmK, p.K, BH, p.Nk, D, BN) ||
@@ -972,7 +983,9 @@ int launch_tc2_kh(const Problem& p, cudaStream_t st, int key_split, bool only_if
     const dim3 grid((p.Nq + BM - 1) / BM, BH);
     auto launch = [&](auto cs_tag) -> int {
         constexpr int CS = decltype(cs_tag)::value;
+        using LY = L2<D, NT, false, CS == 16 ? 2 : 1>;   // (the kernel's own choice of ring depths)
         constexpr int BYTES = LY::SMEM_BYTES + LY::merge_bytes(CS) + 128 * merge_vecs(D) * 16;
+        static_assert(BYTES <= 232448, "shared memory of the two-warpgroup form");
         auto kern = fused_tc2_kernel<D, NT, false, 0, false, CS, true>;
         if (!ensure_dynamic_smem<fused_tc2_kernel<D, NT, false, 0, false, CS, true>>(BYTES)) return FLAT_ERR_CUDA;
         if constexpr (CS > 8) {
