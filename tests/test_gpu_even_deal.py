@@ -243,3 +243,36 @@ def test_two_host_threads_on_two_streams(api):
         for O, status in results[k]:
             assert int(status.item()) == 0
             check_bf16(bf16_to_f64(O).reshape(-1, 64)[rows], ref, "thread %d" % k)
+
+
+def test_while_another_stream_holds_sms(api):
+    """The launch is not a cooperative one: when another stream's kernels hold SMs, some CTAs start late and a CTA
+    that waits for another's part may spin for a while.  Every launch must still finish without a device code and
+    with the bits of an undisturbed launch."""
+    w = inputs.WORKLOADS["c5_cross_masked"]
+    g = torch.Generator(device="cuda").manual_seed(43)
+    Q = torch.randn(w.B, w.H, w.Nq, 64, device="cuda", dtype=torch.bfloat16, generator=g)
+    K = torch.randn(w.B, w.H, w.Nk, 64, device="cuda", dtype=torch.bfloat16, generator=g)
+    V = torch.randn(w.B, w.H, w.Nk, 64, device="cuda", dtype=torch.bfloat16, generator=g)
+    vlt = torch.from_numpy(inputs.make_valid_len(w)).cuda()
+    ref = torch.empty_like(Q)
+    status0 = torch.zeros(1, dtype=torch.int32, device="cuda")
+    api.flat_attn_fwd_ex(Q, K, V, ref, w.scale, k_valid_len=vlt, status=status0, variant=api.FLAT_VARIANT_TC3)
+    torch.cuda.synchronize()
+    assert api.flat_attn_last_schedule() == api.FLAT_SCHEDULE_EVEN_DEAL and int(status0.item()) == 0
+    A = torch.randn(8192, 8192, device="cuda", dtype=torch.bfloat16, generator=g)
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    n = 40
+    status = torch.zeros(n, dtype=torch.int32, device="cuda")
+    outs = []
+    for it in range(n):
+        with torch.cuda.stream(s1):
+            _ = A @ A                                    # (a library GEMM as the disturbance: all SMs for about 0.7 ms)
+            _ = A @ A
+        O = torch.empty_like(Q)
+        api.flat_attn_fwd_ex(Q, K, V, O, w.scale, k_valid_len=vlt, status=status[it:it + 1], variant=api.FLAT_VARIANT_TC3,
+                             stream=s2.cuda_stream)
+        outs.append(O)
+    torch.cuda.synchronize()
+    assert int(status.abs().max().item()) == 0, [hex(c) for c in status.cpu().numpy().tolist() if c]
+    assert all(torch.equal(o, ref) for o in outs)
