@@ -84,3 +84,69 @@ def test_backward_launches_repeat_bit_for_bit(api, case):
         else:
             assert all(torch.equal(a, b) for a, b in zip(first, (dQ, dK, dV))), "launch %d differs" % it
     assert int(status.item()) == 0
+
+
+def _repeat(fn, n):
+    first = None
+    for it in range(n):
+        out = fn()
+        torch.cuda.synchronize()
+        if first is None:
+            first = [o.clone() for o in out]
+        else:
+            assert all(torch.equal(a, b) for a, b in zip(first, out)), "launch %d differs" % it
+
+
+@pytest.mark.parametrize("d", [64, 128])
+@pytest.mark.parametrize("causal", [False, True])
+def test_packed_batches_repeat_bit_for_bit(api, d, causal):
+    H, lens = 8, [3900, 777, 5000, 128, 2049, 1]
+    cu = torch.tensor(np.concatenate([[0], np.cumsum(lens)]), dtype=torch.int32, device="cuda")
+    g = torch.Generator(device="cuda").manual_seed(d)
+    mk = lambda: torch.randn(sum(lens), H, d, device="cuda", dtype=torch.bfloat16, generator=g)
+    Q, K, V = mk(), mk(), mk()
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+
+    def call():
+        O = torch.empty_like(Q)
+        api.flat_attn_varlen_fwd(Q, K, V, O, cu, cu, max(lens), d ** -0.5, causal=causal, status=status)
+        return [O]
+    _repeat(call, 30)
+    assert int(status.item()) == 0
+
+
+def test_bias_pruned_and_layer_calls_repeat_bit_for_bit(api):
+    B, H, Nq, Nk = 2, 8, 1024, 2048
+    g = torch.Generator(device="cuda").manual_seed(7)
+    Q = torch.randn(B, H, Nq, 64, device="cuda", dtype=torch.bfloat16, generator=g)
+    K = torch.randn(B, H, Nk, 64, device="cuda", dtype=torch.bfloat16, generator=g)
+    V = torch.randn(B, H, Nk, 64, device="cuda", dtype=torch.bfloat16, generator=g)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    for shape, dt in (((1, H, Nq, Nk), torch.bfloat16), ((B, H, Nq, Nk), torch.bfloat16), ((1, 1, Nq, Nk), torch.float32)):
+        bias = torch.randn(*shape, device="cuda", dtype=dt, generator=g)
+
+        def call():
+            O = torch.empty_like(Q)
+            api.flat_attn_fwd_ex(Q, K, V, O, 0.125, status=status, bias=bias)
+            return [O]
+        _repeat(call, 20)
+    keep = (torch.rand(1, H, Nq // 128, Nk // 128, device="cuda", generator=g) < 0.5).to(torch.uint8)
+    keep[..., 0] = 1
+
+    def pruned():
+        O = torch.empty_like(Q)
+        api.flat_attn_fwd_ex(Q, K, V, O, 0.125, status=status, block_mask=keep)
+        return [O]
+    _repeat(pruned, 20)
+    Bn, N, Hh, dd, Dm = 2, 1024, 8, 64, 512
+    X = torch.randn(Bn, N, Dm, device="cuda", dtype=torch.bfloat16, generator=g) * 0.5
+    Wqkv = torch.randn(3 * Hh * dd, Dm, device="cuda", dtype=torch.bfloat16, generator=g) * 0.05
+    Wo = torch.randn(Dm, Hh * dd, device="cuda", dtype=torch.bfloat16, generator=g) * 0.05
+
+    def layer():
+        Y = torch.empty_like(X)
+        bufs = [torch.empty(Bn, Hh, N, dd, device="cuda", dtype=torch.bfloat16) for _ in range(4)]
+        api.flat_attn_layer_fwd(X, Wqkv, Wo, Y, *bufs, 0.125, status=status)
+        return [Y]
+    _repeat(layer, 12)
+    assert int(status.item()) == 0
