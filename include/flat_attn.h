@@ -18,7 +18,10 @@
  *       Q, O : [B, H, Nq, d]      K, V : [B, H, Nk, d]      L, A : [B, H, Nq, Nk]
  *   - Unless an argument says HOST, pointers are DEVICE pointers owned by the
  *     caller, 16-byte aligned.  The library allocates and frees no device memory
- *     and keeps no pointer after a call returns.
+ *     and keeps no pointer after a call returns.  (What it needs beyond the caller's
+ *     buffers lives in its own device image: a status word, the workspace of the
+ *     even deal -- see flat_attn_last_schedule -- and that of flat_attn_naive_fwd_static.
+ *     The even deal also records one event per launch, created once per device.)
  *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*; NULL is
  *     the default stream); the library does not synchronise unless stated.
  *   - Return value: FLAT_OK or one of the error codes below.  On an argument
