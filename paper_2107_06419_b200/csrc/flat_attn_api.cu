@@ -177,8 +177,10 @@ int run_fused(const flat::Problem& q, int variant, cudaStream_t st) {
         if (!tc_applies(q) || q.d != 64 || q.block_mask || q.bias) return FLAT_ERR_UNSUPPORTED;
         const int cs = v == FLAT_VARIANT_TC2_HALVES_SPLIT16 ? 16 : 1 << (v - FLAT_VARIANT_TC2_HALVES);
         int rc = flat::launch_fused_tc2_halves(q, st, cs, variant == FLAT_VARIANT_AUTO);
-        if (rc == FLAT_ERR_UNSUPPORTED && cs == 16 && variant == FLAT_VARIANT_AUTO) {
-            // (AUTO asked for sixteen and the device cannot hold all the launch's clusters at once: eight)
+        if (rc != FLAT_OK && cs == 16 && variant == FLAT_VARIANT_AUTO) {
+            // (AUTO asked for sixteen and the device cannot hold all the launch's clusters at once, or refused the
+            // launch: eight)
+            cudaGetLastError();
             v = FLAT_VARIANT_TC2_HALVES_SPLIT8;
             rc = flat::launch_fused_tc2_halves(q, st, 8);
         }
@@ -189,8 +191,10 @@ int run_fused(const flat::Problem& q, int variant, cudaStream_t st) {
         if (!tc_applies(q) || q.block_mask || (v == FLAT_VARIANT_TC2_SPLIT16 && q.d != 128)) return FLAT_ERR_UNSUPPORTED;
         const int cs = v == FLAT_VARIANT_TC2_SPLIT2 ? 2 : v == FLAT_VARIANT_TC2_SPLIT4 ? 4 : v == FLAT_VARIANT_TC2_SPLIT8 ? 8 : 16;
         int rc = flat::launch_fused_tc2_single(q, st, cs, variant == FLAT_VARIANT_AUTO);
-        if (rc == FLAT_ERR_UNSUPPORTED && cs == 16 && variant == FLAT_VARIANT_AUTO) {
-            // (AUTO asked for sixteen and the device cannot hold all the launch's clusters at once: eight)
+        if (rc != FLAT_OK && cs == 16 && variant == FLAT_VARIANT_AUTO) {
+            // (AUTO asked for sixteen and the device cannot hold all the launch's clusters at once, or refused the
+            // launch: eight)
+            cudaGetLastError();
             v = FLAT_VARIANT_TC2_SPLIT8;
             rc = flat::launch_fused_tc2_single(q, st, 8);
         }
