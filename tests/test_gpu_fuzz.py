@@ -199,3 +199,41 @@ def test_bias_and_pruning_map(api, case):
     check_bf16(bf16_to_f64(O), refm["O"], "fuzz pruning map %s" % (case[:7],))
     dead = np.isneginf(refm["LSE"])
     assert np.array_equal(np.isneginf(lse.double().cpu().numpy()), dead)
+
+
+def test_auto_against_the_two_tile_kernel_at_medium_sizes(api):
+    """The dispatcher's choices that only medium-sized problems reach (two warpgroups per tile, key splits over
+    clusters, the even deal, one CTA per item, persistent CTAs): 90 seeded random problems, each run three times
+    with FLAT_VARIANT_AUTO (same bits every time, no device code) and once with the two-tile kernel, whose output
+    the dispatcher's kernel must match within the sum of the two kernels' parity bars."""
+    rng = np.random.default_rng(20210706)
+    seen = set()
+    for it in range(90):
+        d = 64 if rng.random() < 0.6 else 128
+        B, H = int(rng.integers(1, 9)), int(rng.integers(1, 17))
+        Nq = int(rng.integers(1, 13)) * 128 + int(rng.integers(0, 2)) * int(rng.integers(1, 128))
+        Nk = int(rng.integers(2, 64)) * 128 + int(rng.integers(0, 2)) * int(rng.integers(1, 128))
+        causal = bool(rng.random() < 0.25)
+        vl = rng.integers(0, Nk + 1, B).astype(np.int32) if rng.random() < 0.5 else None
+        g = torch.Generator(device="cuda").manual_seed(it)
+        Q = torch.randn(B, H, Nq, d, device="cuda", dtype=torch.bfloat16, generator=g)
+        K = torch.randn(B, H, Nk, d, device="cuda", dtype=torch.bfloat16, generator=g)
+        V = torch.randn(B, H, Nk, d, device="cuda", dtype=torch.bfloat16, generator=g)
+        vlt = None if vl is None else torch.from_numpy(vl).cuda()
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        outs = []
+        for _ in range(3):
+            O = torch.full_like(Q, float("nan"))
+            api.flat_attn_fwd_ex(Q, K, V, O, d ** -0.5, k_valid_len=vlt, status=status, causal=causal)
+            outs.append(O)
+        v = api.flat_attn_last_variant()
+        seen.add((d, v, api.flat_attn_last_schedule() if v == api.FLAT_VARIANT_TC3 else 0))
+        O2 = torch.full_like(Q, float("nan"))
+        api.flat_attn_fwd_ex(Q, K, V, O2, d ** -0.5, k_valid_len=vlt, status=status, causal=causal, variant=api.FLAT_VARIANT_TC2)
+        torch.cuda.synchronize()
+        what = "case %d %s d=%d causal=%d variant %d" % (it, (B, H, Nq, Nk), d, causal, v)
+        assert int(status.item()) == 0, what
+        assert bool(torch.isfinite(outs[0].float()).all()), what
+        assert torch.equal(outs[0], outs[1]) and torch.equal(outs[0], outs[2]), what
+        assert float((outs[0].float() - O2.float()).abs().max()) <= 2 * 2e-2, what
+    assert len(seen) >= 6, seen                          # (the cases do reach the different kernels and deals)
